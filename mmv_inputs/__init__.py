@@ -1,0 +1,215 @@
+"""Seeded synthetic inputs for the segmented scan / sum / SpMV workloads.
+
+This module only draws random numbers and lays them out; it holds none of the
+method's arithmetic and is the one piece of code that both the GPU tests and
+the CPU oracle's tests may share.  Every array is produced in chunks of
+``CHUNK`` elements, each from its own ``SeedSequence([BASE_SEED, config,
+stream, chunk])``, so any chunk of a 2^30-element input can be regenerated
+alone when results are compared piece by piece.
+
+The workloads stand in for the paper's own inputs (segment lengths taken from
+the rows of sparse-matrix collections, and uniformly random segment densities,
+Section 5), whose data files are not available here.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+BASE_SEED = 250623906
+CHUNK = 1 << 24
+
+# stream ids
+S_VALUES, S_FLAGS, S_LENGTHS, S_COLS, S_XVEC = 0, 1, 2, 3, 4
+
+
+def _rng(config: int, stream: int, chunk: int) -> np.random.Generator:
+    return np.random.Generator(np.random.PCG64(np.random.SeedSequence([BASE_SEED, config, stream, chunk])))
+
+
+def _chunks(n: int):
+    c = 0
+    while c * CHUNK < n:
+        yield c, min(CHUNK, n - c * CHUNK)
+        c += 1
+
+
+# --------------------------------------------------------------------------
+# values
+# --------------------------------------------------------------------------
+def f16_uniform_chunk(config: int, chunk: int, m: int = CHUNK, stream: int = S_VALUES) -> np.ndarray:
+    """fp16 values: float32 uniform in [-1, 1) rounded to nearest-even fp16."""
+    u = _rng(config, stream, chunk).random(CHUNK, dtype=np.float32)[:m]
+    return (u * np.float32(2.0) - np.float32(1.0)).astype(np.float16)
+
+
+def f16_normal_chunk(config: int, chunk: int, m: int = CHUNK, stream: int = S_VALUES) -> np.ndarray:
+    g = _rng(config, stream, chunk).standard_normal(CHUNK, dtype=np.float32)[:m]
+    return g.astype(np.float16)
+
+
+def i8_uniform_chunk(config: int, chunk: int, m: int = CHUNK, lo: int = -8, hi: int = 7) -> np.ndarray:
+    return _rng(config, S_VALUES, chunk).integers(lo, hi + 1, size=CHUNK, dtype=np.int8)[:m]
+
+
+def _full(fn, n: int, dtype, *a, **k) -> np.ndarray:
+    out = np.empty(n, dtype)
+    for c, m in _chunks(n):
+        out[c * CHUNK:c * CHUNK + m] = fn(*a, chunk=c, m=m, **k)
+    return out
+
+
+def f16_uniform(config: int, n: int, stream: int = S_VALUES) -> np.ndarray:
+    return _full(f16_uniform_chunk, n, np.float16, config, stream=stream)
+
+
+def f16_normal(config: int, n: int, stream: int = S_VALUES) -> np.ndarray:
+    return _full(f16_normal_chunk, n, np.float16, config, stream=stream)
+
+
+def i8_uniform(config: int, n: int, lo: int = -8, hi: int = 7) -> np.ndarray:
+    return _full(i8_uniform_chunk, n, np.int8, config, lo=lo, hi=hi)
+
+
+# --------------------------------------------------------------------------
+# start flags
+# --------------------------------------------------------------------------
+def flags_chunk(config: int, chunk: int, m: int = CHUNK, p: float = 1.0 / 64, pattern: str = "bernoulli") -> np.ndarray:
+    """uint8 start flags of one chunk.
+
+    pattern: "bernoulli" (probability p per element), "all" (every element
+    starts a segment) or "cycle123" (segment lengths 1,2,3,1,2,3,...).  The
+    first flag of the whole array is always 1.
+    """
+    if pattern == "all":
+        f = np.ones(m, np.uint8)
+    elif pattern == "cycle123":
+        base = (chunk * CHUNK) % 6
+        pat = np.array([1, 1, 0, 1, 0, 0], np.uint8)
+        idx = (np.arange(m, dtype=np.int64) + base) % 6
+        f = pat[idx]
+    elif pattern == "bernoulli":
+        if p <= 0.0:
+            f = np.zeros(m, np.uint8)
+        else:
+            u = _rng(config, S_FLAGS, chunk).random(CHUNK, dtype=np.float32)[:m]
+            f = (u < np.float32(p)).astype(np.uint8)
+    else:
+        raise ValueError(pattern)
+    if chunk == 0 and m > 0:
+        f[0] = 1
+    return f
+
+
+def flags(config: int, n: int, p: float = 1.0 / 64, pattern: str = "bernoulli") -> np.ndarray:
+    return _full(flags_chunk, n, np.uint8, config, p=p, pattern=pattern)
+
+
+# --------------------------------------------------------------------------
+# CSR offsets
+# --------------------------------------------------------------------------
+def offsets_uniform_lengths(config: int, n: int, max_len: int = 4096) -> np.ndarray:
+    """int32 offsets of segments with lengths uniform in {1..max_len} covering exactly n."""
+    if n == 0:
+        return np.zeros(1, np.int32)
+    rng = _rng(config, S_LENGTHS, 0)
+    parts, total = [], 0
+    while total < n:
+        want = max(16, int(2.2 * (n - total) / (max_len + 1)) + 16)
+        l = rng.integers(1, max_len + 1, size=want, dtype=np.int64)
+        parts.append(l)
+        total += int(l.sum())
+    lens = np.concatenate(parts)
+    cs = np.cumsum(lens)
+    k = int(np.searchsorted(cs, n, side="left"))       # first index with cs >= n
+    cs = cs[:k + 1]
+    cs[k] = n                                          # truncate the last length
+    off = np.empty(k + 2, np.int64)
+    off[0] = 0
+    off[1:] = cs
+    return off.astype(np.int32)
+
+
+def zipf_row_lengths(config: int, rows: int, s: float = 1.5, cap: int = 10_000,
+                     empty_fraction: float = 0.0) -> np.ndarray:
+    """Row lengths with P(k) proportional to k^-s on {1..cap} (inverse-CDF table)."""
+    k = np.arange(1, cap + 1, dtype=np.float64)
+    w = k ** (-s)
+    cdf = np.cumsum(w / w.sum())
+    rng = _rng(config, S_LENGTHS, 0)
+    u = rng.random(rows)
+    lens = np.searchsorted(cdf, u, side="left").astype(np.int64) + 1
+    lens = np.minimum(lens, cap)
+    if empty_fraction > 0.0:
+        e = rng.random(rows) < empty_fraction
+        lens[e] = 0
+    return lens
+
+
+def offsets_from_lengths(lens: np.ndarray) -> np.ndarray:
+    off = np.zeros(lens.shape[0] + 1, np.int64)
+    np.cumsum(lens, out=off[1:])
+    if off[-1] >= 2 ** 31:
+        raise ValueError("too many elements for int32 offsets")
+    return off.astype(np.int32)
+
+
+def csr_matrix(config: int, rows: int, cols: int, s: float = 1.5, cap: int = 10_000,
+               empty_fraction: float = 0.0):
+    """(rowptr int32, col int32, val fp16, x fp32) of a random CSR matrix.
+
+    Row lengths follow the truncated power law above; column indices are
+    uniform (unsorted, duplicates allowed); values uniform in [-1, 1); the
+    dense vector is standard normal.
+    """
+    lens = zipf_row_lengths(config, rows, s, cap, empty_fraction)
+    rowptr = offsets_from_lengths(lens)
+    nnz = int(rowptr[-1])
+    col = np.empty(nnz, np.int32)
+    for c, m in _chunks(nnz):
+        col[c * CHUNK:c * CHUNK + m] = _rng(config, S_COLS, c).integers(0, cols, size=CHUNK, dtype=np.int32)[:m]
+    val = f16_uniform(config, nnz)
+    x = _rng(config, S_XVEC, 0).standard_normal(cols, dtype=np.float32)
+    return rowptr, col, val, x
+
+
+# --------------------------------------------------------------------------
+# the five benchmark configurations (sizes can be scaled down for tests)
+# --------------------------------------------------------------------------
+C5_CASES = (
+    ("p0", dict(p=0.0, pattern="bernoulli")),
+    ("p1e-6", dict(p=1e-6, pattern="bernoulli")),
+    ("p1e-3", dict(p=1e-3, pattern="bernoulli")),
+    ("p0.1", dict(p=0.1, pattern="bernoulli")),
+    ("p0.5", dict(p=0.5, pattern="bernoulli")),
+    ("all", dict(p=1.0, pattern="all")),
+    ("cycle123", dict(p=0.5, pattern="cycle123")),
+)
+
+
+def config1(n: int = 1 << 20):
+    """Segmented scan: fp16 uniform values, Bernoulli(1/64) flags."""
+    return f16_uniform(1, n), flags(1, n, p=1.0 / 64)
+
+
+def config2(n: int = 1 << 26, max_len: int = 4096):
+    """Segmented sum: fp16 normal values, CSR offsets with lengths uniform in {1..max_len}."""
+    return f16_normal(2, n), offsets_uniform_lengths(2, n, max_len)
+
+
+def config3(n: int = 1 << 28):
+    """Segmented scan: int8 values uniform in {-8..7}, Bernoulli(1e-3) flags."""
+    return i8_uniform(3, n), flags(3, n, p=1e-3)
+
+
+def config4(rows: int = 1 << 20, cols: int | None = None, empty_fraction: float = 0.0):
+    """CSR SpMV: power-law row lengths capped at 10^4."""
+    return csr_matrix(4, rows, rows if cols is None else cols, empty_fraction=empty_fraction)
+
+
+def config5_values(n: int = 1 << 30):
+    return f16_uniform(5, n)
+
+
+def config5_flags(n: int, case: str):
+    kw = dict(C5_CASES)[case]
+    return flags(5, n, **kw)
