@@ -1,0 +1,150 @@
+/*
+ * mmv.h -- C ABI of the segmented scan / segmented sum / CSR SpMV library for
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel hot path of "Segmented Operations
+ * using Matrix Multiplications" (MMV-RAM): the prefix sums inside each tile are
+ * a tensor-core product of the data tile with a constant triangular all-ones
+ * matrix (Section 1.2 "Notation": z = MATMUL(x, U_s); Algorithm A.1,
+ * BlockSegScan), vector operations revert the speculation at segment
+ * boundaries (Lemma A.1), and the per-block recursion of Section 4.2 is
+ * replaced by a single-pass chained carry between tiles.
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".
+ *     The caller owns every buffer; the library never allocates, frees or
+ *     keeps a pointer after the call returns.
+ *   - `workspace` is caller-provided device scratch of at least
+ *     mmv_workspace_bytes(...) bytes, 256-byte aligned; its content on entry is
+ *     irrelevant (the call initialises what it needs on the stream) and it must
+ *     not be shared by calls that may overlap on the GPU.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL =
+ *     the default stream); the call does not synchronise with the host.
+ *   - x, seg and out must be 16-byte aligned and must not overlap each other.
+ *   - Argument errors are reported synchronously and nothing is enqueued.
+ *     Conditions only the device can detect (a wait that ran out of its time
+ *     budget, segment offsets that are not monotone) set a status word inside
+ *     the workspace; outputs are then unspecified and
+ *     mmv_last_async_status() reports the code.  No device trap, no unbounded
+ *     wait.
+ *   - n == 0 (nnz == 0, rows == 0) is valid: nothing is read; seg-sum / SpMV
+ *     still write their (empty-segment) zeros.
+ *
+ * Segment encodings
+ *   MMV_SEG_FLAGS_U8     n bytes; any non-zero byte marks the first element of a
+ *                        segment.  Byte 0 is never consulted: element 0 always
+ *                        opens a segment (Problem 2.1, Eq. 1: "i = 0 or f(i) = 1").
+ *   MMV_SEG_OFFSETS_I32  nseg+1 int32 values, non-decreasing, the CSR row-pointer
+ *                        convention: segment r covers [off[r], off[r+1]) and may
+ *                        be empty (Section 4.3, remark after Algorithm 4.4;
+ *                        Algorithm A.4 for empty rows).
+ *
+ * Arithmetic
+ *   MMV_F16_TO_F32  fp16 values, fp32 accumulation and output.  Results satisfy
+ *                   |out - exact| <= 2e-3 * (sum of |x| over the summed range) + 1e-6
+ *                   for inputs of the magnitude the library is specified for
+ *                   (|x| of order 1); they are not bit-reproducible from run to
+ *                   run because the grouping of the cross-tile carry chain
+ *                   depends on timing.
+ *   MMV_I8_TO_I32   int8 values, exact int32 result modulo 2^32 (bit-exact and
+ *                   deterministic).
+ */
+#ifndef MMV_H_
+#define MMV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MMV_OK = 0,
+    MMV_ERR_INVALID_ARG = 1,         /* null/misaligned pointer, negative size, bad enum      */
+    MMV_ERR_UNSUPPORTED = 2,         /* combination not implemented                           */
+    MMV_ERR_WORKSPACE_TOO_SMALL = 3,
+    MMV_ERR_BAD_SEGMENTS = 4,        /* offsets not monotone / out of range (device-detected) */
+    MMV_ERR_TIMEOUT = 5,             /* a bounded device-side wait gave up                    */
+    MMV_ERR_CUDA = 6                 /* a CUDA runtime / driver call failed                   */
+} mmv_status;
+
+typedef enum { MMV_F16_TO_F32 = 0, MMV_I8_TO_I32 = 1 } mmv_dtype;
+typedef enum { MMV_SEG_FLAGS_U8 = 0, MMV_SEG_OFFSETS_I32 = 1 } mmv_segfmt;
+typedef enum { MMV_OP_SEG_SCAN = 0, MMV_OP_SEG_SUM = 1, MMV_OP_SPMV_CSR = 2 } mmv_op;
+
+/*
+ * Bytes of device workspace the given call needs (a pure host computation).
+ * n = number of values (nnz for SpMV), nseg = number of segments (rows); nseg is
+ * ignored for flag-encoded segments.  Returns 0 for invalid arguments.
+ */
+size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, int64_t nseg);
+
+/*
+ * Segmented inclusive scan (Problem 2.1, Eq. 1):
+ *     out[i] = x[i]               if i == 0 or i starts a segment
+ *     out[i] = out[i-1] + x[i]    otherwise
+ * x: n values (fp16 or int8 per dt).  seg: n flag bytes, or nseg+1 offsets with
+ * off[0] == 0 and off[nseg] == n (empty segments allowed, they start nothing).
+ * out: n values (fp32 or int32).  Elements past n are never written.
+ */
+mmv_status mmv_seg_scan(const void *x, const void *seg, mmv_segfmt sf, int64_t n, int64_t nseg,
+                        mmv_dtype dt, void *out,
+                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Segmented sum (Section 2: the last element of every segment of the
+ * segmented scan; Algorithm 4.2 computes the same quantity).
+ * Offsets form: out has nseg entries, out[r] = sum of x over [off[r], off[r+1]),
+ * exactly 0 for an empty segment; values outside [off[0], off[nseg]) are
+ * ignored; requires 0 <= off[0] and off[nseg] <= n.  d_num_segments is ignored
+ * (may be NULL).
+ * Flags form: out has capacity n; the K = 1 + #{i >= 1 : flag[i] != 0} segment
+ * sums are written in segment order and K is written to *d_num_segments
+ * (device pointer, int64) when it is not NULL.
+ */
+mmv_status mmv_seg_sum(const void *x, const void *seg, mmv_segfmt sf, int64_t n, int64_t nseg,
+                       mmv_dtype dt, void *out, int64_t *d_num_segments,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * CSR sparse matrix times dense vector built on the segmented sum
+ * (Algorithm 4.4; Algorithms A.4-A.6):  y[r] = sum over k in
+ * [rowptr[r], rowptr[r+1]) of val[k] * x[col[k]], fp32 products and sums, an
+ * empty row gives exactly 0.  rowptr: rows+1 int32 with rowptr[0] == 0 and
+ * rowptr[rows] == nnz; col: nnz int32 in [0, cols) (not checked; duplicates
+ * simply add); val: nnz fp16; x: cols fp32; y: rows fp32.
+ */
+mmv_status mmv_spmv_csr(const int32_t *rowptr, const int32_t *col, const void *val_f16,
+                        const float *x, float *y, int64_t rows, int64_t cols, int64_t nnz,
+                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Synchronises `cuda_stream` and returns the device-side status that the last
+ * call using `workspace` recorded (MMV_OK if none), or MMV_ERR_CUDA if the
+ * stream itself reports an error.
+ */
+mmv_status mmv_last_async_status(const void *workspace, void *cuda_stream);
+
+/* Static, human-readable name of a status code. */
+const char *mmv_status_string(mmv_status s);
+
+/*
+ * Number of kernels the library has launched in this process since it was
+ * loaded (host counter; used by the benchmark to report its launch count).
+ */
+int64_t mmv_kernel_launch_count(void);
+
+/*
+ * Test hook.  wait_budget_ns: time after which a device-side wait gives up
+ * (<= 0 restores the default of 4 s).  skip_publish_span: index of one
+ * 4096-element span of the scan that never publishes its carry, so that its
+ * successors exercise the time-out path without any GPU fault (-1 = off).
+ * Applies to calls made after it returns.
+ */
+void mmv_debug_configure(int64_t wait_budget_ns, int64_t skip_publish_span);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MMV_H_ */

@@ -1,0 +1,175 @@
+"""Python binding of libmmv.so, the C-ABI CUDA library for segmented scan,
+segmented sum and CSR SpMV on B200 (sm_100a).
+
+The binding only marshals arguments: torch supplies device memory and the
+current CUDA stream, every step of the computation runs in the library's own
+kernels.  There is no CPU or PyTorch fallback: if the shared library is missing
+the import of this module fails.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libmmv.so"
+
+# enums of include/mmv.h
+MMV_OK = 0
+F16_TO_F32, I8_TO_I32 = 0, 1
+SEG_FLAGS_U8, SEG_OFFSETS_I32 = 0, 1
+OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR = 0, 1, 2
+
+EXPORTS = (
+    "mmv_workspace_bytes", "mmv_seg_scan", "mmv_seg_sum", "mmv_spmv_csr",
+    "mmv_last_async_status", "mmv_status_string", "mmv_kernel_launch_count", "mmv_debug_configure",
+)
+
+
+class MmvError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (mmv_status {code})")
+
+
+def _load() -> ctypes.CDLL:
+    if not LIB_PATH.exists():
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2506_23906_b200.build` "
+            "(nvcc, sm_100a).  There is no fallback path.")
+    lib = ctypes.CDLL(str(LIB_PATH))
+    vp, i64, sz, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_int
+    lib.mmv_workspace_bytes.restype = sz
+    lib.mmv_workspace_bytes.argtypes = [ci, ci, ci, i64, i64]
+    lib.mmv_seg_scan.restype = ci
+    lib.mmv_seg_scan.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, sz, vp]
+    lib.mmv_seg_sum.restype = ci
+    lib.mmv_seg_sum.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, vp, sz, vp]
+    lib.mmv_spmv_csr.restype = ci
+    lib.mmv_spmv_csr.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, sz, vp]
+    lib.mmv_last_async_status.restype = ci
+    lib.mmv_last_async_status.argtypes = [vp, vp]
+    lib.mmv_status_string.restype = ctypes.c_char_p
+    lib.mmv_status_string.argtypes = [ci]
+    lib.mmv_kernel_launch_count.restype = i64
+    lib.mmv_kernel_launch_count.argtypes = []
+    lib.mmv_debug_configure.restype = None
+    lib.mmv_debug_configure.argtypes = [i64, i64]
+    return lib
+
+
+_lib = _load()
+
+
+def status_string(code: int) -> str:
+    return _lib.mmv_status_string(int(code)).decode()
+
+
+def kernel_launch_count() -> int:
+    return int(_lib.mmv_kernel_launch_count())
+
+
+def debug_configure(wait_budget_ns: int = 0, skip_publish_span: int = -1) -> None:
+    _lib.mmv_debug_configure(int(wait_budget_ns), int(skip_publish_span))
+
+
+def workspace_bytes(op: int, dt: int, sf: int, n: int, nseg: int = 0) -> int:
+    return int(_lib.mmv_workspace_bytes(op, dt, sf, int(n), int(nseg)))
+
+
+def _stream_ptr(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else int(t.data_ptr())
+
+
+def _dtype_code(x: torch.Tensor) -> int:
+    if x.dtype == torch.float16:
+        return F16_TO_F32
+    if x.dtype == torch.int8:
+        return I8_TO_I32
+    raise TypeError("values must be torch.float16 or torch.int8")
+
+
+def _seg_code(seg: torch.Tensor) -> int:
+    if seg.dtype == torch.uint8:
+        return SEG_FLAGS_U8
+    if seg.dtype == torch.int32:
+        return SEG_OFFSETS_I32
+    raise TypeError("segments must be uint8 start flags or int32 offsets")
+
+
+def _check_cuda(*ts):
+    for t in ts:
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("tensors must be contiguous CUDA tensors")
+
+
+def alloc_workspace(op: int, dt: int, sf: int, n: int, nseg: int = 0, device=None) -> torch.Tensor:
+    nbytes = max(256, workspace_bytes(op, dt, sf, n, nseg))
+    return torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
+
+
+def last_async_status(workspace: torch.Tensor, stream=None) -> int:
+    return int(_lib.mmv_last_async_status(_ptr(workspace), _stream_ptr(stream)))
+
+
+def seg_scan(x: torch.Tensor, seg: torch.Tensor, out: torch.Tensor | None = None,
+             workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """mmv_seg_scan: segmented inclusive scan (Problem 2.1, Eq. 1) of x over seg."""
+    _check_cuda(x, seg, out, workspace)
+    dt, sf = _dtype_code(x), _seg_code(seg)
+    n = x.numel()
+    nseg = seg.numel() - 1 if sf == SEG_OFFSETS_I32 else 0
+    if out is None:
+        out = torch.empty(n, dtype=torch.float32 if dt == F16_TO_F32 else torch.int32, device=x.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_SEG_SCAN, dt, sf, n, nseg, x.device)
+    rc = _lib.mmv_seg_scan(_ptr(x), _ptr(seg), sf, n, nseg, dt, _ptr(out), _ptr(workspace),
+                           workspace.numel(), _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_seg_scan")
+    return out
+
+
+def seg_sum(x: torch.Tensor, seg: torch.Tensor, out: torch.Tensor | None = None,
+            num_segments: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
+            stream=None) -> torch.Tensor:
+    """mmv_seg_sum: per-segment sums (Section 2) of x over seg (CSR offsets or flags)."""
+    _check_cuda(x, seg, out, workspace, num_segments)
+    dt, sf = _dtype_code(x), _seg_code(seg)
+    n = x.numel()
+    nseg = seg.numel() - 1 if sf == SEG_OFFSETS_I32 else 0
+    if out is None:
+        cap = nseg if sf == SEG_OFFSETS_I32 else n
+        out = torch.empty(cap, dtype=torch.float32 if dt == F16_TO_F32 else torch.int32, device=x.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_SEG_SUM, dt, sf, n, nseg, x.device)
+    rc = _lib.mmv_seg_sum(_ptr(x), _ptr(seg), sf, n, nseg, dt, _ptr(out), _ptr(num_segments),
+                          _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_seg_sum")
+    return out
+
+
+def spmv_csr(rowptr: torch.Tensor, col: torch.Tensor, val: torch.Tensor, x: torch.Tensor,
+             y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """mmv_spmv_csr: y = A x for a CSR matrix (Algorithm 4.4), fp16 values, fp32 x and y."""
+    _check_cuda(rowptr, col, val, x, y, workspace)
+    if rowptr.dtype != torch.int32 or col.dtype != torch.int32 or val.dtype != torch.float16 or x.dtype != torch.float32:
+        raise TypeError("rowptr/col int32, val float16, x float32 expected")
+    rows, cols, nnz = rowptr.numel() - 1, x.numel(), val.numel()
+    if y is None:
+        y = torch.empty(rows, dtype=torch.float32, device=x.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_SPMV_CSR, F16_TO_F32, SEG_OFFSETS_I32, nnz, rows, x.device)
+    rc = _lib.mmv_spmv_csr(_ptr(rowptr), _ptr(col), _ptr(val), _ptr(x), _ptr(y), rows, cols, nnz,
+                           _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_spmv_csr")
+    return y

@@ -1,0 +1,249 @@
+// Host side of the C ABI declared in include/mmv.h: argument checks, workspace
+// carve-up, tensor-map encoding and kernel launches.  No allocation, no host
+// synchronisation (except mmv_last_async_status, whose job it is).
+#include <atomic>
+#include <cstdint>
+#include <cstring>
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <mutex>
+
+#include "../../include/mmv.h"
+#include "common.cuh"
+#include "seg_scan.cuh"
+#include "seg_sum.cuh"
+
+namespace mmv {
+namespace {
+
+std::atomic<long long> g_launches{0};
+std::atomic<unsigned long long> g_budget_ns{WAIT_BUDGET_NS};
+std::atomic<long long> g_debug_skip_span{-1};
+
+constexpr int kMaxDevices = 64;
+
+struct DeviceInfo {
+    std::once_flag once;
+    int sm_count = 0;
+    bool ok = false;
+};
+DeviceInfo g_dev[kMaxDevices];
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+std::once_flag g_encode_once;
+
+EncodeTiledFn get_encode() {
+    std::call_once(g_encode_once, [] {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    });
+    return g_encode;
+}
+
+template <typename K>
+bool set_smem(K kernel, int bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+// Per-device one-time set-up: SM count and the kernels' dynamic shared-memory limits.
+DeviceInfo* device_info() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    DeviceInfo* d = &g_dev[dev];
+    std::call_once(d->once, [d, dev] {
+        int sm = 0;
+        if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
+        d->sm_count = sm;
+        bool ok = true;
+        ok &= set_smem(seg_scan_kernel<F16Path>, ScanCfg<F16Path>::kSmemBytes);
+        ok &= set_smem(seg_scan_kernel<I8Path>, ScanCfg<I8Path>::kSmemBytes);
+        ok &= seg_sum_set_attributes();
+        d->ok = ok;
+    });
+    return d->ok ? d : nullptr;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// The value vector as a matrix of CHUNK-element rows (full rows only); box = NCOL rows.
+bool encode_rows_map(CUtensorMap* map, const void* x, long long n, bool is_f16) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t rows = static_cast<cuuint64_t>(n / CHUNK);
+    if (rows == 0) {
+        std::memset(map, 0, sizeof(*map));
+        return true;               // never used: every tile takes the plain-load path
+    }
+    const cuuint32_t esz = is_f16 ? 2 : 1;
+    cuuint64_t dims[2] = {CHUNK, rows};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(CHUNK) * esz};
+    cuuint32_t box[2] = {CHUNK, NCOL};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, is_f16 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
+                     const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     is_f16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+struct WorkspacePlan {
+    size_t status_off, status_bytes;
+    size_t flags_off, flags_bytes;     // scratch flag bytes (offset-encoded scan only)
+    size_t total;
+};
+
+long long num_tiles_of(long long n) { return (n + TILE - 1) / TILE; }
+
+WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
+    WorkspacePlan p{};
+    const long long tiles = num_tiles_of(n);
+    p.status_off = sizeof(WorkspaceHeader);
+    p.status_bytes = round_up(static_cast<size_t>(tiles) * SPANS_PER_TILE * sizeof(uint64_t), 256);
+    p.flags_off = p.status_off + p.status_bytes;
+    p.flags_bytes = (op == MMV_OP_SEG_SCAN && sf == MMV_SEG_OFFSETS_I32) ? round_up(static_cast<size_t>(n), 256) : 0;
+    p.total = p.flags_off + p.flags_bytes;
+    return p;
+}
+
+// f[off[r]] = 1 for every non-empty segment r (scratch flags of the offset-encoded scan).
+__global__ void offsets_to_flags_kernel(const int32_t* __restrict__ off, long long nseg, long long n,
+                                        uint8_t* __restrict__ f, WorkspaceHeader* hdr) {
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long r = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; r < nseg; r += stride) {
+        const long long a = off[r], b = off[r + 1];
+        if (a > b || a < 0 || b > n || (r == 0 && a != 0) || (r == nseg - 1 && b != n)) {
+            report_error(hdr, 4u);
+        } else if (a < b) {
+            f[a] = 1;
+        }
+    }
+}
+
+}  // namespace
+}  // namespace mmv
+
+using namespace mmv;
+
+extern "C" {
+
+size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, int64_t nseg) {
+    if (n < 0 || nseg < 0) return 0;
+    if (op != MMV_OP_SEG_SCAN && op != MMV_OP_SEG_SUM && op != MMV_OP_SPMV_CSR) return 0;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return 0;
+    if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return 0;
+    return plan_workspace(op, sf, n).total;
+}
+
+mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
+                        void* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (n < 0 || nseg < 0) return MMV_ERR_INVALID_ARG;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
+    if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
+    if (n == 0) return MMV_OK;
+    if (n >= (1ll << 36)) return MMV_ERR_UNSUPPORTED;
+    if (sf == MMV_SEG_OFFSETS_I32 && n >= (1ll << 31)) return MMV_ERR_INVALID_ARG;
+    if (!x || !seg || !out || !workspace) return MMV_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(seg) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return MMV_ERR_INVALID_ARG;
+    if (sf == MMV_SEG_OFFSETS_I32 && nseg == 0) return MMV_ERR_INVALID_ARG;   // n > 0 needs a segment
+    const WorkspacePlan plan = plan_workspace(MMV_OP_SEG_SCAN, sf, n);
+    if (workspace_bytes < plan.total) return MMV_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo* dev = device_info();
+    if (!dev) return MMV_ERR_CUDA;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    WorkspaceHeader* hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+    if (cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
+
+    const uint8_t* flags = static_cast<const uint8_t*>(seg);
+    if (sf == MMV_SEG_OFFSETS_I32) {
+        uint8_t* f = ws + plan.flags_off;
+        if (cudaMemsetAsync(f, 0, static_cast<size_t>(n), st) != cudaSuccess) return MMV_ERR_CUDA;
+        const int threads = 256;
+        long long blocks = (nseg + threads - 1) / threads;
+        if (blocks > dev->sm_count * 8) blocks = dev->sm_count * 8;
+        offsets_to_flags_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(static_cast<const int32_t*>(seg), nseg,
+                                                                                n, f, hdr);
+        ++g_launches;
+        flags = f;
+    }
+
+    const bool f16 = dt == MMV_F16_TO_F32;
+    CUtensorMap tmap;
+    if (!encode_rows_map(&tmap, x, n, f16)) return MMV_ERR_CUDA;
+
+    ScanParams prm;
+    prm.x = x;
+    prm.flags = flags;
+    prm.out = out;
+    prm.n = n;
+    prm.num_tiles = static_cast<int>(num_tiles_of(n));
+    prm.hdr = hdr;
+    prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
+    prm.budget_ns = g_budget_ns.load();
+    prm.debug_skip_span = g_debug_skip_span.load();
+    const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
+    if (f16)
+        seg_scan_kernel<F16Path><<<grid, SCAN_THREADS, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, prm);
+    else
+        seg_scan_kernel<I8Path><<<grid, SCAN_THREADS, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, prm);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+}
+
+mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
+                       void* out, int64_t* d_num_segments, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream) {
+    (void)d_num_segments;
+    if (n < 0 || nseg < 0) return MMV_ERR_INVALID_ARG;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
+    if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
+    if (sf == MMV_SEG_FLAGS_U8) return MMV_ERR_UNSUPPORTED;
+    return seg_sum_csr_launch(x, static_cast<const int32_t*>(seg), n, nseg, dt, out, workspace, workspace_bytes,
+                              cuda_stream);
+}
+
+mmv_status mmv_spmv_csr(const int32_t* rowptr, const int32_t* col, const void* val_f16, const float* x, float* y,
+                        int64_t rows, int64_t cols, int64_t nnz, void* workspace, size_t workspace_bytes,
+                        void* cuda_stream) {
+    return spmv_csr_launch(rowptr, col, val_f16, x, y, rows, cols, nnz, workspace, workspace_bytes, cuda_stream);
+}
+
+mmv_status mmv_last_async_status(const void* workspace, void* cuda_stream) {
+    if (!workspace) return MMV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return MMV_ERR_CUDA;
+    WorkspaceHeader h;
+    if (cudaMemcpy(&h, workspace, sizeof(unsigned int) * 2, cudaMemcpyDeviceToHost) != cudaSuccess) return MMV_ERR_CUDA;
+    return h.error <= 6u ? static_cast<mmv_status>(h.error) : MMV_ERR_CUDA;
+}
+
+const char* mmv_status_string(mmv_status s) {
+    switch (s) {
+        case MMV_OK: return "ok";
+        case MMV_ERR_INVALID_ARG: return "invalid argument";
+        case MMV_ERR_UNSUPPORTED: return "unsupported combination";
+        case MMV_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case MMV_ERR_BAD_SEGMENTS: return "segment offsets not monotone or out of range";
+        case MMV_ERR_TIMEOUT: return "device-side wait timed out";
+        case MMV_ERR_CUDA: return "CUDA call failed";
+    }
+    return "unknown status";
+}
+
+int64_t mmv_kernel_launch_count(void) { return g_launches.load(); }
+
+void mmv_debug_configure(int64_t wait_budget_ns, int64_t skip_publish_span) {
+    g_budget_ns.store(wait_budget_ns > 0 ? static_cast<unsigned long long>(wait_budget_ns) : WAIT_BUDGET_NS);
+    g_debug_skip_span.store(skip_publish_span);
+}
+
+}  // extern "C"
