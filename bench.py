@@ -1,0 +1,442 @@
+#!/usr/bin/env python
+"""Benchmark of the segmented scan / sum / SpMV library on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one pass of the segmented-scan hot path (tile load, tensor-core block
+prefix, flag pass, revert, carries, look-back, store) over the headline workload:
+the density-sweep configuration (n = 2^30 fp16 values uniform in [-1,1), fp32
+output) with Bernoulli(1e-3) start flags.  The line printed at the end also
+carries, under "configs", short measurements of all five configurations of
+the benchmark spec (N = 1 only).  Inputs are seeded and synthetic (mmv_inputs); they
+are generated on the host and uploaded before the timed region.  Every working
+set here is larger than the 126 MB L2 except configuration 1, for which a
+buffer larger than L2 is rewritten between timed launches.
+
+With --impl reference the same metric is produced by the CPU oracle on the
+box's host cores (a deliberately plain sequential program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import mmv_inputs as gen  # noqa: E402
+
+METRIC = "segmented scan throughput (input elements per second)"
+UNIT = "Gelem/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+# DRAM bytes per element of the headline kernel measured with ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum of one launch divided by its n); see profiles/.  None = not captured yet.
+NCU_TRAFFIC_BYTES_PER_ELEM = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--log2n", type=int, default=30, help="headline size (default 2^30)")
+    ap.add_argument("--case", default="p1e-3", help="flag pattern of the headline workload")
+    ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline")
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.kill()
+            self.proc.wait()
+            self.thread.join(timeout=1.0)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            parts = [p.strip() for p in r.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------
+# the reference arm: the CPU oracle, as it stands
+# ---------------------------------------------------------------------------
+def time_oracle_scan(x, f, reps=3):
+    import oracle
+    best = float("inf")
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        if x.dtype == np.int8:
+            oracle.seg_scan_i8(x, f)
+        else:
+            oracle.seg_scan_f16(x, f)
+        best = min(best, time.perf_counter() - t0)
+    return best
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    n = 1 << min(args.log2n, 27)          # bounded sample of the headline workload
+    x = gen.f16_uniform(5, n)
+    f = gen.config5_flags(n, args.case)
+    for _ in range(max(1, min(args.warmup, 2))):
+        oracle.seg_scan_f16(x, f)
+    steps = max(1, args.steps)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.seg_scan_f16(x, f)
+    dt = (time.perf_counter() - t0) / steps
+    val = n / dt / 1e9
+    sample = f"first 2^{int(np.log2(n))} elements of the headline workload per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"seg-scan fp16->fp32, flags {args.case}, CPU oracle on a sample", "n": n},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ---------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------
+def event_time_ms(torch, fn, steps, flush=None):
+    """Average device time of fn() over `steps` launches, CUDA events on the current stream."""
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1) / steps
+    total = 0.0
+    for _ in range(steps):
+        flush()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        e1.synchronize()
+        total += e0.elapsed_time(e1)
+    return total / steps
+
+
+def verify_scan_sample(torch, mmv, oracle, x, f, out_d, ws):
+    """Checks the device result on the head of the array and on a window that starts at a flag."""
+    n = x.shape[0]
+    m = min(n, 1 << 22)
+    windows = [(0, m)]
+    if n > 2 * m:
+        nz = np.flatnonzero(f[n // 2:n // 2 + m])
+        if nz.size:
+            s = n // 2 + int(nz[0])
+            windows.append((s, min(n, s + m)))
+    worst = 0.0
+    for a, b in windows:
+        got = out_d[a:b].cpu().numpy()
+        if x.dtype == np.int8:
+            want = oracle.seg_scan_i8(x[a:b], f[a:b])
+            if not np.array_equal(got, want):
+                raise SystemExit(f"bench: int8 scan mismatch in window {a}:{b}")
+        else:
+            z, ab = oracle.seg_scan_f16(x[a:b], f[a:b])
+            ok, ratio, i = oracle.check_fp(got, z, ab)
+            worst = max(worst, ratio)
+            if not ok:
+                raise SystemExit(f"bench: fp16 scan outside the bound in window {a}:{b}: ratio {ratio} at {a + i}")
+    return worst
+
+
+def bench_configs(torch, mmv, oracle, peak, steps, warmup, l2_flush):
+    """Short measurements of the five configurations (device-resident inputs)."""
+    res = []
+
+    def rec(name, units, bytes_, ms, extra=None):
+        d = {"config": name, "units": int(units), "ms": ms, "gelem_s": units / ms / 1e6,
+             "gb_s": bytes_ / ms / 1e6, "frac_of_measured_peak": bytes_ / ms / 1e6 / peak,
+             "frac_of_8tbs": bytes_ / ms / 1e6 / NOMINAL_HBM_GBS}
+        if extra:
+            d.update(extra)
+        res.append(d)
+
+    def run_scan(name, x, f, flush=None):
+        n = x.shape[0]
+        dt = mmv.F16_TO_F32 if x.dtype == np.float16 else mmv.I8_TO_I32
+        xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+        out = torch.empty(n, dtype=torch.float32 if dt == mmv.F16_TO_F32 else torch.int32, device="cuda")
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, dt, mmv.SEG_FLAGS_U8, n)
+        fn = lambda: mmv.seg_scan(xd, fd, out=out, workspace=ws)  # noqa: E731
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        ms = event_time_ms(torch, fn, steps, flush)
+        assert mmv.last_async_status(ws) == 0
+        worst = verify_scan_sample(torch, mmv, oracle, x, f, out, ws)
+        bpe = (2 if dt == mmv.F16_TO_F32 else 1) + 1 + 4
+        rec(name, n, n * bpe, ms, {"worst_err_over_bound": worst} if dt == mmv.F16_TO_F32 else {"mismatches": 0})
+        del xd, fd, out, ws
+
+    x, f = gen.config1()
+    run_scan("C1 seg-scan n=2^20 fp16 flags 1/64 (L2 flushed between launches)", x, f, l2_flush)
+
+    x, off = gen.config2()
+    n, nseg = x.shape[0], off.shape[0] - 1
+    xd, od = torch.from_numpy(x).cuda(), torch.from_numpy(off).cuda()
+    out = torch.empty(nseg, dtype=torch.float32, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, n, nseg)
+    fn = lambda: mmv.seg_sum(xd, od, out=out, workspace=ws)  # noqa: E731
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ms = event_time_ms(torch, fn, steps)
+    assert mmv.last_async_status(ws) == 0
+    want, a = oracle.seg_sum_csr_f16(x, off)
+    ok, ratio, i = oracle.check_fp(out.cpu().numpy(), want, a)
+    if not ok:
+        raise SystemExit(f"bench: config 2 outside the bound: ratio {ratio} at segment {i}")
+    rec("C2 seg-sum n=2^26 fp16 N(0,1), CSR offsets len U{1..4096}", n, 2 * n + 4 * (nseg + 1) + 4 * nseg, ms,
+        {"segments": nseg, "worst_err_over_bound": ratio})
+    del xd, od, out, ws
+
+    x, f = gen.config3()
+    run_scan("C3 seg-scan n=2^28 int8 flags 1e-3", x, f)
+
+    rowptr, col, val, xv = gen.config4()
+    rows, nnz = rowptr.shape[0] - 1, val.shape[0]
+    rd, cd, vd, xd = (torch.from_numpy(t).cuda() for t in (rowptr, col, val, xv))
+    y = torch.empty(rows, dtype=torch.float32, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, nnz, rows)
+    fn = lambda: mmv.spmv_csr(rd, cd, vd, xd, y=y, workspace=ws)  # noqa: E731
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ms = event_time_ms(torch, fn, steps)
+    assert mmv.last_async_status(ws) == 0
+    want, a = oracle.spmv_csr(rowptr, col, val, xv)
+    ok, ratio, i = oracle.check_fp(y.cpu().numpy(), want, a)
+    if not ok:
+        raise SystemExit(f"bench: config 4 outside the bound: ratio {ratio} at row {i}")
+    rec("C4 CSR SpMV 2^20 rows, nnz/row Zipf(1.5) cap 1e4", nnz, 6 * nnz + 4 * (rows + 1) + 4 * xv.shape[0] + 4 * rows,
+        ms, {"nnz": nnz, "worst_err_over_bound": ratio})
+    del rd, cd, vd, xd, y, ws
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    import paper_2506_23906_b200 as mmv
+    import oracle
+
+    if rank == 0:
+        oracle.build()
+    n = 1 << args.log2n
+    x = gen.f16_uniform(5, n)
+    f = gen.config5_flags(n, args.case)
+    peak, peak_kind = measured_peak()
+
+    # pinned host buffers (end-to-end leg) and device-resident copies (kernel leg)
+    xh = torch.from_numpy(x).pin_memory()
+    fh = torch.from_numpy(f).pin_memory()
+    oh = torch.empty(n, dtype=torch.float32).pin_memory()
+    xd = torch.empty(n, dtype=torch.float16, device="cuda")
+    fd = torch.empty(n, dtype=torch.uint8, device="cuda")
+    od = torch.empty(n, dtype=torch.float32, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+    xd.copy_(xh)
+    fd.copy_(fh)
+    l2_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def step():
+        mmv.seg_scan(xd, fd, out=od, workspace=ws)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    launches0 = mmv.kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        barrier()
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        barrier()
+    launches = mmv.kernel_launch_count() - launches0
+    ms = e0.elapsed_time(e1) / args.steps
+    if mmv.last_async_status(ws) != 0:
+        raise SystemExit("bench: device-side error status")
+    worst = verify_scan_sample(torch, mmv, oracle, x, f, od, ws)
+
+    # end to end: pinned host -> device, the call, device -> host, every step
+    e2e_steps = max(1, min(args.steps, 5))
+    def e2e_step():
+        xd.copy_(xh, non_blocking=True)
+        fd.copy_(fh, non_blocking=True)
+        mmv.seg_scan(xd, fd, out=od, workspace=ws)
+        oh.copy_(od, non_blocking=True)
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        bytes_per_launch = 7 * n
+        achieved = bytes_per_launch / ms / 1e6
+        line = {
+            "metric": METRIC, "value": world * n / ms / 1e6, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"C5 seg-scan n=2^{args.log2n} fp16 U[-1,1) -> fp32, uint8 flags {args.case}",
+                       "n_per_gpu": n, "timing": "inputs (7 B/elem working set) larger than L2; no flush needed",
+                       "parallelism": f"{world} independent shards, no collective"},
+            "clocks": clk.summary(),
+            "e2e": {"value": world * n / e2e_ms / 1e6, "unit": UNIT, "h2d_bytes_per_step": 3 * n,
+                    "d2h_bytes_per_step": 4 * n, "ms_per_step": e2e_ms, "steps": e2e_steps},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": peak_kind,
+                         "frac_of_8tbs_nominal": achieved / NOMINAL_HBM_GBS,
+                         "algorithmic_bytes_per_elem": 7,
+                         "traffic": None if NCU_TRAFFIC_BYTES_PER_ELEM is None else NCU_TRAFFIC_BYTES_PER_ELEM * n},
+            "worst_err_over_bound": worst,
+        }
+        del xh, fh, oh
+        if not args.no_cpu:
+            sec = time_oracle_scan(x, f, reps=3)
+            line["cpu_baseline"] = {"value": n / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": f"the whole headline workload (n=2^{args.log2n}), best of 3, {sec:.2f} s"}
+        del xd, fd, od
+        torch.cuda.empty_cache()
+        if world == 1 and not args.no_configs:
+            def l2_flush():
+                l2_buf.zero_()
+            cfgs = bench_configs(torch, mmv, oracle, peak, min(args.steps, 20), max(3, args.warmup), l2_flush)
+            # the seven flag patterns of configuration 5 on the headline values
+            xd = torch.from_numpy(x).cuda()
+            od = torch.empty(n, dtype=torch.float32, device="cuda")
+            sweep = []
+            for case, _ in gen.C5_CASES:
+                fc = gen.config5_flags(n, case)
+                fd = torch.from_numpy(fc).cuda()
+                fn = lambda: mmv.seg_scan(xd, fd, out=od, workspace=ws)  # noqa: E731
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                cms = event_time_ms(torch, fn, min(args.steps, 10))
+                assert mmv.last_async_status(ws) == 0
+                w = verify_scan_sample(torch, mmv, oracle, x, fc, od, ws)
+                sweep.append({"case": case, "ms": cms, "gelem_s": n / cms / 1e6, "gb_s": 7 * n / cms / 1e6,
+                              "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
+                              "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS, "worst_err_over_bound": w})
+                del fd
+            line["configs"] = cfgs
+            line["c5_density_sweep"] = sweep
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -63,7 +63,9 @@ DeviceInfo* device_info() {
         bool ok = true;
         ok &= set_smem(seg_scan_kernel<F16Path>, ScanCfg<F16Path>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<I8Path>, ScanCfg<I8Path>::kSmemBytes);
-        ok &= seg_sum_set_attributes();
+        ok &= set_smem(seg_sum_kernel<F16Path>, SumCfg<F16Path>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<I8Path>, SumCfg<I8Path>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<BF16Path>, SumCfg<BF16Path>::kSmemBytes);
         d->ok = ok;
     });
     return d->ok ? d : nullptr;
@@ -93,9 +95,35 @@ bool encode_rows_map(CUtensorMap* map, const void* x, long long n, bool is_f16) 
     return r == CUDA_SUCCESS;
 }
 
+// The value vector as [spans][4 pieces][32 rows][32 elements] (full spans only); one box =
+// piece i of four consecutive spans = the 128 x 32 A operand of one tensor-core product.
+bool encode_span_map(CUtensorMap* map, const void* x, long long n, int elem_bytes, bool bf16) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t spans = static_cast<cuuint64_t>(n / SPAN);
+    if (spans == 0) {
+        std::memset(map, 0, sizeof(*map));
+        return true;
+    }
+    const cuuint64_t rb = static_cast<cuuint64_t>(ROW) * elem_bytes;
+    cuuint64_t dims[4] = {ROW, PIECE_ROWS, PIECES_PER_SPAN, spans};
+    cuuint64_t strides[3] = {rb, rb * PIECE_ROWS, rb * PIECE_ROWS * PIECES_PER_SPAN};
+    cuuint32_t box[4] = {ROW, PIECE_ROWS, 1, SPANS_PER_TILE};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    (void)bf16;
+    CUresult r = enc(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4,
+                     const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     elem_bytes == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 struct WorkspacePlan {
     size_t status_off, status_bytes;
     size_t flags_off, flags_bytes;     // scratch flag bytes (offset-encoded scan only)
+    size_t tileq_off, tileq_bytes;     // per-tile first boundary index (seg-sum, SpMV)
+    size_t prod_off, prod_bytes;       // bf16 hi/lo halves of the products (SpMV)
+    long long n_eff;                   // elements the tiled kernel runs over
     size_t total;
 };
 
@@ -103,13 +131,88 @@ long long num_tiles_of(long long n) { return (n + TILE - 1) / TILE; }
 
 WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     WorkspacePlan p{};
-    const long long tiles = num_tiles_of(n);
+    p.n_eff = (op == MMV_OP_SPMV_CSR) ? 2 * n : n;
+    const long long tiles = num_tiles_of(p.n_eff);
     p.status_off = sizeof(WorkspaceHeader);
     p.status_bytes = round_up(static_cast<size_t>(tiles) * SPANS_PER_TILE * sizeof(uint64_t), 256);
     p.flags_off = p.status_off + p.status_bytes;
     p.flags_bytes = (op == MMV_OP_SEG_SCAN && sf == MMV_SEG_OFFSETS_I32) ? round_up(static_cast<size_t>(n), 256) : 0;
-    p.total = p.flags_off + p.flags_bytes;
+    p.tileq_off = p.flags_off + p.flags_bytes;
+    p.tileq_bytes = (op != MMV_OP_SEG_SCAN) ? round_up(static_cast<size_t>(tiles + 1) * sizeof(int32_t), 256) : 0;
+    p.prod_off = p.tileq_off + p.tileq_bytes;
+    p.prod_bytes = (op == MMV_OP_SPMV_CSR) ? round_up(static_cast<size_t>(n) * 4, 256) : 0;
+    p.total = p.prod_off + p.prod_bytes;
     return p;
+}
+
+// z(k) = val(k) * x(col(k)) in fp32 (Algorithm A.5, CsrGather), written as two bf16 halves
+// (hi = bf16(z), lo = bf16(z - hi)) so that the segmented sum can feed them to the tensor core.
+__global__ void spmv_gather_kernel(const int32_t* __restrict__ col, const __half* __restrict__ val,
+                                   const float* __restrict__ x, uint32_t* __restrict__ prod, long long nnz) {
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    const long long nvec = nnz >> 2;
+    for (long long v = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; v < nvec; v += stride) {
+        const int4 c = __ldg(reinterpret_cast<const int4*>(col) + v);
+        const uint2 hv = __ldg(reinterpret_cast<const uint2*>(val) + v);
+        const __half2 h01 = *reinterpret_cast<const __half2*>(&hv.x);
+        const __half2 h23 = *reinterpret_cast<const __half2*>(&hv.y);
+        float z[4];
+        z[0] = __low2float(h01) * __ldg(x + c.x);
+        z[1] = __high2float(h01) * __ldg(x + c.y);
+        z[2] = __low2float(h23) * __ldg(x + c.z);
+        z[3] = __high2float(h23) * __ldg(x + c.w);
+        uint32_t o[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(z[e]);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(z[e] - __bfloat162float(hi));
+            o[e] = static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(lo)) << 16);
+        }
+        *(reinterpret_cast<uint4*>(prod) + v) = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    // ragged tail (nnz not a multiple of 4)
+    const long long k = (nvec << 2) + static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (k < nnz) {
+        const float z = __half2float(val[k]) * __ldg(x + col[k]);
+        const __nv_bfloat16 hi = __float2bfloat16_rn(z);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(z - __bfloat162float(hi));
+        prod[k] = static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(lo)) << 16);
+    }
+}
+
+// Shared launcher of the tiled segmented-sum kernel.  `values` holds n_eff elements of the
+// path's type; boundaries are off[q] << shift.  The header and status words must have been
+// cleared on the stream already.
+template <typename P>
+mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* off, long long nseg, int shift,
+                          void* out, uint8_t* ws, const WorkspacePlan& plan, DeviceInfo* dev, cudaStream_t st) {
+    const int tiles = static_cast<int>(num_tiles_of(n_eff));
+    int32_t* tile_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
+    {
+        const int warps = tiles + 1;
+        const int threads = 256;
+        const int blocks = (warps * 32 + threads - 1) / threads;
+        partition_offsets_kernel<<<blocks, threads, 0, st>>>(off, nseg, shift, tiles, tile_q, n_eff,
+                                                             reinterpret_cast<WorkspaceHeader*>(ws));
+        ++g_launches;
+    }
+    CUtensorMap tmap;
+    if (!encode_span_map(&tmap, values, n_eff, P::kElemBytes, false)) return MMV_ERR_CUDA;
+    SumParams prm;
+    prm.off = off;
+    prm.nseg = nseg;
+    prm.n = n_eff;
+    prm.off_shift = shift;
+    prm.out = out;
+    prm.num_tiles = tiles;
+    prm.tile_q = tile_q;
+    prm.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+    prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
+    prm.budget_ns = g_budget_ns.load();
+    const int grid = tiles < dev->sm_count ? tiles : dev->sm_count;
+    seg_sum_kernel<P><<<grid, SUM_THREADS, SumCfg<P>::kSmemBytes, st>>>(tmap, values, prm);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
 
 // f[off[r]] = 1 for every non-empty segment r (scratch flags of the offset-encoded scan).
@@ -207,14 +310,60 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
     if (sf == MMV_SEG_FLAGS_U8) return MMV_ERR_UNSUPPORTED;
-    return seg_sum_csr_launch(x, static_cast<const int32_t*>(seg), n, nseg, dt, out, workspace, workspace_bytes,
-                              cuda_stream);
+    if (n >= (1ll << 31)) return MMV_ERR_INVALID_ARG;            // int32 offsets cannot address more
+    if (nseg == 0) return MMV_OK;
+    if (!seg || !out) return MMV_ERR_INVALID_ARG;
+    if (!aligned16(seg) || !aligned16(out)) return MMV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (n == 0) {                                                // every segment is empty
+        return cudaMemsetAsync(out, 0, static_cast<size_t>(nseg) * 4, st) == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+    }
+    if (!x || !workspace) return MMV_ERR_INVALID_ARG;
+    if (!aligned16(x) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MMV_ERR_INVALID_ARG;
+    const WorkspacePlan plan = plan_workspace(MMV_OP_SEG_SUM, sf, n);
+    if (workspace_bytes < plan.total) return MMV_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo* dev = device_info();
+    if (!dev) return MMV_ERR_CUDA;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
+    const int32_t* off = static_cast<const int32_t*>(seg);
+    if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, nseg, 0, out, ws, plan, dev, st);
+    return launch_seg_sum<I8Path>(x, n, off, nseg, 0, out, ws, plan, dev, st);
 }
 
 mmv_status mmv_spmv_csr(const int32_t* rowptr, const int32_t* col, const void* val_f16, const float* x, float* y,
                         int64_t rows, int64_t cols, int64_t nnz, void* workspace, size_t workspace_bytes,
                         void* cuda_stream) {
-    return spmv_csr_launch(rowptr, col, val_f16, x, y, rows, cols, nnz, workspace, workspace_bytes, cuda_stream);
+    if (rows < 0 || cols < 0 || nnz < 0) return MMV_ERR_INVALID_ARG;
+    if (nnz >= (1ll << 30)) return MMV_ERR_INVALID_ARG;          // 2 * nnz must fit int32 offsets
+    if (rows == 0) return MMV_OK;
+    if (!rowptr || !y) return MMV_ERR_INVALID_ARG;
+    if (!aligned16(rowptr) || !aligned16(y)) return MMV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (nnz == 0) {
+        return cudaMemsetAsync(y, 0, static_cast<size_t>(rows) * 4, st) == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+    }
+    if (!col || !val_f16 || !x || !workspace || cols == 0) return MMV_ERR_INVALID_ARG;
+    if (!aligned16(col) || !aligned16(val_f16) || !aligned16(x) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return MMV_ERR_INVALID_ARG;
+    const WorkspacePlan plan = plan_workspace(MMV_OP_SPMV_CSR, MMV_SEG_OFFSETS_I32, nnz);
+    if (workspace_bytes < plan.total) return MMV_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo* dev = device_info();
+    if (!dev) return MMV_ERR_CUDA;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
+    uint32_t* prod = reinterpret_cast<uint32_t*>(ws + plan.prod_off);
+    {
+        const int threads = 256;
+        long long blocks = ((nnz >> 2) + threads - 1) / threads;
+        const long long cap = static_cast<long long>(dev->sm_count) * 16;
+        if (blocks > cap) blocks = cap;
+        if (blocks < 1) blocks = 1;
+        spmv_gather_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(col, static_cast<const __half*>(val_f16), x,
+                                                                              prod, nnz);
+        ++g_launches;
+    }
+    return launch_seg_sum<BF16Path>(prod, 2 * nnz, rowptr, rows, 1, y, ws, plan, dev, st);
 }
 
 mmv_status mmv_last_async_status(const void* workspace, void* cuda_stream) {

@@ -47,6 +47,8 @@ struct F16Path {
     static constexpr int kKStepBytes = 32;
     static constexpr uint32_t kLayoutType = 4;             // SWIZZLE_64B
     static constexpr uint32_t kSbo = 8 * kRowBytes;        // 512
+    static constexpr uint32_t kOneBits = 0x3C00u;          // 1.0 in fp16
+    static constexpr uint32_t kFmtBits = 0u;               // instruction-descriptor A/B format: f16
     __device__ static __forceinline__ Acc from_bits(uint32_t b) { return __uint_as_float(b); }
     __device__ static __forceinline__ uint32_t to_bits(Acc v) { return __float_as_uint(v); }
     __device__ static __forceinline__ Acc add(Acc a, Acc b) { return a + b; }
@@ -62,6 +64,8 @@ struct I8Path {
     static constexpr int kKStepBytes = 32;
     static constexpr uint32_t kLayoutType = 6;             // SWIZZLE_32B
     static constexpr uint32_t kSbo = 8 * kRowBytes;        // 256
+    static constexpr uint32_t kOneBits = 1u;
+    static constexpr uint32_t kFmtBits = 0u;
     __device__ static __forceinline__ Acc from_bits(uint32_t b) { return b; }
     __device__ static __forceinline__ uint32_t to_bits(Acc v) { return v; }
     __device__ static __forceinline__ Acc add(Acc a, Acc b) { return a + b; }

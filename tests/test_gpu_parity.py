@@ -1,0 +1,276 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle.
+
+int8 -> int32 paths are compared bit for bit; fp16 -> fp32 paths must satisfy
+|gpu - oracle| <= 2e-3 * (sum of |x| over the summed range) + 1e-6 per element.
+Sizes span several 16384-element tiles and ragged tails.
+"""
+import numpy as np
+import pytest
+
+import mmv_inputs as gen
+import oracle
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TILE = 16384
+
+
+@pytest.fixture(scope="module")
+def mmv():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2506_23906_b200 as m
+    m.debug_configure(0, -1)
+    return m
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def scan_i8(mmv, x, f, guard=64):
+    n = x.shape[0]
+    seg = dev(f)
+    sf = mmv.SEG_FLAGS_U8 if f.dtype == np.uint8 else mmv.SEG_OFFSETS_I32
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, sf, n, max(0, f.shape[0] - 1))
+    buf = torch.full((n + guard,), -777, dtype=torch.int32, device="cuda")
+    mmv.seg_scan(dev(x), seg, out=buf[:n], workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    got = buf.cpu().numpy()
+    assert (got[n:] == -777).all(), "wrote past the end of the output"
+    return got[:n]
+
+
+def scan_f16(mmv, x, f, guard=64):
+    n = x.shape[0]
+    sf = mmv.SEG_FLAGS_U8 if f.dtype == np.uint8 else mmv.SEG_OFFSETS_I32
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.F16_TO_F32, sf, n, max(0, f.shape[0] - 1))
+    buf = torch.full((n + guard,), -777.0, dtype=torch.float32, device="cuda")
+    mmv.seg_scan(dev(x), dev(f), out=buf[:n], workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    got = buf.cpu().numpy()
+    assert (got[n:] == -777.0).all(), "wrote past the end of the output"
+    return got[:n]
+
+
+def assert_fp(got, z, a, what):
+    ok, ratio, i = oracle.check_fp(got, z, a)
+    assert ok, f"{what}: |err|/bound = {ratio:.3g} at index {i}: got {got[i]!r}, want {z[i]!r}"
+    return ratio
+
+
+SIZES = [1, 2, 31, 32, 33, 1023, 1024, 1025, 4095, 4096, 4097, TILE - 1, TILE, TILE + 1,
+         2 * TILE - 1, 2 * TILE + 1, 5 * TILE + 4099, 100_003]
+
+
+@pytest.mark.parametrize("n", SIZES)
+def test_scan_i8_sizes(mmv, n):
+    rng = np.random.default_rng(n)
+    x = rng.integers(-128, 128, n).astype(np.int8)
+    for p in (0.0, 0.01, 0.3, 1.0):
+        f = (rng.random(n) < p).astype(np.uint8)
+        assert np.array_equal(scan_i8(mmv, x, f), oracle.seg_scan_i8(x, f)), (n, p)
+
+
+@pytest.mark.parametrize("n", SIZES)
+def test_scan_f16_sizes(mmv, n):
+    rng = np.random.default_rng(n + 1)
+    x = rng.uniform(-1, 1, n).astype(np.float16)
+    for p in (0.0, 1.0 / 64, 0.5, 1.0):
+        f = (rng.random(n) < p).astype(np.uint8)
+        z, a = oracle.seg_scan_f16(x, f)
+        assert_fp(scan_f16(mmv, x, f), z, a, f"n={n} p={p}")
+
+
+def test_scan_flag_positions_around_row_and_tile_edges(mmv):
+    n = 3 * TILE
+    rng = np.random.default_rng(5)
+    x = rng.integers(-8, 8, n).astype(np.int8)
+    xf = rng.uniform(-1, 1, n).astype(np.float16)
+    for pos in (1, 31, 32, 33, 1023, 1024, 4095, 4096, 4097, TILE - 1, TILE, TILE + 1, 2 * TILE, n - 1):
+        f = np.zeros(n, np.uint8)
+        f[pos] = 1
+        assert np.array_equal(scan_i8(mmv, x, f), oracle.seg_scan_i8(x, f)), pos
+        f[min(n - 1, pos + 1)] = 1
+        f[pos - 1] = 1
+        assert np.array_equal(scan_i8(mmv, x, f), oracle.seg_scan_i8(x, f)), pos
+        z, a = oracle.seg_scan_f16(xf, f)
+        assert_fp(scan_f16(mmv, xf, f), z, a, f"flags around {pos}")
+
+
+def test_scan_closed_forms(mmv):
+    n = 2 * TILE + 77
+    ones = np.ones(n, np.int8)
+    f = gen.flags(9, n, pattern="cycle123")
+    assert np.array_equal(scan_i8(mmv, ones, f), np.tile([1, 1, 2, 1, 2, 3], n // 6 + 1)[:n])
+    f = np.zeros(n, np.uint8)
+    assert np.array_equal(scan_i8(mmv, ones, f), np.arange(1, n + 1))
+    f = np.ones(n, np.uint8)
+    x = np.random.default_rng(3).uniform(-1, 1, n).astype(np.float16)
+    assert np.array_equal(scan_f16(mmv, x, f), x.astype(np.float32))      # identity, exactly
+    # flag byte values other than 1 count, and flag[0] is ignored
+    f = np.zeros(n, np.uint8)
+    f[[5, 4096, 20000]] = [200, 2, 128]
+    assert np.array_equal(scan_i8(mmv, ones, f), oracle.seg_scan_i8(ones, f))
+
+
+def test_scan_int_wraps_mod_2_32(mmv):
+    n = 1 << 25
+    x = np.full(n, -128, np.int8)
+    f = np.zeros(n, np.uint8)
+    got = scan_i8(mmv, x, f)
+    assert got[-1] == 0 and got[(1 << 24) - 1] == -2 ** 31 and got[1 << 24] == 2 ** 31 - 128
+    assert np.array_equal(got, oracle.seg_scan_i8(x, f))
+
+
+def test_scan_with_offsets(mmv):
+    rng = np.random.default_rng(11)
+    lens = rng.integers(0, 300, 700)
+    off = gen.offsets_from_lengths(lens)
+    n = int(off[-1])
+    x = rng.integers(-128, 128, n).astype(np.int8)
+    f = oracle.flags_from_offsets(off, n)
+    assert np.array_equal(scan_i8(mmv, x, off), oracle.seg_scan_i8(x, f))
+    xf = rng.uniform(-1, 1, n).astype(np.float16)
+    z, a = oracle.seg_scan_f16(xf, f)
+    assert_fp(scan_f16(mmv, xf, off), z, a, "offset-encoded scan")
+
+
+def test_scan_is_deterministic_for_integers(mmv):
+    x, f = gen.config3(1 << 22)
+    a = scan_i8(mmv, x, f)
+    for _ in range(3):
+        assert np.array_equal(scan_i8(mmv, x, f), a)
+
+
+def test_config1_full(mmv):
+    x, f = gen.config1()
+    z, a = oracle.seg_scan_f16(x, f)
+    assert_fp(scan_f16(mmv, x, f), z, a, "config 1")
+
+
+def test_config3_reduced_and_config5_cases_reduced(mmv):
+    x, f = gen.config3(1 << 24)
+    assert np.array_equal(scan_i8(mmv, x, f), oracle.seg_scan_i8(x, f))
+    n = 1 << 23
+    xv = gen.config5_values(n)
+    for case, _ in gen.C5_CASES:
+        f = gen.config5_flags(n, case)
+        z, a = oracle.seg_scan_f16(xv, f)
+        assert_fp(scan_f16(mmv, xv, f), z, a, f"config 5 / {case}")
+
+
+# ---------------------------------------------------------------------------
+# segmented sum over CSR offsets
+# ---------------------------------------------------------------------------
+def sum_csr(mmv, x, off, guard=16):
+    n, nseg = x.shape[0], off.shape[0] - 1
+    dt = mmv.F16_TO_F32 if x.dtype == np.float16 else mmv.I8_TO_I32
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, dt, mmv.SEG_OFFSETS_I32, n, nseg)
+    tdt = torch.float32 if x.dtype == np.float16 else torch.int32
+    buf = torch.full((nseg + guard,), -777, dtype=tdt, device="cuda")
+    xd = dev(x) if n else torch.empty(0, dtype=torch.float16 if x.dtype == np.float16 else torch.int8, device="cuda")
+    mmv.seg_sum(xd, dev(off), out=buf[:nseg], workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    got = buf.cpu().numpy()
+    assert (got[nseg:] == -777).all()
+    return got[:nseg]
+
+
+@pytest.mark.parametrize("maxlen,nseg", [(1, 5000), (3, 40000), (40, 3000), (700, 300), (5000, 60), (40000, 9)])
+def test_seg_sum_csr_random_lengths(mmv, maxlen, nseg):
+    rng = np.random.default_rng(maxlen)
+    lens = rng.integers(0, maxlen + 1, nseg)
+    off = gen.offsets_from_lengths(lens)
+    n = int(off[-1])
+    x = rng.integers(-128, 128, n).astype(np.int8)
+    assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
+    xf = rng.standard_normal(n).astype(np.float16)
+    want, a = oracle.seg_sum_csr_f16(xf, off)
+    got = sum_csr(mmv, xf, off)
+    assert_fp(got, want, a, f"maxlen={maxlen}")
+    assert (got[lens == 0] == 0).all()
+
+
+def test_seg_sum_csr_edges(mmv):
+    g = __import__("conftest").load_golden("csr_examples.txt")
+    x = np.asarray(g["sum_x"], np.int8)
+    off = np.asarray(g["sum_off"], np.int32)
+    assert sum_csr(mmv, x, off).tolist() == g["sum_out"]
+    # one segment covering everything; boundaries exactly on row / piece / span / tile edges
+    n = 3 * TILE + 5
+    x = np.random.default_rng(1).integers(-128, 128, n).astype(np.int8)
+    assert np.array_equal(sum_csr(mmv, x, np.asarray([0, n], np.int32)), oracle.seg_sum_csr_i8(x, np.asarray([0, n], np.int32)))
+    off = np.asarray([0, 0, 32, 1024, 1024, 4096, TILE, TILE, TILE + 1, 2 * TILE + 4096, n, n, n], np.int32)
+    assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
+    # segments that do not cover the ends of x: values outside [off[0], off[-1]) are ignored
+    off = np.asarray([100, 5000, 5000, 40000], np.int32)
+    assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
+    # all segments empty, no values at all
+    off = np.zeros(9, np.int32)
+    assert sum_csr(mmv, np.zeros(0, np.int8), off).tolist() == [0] * 8
+
+
+def test_seg_sum_config2_reduced(mmv):
+    x, off = gen.config2(1 << 22)
+    want, a = oracle.seg_sum_csr_f16(x, off)
+    assert_fp(sum_csr(mmv, x, off), want, a, "config 2 (n = 2^22)")
+
+
+# ---------------------------------------------------------------------------
+# CSR SpMV
+# ---------------------------------------------------------------------------
+def spmv(mmv, rowptr, col, val, x):
+    rows = rowptr.shape[0] - 1
+    ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, val.shape[0], rows)
+    y = mmv.spmv_csr(dev(rowptr), dev(col), dev(val), dev(x), workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    return y.cpu().numpy()
+
+
+def test_spmv_golden_and_random(mmv):
+    g = __import__("conftest").load_golden("csr_examples.txt")
+    y = spmv(mmv, np.asarray(g["spmv_rowptr"], np.int32), np.asarray(g["spmv_col"], np.int32),
+             np.asarray(g["spmv_val"], np.float32).astype(np.float16), np.asarray(g["spmv_x"], np.float32))
+    assert y.tolist() == g["spmv_y"]
+    for rows, frac in ((3000, 0.0), (20000, 0.1)):
+        rowptr, col, val, x = gen.config4(rows=rows, empty_fraction=frac)
+        want, a = oracle.spmv_csr(rowptr, col, val, x)
+        got = spmv(mmv, rowptr, col, val, x)
+        assert_fp(got, want, a, f"spmv rows={rows}")
+        assert (got[np.diff(rowptr) == 0] == 0).all()
+
+
+# ---------------------------------------------------------------------------
+# robustness
+# ---------------------------------------------------------------------------
+def test_bad_offsets_are_reported_not_trapped(mmv):
+    n = 50000
+    x = dev(np.ones(n, np.int8))
+    off = dev(np.asarray([0, 30000, 20000, n], np.int32))
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.I8_TO_I32, mmv.SEG_OFFSETS_I32, n, 3)
+    mmv.seg_sum(x, off, workspace=ws)
+    assert mmv.last_async_status(ws) == 4
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, mmv.SEG_OFFSETS_I32, n, 3)
+    mmv.seg_scan(x, off, workspace=ws)
+    assert mmv.last_async_status(ws) == 4
+    # the context is still usable
+    f = np.zeros(n, np.uint8)
+    assert np.array_equal(scan_i8(mmv, np.ones(n, np.int8), f), np.arange(1, n + 1))
+
+
+def test_lookback_wait_gives_up_with_a_status(mmv):
+    # one span never publishes its carry: its successors must time out, report it and return
+    n = 40 * TILE
+    x, f = dev(np.ones(n, np.int8)), dev(np.zeros(n, np.uint8))
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    try:
+        mmv.debug_configure(20_000_000, 17)           # 20 ms budget, span 17 stays silent
+        mmv.seg_scan(x, f, workspace=ws)
+        assert mmv.last_async_status(ws) == 5
+    finally:
+        mmv.debug_configure(0, -1)
+    out = mmv.seg_scan(x, f, workspace=ws)            # and the next call works
+    assert mmv.last_async_status(ws) == 0
+    assert np.array_equal(out.cpu().numpy(), np.arange(1, n + 1))
