@@ -12,6 +12,8 @@
 #include "common.cuh"
 #include "seg_scan.cuh"
 #include "seg_sum.cuh"
+#include "seg_scan2.cuh"
+#include <cstdlib>
 
 namespace mmv {
 namespace {
@@ -63,6 +65,8 @@ DeviceInfo* device_info() {
         bool ok = true;
         ok &= set_smem(seg_scan_kernel<F16Path>, ScanCfg<F16Path>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<I8Path>, ScanCfg<I8Path>::kSmemBytes);
+        ok &= set_smem(seg_scan2_kernel<F16Path>, Scan2Cfg<F16Path>::kSmemBytes);
+        ok &= set_smem(seg_scan2_kernel<I8Path>, Scan2Cfg<I8Path>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<F16Path>, SumCfg<F16Path>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<I8Path>, SumCfg<I8Path>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<BF16Path>, SumCfg<BF16Path>::kSmemBytes);
@@ -115,6 +119,25 @@ bool encode_span_map(CUtensorMap* map, const void* x, long long n, int elem_byte
                      const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      elem_bytes == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// The output vector as rows of 32 four-byte values (full rows only); box = one 32 x 32 piece.
+bool encode_out_map(CUtensorMap* map, void* out, long long n) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t rows = static_cast<cuuint64_t>(n / ROW);
+    if (rows == 0) {
+        std::memset(map, 0, sizeof(*map));
+        return true;
+    }
+    cuuint64_t dims[2] = {ROW, rows};
+    cuuint64_t strides[1] = {ROW * 4};
+    cuuint32_t box[2] = {ROW, PIECE_ROWS};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, out, dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
@@ -280,8 +303,14 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
     }
 
     const bool f16 = dt == MMV_F16_TO_F32;
-    CUtensorMap tmap;
-    if (!encode_rows_map(&tmap, x, n, f16)) return MMV_ERR_CUDA;
+    static const bool use_v1 = std::getenv("MMV_SCAN_V1") != nullptr;
+    CUtensorMap tmap, tmap_out;
+    if (use_v1) {
+        if (!encode_rows_map(&tmap, x, n, f16)) return MMV_ERR_CUDA;
+    } else {
+        if (!encode_span_map(&tmap, x, n, f16 ? 2 : 1, false)) return MMV_ERR_CUDA;
+        if (!encode_out_map(&tmap_out, out, n)) return MMV_ERR_CUDA;
+    }
 
     ScanParams prm;
     prm.x = x;
@@ -294,10 +323,17 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
     prm.budget_ns = g_budget_ns.load();
     prm.debug_skip_span = g_debug_skip_span.load();
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
-    if (f16)
-        seg_scan_kernel<F16Path><<<grid, SCAN_THREADS, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, prm);
-    else
-        seg_scan_kernel<I8Path><<<grid, SCAN_THREADS, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, prm);
+    if (use_v1) {
+        if (f16)
+            seg_scan_kernel<F16Path><<<grid, SCAN_THREADS, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, prm);
+        else
+            seg_scan_kernel<I8Path><<<grid, SCAN_THREADS, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, prm);
+    } else {
+        if (f16)
+            seg_scan2_kernel<F16Path><<<grid, SC2_THREADS, Scan2Cfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+        else
+            seg_scan2_kernel<I8Path><<<grid, SC2_THREADS, Scan2Cfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+    }
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }

@@ -1,0 +1,493 @@
+// Single-pass segmented inclusive scan (Problem 2.1, Eq. 1) for sm_100a, row-major layout.
+//
+// The value vector is the paper's ceil(n/s) x s matrix with s = ROW = 32.  A warp owns a
+// SPAN of 128 consecutive rows (4096 elements) in four PIECES of 32 rows; a TILE is four
+// spans.  For each tile:
+//   producer warp  one 4-D TMA box per piece index i (the [128 rows x 32] matrix made of
+//                  piece i of the four spans, K-major, hardware swizzle) and one bulk copy
+//                  of the tile's 16 KB of flag bytes.
+//   MMA warp       tcgen05.mma, A = that matrix, B = the constant [U_32 | I_32] (fp16) or
+//                  U_32 (int8):  TMEM lane 32w+l, column j (< 32) = inclusive prefix at
+//                  position j of row l of piece i of span w, the speculative block scan
+//                  z = MATMUL(x, U_s) of Algorithm A.1 (BlockSegScan); columns 32..63 (fp16)
+//                  return the row itself converted exactly to fp32.
+//   epilogue warps (lane = row; two warpgroups on alternating tiles)
+//     pre-pass     flag bytes -> one 32-bit start mask per row; row totals (TMEM column 31);
+//                  from these the span's aggregate (sum of its open tail segment, any flag)
+//                  is formed with a handful of shuffles and published at once; a decoupled
+//                  look-back over the earlier spans' status words returns the carry (this
+//                  replaces the recursion of Section 4.2 / Algorithm A.1's Recurse).
+//     main pass    per piece: revert the speculation inside each row (Lemma A.1: subtract the
+//                  prefix just before the element's segment start; the first element of a
+//                  segment takes the input value itself), segmented scan of the 32 row tails
+//                  with shuffles, add the carry to each row's first segment
+//                  (UpdateFirstSegment), stage the 32 x 32 results in shared memory and
+//                  write them with one TMA store.  Pieces without any flag skip the revert.
+#pragma once
+#include "common.cuh"
+#include "seg_scan.cuh"
+#include "seg_sum.cuh"
+
+namespace mmv {
+
+constexpr int SC2_EPI_WARPS = 8;
+constexpr int SC2_PRODUCER_WARP = 8;
+constexpr int SC2_MMA_WARP = 9;
+constexpr int SC2_THREADS = 320;
+
+template <typename P>
+struct Scan2Cfg {
+    static constexpr int kN = P::kIsFloat ? 2 * ROW : ROW;               // accumulator columns per product
+    static constexpr int kTmemCols = 2 * PIECES_PER_SPAN * kN;           // two tile buffers: 512 / 256
+    static constexpr int kStages = P::kIsFloat ? 3 : 4;
+    static constexpr int kBBytes = kN * P::kRowBytes;                    // constant operand
+    static constexpr int kBSlot = 4096;
+    static constexpr int kXBytes = PIECES_PER_SPAN * P::kSlabBytes;
+    static constexpr int kStageBytes = kXBytes + FLAG_TILE_BYTES;
+    static constexpr int kStageOffset = kBSlot;
+    static constexpr int kOutOffset = kStageOffset + kStages * kStageBytes;
+    static constexpr int kOutBufBytes = PIECE * 4;                       // 32 rows x 128 B
+    static constexpr int kOutBytes = SC2_EPI_WARPS * 2 * kOutBufBytes;   // double-buffered per warp
+    static constexpr int kBarOffset = kOutOffset + kOutBytes;
+    static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
+    static_assert(kBBytes <= kBSlot, "constant operand fits its slot");
+    static_assert(kStageOffset % 1024 == 0 && kStageBytes % 1024 == 0 && kOutOffset % 1024 == 0, "swizzle atoms");
+};
+
+// 32 flag bytes (8 words) -> bit j set iff byte j is non-zero.
+__device__ __forceinline__ uint32_t flag_bytes_to_mask(const uint4& a, const uint4& b) {
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t m = 0u;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        // bit 7 of every byte := byte != 0, then gather the four bits
+        const uint32_t t = (((w[k] & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w[k]) & 0x80808080u;
+        m |= ((t * 0x00204081u) >> 28) << (4 * k);
+    }
+    return m;
+}
+
+template <typename P>
+__global__ void __launch_bounds__(SC2_THREADS, 1)
+seg_scan2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_out,
+                 const ScanParams prm) {
+    using Acc = typename P::Acc;
+    using Cfg = Scan2Cfg<P>;
+    constexpr int S = Cfg::kStages;
+    constexpr int N = Cfg::kN;
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* sB = smem;
+    uint8_t* sStage = smem + Cfg::kStageOffset;
+    uint64_t* bar_full = reinterpret_cast<uint64_t*>(smem + Cfg::kBarOffset);
+    uint64_t* bar_empty = bar_full + S;
+    uint64_t* bar_acc_full = bar_empty + S;
+    uint64_t* bar_acc_empty = bar_acc_full + 2;
+    uint64_t* bar_ready = bar_acc_empty + 2;      // MMA warp -> warpgroup g: "your next tile has landed"
+    int* tile_slot = reinterpret_cast<int*>(bar_ready + 2);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_slot + S);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;
+    const uint32_t lane = lane_id();
+    const uint64_t budget = prm.budget_ns;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < S; ++i) {
+            mbar_init(&bar_full[i], 1);
+            mbar_init(&bar_empty[i], 4);      // the four epilogue warps, once their flag bytes are read
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&bar_acc_full[i], 1);
+            mbar_init(&bar_acc_empty[i], 4);
+            mbar_init(&bar_ready[i], 1);
+        }
+        *abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (warp == SC2_MMA_WARP) {
+        tmem_alloc(tmem_slot, Cfg::kTmemCols);
+        tmem_relinquish();
+    }
+    if (warp == SC2_PRODUCER_WARP && lane == 0) {
+        tma_prefetch_desc(&tmap_x);
+        tma_prefetch_desc(&tmap_out);
+    }
+    {
+        // constant B, K-major: row nn = output column, element k = input position.
+        // nn < 32: 1 iff k <= nn (U_32);  nn >= 32 (fp16 only): 1 iff k == nn - 32 (identity).
+        constexpr int kVecPerRow = P::kRowBytes / 16;
+        constexpr int kElemPerVec = 16 / P::kElemBytes;
+        for (int v = threadIdx.x; v < N * kVecPerRow; v += SC2_THREADS) {
+            const int nn = v / kVecPerRow, cv = v % kVecPerRow;
+            uint32_t words[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int e = 0; e < kElemPerVec; ++e) {
+                const int k = cv * kElemPerVec + e;
+                const bool one = (nn < ROW) ? (k <= nn) : (k == nn - ROW);
+                if (one) {
+                    if constexpr (P::kElemBytes == 2) words[e >> 1] |= static_cast<uint32_t>(P::kOneBits) << ((e & 1) * 16);
+                    else words[e >> 2] |= 1u << ((e & 3) * 8);
+                }
+            }
+            *reinterpret_cast<uint4*>(sB + swz_offset<P::kRowBytes>(nn, cv * 16)) =
+                make_uint4(words[0], words[1], words[2], words[3]);
+        }
+    }
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == SC2_PRODUCER_WARP) {
+        // =========================== producer ===========================
+        int it = 0, sentinels = 0;
+        bool ok = true;
+        while (ok) {
+            const int stage = it % S;
+            if (!wait_bar(&bar_empty[stage], ((it / S) & 1) ^ 1, abort_flag, budget)) { ok = false; break; }
+            int tile = 0;
+            if (lane == 0) tile = static_cast<int>(atomicAdd(&prm.hdr->tile_counter, 1u));
+            tile = __shfl_sync(0xffffffffu, tile, 0);
+            if (tile >= prm.num_tiles) tile = -1;
+            if (lane == 0) tile_slot[stage] = tile;
+            if (tile < 0) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar_full[stage]);
+                ++it;
+                if (++sentinels == 2) break;
+                continue;
+            }
+            uint8_t* xs = sStage + stage * Cfg::kStageBytes;
+            uint8_t* fs = xs + Cfg::kXBytes;
+            const long long tbase = static_cast<long long>(tile) * TILE;
+            if (tbase + TILE <= prm.n) {
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(&bar_full[stage], Cfg::kStageBytes);
+#pragma unroll
+                    for (int i = 0; i < PIECES_PER_SPAN; ++i)
+                        tma_load_4d(xs + i * P::kSlabBytes, &tmap_x, &bar_full[stage], 0, 0, i, tile * SPANS_PER_TILE);
+                    tma_load_1d(fs, prm.flags + tbase, FLAG_TILE_BYTES, &bar_full[stage]);
+                }
+            } else {
+                // ragged last tile: plain loads, zero fill past n (MATMUL zero-pads its operand)
+                const long long cnt = prm.n - tbase;
+                for (int v = lane; v < TILE / 16; v += 32) {
+                    const int e0 = v * 16;
+                    uint4 fv = make_uint4(0u, 0u, 0u, 0u);
+                    if (e0 + 16 <= cnt) {
+                        fv = *reinterpret_cast<const uint4*>(prm.flags + tbase + e0);
+                    } else if (e0 < cnt) {
+                        __align__(16) uint8_t tmp[16];
+                        for (int e = 0; e < 16; ++e) tmp[e] = (e0 + e < cnt) ? prm.flags[tbase + e0 + e] : uint8_t(0);
+                        fv = *reinterpret_cast<const uint4*>(tmp);
+                    }
+                    *reinterpret_cast<uint4*>(fs + e0) = fv;
+                }
+                constexpr int kElemPerVec = 16 / P::kElemBytes;
+                const uint8_t* xt = static_cast<const uint8_t*>(prm.x) + tbase * P::kElemBytes;
+                for (int v = lane; v < TILE / kElemPerVec; v += 32) {
+                    const int e0 = v * kElemPerVec;
+                    uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+                    if (e0 + kElemPerVec <= cnt) {
+                        xv = *reinterpret_cast<const uint4*>(xt + static_cast<size_t>(e0) * P::kElemBytes);
+                    } else if (e0 < cnt) {
+                        __align__(16) uint8_t tmp[16];
+                        for (int b = 0; b < 16; ++b)
+                            tmp[b] = (e0 + b / P::kElemBytes < cnt) ? xt[static_cast<size_t>(e0) * P::kElemBytes + b] : uint8_t(0);
+                        xv = *reinterpret_cast<const uint4*>(tmp);
+                    }
+                    const int w = e0 / SPAN, i = (e0 % SPAN) / PIECE, l = (e0 % PIECE) / ROW, j0 = e0 % ROW;
+                    *reinterpret_cast<uint4*>(xs + i * P::kSlabBytes +
+                                              swz_offset<P::kRowBytes>(w * PIECE_ROWS + l, j0 * P::kElemBytes)) = xv;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar_full[stage]);
+            }
+            ++it;
+        }
+        if (!ok) {
+            *abort_flag = 1;
+            if (lane == 0) report_error(prm.hdr, 5u);
+        }
+        for (int k = (it > S ? it - S : 0); k < it; ++k) mbar_wait(&bar_full[k % S], (k / S) & 1, 2000000ull);
+    } else if (warp == SC2_MMA_WARP) {
+        // =========================== MMA issuer ===========================
+        constexpr uint32_t idesc = P::kIsFloat ? (make_idesc_f16_f32(128, N) | P::kFmtBits) : make_idesc_s8_s32(128, N);
+        int sentinels = 0;
+        for (int it = 0;; ++it) {
+            const int stage = it % S;
+            if (!wait_bar(&bar_full[stage], (it / S) & 1, abort_flag, budget)) {
+                *abort_flag = 1;
+                if (lane == 0) report_error(prm.hdr, 5u);
+                break;
+            }
+            const int tile = tile_slot[stage];
+            const int acc = it & 1;
+            // the warpgroup that owns this iteration has finished its previous tile (so it has also
+            // consumed the previous phase of bar_ready): hand it the new one
+            if (!wait_bar(&bar_acc_empty[acc], ((it >> 1) & 1) ^ 1, abort_flag, budget)) {
+                *abort_flag = 1;
+                if (lane == 0) report_error(prm.hdr, 5u);
+                break;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_ready[acc]);
+            if (tile < 0) {
+                if (++sentinels == 2) break;
+                continue;
+            }
+            tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t xs = smem_u32(sStage + stage * Cfg::kStageBytes);
+                const uint32_t bs = smem_u32(sB);
+#pragma unroll
+                for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                    const uint32_t d = tmem_base + acc * (PIECES_PER_SPAN * N) + i * N;
+#pragma unroll
+                    for (int ks = 0; ks < P::kMmaPerSlab; ++ks) {
+                        const uint64_t da = make_desc(xs + i * P::kSlabBytes + ks * P::kKStepBytes, P::kSbo, P::kLayoutType);
+                        const uint64_t db = make_desc(bs + ks * P::kKStepBytes, P::kSbo, P::kLayoutType);
+                        if constexpr (P::kIsFloat) mma_f16_ss(d, da, db, idesc, ks != 0);
+                        else mma_i8_ss(d, da, db, idesc, ks != 0);
+                    }
+                }
+                tc_commit(&bar_acc_full[acc]);
+            }
+            __syncwarp();
+        }
+    } else {
+        // =========================== epilogue ===========================
+        const int g = warp >> 2;
+        const int w = warp & 3;
+        Acc* outp = static_cast<Acc*>(prm.out);
+        uint8_t* stg = smem + Cfg::kOutOffset + warp * 2 * Cfg::kOutBufBytes;
+        const long long nrows_full = prm.n / ROW;
+        int obuf = 0;
+        for (int it = g;; it += 2) {
+            const int stage = it % S;
+            // every phase of bar_ready[g] is seen by this warpgroup, so parity waits cannot alias
+            // (bar_full is shared with the other warpgroup's iterations when S is odd)
+            if (!wait_bar(&bar_ready[g], (it >> 1) & 1, abort_flag, budget)) {
+                *abort_flag = 1;
+                if (lane == 0) report_error(prm.hdr, 5u);
+                break;
+            }
+            const int tile = tile_slot[stage];
+            if (tile < 0) break;
+            const long long s = static_cast<long long>(tile) * SPANS_PER_TILE + w;
+
+            // ---- flag bytes -> one start mask per row (registers), then the stage is free ----
+            uint32_t fm[PIECES_PER_SPAN];
+            {
+                const uint8_t* fs = sStage + stage * Cfg::kStageBytes + Cfg::kXBytes + w * SPAN + lane * ROW;
+#pragma unroll
+                for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                    const uint4 a = *reinterpret_cast<const uint4*>(fs + i * PIECE);
+                    const uint4 b = *reinterpret_cast<const uint4*>(fs + i * PIECE + 16);
+                    const uint32_t any = a.x | a.y | a.z | a.w | b.x | b.y | b.z | b.w;
+                    fm[i] = any ? flag_bytes_to_mask(a, b) : 0u;
+                }
+            }
+            if (!wait_bar(&bar_acc_full[g], (it >> 1) & 1, abort_flag, budget)) {
+                *abort_flag = 1;
+                if (lane == 0) report_error(prm.hdr, 5u);
+                break;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_empty[stage]);
+            tc_fence_after_sync();
+
+            const uint32_t taddr = tmem_base + g * (PIECES_PER_SPAN * N) + ((static_cast<uint32_t>(w) * 32u) << 16);
+
+            // ---- pre-pass: row totals, span aggregate, publish, look back ----
+            Acc tot[PIECES_PER_SPAN];
+            uint32_t pm[PIECES_PER_SPAN];
+#pragma unroll
+            for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * N + (ROW - 1)));
+            tmem_ld_wait();
+            uint32_t anyp = 0u;
+#pragma unroll
+            for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                pm[i] = __ballot_sync(0xffffffffu, fm[i] != 0u);
+                anyp |= pm[i];
+            }
+            const bool flagged = anyp != 0u;
+            Acc tail_span;
+            if (!flagged) {
+                tail_span = warp_sum<P>(P::add(P::add(tot[0], tot[1]), P::add(tot[2], tot[3])));
+            } else {
+                int istar = 0;
+#pragma unroll
+                for (int i = 0; i < PIECES_PER_SPAN; ++i)
+                    if (pm[i]) istar = i;
+                uint32_t pms = pm[0], fms = fm[0];
+                Acc tots = tot[0];
+#pragma unroll
+                for (int i = 1; i < PIECES_PER_SPAN; ++i)
+                    if (istar == i) { pms = pm[i]; fms = fm[i]; tots = tot[i]; }
+                const int lstar = 31 - __clz(pms);
+                const uint32_t fmstar = __shfl_sync(0xffffffffu, fms, lstar);
+                const int pl = 31 - __clz(fmstar);            // last flag of the last flagged row
+                Acc after = Acc(0);                            // totals of the rows behind it
+#pragma unroll
+                for (int i = 0; i < PIECES_PER_SPAN; ++i)
+                    if (i > istar) after = P::add(after, tot[i]);
+                if (static_cast<int>(lane) > lstar) after = P::add(after, tots);
+                after = warp_sum<P>(after);
+                Acc before = Acc(0);
+                if (pl > 0) {
+                    before = P::from_bits(tmem_ld_32x1(taddr + istar * N + (pl - 1)));
+                    tmem_ld_wait();
+                }
+                Acc row_tail = P::sub(tots, before);
+                if constexpr (P::kIsFloat) {
+                    if (pl == ROW - 1) {          // the tail is a segment's first element: the input value itself
+                        row_tail = P::from_bits(tmem_ld_32x1(taddr + istar * N + ROW + (ROW - 1)));
+                        tmem_ld_wait();
+                    }
+                }
+                tail_span = P::add(__shfl_sync(0xffffffffu, row_tail, lstar), after);
+            }
+            Acc run = Acc(0);
+            const bool skip_publish = (s == prm.debug_skip_span);
+            if (s == 0) {
+                if (lane == 0 && !skip_publish) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(tail_span)));
+            } else {
+                if (lane == 0 && !skip_publish)
+                    st_relaxed_gpu_u64(prm.status + s, pack_status(flagged ? ST_PREFIX : ST_AGG, P::to_bits(tail_span)));
+                if (!lookback<P>(prm.status, s, run, abort_flag, budget)) {
+                    *abort_flag = 1;
+                    if (lane == 0) {
+                        report_error(prm.hdr, 5u);
+                        st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
+                    }
+                    break;
+                }
+                if (!flagged && lane == 0 && !skip_publish)
+                    st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(run, tail_span))));
+            }
+
+            // ---- main pass ----
+            const long long row0 = s * (SPAN / ROW);
+#pragma unroll 1
+            for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                uint32_t r[32];
+                tmem_ld_32x32(taddr + i * N, r);
+                uint32_t fmi = fm[0];
+                uint32_t pmi = pm[0];
+                Acc toti = tot[0];
+#pragma unroll
+                for (int k = 1; k < PIECES_PER_SPAN; ++k)
+                    if (i == k) { fmi = fm[k]; pmi = pm[k]; toti = tot[k]; }
+                tmem_ld_wait();
+                if (pmi == 0u) {
+                    // no flag in the piece: plain prefix of the row totals, one add per element
+                    Acc inc = toti;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const Acc t = __shfl_up_sync(0xffffffffu, inc, o);
+                        if (static_cast<int>(lane) >= o) inc = P::add(t, inc);
+                    }
+                    const Acc carry_row = P::add(run, P::sub(inc, toti));
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = P::to_bits(P::add(carry_row, P::from_bits(r[j])));
+                    run = P::add(run, __shfl_sync(0xffffffffu, inc, 31));
+                } else {
+                    // revert the speculation inside each row (Lemma A.1)
+                    if constexpr (P::kIsFloat) {
+                        uint32_t raw[32], z[32];
+                        tmem_ld_32x32(taddr + i * N + ROW, raw);
+                        tmem_ld_wait();
+                        Acc base = Acc(0);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const bool pj = (fmi >> j) & 1u;
+                            if (j > 0) base = pj ? P::from_bits(r[j - 1]) : base;
+                            // the first element of a segment is the input value itself, exactly
+                            z[j] = pj ? raw[j] : P::to_bits(P::sub(P::from_bits(r[j]), base));
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = z[j];
+                    } else {
+                        Acc base = Acc(0);
+                        uint32_t prev = 0u;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const bool pj = (fmi >> j) & 1u;
+                            if (j > 0) base = pj ? prev : base;
+                            prev = r[j];
+                            r[j] = P::sub(r[j], base);
+                        }
+                    }
+                    // segmented scan of the row tails across the 32 rows
+                    const bool rowflag = fmi != 0u;
+                    Acc val = P::from_bits(r[31]);
+                    if (lane == 0 && !rowflag) val = P::add(run, val);
+                    uint32_t flg = rowflag ? 1u : 0u;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const Acc tv = __shfl_up_sync(0xffffffffu, val, o);
+                        const uint32_t tf = __shfl_up_sync(0xffffffffu, flg, o);
+                        if (static_cast<int>(lane) >= o) {
+                            if (!flg) val = P::add(tv, val);
+                            flg |= tf;
+                        }
+                    }
+                    Acc carry_row = __shfl_up_sync(0xffffffffu, val, 1);
+                    if (lane == 0) carry_row = run;
+                    run = __shfl_sync(0xffffffffu, val, 31);
+                    const int f0 = rowflag ? (__ffs(fmi) - 1) : 32;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < f0) r[j] = P::to_bits(P::add(carry_row, P::from_bits(r[j])));
+                }
+
+                // ---- stage the 32 x 32 block and store it ----
+                uint8_t* ob = stg + obuf * Cfg::kOutBufBytes;
+                if (lane == 0) tma_store_wait_read<1>();      // the buffer used two stores ago is free again
+                __syncwarp();
+#pragma unroll
+                for (int c4 = 0; c4 < 8; ++c4)
+                    *reinterpret_cast<uint4*>(ob + lane * 128 + ((c4 ^ (lane & 7)) << 4)) =
+                        make_uint4(r[4 * c4], r[4 * c4 + 1], r[4 * c4 + 2], r[4 * c4 + 3]);
+                fence_proxy_async_smem();
+                __syncwarp();
+                const long long prow = row0 + i * PIECE_ROWS;
+                if (lane == 0 && prow < nrows_full) {
+                    tma_store_2d(&tmap_out, ob, 0, static_cast<int>(prow));
+                    tma_store_commit();
+                }
+                // the one row that straddles n (n not a multiple of 32) is written with plain stores
+                if (prow + lane == nrows_full) {
+                    const int cnt = static_cast<int>(prm.n - nrows_full * ROW);
+                    for (int j = 0; j < cnt; ++j) {
+                        uint32_t v = r[0];
+#pragma unroll
+                        for (int k = 1; k < 32; ++k)
+                            if (j == k) v = r[k];
+                        reinterpret_cast<uint32_t*>(outp)[nrows_full * ROW + j] = v;
+                    }
+                }
+                obuf ^= 1;
+            }
+
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_acc_empty[g]);
+        }
+        if (lane == 0) tma_store_wait_all<0>();
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == SC2_MMA_WARP) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, Cfg::kTmemCols);
+    }
+}
+
+}  // namespace mmv
