@@ -27,7 +27,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
     tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
     cmd = [NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "--use_fast_math" if False else "-DNDEBUG",
-           "-o", str(tmp)] + [str(s) for s in SOURCES]
+           "-o", str(tmp)] + os.environ.get("MMV_NVCC_FLAGS", "").split() + [str(s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

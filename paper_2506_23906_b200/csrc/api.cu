@@ -12,8 +12,6 @@
 #include "common.cuh"
 #include "seg_scan.cuh"
 #include "seg_sum.cuh"
-#include "seg_scan2.cuh"
-#include <cstdlib>
 
 namespace mmv {
 namespace {
@@ -65,8 +63,6 @@ DeviceInfo* device_info() {
         bool ok = true;
         ok &= set_smem(seg_scan_kernel<F16Path>, ScanCfg<F16Path>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<I8Path>, ScanCfg<I8Path>::kSmemBytes);
-        ok &= set_smem(seg_scan2_kernel<F16Path>, Scan2Cfg<F16Path>::kSmemBytes);
-        ok &= set_smem(seg_scan2_kernel<I8Path>, Scan2Cfg<I8Path>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<F16Path>, SumCfg<F16Path>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<I8Path>, SumCfg<I8Path>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<BF16Path>, SumCfg<BF16Path>::kSmemBytes);
@@ -78,43 +74,21 @@ DeviceInfo* device_info() {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// The value vector as a matrix of CHUNK-element rows (full rows only); box = NCOL rows.
-bool encode_rows_map(CUtensorMap* map, const void* x, long long n, bool is_f16) {
-    EncodeTiledFn enc = get_encode();
-    if (!enc) return false;
-    const cuuint64_t rows = static_cast<cuuint64_t>(n / CHUNK);
-    if (rows == 0) {
-        std::memset(map, 0, sizeof(*map));
-        return true;               // never used: every tile takes the plain-load path
-    }
-    const cuuint32_t esz = is_f16 ? 2 : 1;
-    cuuint64_t dims[2] = {CHUNK, rows};
-    cuuint64_t strides[1] = {static_cast<cuuint64_t>(CHUNK) * esz};
-    cuuint32_t box[2] = {CHUNK, NCOL};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = enc(map, is_f16 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2,
-                     const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     is_f16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B,
-                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
-
 // The value vector as [spans][4 pieces][32 rows][32 elements] (full spans only); one box =
 // piece i of four consecutive spans = the 128 x 32 A operand of one tensor-core product.
-bool encode_span_map(CUtensorMap* map, const void* x, long long n, int elem_bytes, bool bf16) {
+bool encode_span_map(CUtensorMap* map, const void* x, long long n, int elem_bytes, int pieces_per_unit) {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
-    const cuuint64_t spans = static_cast<cuuint64_t>(n / SPAN);
+    const cuuint64_t spans = static_cast<cuuint64_t>(n / (static_cast<long long>(pieces_per_unit) * PIECE));
     if (spans == 0) {
         std::memset(map, 0, sizeof(*map));
         return true;
     }
     const cuuint64_t rb = static_cast<cuuint64_t>(ROW) * elem_bytes;
-    cuuint64_t dims[4] = {ROW, PIECE_ROWS, PIECES_PER_SPAN, spans};
-    cuuint64_t strides[3] = {rb, rb * PIECE_ROWS, rb * PIECE_ROWS * PIECES_PER_SPAN};
+    cuuint64_t dims[4] = {ROW, PIECE_ROWS, static_cast<cuuint64_t>(pieces_per_unit), spans};
+    cuuint64_t strides[3] = {rb, rb * PIECE_ROWS, rb * PIECE_ROWS * pieces_per_unit};
     cuuint32_t box[4] = {ROW, PIECE_ROWS, 1, SPANS_PER_TILE};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    (void)bf16;
     CUresult r = enc(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4,
                      const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                      elem_bytes == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B,
@@ -151,13 +125,15 @@ struct WorkspacePlan {
 };
 
 long long num_tiles_of(long long n) { return (n + TILE - 1) / TILE; }
+long long num_scan_tiles_of(long long n) { return (n + SCAN_TILE - 1) / SCAN_TILE; }
 
 WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     WorkspacePlan p{};
     p.n_eff = (op == MMV_OP_SPMV_CSR) ? 2 * n : n;
     const long long tiles = num_tiles_of(p.n_eff);
+    const long long units = (op == MMV_OP_SEG_SCAN) ? num_scan_tiles_of(n) * SPANS_PER_TILE : tiles * SPANS_PER_TILE;
     p.status_off = sizeof(WorkspaceHeader);
-    p.status_bytes = round_up(static_cast<size_t>(tiles) * SPANS_PER_TILE * sizeof(uint64_t), 256);
+    p.status_bytes = round_up(static_cast<size_t>(units) * sizeof(uint64_t), 256);
     p.flags_off = p.status_off + p.status_bytes;
     p.flags_bytes = (op == MMV_OP_SEG_SCAN && sf == MMV_SEG_OFFSETS_I32) ? round_up(static_cast<size_t>(n), 256) : 0;
     p.tileq_off = p.flags_off + p.flags_bytes;
@@ -220,7 +196,7 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
         ++g_launches;
     }
     CUtensorMap tmap;
-    if (!encode_span_map(&tmap, values, n_eff, P::kElemBytes, false)) return MMV_ERR_CUDA;
+    if (!encode_span_map(&tmap, values, n_eff, P::kElemBytes, PIECES_PER_SPAN)) return MMV_ERR_CUDA;
     SumParams prm;
     prm.off = off;
     prm.nseg = nseg;
@@ -303,37 +279,25 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
     }
 
     const bool f16 = dt == MMV_F16_TO_F32;
-    static const bool use_v1 = std::getenv("MMV_SCAN_V1") != nullptr;
     CUtensorMap tmap, tmap_out;
-    if (use_v1) {
-        if (!encode_rows_map(&tmap, x, n, f16)) return MMV_ERR_CUDA;
-    } else {
-        if (!encode_span_map(&tmap, x, n, f16 ? 2 : 1, false)) return MMV_ERR_CUDA;
-        if (!encode_out_map(&tmap_out, out, n)) return MMV_ERR_CUDA;
-    }
+    if (!encode_span_map(&tmap, x, n, f16 ? 2 : 1, SCAN_UP)) return MMV_ERR_CUDA;
+    if (!encode_out_map(&tmap_out, out, n)) return MMV_ERR_CUDA;
 
     ScanParams prm;
     prm.x = x;
     prm.flags = flags;
     prm.out = out;
     prm.n = n;
-    prm.num_tiles = static_cast<int>(num_tiles_of(n));
+    prm.num_tiles = static_cast<int>(num_scan_tiles_of(n));
     prm.hdr = hdr;
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();
     prm.debug_skip_span = g_debug_skip_span.load();
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
-    if (use_v1) {
-        if (f16)
-            seg_scan_kernel<F16Path><<<grid, SCAN_THREADS, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, prm);
-        else
-            seg_scan_kernel<I8Path><<<grid, SCAN_THREADS, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, prm);
-    } else {
-        if (f16)
-            seg_scan2_kernel<F16Path><<<grid, SC2_THREADS, Scan2Cfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
-        else
-            seg_scan2_kernel<I8Path><<<grid, SC2_THREADS, Scan2Cfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
-    }
+    if (f16)
+        seg_scan_kernel<F16Path><<<grid, SCAN_THREADS, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+    else
+        seg_scan_kernel<I8Path><<<grid, SCAN_THREADS, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
@@ -425,6 +389,16 @@ const char* mmv_status_string(mmv_status s) {
 }
 
 int64_t mmv_kernel_launch_count(void) { return g_launches.load(); }
+
+#ifdef MMV_PHASE_TIMERS
+// Development aid: reads and clears the phase-cycle counters of the scan kernel.
+void mmv_debug_phase_cycles(unsigned long long* host16) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(host16, g_phase_cycles, 16 * sizeof(unsigned long long));
+    unsigned long long z[16] = {0};
+    cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z));
+}
+#endif
 
 void mmv_debug_configure(int64_t wait_budget_ns, int64_t skip_publish_span) {
     g_budget_ns.store(wait_budget_ns > 0 ? static_cast<unsigned long long>(wait_budget_ns) : WAIT_BUDGET_NS);

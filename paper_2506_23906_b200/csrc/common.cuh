@@ -6,17 +6,19 @@
 
 namespace mmv {
 
-// Geometry.  The value vector is viewed as rows of CHUNK consecutive elements
-// (the paper's ceil(n/s) x s matrix view of MATMUL(x, U_s), with s = CHUNK).  A
-// warp owns a SPAN of NCOL consecutive rows: its 32 lanes are the 32 positions
-// of a row and the rows are the columns of its TMEM accumulator.  A TILE is the
-// four spans handled by the four warps of one epilogue warpgroup and is the
-// unit of one tensor-core product.
-constexpr int CHUNK = 32;
-constexpr int NCOL = 128;
-constexpr int SPAN = CHUNK * NCOL;       // 4096 elements
+// Geometry.  The value vector is viewed as rows of ROW consecutive elements (the paper's
+// ceil(n/s) x s matrix view of MATMUL(x, U_s), with s = ROW).  A warp owns a SPAN of 128
+// consecutive rows in four PIECES of 32 rows (one row per lane); a TILE is the four spans
+// handled by the four warps of one epilogue warpgroup.  Tensor-core product i of a tile
+// multiplies the 128 x 32 matrix made of piece i of the four spans.
+constexpr int ROW = 32;
+constexpr int PIECE_ROWS = 32;
+constexpr int PIECE = ROW * PIECE_ROWS;        // 1024 elements
+constexpr int PIECES_PER_SPAN = 4;
+constexpr int SPAN = PIECES_PER_SPAN * PIECE;  // 4096 elements
 constexpr int SPANS_PER_TILE = 4;
-constexpr int TILE = SPANS_PER_TILE * SPAN;   // 16384 elements
+constexpr int TILE = SPANS_PER_TILE * SPAN;    // 16384 elements
+constexpr int OPERAND_ROWS = SPANS_PER_TILE * PIECE_ROWS;   // 128 = M of one product
 constexpr int FLAG_TILE_BYTES = TILE;
 
 // Every device-side wait (mbarrier, look-back) gives up after this long.
@@ -41,8 +43,8 @@ struct F16Path {
     using Acc = float;
     static constexpr int kElemBytes = 2;
     static constexpr bool kIsFloat = true;
-    static constexpr int kRowBytes = CHUNK * 2;            // 64-byte rows -> 64-byte swizzle
-    static constexpr int kSlabBytes = NCOL * kRowBytes;    // one K-slab of an operand: 8 KB
+    static constexpr int kRowBytes = ROW * 2;            // 64-byte rows -> 64-byte swizzle
+    static constexpr int kSlabBytes = OPERAND_ROWS * kRowBytes;    // one K-slab of an operand: 8 KB
     static constexpr int kMmaPerSlab = 2;                  // K = 16 per instruction
     static constexpr int kKStepBytes = 32;
     static constexpr uint32_t kLayoutType = 4;             // SWIZZLE_64B
@@ -58,8 +60,8 @@ struct I8Path {
     using Acc = uint32_t;                                  // wrap-around arithmetic on unsigned
     static constexpr int kElemBytes = 1;
     static constexpr bool kIsFloat = false;
-    static constexpr int kRowBytes = CHUNK;                // 32-byte rows -> 32-byte swizzle
-    static constexpr int kSlabBytes = NCOL * kRowBytes;    // 4 KB
+    static constexpr int kRowBytes = ROW;                  // 32-byte rows -> 32-byte swizzle
+    static constexpr int kSlabBytes = OPERAND_ROWS * kRowBytes;    // 4 KB
     static constexpr int kMmaPerSlab = 1;                  // K = 32 per instruction
     static constexpr int kKStepBytes = 32;
     static constexpr uint32_t kLayoutType = 6;             // SWIZZLE_32B
@@ -97,6 +99,110 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t sbo_bytes,
 
 __device__ __forceinline__ void report_error(WorkspaceHeader* hdr, unsigned int code) {
     atomicCAS(&hdr->error, 0u, code);
+}
+
+// Bounded mbarrier wait that also gives up when another role of the CTA has aborted.
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                         uint64_t budget_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    uint32_t polls = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++polls & 31u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > budget_ns) return false;
+        }
+    }
+    return true;
+}
+
+template <typename P>
+__device__ __forceinline__ typename P::Acc warp_sum(typename P::Acc v) {
+    if constexpr (P::kIsFloat) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        return v;
+    } else {
+        return __reduce_add_sync(0xffffffffu, v);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Decoupled look-back over per-span status words.
+//
+// Span s publishes either its aggregate (ST_AGG: sum of all its elements, it holds no segment
+// start) or an inclusive prefix (ST_PREFIX: sum of the segment that is open at its end).  The
+// carry into span s is the sum of the aggregates of s-1, s-2, ... down to and including the
+// first span that published a prefix.  A window is LB_WINDOW consecutive predecessors, LB_WORDS
+// per lane, nearest first: lane l holds positions LB_WORDS*l .. LB_WORDS*l + LB_WORDS-1.
+// ---------------------------------------------------------------------------
+constexpr int LB_WORDS = 1;
+constexpr int LB_WINDOW = 32 * LB_WORDS;
+
+struct LookbackWindow {
+    uint64_t w[LB_WORDS];
+};
+
+// Issues the loads of the window whose nearest predecessor is `idx` (no wait on the data).
+__device__ __forceinline__ void lookback_load(const uint64_t* status, long long idx, LookbackWindow& win) {
+    const long long first = idx - static_cast<long long>(LB_WORDS) * lane_id();
+#pragma unroll
+    for (int q = 0; q < LB_WORDS; ++q) {
+        const long long my = first - q;
+        win.w[q] = (my >= 0) ? ld_relaxed_gpu_u64(status + my) : pack_status(ST_PREFIX, 0u);   // nothing before span 0
+    }
+}
+
+// Returns the carry into span s.  `win` may hold a window loaded earlier with lookback_load
+// (preloaded = true) so that the first round trip overlaps the caller's work.  Bounded: returns
+// false on time-out, when another role of the CTA aborted, or when a predecessor aborted.
+template <typename P>
+__device__ __forceinline__ bool lookback(const uint64_t* status, long long s, typename P::Acc& carry,
+                                         volatile int* abort_flag, uint64_t budget_ns, LookbackWindow& win,
+                                         bool preloaded) {
+    using Acc = typename P::Acc;
+    const uint32_t lane = lane_id();
+    Acc acc = Acc(0);
+    long long idx = s - 1;
+    uint64_t t0 = global_timer_ns();
+    uint32_t polls = 0;
+    if (!preloaded) lookback_load(status, idx, win);
+    while (true) {
+        uint32_t tmask = 0u, rmask = 0u, xmask = 0u;
+#pragma unroll
+        for (int q = 0; q < LB_WORDS; ++q) {
+            const uint32_t st = static_cast<uint32_t>(win.w[q] >> 32);
+            rmask |= (st != ST_NONE) ? (1u << q) : 0u;
+            tmask |= (st == ST_PREFIX || st == ST_ABORT) ? (1u << q) : 0u;
+            xmask |= (st == ST_ABORT) ? (1u << q) : 0u;
+        }
+        const uint32_t lanes_t = __ballot_sync(0xffffffffu, tmask != 0u);
+        const int L = lanes_t ? (__ffs(lanes_t) - 1) : 32;            // first lane that holds a terminal word
+        const int qt = tmask ? (__ffs(tmask) - 1) : LB_WORDS;         // this lane's first terminal word
+        // words this lane must contribute: all of them before lane L, up to its terminal in lane L
+        const int need = (static_cast<int>(lane) < L) ? LB_WORDS : ((static_cast<int>(lane) == L) ? qt + 1 : 0);
+        const uint32_t need_mask = (1u << need) - 1u;
+        const bool lane_ready = (rmask & need_mask) == need_mask;
+        if (__all_sync(0xffffffffu, lane_ready)) {
+            if (__any_sync(0xffffffffu, (xmask & need_mask) != 0u)) return false;
+            Acc v = Acc(0);
+#pragma unroll
+            for (int q = LB_WORDS - 1; q >= 0; --q)
+                if (q < need) v = P::add(P::from_bits(static_cast<uint32_t>(win.w[q])), v);
+            v = warp_sum<P>(v);
+            acc = P::add(v, acc);
+            if (L < 32) {
+                carry = acc;
+                return true;
+            }
+            idx -= LB_WINDOW;
+            t0 = global_timer_ns();
+        } else if ((++polls & 7u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > budget_ns) return false;
+        }
+        lookback_load(status, idx, win);
+    }
 }
 
 }  // namespace mmv

@@ -1,42 +1,49 @@
-// Single-pass segmented inclusive scan (Problem 2.1, Eq. 1) for sm_100a.
+// Single-pass segmented inclusive scan (Problem 2.1, Eq. 1) for sm_100a, row-major layout.
 //
-// Per tile of TILE = 4 x 128 x 32 elements:
-//   producer warp   TMA: four [128 rows x 32 elements] boxes of x (one per span,
-//                   K-major, hardware swizzle) and the tile's flag bytes.
-//   MMA warp        tcgen05.mma  D[128 x 128] = A . B^T  with B the x boxes and A the
-//                   constant block-diagonal lower-triangular all-ones matrix
-//                   (I_4 (x) L_32): TMEM lane 32w+l, column c holds the inclusive
-//                   prefix at position l of row c of span w -- the speculative
-//                   block scan MATMUL(x, U_s) of Algorithm A.1 (BlockSegScan),
-//                   transposed so that a warp's lanes are consecutive elements.
-//   epilogue warps  (two warpgroups on alternating tiles) per row: ballot of the flag
-//                   bytes -> boundary mask; revert the speculation by subtracting the
-//                   prefix just before the element's segment start (Lemma A.1), one
-//                   shuffle; chain the row tails through the span; publish the span's
-//                   aggregate, look back over earlier spans (decoupled look-back:
-//                   the recursion of Section 4.2 folded into one pass), add the carry
-//                   to the elements before the span's first flag (UpdateFirstSegment of
-//                   Algorithm A.1) and store with 128-byte coalesced warp stores.
+// The value vector is the paper's ceil(n/s) x s matrix with s = ROW = 32.  A warp owns a
+// SPAN of 128 consecutive rows (4096 elements) in four PIECES of 32 rows; a TILE is four
+// spans.  For each tile:
+//   producer warp  one 4-D TMA box per piece index i (the [128 rows x 32] matrix made of
+//                  piece i of the four spans, K-major, hardware swizzle) and one bulk copy
+//                  of the tile's 16 KB of flag bytes, several tiles ahead.
+//   tensor core    tcgen05.mma issued by the leader of the warpgroup that takes the tile:
+//                  A = that matrix, B = the constant [U_32 | I_32] (fp16) or U_32 (int8):
+//                  TMEM lane 32w+l, column j (< 32) = inclusive prefix at position j of row l
+//                  of piece i of span w, the speculative block scan z = MATMUL(x, U_s) of
+//                  Algorithm A.1 (BlockSegScan); columns 32..63 (fp16) return the row itself
+//                  converted exactly to fp32.
+//   epilogue warps (lane = row; two warpgroups on alternating tiles)
+//     pre-pass     flag bytes -> one 32-bit start mask per row; row totals (TMEM column 31);
+//                  from these the span's aggregate (sum of its open tail segment, any flag)
+//                  is formed with a handful of shuffles and published at once.
+//     main pass    per piece: revert the speculation inside each row (Lemma A.1: subtract the
+//                  prefix just before the element's segment start; the first element of a
+//                  segment takes the input value itself), segmented scan of the 32 row tails
+//                  with shuffles, add the row carries (UpdateFirstSegment inside the span),
+//                  stage the 32 x 32 results in shared memory and write them with one TMA
+//                  store.  Pieces without any flag skip the revert.  Pieces that reach back
+//                  to the start of the span (up to and including the first flagged one) are
+//                  parked in TMEM instead.
+//     look-back    decoupled look-back over the earlier spans' status words returns the carry
+//                  (this replaces the recursion of Section 4.2 / Algorithm A.1's Recurse); its
+//                  latency is covered by the main pass.  The parked pieces then receive the
+//                  carry on the elements before the span's first flag and are stored.
 #pragma once
 #include "common.cuh"
 
 namespace mmv {
 
-constexpr int SCAN_EPI_WARPS = 8;
-constexpr int SCAN_PRODUCER_WARP = 8;
-constexpr int SCAN_MMA_WARP = 9;
-constexpr int SCAN_THREADS = 320;
-constexpr int SCAN_TMEM_COLS = 256;          // two 128-column accumulators
-
-template <typename P>
-struct ScanCfg {
-    static constexpr int kStages = P::kIsFloat ? 4 : 6;
-    static constexpr int kABytes = 4 * P::kSlabBytes;
-    static constexpr int kXBytes = 4 * P::kSlabBytes;
-    static constexpr int kStageBytes = kXBytes + FLAG_TILE_BYTES;
-    static constexpr int kBarOffset = kABytes + kStages * kStageBytes;
-    static constexpr int kSmemBytes = kBarOffset + 512 + 1024;   // + barriers/slots + alignment slack
-};
+// Optional phase timers (compile with -DMMV_PHASE_TIMERS): cycles summed over all epilogue warps.
+#ifdef MMV_PHASE_TIMERS
+__device__ unsigned long long g_phase_cycles[16];
+#define MMV_T_DECL long long t_prev = clock64(); unsigned long long t_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#define MMV_T_MARK(k) { const long long t_now = clock64(); t_acc[k] += static_cast<unsigned long long>(t_now - t_prev); t_prev = t_now; }
+#define MMV_T_FLUSH() { if (lane == 0) { for (int k = 0; k < 8; ++k) atomicAdd(&g_phase_cycles[k], t_acc[k]); } }
+#else
+#define MMV_T_DECL
+#define MMV_T_MARK(k)
+#define MMV_T_FLUSH()
+#endif
 
 struct ScanParams {
     const void* x;
@@ -50,109 +57,108 @@ struct ScanParams {
     long long debug_skip_span;   // test hook: this span never publishes (-1 = off)
 };
 
-// Bounded mbarrier wait that also gives up when another role of the CTA has aborted.
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                         uint64_t budget_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
-    uint32_t polls = 0;
-    while (!mbar_try_wait(bar, parity)) {
-        if ((++polls & 31u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > budget_ns) return false;
-        }
-    }
-    return true;
-}
+// Scan geometry: a warp owns a UNIT of SCAN_UP consecutive pieces (the grain of the carry
+// chain: one status word per unit); a scan tile is four units and SCAN_UP tensor-core products.
+// SCAN_GROUPS warpgroups take alternating tiles; each has two TMEM buffers so that the products
+// of its next tile are finished before it gets there.
+constexpr int SCAN_UP = 4;
+constexpr int SCAN_UNIT = SCAN_UP * PIECE;                  // 4096 elements
+constexpr int SCAN_TILE = SPANS_PER_TILE * SCAN_UNIT;       // 16384 elements
+constexpr int SCAN_GROUPS = 2;
+constexpr int SCAN_BUFS = 2 * SCAN_GROUPS;                  // TMEM tile buffers
+constexpr int SCAN_EPI_WARPS = 4 * SCAN_GROUPS;             // 8
+constexpr int SCAN_PRODUCER_WARP = SCAN_EPI_WARPS;
+constexpr int SCAN_MMA_WARP = SCAN_EPI_WARPS + 1;
+constexpr int SCAN_THREADS = (SCAN_EPI_WARPS + 2) * 32;     // 320
 
 template <typename P>
-__device__ __forceinline__ typename P::Acc warp_sum(typename P::Acc v) {
-    if constexpr (P::kIsFloat) {
+struct ScanCfg {
+    // fp16: the product also returns the rows themselves (exact fp32 copies, columns 32..63), so a
+    // tile needs 256 TMEM columns and each warpgroup has one buffer; int8: 128 columns, two buffers.
+    static constexpr int kN = P::kIsFloat ? 2 * ROW : ROW;               // accumulator columns per product
+    static constexpr int kBufsPerGroup = P::kIsFloat ? 1 : 2;
+    static constexpr int kTmemCols = SCAN_GROUPS * kBufsPerGroup * SCAN_UP * kN;   // 512
+    static constexpr int kStages = P::kIsFloat ? 3 : 4;
+    static constexpr int kBBytes = kN * P::kRowBytes;                    // constant operand [U_32 | I_32] / U_32
+    static constexpr int kBSlot = 4096;
+    static constexpr int kXBytes = SCAN_UP * P::kSlabBytes;
+    static constexpr int kFlagBytes = SCAN_TILE;
+    static constexpr int kStageBytes = kXBytes + kFlagBytes;
+    static constexpr int kStageOffset = kBSlot;
+    static constexpr int kOutOffset = kStageOffset + kStages * kStageBytes;
+    static constexpr int kOutBufBytes = PIECE * 4;                       // 32 rows x 128 B
+    static constexpr int kOutBufs = 2;                                   // staging buffers per warp
+    static constexpr int kOutBytes = SCAN_EPI_WARPS * kOutBufs * kOutBufBytes;
+    static constexpr int kBarOffset = kOutOffset + kOutBytes;
+    static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
+    static_assert(kBBytes <= kBSlot, "constant operand fits its slot");
+    static_assert(kStageOffset % 1024 == 0 && kStageBytes % 1024 == 0 && kOutOffset % 1024 == 0, "swizzle atoms");
+};
+
+// 32 flag bytes (8 words) -> bit j set iff byte j is non-zero.
+__device__ __forceinline__ uint32_t flag_bytes_to_mask(const uint4& a, const uint4& b) {
+    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    uint32_t m = 0u;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        return v;
-    } else {
-        return __reduce_add_sync(0xffffffffu, v);
+    for (int k = 0; k < 8; ++k) {
+        // bit 7 of every byte := byte != 0, then gather the four bits
+        const uint32_t t = (((w[k] & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w[k]) & 0x80808080u;
+        m |= ((t * 0x00204081u) >> 28) << (4 * k);
     }
+    return m;
 }
 
-// Decoupled look-back: exclusive carry of span s = running sum of the open segment at the
-// end of span s-1.  Walks predecessor status words, 32 per step, adding aggregates until it
-// meets a span that published an inclusive prefix.  Bounded: returns false on time-out or if
-// a predecessor aborted.
-template <typename P>
-__device__ __forceinline__ bool lookback(const uint64_t* status, long long s, typename P::Acc& carry,
-                                         volatile int* abort_flag, uint64_t budget_ns) {
-    using Acc = typename P::Acc;
-    const uint32_t lane = lane_id();
-    Acc acc = Acc(0);
-    long long idx = s - 1;
-    uint64_t t0 = global_timer_ns();
-    uint32_t polls = 0;
-    while (true) {
-        const long long my = idx - lane;
-        const uint64_t wv = (my >= 0) ? ld_relaxed_gpu_u64(status + my) : pack_status(ST_PREFIX, 0u);
-        const uint32_t st = static_cast<uint32_t>(wv >> 32);
-        const uint32_t rdy = __ballot_sync(0xffffffffu, st != ST_NONE);
-        const uint32_t pm = __ballot_sync(0xffffffffu, st == ST_PREFIX);
-        const uint32_t xm = __ballot_sync(0xffffffffu, st == ST_ABORT);
-        const uint32_t term = pm | xm;
-        uint32_t need = 0xffffffffu;
-        int t = 32;
-        if (term) {
-            t = __ffs(term) - 1;
-            need = (t == 31) ? 0xffffffffu : ((2u << t) - 1u);
-        }
-        if ((rdy & need) == need) {
-            if (term && ((xm >> t) & 1u)) return false;
-            Acc v = ((need >> lane) & 1u) ? P::from_bits(static_cast<uint32_t>(wv)) : Acc(0);
-            v = warp_sum<P>(v);
-            acc = P::add(v, acc);
-            if (term) {
-                carry = acc;
-                return true;
+// Waits until shared-memory stage `stage` holds iteration `it` (the producer writes the iteration
+// number before it arms the barrier) and its bytes have landed.  Checking the iteration number
+// first makes the parity wait unambiguous even for a waiter that does not see every phase.
+__device__ __forceinline__ bool wait_stage(const volatile int* stage_iter, int it, uint64_t* bar, uint32_t parity,
+                                           volatile int* abort_flag, uint64_t budget_ns) {
+    if (*stage_iter != it) {
+        const uint64_t t0 = global_timer_ns();
+        uint32_t polls = 0;
+        while (*stage_iter != it) {
+            if ((++polls & 31u) == 0u) {
+                if (*abort_flag) return false;
+                if (global_timer_ns() - t0 > budget_ns) return false;
             }
-            idx -= 32;
-            t0 = global_timer_ns();
-            continue;
-        }
-        if ((++polls & 7u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > budget_ns) return false;
         }
     }
+    return wait_bar(bar, parity, abort_flag, budget_ns);
 }
 
 template <typename P>
 __global__ void __launch_bounds__(SCAN_THREADS, 1)
-seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const ScanParams prm) {
+seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_out,
+                 const ScanParams prm) {
     using Acc = typename P::Acc;
     using Cfg = ScanCfg<P>;
     constexpr int S = Cfg::kStages;
+    constexpr int N = Cfg::kN;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* sA = smem;
-    uint8_t* sStage = smem + Cfg::kABytes;
+    uint8_t* sB = smem;
+    uint8_t* sStage = smem + Cfg::kStageOffset;
     uint64_t* bar_full = reinterpret_cast<uint64_t*>(smem + Cfg::kBarOffset);
     uint64_t* bar_empty = bar_full + S;
-    uint64_t* bar_acc_full = bar_empty + S;
-    uint64_t* bar_acc_empty = bar_acc_full + 2;
-    int* tile_slot = reinterpret_cast<int*>(bar_acc_empty + 2);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_slot + S);
+    uint64_t* bar_acc_full = bar_empty + S;                // per TMEM buffer: the tile's products are in it
+    uint64_t* bar_acc_empty = bar_acc_full + SCAN_BUFS;    // per TMEM buffer: the four warps are done with it
+    int* tile_slot = reinterpret_cast<int*>(bar_acc_empty + SCAN_BUFS);
+    volatile int* stage_iter = tile_slot + S;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_slot + 2 * S);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5;
     const uint32_t lane = lane_id();
     const uint64_t budget = prm.budget_ns;
 
-    // ---- set-up: barriers, TMEM, the constant operand A = I_4 (x) L_32 ----
     if (threadIdx.x == 0) {
         for (int i = 0; i < S; ++i) {
             mbar_init(&bar_full[i], 1);
-            mbar_init(&bar_empty[i], 4);
+            mbar_init(&bar_empty[i], 4);      // the group's four warps, once their flag bytes are read
+            stage_iter[i] = -1;
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < SCAN_BUFS; ++i) {
             mbar_init(&bar_acc_full[i], 1);
             mbar_init(&bar_acc_empty[i], 4);
         }
@@ -160,31 +166,32 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const ScanParams prm
         mbar_fence_init();
     }
     if (warp == SCAN_MMA_WARP) {
-        tmem_alloc(tmem_slot, SCAN_TMEM_COLS);
+        tmem_alloc(tmem_slot, Cfg::kTmemCols);
         tmem_relinquish();
     }
-    if (warp == SCAN_PRODUCER_WARP && lane == 0) tma_prefetch_desc(&tmap_x);
+    if (warp == SCAN_PRODUCER_WARP && lane == 0) {
+        tma_prefetch_desc(&tmap_x);
+        tma_prefetch_desc(&tmap_out);
+    }
     {
-        // slab w, row m, element k of the row: 1 iff m belongs to block w and k <= m mod 32
+        // constant B, K-major: row nn = output column, element k = input position.
+        // nn < 32: 1 iff k <= nn (U_32);  nn >= 32 (fp16 only): 1 iff k == nn - 32 (identity).
         constexpr int kVecPerRow = P::kRowBytes / 16;
         constexpr int kElemPerVec = 16 / P::kElemBytes;
-        for (int v = threadIdx.x; v < 4 * NCOL * kVecPerRow; v += SCAN_THREADS) {
-            const int w = v / (NCOL * kVecPerRow);
-            const int m = (v / kVecPerRow) % NCOL;
-            const int cv = v % kVecPerRow;
+        for (int v = threadIdx.x; v < N * kVecPerRow; v += SCAN_THREADS) {
+            const int nn = v / kVecPerRow, cv = v % kVecPerRow;
             uint32_t words[4] = {0u, 0u, 0u, 0u};
-            if ((m >> 5) == w) {
 #pragma unroll
-                for (int e = 0; e < kElemPerVec; ++e) {
-                    const int k = cv * kElemPerVec + e;
-                    if (k <= (m & 31)) {
-                        if constexpr (P::kIsFloat) words[e >> 1] |= 0x3C00u << ((e & 1) * 16);   // fp16 1.0
-                        else words[e >> 2] |= 1u << ((e & 3) * 8);
-                    }
+            for (int e = 0; e < kElemPerVec; ++e) {
+                const int k = cv * kElemPerVec + e;
+                const bool one = (nn < ROW) ? (k <= nn) : (k == nn - ROW);
+                if (one) {
+                    if constexpr (P::kElemBytes == 2) words[e >> 1] |= static_cast<uint32_t>(P::kOneBits) << ((e & 1) * 16);
+                    else words[e >> 2] |= 1u << ((e & 3) * 8);
                 }
             }
-            uint4* dst = reinterpret_cast<uint4*>(sA + w * P::kSlabBytes + swz_offset<P::kRowBytes>(m, cv * 16));
-            *dst = make_uint4(words[0], words[1], words[2], words[3]);
+            *reinterpret_cast<uint4*>(sB + swz_offset<P::kRowBytes>(nn, cv * 16)) =
+                make_uint4(words[0], words[1], words[2], words[3]);
         }
     }
     fence_proxy_async_smem();
@@ -200,59 +207,64 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const ScanParams prm
         while (ok) {
             const int stage = it % S;
             if (!wait_bar(&bar_empty[stage], ((it / S) & 1) ^ 1, abort_flag, budget)) { ok = false; break; }
-            int tile = 0;
-            if (lane == 0) tile = static_cast<int>(atomicAdd(&prm.hdr->tile_counter, 1u));
-            tile = __shfl_sync(0xffffffffu, tile, 0);
+            // static round-robin tile assignment: all CTAs are resident (grid <= SM count, one CTA per
+            // SM), so iteration `it` of every CTA runs at about the same time and a tile's predecessors
+            // are always in flight or finished
+            int tile = static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
             if (tile >= prm.num_tiles) tile = -1;
-            if (lane == 0) tile_slot[stage] = tile;
+            if (lane == 0) {
+                tile_slot[stage] = tile;
+                stage_iter[stage] = it;
+            }
             if (tile < 0) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar_full[stage]);
                 ++it;
-                if (++sentinels == 2) break;
+                if (++sentinels == SCAN_GROUPS) break;
                 continue;
             }
             uint8_t* xs = sStage + stage * Cfg::kStageBytes;
             uint8_t* fs = xs + Cfg::kXBytes;
-            const long long tbase = static_cast<long long>(tile) * TILE;
-            if (tbase + TILE <= prm.n) {
+            const long long tbase = static_cast<long long>(tile) * SCAN_TILE;
+            if (tbase + SCAN_TILE <= prm.n) {
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&bar_full[stage], Cfg::kXBytes + FLAG_TILE_BYTES);
+                    mbar_arrive_expect_tx(&bar_full[stage], Cfg::kStageBytes);
 #pragma unroll
-                    for (int w = 0; w < 4; ++w)
-                        tma_load_2d(xs + w * P::kSlabBytes, &tmap_x, &bar_full[stage], 0, tile * (TILE / CHUNK) + w * NCOL);
-                    tma_load_1d(fs, prm.flags + tbase, FLAG_TILE_BYTES, &bar_full[stage]);
+                    for (int i = 0; i < SCAN_UP; ++i)
+                        tma_load_4d(xs + i * P::kSlabBytes, &tmap_x, &bar_full[stage], 0, 0, i, tile * SPANS_PER_TILE);
+                    tma_load_1d(fs, prm.flags + tbase, Cfg::kFlagBytes, &bar_full[stage]);
                 }
             } else {
-                // ragged last tile: plain loads, zero fill past n (the paper zero-pads MATMUL's operand)
+                // ragged last tile: plain loads, zero fill past n (MATMUL zero-pads its operand)
                 const long long cnt = prm.n - tbase;
-                for (int v = lane; v < TILE / 16; v += 32) {
+                for (int v = lane; v < SCAN_TILE / 16; v += 32) {
                     const int e0 = v * 16;
                     uint4 fv = make_uint4(0u, 0u, 0u, 0u);
                     if (e0 + 16 <= cnt) {
                         fv = *reinterpret_cast<const uint4*>(prm.flags + tbase + e0);
                     } else if (e0 < cnt) {
-                        uint8_t tmp[16];
+                        __align__(16) uint8_t tmp[16];
                         for (int e = 0; e < 16; ++e) tmp[e] = (e0 + e < cnt) ? prm.flags[tbase + e0 + e] : uint8_t(0);
                         fv = *reinterpret_cast<const uint4*>(tmp);
                     }
                     *reinterpret_cast<uint4*>(fs + e0) = fv;
                 }
                 constexpr int kElemPerVec = 16 / P::kElemBytes;
-                const uint8_t* xg = static_cast<const uint8_t*>(prm.x) + tbase * P::kElemBytes;
-                for (int v = lane; v < TILE / kElemPerVec; v += 32) {
+                const uint8_t* xt = static_cast<const uint8_t*>(prm.x) + tbase * P::kElemBytes;
+                for (int v = lane; v < SCAN_TILE / kElemPerVec; v += 32) {
                     const int e0 = v * kElemPerVec;
                     uint4 xv = make_uint4(0u, 0u, 0u, 0u);
                     if (e0 + kElemPerVec <= cnt) {
-                        xv = *reinterpret_cast<const uint4*>(xg + static_cast<size_t>(e0) * P::kElemBytes);
+                        xv = *reinterpret_cast<const uint4*>(xt + static_cast<size_t>(e0) * P::kElemBytes);
                     } else if (e0 < cnt) {
                         __align__(16) uint8_t tmp[16];
                         for (int b = 0; b < 16; ++b)
-                            tmp[b] = (e0 + b / P::kElemBytes < cnt) ? xg[static_cast<size_t>(e0) * P::kElemBytes + b] : uint8_t(0);
+                            tmp[b] = (e0 + b / P::kElemBytes < cnt) ? xt[static_cast<size_t>(e0) * P::kElemBytes + b] : uint8_t(0);
                         xv = *reinterpret_cast<const uint4*>(tmp);
                     }
-                    const int w = e0 / SPAN, c = (e0 % SPAN) / CHUNK, j0 = e0 % CHUNK;
-                    *reinterpret_cast<uint4*>(xs + w * P::kSlabBytes + swz_offset<P::kRowBytes>(c, j0 * P::kElemBytes)) = xv;
+                    const int w = e0 / SCAN_UNIT, i = (e0 % SCAN_UNIT) / PIECE, l = (e0 % PIECE) / ROW, j0 = e0 % ROW;
+                    *reinterpret_cast<uint4*>(xs + i * P::kSlabBytes +
+                                              swz_offset<P::kRowBytes>(w * PIECE_ROWS + l, j0 * P::kElemBytes)) = xv;
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
@@ -264,11 +276,12 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const ScanParams prm
             *abort_flag = 1;
             if (lane == 0) report_error(prm.hdr, 5u);
         }
-        // wait (bounded) for copies still in flight before the CTA may exit
         for (int k = (it > S ? it - S : 0); k < it; ++k) mbar_wait(&bar_full[k % S], (k / S) & 1, 2000000ull);
     } else if (warp == SCAN_MMA_WARP) {
         // =========================== MMA issuer ===========================
-        constexpr uint32_t idesc = P::kIsFloat ? make_idesc_f16_f32(128, NCOL) : make_idesc_s8_s32(128, NCOL);
+        // Runs ahead of the epilogue: the products of a warpgroup's next tile go to its other buffer.
+        constexpr uint32_t idesc = P::kIsFloat ? (make_idesc_f16_f32(128, N) | P::kFmtBits) : make_idesc_s8_s32(128, N);
+        int sentinels = 0;
         for (int it = 0;; ++it) {
             const int stage = it % S;
             if (!wait_bar(&bar_full[stage], (it / S) & 1, abort_flag, budget)) {
@@ -276,9 +289,13 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const ScanParams prm
                 if (lane == 0) report_error(prm.hdr, 5u);
                 break;
             }
-            if (tile_slot[stage] < 0) break;
-            const int acc = it & 1;
-            if (!wait_bar(&bar_acc_empty[acc], ((it >> 1) & 1) ^ 1, abort_flag, budget)) {
+            if (tile_slot[stage] < 0) {
+                if (++sentinels == SCAN_GROUPS) break;
+                continue;
+            }
+            const int g = it % SCAN_GROUPS, k = it / SCAN_GROUPS;
+            const int buf = g * Cfg::kBufsPerGroup + (k % Cfg::kBufsPerGroup);
+            if (!wait_bar(&bar_acc_empty[buf], ((k / Cfg::kBufsPerGroup) & 1) ^ 1, abort_flag, budget)) {
                 *abort_flag = 1;
                 if (lane == 0) report_error(prm.hdr, 5u);
                 break;
@@ -286,155 +303,291 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const ScanParams prm
             tc_fence_after_sync();
             if (lane == 0) {
                 const uint32_t xs = smem_u32(sStage + stage * Cfg::kStageBytes);
-                const uint32_t as = smem_u32(sA);
-                const uint32_t d = tmem_base + acc * NCOL;
+                const uint32_t bs = smem_u32(sB);
 #pragma unroll
-                for (int w = 0; w < 4; ++w) {
+                for (int i = 0; i < SCAN_UP; ++i) {
+                    const uint32_t d = tmem_base + buf * (SCAN_UP * N) + i * N;
 #pragma unroll
                     for (int ks = 0; ks < P::kMmaPerSlab; ++ks) {
-                        const uint32_t off = w * P::kSlabBytes + ks * P::kKStepBytes;
-                        const uint64_t da = make_desc(as + off, P::kSbo, P::kLayoutType);
-                        const uint64_t db = make_desc(xs + off, P::kSbo, P::kLayoutType);
-                        if constexpr (P::kIsFloat) mma_f16_ss(d, da, db, idesc, (w | ks) != 0);
-                        else mma_i8_ss(d, da, db, idesc, (w | ks) != 0);
+                        const uint64_t da = make_desc(xs + i * P::kSlabBytes + ks * P::kKStepBytes, P::kSbo, P::kLayoutType);
+                        const uint64_t db = make_desc(bs + ks * P::kKStepBytes, P::kSbo, P::kLayoutType);
+                        if constexpr (P::kIsFloat) mma_f16_ss(d, da, db, idesc, ks != 0);
+                        else mma_i8_ss(d, da, db, idesc, ks != 0);
                     }
                 }
-                tc_commit(&bar_acc_full[acc]);
+                tc_commit(&bar_acc_full[buf]);
             }
             __syncwarp();
         }
     } else {
         // =========================== epilogue ===========================
-        const int g = warp >> 2;            // warpgroup: handles iterations it = g, g+2, ...
-        const int w = warp & 3;             // span inside the tile = TMEM lane block
-        const uint32_t lanemask_le = 0xffffffffu >> (31u - lane);
+        constexpr int UP = SCAN_UP;
+        const int g = warp >> 2;            // warpgroup: iterations g, g + SCAN_GROUPS, ...
+        const int w = warp & 3;             // unit inside the tile = TMEM lane quarter
         Acc* outp = static_cast<Acc*>(prm.out);
-        for (int it = g;; it += 2) {
-            const int stage = it % S;
-            if (!wait_bar(&bar_full[stage], (it / S) & 1, abort_flag, budget)) {
-                *abort_flag = 1;
-                if (lane == 0) report_error(prm.hdr, 5u);
-                break;
+        uint8_t* stg = smem + Cfg::kOutOffset + warp * Cfg::kOutBufs * Cfg::kOutBufBytes;
+        const long long nrows_full = prm.n / ROW;
+        // first accumulator column of this warp's unit, in its lane quarter
+        int obuf = 0;
+        bool failed = false;
+
+        MMV_T_DECL
+        // stages the 32 x 32 block held in r (lane = row) and stores it with one TMA store
+        auto store_piece = [&](const uint32_t (&r)[32], long long prow) {
+            uint8_t* ob = stg + obuf * Cfg::kOutBufBytes;
+            if (lane == 0) tma_store_wait_read<Cfg::kOutBufs - 1>();   // the buffer about to be reused is free again
+            __syncwarp();
+            MMV_T_MARK(6)
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4)
+                *reinterpret_cast<uint4*>(ob + lane * 128 + ((c4 ^ (lane & 7)) << 4)) =
+                    make_uint4(r[4 * c4], r[4 * c4 + 1], r[4 * c4 + 2], r[4 * c4 + 3]);
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0 && prow < nrows_full) {
+                tma_store_2d(&tmap_out, ob, 0, static_cast<int>(prow));
+                tma_store_commit();
             }
+            // the one row that straddles n (n not a multiple of 32) is written with plain stores
+            if (prow + lane == nrows_full) {
+                const int cnt = static_cast<int>(prm.n - nrows_full * ROW);
+                for (int j = 0; j < cnt; ++j) {
+                    uint32_t v = r[0];
+#pragma unroll
+                    for (int q = 1; q < 32; ++q)
+                        if (j == q) v = r[q];
+                    reinterpret_cast<uint32_t*>(outp)[nrows_full * ROW + j] = v;
+                }
+            }
+            obuf = (obuf + 1) % Cfg::kOutBufs;
+        };
+
+        for (int k = 0;; ++k) {
+            const int it = g + SCAN_GROUPS * k;
+            const int stage = it % S;
+            if (!wait_stage(&stage_iter[stage], it, &bar_full[stage], (it / S) & 1, abort_flag, budget)) { failed = true; break; }
             const int tile = tile_slot[stage];
             if (tile < 0) break;
-            if (!wait_bar(&bar_acc_full[g], (it >> 1) & 1, abort_flag, budget)) {
-                *abort_flag = 1;
-                if (lane == 0) report_error(prm.hdr, 5u);
-                break;
+            MMV_T_MARK(0)
+
+            const int buf = g * Cfg::kBufsPerGroup + (k % Cfg::kBufsPerGroup);
+            const uint32_t taddr = tmem_base + buf * (UP * N) + ((static_cast<uint32_t>(w) * 32u) << 16);
+            const long long s = static_cast<long long>(tile) * SPANS_PER_TILE + w;      // this warp's unit
+
+            // ---- flag bytes -> one start mask per row (registers) ----
+            uint32_t fm[UP];
+            uint32_t pm[UP];
+            {
+                const uint8_t* fs = sStage + stage * Cfg::kStageBytes + Cfg::kXBytes + w * SCAN_UNIT + lane * ROW;
+#pragma unroll
+                for (int i = 0; i < UP; ++i) {
+                    const uint4 a = *reinterpret_cast<const uint4*>(fs + i * PIECE);
+                    const uint4 b = *reinterpret_cast<const uint4*>(fs + i * PIECE + 16);
+                    const uint32_t any = a.x | a.y | a.z | a.w | b.x | b.y | b.z | b.w;
+                    fm[i] = any ? flag_bytes_to_mask(a, b) : 0u;
+                    pm[i] = __ballot_sync(0xffffffffu, fm[i] != 0u);
+                }
             }
+            MMV_T_MARK(1)
+            if (!wait_bar(&bar_acc_full[buf], (k / Cfg::kBufsPerGroup) & 1, abort_flag, budget)) { failed = true; break; }
+            MMV_T_MARK(2)
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_empty[stage]);      // operands consumed, flags in registers
             tc_fence_after_sync();
 
-            const uint8_t* xs = sStage + stage * Cfg::kStageBytes + w * P::kSlabBytes;
-            const uint8_t* fs = sStage + stage * Cfg::kStageBytes + Cfg::kXBytes + w * SPAN;
-            const long long s = static_cast<long long>(tile) * SPANS_PER_TILE + w;
-            const long long base = s * SPAN;
-            const long long rem = prm.n - base;           // elements of this span that exist (may be <= 0)
-            const int lim = rem >= SPAN ? SPAN : (rem > 0 ? static_cast<int>(rem) : 0);
-            const uint32_t taddr = tmem_base + g * NCOL + ((static_cast<uint32_t>(w) * 32u) << 16);
-
-            // ---- pass A: local segmented scan of the span ----
-            Acc run = Acc(0);                 // sum of the open segment so far (uniform)
-            bool seen = false;                // a flag occurred in this span (uniform)
-            int ffc = NCOL;                   // chunk of the span's first flag
-            uint32_t ffm = 0u;                // flag mask of that chunk
-            int ndef = 0;                     // leading groups whose store waits for the carry
-            uint32_t r[32];
-#pragma unroll 1
-            for (int gg = 0; gg < NCOL / 32; ++gg) {
-                tmem_ld_32x32(taddr + gg * 32, r);
-                tmem_ld_wait();
-                const bool defer = !seen;
+            // ---- pre-pass: row totals, unit aggregate, publish ----
+            Acc tot[UP];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int c = gg * 32 + j;
-                    const uint32_t fb = fs[c * CHUNK + lane];
-                    uint32_t m = __ballot_sync(0xffffffffu, fb != 0u);
-                    if (s == 0 && c == 0) m |= 1u;        // element 0 always opens a segment
-                    const Acc xb = P::from_bits(r[j]);
-                    const uint32_t le = m & lanemask_le;
-                    const int p = 31 - __clz(le);         // last flag at or before this lane, -1 if none
-                    const Acc v = __shfl_sync(0xffffffffu, xb, (p - 1) & 31);
-                    Acc zl = (p > 0) ? P::sub(xb, v) : xb;
+            for (int i = 0; i < UP; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * N + (ROW - 1)));
+            tmem_ld_wait();
+            uint32_t anyp = 0u;
+            int i0 = UP;                    // first piece with a flag
+#pragma unroll
+            for (int i = UP - 1; i >= 0; --i) {
+                anyp |= pm[i];
+                if (pm[i]) i0 = i;
+            }
+            const bool flagged = anyp != 0u;
+            Acc tail_unit;
+            if (!flagged) {
+                Acc t = tot[0];
+#pragma unroll
+                for (int i = 1; i < UP; ++i) t = P::add(t, tot[i]);
+                tail_unit = warp_sum<P>(t);
+            } else {
+                int istar = 0;
+#pragma unroll
+                for (int i = 0; i < UP; ++i)
+                    if (pm[i]) istar = i;
+                uint32_t pms = pm[0], fms = fm[0];
+                Acc tots = tot[0];
+#pragma unroll
+                for (int i = 1; i < UP; ++i)
+                    if (istar == i) { pms = pm[i]; fms = fm[i]; tots = tot[i]; }
+                const int lstar = 31 - __clz(pms);
+                const uint32_t fmstar = __shfl_sync(0xffffffffu, fms, lstar);
+                const int pl = 31 - __clz(fmstar);            // last flag of the last flagged row
+                Acc after = Acc(0);                            // totals of the rows behind it
+#pragma unroll
+                for (int i = 0; i < UP; ++i)
+                    if (i > istar) after = P::add(after, tot[i]);
+                if (static_cast<int>(lane) > lstar) after = P::add(after, tots);
+                after = warp_sum<P>(after);
+                Acc before = Acc(0);
+                if (pl > 0) {
+                    before = P::from_bits(tmem_ld_32x1(taddr + istar * N + (pl - 1)));
+                    tmem_ld_wait();
+                }
+                Acc row_tail = P::sub(tots, before);
+                if constexpr (P::kIsFloat) {
+                    if (pl == ROW - 1) {          // the tail is a segment's first element: the input value itself
+                        row_tail = P::from_bits(tmem_ld_32x1(taddr + istar * N + ROW + (ROW - 1)));
+                        tmem_ld_wait();
+                    }
+                }
+                tail_unit = P::add(__shfl_sync(0xffffffffu, row_tail, lstar), after);
+            }
+            const bool skip_publish = (s == prm.debug_skip_span);
+            if (lane == 0 && !skip_publish)
+                st_relaxed_gpu_u64(prm.status + s,
+                                   pack_status((flagged || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail_unit)));
+            MMV_T_MARK(3)
+
+            // ---- main pass: everything that does not need the carry of earlier units ----
+            const long long row0 = s * (SCAN_UNIT / ROW);
+            Acc run = Acc(0);                 // sum of the open segment inside this unit so far
+            uint32_t fm0 = 0u, pm0 = 0u;      // masks of the first flagged piece
+            LookbackWindow lbw;
+#pragma unroll
+            for (int i = 0; i < UP; ++i) {
+                // the first look-back window travels while the last piece is processed
+                if (i == UP - 1) lookback_load(prm.status, s - 1, lbw);
+                const uint32_t fmi = fm[i];
+                const uint32_t pmi = pm[i];
+                const Acc toti = tot[i];
+                if (i == i0) { fm0 = fmi; pm0 = pmi; }
+                uint32_t r[32];
+                uint32_t raw[P::kIsFloat ? 32 : 1];
+                tmem_ld_32x32(taddr + i * N, r);
+                if constexpr (P::kIsFloat) {
+                    if (pmi != 0u) tmem_ld_32x32(taddr + i * N + ROW, raw);
+                }
+                tmem_ld_wait();
+                MMV_T_MARK(4)
+                if (pmi == 0u) {
+                    // no flag in the piece: plain prefix of the row totals, one add per element
+                    Acc inc = toti;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const Acc t = __shfl_up_sync(0xffffffffu, inc, o);
+                        if (static_cast<int>(lane) >= o) inc = P::add(t, inc);
+                    }
+                    const Acc carry_row = P::add(run, P::sub(inc, toti));
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = P::to_bits(P::add(carry_row, P::from_bits(r[j])));
+                    run = P::add(run, __shfl_sync(0xffffffffu, inc, 31));
+                } else {
+                    // revert the speculation inside each row (Lemma A.1)
                     if constexpr (P::kIsFloat) {
-                        // the first element of a segment is the input value itself, exactly
-                        if ((m >> lane) & 1u) {
-                            const __half hx = *reinterpret_cast<const __half*>(xs + swz_offset<P::kRowBytes>(c, lane * 2));
-                            zl = __half2float(hx);
+                        Acc base = Acc(0);
+                        uint32_t prev = 0u;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const bool pj = (fmi >> j) & 1u;
+                            if (j > 0) base = pj ? P::from_bits(prev) : base;
+                            prev = r[j];
+                            // the first element of a segment is the input value itself, exactly
+                            r[j] = pj ? raw[j] : P::to_bits(P::sub(P::from_bits(r[j]), base));
+                        }
+                    } else {
+                        Acc base = Acc(0);
+                        uint32_t prev = 0u;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const bool pj = (fmi >> j) & 1u;
+                            if (j > 0) base = pj ? prev : base;
+                            prev = r[j];
+                            r[j] = P::sub(r[j], base);
                         }
                     }
-                    const Acc tail = __shfl_sync(0xffffffffu, zl, 31);
-                    const Acc z = (le == 0u) ? P::add(run, zl) : zl;
-                    run = (m != 0u) ? tail : P::add(run, tail);
-                    if (m != 0u && !seen) {
-                        seen = true;
-                        ffc = c;
-                        ffm = m;
+                    // segmented scan of the row tails across the 32 rows
+                    const bool rowflag = fmi != 0u;
+                    Acc val = P::from_bits(r[31]);
+                    if (lane == 0 && !rowflag) val = P::add(run, val);
+                    uint32_t flg = rowflag ? 1u : 0u;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const Acc tv = __shfl_up_sync(0xffffffffu, val, o);
+                        const uint32_t tf = __shfl_up_sync(0xffffffffu, flg, o);
+                        if (static_cast<int>(lane) >= o) {
+                            if (!flg) val = P::add(tv, val);
+                            flg |= tf;
+                        }
                     }
-                    r[j] = P::to_bits(z);
-                    if (!defer) {
-                        if (c * CHUNK + static_cast<int>(lane) < lim) outp[base + c * CHUNK + lane] = z;
-                    }
+                    Acc carry_row = __shfl_up_sync(0xffffffffu, val, 1);
+                    if (lane == 0) carry_row = run;
+                    run = __shfl_sync(0xffffffffu, val, 31);
+                    const int f0 = rowflag ? (__ffs(fmi) - 1) : 32;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < f0) r[j] = P::to_bits(P::add(carry_row, P::from_bits(r[j])));
                 }
-                if (defer) {
-                    tmem_st_32x32(taddr + gg * 32, r);
-                    ndef = gg + 1;
+                MMV_T_MARK(5)
+                if (i > i0) {
+                    store_piece(r, row0 + i * PIECE_ROWS);       // complete: no element reaches back past a flag
+                } else {
+                    tmem_st_32x32(taddr + i * N, r);             // parked until the carry is known
                 }
+                MMV_T_MARK(4)
             }
             tmem_st_wait();
 
-            // ---- publish, look back, publish ----
+            // ---- look back (most of its latency has been covered by the main pass) ----
             Acc carry = Acc(0);
-            bool ok = true;
-            const bool skip_publish = (s == prm.debug_skip_span);
-            if (s == 0) {
-                if (lane == 0 && !skip_publish) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(run)));
-            } else {
-                if (lane == 0 && !skip_publish)
-                    st_relaxed_gpu_u64(prm.status + s, pack_status(seen ? ST_PREFIX : ST_AGG, P::to_bits(run)));
-                ok = lookback<P>(prm.status, s, carry, abort_flag, budget);
-                if (!ok) {
-                    *abort_flag = 1;
-                    if (lane == 0) {
-                        report_error(prm.hdr, 5u);
-                        st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
-                    }
+            if (s != 0) {
+                if (!lookback<P>(prm.status, s, carry, abort_flag, budget, lbw, true)) {
+                    if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
+                    failed = true;
                     break;
                 }
-                if (!seen && lane == 0 && !skip_publish)
-                    st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(carry, run))));
+                if (!flagged && lane == 0 && !skip_publish)
+                    st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(carry, tail_unit))));
             }
 
-            // ---- pass B: add the carry before the span's first flag, store the deferred groups ----
+            // ---- parked pieces: add the carry in front of the unit's first flag, store ----
+            const int l0 = pm0 ? (__ffs(pm0) - 1) : 32;                       // first flagged row of piece i0
+            const int fpos = __ffs(__shfl_sync(0xffffffffu, fm0, l0 & 31)) - 1;  // its first flag
 #pragma unroll 1
-            for (int gg = 0; gg < ndef; ++gg) {
-                tmem_ld_32x32(taddr + gg * 32, r);
+            for (int i = 0; i <= i0 && i < UP; ++i) {
+                uint32_t r[32];
+                tmem_ld_32x32(taddr + i * N, r);
+                int limit = 32;
+                if (i == i0) limit = (static_cast<int>(lane) < l0) ? 32 : ((static_cast<int>(lane) == l0) ? fpos : 0);
                 tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const int c = gg * 32 + j;
-                    Acc z = P::from_bits(r[j]);
-                    const bool pre = (c < ffc) || (c == ffc && (ffm & lanemask_le) == 0u);
-                    if (pre) z = P::add(carry, z);
-                    if (c * CHUNK + static_cast<int>(lane) < lim) outp[base + c * CHUNK + lane] = z;
-                }
+                for (int j = 0; j < 32; ++j)
+                    if (j < limit) r[j] = P::to_bits(P::add(carry, P::from_bits(r[j])));
+                store_piece(r, row0 + i * PIECE_ROWS);
             }
+            MMV_T_MARK(7)
 
-            // ---- release the accumulator and the shared-memory stage ----
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(&bar_acc_empty[g]);
-                mbar_arrive(&bar_empty[stage]);
-            }
+            if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
         }
+        if (failed) {
+            *abort_flag = 1;
+            if (lane == 0) report_error(prm.hdr, 5u);
+        }
+        if (lane == 0) tma_store_wait_all<0>();
+        MMV_T_FLUSH()
     }
 
     tc_fence_before_sync();
     __syncthreads();
     if (warp == SCAN_MMA_WARP) {
         tc_fence_after_sync();
-        tmem_dealloc(tmem_base, SCAN_TMEM_COLS);
+        tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
 }
 

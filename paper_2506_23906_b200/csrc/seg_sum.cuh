@@ -21,14 +21,8 @@
 #include <cuda_runtime.h>
 #include "../../include/mmv.h"
 #include "common.cuh"
-#include "seg_scan.cuh"
 
 namespace mmv {
-
-constexpr int ROW = 32;
-constexpr int PIECE_ROWS = 32;
-constexpr int PIECE = ROW * PIECE_ROWS;        // 1024 elements
-constexpr int PIECES_PER_SPAN = SPAN / PIECE;  // 4
 
 constexpr int SUM_EPI_WARPS = 8;
 constexpr int SUM_PRODUCER_WARP = 8;
@@ -184,9 +178,10 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         while (ok) {
             const int stage = it % S;
             if (!wait_bar(&bar_empty[stage], ((it / S) & 1) ^ 1, abort_flag, budget)) { ok = false; break; }
-            int tile = 0;
-            if (lane == 0) tile = static_cast<int>(atomicAdd(&prm.hdr->tile_counter, 1u));
-            tile = __shfl_sync(0xffffffffu, tile, 0);
+            // static round-robin tile assignment: all CTAs are resident (grid <= SM count, one CTA per
+            // SM), so iteration `it` of every CTA runs at about the same time and a tile's predecessors
+            // are always in flight or finished
+            int tile = static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
             if (tile >= prm.num_tiles) tile = -1;
             if (lane == 0) tile_slot[stage] = tile;
             if (tile < 0) {
@@ -444,7 +439,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(seen ? ST_PREFIX : ST_AGG, P::to_bits(run)));
                 Acc carry = Acc(0);
                 if (!seen || def_r >= 0) {
-                    if (!lookback<P>(prm.status, s, carry, abort_flag, budget)) {
+                    LookbackWindow lbw;
+                    if (!lookback<P>(prm.status, s, carry, abort_flag, budget, lbw, false)) {
                         *abort_flag = 1;
                         if (lane == 0) {
                             report_error(prm.hdr, 5u);
