@@ -54,6 +54,8 @@ def parse_args():
     ap.add_argument("--case", default="p1e-3", help="flag pattern of the headline workload")
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline")
+    ap.add_argument("--profile-case", default=None, choices=["scan_f16", "scan_i8", "seg_sum", "spmv"],
+                    help="run one small case a few times and exit (the command profiled with ncu)")
     return ap.parse_args()
 
 
@@ -430,9 +432,43 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_profile_case(args):
+    """One small case, `steps` launches, no timing: the target of the ncu captures under profiles/."""
+    import torch
+    import paper_2506_23906_b200 as mmv
+    torch.cuda.set_device(0)
+    n = 1 << min(args.log2n, 27)
+    if args.profile_case in ("scan_f16", "scan_i8"):
+        f16 = args.profile_case == "scan_f16"
+        x = gen.f16_uniform(5, n) if f16 else gen.i8_uniform(3, n)
+        f = gen.config5_flags(n, args.case)
+        xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+        out = torch.empty(n, dtype=torch.float32 if f16 else torch.int32, device="cuda")
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.F16_TO_F32 if f16 else mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+        fn = lambda: mmv.seg_scan(xd, fd, out=out, workspace=ws)  # noqa: E731
+    elif args.profile_case == "seg_sum":
+        x, off = gen.config2(n)
+        xd, od = torch.from_numpy(x).cuda(), torch.from_numpy(off).cuda()
+        out = torch.empty(off.shape[0] - 1, dtype=torch.float32, device="cuda")
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, n, off.shape[0] - 1)
+        fn = lambda: mmv.seg_sum(xd, od, out=out, workspace=ws)  # noqa: E731
+    else:
+        rowptr, col, val, xv = gen.config4(rows=1 << 18)
+        rd, cd, vd, xd = (torch.from_numpy(t).cuda() for t in (rowptr, col, val, xv))
+        y = torch.empty(rowptr.shape[0] - 1, dtype=torch.float32, device="cuda")
+        ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, val.shape[0], rowptr.shape[0] - 1)
+        fn = lambda: mmv.spmv_csr(rd, cd, vd, xd, y=y, workspace=ws)  # noqa: E731
+    for _ in range(max(1, args.steps)):
+        fn()
+    torch.cuda.synchronize()
+    print(json.dumps({"profile_case": args.profile_case, "n": n, "status": mmv.last_async_status(ws)}))
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.profile_case:
+        run_profile_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
