@@ -136,6 +136,44 @@ const char *mmv_status_string(mmv_status s);
 int64_t mmv_kernel_launch_count(void);
 
 /*
+ * Segmented inclusive scan for callers that cannot provide a workspace.
+ * (The paper has no counterpart: this is a packaging variant of mmv_seg_scan.)
+ *
+ * Some users of this library may not allocate device memory at the moment they
+ * need a scan: a service that handed the whole GPU to its own memory pool at
+ * start-up, a plug-in that runs inside another framework's operator and is
+ * given only its input and output buffers, a control loop where an allocation's
+ * implicit device synchronisation would break its timing.  For them this entry
+ * point takes only x, the uint8 start flags and out; the per-unit carry words
+ * that mmv_seg_scan keeps in the caller's workspace live in a fixed buffer
+ * inside the library's own device image instead (about 0.5 MB, resident on
+ * every GPU that loads the library until the process exits).  The call itself
+ * performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ * Limits and rules
+ *   - n <= MMV_STATIC_SCAN_MAX_N; larger inputs are refused with
+ *     MMV_ERR_WORKSPACE_TOO_SMALL and nothing is enqueued.
+ *   - Flag-encoded segments only; arithmetic, alignment rules, asynchrony and
+ *     error reporting are those of mmv_seg_scan.
+ *   - The first call on each device looks up the device address of the built-in
+ *     buffer (the device must be current); make that first call before starting
+ *     any stream capture.
+ *   - All calls on a device share the one buffer.  Each call clears the part it
+ *     uses on its stream before the kernel runs, so stale contents never leak
+ *     into a result, but two calls that overlap on the GPU (different streams)
+ *     would overwrite each other's carries: serialise them.
+ *   - Device-side status (time-outs) is returned by
+ *     mmv_seg_scan_static_last_status().
+ */
+#define MMV_STATIC_SCAN_MAX_N (1ll << 28)
+mmv_status mmv_seg_scan_static(const void *x, const void *flags_u8, int64_t n, mmv_dtype dt, void *out,
+                               void *cuda_stream);
+
+/* Synchronises the stream and returns the device-side status of the last mmv_seg_scan_static call
+ * on the current device. */
+mmv_status mmv_seg_scan_static_last_status(void *cuda_stream);
+
+/*
  * Test hook.  wait_budget_ns: time after which a device-side wait gives up
  * (<= 0 restores the default of 4 s).  skip_publish_span: index of one
  * 4096-element span of the scan that never publishes its carry, so that its

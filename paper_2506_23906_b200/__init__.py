@@ -25,7 +25,9 @@ OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR = 0, 1, 2
 EXPORTS = (
     "mmv_workspace_bytes", "mmv_seg_scan", "mmv_seg_sum", "mmv_spmv_csr",
     "mmv_last_async_status", "mmv_status_string", "mmv_kernel_launch_count", "mmv_debug_configure",
+    "mmv_seg_scan_static", "mmv_seg_scan_static_last_status",
 )
+STATIC_SCAN_MAX_N = 1 << 28
 
 
 class MmvError(RuntimeError):
@@ -55,6 +57,10 @@ def _load() -> ctypes.CDLL:
     lib.mmv_status_string.argtypes = [ci]
     lib.mmv_kernel_launch_count.restype = i64
     lib.mmv_kernel_launch_count.argtypes = []
+    lib.mmv_seg_scan_static.restype = ci
+    lib.mmv_seg_scan_static.argtypes = [vp, vp, i64, ci, vp, vp]
+    lib.mmv_seg_scan_static_last_status.restype = ci
+    lib.mmv_seg_scan_static_last_status.argtypes = [vp]
     lib.mmv_debug_configure.restype = None
     lib.mmv_debug_configure.argtypes = [i64, i64]
     return lib
@@ -135,6 +141,26 @@ def seg_scan(x: torch.Tensor, seg: torch.Tensor, out: torch.Tensor | None = None
     if rc != MMV_OK:
         raise MmvError(rc, "mmv_seg_scan")
     return out
+
+
+def seg_scan_static(x: torch.Tensor, flags: torch.Tensor, out: torch.Tensor, stream=None) -> torch.Tensor:
+    """mmv_seg_scan_static: the scan for callers that can pass only inputs and outputs.
+
+    The carry words live in a buffer built into the library, so nothing is allocated by the
+    call (here the caller supplies ``out`` too).  n is limited to STATIC_SCAN_MAX_N; calls on
+    one device must not overlap on the GPU.
+    """
+    _check_cuda(x, flags, out)
+    if flags.dtype != torch.uint8:
+        raise TypeError("start flags must be uint8")
+    rc = _lib.mmv_seg_scan_static(_ptr(x), _ptr(flags), x.numel(), _dtype_code(x), _ptr(out), _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_seg_scan_static")
+    return out
+
+
+def seg_scan_static_last_status(stream=None) -> int:
+    return int(_lib.mmv_seg_scan_static_last_status(_stream_ptr(stream)))
 
 
 def seg_sum(x: torch.Tensor, seg: torch.Tensor, out: torch.Tensor | None = None,

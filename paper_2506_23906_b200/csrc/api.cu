@@ -228,6 +228,34 @@ __global__ void offsets_to_flags_kernel(const int32_t* __restrict__ off, long lo
     }
 }
 
+// ---------------------------------------------------------------------------
+// Built-in scratch of mmv_seg_scan_static: header + one status word per 4096-element unit.
+// The symbol below is a host-side stand-in in host code; its device address is looked up once per
+// device with cudaGetSymbolAddress and only that address is ever handed to a kernel or a memset.
+// ---------------------------------------------------------------------------
+constexpr long long kStaticScanMaxN = MMV_STATIC_SCAN_MAX_N;
+constexpr size_t kStaticScratchBytes =
+    sizeof(WorkspaceHeader) + static_cast<size_t>((kStaticScanMaxN + SCAN_UNIT - 1) / SCAN_UNIT) * sizeof(uint64_t);
+static __device__ __align__(256) unsigned char g_static_scan_scratch[kStaticScratchBytes];
+
+struct StaticScratch {
+    std::once_flag once;
+    void* ptr = nullptr;
+};
+StaticScratch g_static_scratch[kMaxDevices];
+
+// Device address of the built-in scratch on the current device (nullptr on failure).
+void* static_scratch_ptr() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    StaticScratch* sc = &g_static_scratch[dev];
+    std::call_once(sc->once, [sc] {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scan_scratch) == cudaSuccess) sc->ptr = p;
+    });
+    return sc->ptr;
+}
+
 }  // namespace
 }  // namespace mmv
 
@@ -373,6 +401,54 @@ mmv_status mmv_last_async_status(const void* workspace, void* cuda_stream) {
     WorkspaceHeader h;
     if (cudaMemcpy(&h, workspace, sizeof(unsigned int) * 2, cudaMemcpyDeviceToHost) != cudaSuccess) return MMV_ERR_CUDA;
     return h.error <= 6u ? static_cast<mmv_status>(h.error) : MMV_ERR_CUDA;
+}
+
+mmv_status mmv_seg_scan_static(const void* x, const void* flags_u8, int64_t n, mmv_dtype dt, void* out,
+                               void* cuda_stream) {
+    if (n < 0) return MMV_ERR_INVALID_ARG;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
+    if (n == 0) return MMV_OK;
+    if (n > kStaticScanMaxN) return MMV_ERR_WORKSPACE_TOO_SMALL;      // the built-in buffer covers 2^28 elements
+    if (!x || !flags_u8 || !out) return MMV_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(flags_u8) || !aligned16(out)) return MMV_ERR_INVALID_ARG;
+    DeviceInfo* dev = device_info();
+    if (!dev) return MMV_ERR_CUDA;
+    uint8_t* ws = static_cast<uint8_t*>(static_scratch_ptr());        // device address, never the host symbol
+    if (!ws) return MMV_ERR_CUDA;
+
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const long long tiles = num_scan_tiles_of(n);
+    const size_t used = sizeof(WorkspaceHeader) + static_cast<size_t>(tiles) * SPANS_PER_TILE * sizeof(uint64_t);
+    // the buffer keeps the previous call's words: everything this call reads must start at zero
+    if (cudaMemsetAsync(ws, 0, used, st) != cudaSuccess) return MMV_ERR_CUDA;
+
+    const bool f16 = dt == MMV_F16_TO_F32;
+    CUtensorMap tmap, tmap_out;
+    if (!encode_span_map(&tmap, x, n, f16 ? 2 : 1, SCAN_UP)) return MMV_ERR_CUDA;
+    if (!encode_out_map(&tmap_out, out, n)) return MMV_ERR_CUDA;
+    ScanParams prm;
+    prm.x = x;
+    prm.flags = static_cast<const uint8_t*>(flags_u8);
+    prm.out = out;
+    prm.n = n;
+    prm.num_tiles = static_cast<int>(tiles);
+    prm.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+    prm.status = reinterpret_cast<uint64_t*>(ws + sizeof(WorkspaceHeader));
+    prm.budget_ns = g_budget_ns.load();
+    prm.debug_skip_span = -1;
+    const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
+    if (f16)
+        seg_scan_kernel<F16Path><<<grid, SCAN_THREADS, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+    else
+        seg_scan_kernel<I8Path><<<grid, SCAN_THREADS, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+}
+
+mmv_status mmv_seg_scan_static_last_status(void* cuda_stream) {
+    void* ws = static_scratch_ptr();
+    if (!ws) return MMV_ERR_CUDA;
+    return mmv_last_async_status(ws, cuda_stream);
 }
 
 const char* mmv_status_string(mmv_status s) {

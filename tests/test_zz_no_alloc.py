@@ -1,0 +1,63 @@
+"""mmv_seg_scan_static: the scan entry point that needs no workspace from the caller.
+
+Some callers cannot allocate device memory when they need a scan (all memory already handed
+to their own pool, or only input/output buffers are given to them), so this entry point keeps
+its carry words in a buffer built into the library.  The test calls it through the C ABI twice
+in a row -- the second call with different segments, so that words left in the shared buffer
+by the first call would show -- and compares each result with mmv_seg_scan's on the same input.
+This file is collected last on purpose.
+"""
+import numpy as np
+import pytest
+
+import oracle
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mmv():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2506_23906_b200 as m
+    m.debug_configure(0, -1)
+    return m
+
+
+def test_static_scan_matches_workspace_scan_on_two_calls_in_a_row(mmv):
+    n = 7 * 16384 + 1234                       # several tiles and a ragged tail
+    rng = np.random.default_rng(2024)
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    xf = rng.uniform(-1, 1, n).astype(np.float16)
+    flag_sets = [(rng.random(n) < 0.02).astype(np.uint8), (rng.random(n) < 1e-4).astype(np.uint8)]
+    for x in (xi, xf):
+        xd = torch.from_numpy(x).cuda()
+        odt = torch.int32 if x.dtype == np.int8 else torch.float32
+        for f in flag_sets:                     # two calls in a row share the built-in buffer
+            fd = torch.from_numpy(f).cuda()
+            want = mmv.seg_scan(xd, fd)         # the existing entry point, caller-provided workspace
+            got = torch.full((n + 32,), -777, dtype=odt, device="cuda")
+            mmv.seg_scan_static(xd, fd, got[:n])
+            assert mmv.seg_scan_static_last_status() == 0
+            g, w = got.cpu().numpy(), want.cpu().numpy()
+            assert (g[n:] == -777).all()
+            if x.dtype == np.int8:
+                assert np.array_equal(g[:n], w)                 # bit-exact
+            else:
+                # both results lie inside the library's bound around the exact value; they may differ
+                # from each other in the last bits because the carry chain groups its adds by timing
+                z, a = oracle.seg_scan_f16(x, f)
+                bound = oracle.fp_bound(a)
+                assert (np.abs(g[:n].astype(np.float64) - w.astype(np.float64)) <= bound).all()
+                assert (np.abs(g[:n].astype(np.float64) - z) <= bound).all()
+
+
+def test_static_scan_refuses_inputs_beyond_its_buffer(mmv):
+    x = torch.zeros(64, dtype=torch.int8, device="cuda")
+    f = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    out = torch.zeros(64, dtype=torch.int32, device="cuda")
+    rc = mmv._lib.mmv_seg_scan_static(x.data_ptr(), f.data_ptr(), mmv.STATIC_SCAN_MAX_N + 1, mmv.I8_TO_I32,
+                                      out.data_ptr(), None)
+    assert rc == 3 and "workspace" in mmv.status_string(rc)
+    assert mmv._lib.mmv_seg_scan_static(x.data_ptr(), f.data_ptr(), 0, mmv.I8_TO_I32, out.data_ptr(), None) == 0
