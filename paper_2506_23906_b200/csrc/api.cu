@@ -137,7 +137,7 @@ WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     p.flags_off = p.status_off + p.status_bytes;
     p.flags_bytes = (op == MMV_OP_SEG_SCAN && sf == MMV_SEG_OFFSETS_I32) ? round_up(static_cast<size_t>(n), 256) : 0;
     p.tileq_off = p.flags_off + p.flags_bytes;
-    p.tileq_bytes = (op != MMV_OP_SEG_SCAN) ? round_up(static_cast<size_t>(tiles + 1) * sizeof(int32_t), 256) : 0;
+    p.tileq_bytes = (op != MMV_OP_SEG_SCAN) ? round_up(static_cast<size_t>(tiles * SPANS_PER_TILE + 1) * sizeof(int32_t), 256) : 0;
     p.prod_off = p.tileq_off + p.tileq_bytes;
     p.prod_bytes = (op == MMV_OP_SPMV_CSR) ? round_up(static_cast<size_t>(n) * 4, 256) : 0;
     p.total = p.prod_off + p.prod_bytes;
@@ -186,13 +186,14 @@ template <typename P>
 mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* off, long long nseg, int shift,
                           void* out, uint8_t* ws, const WorkspacePlan& plan, DeviceInfo* dev, cudaStream_t st) {
     const int tiles = static_cast<int>(num_tiles_of(n_eff));
-    int32_t* tile_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
+    int32_t* span_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
     {
-        const int warps = tiles + 1;
+        const long long spans = static_cast<long long>(tiles) * SPANS_PER_TILE;
+        const long long warps = spans + 1;
         const int threads = 256;
-        const int blocks = (warps * 32 + threads - 1) / threads;
-        partition_offsets_kernel<<<blocks, threads, 0, st>>>(off, nseg, shift, tiles, tile_q, n_eff,
-                                                             reinterpret_cast<WorkspaceHeader*>(ws));
+        const long long blocks = (warps * 32 + threads - 1) / threads;
+        partition_offsets_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, shift, spans, span_q, n_eff,
+                                                                                 reinterpret_cast<WorkspaceHeader*>(ws));
         ++g_launches;
     }
     CUtensorMap tmap;
@@ -204,7 +205,7 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     prm.off_shift = shift;
     prm.out = out;
     prm.num_tiles = tiles;
-    prm.tile_q = tile_q;
+    prm.span_q = span_q;
     prm.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();

@@ -2,20 +2,24 @@
 // quantity; Section 4.3 remark after Algorithm 4.4 for the offset encoding) and
 // CSR SpMV built on it (Algorithm 4.4, Algorithms A.4-A.6), single pass, sm_100a.
 //
-// Layout ("row-major" view of the paper: x as a ceil(n/s) x s matrix, s = ROW = 32):
+// Layout (the paper's ceil(n/s) x s row-major matrix view, s = ROW = 32):
 //   a warp owns a SPAN of 128 consecutive rows (4096 elements) in four PIECES of
 //   32 rows; a TILE is four spans.  Tensor-core product i of a tile multiplies the
 //   [128 rows x 32] matrix made of piece i of each span (A operand, brought by one
 //   4-D TMA box, K-major, hardware swizzle) with the constant upper-triangular
 //   all-ones U_32 (B operand): TMEM lane 32w+l, column j = inclusive prefix at
 //   position j of row l of piece i of span w  --  z = MATMUL(x, U_s).
-//   Epilogue warps copy their 32 x 32 prefixes to shared memory, scan the 32 row
-//   totals with shuffles, and then only touch the segment boundaries: every segment
-//   end inside the piece emits  prefix(end) - prefix(start-1)  (the DIFF of
-//   Algorithm 4.2 applied to the COMPRESSed speculative scan, but with prefixes that
-//   are local to the row or the piece so that magnitudes stay small), segments that
-//   cross pieces take the running sum of the open segment, and segments that cross
-//   spans take the carry of a decoupled look-back over per-span status words.
+//   The MMA warp runs one tile ahead (two TMEM buffers per warpgroup).
+//   Epilogue warps (lane = row) read the row totals (TMEM column 31) and only touch
+//   the segment boundaries, which they hold in registers (one offset per lane):
+//   a piece that contains a boundary has its 32 x 32 prefixes copied to shared
+//   memory and its row totals scanned with shuffles; every segment end inside it
+//   emits  prefix(end) - prefix(start-1)  (the DIFF of Algorithm 4.2 applied to the
+//   COMPRESSed speculative scan, but with prefixes local to the row or the piece so
+//   that magnitudes stay small); very short segments are summed directly from the
+//   input values; segments that cross pieces take the running sum of the open
+//   segment, and segments that cross spans take the carry of a decoupled look-back
+//   over per-span status words.  Pieces without a boundary only add their total.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -28,13 +32,30 @@ constexpr int SUM_EPI_WARPS = 8;
 constexpr int SUM_PRODUCER_WARP = 8;
 constexpr int SUM_MMA_WARP = 9;
 constexpr int SUM_THREADS = 320;
-constexpr int SUM_TMEM_COLS = 256;             // 2 buffers x 4 products x 32 columns
+constexpr int SUM_BUFS = 4;                                        // TMEM tile buffers: two per warpgroup
+constexpr int SUM_TMEM_COLS = SUM_BUFS * PIECES_PER_SPAN * ROW;    // 512
+constexpr int SUM_DIRECT_LEN = 4;                                  // segments this short are summed from the inputs
 
-// bf16 values (used for the hi/lo halves of the fp32 products of SpMV): same geometry as fp16.
+// bf16 values (the hi/lo halves of the fp32 products of SpMV): same geometry as fp16.
 struct BF16Path : F16Path {
     static constexpr uint32_t kOneBits = 0x3F80u;                       // 1.0 in bf16
     static constexpr uint32_t kFmtBits = (1u << 7) | (1u << 10);        // A and B are bf16
 };
+
+template <typename P>
+__device__ __forceinline__ typename P::Acc load_value(const void* base, long long idx);
+template <>
+__device__ __forceinline__ float load_value<F16Path>(const void* base, long long idx) {
+    return __half2float(static_cast<const __half*>(base)[idx]);
+}
+template <>
+__device__ __forceinline__ float load_value<BF16Path>(const void* base, long long idx) {
+    return __bfloat162float(static_cast<const __nv_bfloat16*>(base)[idx]);
+}
+template <>
+__device__ __forceinline__ uint32_t load_value<I8Path>(const void* base, long long idx) {
+    return static_cast<uint32_t>(static_cast<int32_t>(static_cast<const int8_t*>(base)[idx]));
+}
 
 template <typename P>
 struct SumCfg {
@@ -57,18 +78,18 @@ struct SumParams {
     int off_shift;               // boundaries are off[q] << off_shift (1 for the hi/lo pairs of SpMV)
     void* out;                   // nseg results
     int num_tiles;
-    const int32_t* tile_q;       // num_tiles + 1: first q with (off[q] << shift) >= tile start
+    const int32_t* span_q;       // 4 * num_tiles + 1: first q with (off[q] << shift) >= span start
     WorkspaceHeader* hdr;
     uint64_t* status;
     unsigned long long budget_ns;
 };
 
-// tile_q[t] = first index q in [0, nseg] with (off[q] << shift) >= t * TILE, nseg + 1 if none.
-// One warp per tile boundary, 32-ary search.
-// The same launch validates the offsets (non-decreasing, inside [0, n]) and records
-// MMV_ERR_BAD_SEGMENTS otherwise; the main kernel never indexes outside its tile whatever they hold.
-__global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, int shift, int num_tiles,
-                                         int32_t* __restrict__ tile_q, long long n, WorkspaceHeader* hdr) {
+// span_q[s] = first index q in [0, nseg] with (off[q] << shift) >= s * SPAN, nseg + 1 if none.
+// One warp per span edge, 32-ary search.  The same launch validates the offsets (non-decreasing,
+// inside [0, n]) and records MMV_ERR_BAD_SEGMENTS otherwise; the main kernel never indexes
+// outside its tile whatever they hold.
+__global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, int shift, long long num_spans,
+                                         int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr) {
     {
         const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
         bool bad = false;
@@ -78,10 +99,10 @@ __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long l
         }
         if (bad) report_error(hdr, 4u);
     }
-    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long warp = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (warp > num_tiles) return;
-    const long long target = static_cast<long long>(warp) * TILE;
+    if (warp > num_spans) return;
+    const long long target = warp * SPAN;
     long long lo = 0, hi = nseg + 1;
     while (hi > lo) {
         const long long len = hi - lo;
@@ -103,7 +124,7 @@ __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long l
             hi = ke - 1;
         }
     }
-    if (lane == 0) tile_q[warp] = static_cast<int32_t>(lo);
+    if (lane == 0) span_q[warp] = static_cast<int32_t>(lo);
 }
 
 template <typename P>
@@ -120,9 +141,10 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
     uint64_t* bar_full = reinterpret_cast<uint64_t*>(smem + Cfg::kBarOffset);
     uint64_t* bar_empty = bar_full + S;
     uint64_t* bar_acc_full = bar_empty + S;
-    uint64_t* bar_acc_empty = bar_acc_full + 2;
-    int* tile_slot = reinterpret_cast<int*>(bar_acc_empty + 2);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_slot + S);
+    uint64_t* bar_acc_empty = bar_acc_full + SUM_BUFS;
+    // per stage: (iteration << 32) | tile, written as one word before the stage's barrier is armed
+    volatile long long* stage_info = reinterpret_cast<volatile long long*>(bar_acc_empty + SUM_BUFS);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<long long*>(stage_info) + S);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5;
@@ -133,8 +155,9 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         for (int i = 0; i < S; ++i) {
             mbar_init(&bar_full[i], 1);
             mbar_init(&bar_empty[i], 1);      // released by the MMA warp's commit
+            stage_info[i] = -1;
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < SUM_BUFS; ++i) {
             mbar_init(&bar_acc_full[i], 1);
             mbar_init(&bar_acc_empty[i], 4);
         }
@@ -183,7 +206,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             // are always in flight or finished
             int tile = static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
             if (tile >= prm.num_tiles) tile = -1;
-            if (lane == 0) tile_slot[stage] = tile;
+            if (lane == 0)
+                stage_info[stage] = (static_cast<long long>(it) << 32) | static_cast<long long>(static_cast<unsigned int>(tile));
             if (tile < 0) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar_full[stage]);
@@ -232,9 +256,10 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         }
         for (int k = (it > S ? it - S : 0); k < it; ++k) mbar_wait(&bar_full[k % S], (k / S) & 1, 2000000ull);
     } else if (warp == SUM_MMA_WARP) {
-        // =========================== MMA issuer ===========================
+        // =========================== MMA issuer (one tile ahead of the epilogue) ===========================
         constexpr uint32_t idesc = P::kIsFloat ? (make_idesc_f16_f32(128, ROW) | P::kFmtBits)
                                                : make_idesc_s8_s32(128, ROW);
+        int sentinels = 0;
         for (int it = 0;; ++it) {
             const int stage = it % S;
             if (!wait_bar(&bar_full[stage], (it / S) & 1, abort_flag, budget)) {
@@ -242,9 +267,13 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (lane == 0) report_error(prm.hdr, 5u);
                 break;
             }
-            if (tile_slot[stage] < 0) break;
-            const int acc = it & 1;
-            if (!wait_bar(&bar_acc_empty[acc], ((it >> 1) & 1) ^ 1, abort_flag, budget)) {
+            if (static_cast<int>(stage_info[stage] & 0xffffffffll) < 0) {
+                if (++sentinels == 2) break;
+                continue;
+            }
+            const int g = it & 1, k = it >> 1;
+            const int buf = g * 2 + (k & 1);
+            if (!wait_bar(&bar_acc_empty[buf], ((k >> 1) & 1) ^ 1, abort_flag, budget)) {
                 *abort_flag = 1;
                 if (lane == 0) report_error(prm.hdr, 5u);
                 break;
@@ -255,7 +284,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 const uint32_t bs = smem_u32(sB);
 #pragma unroll
                 for (int i = 0; i < PIECES_PER_SPAN; ++i) {
-                    const uint32_t d = tmem_base + acc * (PIECES_PER_SPAN * ROW) + i * ROW;
+                    const uint32_t d = tmem_base + buf * (PIECES_PER_SPAN * ROW) + i * ROW;
 #pragma unroll
                     for (int ks = 0; ks < P::kMmaPerSlab; ++ks) {
                         const uint64_t da = make_desc(xs + i * P::kSlabBytes + ks * P::kKStepBytes, P::kSbo, P::kLayoutType);
@@ -265,7 +294,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     }
                 }
                 tc_commit(&bar_empty[stage]);       // operands consumed: the stage may be refilled
-                tc_commit(&bar_acc_full[acc]);
+                tc_commit(&bar_acc_full[buf]);
             }
             __syncwarp();
         }
@@ -278,98 +307,109 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         Acc* rowpre = reinterpret_cast<Acc*>(smem + Cfg::kRowpreOffset) + warp * PIECE_ROWS;
         const int sh = prm.off_shift;
         const long long nq = prm.nseg + 1;
-        // inclusive prefix inside the piece at element offset j (0..1023); j = -1 gives 0
+        bool failed = false;
+        // inclusive prefix inside the piece at element offset j (0..1023)
         auto piece_prefix = [&](int j, Acc& rowpart, int& row) -> Acc {
             row = j >> 5;
             const int pos = j & 31;
             rowpart = *reinterpret_cast<const Acc*>(dump + row * 128 + ((((pos >> 2) ^ (row & 7)) << 4) | ((pos & 3) << 2)));
             return P::add(rowpre[row], rowpart);
         };
-        for (int it = g;; it += 2) {
-            const int stage = it % S;
-            if (!wait_bar(&bar_full[stage], (it / S) & 1, abort_flag, budget)) {
-                *abort_flag = 1;
-                if (lane == 0) report_error(prm.hdr, 5u);
-                break;
-            }
-            const int tile = tile_slot[stage];
+        for (int k = 0;; ++k) {
+            const int it = g + 2 * k;
+            // the epilogue never reads the operand stage (the MMA warp releases it); with the static
+            // tile order it knows its tile without being told
+            int tile = static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
+            if (tile >= prm.num_tiles) tile = -1;
             if (tile < 0) break;
-            if (!wait_bar(&bar_acc_full[g], (it >> 1) & 1, abort_flag, budget)) {
-                *abort_flag = 1;
-                if (lane == 0) report_error(prm.hdr, 5u);
-                break;
-            }
-            tc_fence_after_sync();
-
+            const int buf = g * 2 + (k & 1);
             const long long s = static_cast<long long>(tile) * SPANS_PER_TILE + w;
             const long long sbase = s * SPAN;
-            const uint32_t taddr = tmem_base + g * (PIECES_PER_SPAN * ROW) + ((static_cast<uint32_t>(w) * 32u) << 16);
+            const long long send = sbase + SPAN;
+            const uint32_t taddr = tmem_base + buf * (PIECES_PER_SPAN * ROW) + ((static_cast<uint32_t>(w) * 32u) << 16);
 
-            // first boundary index of this span: first q in the tile's range with bnd(q) >= sbase
-            long long q;
+            // ---- the span's boundaries: one offset per lane, requested before the products are awaited ----
+            long long q = prm.span_q[s];                       // first q with bnd(q) >= sbase
+            const long long cq = q;                            // index held by lane 0 of the cache
+            long long cb = -1, csb = -1;                       // cached boundary and its predecessor
             {
-                long long lo = prm.tile_q[tile], hi = prm.tile_q[tile + 1];
-                while (hi > lo) {
-                    const long long len = hi - lo, step = (len + 31) / 32;
-                    const long long bstart = lo + lane * step;
-                    long long bend = bstart + step;
-                    if (bend > hi) bend = hi;
-                    bool pred = false;
-                    if (bstart < hi) pred = (static_cast<long long>(prm.off[bend - 1]) << sh) >= sbase;
-                    const unsigned m = __ballot_sync(0xffffffffu, pred);
-                    if (m == 0u) {
-                        lo = hi;
-                    } else {
-                        const int k = __ffs(m) - 1;
-                        const long long ks = lo + k * step;
-                        long long ke = ks + step;
-                        if (ke > hi) ke = hi;
-                        lo = ks;
-                        hi = ke - 1;
-                    }
-                }
-                q = lo;
+                const long long qi = q + lane;
+                if (qi < nq) cb = static_cast<long long>(prm.off[qi]) << sh;
+                if (qi >= 1 && qi < nq) csb = static_cast<long long>(prm.off[qi - 1]) << sh;
             }
+            // the cache covers the span if it reaches past the span's end (or the end of the offsets)
+            const bool covers = __any_sync(0xffffffffu, (q + lane >= nq) || (cb > send));
+
+            if (!wait_bar(&bar_acc_full[buf], (k >> 1) & 1, abort_flag, budget)) { failed = true; break; }
+            tc_fence_after_sync();
+
+            // row totals of the four pieces
+            Acc tot[PIECES_PER_SPAN];
+#pragma unroll
+            for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * ROW + (ROW - 1)));
+            tmem_ld_wait();
 
             Acc run = Acc(0);              // sum of the open segment inside this span so far
             bool seen = false;             // a segment start lies inside this span
             long long def_r = -1;          // segment that began before the span and ends inside it
             Acc def_val = Acc(0);
-            uint32_t r[32];
 #pragma unroll 1
             for (int i = 0; i < PIECES_PER_SPAN; ++i) {
                 const long long pbase = sbase + i * PIECE;
+                const long long pend = pbase + PIECE;
+                Acc toti = tot[0];
+#pragma unroll
+                for (int t = 1; t < PIECES_PER_SPAN; ++t)
+                    if (i == t) toti = tot[t];
+                // any boundary with pbase <= bnd <= pend (END in (pbase, pend], START in [pbase, pend))?
+                bool touched = true;
+                if (covers) {
+                    const long long qi = cq + lane;
+                    touched = __any_sync(0xffffffffu, (qi >= q) && (qi < nq) && (cb >= pbase) && (cb <= pend));
+                }
+                if (!touched) {
+                    run = P::add(run, warp_sum<P>(toti));
+                    continue;
+                }
+
+                // ---- prefixes of the piece -> shared memory, exclusive scan of the 32 row totals ----
+                uint32_t r[32];
                 tmem_ld_32x32(taddr + i * ROW, r);
                 tmem_ld_wait();
-                // row prefixes -> shared memory (16-byte chunks rotated by the row to avoid bank conflicts)
 #pragma unroll
                 for (int c4 = 0; c4 < 8; ++c4)
                     *reinterpret_cast<uint4*>(dump + lane * 128 + ((c4 ^ (lane & 7)) << 4)) =
                         make_uint4(r[4 * c4], r[4 * c4 + 1], r[4 * c4 + 2], r[4 * c4 + 3]);
-                // exclusive scan of the 32 row totals
-                const Acc tot = P::from_bits(r[31]);
-                Acc inc = tot;
+                Acc inc = toti;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
                     const Acc t = __shfl_up_sync(0xffffffffu, inc, o);
                     if (static_cast<int>(lane) >= o) inc = P::add(t, inc);
                 }
-                rowpre[lane] = P::sub(inc, tot);
+                rowpre[lane] = P::sub(inc, toti);
                 const Acc piece_total = __shfl_sync(0xffffffffu, inc, 31);
                 __syncwarp();
 
-                // boundaries with pbase <= bnd(q) <= pbase + PIECE, 32 at a time (sorted, so the
-                // ones of this piece are a prefix of every batch)
-                const long long pend = pbase + PIECE;
+                // ---- boundaries with pbase <= bnd(q) <= pend, 32 at a time (sorted: a prefix of every batch) ----
                 bool piece_has_start = false;
                 long long last_start = -1;
                 long long qp = q;              // batch pointer
                 int advance = 0;               // boundaries strictly before pend: consumed for good
                 while (true) {
                     const long long qi = qp + lane;
-                    long long b = -1;
-                    if (qi < nq) b = static_cast<long long>(prm.off[qi]) << sh;
-                    const bool in_piece = (qi < nq) && (b <= pend);
+                    long long b = -1, sb = -1;
+                    if (covers && qp == q) {
+                        // the batch is the cache shifted by (q - cq) lanes; lanes shifted in from beyond the
+                        // cache lie past the span's end by construction
+                        const int d = static_cast<int>(q - cq);
+                        b = __shfl_down_sync(0xffffffffu, cb, d);
+                        sb = __shfl_down_sync(0xffffffffu, csb, d);
+                        if (static_cast<int>(lane) + d >= 32) { b = send + 1; sb = send + 1; }
+                    } else {
+                        if (qi < nq) b = static_cast<long long>(prm.off[qi]) << sh;
+                        if (qi >= 1 && qi < nq) sb = static_cast<long long>(prm.off[qi - 1]) << sh;
+                    }
+                    const bool in_piece = (qi < nq) && (b >= 0) && (b <= pend);
                     const unsigned inm = __ballot_sync(0xffffffffu, in_piece);
                     const int cnt = (inm == 0xffffffffu) ? 32 : (__ffs(~inm) - 1);
                     const bool mine = static_cast<int>(lane) < cnt;
@@ -377,24 +417,28 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     Acc val = Acc(0);
                     // as the END of segment qi-1: bnd in (pbase, pend], or 0 for leading empty segments
                     if (mine && qi >= 1 && (b > pbase || (pbase == 0 && b == 0))) {
-                        const long long sb = static_cast<long long>(prm.off[qi - 1]) << sh;
                         if (sb > b || sb < 0 || b > prm.n) {
                             report_error(prm.hdr, 4u);
                         } else {
                             if (b != sb) {
-                                Acc ep, sp = Acc(0);
-                                int erow, srow;
-                                const Acc e_full = piece_prefix(static_cast<int>(b - 1 - pbase), ep, erow);
-                                if (sb >= pbase) {
-                                    Acc s_full = Acc(0);
-                                    if (sb > pbase) s_full = piece_prefix(static_cast<int>(sb - 1 - pbase), sp, srow);
-                                    if (static_cast<int>((sb - pbase) >> 5) == erow)
-                                        val = ((sb - pbase) & 31) ? P::sub(ep, sp) : ep;   // inside one row
-                                    else
-                                        val = P::sub(e_full, s_full);
+                                if (b - sb <= SUM_DIRECT_LEN) {
+                                    // a very short segment: add the input values themselves
+                                    for (long long e = sb; e < b; ++e) val = P::add(val, load_value<P>(xg, e));
                                 } else {
-                                    val = P::add(run, e_full);
-                                    deferred = sb < sbase;
+                                    Acc ep, sp = Acc(0);
+                                    int erow, srow;
+                                    const Acc e_full = piece_prefix(static_cast<int>(b - 1 - pbase), ep, erow);
+                                    if (sb >= pbase) {
+                                        Acc s_full = Acc(0);
+                                        if (sb > pbase) s_full = piece_prefix(static_cast<int>(sb - 1 - pbase), sp, srow);
+                                        if (static_cast<int>((sb - pbase) >> 5) == erow)
+                                            val = ((sb - pbase) & 31) ? P::sub(ep, sp) : ep;   // inside one row
+                                        else
+                                            val = P::sub(e_full, s_full);
+                                    } else {
+                                        val = P::add(run, e_full);
+                                        deferred = sb < sbase;
+                                    }
                                 }
                             }
                             if (!deferred) outp[qi - 1] = val;
@@ -431,7 +475,10 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 __syncwarp();
             }
 
-            // ---- publish, look back, emit the segment that began before this span ----
+            // ---- the TMEM buffer is free; publish, look back, emit the segment that began before this span ----
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
             if (s == 0) {
                 if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(run)));
                 if (def_r >= 0 && lane == 0) outp[def_r] = def_val;
@@ -441,11 +488,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (!seen || def_r >= 0) {
                     LookbackWindow lbw;
                     if (!lookback<P>(prm.status, s, carry, abort_flag, budget, lbw, false)) {
-                        *abort_flag = 1;
-                        if (lane == 0) {
-                            report_error(prm.hdr, 5u);
-                            st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
-                        }
+                        if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
+                        failed = true;
                         break;
                     }
                     if (!seen && lane == 0)
@@ -453,10 +497,10 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     if (def_r >= 0 && lane == 0) outp[def_r] = P::add(carry, def_val);
                 }
             }
-
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar_acc_empty[g]);
+        }
+        if (failed) {
+            *abort_flag = 1;
+            if (lane == 0) report_error(prm.hdr, 5u);
         }
     }
 
