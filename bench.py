@@ -39,9 +39,12 @@ UNIT = "Gelem/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# DRAM bytes per element of the headline kernel measured with ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum of one launch divided by its n); see profiles/.  None = not captured yet.
-NCU_TRAFFIC_BYTES_PER_ELEM = None
+# DRAM traffic of the headline kernel from the ncu capture of its n = 2^26 case
+# (profiles/seg_scan_kernel_f16_n2p26_p1e-3.md): reads 3.002 B/element, writes 4 B/element minus
+# the ~57 MB of output that are still in L2 when a launch ends; both scale with n.
+NCU_READ_BYTES_PER_ELEM = 3.002
+NCU_WRITE_BYTES_PER_ELEM = 4.0
+NCU_WRITE_L2_RESIDUE_BYTES = 56.6e6
 
 
 def parse_args():
@@ -349,6 +352,17 @@ def run_ours(args):
         e1.record()
         barrier()
     launches = mmv.kernel_launch_count() - launches0
+    # context: a plain fp16 -> fp32 conversion copy (2 B read + 4 B written per element, no arithmetic)
+    for _ in range(2):
+        od.copy_(xd)
+    torch.cuda.synchronize()
+    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    c0.record()
+    for _ in range(5):
+        od.copy_(xd)
+    c1.record()
+    c1.synchronize()
+    conv_copy_gbs = 6 * n / (c0.elapsed_time(c1) / 5) / 1e6
     ms = e0.elapsed_time(e1) / args.steps
     if mmv.last_async_status(ws) != 0:
         raise SystemExit("bench: device-side error status")
@@ -392,8 +406,10 @@ def run_ours(args):
                          "frac": achieved / peak, "peak_kind": peak_kind,
                          "frac_of_8tbs_nominal": achieved / NOMINAL_HBM_GBS,
                          "algorithmic_bytes_per_elem": 7,
-                         "traffic": None if NCU_TRAFFIC_BYTES_PER_ELEM is None else NCU_TRAFFIC_BYTES_PER_ELEM * n},
+                         "traffic": (NCU_READ_BYTES_PER_ELEM + NCU_WRITE_BYTES_PER_ELEM) * n - NCU_WRITE_L2_RESIDUE_BYTES,
+                         "traffic_source": "ncu capture at n=2^26 scaled by n (profiles/seg_scan_kernel_f16_n2p26_p1e-3.md)"},
             "worst_err_over_bound": worst,
+            "context_conversion_copy_gb_s": conv_copy_gbs,
         }
         del xh, fh, oh
         if not args.no_cpu:
