@@ -352,6 +352,10 @@ def run_ours(args):
         e1.record()
         barrier()
     launches = mmv.kernel_launch_count() - launches0
+    ms = e0.elapsed_time(e1) / args.steps
+    if mmv.last_async_status(ws) != 0:
+        raise SystemExit("bench: device-side error status")
+    worst = verify_scan_sample(torch, mmv, oracle, x, f, od, ws)
     # context: a plain fp16 -> fp32 conversion copy (2 B read + 4 B written per element, no arithmetic)
     for _ in range(2):
         od.copy_(xd)
@@ -363,10 +367,6 @@ def run_ours(args):
     c1.record()
     c1.synchronize()
     conv_copy_gbs = 6 * n / (c0.elapsed_time(c1) / 5) / 1e6
-    ms = e0.elapsed_time(e1) / args.steps
-    if mmv.last_async_status(ws) != 0:
-        raise SystemExit("bench: device-side error status")
-    worst = verify_scan_sample(torch, mmv, oracle, x, f, od, ws)
 
     # end to end: pinned host -> device, the call, device -> host, every step
     e2e_steps = max(1, min(args.steps, 5))
