@@ -315,12 +315,29 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             rowpart = *reinterpret_cast<const Acc*>(dump + row * 128 + ((((pos >> 2) ^ (row & 7)) << 4) | ((pos & 3) << 2)));
             return P::add(rowpre[row], rowpart);
         };
+        // The boundaries of the NEXT tile's span are requested one tile ahead (first the span's first
+        // offset index, then one offset per lane), so that their two dependent round trips never
+        // sit on the critical path.
+        auto tile_of = [&](int kk) -> int {
+            const int t = static_cast<int>(blockIdx.x) + (g + 2 * kk) * static_cast<int>(gridDim.x);
+            return t < prm.num_tiles ? t : -1;
+        };
+        auto load_offsets = [&](long long q0, long long& b, long long& sb) {
+            const long long qi = q0 + lane;
+            b = -1;
+            sb = -1;
+            if (qi < nq) b = static_cast<long long>(prm.off[qi]) << sh;
+            if (qi >= 1 && qi < nq) sb = static_cast<long long>(prm.off[qi - 1]) << sh;
+        };
+        long long q_next = 0, nb = -1, nsb = -1;
+        if (tile_of(0) >= 0) {
+            q_next = prm.span_q[static_cast<long long>(tile_of(0)) * SPANS_PER_TILE + w];
+            load_offsets(q_next, nb, nsb);
+        }
         for (int k = 0;; ++k) {
-            const int it = g + 2 * k;
             // the epilogue never reads the operand stage (the MMA warp releases it); with the static
             // tile order it knows its tile without being told
-            int tile = static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
-            if (tile >= prm.num_tiles) tile = -1;
+            const int tile = tile_of(k);
             if (tile < 0) break;
             const int buf = g * 2 + (k & 1);
             const long long s = static_cast<long long>(tile) * SPANS_PER_TILE + w;
@@ -328,15 +345,12 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             const long long send = sbase + SPAN;
             const uint32_t taddr = tmem_base + buf * (PIECES_PER_SPAN * ROW) + ((static_cast<uint32_t>(w) * 32u) << 16);
 
-            // ---- the span's boundaries: one offset per lane, requested before the products are awaited ----
-            long long q = prm.span_q[s];                       // first q with bnd(q) >= sbase
+            // ---- the span's boundaries: one offset per lane (requested during the previous tile) ----
+            long long q = q_next;                              // first q with bnd(q) >= sbase
             const long long cq = q;                            // index held by lane 0 of the cache
-            long long cb = -1, csb = -1;                       // cached boundary and its predecessor
-            {
-                const long long qi = q + lane;
-                if (qi < nq) cb = static_cast<long long>(prm.off[qi]) << sh;
-                if (qi >= 1 && qi < nq) csb = static_cast<long long>(prm.off[qi - 1]) << sh;
-            }
+            const long long cb = nb, csb = nsb;                // cached boundary and its predecessor
+            const int tile_n = tile_of(k + 1);
+            if (tile_n >= 0) q_next = prm.span_q[static_cast<long long>(tile_n) * SPANS_PER_TILE + w];
             // the cache covers the span if it reaches past the span's end (or the end of the offsets)
             const bool covers = __any_sync(0xffffffffu, (q + lane >= nq) || (cb > send));
 
@@ -348,6 +362,41 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
 #pragma unroll
             for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * ROW + (ROW - 1)));
             tmem_ld_wait();
+
+            // ---- pre-pass (all boundaries in registers): the span's aggregate from the row totals and one
+            //      prefix, published before the boundaries are worked through ----
+            LookbackWindow lbw;
+            bool published = false;
+            if (covers) {
+                const bool isstart = (cq + lane < nq) && (cb >= sbase) && (cb < send);
+                const int rel = isstart ? static_cast<int>(cb - sbase) : -1;
+                const int lastrel = __reduce_max_sync(0xffffffffu, rel);     // last segment start inside the span
+                Acc tail;
+                if (lastrel < 0) {
+                    tail = warp_sum<P>(P::add(P::add(tot[0], tot[1]), P::add(tot[2], tot[3])));
+                } else {
+                    const int il = lastrel >> 10, rl = (lastrel >> 5) & 31, pos = lastrel & 31;
+                    Acc after = Acc(0), totl = tot[0];
+#pragma unroll
+                    for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                        if (i > il) after = P::add(after, tot[i]);
+                        if (i == il) totl = tot[i];
+                    }
+                    if (static_cast<int>(lane) > rl) after = P::add(after, totl);
+                    after = warp_sum<P>(after);
+                    Acc before = Acc(0);
+                    if (pos > 0) {
+                        before = P::from_bits(tmem_ld_32x1(taddr + il * ROW + (pos - 1)));
+                        tmem_ld_wait();
+                    }
+                    tail = P::add(__shfl_sync(0xffffffffu, P::sub(totl, before), rl), after);
+                }
+                if (lane == 0)
+                    st_relaxed_gpu_u64(prm.status + s,
+                                       pack_status((lastrel >= 0 || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail)));
+                published = true;
+                if (s != 0) lookback_load(prm.status, s - 1, lbw);     // travels while the boundaries are processed
+            }
 
             Acc run = Acc(0);              // sum of the open segment inside this span so far
             bool seen = false;             // a segment start lies inside this span
@@ -479,23 +528,22 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
+            // request the next tile's offsets (its first index has arrived by now)
+            if (tile_n >= 0) load_offsets(q_next, nb, nsb);
+            if (!published && lane == 0)
+                st_relaxed_gpu_u64(prm.status + s, pack_status((seen || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(run)));
             if (s == 0) {
-                if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(run)));
                 if (def_r >= 0 && lane == 0) outp[def_r] = def_val;
-            } else {
-                if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(seen ? ST_PREFIX : ST_AGG, P::to_bits(run)));
+            } else if (!seen || def_r >= 0) {
                 Acc carry = Acc(0);
-                if (!seen || def_r >= 0) {
-                    LookbackWindow lbw;
-                    if (!lookback<P>(prm.status, s, carry, abort_flag, budget, lbw, false)) {
-                        if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
-                        failed = true;
-                        break;
-                    }
-                    if (!seen && lane == 0)
-                        st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(carry, run))));
-                    if (def_r >= 0 && lane == 0) outp[def_r] = P::add(carry, def_val);
+                if (!lookback<P>(prm.status, s, carry, abort_flag, budget, lbw, published)) {
+                    if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
+                    failed = true;
+                    break;
                 }
+                if (!seen && lane == 0)
+                    st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(carry, run))));
+                if (def_r >= 0 && lane == 0) outp[def_r] = P::add(carry, def_val);
             }
         }
         if (failed) {
