@@ -133,32 +133,32 @@ __device__ __forceinline__ typename P::Acc warp_sum(typename P::Acc v) {
 // Span s publishes either its aggregate (ST_AGG: sum of all its elements, it holds no segment
 // start) or an inclusive prefix (ST_PREFIX: sum of the segment that is open at its end).  The
 // carry into span s is the sum of the aggregates of s-1, s-2, ... down to and including the
-// first span that published a prefix.  A window is LB_WINDOW consecutive predecessors, LB_WORDS
-// per lane, nearest first: lane l holds positions LB_WORDS*l .. LB_WORDS*l + LB_WORDS-1.
+// first one that published a prefix.  A window is 32 * W consecutive predecessors, W per lane,
+// nearest first: lane l holds positions W*l .. W*l + W-1.
 // ---------------------------------------------------------------------------
-constexpr int LB_WORDS = 1;
-constexpr int LB_WINDOW = 32 * LB_WORDS;
-
+// W = words per lane: a window is 32 * W consecutive predecessors.
+template <int W>
 struct LookbackWindow {
-    uint64_t w[LB_WORDS];
+    uint64_t w[W];
 };
 
 // Issues the loads of the window whose nearest predecessor is `idx` (no wait on the data).
-__device__ __forceinline__ void lookback_load(const uint64_t* status, long long idx, LookbackWindow& win) {
-    const long long first = idx - static_cast<long long>(LB_WORDS) * lane_id();
+template <int W>
+__device__ __forceinline__ void lookback_load(const uint64_t* status, long long idx, LookbackWindow<W>& win) {
+    const long long first = idx - static_cast<long long>(W) * lane_id();
 #pragma unroll
-    for (int q = 0; q < LB_WORDS; ++q) {
+    for (int q = 0; q < W; ++q) {
         const long long my = first - q;
-        win.w[q] = (my >= 0) ? ld_relaxed_gpu_u64(status + my) : pack_status(ST_PREFIX, 0u);   // nothing before span 0
+        win.w[q] = (my >= 0) ? ld_relaxed_gpu_u64(status + my) : pack_status(ST_PREFIX, 0u);   // nothing before word 0
     }
 }
 
-// Returns the carry into span s.  `win` may hold a window loaded earlier with lookback_load
+// Returns the carry into position s.  `win` may hold a window loaded earlier with lookback_load
 // (preloaded = true) so that the first round trip overlaps the caller's work.  Bounded: returns
 // false on time-out, when another role of the CTA aborted, or when a predecessor aborted.
-template <typename P>
+template <typename P, int W>
 __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, typename P::Acc& carry,
-                                         volatile int* abort_flag, uint64_t budget_ns, LookbackWindow& win,
+                                         volatile int* abort_flag, uint64_t budget_ns, LookbackWindow<W>& win,
                                          bool preloaded) {
     using Acc = typename P::Acc;
     const uint32_t lane = lane_id();
@@ -166,11 +166,11 @@ __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, ty
     long long idx = s - 1;
     uint64_t t0 = global_timer_ns();
     uint32_t polls = 0;
-    if (!preloaded) lookback_load(status, idx, win);
+    if (!preloaded) lookback_load<W>(status, idx, win);
     while (true) {
         uint32_t tmask = 0u, rmask = 0u, xmask = 0u;
 #pragma unroll
-        for (int q = 0; q < LB_WORDS; ++q) {
+        for (int q = 0; q < W; ++q) {
             const uint32_t st = static_cast<uint32_t>(win.w[q] >> 32);
             rmask |= (st != ST_NONE) ? (1u << q) : 0u;
             tmask |= (st == ST_PREFIX || st == ST_ABORT) ? (1u << q) : 0u;
@@ -178,16 +178,16 @@ __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, ty
         }
         const uint32_t lanes_t = __ballot_sync(0xffffffffu, tmask != 0u);
         const int L = lanes_t ? (__ffs(lanes_t) - 1) : 32;            // first lane that holds a terminal word
-        const int qt = tmask ? (__ffs(tmask) - 1) : LB_WORDS;         // this lane's first terminal word
+        const int qt = tmask ? (__ffs(tmask) - 1) : W;                // this lane's first terminal word
         // words this lane must contribute: all of them before lane L, up to its terminal in lane L
-        const int need = (static_cast<int>(lane) < L) ? LB_WORDS : ((static_cast<int>(lane) == L) ? qt + 1 : 0);
+        const int need = (static_cast<int>(lane) < L) ? W : ((static_cast<int>(lane) == L) ? qt + 1 : 0);
         const uint32_t need_mask = (1u << need) - 1u;
         const bool lane_ready = (rmask & need_mask) == need_mask;
         if (__all_sync(0xffffffffu, lane_ready)) {
             if (__any_sync(0xffffffffu, (xmask & need_mask) != 0u)) return false;
             Acc v = Acc(0);
 #pragma unroll
-            for (int q = LB_WORDS - 1; q >= 0; --q)
+            for (int q = W - 1; q >= 0; --q)
                 if (q < need) v = P::add(P::from_bits(static_cast<uint32_t>(win.w[q])), v);
             v = warp_sum<P>(v);
             acc = P::add(v, acc);
@@ -195,13 +195,16 @@ __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, ty
                 carry = acc;
                 return true;
             }
-            idx -= LB_WINDOW;
+            idx -= 32 * W;
             t0 = global_timer_ns();
-        } else if ((++polls & 7u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > budget_ns) return false;
+        } else {
+            if ((++polls & 7u) == 0u) {
+                if (*abort_flag) return false;
+                if (global_timer_ns() - t0 > budget_ns) return false;
+            }
+            __nanosleep(40);        // keep the polling traffic in L2 small
         }
-        lookback_load(status, idx, win);
+        lookback_load<W>(status, idx, win);
     }
 }
 

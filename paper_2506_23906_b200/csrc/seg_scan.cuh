@@ -70,6 +70,7 @@ constexpr int SCAN_EPI_WARPS = 4 * SCAN_GROUPS;             // 8
 constexpr int SCAN_PRODUCER_WARP = SCAN_EPI_WARPS;
 constexpr int SCAN_MMA_WARP = SCAN_EPI_WARPS + 1;
 constexpr int SCAN_THREADS = (SCAN_EPI_WARPS + 2) * 32;     // 320
+constexpr int SCAN_LB_WORDS = 1;                            // look-back window: 128 tiles per poll
 
 template <typename P>
 struct ScanCfg {
@@ -143,7 +144,11 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     uint64_t* bar_empty = bar_full + S;
     uint64_t* bar_acc_full = bar_empty + S;                // per TMEM buffer: the tile's products are in it
     uint64_t* bar_acc_empty = bar_acc_full + SCAN_BUFS;    // per TMEM buffer: the four warps are done with it
-    int* tile_slot = reinterpret_cast<int*>(bar_acc_empty + SCAN_BUFS);
+    uint64_t* bar_agg = bar_acc_empty + SCAN_BUFS;          // per warpgroup: its four unit aggregates are in agg_slot
+    uint64_t* bar_carry = bar_agg + SCAN_GROUPS;           // per warpgroup: the tile's carry is in carry_slot
+    uint64_t* agg_slot = bar_carry + SCAN_GROUPS;          // [group][unit]: (flag << 32) | payload
+    uint32_t* carry_slot = reinterpret_cast<uint32_t*>(agg_slot + SCAN_GROUPS * SPANS_PER_TILE);   // [group]
+    int* tile_slot = reinterpret_cast<int*>(carry_slot + SCAN_GROUPS);
     volatile int* stage_iter = tile_slot + S;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_slot + 2 * S);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -157,6 +162,10 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             mbar_init(&bar_full[i], 1);
             mbar_init(&bar_empty[i], 4);      // the group's four warps, once their flag bytes are read
             stage_iter[i] = -1;
+        }
+        for (int i = 0; i < SCAN_GROUPS; ++i) {
+            mbar_init(&bar_agg[i], SPANS_PER_TILE);
+            mbar_init(&bar_carry[i], 1);
         }
         for (int i = 0; i < SCAN_BUFS; ++i) {
             mbar_init(&bar_acc_full[i], 1);
@@ -447,21 +456,42 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 }
                 tail_unit = P::add(__shfl_sync(0xffffffffu, row_tail, lstar), after);
             }
-            const bool skip_publish = (s == prm.debug_skip_span);
-            if (lane == 0 && !skip_publish)
-                st_relaxed_gpu_u64(prm.status + s,
-                                   pack_status((flagged || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail_unit)));
+            // ---- the four units of the tile exchange their aggregates through shared memory; the carry
+            //      chain between CTAs runs over one status word per TILE, published by the first warp ----
+            if (lane == 0) {
+                agg_slot[g * SPANS_PER_TILE + w] = (static_cast<uint64_t>(flagged ? 1u : 0u) << 32) | P::to_bits(tail_unit);
+                mbar_arrive(&bar_agg[g]);
+            }
+            if (!wait_bar(&bar_agg[g], k & 1, abort_flag, budget)) { failed = true; break; }
+            Acc ex = Acc(0);                  // open-segment sum of the tile's units before this one
+            bool exflag = false;              // ... and whether one of them holds a flag
+            Acc tail_tile = Acc(0);
+            bool flag_tile = false;
+#pragma unroll
+            for (int j = 0; j < SPANS_PER_TILE; ++j) {
+                const uint64_t a = agg_slot[g * SPANS_PER_TILE + j];
+                const bool fj = (a >> 32) != 0u;
+                const Acc tj = P::from_bits(static_cast<uint32_t>(a));
+                if (j == w) { ex = tail_tile; exflag = flag_tile; }
+                tail_tile = fj ? tj : P::add(tail_tile, tj);
+                flag_tile = flag_tile || fj;
+            }
+            const bool need_global = !exflag && tile != 0;      // the carry reaches back past the tile
+            const bool skip_publish = (prm.debug_skip_span >= 0) && ((prm.debug_skip_span >> 2) == tile);
+            if (w == 0 && lane == 0 && !skip_publish)
+                st_relaxed_gpu_u64(prm.status + tile,
+                                   pack_status((flag_tile || tile == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail_tile)));
             MMV_T_MARK(3)
 
             // ---- main pass: everything that does not need the carry of earlier units ----
             const long long row0 = s * (SCAN_UNIT / ROW);
             Acc run = Acc(0);                 // sum of the open segment inside this unit so far
             uint32_t fm0 = 0u, pm0 = 0u;      // masks of the first flagged piece
-            LookbackWindow lbw;
+            LookbackWindow<SCAN_LB_WORDS> lbw;
 #pragma unroll
             for (int i = 0; i < UP; ++i) {
                 // the first look-back window travels while the last piece is processed
-                if (i == UP - 1) lookback_load(prm.status, s - 1, lbw);
+                if (i == UP - 1 && need_global && w == 0) lookback_load<SCAN_LB_WORDS>(prm.status, tile - 1, lbw);
                 const uint32_t fmi = fm[i];
                 const uint32_t pmi = pm[i];
                 const Acc toti = tot[i];
@@ -543,15 +573,29 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             tmem_st_wait();
 
             // ---- look back (most of its latency has been covered by the main pass) ----
-            Acc carry = Acc(0);
-            if (s != 0) {
-                if (!lookback<P>(prm.status, s, carry, abort_flag, budget, lbw, true)) {
-                    if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
-                    failed = true;
-                    break;
+            // Only the tile's first warp polls the other CTAs' status words; it hands the tile's carry to
+            // its siblings through shared memory (they have passed bar_agg of this tile, so the previous
+            // phase of bar_carry is complete and the parity wait cannot alias).
+            Acc carry = ex;
+            if (w == 0) {
+                Acc carry_tile = Acc(0);
+                if (tile != 0) {
+                    if (!lookback<P, SCAN_LB_WORDS>(prm.status, tile, carry_tile, abort_flag, budget, lbw, true)) {
+                        if (lane == 0) st_relaxed_gpu_u64(prm.status + tile, pack_status(ST_ABORT, 0u));
+                        failed = true;
+                        break;
+                    }
+                    if (!flag_tile && lane == 0 && !skip_publish)
+                        st_relaxed_gpu_u64(prm.status + tile, pack_status(ST_PREFIX, P::to_bits(P::add(carry_tile, tail_tile))));
                 }
-                if (!flagged && lane == 0 && !skip_publish)
-                    st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(carry, tail_unit))));
+                if (lane == 0) {
+                    carry_slot[g] = P::to_bits(carry_tile);
+                    mbar_arrive(&bar_carry[g]);
+                }
+                carry = carry_tile;
+            } else if (need_global) {
+                if (!wait_bar(&bar_carry[g], k & 1, abort_flag, budget)) { failed = true; break; }
+                carry = P::add(P::from_bits(carry_slot[g]), ex);
             }
 
             // ---- parked pieces: add the carry in front of the unit's first flag, store ----

@@ -365,7 +365,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
 
             // ---- pre-pass (all boundaries in registers): the span's aggregate from the row totals and one
             //      prefix, published before the boundaries are worked through ----
-            LookbackWindow lbw;
+            LookbackWindow<1> lbw;
             bool published = false;
             if (covers) {
                 const bool isstart = (cq + lane < nq) && (cb >= sbase) && (cb < send);
@@ -395,7 +395,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     st_relaxed_gpu_u64(prm.status + s,
                                        pack_status((lastrel >= 0 || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail)));
                 published = true;
-                if (s != 0) lookback_load(prm.status, s - 1, lbw);     // travels while the boundaries are processed
+                if (s != 0) lookback_load<1>(prm.status, s - 1, lbw);     // travels while the boundaries are processed
             }
 
             Acc run = Acc(0);              // sum of the open segment inside this span so far
@@ -536,7 +536,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (def_r >= 0 && lane == 0) outp[def_r] = def_val;
             } else if (!seen || def_r >= 0) {
                 Acc carry = Acc(0);
-                if (!lookback<P>(prm.status, s, carry, abort_flag, budget, lbw, published)) {
+                if (!lookback<P, 1>(prm.status, s, carry, abort_flag, budget, lbw, published)) {
                     if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
                     failed = true;
                     break;
