@@ -488,13 +488,16 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             Acc run = Acc(0);                 // sum of the open segment inside this unit so far
             uint32_t fm0 = 0u, pm0 = 0u;      // masks of the first flagged piece
             LookbackWindow<SCAN_LB_WORDS> lbw;
-#pragma unroll
+            // (not unrolled: the body is large and the instruction cache is the scarcer resource)
+#pragma unroll 1
             for (int i = 0; i < UP; ++i) {
                 // the first look-back window travels while the last piece is processed
                 if (i == UP - 1 && need_global && w == 0) lookback_load<SCAN_LB_WORDS>(prm.status, tile - 1, lbw);
-                const uint32_t fmi = fm[i];
-                const uint32_t pmi = pm[i];
-                const Acc toti = tot[i];
+                uint32_t fmi = fm[0], pmi = pm[0];
+                Acc toti = tot[0];
+#pragma unroll
+                for (int q = 1; q < UP; ++q)
+                    if (i == q) { fmi = fm[q]; pmi = pm[q]; toti = tot[q]; }
                 if (i == i0) { fm0 = fmi; pm0 = pmi; }
                 uint32_t r[32];
                 uint32_t raw[P::kIsFloat ? 32 : 1];
