@@ -187,6 +187,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         // nn < 32: 1 iff k <= nn (U_32);  nn >= 32 (fp16 only): 1 iff k == nn - 32 (identity).
         constexpr int kVecPerRow = P::kRowBytes / 16;
         constexpr int kElemPerVec = 16 / P::kElemBytes;
+#pragma unroll 1
         for (int v = threadIdx.x; v < N * kVecPerRow; v += SCAN_THREADS) {
             const int nn = v / kVecPerRow, cv = v % kVecPerRow;
             uint32_t words[4] = {0u, 0u, 0u, 0u};
@@ -246,6 +247,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             } else {
                 // ragged last tile: plain loads, zero fill past n (MATMUL zero-pads its operand)
                 const long long cnt = prm.n - tbase;
+#pragma unroll 1
                 for (int v = lane; v < SCAN_TILE / 16; v += 32) {
                     const int e0 = v * 16;
                     uint4 fv = make_uint4(0u, 0u, 0u, 0u);
@@ -253,6 +255,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                         fv = *reinterpret_cast<const uint4*>(prm.flags + tbase + e0);
                     } else if (e0 < cnt) {
                         __align__(16) uint8_t tmp[16];
+#pragma unroll 1
                         for (int e = 0; e < 16; ++e) tmp[e] = (e0 + e < cnt) ? prm.flags[tbase + e0 + e] : uint8_t(0);
                         fv = *reinterpret_cast<const uint4*>(tmp);
                     }
@@ -260,6 +263,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 }
                 constexpr int kElemPerVec = 16 / P::kElemBytes;
                 const uint8_t* xt = static_cast<const uint8_t*>(prm.x) + tbase * P::kElemBytes;
+#pragma unroll 1
                 for (int v = lane; v < SCAN_TILE / kElemPerVec; v += 32) {
                     const int e0 = v * kElemPerVec;
                     uint4 xv = make_uint4(0u, 0u, 0u, 0u);
@@ -267,6 +271,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                         xv = *reinterpret_cast<const uint4*>(xt + static_cast<size_t>(e0) * P::kElemBytes);
                     } else if (e0 < cnt) {
                         __align__(16) uint8_t tmp[16];
+#pragma unroll 1
                         for (int b = 0; b < 16; ++b)
                             tmp[b] = (e0 + b / P::kElemBytes < cnt) ? xt[static_cast<size_t>(e0) * P::kElemBytes + b] : uint8_t(0);
                         xv = *reinterpret_cast<const uint4*>(tmp);
@@ -357,16 +362,14 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 tma_store_2d(&tmap_out, ob, 0, static_cast<int>(prow));
                 tma_store_commit();
             }
-            // the one row that straddles n (n not a multiple of 32) is written with plain stores
+            // the one row that straddles n (n not a multiple of 32) is written with plain stores,
+            // read back from the staging buffer
             if (prow + lane == nrows_full) {
                 const int cnt = static_cast<int>(prm.n - nrows_full * ROW);
-                for (int j = 0; j < cnt; ++j) {
-                    uint32_t v = r[0];
-#pragma unroll
-                    for (int q = 1; q < 32; ++q)
-                        if (j == q) v = r[q];
-                    reinterpret_cast<uint32_t*>(outp)[nrows_full * ROW + j] = v;
-                }
+#pragma unroll 1
+                for (int j = 0; j < cnt; ++j)
+                    reinterpret_cast<uint32_t*>(outp)[nrows_full * ROW + j] =
+                        *reinterpret_cast<const uint32_t*>(ob + lane * 128 + ((((j >> 2) ^ (lane & 7)) << 4) | ((j & 3) << 2)));
             }
             obuf = (obuf + 1) % Cfg::kOutBufs;
         };
