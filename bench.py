@@ -374,17 +374,6 @@ def run_ours(args):
     if mmv.last_async_status(ws) != 0:
         raise SystemExit("bench: device-side error status")
     worst = verify_scan_sample(torch, mmv, oracle, x, f, od, ws)
-    # context: a plain fp16 -> fp32 conversion copy (2 B read + 4 B written per element, no arithmetic)
-    for _ in range(2):
-        od.copy_(xd)
-    torch.cuda.synchronize()
-    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    c0.record()
-    for _ in range(5):
-        od.copy_(xd)
-    c1.record()
-    c1.synchronize()
-    conv_copy_gbs = 6 * n / (c0.elapsed_time(c1) / 5) / 1e6
 
     # end to end: pinned host -> device, the call, device -> host, every step
     e2e_steps = max(1, min(args.steps, 5))
@@ -424,7 +413,6 @@ def run_ours(args):
                          "traffic": (NCU_READ_BYTES_PER_ELEM + NCU_WRITE_BYTES_PER_ELEM) * n - NCU_WRITE_L2_RESIDUE_BYTES,
                          "traffic_source": "ncu capture at n=2^26 scaled by n (profiles/seg_scan_kernel_f16_n2p26_p1e-3.md)"},
             "worst_err_over_bound": worst,
-            "context_conversion_copy_gb_s": conv_copy_gbs,
         }
         del xh, fh, oh
         if not args.no_cpu:
