@@ -6,6 +6,18 @@
 
 namespace mmv {
 
+// Optional phase timers (compile with -DMMV_PHASE_TIMERS): cycles summed over all epilogue warps.
+#ifdef MMV_PHASE_TIMERS
+__device__ unsigned long long g_phase_cycles[16];
+#define MMV_T_DECL long long t_prev = clock64(); unsigned long long t_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#define MMV_T_MARK(k) { const long long t_now = clock64(); t_acc[k] += static_cast<unsigned long long>(t_now - t_prev); t_prev = t_now; }
+#define MMV_T_FLUSH() { if (lane == 0) { for (int k = 0; k < 8; ++k) atomicAdd(&g_phase_cycles[k], t_acc[k]); } }
+#else
+#define MMV_T_DECL
+#define MMV_T_MARK(k)
+#define MMV_T_FLUSH()
+#endif
+
 // Geometry.  The value vector is viewed as rows of ROW consecutive elements (the paper's
 // ceil(n/s) x s matrix view of MATMUL(x, U_s), with s = ROW).  A warp owns a SPAN of 128
 // consecutive rows in four PIECES of 32 rows (one row per lane); a TILE is the four spans

@@ -33,18 +33,6 @@
 
 namespace mmv {
 
-// Optional phase timers (compile with -DMMV_PHASE_TIMERS): cycles summed over all epilogue warps.
-#ifdef MMV_PHASE_TIMERS
-__device__ unsigned long long g_phase_cycles[16];
-#define MMV_T_DECL long long t_prev = clock64(); unsigned long long t_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-#define MMV_T_MARK(k) { const long long t_now = clock64(); t_acc[k] += static_cast<unsigned long long>(t_now - t_prev); t_prev = t_now; }
-#define MMV_T_FLUSH() { if (lane == 0) { for (int k = 0; k < 8; ++k) atomicAdd(&g_phase_cycles[k], t_acc[k]); } }
-#else
-#define MMV_T_DECL
-#define MMV_T_MARK(k)
-#define MMV_T_FLUSH()
-#endif
-
 struct ScanParams {
     const void* x;
     const uint8_t* flags;
@@ -146,8 +134,10 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     uint64_t* bar_acc_empty = bar_acc_full + SCAN_BUFS;    // per TMEM buffer: the four warps are done with it
     uint64_t* bar_agg = bar_acc_empty + SCAN_BUFS;          // per warpgroup: its four unit aggregates are in agg_slot
     uint64_t* bar_carry = bar_agg + SCAN_GROUPS;           // per warpgroup: the tile's carry is in carry_slot
-    uint64_t* agg_slot = bar_carry + SCAN_GROUPS;          // [group][unit]: (flag << 32) | payload
-    uint32_t* carry_slot = reinterpret_cast<uint32_t*>(agg_slot + SCAN_GROUPS * SPANS_PER_TILE);   // [group]
+    // [group][tile parity][unit]: (flag << 32) | payload; two sets so that a warp's next-tile write
+    // can never meet a sibling's read of this tile's values
+    uint64_t* agg_slot = bar_carry + SCAN_GROUPS;
+    uint32_t* carry_slot = reinterpret_cast<uint32_t*>(agg_slot + SCAN_GROUPS * 2 * SPANS_PER_TILE);   // [group]
     int* tile_slot = reinterpret_cast<int*>(carry_slot + SCAN_GROUPS);
     volatile int* stage_iter = tile_slot + S;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_slot + 2 * S);
@@ -462,7 +452,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             // ---- the four units of the tile exchange their aggregates through shared memory; the carry
             //      chain between CTAs runs over one status word per TILE, published by the first warp ----
             if (lane == 0) {
-                agg_slot[g * SPANS_PER_TILE + w] = (static_cast<uint64_t>(flagged ? 1u : 0u) << 32) | P::to_bits(tail_unit);
+                agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + w] = (static_cast<uint64_t>(flagged ? 1u : 0u) << 32) | P::to_bits(tail_unit);
                 mbar_arrive(&bar_agg[g]);
             }
             if (!wait_bar(&bar_agg[g], k & 1, abort_flag, budget)) { failed = true; break; }
@@ -472,7 +462,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             bool flag_tile = false;
 #pragma unroll
             for (int j = 0; j < SPANS_PER_TILE; ++j) {
-                const uint64_t a = agg_slot[g * SPANS_PER_TILE + j];
+                const uint64_t a = agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + j];
                 const bool fj = (a >> 32) != 0u;
                 const Acc tj = P::from_bits(static_cast<uint32_t>(a));
                 if (j == w) { ex = tail_tile; exflag = flag_tile; }

@@ -34,6 +34,7 @@ constexpr int SUM_MMA_WARP = 9;
 constexpr int SUM_THREADS = 320;
 constexpr int SUM_BUFS = 4;                                        // TMEM tile buffers: two per warpgroup
 constexpr int SUM_TMEM_COLS = SUM_BUFS * PIECES_PER_SPAN * ROW;    // 512
+constexpr int SUM_SPARSE_MAX = 8;                                  // spans with at most this many boundaries read single prefixes from TMEM
 constexpr int SUM_DIRECT_LEN = 4;                                  // segments this short are summed from the inputs
 
 // bf16 values (the hi/lo halves of the fp32 products of SpMV): same geometry as fp16.
@@ -143,7 +144,11 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
     uint64_t* bar_acc_full = bar_empty + S;
     uint64_t* bar_acc_empty = bar_acc_full + SUM_BUFS;
     // per stage: (iteration << 32) | tile, written as one word before the stage's barrier is armed
-    volatile long long* stage_info = reinterpret_cast<volatile long long*>(bar_acc_empty + SUM_BUFS);
+    uint64_t* bar_agg = bar_acc_empty + SUM_BUFS;          // per warpgroup: its four span aggregates are in agg_slot
+    // [group][tile parity][span]: (has start << 32) | open-segment sum.  Two sets, because a warp may
+    // write its next tile's aggregate while a sibling still reads this tile's.
+    uint64_t* agg_slot = bar_agg + 2;
+    volatile long long* stage_info = reinterpret_cast<volatile long long*>(agg_slot + 2 * 2 * SPANS_PER_TILE);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<long long*>(stage_info) + S);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -157,6 +162,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             mbar_init(&bar_empty[i], 1);      // released by the MMA warp's commit
             stage_info[i] = -1;
         }
+        for (int i = 0; i < 2; ++i) mbar_init(&bar_agg[i], SPANS_PER_TILE);
         for (int i = 0; i < SUM_BUFS; ++i) {
             mbar_init(&bar_acc_full[i], 1);
             mbar_init(&bar_acc_empty[i], 4);
@@ -329,6 +335,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             if (qi < nq) b = static_cast<long long>(prm.off[qi]) << sh;
             if (qi >= 1 && qi < nq) sb = static_cast<long long>(prm.off[qi - 1]) << sh;
         };
+        MMV_T_DECL
         long long q_next = 0, nb = -1, nsb = -1;
         if (tile_of(0) >= 0) {
             q_next = prm.span_q[static_cast<long long>(tile_of(0)) * SPANS_PER_TILE + w];
@@ -354,8 +361,10 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             // the cache covers the span if it reaches past the span's end (or the end of the offsets)
             const bool covers = __any_sync(0xffffffffu, (q + lane >= nq) || (cb > send));
 
+            MMV_T_MARK(0)
             if (!wait_bar(&bar_acc_full[buf], (k >> 1) & 1, abort_flag, budget)) { failed = true; break; }
             tc_fence_after_sync();
+            MMV_T_MARK(1)
 
             // row totals of the four pieces
             Acc tot[PIECES_PER_SPAN];
@@ -367,10 +376,12 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             //      prefix, published before the boundaries are worked through ----
             LookbackWindow<1> lbw;
             bool published = false;
+            int lastrel = -1;
+            Acc tail_pre = Acc(0);
             if (covers) {
                 const bool isstart = (cq + lane < nq) && (cb >= sbase) && (cb < send);
                 const int rel = isstart ? static_cast<int>(cb - sbase) : -1;
-                const int lastrel = __reduce_max_sync(0xffffffffu, rel);     // last segment start inside the span
+                lastrel = __reduce_max_sync(0xffffffffu, rel);               // last segment start inside the span
                 Acc tail;
                 if (lastrel < 0) {
                     tail = warp_sum<P>(P::add(P::add(tot[0], tot[1]), P::add(tot[2], tot[3])));
@@ -395,15 +406,111 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     st_relaxed_gpu_u64(prm.status + s,
                                        pack_status((lastrel >= 0 || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail)));
                 published = true;
-                if (s != 0) lookback_load<1>(prm.status, s - 1, lbw);     // travels while the boundaries are processed
+                tail_pre = tail;
+                if (lane == 0) {
+                    agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + w] = (static_cast<uint64_t>(lastrel >= 0 ? 1u : 0u) << 32) | P::to_bits(tail);
+                    mbar_arrive(&bar_agg[g]);
+                }
+                // the first window beyond the tile travels while the boundaries are processed
+                if (tile != 0) lookback_load<1>(prm.status, s - w - 1, lbw);
             }
 
+            MMV_T_MARK(2)
             Acc run = Acc(0);              // sum of the open segment inside this span so far
             bool seen = false;             // a segment start lies inside this span
             long long def_r = -1;          // segment that began before the span and ends inside it
             Acc def_val = Acc(0);
+            // number of boundaries with sbase <= bnd <= send (a prefix of the cache lanes)
+            const int nb_span = __popc(__ballot_sync(0xffffffffu, (cq + lane < nq) && (cb >= 0) && (cb <= send)));
+            const bool sparse = covers && nb_span <= SUM_SPARSE_MAX;
+            if (sparse) {
+                // ---- few boundaries: no copy of the prefixes; the one prefix each boundary needs is read
+                //      straight from TMEM (one column, the lane of its row) ----
+                seen = lastrel >= 0;
+                run = tail_pre;               // the open segment's sum at the end of the span
+                uint32_t vv[SUM_SPARSE_MAX];
+#pragma unroll
+                for (int j = 0; j < SUM_SPARSE_MAX; ++j) {
+                    vv[j] = 0u;
+                    if (j < nb_span) {
+                        const int e = static_cast<int>(__shfl_sync(0xffffffffu, cb, j) - 1 - sbase);   // element before the boundary
+                        if (e >= 0) vv[j] = tmem_ld_32x1(taddr + (e >> 10) * ROW + (e & 31));
+                    }
+                }
+                tmem_ld_wait();
+                // exclusive prefix of the 128 row totals of the span (four interleaved warp scans)
+                Acc inc[PIECES_PER_SPAN];
+#pragma unroll
+                for (int i = 0; i < PIECES_PER_SPAN; ++i) inc[i] = tot[i];
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+                    for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                        const Acc t = __shfl_up_sync(0xffffffffu, inc[i], o);
+                        if (static_cast<int>(lane) >= o) inc[i] = P::add(t, inc[i]);
+                    }
+                }
+                Acc pbase_acc = Acc(0), rowpre_span[PIECES_PER_SPAN];
+#pragma unroll
+                for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                    rowpre_span[i] = P::add(pbase_acc, P::sub(inc[i], tot[i]));
+                    pbase_acc = P::add(pbase_acc, __shfl_sync(0xffffffffu, inc[i], 31));
+                }
+                // lane j keeps, for boundary j: the prefix inside its row, the prefix of the rows before, the row
+                Acc mylocal = Acc(0), myrp = Acc(0);
+                int myrow = -1;
+#pragma unroll
+                for (int j = 0; j < SUM_SPARSE_MAX; ++j) {
+                    if (j < nb_span) {
+                        const int e = static_cast<int>(__shfl_sync(0xffffffffu, cb, j) - 1 - sbase);
+                        if (e >= 0) {
+                            const int piece = e >> 10, row = (e >> 5) & 31;
+                            Acc rsel = rowpre_span[0];
+#pragma unroll
+                            for (int i = 1; i < PIECES_PER_SPAN; ++i)
+                                if (piece == i) rsel = rowpre_span[i];
+                            const Acc lj = P::from_bits(__shfl_sync(0xffffffffu, vv[j], row));
+                            const Acc rj = __shfl_sync(0xffffffffu, rsel, row);
+                            if (static_cast<int>(lane) == j) { mylocal = lj; myrp = rj; myrow = e >> 5; }
+                        }
+                    }
+                }
+                const Acc plocal = __shfl_up_sync(0xffffffffu, mylocal, 1);
+                const Acc prp = __shfl_up_sync(0xffffffffu, myrp, 1);
+                const int prow = __shfl_up_sync(0xffffffffu, myrow, 1);
+                const long long qi = cq + lane;
+                bool deferred = false;
+                Acc val = Acc(0);
+                // lane j: boundary j as the END of segment qi-1 (bnd in (sbase, send], or 0 for leading empties)
+                if (static_cast<int>(lane) < nb_span && qi >= 1 && (cb > sbase || (sbase == 0 && cb == 0))) {
+                    if (csb > cb || csb < 0 || cb > prm.n) {
+                        report_error(prm.hdr, 4u);
+                    } else {
+                        if (cb != csb) {
+                            if (cb - csb <= SUM_DIRECT_LEN) {
+                                for (long long e = csb; e < cb; ++e) val = P::add(val, load_value<P>(xg, e));
+                            } else if (csb > sbase) {
+                                // the start is the previous boundary (lane - 1), inside this span
+                                val = (prow == myrow) ? P::sub(mylocal, plocal)
+                                                      : P::sub(P::add(myrp, mylocal), P::add(prp, plocal));
+                            } else {
+                                val = P::add(myrp, mylocal);        // from the span's first element
+                                deferred = csb < sbase;
+                            }
+                        }
+                        if (!deferred) outp[qi - 1] = val;
+                    }
+                }
+                const unsigned dm = __ballot_sync(0xffffffffu, deferred);
+                if (dm) {
+                    const int src = __ffs(dm) - 1;
+                    def_r = cq + src - 1;
+                    def_val = __shfl_sync(0xffffffffu, val, src);
+                }
+                MMV_T_MARK(5)
+            }
 #pragma unroll 1
-            for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+            for (int i = 0; i < (sparse ? 0 : PIECES_PER_SPAN); ++i) {
                 const long long pbase = sbase + i * PIECE;
                 const long long pend = pbase + PIECE;
                 Acc toti = tot[0];
@@ -418,6 +525,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 }
                 if (!touched) {
                     run = P::add(run, warp_sum<P>(toti));
+                    MMV_T_MARK(3)
                     continue;
                 }
 
@@ -438,6 +546,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 rowpre[lane] = P::sub(inc, toti);
                 const Acc piece_total = __shfl_sync(0xffffffffu, inc, 31);
                 __syncwarp();
+                MMV_T_MARK(4)
 
                 // ---- boundaries with pbase <= bnd(q) <= pend, 32 at a time (sorted: a prefix of every batch) ----
                 bool piece_has_start = false;
@@ -522,30 +631,56 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     run = P::add(run, piece_total);
                 }
                 __syncwarp();
+                MMV_T_MARK(5)
             }
 
             // ---- the TMEM buffer is free; publish, look back, emit the segment that began before this span ----
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
+            MMV_T_MARK(6)
             // request the next tile's offsets (its first index has arrived by now)
             if (tile_n >= 0) load_offsets(q_next, nb, nsb);
-            if (!published && lane == 0)
+            if (!published && lane == 0) {
                 st_relaxed_gpu_u64(prm.status + s, pack_status((seen || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(run)));
+                agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + w] = (static_cast<uint64_t>(seen ? 1u : 0u) << 32) | P::to_bits(run);
+                mbar_arrive(&bar_agg[g]);
+            }
+            // Every warp waits on every phase of bar_agg (parity waits must not skip phases).  The carry
+            // into this span is first sought among the tile's earlier spans (shared memory); only if
+            // none of them holds a segment start does the look-back go out to the other CTAs' words.
+            if (!wait_bar(&bar_agg[g], k & 1, abort_flag, budget)) { failed = true; break; }
             if (s == 0) {
                 if (def_r >= 0 && lane == 0) outp[def_r] = def_val;
             } else if (!seen || def_r >= 0) {
-                Acc carry = Acc(0);
-                if (!lookback<P, 1>(prm.status, s, carry, abort_flag, budget, lbw, published)) {
-                    if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
-                    failed = true;
-                    break;
+                Acc ex = Acc(0);
+                bool exflag = false;
+#pragma unroll
+                for (int j = 0; j < SPANS_PER_TILE; ++j) {
+                    if (j < w) {
+                        const uint64_t a = agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + j];
+                        const Acc tj = P::from_bits(static_cast<uint32_t>(a));
+                        if ((a >> 32) != 0u) { ex = tj; exflag = true; }
+                        else ex = P::add(ex, tj);
+                    }
+                }
+                Acc carry = ex;
+                if (!exflag && tile != 0) {
+                    Acc carry_out = Acc(0);
+                    if (!lookback<P, 1>(prm.status, s - w, carry_out, abort_flag, budget, lbw, published)) {
+                        if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
+                        failed = true;
+                        break;
+                    }
+                    carry = P::add(carry_out, ex);
                 }
                 if (!seen && lane == 0)
                     st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(carry, run))));
                 if (def_r >= 0 && lane == 0) outp[def_r] = P::add(carry, def_val);
             }
+            MMV_T_MARK(7)
         }
+        MMV_T_FLUSH()
         if (failed) {
             *abort_flag = 1;
             if (lane == 0) report_error(prm.hdr, 5u);

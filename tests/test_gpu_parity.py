@@ -212,6 +212,22 @@ def test_seg_sum_csr_edges(mmv):
     assert sum_csr(mmv, np.zeros(0, np.int8), off).tolist() == [0] * 8
 
 
+@pytest.mark.parametrize("maxlen", [3, 60, 3000])
+def test_seg_sum_csr_many_tiles_per_cta(mmv, maxlen):
+    # more tiles than 2 x 148, so every CTA runs several tiles back to back in both warpgroups
+    rng = np.random.default_rng(1000 + maxlen)
+    n = (1 << 23) + 4321
+    lens = rng.integers(0, maxlen + 1, int(2.2 * n / maxlen) + 10)
+    cs = np.cumsum(lens)
+    keep = int(np.searchsorted(cs, n, side="right"))
+    off = np.concatenate([[0], cs[:keep], [n]]).astype(np.int32)
+    x = rng.integers(-128, 128, n).astype(np.int8)
+    assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
+    xf = rng.standard_normal(n).astype(np.float16)
+    want, a = oracle.seg_sum_csr_f16(xf, off)
+    assert_fp(sum_csr(mmv, xf, off), want, a, f"many tiles, maxlen={maxlen}")
+
+
 def test_seg_sum_config2_reduced(mmv):
     x, off = gen.config2(1 << 22)
     want, a = oracle.seg_sum_csr_f16(x, off)
@@ -234,7 +250,7 @@ def test_spmv_golden_and_random(mmv):
     y = spmv(mmv, np.asarray(g["spmv_rowptr"], np.int32), np.asarray(g["spmv_col"], np.int32),
              np.asarray(g["spmv_val"], np.float32).astype(np.float16), np.asarray(g["spmv_x"], np.float32))
     assert y.tolist() == g["spmv_y"]
-    for rows, frac in ((3000, 0.0), (20000, 0.1)):
+    for rows, frac in ((3000, 0.0), (20000, 0.1), (1 << 17, 0.05)):
         rowptr, col, val, x = gen.config4(rows=rows, empty_fraction=frac)
         want, a = oracle.spmv_csr(rowptr, col, val, x)
         got = spmv(mmv, rowptr, col, val, x)
