@@ -9,9 +9,9 @@ namespace mmv {
 // Optional phase timers (compile with -DMMV_PHASE_TIMERS): cycles summed over all epilogue warps.
 #ifdef MMV_PHASE_TIMERS
 __device__ unsigned long long g_phase_cycles[16];
-#define MMV_T_DECL long long t_prev = clock64(); unsigned long long t_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#define MMV_T_DECL long long t_prev = clock64(); unsigned long long t_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
 #define MMV_T_MARK(k) { const long long t_now = clock64(); t_acc[k] += static_cast<unsigned long long>(t_now - t_prev); t_prev = t_now; }
-#define MMV_T_FLUSH() { if (lane == 0) { for (int k = 0; k < 8; ++k) atomicAdd(&g_phase_cycles[k], t_acc[k]); } }
+#define MMV_T_FLUSH() { if (lane == 0) { for (int k = 0; k < 16; ++k) atomicAdd(&g_phase_cycles[k], t_acc[k]); } }
 #else
 #define MMV_T_DECL
 #define MMV_T_MARK(k)

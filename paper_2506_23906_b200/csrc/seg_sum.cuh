@@ -36,6 +36,8 @@ constexpr int SUM_BUFS = 4;                                        // TMEM tile 
 constexpr int SUM_TMEM_COLS = SUM_BUFS * PIECES_PER_SPAN * ROW;    // 512
 constexpr int SUM_SPARSE_MAX = 8;                                  // spans with at most this many boundaries read single prefixes from TMEM
 constexpr int SUM_DIRECT_LEN = 4;                                  // segments this short are summed from the inputs
+constexpr int SUM_TBL = 128;                                       // boundaries of a span kept in shared memory
+constexpr int SUM_TBL_BYTES = (SUM_TBL + 4) * 4 + SUM_TBL * 4;     // offsets (one predecessor in front) + direct sums
 
 // bf16 values (the hi/lo halves of the fp32 products of SpMV): same geometry as fp16.
 struct BF16Path : F16Path {
@@ -58,6 +60,87 @@ __device__ __forceinline__ uint32_t load_value<I8Path>(const void* base, long lo
     return static_cast<uint32_t>(static_cast<int32_t>(static_cast<const int8_t*>(base)[idx]));
 }
 
+// One input element given as its bit pattern in the low bits of a word.
+template <typename P>
+__device__ __forceinline__ typename P::Acc elem_bits_to_acc(uint32_t bits);
+template <>
+__device__ __forceinline__ float elem_bits_to_acc<F16Path>(uint32_t bits) {
+    return __half2float(__ushort_as_half(static_cast<unsigned short>(bits)));
+}
+template <>
+__device__ __forceinline__ float elem_bits_to_acc<BF16Path>(uint32_t bits) {
+    return __uint_as_float(bits << 16);
+}
+template <>
+__device__ __forceinline__ uint32_t elem_bits_to_acc<I8Path>(uint32_t bits) {
+    return static_cast<uint32_t>(static_cast<int32_t>(static_cast<int8_t>(bits)));
+}
+
+// Sum of the elements [sb, cb) of a very short segment, taken from the input values themselves.
+template <typename P>
+__device__ __forceinline__ typename P::Acc direct_sum(const void* xg, long long sb, long long cb) {
+    typename P::Acc val = typename P::Acc(0);
+    for (long long e = sb; e < cb; ++e) val = P::add(val, load_value<P>(xg, e));
+    return val;
+}
+
+// The same sum in two steps, so that the loads can be in flight while other work is done:
+// window_load fetches the two aligned words of four elements each that hold [sb, sb + 4) (no
+// arithmetic on them), window_sum adds up the first `len` elements once they are needed.
+// Falls back to element loads where an aligned word would reach past the n input values.
+struct ValueWindow {
+    uint32_t r[4];
+    bool wide;
+};
+template <typename P>
+__device__ __forceinline__ void window_load(const void* xg, long long sb, int len, long long n, ValueWindow& win) {
+    constexpr int EB = P::kElemBytes;                   // 2 or 1: a word of four elements is 8 or 4 bytes
+    const long long base = sb & ~3ll;
+    const int sh = static_cast<int>(sb & 3);
+    win.r[0] = win.r[1] = win.r[2] = win.r[3] = 0u;
+    win.wide = (base + 4 <= n) && (sh + len <= 4 || base + 8 <= n);
+    if (!win.wide) return;
+    const uint8_t* p = static_cast<const uint8_t*>(xg) + base * EB;
+    if constexpr (EB == 2) {
+        const uint2 a = *reinterpret_cast<const uint2*>(p);
+        win.r[0] = a.x;
+        win.r[1] = a.y;
+        if (sh + len > 4) {
+            const uint2 b = *reinterpret_cast<const uint2*>(p + 8);
+            win.r[2] = b.x;
+            win.r[3] = b.y;
+        }
+    } else {
+        win.r[0] = *reinterpret_cast<const uint32_t*>(p);
+        if (sh + len > 4) win.r[1] = *reinterpret_cast<const uint32_t*>(p + 4);
+    }
+}
+template <typename P>
+__device__ __forceinline__ typename P::Acc window_sum(const void* xg, long long sb, int len, const ValueWindow& win) {
+    using Acc = typename P::Acc;
+    if (!win.wide) return direct_sum<P>(xg, sb, sb + len);
+    constexpr int EB = P::kElemBytes;
+    const int sh = static_cast<int>(sb & 3);
+    Acc val = Acc(0);
+    if constexpr (EB == 2) {
+        const int bits = sh * 16;
+        const uint32_t a0 = bits >= 32 ? win.r[1] : win.r[0];
+        const uint32_t a1 = bits >= 32 ? win.r[2] : win.r[1];
+        const uint32_t a2 = bits >= 32 ? win.r[3] : win.r[2];
+        const uint32_t o0 = __funnelshift_r(a0, a1, bits & 31), o1 = __funnelshift_r(a1, a2, bits & 31);
+        const uint32_t e[4] = {o0 & 0xffffu, o0 >> 16, o1 & 0xffffu, o1 >> 16};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (i < len) val = P::add(val, elem_bits_to_acc<P>(e[i]));
+    } else {
+        const uint32_t o = __funnelshift_r(win.r[0], win.r[1], sh * 8);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (i < len) val = P::add(val, elem_bits_to_acc<P>((o >> (8 * i)) & 0xffu));
+    }
+    return val;
+}
+
 template <typename P>
 struct SumCfg {
     static constexpr int kStages = 4;
@@ -67,7 +150,8 @@ struct SumCfg {
     static constexpr int kStageOffset = 2048;                        // after the constant operand
     static constexpr int kDumpOffset = kStageOffset + kStages * kXBytes;
     static constexpr int kRowpreOffset = kDumpOffset + SUM_EPI_WARPS * kDumpBytes;
-    static constexpr int kBarOffset = kRowpreOffset + SUM_EPI_WARPS * PIECE_ROWS * 4;
+    static constexpr int kTblOffset = kRowpreOffset + SUM_EPI_WARPS * PIECE_ROWS * 4;
+    static constexpr int kBarOffset = kTblOffset + SUM_EPI_WARPS * SUM_TBL_BYTES;
     static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
     static_assert(kBBytes <= 2048, "constant operand fits its slot");
 };
@@ -311,6 +395,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         Acc* outp = static_cast<Acc*>(prm.out);
         uint8_t* dump = smem + Cfg::kDumpOffset + warp * Cfg::kDumpBytes;      // [32 rows][32] swizzled by row
         Acc* rowpre = reinterpret_cast<Acc*>(smem + Cfg::kRowpreOffset) + warp * PIECE_ROWS;
+        int32_t* tbl = reinterpret_cast<int32_t*>(smem + Cfg::kTblOffset + warp * SUM_TBL_BYTES);   // [0] = offset before the first
+        Acc* dvt = reinterpret_cast<Acc*>(tbl + SUM_TBL + 4);
         const int sh = prm.off_shift;
         const long long nq = prm.nseg + 1;
         bool failed = false;
@@ -328,19 +414,40 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             const int t = static_cast<int>(blockIdx.x) + (g + 2 * kk) * static_cast<int>(gridDim.x);
             return t < prm.num_tiles ? t : -1;
         };
-        auto load_offsets = [&](long long q0, long long& b, long long& sb) {
-            const long long qi = q0 + lane;
-            b = -1;
-            sb = -1;
-            if (qi < nq) b = static_cast<long long>(prm.off[qi]) << sh;
-            if (qi >= 1 && qi < nq) sb = static_cast<long long>(prm.off[qi - 1]) << sh;
+        // raw offset -> position (index checks against nq are made where an entry is used)
+        auto cvt = [&](int32_t raw) -> long long { return static_cast<long long>(raw) << sh; };
+        constexpr int32_t kNoOffset = 0;
+        // offsets q0 + lane + 32 j (j < 4), the one before q0, and the last one below the span's end
+        auto load_offsets = [&](long long q0, long long qe, int32_t (&raw)[4], int32_t& rawp, long long& last) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const long long qi = q0 + lane + 32 * j;
+                raw[j] = kNoOffset;
+                if (qi < nq) raw[j] = prm.off[qi];
+            }
+            rawp = kNoOffset;
+            if (q0 >= 1 && q0 - 1 < nq) rawp = prm.off[q0 - 1];
+            last = -1;
+            if (qe > q0 && qe <= nq) last = static_cast<long long>(prm.off[qe - 1]) << sh;
+        };
+        auto load_span_q = [&](int t, long long& q0, long long& qe) {
+            const int32_t* sq = prm.span_q + static_cast<long long>(t) * SPANS_PER_TILE + w;
+            q0 = sq[0];
+            qe = sq[1];
         };
         MMV_T_DECL
-        long long q_next = 0, nb = -1, nsb = -1;
+        // The boundaries of the NEXT tile's span are prefetched one tile ahead.
+        long long q_next = 0, qe_next = 0, nlast = -1;
+        int32_t nraw[4] = {kNoOffset, kNoOffset, kNoOffset, kNoOffset}, nrawp = kNoOffset;
         if (tile_of(0) >= 0) {
-            q_next = prm.span_q[static_cast<long long>(tile_of(0)) * SPANS_PER_TILE + w];
-            load_offsets(q_next, nb, nsb);
+            load_span_q(tile_of(0), q_next, qe_next);
+            load_offsets(q_next, qe_next, nraw, nrawp, nlast);
         }
+        // a segment that began before an earlier span of this warp and still waits for its carry
+        bool pending = false;
+        long long pend_s = 0, pend_r = -1;
+        Acc pend_val = Acc(0), pend_ex = Acc(0);
+        LookbackWindow<1> plw;
         for (int k = 0;; ++k) {
             // the epilogue never reads the operand stage (the MMA warp releases it); with the static
             // tile order it knows its tile without being told
@@ -355,11 +462,43 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             // ---- the span's boundaries: one offset per lane (requested during the previous tile) ----
             long long q = q_next;                              // first q with bnd(q) >= sbase
             const long long cq = q;                            // index held by lane 0 of the cache
-            const long long cb = nb, csb = nsb;                // cached boundary and its predecessor
+            int32_t raw[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) raw[j] = nraw[j];
+            const int32_t rawp = nrawp;
+            const long long last_b = nlast;                    // last boundary below the span's end
             const int tile_n = tile_of(k + 1);
-            if (tile_n >= 0) q_next = prm.span_q[static_cast<long long>(tile_n) * SPANS_PER_TILE + w];
-            // the cache covers the span if it reaches past the span's end (or the end of the offsets)
+            if (tile_n >= 0) load_span_q(tile_n, q_next, qe_next);
+            // table entry t <-> boundary index cq + t; lane holds entries lane + 32 j
+            long long bj[4], sbj[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                int32_t pr = __shfl_up_sync(0xffffffffu, raw[j], 1);
+                const int32_t wrap = __shfl_sync(0xffffffffu, j == 0 ? rawp : raw[j > 0 ? j - 1 : 0], j == 0 ? 0 : 31);
+                if (lane == 0) pr = wrap;
+                bj[j] = (cq + lane + 32 * j < nq) ? cvt(raw[j]) : -1ll;
+                sbj[j] = (cq + lane + 32 * j >= 1) ? cvt(pr) : -1ll;
+                tbl[1 + lane + 32 * j] = raw[j];
+            }
+            if (lane == 0) tbl[0] = rawp;
+            const long long cb = bj[0], csb = sbj[0];          // the first 32 boundaries, one per lane
+            // the first 32 entries cover the span if they reach past its end (or the end of the offsets)
             const bool covers = __any_sync(0xffffffffu, (q + lane >= nq) || (cb > send));
+            // ... and so does the whole table
+            bool tc = false;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) tc |= (cq + lane + 32 * j >= nq) || (bj[j] > send);
+            const bool tcovers = __any_sync(0xffffffffu, tc);
+            // very short segments that end in this span are summed from the inputs; the loads go out
+            // now and return while the accumulators are awaited
+            bool isdir[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                isdir[j] = cq + lane + 32 * j >= 1 && cq + lane + 32 * j < nq && sbj[j] >= 0 && bj[j] > sbj[j] &&
+                           bj[j] - sbj[j] <= SUM_DIRECT_LEN && bj[j] > sbase && bj[j] <= send && bj[j] <= prm.n;
+            ValueWindow win0;
+            win0.wide = false;
+            if (isdir[0]) window_load<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), prm.n, win0);
 
             MMV_T_MARK(0)
             if (!wait_bar(&bar_acc_full[buf], (k >> 1) & 1, abort_flag, budget)) { failed = true; break; }
@@ -372,16 +511,13 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * ROW + (ROW - 1)));
             tmem_ld_wait();
 
-            // ---- pre-pass (all boundaries in registers): the span's aggregate from the row totals and one
-            //      prefix, published before the boundaries are worked through ----
+            // ---- pre-pass: the span's aggregate from the row totals and the one prefix before the span's
+            //      last segment start, published before the boundaries are worked through ----
             LookbackWindow<1> lbw;
-            bool published = false;
-            int lastrel = -1;
+            // the last segment start inside the span, or -1
+            const int lastrel = (last_b >= sbase && last_b < send) ? static_cast<int>(last_b - sbase) : -1;
             Acc tail_pre = Acc(0);
-            if (covers) {
-                const bool isstart = (cq + lane < nq) && (cb >= sbase) && (cb < send);
-                const int rel = isstart ? static_cast<int>(cb - sbase) : -1;
-                lastrel = __reduce_max_sync(0xffffffffu, rel);               // last segment start inside the span
+            {
                 Acc tail;
                 if (lastrel < 0) {
                     tail = warp_sum<P>(P::add(P::add(tot[0], tot[1]), P::add(tot[2], tot[3])));
@@ -405,19 +541,35 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (lane == 0)
                     st_relaxed_gpu_u64(prm.status + s,
                                        pack_status((lastrel >= 0 || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail)));
-                published = true;
                 tail_pre = tail;
                 if (lane == 0) {
                     agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + w] = (static_cast<uint64_t>(lastrel >= 0 ? 1u : 0u) << 32) | P::to_bits(tail);
                     mbar_arrive(&bar_agg[g]);
                 }
                 // the first window beyond the tile travels while the boundaries are processed
-                if (tile != 0) lookback_load<1>(prm.status, s - w - 1, lbw);
+                if (tile != 0 && lastrel < 0) lookback_load<1>(prm.status, s - w - 1, lbw);
+                if (pending) lookback_load<1>(prm.status, pend_s - w - 1, plw);
             }
+            // direct sums: the first 32 boundaries' values have arrived by now; the others (spans with
+            // more than 32 boundaries) are fetched here, all at once
+            const Acc dval = isdir[0] ? window_sum<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), win0) : Acc(0);
+            dvt[lane] = dval;
+            if (!covers) {
+                ValueWindow wn[3];
+#pragma unroll
+                for (int j = 1; j < 4; ++j) {
+                    wn[j - 1].wide = false;
+                    if (isdir[j]) window_load<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), prm.n, wn[j - 1]);
+                }
+#pragma unroll
+                for (int j = 1; j < 4; ++j)
+                    dvt[lane + 32 * j] = isdir[j] ? window_sum<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), wn[j - 1]) : Acc(0);
+            }
+            __syncwarp();
 
             MMV_T_MARK(2)
             Acc run = Acc(0);              // sum of the open segment inside this span so far
-            bool seen = false;             // a segment start lies inside this span
+            const bool seen = lastrel >= 0;   // a segment start lies inside this span
             long long def_r = -1;          // segment that began before the span and ends inside it
             Acc def_val = Acc(0);
             // number of boundaries with sbase <= bnd <= send (a prefix of the cache lanes)
@@ -426,7 +578,6 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             if (sparse) {
                 // ---- few boundaries: no copy of the prefixes; the one prefix each boundary needs is read
                 //      straight from TMEM (one column, the lane of its row) ----
-                seen = lastrel >= 0;
                 run = tail_pre;               // the open segment's sum at the end of the span
                 uint32_t vv[SUM_SPARSE_MAX];
 #pragma unroll
@@ -488,7 +639,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     } else {
                         if (cb != csb) {
                             if (cb - csb <= SUM_DIRECT_LEN) {
-                                for (long long e = csb; e < cb; ++e) val = P::add(val, load_value<P>(xg, e));
+                                val = dval;
                             } else if (csb > sbase) {
                                 // the start is the previous boundary (lane - 1), inside this span
                                 val = (prow == myrow) ? P::sub(mylocal, plocal)
@@ -519,9 +670,11 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     if (i == t) toti = tot[t];
                 // any boundary with pbase <= bnd <= pend (END in (pbase, pend], START in [pbase, pend))?
                 bool touched = true;
-                if (covers) {
-                    const long long qi = cq + lane;
-                    touched = __any_sync(0xffffffffu, (qi >= q) && (qi < nq) && (cb >= pbase) && (cb <= pend));
+                if (tcovers) {
+                    bool t4 = false;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) t4 |= (cq + lane + 32 * j >= q) && (bj[j] >= pbase) && (bj[j] <= pend);
+                    touched = __any_sync(0xffffffffu, t4);
                 }
                 if (!touched) {
                     run = P::add(run, warp_sum<P>(toti));
@@ -556,13 +709,13 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 while (true) {
                     const long long qi = qp + lane;
                     long long b = -1, sb = -1;
-                    if (covers && qp == q) {
-                        // the batch is the cache shifted by (q - cq) lanes; lanes shifted in from beyond the
-                        // cache lie past the span's end by construction
-                        const int d = static_cast<int>(q - cq);
-                        b = __shfl_down_sync(0xffffffffu, cb, d);
-                        sb = __shfl_down_sync(0xffffffffu, csb, d);
-                        if (static_cast<int>(lane) + d >= 32) { b = send + 1; sb = send + 1; }
+                    Acc dv = Acc(0);
+                    const long long rel = qi - cq;
+                    const bool cached = rel < SUM_TBL;
+                    if (cached) {
+                        if (qi < nq) b = cvt(tbl[1 + rel]);
+                        if (qi >= 1 && qi < nq) sb = cvt(tbl[rel]);
+                        dv = dvt[rel];
                     } else {
                         if (qi < nq) b = static_cast<long long>(prm.off[qi]) << sh;
                         if (qi >= 1 && qi < nq) sb = static_cast<long long>(prm.off[qi - 1]) << sh;
@@ -581,7 +734,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                             if (b != sb) {
                                 if (b - sb <= SUM_DIRECT_LEN) {
                                     // a very short segment: add the input values themselves
-                                    for (long long e = sb; e < b; ++e) val = P::add(val, load_value<P>(xg, e));
+                                    val = cached ? dv : direct_sum<P>(xg, sb, b);
                                 } else {
                                     Acc ep, sp = Acc(0);
                                     int erow, srow;
@@ -626,7 +779,6 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     Acc before = Acc(0);
                     if (last_start > pbase) before = piece_prefix(static_cast<int>(last_start - 1 - pbase), sp2, srow2);
                     run = P::sub(piece_total, before);
-                    seen = true;
                 } else {
                     run = P::add(run, piece_total);
                 }
@@ -640,16 +792,19 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
             MMV_T_MARK(6)
             // request the next tile's offsets (its first index has arrived by now)
-            if (tile_n >= 0) load_offsets(q_next, nb, nsb);
-            if (!published && lane == 0) {
-                st_relaxed_gpu_u64(prm.status + s, pack_status((seen || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(run)));
-                agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + w] = (static_cast<uint64_t>(seen ? 1u : 0u) << 32) | P::to_bits(run);
-                mbar_arrive(&bar_agg[g]);
-            }
+            if (tile_n >= 0) load_offsets(q_next, qe_next, nraw, nrawp, nlast);
             // Every warp waits on every phase of bar_agg (parity waits must not skip phases).  The carry
             // into this span is first sought among the tile's earlier spans (shared memory); only if
             // none of them holds a segment start does the look-back go out to the other CTAs' words.
             if (!wait_bar(&bar_agg[g], k & 1, abort_flag, budget)) { failed = true; break; }
+            // the segment parked at this warp's previous tile: its look-back window was requested during
+            // this tile's pre-pass, so the predecessor's word has normally arrived
+            if (pending) {
+                Acc carry_out = Acc(0);
+                if (!lookback<P, 1>(prm.status, pend_s - w, carry_out, abort_flag, budget, plw, true)) { failed = true; break; }
+                if (lane == 0) outp[pend_r] = P::add(P::add(carry_out, pend_ex), pend_val);
+                pending = false;
+            }
             if (s == 0) {
                 if (def_r >= 0 && lane == 0) outp[def_r] = def_val;
             } else if (!seen || def_r >= 0) {
@@ -664,21 +819,39 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                         else ex = P::add(ex, tj);
                     }
                 }
-                Acc carry = ex;
-                if (!exflag && tile != 0) {
+                if (exflag || tile == 0) {
+                    // the carry is complete inside the tile
+                    if (!seen && lane == 0)
+                        st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(ex, run))));
+                    if (def_r >= 0 && lane == 0) outp[def_r] = P::add(ex, def_val);
+                } else if (seen) {
+                    // The span's own word is final already; only the segment that ends here waits for the
+                    // carry from the other CTAs.  It is parked until this warp's next tile is done, which
+                    // keeps the CTAs from falling into step with their slowest neighbour.
+                    pending = true;
+                    pend_s = s;
+                    pend_r = def_r;
+                    pend_val = def_val;
+                    pend_ex = ex;
+                } else {
                     Acc carry_out = Acc(0);
-                    if (!lookback<P, 1>(prm.status, s - w, carry_out, abort_flag, budget, lbw, published)) {
+                    if (!lookback<P, 1>(prm.status, s - w, carry_out, abort_flag, budget, lbw, true)) {
                         if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
                         failed = true;
                         break;
                     }
-                    carry = P::add(carry_out, ex);
+                    const Acc carry = P::add(carry_out, ex);
+                    if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(carry, run))));
+                    if (def_r >= 0 && lane == 0) outp[def_r] = P::add(carry, def_val);
                 }
-                if (!seen && lane == 0)
-                    st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(carry, run))));
-                if (def_r >= 0 && lane == 0) outp[def_r] = P::add(carry, def_val);
             }
             MMV_T_MARK(7)
+        }
+        if (pending && !failed) {
+            Acc carry_out = Acc(0);
+            LookbackWindow<1> lw;
+            if (!lookback<P, 1>(prm.status, pend_s - w, carry_out, abort_flag, budget, lw, false)) failed = true;
+            else if (lane == 0) outp[pend_r] = P::add(P::add(carry_out, pend_ex), pend_val);
         }
         MMV_T_FLUSH()
         if (failed) {
