@@ -114,9 +114,7 @@ __device__ __forceinline__ void report_error(WorkspaceHeader* hdr, unsigned int 
 }
 
 // Bounded mbarrier wait that also gives up when another role of the CTA has aborted.
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                         uint64_t budget_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
+__device__ __noinline__ bool wait_bar_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint64_t budget_ns) {
     const uint64_t t0 = global_timer_ns();
     uint32_t polls = 0;
     while (!mbar_try_wait(bar, parity)) {
@@ -126,6 +124,13 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
         }
     }
     return true;
+}
+// (The polling loop is out of line: there are dozens of wait sites and the epilogues have to
+// stay inside the instruction cache.)
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                         uint64_t budget_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return wait_bar_slow(bar, parity, abort_flag, budget_ns);
 }
 
 template <typename P>

@@ -77,8 +77,9 @@ __device__ __forceinline__ uint32_t elem_bits_to_acc<I8Path>(uint32_t bits) {
 }
 
 // Sum of the elements [sb, cb) of a very short segment, taken from the input values themselves.
+// (Not inlined: it is the rare path, and the epilogue has to stay inside the instruction cache.)
 template <typename P>
-__device__ __forceinline__ typename P::Acc direct_sum(const void* xg, long long sb, long long cb) {
+__device__ __noinline__ typename P::Acc direct_sum(const void* xg, long long sb, long long cb) {
     typename P::Acc val = typename P::Acc(0);
     for (long long e = sb; e < cb; ++e) val = P::add(val, load_value<P>(xg, e));
     return val;
@@ -139,6 +140,18 @@ __device__ __forceinline__ typename P::Acc window_sum(const void* xg, long long 
             if (i < len) val = P::add(val, elem_bits_to_acc<P>((o >> (8 * i)) & 0xffu));
     }
     return val;
+}
+
+// The look-back of the segmented sum behind one signature for its three call sites.
+template <typename P>
+__device__ __forceinline__ bool sum_lookback(const uint64_t* status, long long s, typename P::Acc* carry,
+                                          volatile int* abort_flag, uint64_t budget_ns, uint64_t window, bool preloaded) {
+    LookbackWindow<1> win;
+    win.w[0] = window;
+    typename P::Acc c = typename P::Acc(0);
+    const bool ok = lookback<P, 1>(status, s, c, abort_flag, budget_ns, win, preloaded);
+    *carry = c;
+    return ok;
 }
 
 template <typename P>
@@ -801,7 +814,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             // this tile's pre-pass, so the predecessor's word has normally arrived
             if (pending) {
                 Acc carry_out = Acc(0);
-                if (!lookback<P, 1>(prm.status, pend_s - w, carry_out, abort_flag, budget, plw, true)) { failed = true; break; }
+                if (!sum_lookback<P>(prm.status, pend_s - w, &carry_out, abort_flag, budget, plw.w[0], true)) { failed = true; break; }
                 if (lane == 0) outp[pend_r] = P::add(P::add(carry_out, pend_ex), pend_val);
                 pending = false;
             }
@@ -835,7 +848,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     pend_ex = ex;
                 } else {
                     Acc carry_out = Acc(0);
-                    if (!lookback<P, 1>(prm.status, s - w, carry_out, abort_flag, budget, lbw, true)) {
+                    if (!sum_lookback<P>(prm.status, s - w, &carry_out, abort_flag, budget, lbw.w[0], true)) {
                         if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
                         failed = true;
                         break;
@@ -849,8 +862,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         }
         if (pending && !failed) {
             Acc carry_out = Acc(0);
-            LookbackWindow<1> lw;
-            if (!lookback<P, 1>(prm.status, pend_s - w, carry_out, abort_flag, budget, lw, false)) failed = true;
+            if (!sum_lookback<P>(prm.status, pend_s - w, &carry_out, abort_flag, budget, 0ull, false)) failed = true;
             else if (lane == 0) outp[pend_r] = P::add(P::add(carry_out, pend_ex), pend_val);
         }
         MMV_T_FLUSH()
