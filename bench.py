@@ -42,9 +42,9 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic of the headline kernel from the ncu capture of its n = 2^26 case
 # (profiles/seg_scan_kernel_f16_n2p26_p1e-3.md): reads 3.002 B/element, writes 4 B/element minus
 # the ~57 MB of output that are still in L2 when a launch ends; both scale with n.
-NCU_READ_BYTES_PER_ELEM = 3.002
+NCU_READ_BYTES_PER_ELEM = 3.001
 NCU_WRITE_BYTES_PER_ELEM = 4.0
-NCU_WRITE_L2_RESIDUE_BYTES = 56.6e6
+NCU_WRITE_L2_RESIDUE_BYTES = 58.9e6
 
 
 def parse_args():
@@ -73,7 +73,11 @@ def measured_peak():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs.
+
+    Every sample is stamped when it arrives; summary(t0, t1) keeps the ones taken inside the
+    window, i.e. while the GPU was under the benchmark's load.
+    """
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -86,7 +90,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -96,19 +100,23 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append(line.strip())
+            self.rows.append((time.perf_counter(), line.strip()))
 
     def __exit__(self, *a):
         if self.proc is not None:
-            time.sleep(0.15)
             self.proc.kill()
             self.proc.wait()
             self.thread.join(timeout=1.0)
 
-    def summary(self):
+    def count_between(self, t0, t1):
+        return sum(1 for t, _ in list(self.rows) if t0 <= t <= t1)
+
+    def summary(self, t0=float("-inf"), t1=float("inf")):
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for t, r in list(self.rows):
+            if not (t0 <= t <= t1):
+                continue
             parts = [p.strip() for p in r.split(",")]
             if len(parts) < 7:
                 continue
@@ -357,19 +365,29 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(max(3, args.warmup)):
-        step()
-    barrier()
-    launches0 = mmv.kernel_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local) as clk:
+        for _ in range(max(3, args.warmup)):
+            step()
         barrier()
+        launches0 = mmv.kernel_launch_count()
+        t_load0 = time.perf_counter()
         e0.record()
         for _ in range(args.steps):
             step()
         e1.record()
         barrier()
-    launches = mmv.kernel_launch_count() - launches0
+        launches = mmv.kernel_launch_count() - launches0
+        # The timed region can be shorter than the sampler's period: keep the GPU under the very same
+        # load (untimed) until a handful of clock samples have been taken inside the window.
+        t_extra0 = time.perf_counter()
+        while clk.count_between(t_load0, time.perf_counter()) < 6 and time.perf_counter() - t_extra0 < 1.5:
+            for _ in range(16):
+                step()
+            torch.cuda.synchronize()
+        t_load1 = time.perf_counter()
+    clocks = clk.summary(t_load0, t_load1)
+    clocks["window"] = "timed steps followed by identical untimed steps until >= 6 samples"
     ms = e0.elapsed_time(e1) / args.steps
     if mmv.last_async_status(ws) != 0:
         raise SystemExit("bench: device-side error status")
@@ -402,7 +420,7 @@ def run_ours(args):
             "config": {"workload": f"C5 seg-scan n=2^{args.log2n} fp16 U[-1,1) -> fp32, uint8 flags {args.case}",
                        "n_per_gpu": n, "timing": "inputs (7 B/elem working set) larger than L2; no flush needed",
                        "parallelism": f"{world} independent shards, no collective"},
-            "clocks": clk.summary(),
+            "clocks": clocks,
             "e2e": {"value": whole_job_value(world, n, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": 3 * n,
                     "d2h_bytes_per_step": 4 * n, "ms_per_step": e2e_ms, "steps": e2e_steps},
             "gpu_launches": int(launches),
