@@ -431,7 +431,10 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         auto cvt = [&](int32_t raw) -> long long { return static_cast<long long>(raw) << sh; };
         constexpr int32_t kNoOffset = 0;
         // offsets q0 + lane + 32 j (j < 4), the one before q0, and the last one below the span's end
-        auto load_offsets = [&](long long q0, long long qe, int32_t (&raw)[4], int32_t& rawp, long long& last) {
+        // (No arithmetic may touch a prefetched value before the tile that uses it: even a sign
+        // extension would make the warp wait for the load on the spot.  `last_ok` says whether `last`
+        // was loaded at all.)
+        auto load_offsets = [&](long long q0, long long qe, int32_t (&raw)[4], int32_t& rawp, int32_t& last, bool& last_ok) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const long long qi = q0 + lane + 32 * j;
@@ -440,21 +443,23 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             }
             rawp = kNoOffset;
             if (q0 >= 1 && q0 - 1 < nq) rawp = prm.off[q0 - 1];
-            last = -1;
-            if (qe > q0 && qe <= nq) last = static_cast<long long>(prm.off[qe - 1]) << sh;
+            last = kNoOffset;
+            last_ok = qe > q0 && qe <= nq;
+            if (last_ok) last = prm.off[qe - 1];
         };
-        auto load_span_q = [&](int t, long long& q0, long long& qe) {
+        auto load_span_q = [&](int t, int32_t& q0, int32_t& qe) {
             const int32_t* sq = prm.span_q + static_cast<long long>(t) * SPANS_PER_TILE + w;
             q0 = sq[0];
             qe = sq[1];
         };
         MMV_T_DECL
         // The boundaries of the NEXT tile's span are prefetched one tile ahead.
-        long long q_next = 0, qe_next = 0, nlast = -1;
+        int32_t q_next = 0, qe_next = 0, nlast = kNoOffset;
+        bool nlast_ok = false;
         int32_t nraw[4] = {kNoOffset, kNoOffset, kNoOffset, kNoOffset}, nrawp = kNoOffset;
         if (tile_of(0) >= 0) {
             load_span_q(tile_of(0), q_next, qe_next);
-            load_offsets(q_next, qe_next, nraw, nrawp, nlast);
+            load_offsets(q_next, qe_next, nraw, nrawp, nlast, nlast_ok);
         }
         // a segment that began before an earlier span of this warp and still waits for its carry
         bool pending = false;
@@ -479,129 +484,98 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
 #pragma unroll
             for (int j = 0; j < 4; ++j) raw[j] = nraw[j];
             const int32_t rawp = nrawp;
-            const long long last_b = nlast;                    // last boundary below the span's end
+            const long long last_b = nlast_ok ? cvt(nlast) : -1ll;   // last boundary below the span's end
+            MMV_T_MARK(8)
             const int tile_n = tile_of(k + 1);
             if (tile_n >= 0) load_span_q(tile_n, q_next, qe_next);
-            // table entry t <-> boundary index cq + t; lane holds entries lane + 32 j
-            long long bj[4], sbj[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                int32_t pr = __shfl_up_sync(0xffffffffu, raw[j], 1);
-                const int32_t wrap = __shfl_sync(0xffffffffu, j == 0 ? rawp : raw[j > 0 ? j - 1 : 0], j == 0 ? 0 : 31);
-                if (lane == 0) pr = wrap;
-                bj[j] = (cq + lane + 32 * j < nq) ? cvt(raw[j]) : -1ll;
-                sbj[j] = (cq + lane + 32 * j >= 1) ? cvt(pr) : -1ll;
-                tbl[1 + lane + 32 * j] = raw[j];
+            MMV_T_MARK(10)
+            // table entry t <-> boundary index cq + t; lane holds entries lane + 32 j.  Block 0 first: it
+            // decides between the path for spans with few boundaries and the general one.
+            long long bj[4] = {-1, -1, -1, -1}, sbj[4] = {-1, -1, -1, -1};
+            {
+                int32_t pr = __shfl_up_sync(0xffffffffu, raw[0], 1);
+                if (lane == 0) pr = rawp;
+                if (cq + lane < nq) bj[0] = cvt(raw[0]);
+                if (cq + lane >= 1) sbj[0] = cvt(pr);
             }
-            if (lane == 0) tbl[0] = rawp;
             const long long cb = bj[0], csb = sbj[0];          // the first 32 boundaries, one per lane
             // the first 32 entries cover the span if they reach past its end (or the end of the offsets)
             const bool covers = __any_sync(0xffffffffu, (q + lane >= nq) || (cb > send));
-            // ... and so does the whole table
-            bool tc = false;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) tc |= (cq + lane + 32 * j >= nq) || (bj[j] > send);
-            const bool tcovers = __any_sync(0xffffffffu, tc);
+            // number of boundaries with sbase <= bnd <= send (a prefix of the lanes)
+            const int nb_span = __popc(__ballot_sync(0xffffffffu, (cq + lane < nq) && (cb >= 0) && (cb <= send)));
+            const bool sparse = covers && nb_span <= SUM_SPARSE_MAX;
+            // the last segment start inside the span, or -1
+            const int lastrel = (last_b >= sbase && last_b < send) ? static_cast<int>(last_b - sbase) : -1;
+            const bool seen = lastrel >= 0;   // a segment start lies inside this span
+            MMV_T_MARK(9)
             // very short segments that end in this span are summed from the inputs; the loads go out
             // now and return while the accumulators are awaited
-            bool isdir[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                isdir[j] = cq + lane + 32 * j >= 1 && cq + lane + 32 * j < nq && sbj[j] >= 0 && bj[j] > sbj[j] &&
-                           bj[j] - sbj[j] <= SUM_DIRECT_LEN && bj[j] > sbase && bj[j] <= send && bj[j] <= prm.n;
+            bool isdir[4] = {false, false, false, false};
+            isdir[0] = cq + lane >= 1 && cq + lane < nq && sbj[0] >= 0 && bj[0] > sbj[0] && bj[0] - sbj[0] <= SUM_DIRECT_LEN &&
+                       bj[0] > sbase && bj[0] <= send && bj[0] <= prm.n;
             ValueWindow win0;
             win0.wide = false;
             if (isdir[0]) window_load<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), prm.n, win0);
+            bool tcovers = covers;
+            if (!sparse) {
+                // the general path keeps up to 128 boundaries in a shared-memory table
+                bool tc = false;
+                tbl[1 + lane] = raw[0];
+                if (lane == 0) tbl[0] = rawp;
+#pragma unroll
+                for (int j = 1; j < 4; ++j) {
+                    int32_t pr = __shfl_up_sync(0xffffffffu, raw[j], 1);
+                    const int32_t wrap = __shfl_sync(0xffffffffu, raw[j - 1], 31);
+                    if (lane == 0) pr = wrap;
+                    if (cq + lane + 32 * j < nq) bj[j] = cvt(raw[j]);
+                    sbj[j] = cvt(pr);
+                    tbl[1 + lane + 32 * j] = raw[j];
+                    tc |= (cq + lane + 32 * j >= nq) || (bj[j] > send);
+                    isdir[j] = cq + lane + 32 * j < nq && sbj[j] >= 0 && bj[j] > sbj[j] && bj[j] - sbj[j] <= SUM_DIRECT_LEN &&
+                               bj[j] > sbase && bj[j] <= send && bj[j] <= prm.n;
+                }
+                tcovers = __any_sync(0xffffffffu, tc) || covers;
+            }
 
             MMV_T_MARK(0)
             if (!wait_bar(&bar_acc_full[buf], (k >> 1) & 1, abort_flag, budget)) { failed = true; break; }
             tc_fence_after_sync();
             MMV_T_MARK(1)
 
-            // row totals of the four pieces
-            Acc tot[PIECES_PER_SPAN];
-#pragma unroll
-            for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * ROW + (ROW - 1)));
-            tmem_ld_wait();
-
-            // ---- pre-pass: the span's aggregate from the row totals and the one prefix before the span's
-            //      last segment start, published before the boundaries are worked through ----
             LookbackWindow<1> lbw;
-            // the last segment start inside the span, or -1
-            const int lastrel = (last_b >= sbase && last_b < send) ? static_cast<int>(last_b - sbase) : -1;
-            Acc tail_pre = Acc(0);
-            {
-                Acc tail;
-                if (lastrel < 0) {
-                    tail = warp_sum<P>(P::add(P::add(tot[0], tot[1]), P::add(tot[2], tot[3])));
-                } else {
-                    const int il = lastrel >> 10, rl = (lastrel >> 5) & 31, pos = lastrel & 31;
-                    Acc after = Acc(0), totl = tot[0];
-#pragma unroll
-                    for (int i = 0; i < PIECES_PER_SPAN; ++i) {
-                        if (i > il) after = P::add(after, tot[i]);
-                        if (i == il) totl = tot[i];
-                    }
-                    if (static_cast<int>(lane) > rl) after = P::add(after, totl);
-                    after = warp_sum<P>(after);
-                    Acc before = Acc(0);
-                    if (pos > 0) {
-                        before = P::from_bits(tmem_ld_32x1(taddr + il * ROW + (pos - 1)));
-                        tmem_ld_wait();
-                    }
-                    tail = P::add(__shfl_sync(0xffffffffu, P::sub(totl, before), rl), after);
-                }
-                if (lane == 0)
-                    st_relaxed_gpu_u64(prm.status + s,
-                                       pack_status((lastrel >= 0 || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail)));
-                tail_pre = tail;
+            Acc tot[PIECES_PER_SPAN];
+            Acc run = Acc(0);              // sum of the open segment inside this span so far
+            long long def_r = -1;          // segment that began before the span and ends inside it
+            Acc def_val = Acc(0);
+            // the span's aggregate: published before the boundaries are worked through, kept for the siblings
+            auto publish = [&](Acc tail) {
                 if (lane == 0) {
-                    agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + w] = (static_cast<uint64_t>(lastrel >= 0 ? 1u : 0u) << 32) | P::to_bits(tail);
+                    st_relaxed_gpu_u64(prm.status + s, pack_status((seen || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail)));
+                    agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + w] = (static_cast<uint64_t>(seen ? 1u : 0u) << 32) | P::to_bits(tail);
                     mbar_arrive(&bar_agg[g]);
                 }
                 // the first window beyond the tile travels while the boundaries are processed
-                if (tile != 0 && lastrel < 0) lookback_load<1>(prm.status, s - w - 1, lbw);
+                if (tile != 0 && !seen) lookback_load<1>(prm.status, s - w - 1, lbw);
                 if (pending) lookback_load<1>(prm.status, pend_s - w - 1, plw);
-            }
-            // direct sums: the first 32 boundaries' values have arrived by now; the others (spans with
-            // more than 32 boundaries) are fetched here, all at once
-            const Acc dval = isdir[0] ? window_sum<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), win0) : Acc(0);
-            dvt[lane] = dval;
-            if (!covers) {
-                ValueWindow wn[3];
-#pragma unroll
-                for (int j = 1; j < 4; ++j) {
-                    wn[j - 1].wide = false;
-                    if (isdir[j]) window_load<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), prm.n, wn[j - 1]);
-                }
-#pragma unroll
-                for (int j = 1; j < 4; ++j)
-                    dvt[lane + 32 * j] = isdir[j] ? window_sum<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), wn[j - 1]) : Acc(0);
-            }
-            __syncwarp();
-
-            MMV_T_MARK(2)
-            Acc run = Acc(0);              // sum of the open segment inside this span so far
-            const bool seen = lastrel >= 0;   // a segment start lies inside this span
-            long long def_r = -1;          // segment that began before the span and ends inside it
-            Acc def_val = Acc(0);
-            // number of boundaries with sbase <= bnd <= send (a prefix of the cache lanes)
-            const int nb_span = __popc(__ballot_sync(0xffffffffu, (cq + lane < nq) && (cb >= 0) && (cb <= send)));
-            const bool sparse = covers && nb_span <= SUM_SPARSE_MAX;
+            };
             if (sparse) {
-                // ---- few boundaries: no copy of the prefixes; the one prefix each boundary needs is read
-                //      straight from TMEM (one column, the lane of its row) ----
-                run = tail_pre;               // the open segment's sum at the end of the span
+                // ---- few boundaries (lane j <-> boundary j): the one prefix each boundary needs is read
+                //      straight from TMEM (one column; it sits in the lane of its row), together with the
+                //      row totals (column 31), with a single wait ----
+                const int crel = static_cast<int>(cb - sbase);          // 0..SPAN for lanes < nb_span
                 uint32_t vv[SUM_SPARSE_MAX];
+#pragma unroll
+                for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * ROW + (ROW - 1)));
 #pragma unroll
                 for (int j = 0; j < SUM_SPARSE_MAX; ++j) {
                     vv[j] = 0u;
                     if (j < nb_span) {
-                        const int e = static_cast<int>(__shfl_sync(0xffffffffu, cb, j) - 1 - sbase);   // element before the boundary
+                        const int e = __shfl_sync(0xffffffffu, crel, j) - 1;                 // element before the boundary
                         if (e >= 0) vv[j] = tmem_ld_32x1(taddr + (e >> 10) * ROW + (e & 31));
                     }
                 }
                 tmem_ld_wait();
+                MMV_T_MARK(12)
                 // exclusive prefix of the 128 row totals of the span (four interleaved warp scans)
                 Acc inc[PIECES_PER_SPAN];
 #pragma unroll
@@ -614,31 +588,51 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                         if (static_cast<int>(lane) >= o) inc[i] = P::add(t, inc[i]);
                     }
                 }
-                Acc pbase_acc = Acc(0), rowpre_span[PIECES_PER_SPAN];
+                Acc span_total = Acc(0), rowpre_span[PIECES_PER_SPAN];
 #pragma unroll
                 for (int i = 0; i < PIECES_PER_SPAN; ++i) {
-                    rowpre_span[i] = P::add(pbase_acc, P::sub(inc[i], tot[i]));
-                    pbase_acc = P::add(pbase_acc, __shfl_sync(0xffffffffu, inc[i], 31));
+                    rowpre_span[i] = P::add(span_total, P::sub(inc[i], tot[i]));
+                    span_total = P::add(span_total, __shfl_sync(0xffffffffu, inc[i], 31));
                 }
-                // lane j keeps, for boundary j: the prefix inside its row, the prefix of the rows before, the row
+                MMV_T_MARK(13)
+                // lane j fetches, for its boundary: the prefix inside the row and the prefix of the rows before
+                const int e = crel - 1;
+                const bool have = static_cast<int>(lane) < nb_span && e >= 0;
+                const int myrow = have ? (e >> 5) : -1;                  // row inside the span (0..127)
+                const int src = have ? (myrow & 31) : 0;
                 Acc mylocal = Acc(0), myrp = Acc(0);
-                int myrow = -1;
 #pragma unroll
                 for (int j = 0; j < SUM_SPARSE_MAX; ++j) {
-                    if (j < nb_span) {
-                        const int e = static_cast<int>(__shfl_sync(0xffffffffu, cb, j) - 1 - sbase);
-                        if (e >= 0) {
-                            const int piece = e >> 10, row = (e >> 5) & 31;
-                            Acc rsel = rowpre_span[0];
-#pragma unroll
-                            for (int i = 1; i < PIECES_PER_SPAN; ++i)
-                                if (piece == i) rsel = rowpre_span[i];
-                            const Acc lj = P::from_bits(__shfl_sync(0xffffffffu, vv[j], row));
-                            const Acc rj = __shfl_sync(0xffffffffu, rsel, row);
-                            if (static_cast<int>(lane) == j) { mylocal = lj; myrp = rj; myrow = e >> 5; }
-                        }
-                    }
+                    const uint32_t t = __shfl_sync(0xffffffffu, vv[j], src);
+                    if (static_cast<int>(lane) == j) mylocal = P::from_bits(t);
                 }
+#pragma unroll
+                for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                    const Acc t = __shfl_sync(0xffffffffu, rowpre_span[i], src);
+                    if ((e >> 10) == i) myrp = t;
+                }
+                if (!have) { mylocal = Acc(0); myrp = Acc(0); }
+                // the span's aggregate = sum of the segment open at its end
+                Acc tail = span_total;
+                if (seen) {
+                    // the last start is the last boundary below the span's end: lane jl
+                    const int jl = __popc(__ballot_sync(0xffffffffu, static_cast<int>(lane) < nb_span && crel < SPAN)) - 1;
+                    const int il = lastrel >> 10, rl = (lastrel >> 5) & 31, pos = lastrel & 31;
+                    Acc after = Acc(0), totl = tot[0];
+#pragma unroll
+                    for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                        if (i > il) after = P::add(after, tot[i]);
+                        if (i == il) totl = tot[i];
+                    }
+                    if (static_cast<int>(lane) > rl) after = P::add(after, totl);
+                    after = warp_sum<P>(after);
+                    const Acc before = (pos > 0) ? __shfl_sync(0xffffffffu, mylocal, jl & 31) : Acc(0);
+                    tail = P::add(P::sub(__shfl_sync(0xffffffffu, totl, rl), before), after);
+                }
+                publish(tail);
+                run = tail;
+                MMV_T_MARK(2)
+                const Acc dval = isdir[0] ? window_sum<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), win0) : Acc(0);
                 const Acc plocal = __shfl_up_sync(0xffffffffu, mylocal, 1);
                 const Acc prp = __shfl_up_sync(0xffffffffu, myrp, 1);
                 const int prow = __shfl_up_sync(0xffffffffu, myrow, 1);
@@ -667,11 +661,54 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 }
                 const unsigned dm = __ballot_sync(0xffffffffu, deferred);
                 if (dm) {
-                    const int src = __ffs(dm) - 1;
-                    def_r = cq + src - 1;
-                    def_val = __shfl_sync(0xffffffffu, val, src);
+                    const int srcl = __ffs(dm) - 1;
+                    def_r = cq + srcl - 1;
+                    def_val = __shfl_sync(0xffffffffu, val, srcl);
                 }
                 MMV_T_MARK(5)
+            } else {
+                // ---- general path: row totals, pre-pass, table of direct sums ----
+#pragma unroll
+                for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * ROW + (ROW - 1)));
+                tmem_ld_wait();
+                MMV_T_MARK(11)
+                Acc tail;
+                if (!seen) {
+                    tail = warp_sum<P>(P::add(P::add(tot[0], tot[1]), P::add(tot[2], tot[3])));
+                } else {
+                    const int il = lastrel >> 10, rl = (lastrel >> 5) & 31, pos = lastrel & 31;
+                    Acc after = Acc(0), totl = tot[0];
+#pragma unroll
+                    for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                        if (i > il) after = P::add(after, tot[i]);
+                        if (i == il) totl = tot[i];
+                    }
+                    if (static_cast<int>(lane) > rl) after = P::add(after, totl);
+                    after = warp_sum<P>(after);
+                    Acc before = Acc(0);
+                    if (pos > 0) {
+                        before = P::from_bits(tmem_ld_32x1(taddr + il * ROW + (pos - 1)));
+                        tmem_ld_wait();
+                    }
+                    tail = P::add(__shfl_sync(0xffffffffu, P::sub(totl, before), rl), after);
+                }
+                publish(tail);
+                // direct sums: the first 32 boundaries' values have arrived by now; the others (spans with
+                // more than 32 boundaries) are fetched here, all at once
+                dvt[lane] = isdir[0] ? window_sum<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), win0) : Acc(0);
+                if (!covers) {
+                    ValueWindow wn[3];
+#pragma unroll
+                    for (int j = 1; j < 4; ++j) {
+                        wn[j - 1].wide = false;
+                        if (isdir[j]) window_load<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), prm.n, wn[j - 1]);
+                    }
+#pragma unroll
+                    for (int j = 1; j < 4; ++j)
+                        dvt[lane + 32 * j] = isdir[j] ? window_sum<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), wn[j - 1]) : Acc(0);
+                }
+                __syncwarp();
+                MMV_T_MARK(2)
             }
 #pragma unroll 1
             for (int i = 0; i < (sparse ? 0 : PIECES_PER_SPAN); ++i) {
@@ -805,11 +842,12 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
             MMV_T_MARK(6)
             // request the next tile's offsets (its first index has arrived by now)
-            if (tile_n >= 0) load_offsets(q_next, qe_next, nraw, nrawp, nlast);
+            if (tile_n >= 0) load_offsets(q_next, qe_next, nraw, nrawp, nlast, nlast_ok);
             // Every warp waits on every phase of bar_agg (parity waits must not skip phases).  The carry
             // into this span is first sought among the tile's earlier spans (shared memory); only if
             // none of them holds a segment start does the look-back go out to the other CTAs' words.
             if (!wait_bar(&bar_agg[g], k & 1, abort_flag, budget)) { failed = true; break; }
+            MMV_T_MARK(14)
             // the segment parked at this warp's previous tile: its look-back window was requested during
             // this tile's pre-pass, so the predecessor's word has normally arrived
             if (pending) {
@@ -818,6 +856,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (lane == 0) outp[pend_r] = P::add(P::add(carry_out, pend_ex), pend_val);
                 pending = false;
             }
+            MMV_T_MARK(15)
             if (s == 0) {
                 if (def_r >= 0 && lane == 0) outp[def_r] = def_val;
             } else if (!seen || def_r >= 0) {
