@@ -298,6 +298,46 @@ def bench_configs(torch, mmv, oracle, peak, steps, warmup, l2_flush):
         {"segments": nseg, "worst_err_over_bound": ratio})
     del xd, od, out, ws
 
+    # the same recipe four times larger (the n >= 2^28 point of the target), and the flag-encoded
+    # form of the segmented sum over the same segments (start flags instead of offsets)
+    x, off = gen.config2(1 << 28)
+    n, nseg = x.shape[0], off.shape[0] - 1
+    xd, od = torch.from_numpy(x).cuda(), torch.from_numpy(off).cuda()
+    out = torch.empty(nseg, dtype=torch.float32, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, n, nseg)
+    fn = lambda: mmv.seg_sum(xd, od, out=out, workspace=ws)  # noqa: E731
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ms = event_time_ms(torch, fn, steps)
+    assert mmv.last_async_status(ws) == 0
+    want, a = oracle.seg_sum_csr_f16(x, off)
+    ok, ratio, i = oracle.check_fp(out.cpu().numpy(), want, a)
+    if not ok:
+        raise SystemExit(f"bench: config 2 (n = 2^28) outside the bound: ratio {ratio} at segment {i}")
+    rec("C2x4 seg-sum n=2^28 fp16 N(0,1), CSR offsets len U{1..4096}", n, 2 * n + 4 * (nseg + 1) + 4 * nseg, ms,
+        {"segments": nseg, "worst_err_over_bound": ratio})
+    del od, ws
+    f = gen.start_flags_of_offsets(off, n)
+    fd = torch.from_numpy(f).cuda()
+    outf = torch.empty(n, dtype=torch.float32, device="cuda")
+    kd = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+    fn = lambda: mmv.seg_sum(xd, fd, out=outf, num_segments=kd, workspace=ws)  # noqa: E731
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ms = event_time_ms(torch, fn, steps)
+    assert mmv.last_async_status(ws) == 0
+    k = int(kd.item())
+    wantf, af = oracle.seg_sum_flags_f16(x, f)
+    ok, ratio, i = oracle.check_fp(outf[:k].cpu().numpy(), wantf, af) if k == wantf.shape[0] else (False, float("inf"), -1)
+    if not ok:
+        raise SystemExit(f"bench: flag-form seg-sum outside the bound: ratio {ratio} at segment {i} (K = {k})")
+    rec("N1 seg-sum (start flags) n=2^28 fp16 N(0,1), same segments as C2x4", n, 2 * n + n + 4 * k, ms,
+        {"segments": k, "worst_err_over_bound": ratio})
+    del xd, fd, out, outf, ws
+
     x, f = gen.config3()
     run_scan("C3 seg-scan n=2^28 int8 flags 1e-3", x, f)
 

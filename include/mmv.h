@@ -100,8 +100,12 @@ mmv_status mmv_seg_scan(const void *x, const void *seg, mmv_segfmt sf, int64_t n
  * ignored; requires 0 <= off[0] and off[nseg] <= n.  d_num_segments is ignored
  * (may be NULL).
  * Flags form: out has capacity n; the K = 1 + #{i >= 1 : flag[i] != 0} segment
- * sums are written in segment order and K is written to *d_num_segments
- * (device pointer, int64) when it is not NULL.
+ * sums are written in segment order, nothing beyond out[K-1] is touched, and K
+ * is written to *d_num_segments (device pointer, int64, 8-byte aligned) when it
+ * is not NULL.  The start flags are first compacted into K + 1 offsets inside
+ * the workspace (COMPRESS, Section 2; the compaction step of Algorithm 4.2),
+ * which therefore holds 4 (n + 1) bytes more than for the offsets form; nseg is
+ * ignored.  n < 2^31 in both forms.
  */
 mmv_status mmv_seg_sum(const void *x, const void *seg, mmv_segfmt sf, int64_t n, int64_t nseg,
                        mmv_dtype dt, void *out, int64_t *d_num_segments,

@@ -153,6 +153,15 @@ def offsets_from_lengths(lens: np.ndarray) -> np.ndarray:
     return off.astype(np.int32)
 
 
+def start_flags_of_offsets(off: np.ndarray, n: int) -> np.ndarray:
+    """The same segments as start flags: byte i is 1 iff a non-empty segment starts at i."""
+    off = np.asarray(off, np.int64)
+    f = np.zeros(n, np.uint8)
+    starts = off[:-1][off[1:] > off[:-1]]
+    f[starts] = 1
+    return f
+
+
 def csr_matrix(config: int, rows: int, cols: int, s: float = 1.5, cap: int = 10_000,
                empty_fraction: float = 0.0):
     """(rowptr int32, col int32, val fp16, x fp32) of a random CSR matrix.

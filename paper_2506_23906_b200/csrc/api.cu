@@ -12,6 +12,7 @@
 #include "common.cuh"
 #include "seg_scan.cuh"
 #include "seg_sum.cuh"
+#include "compress.cuh"
 
 namespace mmv {
 namespace {
@@ -120,6 +121,8 @@ struct WorkspacePlan {
     size_t flags_off, flags_bytes;     // scratch flag bytes (offset-encoded scan only)
     size_t tileq_off, tileq_bytes;     // per-tile first boundary index (seg-sum, SpMV)
     size_t prod_off, prod_bytes;       // bf16 hi/lo halves of the products (SpMV)
+    size_t cmp_off, cmp_bytes;         // flag-encoded seg-sum: chunk counts, chunk bases, segment count
+    size_t off_off, off_bytes;         // flag-encoded seg-sum: the compacted offsets (n + 1 entries at most)
     long long n_eff;                   // elements the tiled kernel runs over
     size_t total;
 };
@@ -140,7 +143,13 @@ WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     p.tileq_bytes = (op != MMV_OP_SEG_SCAN) ? round_up(static_cast<size_t>(tiles * SPANS_PER_TILE + 1) * sizeof(int32_t), 256) : 0;
     p.prod_off = p.tileq_off + p.tileq_bytes;
     p.prod_bytes = (op == MMV_OP_SPMV_CSR) ? round_up(static_cast<size_t>(n) * 4, 256) : 0;
-    p.total = p.prod_off + p.prod_bytes;
+    const bool flagsum = op == MMV_OP_SEG_SUM && sf == MMV_SEG_FLAGS_U8;
+    const long long nchunks = (n + CMP_CHUNK - 1) / CMP_CHUNK;
+    p.cmp_off = p.prod_off + p.prod_bytes;
+    p.cmp_bytes = flagsum ? round_up(static_cast<size_t>(2 * nchunks) * sizeof(int32_t) + 16, 256) : 0;
+    p.off_off = p.cmp_off + p.cmp_bytes;
+    p.off_bytes = flagsum ? round_up(static_cast<size_t>(n + 1) * sizeof(int32_t), 256) : 0;
+    p.total = p.off_off + p.off_bytes;
     return p;
 }
 
@@ -184,7 +193,8 @@ __global__ void spmv_gather_kernel(const int32_t* __restrict__ col, const __half
 // cleared on the stream already.
 template <typename P>
 mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* off, long long nseg, int shift,
-                          void* out, uint8_t* ws, const WorkspacePlan& plan, DeviceInfo* dev, cudaStream_t st) {
+                          void* out, uint8_t* ws, const WorkspacePlan& plan, DeviceInfo* dev, cudaStream_t st,
+                          const long long* nseg_dev = nullptr) {
     const int tiles = static_cast<int>(num_tiles_of(n_eff));
     int32_t* span_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
     {
@@ -193,7 +203,7 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
         const int threads = 256;
         const long long blocks = (warps * 32 + threads - 1) / threads;
         partition_offsets_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, shift, spans, span_q, n_eff,
-                                                                                 reinterpret_cast<WorkspaceHeader*>(ws));
+                                                                                 reinterpret_cast<WorkspaceHeader*>(ws), nseg_dev);
         ++g_launches;
     }
     CUtensorMap tmap;
@@ -209,6 +219,7 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     prm.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();
+    prm.nseg_dev = nseg_dev;
     const int grid = tiles < dev->sm_count ? tiles : dev->sm_count;
     seg_sum_kernel<P><<<grid, SUM_THREADS, SumCfg<P>::kSmemBytes, st>>>(tmap, values, prm);
     ++g_launches;
@@ -334,12 +345,45 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
 mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
                        void* out, int64_t* d_num_segments, void* workspace, size_t workspace_bytes,
                        void* cuda_stream) {
-    (void)d_num_segments;
     if (n < 0 || nseg < 0) return MMV_ERR_INVALID_ARG;
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
-    if (sf == MMV_SEG_FLAGS_U8) return MMV_ERR_UNSUPPORTED;
     if (n >= (1ll << 31)) return MMV_ERR_INVALID_ARG;            // int32 offsets cannot address more
+    if (sf == MMV_SEG_FLAGS_U8) {
+        // COMPRESS the start flags into offsets (in the workspace), then the offset-encoded kernel with
+        // the segment count read on the device.
+        cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+        if (n == 0) {
+            if (d_num_segments && cudaMemsetAsync(d_num_segments, 0, sizeof(int64_t), st) != cudaSuccess) return MMV_ERR_CUDA;
+            return MMV_OK;
+        }
+        if (!x || !seg || !out || !workspace) return MMV_ERR_INVALID_ARG;
+        if (!aligned16(x) || !aligned16(seg) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+            return MMV_ERR_INVALID_ARG;
+        if (d_num_segments && (reinterpret_cast<uintptr_t>(d_num_segments) & 7u)) return MMV_ERR_INVALID_ARG;
+        const WorkspacePlan plan = plan_workspace(MMV_OP_SEG_SUM, sf, n);
+        if (workspace_bytes < plan.total) return MMV_ERR_WORKSPACE_TOO_SMALL;
+        DeviceInfo* dev = device_info();
+        if (!dev) return MMV_ERR_CUDA;
+        uint8_t* ws = static_cast<uint8_t*>(workspace);
+        if (cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
+        const long long nchunks = (n + CMP_CHUNK - 1) / CMP_CHUNK;
+        long long* nseg_dev = reinterpret_cast<long long*>(ws + plan.cmp_off);
+        int32_t* chunk_count = reinterpret_cast<int32_t*>(ws + plan.cmp_off + 16);
+        int32_t* chunk_base = chunk_count + nchunks;
+        int32_t* off = reinterpret_cast<int32_t*>(ws + plan.off_off);
+        const uint8_t* f = static_cast<const uint8_t*>(seg);
+        const long long cap = static_cast<long long>(dev->sm_count) * 8;
+        const unsigned blocks = static_cast<unsigned>(nchunks < cap ? nchunks : cap);
+        flag_count_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_count);
+        chunk_scan_kernel<<<1, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, nseg_dev,
+                                              reinterpret_cast<long long*>(d_num_segments), off, n);
+        flag_scatter_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_base, off);
+        g_launches += 3;
+        if (cudaGetLastError() != cudaSuccess) return MMV_ERR_CUDA;
+        if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev);
+        return launch_seg_sum<I8Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev);
+    }
     if (nseg == 0) return MMV_OK;
     if (!seg || !out) return MMV_ERR_INVALID_ARG;
     if (!aligned16(seg) || !aligned16(out)) return MMV_ERR_INVALID_ARG;

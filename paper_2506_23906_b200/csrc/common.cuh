@@ -214,6 +214,9 @@ __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, ty
             }
             idx -= 32 * W;
             t0 = global_timer_ns();
+#ifdef MMV_PHASE_TIMERS
+            if (lane == 0) atomicAdd(&g_phase_cycles[14], 1ull);  // windows walked past
+#endif
         } else {
             if ((++polls & 7u) == 0u) {
                 if (*abort_flag) return false;
@@ -221,6 +224,9 @@ __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, ty
             }
             __nanosleep(40);        // keep the polling traffic in L2 small
         }
+#ifdef MMV_PHASE_TIMERS
+        if (lane == 0) atomicAdd(&g_phase_cycles[13], 1ull);      // polls after the first window
+#endif
         lookback_load<W>(status, idx, win);
     }
 }

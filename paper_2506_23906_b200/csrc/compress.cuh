@@ -1,0 +1,139 @@
+// COMPRESS of the segment-start flags (Section 2; the compaction step of Algorithm 4.2):
+// the positions of the start flags, in order, are exactly the CSR offsets of the segments,
+//     off[r] = position of the r-th start,   off[K] = n,   K = 1 + #{i >= 1 : f(i) != 0},
+// so the flag-encoded segmented sum is this compaction followed by the offset-encoded kernel.
+// Three small streaming kernels: per-chunk counts, one-block exclusive scan of the counts,
+// in-order scatter of the positions.  Element 0 always starts a segment, whatever f(0) holds.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mmv {
+
+constexpr int CMP_THREADS = 256;
+constexpr int CMP_PER_THREAD = 64;                              // flag bytes per thread: four 16-byte vectors
+constexpr int CMP_CHUNK = CMP_THREADS * CMP_PER_THREAD;         // 16384 flags per block iteration
+
+// number of non-zero bytes of a word
+__device__ __forceinline__ int nonzero_bytes(uint32_t w) {
+    return __popc((((w & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w) & 0x80808080u);
+}
+
+// The 64 flag bytes of thread t of chunk c as 16 words (zero past n; byte 0 of the vector forced to 1).
+__device__ __forceinline__ void load_thread_flags(const uint8_t* __restrict__ f, long long n, long long base, uint32_t (&w)[16]) {
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+        const long long p = base + 16 * v;
+        uint4 q = make_uint4(0u, 0u, 0u, 0u);
+        if (p + 16 <= n) {
+            q = *reinterpret_cast<const uint4*>(f + p);
+        } else if (p < n) {
+            uint32_t t[4] = {0u, 0u, 0u, 0u};
+            for (int b = 0; b < 16 && p + b < n; ++b) t[b >> 2] |= static_cast<uint32_t>(f[p + b]) << (8 * (b & 3));
+            q = make_uint4(t[0], t[1], t[2], t[3]);
+        }
+        w[4 * v] = q.x;
+        w[4 * v + 1] = q.y;
+        w[4 * v + 2] = q.z;
+        w[4 * v + 3] = q.w;
+    }
+    if (base == 0) w[0] |= 1u;          // element 0 starts the first segment
+}
+
+// Exclusive scan of one int per thread over the block; returns this thread's offset, *total = block sum.
+__device__ __forceinline__ int block_exclusive_scan(int v, int* total, int* warp_sums /* >= 32 ints of shared memory */) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        int s = lane < nwarps ? warp_sums[lane] : 0;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, s, o);
+            if (lane >= o) s += t;
+        }
+        warp_sums[lane] = s;            // inclusive over warps
+    }
+    __syncthreads();
+    const int before = warp ? warp_sums[warp - 1] : 0;
+    *total = warp_sums[nwarps - 1];
+    __syncthreads();                    // warp_sums may be reused by the caller's next round
+    return before + inc - v;
+}
+
+// chunk_count[c] = number of segment starts among the flags of chunk c.
+__global__ void __launch_bounds__(CMP_THREADS)
+flag_count_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks, int32_t* __restrict__ chunk_count) {
+    __shared__ int warp_sums[32];
+    for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
+        uint32_t w[16];
+        load_thread_flags(f, n, c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD, w);
+        int cnt = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) cnt += nonzero_bytes(w[i]);
+        int total;
+        block_exclusive_scan(cnt, &total, warp_sums);
+        if (threadIdx.x == 0) chunk_count[c] = total;
+    }
+}
+
+// One block: chunk_base = exclusive scan of chunk_count; K = total is written to nseg_dev and, when given,
+// to the caller's d_num_segments; off[K] = n closes the last segment.
+__global__ void __launch_bounds__(1024)
+chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, int32_t* __restrict__ chunk_base,
+                  long long* __restrict__ nseg_dev, long long* __restrict__ d_num_segments, int32_t* __restrict__ off,
+                  long long n) {
+    __shared__ int warp_sums[32];
+    const long long per = (nchunks + blockDim.x - 1) / blockDim.x;
+    const long long lo = static_cast<long long>(threadIdx.x) * per;
+    const long long hi = lo + per < nchunks ? lo + per : nchunks;
+    int local = 0;
+    for (long long c = lo; c < hi; ++c) local += chunk_count[c];
+    int total;
+    int run = block_exclusive_scan(local, &total, warp_sums);
+    for (long long c = lo; c < hi; ++c) {
+        chunk_base[c] = run;
+        run += chunk_count[c];
+    }
+    if (threadIdx.x == 0) {
+        *nseg_dev = total;
+        if (d_num_segments) *d_num_segments = total;
+        off[total] = static_cast<int32_t>(n);
+    }
+}
+
+// off[chunk_base[c] + j] = position of the j-th start flag of chunk c (in order).
+__global__ void __launch_bounds__(CMP_THREADS)
+flag_scatter_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks, const int32_t* __restrict__ chunk_base,
+                    int32_t* __restrict__ off) {
+    __shared__ int warp_sums[32];
+    for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
+        const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
+        uint32_t w[16];
+        load_thread_flags(f, n, base, w);
+        int cnt = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) cnt += nonzero_bytes(w[i]);
+        int total;
+        int slot = chunk_base[c] + block_exclusive_scan(cnt, &total, warp_sums);
+        if (cnt) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                uint32_t m = (((w[i] & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w[i]) & 0x80808080u;     // bit 8b+7 set: byte b non-zero
+                while (m) {
+                    const int b = (__ffs(m) - 1) >> 3;
+                    off[slot++] = static_cast<int32_t>(base + 4 * i + b);
+                    m &= m - 1;
+                }
+            }
+        }
+    }
+}
+
+}  // namespace mmv

@@ -573,6 +573,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             // its siblings through shared memory (they have passed bar_agg of this tile, so the previous
             // phase of bar_carry is complete and the parity wait cannot alias).
             Acc carry = ex;
+            MMV_T_MARK(8)
             if (w == 0) {
                 Acc carry_tile = Acc(0);
                 if (tile != 0) {
@@ -589,9 +590,11 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                     mbar_arrive(&bar_carry[g]);
                 }
                 carry = carry_tile;
+                MMV_T_MARK(10)
             } else if (need_global) {
                 if (!wait_bar(&bar_carry[g], k & 1, abort_flag, budget)) { failed = true; break; }
                 carry = P::add(P::from_bits(carry_slot[g]), ex);
+                MMV_T_MARK(9)
             }
 
             // ---- parked pieces: add the carry in front of the unit's first flag, store ----

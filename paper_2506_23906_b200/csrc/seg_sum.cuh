@@ -180,6 +180,8 @@ struct SumParams {
     WorkspaceHeader* hdr;
     uint64_t* status;
     unsigned long long budget_ns;
+    const long long* nseg_dev;   // when not null: the number of segments is read from here (flag-encoded
+                                 // segments, whose count is only known on the device); nseg is ignored
 };
 
 // span_q[s] = first index q in [0, nseg] with (off[q] << shift) >= s * SPAN, nseg + 1 if none.
@@ -187,7 +189,9 @@ struct SumParams {
 // inside [0, n]) and records MMV_ERR_BAD_SEGMENTS otherwise; the main kernel never indexes
 // outside its tile whatever they hold.
 __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, int shift, long long num_spans,
-                                         int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr) {
+                                         int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr,
+                                         const long long* __restrict__ nseg_dev) {
+    if (nseg_dev) nseg = *nseg_dev;
     {
         const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
         bool bad = false;
@@ -411,7 +415,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         int32_t* tbl = reinterpret_cast<int32_t*>(smem + Cfg::kTblOffset + warp * SUM_TBL_BYTES);   // [0] = offset before the first
         Acc* dvt = reinterpret_cast<Acc*>(tbl + SUM_TBL + 4);
         const int sh = prm.off_shift;
-        const long long nq = prm.nseg + 1;
+        const long long nq = (prm.nseg_dev ? *prm.nseg_dev : prm.nseg) + 1;
         bool failed = false;
         // inclusive prefix inside the piece at element offset j (0..1023)
         auto piece_prefix = [&](int j, Acc& rowpart, int& row) -> Acc {

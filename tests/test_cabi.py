@@ -73,6 +73,7 @@ def test_argument_errors_are_synchronous(lib):
     assert lib.mmv_seg_scan(16, 16, 0, 8, 0, 0, 16, 256, 16, None) == 3             # workspace too small
     assert lib.mmv_seg_sum(None, None, 1, 0, 0, 0, None, None, None, 0, None) == 0  # nothing to do
     assert lib.mmv_seg_sum(16, 16, 1, -5, 1, 0, 16, None, 256, 4096, None) == 1
-    assert lib.mmv_seg_sum(16, 16, 0, 8, 0, 0, 16, None, 256, 4096, None) == 2      # flag form: not implemented
+    assert lib.mmv_seg_sum(16, 16, 0, 8, 0, 0, 16, None, 256, 16, None) == 3        # flag form: workspace too small
+    assert lib.mmv_seg_sum(16, 16, 0, 8, 0, 0, 16, 12, 256, 1 << 20, None) == 1     # misaligned segment counter
     assert lib.mmv_spmv_csr(None, None, None, None, None, -1, 1, 1, None, 0, None) == 1
     assert lib.mmv_spmv_csr(None, None, None, None, None, 0, 1, 0, None, 0, None) == 0

@@ -235,6 +235,46 @@ def test_seg_sum_config2_reduced(mmv):
 
 
 # ---------------------------------------------------------------------------
+# segmented sum over start flags (COMPRESS of the flags, then the offset kernel)
+# ---------------------------------------------------------------------------
+def sum_flags(mmv, x, f, guard=16):
+    n = x.shape[0]
+    dt = mmv.F16_TO_F32 if x.dtype == np.float16 else mmv.I8_TO_I32
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, dt, mmv.SEG_FLAGS_U8, n)
+    tdt = torch.float32 if x.dtype == np.float16 else torch.int32
+    buf = torch.full((n + guard,), -777, dtype=tdt, device="cuda")
+    k = torch.full((1,), -1, dtype=torch.int64, device="cuda")
+    mmv.seg_sum(dev(x), dev(f), out=buf[:n], num_segments=k, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    got, kk = buf.cpu().numpy(), int(k.item())
+    assert (got[kk:] == -777).all()          # nothing beyond the K sums is written
+    return got[:kk]
+
+
+@pytest.mark.parametrize("n,p", [(1, 0.5), (31, 0.3), (4097, 0.01), (3 * TILE + 777, 0.0), (3 * TILE + 777, 1e-3),
+                                 (5 * TILE + 13, 0.2), (2 * TILE, 1.0), ((1 << 22) + 5, 1e-4), ((1 << 21) + 99, 0.6)])
+def test_seg_sum_flags(mmv, n, p):
+    rng = np.random.default_rng(int(n * 7 + p * 1000))
+    f = (rng.random(n) < p).astype(np.uint8) * rng.integers(1, 256, n).astype(np.uint8)   # any non-zero byte counts
+    x = rng.integers(-128, 128, n).astype(np.int8)
+    want = oracle.seg_sum_flags_i8(x, f)
+    got = sum_flags(mmv, x, f)
+    assert got.shape == want.shape and np.array_equal(got, want)
+    xf = rng.standard_normal(n).astype(np.float16)
+    wantf, a = oracle.seg_sum_flags_f16(xf, f)
+    gotf = sum_flags(mmv, xf, f)
+    assert gotf.shape == wantf.shape
+    assert_fp(gotf, wantf, a, f"flag-form seg-sum n={n} p={p}")
+
+
+def test_seg_sum_flags_matches_paper_example(mmv):
+    g = __import__("conftest").load_golden("sec2_worked_example.txt")
+    x = np.asarray(g["x"], np.int8)
+    f = np.asarray(g["f"], np.uint8)
+    assert sum_flags(mmv, x, f).tolist() == g["seg_sum"]
+
+
+# ---------------------------------------------------------------------------
 # CSR SpMV
 # ---------------------------------------------------------------------------
 def spmv(mmv, rowptr, col, val, x):

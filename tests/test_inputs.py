@@ -36,3 +36,11 @@ def test_config_shapes():
     assert col.shape[0] == val.shape[0] == rowptr[-1] and col.max() < 4096 and xv.dtype == np.float32
     rowptr, *_ = gen.config4(rows=4096, empty_fraction=0.1)
     assert 0.05 < (np.diff(rowptr) == 0).mean() < 0.15
+
+
+def test_start_flags_of_offsets_agree_with_the_oracle_encoding():
+    import oracle
+    off = np.asarray([0, 0, 3, 3, 7, 12, 12], np.int32)
+    f = gen.start_flags_of_offsets(off, 12)
+    assert f.tolist() == [1, 0, 0, 1, 0, 0, 0, 1, 0, 0, 0, 0]
+    assert np.array_equal(f, oracle.flags_from_offsets(off, 12))
