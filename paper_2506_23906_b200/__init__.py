@@ -25,7 +25,7 @@ OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR = 0, 1, 2
 EXPORTS = (
     "mmv_workspace_bytes", "mmv_seg_scan", "mmv_seg_sum", "mmv_spmv_csr",
     "mmv_last_async_status", "mmv_status_string", "mmv_kernel_launch_count", "mmv_debug_configure",
-    "mmv_seg_scan_static", "mmv_seg_scan_static_last_status",
+    "mmv_seg_scan_static", "mmv_seg_scan_static_last_status", "mmv_debug_force_sum_groups",
 )
 STATIC_SCAN_MAX_N = 1 << 28
 
@@ -39,7 +39,7 @@ class MmvError(RuntimeError):
 def _load() -> ctypes.CDLL:
     if not LIB_PATH.exists():
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2506_23906_b200.build` "
+            f"{LIB_PATH} is missing: build it with `python paper_2506_23906_b200/build.py` "
             "(nvcc, sm_100a).  There is no fallback path.")
     lib = ctypes.CDLL(str(LIB_PATH))
     vp, i64, sz, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t, ctypes.c_int
@@ -63,6 +63,8 @@ def _load() -> ctypes.CDLL:
     lib.mmv_seg_scan_static_last_status.argtypes = [vp]
     lib.mmv_debug_configure.restype = None
     lib.mmv_debug_configure.argtypes = [i64, i64]
+    lib.mmv_debug_force_sum_groups.restype = None
+    lib.mmv_debug_force_sum_groups.argtypes = [ci]
     return lib
 
 
@@ -79,6 +81,10 @@ def kernel_launch_count() -> int:
 
 def debug_configure(wait_budget_ns: int = 0, skip_publish_span: int = -1) -> None:
     _lib.mmv_debug_configure(int(wait_budget_ns), int(skip_publish_span))
+
+
+def debug_force_sum_groups(groups: int = 0) -> None:
+    _lib.mmv_debug_force_sum_groups(int(groups))
 
 
 def workspace_bytes(op: int, dt: int, sf: int, n: int, nseg: int = 0) -> int:

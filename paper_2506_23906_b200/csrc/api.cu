@@ -7,6 +7,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <mutex>
+#include <type_traits>
 
 #include "../../include/mmv.h"
 #include "common.cuh"
@@ -20,6 +21,7 @@ namespace {
 std::atomic<long long> g_launches{0};
 std::atomic<unsigned long long> g_budget_ns{WAIT_BUDGET_NS};
 std::atomic<long long> g_debug_skip_span{-1};
+std::atomic<int> g_force_groups{0};
 
 constexpr int kMaxDevices = 64;
 
@@ -64,9 +66,11 @@ DeviceInfo* device_info() {
         bool ok = true;
         ok &= set_smem(seg_scan_kernel<F16Path>, ScanCfg<F16Path>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<I8Path>, ScanCfg<I8Path>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<F16Path>, SumCfg<F16Path>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<I8Path>, SumCfg<I8Path>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<BF16Path>, SumCfg<BF16Path>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<F16Path, 2>, SumCfg<F16Path, 2>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<I8Path, 2>, SumCfg<I8Path, 2>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<BF16Path, 2>, SumCfg<BF16Path, 2>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<F16Path, 4>, SumCfg<F16Path, 4>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<I8Path, 4>, SumCfg<I8Path, 4>::kSmemBytes);
         d->ok = ok;
     });
     return d->ok ? d : nullptr;
@@ -221,7 +225,20 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     prm.budget_ns = g_budget_ns.load();
     prm.nseg_dev = nseg_dev;
     const int grid = tiles < dev->sm_count ? tiles : dev->sm_count;
-    seg_sum_kernel<P><<<grid, SUM_THREADS, SumCfg<P>::kSmemBytes, st>>>(tmap, values, prm);
+    // Long segments (few boundaries per 4096-element span): sixteen epilogue warps on the light path.
+    // The segment count of the flag-encoded form is not known here; it takes the eight-warp kernel.
+    bool many_warps = false;
+    if constexpr (!std::is_same<P, BF16Path>::value) many_warps = !nseg_dev && nseg > 0 && n_eff / nseg >= 256;
+    if (g_force_groups.load() == 2) many_warps = false;
+    if (g_force_groups.load() == 4 && !std::is_same<P, BF16Path>::value) many_warps = true;
+    if constexpr (!std::is_same<P, BF16Path>::value) {
+        if (many_warps) {
+            seg_sum_kernel<P, 4><<<grid, SumShape<4>::kThreads, SumCfg<P, 4>::kSmemBytes, st>>>(tmap, values, prm);
+            ++g_launches;
+            return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+        }
+    }
+    seg_sum_kernel<P, 2><<<grid, SumShape<2>::kThreads, SumCfg<P, 2>::kSmemBytes, st>>>(tmap, values, prm);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
@@ -520,6 +537,8 @@ void mmv_debug_phase_cycles(unsigned long long* host16) {
     cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z));
 }
 #endif
+
+void mmv_debug_force_sum_groups(int groups) { g_force_groups.store(groups == 2 || groups == 4 ? groups : 0); }
 
 void mmv_debug_configure(int64_t wait_budget_ns, int64_t skip_publish_span) {
     g_budget_ns.store(wait_budget_ns > 0 ? static_cast<unsigned long long>(wait_budget_ns) : WAIT_BUDGET_NS);

@@ -28,12 +28,22 @@
 
 namespace mmv {
 
-constexpr int SUM_EPI_WARPS = 8;
-constexpr int SUM_PRODUCER_WARP = 8;
-constexpr int SUM_MMA_WARP = 9;
-constexpr int SUM_THREADS = 320;
-constexpr int SUM_BUFS = 4;                                        // TMEM tile buffers: two per warpgroup
+// The kernel comes with G = 2 or 4 epilogue warpgroups (4 G epilogue warps, then the TMA producer
+// warp and the MMA warp).  The epilogue is a chain of dependent instructions per span, so its
+// throughput grows with the number of warps: G = 4 (16 epilogue warps, at most 112 registers) is
+// used when segments are long and the light few-boundaries path does the work, G = 2 (8 warps,
+// 168 registers, the MMA warp one tile ahead) when boundaries are dense.
+constexpr int SUM_BUFS = 4;                                        // TMEM tile buffers, shared out among the warpgroups
 constexpr int SUM_TMEM_COLS = SUM_BUFS * PIECES_PER_SPAN * ROW;    // 512
+template <int G>
+struct SumShape {
+    static_assert(G == 2 || G == 4, "two or four epilogue warpgroups");
+    static constexpr int kEpiWarps = 4 * G;
+    static constexpr int kProducerWarp = 4 * G;
+    static constexpr int kMmaWarp = 4 * G + 1;
+    static constexpr int kThreads = (4 * G + 2) * 32;
+    static constexpr int kBufsPerGroup = SUM_BUFS / G;
+};
 constexpr int SUM_SPARSE_MAX = 8;                                  // spans with at most this many boundaries read single prefixes from TMEM
 constexpr int SUM_DIRECT_LEN = 4;                                  // segments this short are summed from the inputs
 constexpr int SUM_TBL = 128;                                       // boundaries of a span kept in shared memory
@@ -154,7 +164,7 @@ __device__ __forceinline__ bool sum_lookback(const uint64_t* status, long long s
     return ok;
 }
 
-template <typename P>
+template <typename P, int G>
 struct SumCfg {
     static constexpr int kStages = 4;
     static constexpr int kBBytes = ROW * P::kRowBytes;               // constant U_32: 32 rows
@@ -162,9 +172,9 @@ struct SumCfg {
     static constexpr int kDumpBytes = PIECE * 4;                     // per epilogue warp
     static constexpr int kStageOffset = 2048;                        // after the constant operand
     static constexpr int kDumpOffset = kStageOffset + kStages * kXBytes;
-    static constexpr int kRowpreOffset = kDumpOffset + SUM_EPI_WARPS * kDumpBytes;
-    static constexpr int kTblOffset = kRowpreOffset + SUM_EPI_WARPS * PIECE_ROWS * 4;
-    static constexpr int kBarOffset = kTblOffset + SUM_EPI_WARPS * SUM_TBL_BYTES;
+    static constexpr int kRowpreOffset = kDumpOffset + SumShape<G>::kEpiWarps * kDumpBytes;
+    static constexpr int kTblOffset = kRowpreOffset + SumShape<G>::kEpiWarps * PIECE_ROWS * 4;
+    static constexpr int kBarOffset = kTblOffset + SumShape<G>::kEpiWarps * SUM_TBL_BYTES;
     static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
     static_assert(kBBytes <= 2048, "constant operand fits its slot");
 };
@@ -229,11 +239,13 @@ __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long l
     if (lane == 0) span_q[warp] = static_cast<int32_t>(lo);
 }
 
-template <typename P>
-__global__ void __launch_bounds__(SUM_THREADS, 1)
+template <typename P, int G>
+__global__ void __launch_bounds__(SumShape<G>::kThreads, 1)
 seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restrict__ xg, const SumParams prm) {
     using Acc = typename P::Acc;
-    using Cfg = SumCfg<P>;
+    using Cfg = SumCfg<P, G>;
+    using Shape = SumShape<G>;
+    constexpr int BPG = Shape::kBufsPerGroup;
     constexpr int S = Cfg::kStages;
 
     extern __shared__ uint8_t smem_raw[];
@@ -248,8 +260,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
     uint64_t* bar_agg = bar_acc_empty + SUM_BUFS;          // per warpgroup: its four span aggregates are in agg_slot
     // [group][tile parity][span]: (has start << 32) | open-segment sum.  Two sets, because a warp may
     // write its next tile's aggregate while a sibling still reads this tile's.
-    uint64_t* agg_slot = bar_agg + 2;
-    volatile long long* stage_info = reinterpret_cast<volatile long long*>(agg_slot + 2 * 2 * SPANS_PER_TILE);
+    uint64_t* agg_slot = bar_agg + G;
+    volatile long long* stage_info = reinterpret_cast<volatile long long*>(agg_slot + G * 2 * SPANS_PER_TILE);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<long long*>(stage_info) + S);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -263,7 +275,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             mbar_init(&bar_empty[i], 1);      // released by the MMA warp's commit
             stage_info[i] = -1;
         }
-        for (int i = 0; i < 2; ++i) mbar_init(&bar_agg[i], SPANS_PER_TILE);
+        for (int i = 0; i < G; ++i) mbar_init(&bar_agg[i], SPANS_PER_TILE);
         for (int i = 0; i < SUM_BUFS; ++i) {
             mbar_init(&bar_acc_full[i], 1);
             mbar_init(&bar_acc_empty[i], 4);
@@ -271,16 +283,16 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         *abort_flag = 0;
         mbar_fence_init();
     }
-    if (warp == SUM_MMA_WARP) {
+    if (warp == Shape::kMmaWarp) {
         tmem_alloc(tmem_slot, SUM_TMEM_COLS);
         tmem_relinquish();
     }
-    if (warp == SUM_PRODUCER_WARP && lane == 0) tma_prefetch_desc(&tmap_x);
+    if (warp == Shape::kProducerWarp && lane == 0) tma_prefetch_desc(&tmap_x);
     {
         // constant B = U_32 stored K-major: row nn (output position), element k (input position): 1 iff k <= nn
         constexpr int kVecPerRow = P::kRowBytes / 16;
         constexpr int kElemPerVec = 16 / P::kElemBytes;
-        for (int v = threadIdx.x; v < ROW * kVecPerRow; v += SUM_THREADS) {
+        for (int v = threadIdx.x; v < ROW * kVecPerRow; v += Shape::kThreads) {
             const int nn = v / kVecPerRow, cv = v % kVecPerRow;
             uint32_t words[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
@@ -301,7 +313,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == SUM_PRODUCER_WARP) {
+    if (warp == Shape::kProducerWarp) {
         // =========================== producer ===========================
         int it = 0, sentinels = 0;
         bool ok = true;
@@ -362,7 +374,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             if (lane == 0) report_error(prm.hdr, 5u);
         }
         for (int k = (it > S ? it - S : 0); k < it; ++k) mbar_wait(&bar_full[k % S], (k / S) & 1, 2000000ull);
-    } else if (warp == SUM_MMA_WARP) {
+    } else if (warp == Shape::kMmaWarp) {
         // =========================== MMA issuer (one tile ahead of the epilogue) ===========================
         constexpr uint32_t idesc = P::kIsFloat ? (make_idesc_f16_f32(128, ROW) | P::kFmtBits)
                                                : make_idesc_s8_s32(128, ROW);
@@ -378,9 +390,9 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (++sentinels == 2) break;
                 continue;
             }
-            const int g = it & 1, k = it >> 1;
-            const int buf = g * 2 + (k & 1);
-            if (!wait_bar(&bar_acc_empty[buf], ((k >> 1) & 1) ^ 1, abort_flag, budget)) {
+            const int g = it % G, k = it / G;
+            const int buf = g * BPG + (k % BPG);
+            if (!wait_bar(&bar_acc_empty[buf], ((k / BPG) & 1) ^ 1, abort_flag, budget)) {
                 *abort_flag = 1;
                 if (lane == 0) report_error(prm.hdr, 5u);
                 break;
@@ -428,7 +440,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         // offset index, then one offset per lane), so that their two dependent round trips never
         // sit on the critical path.
         auto tile_of = [&](int kk) -> int {
-            const int t = static_cast<int>(blockIdx.x) + (g + 2 * kk) * static_cast<int>(gridDim.x);
+            const int t = static_cast<int>(blockIdx.x) + (g + G * kk) * static_cast<int>(gridDim.x);
             return t < prm.num_tiles ? t : -1;
         };
         // raw offset -> position (index checks against nq are made where an entry is used)
@@ -475,7 +487,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             // tile order it knows its tile without being told
             const int tile = tile_of(k);
             if (tile < 0) break;
-            const int buf = g * 2 + (k & 1);
+            const int buf = g * BPG + (k % BPG);
             const long long s = static_cast<long long>(tile) * SPANS_PER_TILE + w;
             const long long sbase = s * SPAN;
             const long long send = sbase + SPAN;
@@ -542,7 +554,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             }
 
             MMV_T_MARK(0)
-            if (!wait_bar(&bar_acc_full[buf], (k >> 1) & 1, abort_flag, budget)) { failed = true; break; }
+            if (!wait_bar(&bar_acc_full[buf], (k / BPG) & 1, abort_flag, budget)) { failed = true; break; }
             tc_fence_after_sync();
             MMV_T_MARK(1)
 
@@ -917,7 +929,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == SUM_MMA_WARP) {
+    if (warp == Shape::kMmaWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, SUM_TMEM_COLS);
     }

@@ -228,6 +228,26 @@ def test_seg_sum_csr_many_tiles_per_cta(mmv, maxlen):
     assert_fp(sum_csr(mmv, xf, off), want, a, f"many tiles, maxlen={maxlen}")
 
 
+@pytest.mark.parametrize("groups", [2, 4])
+def test_seg_sum_both_kernel_shapes(mmv, groups):
+    # the kernel exists with 8 and with 16 epilogue warps; the library picks by average segment
+    # length, here each shape is forced over sparse, dense and empty-heavy boundaries
+    mmv.debug_force_sum_groups(groups)
+    try:
+        for maxlen, nseg in [(2, 200000), (90, 40000), (6000, 1500), (70000, 40)]:
+            rng = np.random.default_rng(groups * 100 + maxlen)
+            lens = rng.integers(0, maxlen + 1, nseg)
+            off = gen.offsets_from_lengths(lens)
+            n = int(off[-1])
+            x = rng.integers(-128, 128, n).astype(np.int8)
+            assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
+            xf = rng.standard_normal(n).astype(np.float16)
+            want, a = oracle.seg_sum_csr_f16(xf, off)
+            assert_fp(sum_csr(mmv, xf, off), want, a, f"groups={groups} maxlen={maxlen}")
+    finally:
+        mmv.debug_force_sum_groups(0)
+
+
 def test_seg_sum_config2_reduced(mmv):
     x, off = gen.config2(1 << 22)
     want, a = oracle.seg_sum_csr_f16(x, off)
