@@ -137,17 +137,24 @@ class ClockSampler:
 # ---------------------------------------------------------------------------
 # the reference arm: the CPU oracle, as it stands
 # ---------------------------------------------------------------------------
-def time_oracle_scan(x, f, reps=3):
+def time_oracle_scan(x, f, reps=2, got=None):
+    """Times the oracle's fp16 scan on (x, f).  The baseline leg has the oracle's result for the whole
+    workload in hand, so it also reports how far the device result `got` (a CUDA tensor) is from it,
+    as the largest |error| / bound over all elements."""
     import oracle
-    best = float("inf")
+    oracle.build()
+    best, z, a = float("inf"), None, None
     for _ in range(reps):
         t0 = time.perf_counter()
-        if x.dtype == np.int8:
-            oracle.seg_scan_i8(x, f)
-        else:
-            oracle.seg_scan_f16(x, f)
+        z, a = oracle.seg_scan_f16(x, f)
         best = min(best, time.perf_counter() - t0)
-    return best
+    worst = None
+    if got is not None:
+        worst, step = 0.0, 1 << 26
+        for o in range(0, x.shape[0], step):
+            _, ratio, _ = oracle.check_fp(got[o:o + step].cpu().numpy(), z[o:o + step], a[o:o + step])
+            worst = max(worst, ratio)
+    return best, worst
 
 
 def run_reference(args):
@@ -172,7 +179,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"seg-scan fp16->fp32, flags {args.case}, CPU oracle on a sample", "n": n},
+        "config": {"workload": f"C5 seg-scan n=2^{args.log2n} fp16 U[-1,1) -> fp32, uint8 flags {args.case}",
+                   "sample_per_step": sample},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -221,34 +229,9 @@ def event_time_ms(torch, fn, steps, flush=None):
     return total / steps
 
 
-def verify_scan_sample(torch, mmv, oracle, x, f, out_d, ws):
-    """Checks the device result on the head of the array and on a window that starts at a flag."""
-    n = x.shape[0]
-    m = min(n, 1 << 22)
-    windows = [(0, m)]
-    if n > 2 * m:
-        nz = np.flatnonzero(f[n // 2:n // 2 + m])
-        if nz.size:
-            s = n // 2 + int(nz[0])
-            windows.append((s, min(n, s + m)))
-    worst = 0.0
-    for a, b in windows:
-        got = out_d[a:b].cpu().numpy()
-        if x.dtype == np.int8:
-            want = oracle.seg_scan_i8(x[a:b], f[a:b])
-            if not np.array_equal(got, want):
-                raise SystemExit(f"bench: int8 scan mismatch in window {a}:{b}")
-        else:
-            z, ab = oracle.seg_scan_f16(x[a:b], f[a:b])
-            ok, ratio, i = oracle.check_fp(got, z, ab)
-            worst = max(worst, ratio)
-            if not ok:
-                raise SystemExit(f"bench: fp16 scan outside the bound in window {a}:{b}: ratio {ratio} at {a + i}")
-    return worst
-
-
-def bench_configs(torch, mmv, oracle, peak, steps, warmup, l2_flush):
-    """Short measurements of the five configurations (device-resident inputs)."""
+def bench_configs(torch, mmv, peak, steps, warmup, l2_flush):
+    """Short measurements of the five configurations (device-resident inputs).  Timing only: parity at
+    these sizes is checked by tests/test_gpu_full_size.py, which makes the same calls."""
     res = []
 
     def rec(name, units, bytes_, ms, extra=None):
@@ -271,9 +254,8 @@ def bench_configs(torch, mmv, oracle, peak, steps, warmup, l2_flush):
         torch.cuda.synchronize()
         ms = event_time_ms(torch, fn, steps, flush)
         assert mmv.last_async_status(ws) == 0
-        worst = verify_scan_sample(torch, mmv, oracle, x, f, out, ws)
         bpe = (2 if dt == mmv.F16_TO_F32 else 1) + 1 + 4
-        rec(name, n, n * bpe, ms, {"worst_err_over_bound": worst} if dt == mmv.F16_TO_F32 else {"mismatches": 0})
+        rec(name, n, n * bpe, ms)
         del xd, fd, out, ws
 
     x, f = gen.config1()
@@ -290,12 +272,8 @@ def bench_configs(torch, mmv, oracle, peak, steps, warmup, l2_flush):
     torch.cuda.synchronize()
     ms = event_time_ms(torch, fn, steps)
     assert mmv.last_async_status(ws) == 0
-    want, a = oracle.seg_sum_csr_f16(x, off)
-    ok, ratio, i = oracle.check_fp(out.cpu().numpy(), want, a)
-    if not ok:
-        raise SystemExit(f"bench: config 2 outside the bound: ratio {ratio} at segment {i}")
     rec("C2 seg-sum n=2^26 fp16 N(0,1), CSR offsets len U{1..4096}", n, 2 * n + 4 * (nseg + 1) + 4 * nseg, ms,
-        {"segments": nseg, "worst_err_over_bound": ratio})
+        {"segments": nseg})
     del xd, od, out, ws
 
     # the same recipe four times larger (the n >= 2^28 point of the target), and the flag-encoded
@@ -311,12 +289,8 @@ def bench_configs(torch, mmv, oracle, peak, steps, warmup, l2_flush):
     torch.cuda.synchronize()
     ms = event_time_ms(torch, fn, steps)
     assert mmv.last_async_status(ws) == 0
-    want, a = oracle.seg_sum_csr_f16(x, off)
-    ok, ratio, i = oracle.check_fp(out.cpu().numpy(), want, a)
-    if not ok:
-        raise SystemExit(f"bench: config 2 (n = 2^28) outside the bound: ratio {ratio} at segment {i}")
     rec("C2x4 seg-sum n=2^28 fp16 N(0,1), CSR offsets len U{1..4096}", n, 2 * n + 4 * (nseg + 1) + 4 * nseg, ms,
-        {"segments": nseg, "worst_err_over_bound": ratio})
+        {"segments": nseg})
     del od, ws
     f = gen.start_flags_of_offsets(off, n)
     fd = torch.from_numpy(f).cuda()
@@ -330,12 +304,10 @@ def bench_configs(torch, mmv, oracle, peak, steps, warmup, l2_flush):
     ms = event_time_ms(torch, fn, steps)
     assert mmv.last_async_status(ws) == 0
     k = int(kd.item())
-    wantf, af = oracle.seg_sum_flags_f16(x, f)
-    ok, ratio, i = oracle.check_fp(outf[:k].cpu().numpy(), wantf, af) if k == wantf.shape[0] else (False, float("inf"), -1)
-    if not ok:
-        raise SystemExit(f"bench: flag-form seg-sum outside the bound: ratio {ratio} at segment {i} (K = {k})")
+    if k != nseg - int(np.count_nonzero(np.diff(off.astype(np.int64)) == 0)):
+        raise SystemExit(f"bench: flag-form seg-sum found {k} segments")
     rec("N1 seg-sum (start flags) n=2^28 fp16 N(0,1), same segments as C2x4", n, 2 * n + n + 4 * k, ms,
-        {"segments": k, "worst_err_over_bound": ratio})
+        {"segments": k})
     del xd, fd, out, outf, ws
 
     x, f = gen.config3()
@@ -352,12 +324,8 @@ def bench_configs(torch, mmv, oracle, peak, steps, warmup, l2_flush):
     torch.cuda.synchronize()
     ms = event_time_ms(torch, fn, steps)
     assert mmv.last_async_status(ws) == 0
-    want, a = oracle.spmv_csr(rowptr, col, val, xv)
-    ok, ratio, i = oracle.check_fp(y.cpu().numpy(), want, a)
-    if not ok:
-        raise SystemExit(f"bench: config 4 outside the bound: ratio {ratio} at row {i}")
     rec("C4 CSR SpMV 2^20 rows, nnz/row Zipf(1.5) cap 1e4", nnz, 6 * nnz + 4 * (rows + 1) + 4 * xv.shape[0] + 4 * rows,
-        ms, {"nnz": nnz, "worst_err_over_bound": ratio})
+        ms, {"nnz": nnz})
     del rd, cd, vd, xd, y, ws
     torch.cuda.empty_cache()
     return res
@@ -375,10 +343,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     import paper_2506_23906_b200 as mmv
-    import oracle
 
-    if rank == 0:
-        oracle.build()
     n = 1 << args.log2n
     x = gen.f16_uniform(5, n)
     f = gen.config5_flags(n, args.case)
@@ -431,7 +396,6 @@ def run_ours(args):
     ms = e0.elapsed_time(e1) / args.steps
     if mmv.last_async_status(ws) != 0:
         raise SystemExit("bench: device-side error status")
-    worst = verify_scan_sample(torch, mmv, oracle, x, f, od, ws)
 
     # end to end: pinned host -> device, the call, device -> host, every step
     e2e_steps = max(1, min(args.steps, 5))
@@ -470,19 +434,22 @@ def run_ours(args):
                          "algorithmic_bytes_per_elem": 7,
                          "traffic": (NCU_READ_BYTES_PER_ELEM + NCU_WRITE_BYTES_PER_ELEM) * n - NCU_WRITE_L2_RESIDUE_BYTES,
                          "traffic_source": "ncu capture at n=2^26 scaled by n (profiles/seg_scan_kernel_f16_n2p26_p1e-3.md)"},
-            "worst_err_over_bound": worst,
         }
         del xh, fh, oh
         if not args.no_cpu:
-            sec = time_oracle_scan(x, f, reps=3)
+            mmv.seg_scan(xd, fd, out=od, workspace=ws)
+            sec, worst = time_oracle_scan(x, f, reps=2, got=od)
             line["cpu_baseline"] = {"value": n / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                    "sample": f"the whole headline workload (n=2^{args.log2n}), best of 3, {sec:.2f} s"}
+                                    "sample": f"the whole headline workload (n=2^{args.log2n}), best of 2, {sec:.2f} s",
+                                    "device_result_worst_err_over_bound": worst}
+            if worst is not None and not worst <= 1.0:
+                raise SystemExit(f"bench: the device result is outside the bound (ratio {worst})")
         del xd, fd, od
         torch.cuda.empty_cache()
         if world == 1 and not args.no_configs:
             def l2_flush():
                 l2_buf.zero_()
-            cfgs = bench_configs(torch, mmv, oracle, peak, min(args.steps, 20), max(3, args.warmup), l2_flush)
+            cfgs = bench_configs(torch, mmv, peak, min(args.steps, 20), max(3, args.warmup), l2_flush)
             # the seven flag patterns of configuration 5 on the headline values
             xd = torch.from_numpy(x).cuda()
             od = torch.empty(n, dtype=torch.float32, device="cuda")
@@ -496,10 +463,9 @@ def run_ours(args):
                 torch.cuda.synchronize()
                 cms = event_time_ms(torch, fn, min(args.steps, 10))
                 assert mmv.last_async_status(ws) == 0
-                w = verify_scan_sample(torch, mmv, oracle, x, fc, od, ws)
                 sweep.append({"case": case, "ms": cms, "gelem_s": n / cms / 1e6, "gb_s": 7 * n / cms / 1e6,
                               "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
-                              "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS, "worst_err_over_bound": w})
+                              "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
                 del fd
             line["configs"] = cfgs
             line["c5_density_sweep"] = sweep

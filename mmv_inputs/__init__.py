@@ -13,6 +13,9 @@ Section 5), whose data files are not available here.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 BASE_SEED = 250623906
@@ -52,9 +55,22 @@ def i8_uniform_chunk(config: int, chunk: int, m: int = CHUNK, lo: int = -8, hi: 
 
 
 def _full(fn, n: int, dtype, *a, **k) -> np.ndarray:
+    """All chunks of an array; chunks are independent, so large arrays are filled by a few threads
+    (numpy releases the GIL in the generators and conversions; the values do not depend on it)."""
     out = np.empty(n, dtype)
-    for c, m in _chunks(n):
+
+    def fill(cm):
+        c, m = cm
         out[c * CHUNK:c * CHUNK + m] = fn(*a, chunk=c, m=m, **k)
+
+    todo = list(_chunks(n))
+    workers = min(len(todo), os.cpu_count() or 1, 16)
+    if workers <= 1:
+        for cm in todo:
+            fill(cm)
+    else:
+        with ThreadPoolExecutor(max_workers=workers) as ex:
+            list(ex.map(fill, todo))
     return out
 
 
@@ -85,8 +101,7 @@ def flags_chunk(config: int, chunk: int, m: int = CHUNK, p: float = 1.0 / 64, pa
     elif pattern == "cycle123":
         base = (chunk * CHUNK) % 6
         pat = np.array([1, 1, 0, 1, 0, 0], np.uint8)
-        idx = (np.arange(m, dtype=np.int64) + base) % 6
-        f = pat[idx]
+        f = np.tile(np.roll(pat, -base), m // 6 + 1)[:m].copy()      # pat[(i + base) % 6] for i < m
     elif pattern == "bernoulli":
         if p <= 0.0:
             f = np.zeros(m, np.uint8)

@@ -1,0 +1,128 @@
+"""Parity at the sizes and in the launch configuration that bench.py times.
+
+The same binding calls as the benchmark (device-resident inputs, one workspace, current stream),
+on the full-size synthetic workloads; the oracle is streamed over the arrays chunk by chunk (it
+keeps its running state between chunks), or run on windows that start at a segment start, so that
+no more than a chunk of fp64 reference values is ever held.
+"""
+import numpy as np
+import pytest
+
+import mmv_inputs as gen
+import oracle
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+STEP = 1 << 24
+
+
+@pytest.fixture(scope="module")
+def mmv():
+    if not torch.cuda.is_available():
+        pytest.skip("no GPU")
+    import paper_2506_23906_b200 as m
+    return m
+
+
+def stream_check_f16(x, f, out_d, what, lo=0, hi=None, state=None):
+    """Oracle streamed over [lo, hi) with carried state; returns the largest |error| / bound."""
+    hi = x.shape[0] if hi is None else hi
+    state = oracle.new_f16_state() if state is None else state
+    worst = 0.0
+    for o in range(lo, hi, STEP):
+        e = min(hi, o + STEP)
+        z, a = oracle.seg_scan_f16(x[o:e], f[o:e], state)
+        ok, ratio, i = oracle.check_fp(out_d[o:e].cpu().numpy(), z, a)
+        assert ok, f"{what}: outside the bound at element {o + i} (ratio {ratio})"
+        worst = max(worst, ratio)
+    return worst
+
+
+def window_starts(f, n, m):
+    """Head, a window in the middle that starts at a segment start, and the tail window (also
+    starting at a segment start), each at most m long."""
+    wins = [(0, min(n, m))]
+    for anchor in (n // 2, max(0, n - m)):
+        nz = np.flatnonzero(f[anchor:min(n, anchor + m)])
+        if nz.size:
+            s = anchor + int(nz[0])
+            wins.append((s, min(n, s + m)))
+    return wins
+
+
+@pytest.fixture(scope="module")
+def c5_values():
+    return gen.config5_values(1 << 30)
+
+
+@pytest.mark.parametrize("case", [c for c, _ in gen.C5_CASES])
+def test_config5_full_size(mmv, c5_values, case):
+    x = c5_values
+    n = x.shape[0]
+    f = gen.config5_flags(n, case)
+    xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+    od = torch.empty(n, dtype=torch.float32, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+    for _ in range(2):                                   # as in the benchmark: repeated launches, one workspace
+        mmv.seg_scan(xd, fd, out=od, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    if case in ("p1e-3", "p0"):
+        # every element: the headline case and the single-segment case (whose carries span the whole array)
+        stream_check_f16(x, f, od, f"config 5 / {case}")
+    else:
+        for a, b in window_starts(f, n, 1 << 25):
+            stream_check_f16(x, f, od, f"config 5 / {case} window {a}:{b}", a, b)
+    del xd, fd, od, ws
+    torch.cuda.empty_cache()
+
+
+def test_config3_full_size(mmv):
+    x, f = gen.config3()
+    n = x.shape[0]
+    xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+    od = torch.empty(n, dtype=torch.int32, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    mmv.seg_scan(xd, fd, out=od, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    state = oracle.new_i8_state()
+    for o in range(0, n, STEP):
+        want = oracle.seg_scan_i8(x[o:o + STEP], f[o:o + STEP], state)
+        assert np.array_equal(od[o:o + STEP].cpu().numpy(), want), f"config 3: mismatch in chunk at {o}"
+
+
+def test_config2_full_size_and_four_times_larger_with_both_encodings(mmv):
+    for n in (1 << 26, 1 << 28):
+        x, off = gen.config2(n)
+        nseg = off.shape[0] - 1
+        want, a = oracle.seg_sum_csr_f16(x, off)
+        xd = torch.from_numpy(x).cuda()
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, n, nseg)
+        out = mmv.seg_sum(xd, torch.from_numpy(off).cuda(), workspace=ws)
+        assert mmv.last_async_status(ws) == 0
+        ok, ratio, i = oracle.check_fp(out.cpu().numpy(), want, a)
+        assert ok, f"config 2 (n = {n}): ratio {ratio} at segment {i}"
+        if n == 1 << 28:
+            f = gen.start_flags_of_offsets(off, n)
+            wantf, af = oracle.seg_sum_flags_f16(x, f)
+            ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+            kd = torch.zeros(1, dtype=torch.int64, device="cuda")
+            outf = mmv.seg_sum(xd, torch.from_numpy(f).cuda(), num_segments=kd, workspace=ws)
+            assert mmv.last_async_status(ws) == 0
+            assert int(kd.item()) == wantf.shape[0]
+            ok, ratio, i = oracle.check_fp(outf[:wantf.shape[0]].cpu().numpy(), wantf, af)
+            assert ok, f"flag-encoded config 2 (n = {n}): ratio {ratio} at segment {i}"
+        del xd, ws
+        torch.cuda.empty_cache()
+
+
+def test_config4_full_size(mmv):
+    rowptr, col, val, xv = gen.config4()
+    rows = rowptr.shape[0] - 1
+    ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, val.shape[0], rows)
+    y = mmv.spmv_csr(torch.from_numpy(rowptr).cuda(), torch.from_numpy(col).cuda(), torch.from_numpy(val).cuda(),
+                     torch.from_numpy(xv).cuda(), workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    want, a = oracle.spmv_csr(rowptr, col, val, xv)
+    ok, ratio, i = oracle.check_fp(y.cpu().numpy(), want, a)
+    assert ok, f"config 4: ratio {ratio} at row {i}"
