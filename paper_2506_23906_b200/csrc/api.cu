@@ -352,9 +352,9 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
     prm.debug_skip_span = g_debug_skip_span.load();
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
     if (f16)
-        seg_scan_kernel<F16Path><<<grid, SCAN_THREADS, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+        seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
     else
-        seg_scan_kernel<I8Path><<<grid, SCAN_THREADS, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+        seg_scan_kernel<I8Path><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
@@ -500,9 +500,9 @@ mmv_status mmv_seg_scan_static(const void* x, const void* flags_u8, int64_t n, m
     prm.debug_skip_span = -1;
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
     if (f16)
-        seg_scan_kernel<F16Path><<<grid, SCAN_THREADS, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+        seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
     else
-        seg_scan_kernel<I8Path><<<grid, SCAN_THREADS, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+        seg_scan_kernel<I8Path><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }

@@ -47,27 +47,33 @@ struct ScanParams {
 
 // Scan geometry: a warp owns a UNIT of SCAN_UP consecutive pieces (the grain of the carry
 // chain: one status word per unit); a scan tile is four units and SCAN_UP tensor-core products.
-// SCAN_GROUPS warpgroups take alternating tiles; each has two TMEM buffers so that the products
-// of its next tile are finished before it gets there.
+// The warpgroups of the epilogue (two for fp16, three for int8) take tiles in turn; with two TMEM
+// buffers per warpgroup (int8 built with two groups) the products of a group's next tile are
+// finished before it gets there.
 constexpr int SCAN_UP = 4;
 constexpr int SCAN_UNIT = SCAN_UP * PIECE;                  // 4096 elements
 constexpr int SCAN_TILE = SPANS_PER_TILE * SCAN_UNIT;       // 16384 elements
-constexpr int SCAN_GROUPS = 2;
-constexpr int SCAN_BUFS = 2 * SCAN_GROUPS;                  // TMEM tile buffers
-constexpr int SCAN_EPI_WARPS = 4 * SCAN_GROUPS;             // 8
-constexpr int SCAN_PRODUCER_WARP = SCAN_EPI_WARPS;
-constexpr int SCAN_MMA_WARP = SCAN_EPI_WARPS + 1;
-constexpr int SCAN_THREADS = (SCAN_EPI_WARPS + 2) * 32;     // 320
-constexpr int SCAN_LB_WORDS = 1;                            // look-back window: 128 tiles per poll
+constexpr int SCAN_LB_WORDS = 1;                            // look-back window: 32 tiles per poll
+#ifndef MMV_SCAN_I8_GROUPS
+#define MMV_SCAN_I8_GROUPS 3
+#endif
 
 template <typename P>
 struct ScanCfg {
     // fp16: the product also returns the rows themselves (exact fp32 copies, columns 32..63), so a
     // tile needs 256 TMEM columns and each warpgroup has one buffer; int8: 128 columns, two buffers.
+    // The epilogue is latency-bound, so the narrower int8 tiles are spread over a third warpgroup.
     static constexpr int kN = P::kIsFloat ? 2 * ROW : ROW;               // accumulator columns per product
-    static constexpr int kBufsPerGroup = P::kIsFloat ? 1 : 2;
-    static constexpr int kTmemCols = SCAN_GROUPS * kBufsPerGroup * SCAN_UP * kN;   // 512
-    static constexpr int kStages = P::kIsFloat ? 3 : 4;
+    static constexpr int kGroups = P::kIsFloat ? 2 : MMV_SCAN_I8_GROUPS;
+    static constexpr int kBufsPerGroup = P::kIsFloat ? 1 : (kGroups == 2 ? 2 : 1);
+    static constexpr int kBufs = kGroups * kBufsPerGroup;                // TMEM tile buffers
+    static constexpr int kEpiWarps = 4 * kGroups;
+    static constexpr int kProducerWarp = kEpiWarps;
+    static constexpr int kMmaWarp = kEpiWarps + 1;
+    static constexpr int kThreads = (kEpiWarps + 2) * 32;
+    static constexpr int kTmemCols = 512;
+    static constexpr int kStages = P::kIsFloat ? 3 : (kGroups == 2 ? 4 : 3);
+    static_assert(kBufs * SCAN_UP * kN <= kTmemCols, "tile buffers fit the tensor memory");
     static constexpr int kBBytes = kN * P::kRowBytes;                    // constant operand [U_32 | I_32] / U_32
     static constexpr int kBSlot = 4096;
     static constexpr int kXBytes = SCAN_UP * P::kSlabBytes;
@@ -77,9 +83,10 @@ struct ScanCfg {
     static constexpr int kOutOffset = kStageOffset + kStages * kStageBytes;
     static constexpr int kOutBufBytes = PIECE * 4;                       // 32 rows x 128 B
     static constexpr int kOutBufs = 2;                                   // staging buffers per warp
-    static constexpr int kOutBytes = SCAN_EPI_WARPS * kOutBufs * kOutBufBytes;
+    static constexpr int kOutBytes = kEpiWarps * kOutBufs * kOutBufBytes;
     static constexpr int kBarOffset = kOutOffset + kOutBytes;
     static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
+    static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of one CTA");
     static_assert(kBBytes <= kBSlot, "constant operand fits its slot");
     static_assert(kStageOffset % 1024 == 0 && kStageBytes % 1024 == 0 && kOutOffset % 1024 == 0, "swizzle atoms");
 };
@@ -116,7 +123,7 @@ __device__ __forceinline__ bool wait_stage(const volatile int* stage_iter, int i
 }
 
 template <typename P>
-__global__ void __launch_bounds__(SCAN_THREADS, 1)
+__global__ void __launch_bounds__(ScanCfg<P>::kThreads, 1)
 seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_out,
                  const ScanParams prm) {
     using Acc = typename P::Acc;
@@ -131,14 +138,14 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     uint64_t* bar_full = reinterpret_cast<uint64_t*>(smem + Cfg::kBarOffset);
     uint64_t* bar_empty = bar_full + S;
     uint64_t* bar_acc_full = bar_empty + S;                // per TMEM buffer: the tile's products are in it
-    uint64_t* bar_acc_empty = bar_acc_full + SCAN_BUFS;    // per TMEM buffer: the four warps are done with it
-    uint64_t* bar_agg = bar_acc_empty + SCAN_BUFS;          // per warpgroup: its four unit aggregates are in agg_slot
-    uint64_t* bar_carry = bar_agg + SCAN_GROUPS;           // per warpgroup: the tile's carry is in carry_slot
+    uint64_t* bar_acc_empty = bar_acc_full + Cfg::kBufs;    // per TMEM buffer: the four warps are done with it
+    uint64_t* bar_agg = bar_acc_empty + Cfg::kBufs;          // per warpgroup: its four unit aggregates are in agg_slot
+    uint64_t* bar_carry = bar_agg + Cfg::kGroups;           // per warpgroup: the tile's carry is in carry_slot
     // [group][tile parity][unit]: (flag << 32) | payload; two sets so that a warp's next-tile write
     // can never meet a sibling's read of this tile's values
-    uint64_t* agg_slot = bar_carry + SCAN_GROUPS;
-    uint32_t* carry_slot = reinterpret_cast<uint32_t*>(agg_slot + SCAN_GROUPS * 2 * SPANS_PER_TILE);   // [group]
-    int* tile_slot = reinterpret_cast<int*>(carry_slot + SCAN_GROUPS);
+    uint64_t* agg_slot = bar_carry + Cfg::kGroups;
+    uint32_t* carry_slot = reinterpret_cast<uint32_t*>(agg_slot + Cfg::kGroups * 2 * SPANS_PER_TILE);   // [group]
+    int* tile_slot = reinterpret_cast<int*>(carry_slot + Cfg::kGroups);
     volatile int* stage_iter = tile_slot + S;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_slot + 2 * S);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -153,22 +160,22 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             mbar_init(&bar_empty[i], 4);      // the group's four warps, once their flag bytes are read
             stage_iter[i] = -1;
         }
-        for (int i = 0; i < SCAN_GROUPS; ++i) {
+        for (int i = 0; i < Cfg::kGroups; ++i) {
             mbar_init(&bar_agg[i], SPANS_PER_TILE);
             mbar_init(&bar_carry[i], 1);
         }
-        for (int i = 0; i < SCAN_BUFS; ++i) {
+        for (int i = 0; i < Cfg::kBufs; ++i) {
             mbar_init(&bar_acc_full[i], 1);
             mbar_init(&bar_acc_empty[i], 4);
         }
         *abort_flag = 0;
         mbar_fence_init();
     }
-    if (warp == SCAN_MMA_WARP) {
+    if (warp == Cfg::kMmaWarp) {
         tmem_alloc(tmem_slot, Cfg::kTmemCols);
         tmem_relinquish();
     }
-    if (warp == SCAN_PRODUCER_WARP && lane == 0) {
+    if (warp == Cfg::kProducerWarp && lane == 0) {
         tma_prefetch_desc(&tmap_x);
         tma_prefetch_desc(&tmap_out);
     }
@@ -178,7 +185,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         constexpr int kVecPerRow = P::kRowBytes / 16;
         constexpr int kElemPerVec = 16 / P::kElemBytes;
 #pragma unroll 1
-        for (int v = threadIdx.x; v < N * kVecPerRow; v += SCAN_THREADS) {
+        for (int v = threadIdx.x; v < N * kVecPerRow; v += Cfg::kThreads) {
             const int nn = v / kVecPerRow, cv = v % kVecPerRow;
             uint32_t words[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
@@ -200,7 +207,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == SCAN_PRODUCER_WARP) {
+    if (warp == Cfg::kProducerWarp) {
         // =========================== producer ===========================
         int it = 0, sentinels = 0;
         bool ok = true;
@@ -220,7 +227,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar_full[stage]);
                 ++it;
-                if (++sentinels == SCAN_GROUPS) break;
+                if (++sentinels == Cfg::kGroups) break;
                 continue;
             }
             uint8_t* xs = sStage + stage * Cfg::kStageBytes;
@@ -281,7 +288,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             if (lane == 0) report_error(prm.hdr, 5u);
         }
         for (int k = (it > S ? it - S : 0); k < it; ++k) mbar_wait(&bar_full[k % S], (k / S) & 1, 2000000ull);
-    } else if (warp == SCAN_MMA_WARP) {
+    } else if (warp == Cfg::kMmaWarp) {
         // =========================== MMA issuer ===========================
         // Runs ahead of the epilogue: the products of a warpgroup's next tile go to its other buffer.
         constexpr uint32_t idesc = P::kIsFloat ? (make_idesc_f16_f32(128, N) | P::kFmtBits) : make_idesc_s8_s32(128, N);
@@ -294,10 +301,10 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 break;
             }
             if (tile_slot[stage] < 0) {
-                if (++sentinels == SCAN_GROUPS) break;
+                if (++sentinels == Cfg::kGroups) break;
                 continue;
             }
-            const int g = it % SCAN_GROUPS, k = it / SCAN_GROUPS;
+            const int g = it % Cfg::kGroups, k = it / Cfg::kGroups;
             const int buf = g * Cfg::kBufsPerGroup + (k % Cfg::kBufsPerGroup);
             if (!wait_bar(&bar_acc_empty[buf], ((k / Cfg::kBufsPerGroup) & 1) ^ 1, abort_flag, budget)) {
                 *abort_flag = 1;
@@ -326,7 +333,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     } else {
         // =========================== epilogue ===========================
         constexpr int UP = SCAN_UP;
-        const int g = warp >> 2;            // warpgroup: iterations g, g + SCAN_GROUPS, ...
+        const int g = warp >> 2;            // warpgroup: iterations g, g + Cfg::kGroups, ...
         const int w = warp & 3;             // unit inside the tile = TMEM lane quarter
         Acc* outp = static_cast<Acc*>(prm.out);
         uint8_t* stg = smem + Cfg::kOutOffset + warp * Cfg::kOutBufs * Cfg::kOutBufBytes;
@@ -365,7 +372,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         };
 
         for (int k = 0;; ++k) {
-            const int it = g + SCAN_GROUPS * k;
+            const int it = g + Cfg::kGroups * k;
             const int stage = it % S;
             if (!wait_stage(&stage_iter[stage], it, &bar_full[stage], (it / S) & 1, abort_flag, budget)) { failed = true; break; }
             const int tile = tile_slot[stage];
@@ -628,7 +635,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == SCAN_MMA_WARP) {
+    if (warp == Cfg::kMmaWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, Cfg::kTmemCols);
     }
