@@ -178,6 +178,27 @@ mmv_status mmv_seg_scan_static(const void *x, const void *flags_u8, int64_t n, m
 mmv_status mmv_seg_scan_static_last_status(void *cuda_stream);
 
 /*
+ * Segmented scan (Problem 2.1) of vectors that live in HOST memory: x_host (n values), flags_host
+ * (n start-flag bytes) and out_host (n results) are host pointers.  The vectors are cut into
+ * chunks of chunk_elems elements (a positive multiple of 16384); the chunks are copied to the
+ * device, scanned and copied back on three internal streams, so that the copy-in, the kernels
+ * and the copy-out of neighbouring chunks overlap; the running sum at the end of a chunk is
+ * handed to the next chunk's kernel on the device.  Results are identical to mmv_seg_scan on
+ * the whole vector.  device_scratch: device memory, 256-byte aligned, at least
+ * mmv_seg_scan_host_scratch_bytes(dt, chunk_elems) bytes (two chunk buffers and their carry
+ * words).  The work is ordered after everything already in cuda_stream, and cuda_stream
+ * continues only when all results are on the host; the call itself returns without waiting, so
+ * the host vectors must stay valid and untouched until the stream has drained.  Use pinned
+ * (page-locked) host memory: with pageable memory the copies do not overlap.  The internal
+ * streams are shared by all calls on a device, which therefore must not overlap in time.
+ * Device-side status: mmv_last_async_status(device_scratch, cuda_stream).
+ */
+size_t mmv_seg_scan_host_scratch_bytes(mmv_dtype dt, int64_t chunk_elems);
+mmv_status mmv_seg_scan_host(const void *x_host, const void *flags_host, int64_t n, mmv_dtype dt, void *out_host,
+                             int64_t chunk_elems, void *device_scratch, size_t device_scratch_bytes,
+                             void *cuda_stream);
+
+/*
  * Test hook.  wait_budget_ns: time after which a device-side wait gives up
  * (<= 0 restores the default of 4 s).  skip_publish_span: index of one
  * 4096-element span of the scan that never publishes its carry, so that its

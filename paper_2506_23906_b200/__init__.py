@@ -26,6 +26,7 @@ EXPORTS = (
     "mmv_workspace_bytes", "mmv_seg_scan", "mmv_seg_sum", "mmv_spmv_csr",
     "mmv_last_async_status", "mmv_status_string", "mmv_kernel_launch_count", "mmv_debug_configure",
     "mmv_seg_scan_static", "mmv_seg_scan_static_last_status", "mmv_debug_force_sum_groups",
+    "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes",
 )
 STATIC_SCAN_MAX_N = 1 << 28
 
@@ -63,6 +64,10 @@ def _load() -> ctypes.CDLL:
     lib.mmv_seg_scan_static_last_status.argtypes = [vp]
     lib.mmv_debug_configure.restype = None
     lib.mmv_debug_configure.argtypes = [i64, i64]
+    lib.mmv_seg_scan_host_scratch_bytes.restype = sz
+    lib.mmv_seg_scan_host_scratch_bytes.argtypes = [ci, i64]
+    lib.mmv_seg_scan_host.restype = ci
+    lib.mmv_seg_scan_host.argtypes = [vp, vp, i64, ci, vp, i64, vp, sz, vp]
     lib.mmv_debug_force_sum_groups.restype = None
     lib.mmv_debug_force_sum_groups.argtypes = [ci]
     return lib
@@ -162,6 +167,35 @@ def seg_scan_static(x: torch.Tensor, flags: torch.Tensor, out: torch.Tensor, str
     rc = _lib.mmv_seg_scan_static(_ptr(x), _ptr(flags), x.numel(), _dtype_code(x), _ptr(out), _stream_ptr(stream))
     if rc != MMV_OK:
         raise MmvError(rc, "mmv_seg_scan_static")
+    return out
+
+
+def host_scan_scratch(dt: int, chunk: int, device=None) -> torch.Tensor:
+    nbytes = int(_lib.mmv_seg_scan_host_scratch_bytes(dt, int(chunk)))
+    if nbytes == 0:
+        raise ValueError("chunk must be a positive multiple of 16384")
+    return torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
+
+
+def seg_scan_host(x: torch.Tensor, flags: torch.Tensor, out: torch.Tensor | None = None, chunk: int = 1 << 26,
+                  scratch: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """mmv_seg_scan_host: the scan of HOST tensors (pinned memory recommended), copies and kernels
+    of neighbouring chunks overlapped.  Returns ``out`` (a pinned host tensor unless one is given);
+    the results are complete once the stream has been synchronised."""
+    if x.is_cuda or flags.is_cuda or (out is not None and out.is_cuda):
+        raise ValueError("seg_scan_host takes host tensors")
+    if flags.dtype != torch.uint8 or not x.is_contiguous() or not flags.is_contiguous():
+        raise TypeError("contiguous values and uint8 start flags expected")
+    dt = _dtype_code(x)
+    n = x.numel()
+    if out is None:
+        out = torch.empty(n, dtype=torch.float32 if dt == F16_TO_F32 else torch.int32, pin_memory=True)
+    if scratch is None:
+        scratch = host_scan_scratch(dt, chunk)
+    rc = _lib.mmv_seg_scan_host(_ptr(x), _ptr(flags), n, dt, _ptr(out), int(chunk), _ptr(scratch), scratch.numel(),
+                                _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_seg_scan_host")
     return out
 
 

@@ -29,6 +29,12 @@ struct DeviceInfo {
     std::once_flag once;
     int sm_count = 0;
     bool ok = false;
+    // copy-in / kernel / copy-out streams and their events for mmv_seg_scan_host (made on first use)
+    std::once_flag pipe_once;
+    bool pipe_ok = false;
+    cudaStream_t s_in = nullptr, s_k = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_end_k = nullptr, ev_end_out = nullptr;
+    cudaEvent_t in_done[2] = {nullptr, nullptr}, k_done[2] = {nullptr, nullptr}, out_done[2] = {nullptr, nullptr};
 };
 DeviceInfo g_dev[kMaxDevices];
 
@@ -71,6 +77,7 @@ DeviceInfo* device_info() {
         ok &= set_smem(seg_sum_kernel<BF16Path, 2>, SumCfg<BF16Path, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<F16Path, 4>, SumCfg<F16Path, 4>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<I8Path, 4>, SumCfg<I8Path, 4>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<BF16Path, 4>, SumCfg<BF16Path, 4>::kSmemBytes);
         d->ok = ok;
     });
     return d->ok ? d : nullptr;
@@ -227,11 +234,10 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     const int grid = tiles < dev->sm_count ? tiles : dev->sm_count;
     // Long segments (few boundaries per 4096-element span): sixteen epilogue warps on the light path.
     // The segment count of the flag-encoded form is not known here; it takes the eight-warp kernel.
-    bool many_warps = false;
-    if constexpr (!std::is_same<P, BF16Path>::value) many_warps = !nseg_dev && nseg > 0 && n_eff / nseg >= 256;
+    bool many_warps = !nseg_dev && nseg > 0 && n_eff / nseg >= 256;
     if (g_force_groups.load() == 2) many_warps = false;
-    if (g_force_groups.load() == 4 && !std::is_same<P, BF16Path>::value) many_warps = true;
-    if constexpr (!std::is_same<P, BF16Path>::value) {
+    if (g_force_groups.load() == 4) many_warps = true;
+    {
         if (many_warps) {
             seg_sum_kernel<P, 4><<<grid, SumShape<4>::kThreads, SumCfg<P, 4>::kSmemBytes, st>>>(tmap, values, prm);
             ++g_launches;
@@ -350,6 +356,7 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();
     prm.debug_skip_span = g_debug_skip_span.load();
+    prm.carry_in = nullptr;
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
     if (f16)
         seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
@@ -357,6 +364,142 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
         seg_scan_kernel<I8Path><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------
+// Scan of host-resident vectors: chunks travel host -> device, are scanned, and travel back on
+// three streams, so that the copies of neighbouring chunks overlap each other and the kernels.
+// Chunk c + 1 continues the open segment of chunk c through the kernel's carry-in word (the last
+// output element of chunk c, still in its device buffer).
+// ---------------------------------------------------------------------------
+namespace {
+
+struct HostScanPlan {
+    size_t status_off, status_bytes;      // per buffer
+    size_t x_off, f_off, out_off;         // per buffer, relative to the buffer's base
+    size_t buf_bytes;
+    size_t total;
+};
+
+HostScanPlan plan_host_scan(mmv_dtype dt, long long chunk) {
+    HostScanPlan p{};
+    const size_t eb = dt == MMV_F16_TO_F32 ? 2 : 1;
+    p.status_off = 0;
+    p.status_bytes = round_up(static_cast<size_t>(num_scan_tiles_of(chunk)) * SPANS_PER_TILE * sizeof(uint64_t), 256);
+    p.x_off = p.status_bytes;
+    p.f_off = p.x_off + round_up(static_cast<size_t>(chunk) * eb, 256);
+    p.out_off = p.f_off + round_up(static_cast<size_t>(chunk), 256);
+    p.buf_bytes = p.out_off + round_up(static_cast<size_t>(chunk) * 4, 256);
+    p.total = sizeof(WorkspaceHeader) + 2 * p.buf_bytes;
+    return p;
+}
+
+bool pipe_streams(DeviceInfo* d) {
+    std::call_once(d->pipe_once, [d] {
+        bool ok = true;
+        ok &= cudaStreamCreateWithFlags(&d->s_in, cudaStreamNonBlocking) == cudaSuccess;
+        ok &= cudaStreamCreateWithFlags(&d->s_k, cudaStreamNonBlocking) == cudaSuccess;
+        ok &= cudaStreamCreateWithFlags(&d->s_out, cudaStreamNonBlocking) == cudaSuccess;
+        cudaEvent_t* evs[] = {&d->ev_start, &d->ev_end_k, &d->ev_end_out, &d->in_done[0], &d->in_done[1],
+                              &d->k_done[0], &d->k_done[1], &d->out_done[0], &d->out_done[1]};
+        for (cudaEvent_t* e : evs) ok &= cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+        d->pipe_ok = ok;
+    });
+    return d->pipe_ok;
+}
+
+}  // namespace
+
+size_t mmv_seg_scan_host_scratch_bytes(mmv_dtype dt, int64_t chunk_elems) {
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return 0;
+    if (chunk_elems <= 0 || chunk_elems % SCAN_TILE != 0 || chunk_elems >= (1ll << 36)) return 0;
+    return plan_host_scan(dt, chunk_elems).total;
+}
+
+mmv_status mmv_seg_scan_host(const void* x_host, const void* flags_host, int64_t n, mmv_dtype dt, void* out_host,
+                             int64_t chunk_elems, void* device_scratch, size_t device_scratch_bytes, void* cuda_stream) {
+    if (n < 0) return MMV_ERR_INVALID_ARG;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
+    if (chunk_elems <= 0 || chunk_elems % SCAN_TILE != 0 || chunk_elems >= (1ll << 36)) return MMV_ERR_INVALID_ARG;
+    if (n == 0) return MMV_OK;
+    if (!x_host || !flags_host || !out_host || !device_scratch) return MMV_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(device_scratch) & 255u) return MMV_ERR_INVALID_ARG;
+    const HostScanPlan plan = plan_host_scan(dt, chunk_elems);
+    if (device_scratch_bytes < plan.total) return MMV_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo* dev = device_info();
+    if (!dev || !pipe_streams(dev)) return MMV_ERR_CUDA;
+
+    const bool f16 = dt == MMV_F16_TO_F32;
+    const size_t eb = f16 ? 2 : 1;
+    cudaStream_t user = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* base = static_cast<uint8_t*>(device_scratch);
+    WorkspaceHeader* hdr = reinterpret_cast<WorkspaceHeader*>(base);
+    uint8_t* buf[2] = {base + sizeof(WorkspaceHeader), base + sizeof(WorkspaceHeader) + plan.buf_bytes};
+    bool ok = true;
+    ok &= cudaMemsetAsync(hdr, 0, sizeof(WorkspaceHeader), user) == cudaSuccess;
+    ok &= cudaEventRecord(dev->ev_start, user) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(dev->s_in, dev->ev_start, 0) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(dev->s_k, dev->ev_start, 0) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(dev->s_out, dev->ev_start, 0) == cudaSuccess;
+    if (!ok) return MMV_ERR_CUDA;
+
+    const long long nchunks = (n + chunk_elems - 1) / chunk_elems;
+    const void* carry = nullptr;
+    for (long long c = 0; c < nchunks; ++c) {
+        const int b = static_cast<int>(c & 1);
+        const long long o = c * chunk_elems;
+        const long long m = n - o < chunk_elems ? n - o : chunk_elems;
+        uint8_t* xd = buf[b] + plan.x_off;
+        uint8_t* fd = buf[b] + plan.f_off;
+        uint8_t* od = buf[b] + plan.out_off;
+        // copy in: the buffer's previous kernel (chunk c - 2) must be done with it
+        if (c >= 2) ok &= cudaStreamWaitEvent(dev->s_in, dev->k_done[b], 0) == cudaSuccess;
+        ok &= cudaMemcpyAsync(xd, static_cast<const uint8_t*>(x_host) + static_cast<size_t>(o) * eb, static_cast<size_t>(m) * eb,
+                              cudaMemcpyHostToDevice, dev->s_in) == cudaSuccess;
+        ok &= cudaMemcpyAsync(fd, static_cast<const uint8_t*>(flags_host) + o, static_cast<size_t>(m), cudaMemcpyHostToDevice,
+                              dev->s_in) == cudaSuccess;
+        ok &= cudaEventRecord(dev->in_done[b], dev->s_in) == cudaSuccess;
+        // scan: needs the inputs, and the buffer's previous output (chunk c - 2) copied out
+        ok &= cudaStreamWaitEvent(dev->s_k, dev->in_done[b], 0) == cudaSuccess;
+        if (c >= 2) ok &= cudaStreamWaitEvent(dev->s_k, dev->out_done[b], 0) == cudaSuccess;
+        ok &= cudaMemsetAsync(buf[b] + plan.status_off, 0, plan.status_bytes, dev->s_k) == cudaSuccess;
+        if (!ok) return MMV_ERR_CUDA;
+        CUtensorMap tmap, tmap_out;
+        if (!encode_span_map(&tmap, xd, m, f16 ? 2 : 1, SCAN_UP)) return MMV_ERR_CUDA;
+        if (!encode_out_map(&tmap_out, od, m)) return MMV_ERR_CUDA;
+        ScanParams prm;
+        prm.x = xd;
+        prm.flags = fd;
+        prm.out = od;
+        prm.n = m;
+        prm.num_tiles = static_cast<int>(num_scan_tiles_of(m));
+        prm.hdr = hdr;
+        prm.status = reinterpret_cast<uint64_t*>(buf[b] + plan.status_off);
+        prm.budget_ns = g_budget_ns.load();
+        prm.debug_skip_span = -1;
+        prm.carry_in = carry;
+        const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
+        if (f16)
+            seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, dev->s_k>>>(tmap, tmap_out, prm);
+        else
+            seg_scan_kernel<I8Path><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, dev->s_k>>>(tmap, tmap_out, prm);
+        ++g_launches;
+        ok &= cudaGetLastError() == cudaSuccess;
+        ok &= cudaEventRecord(dev->k_done[b], dev->s_k) == cudaSuccess;
+        carry = od + static_cast<size_t>(m - 1) * 4;           // the running sum at the end of this chunk
+        // copy out
+        ok &= cudaStreamWaitEvent(dev->s_out, dev->k_done[b], 0) == cudaSuccess;
+        ok &= cudaMemcpyAsync(static_cast<uint8_t*>(out_host) + static_cast<size_t>(o) * 4, od, static_cast<size_t>(m) * 4,
+                              cudaMemcpyDeviceToHost, dev->s_out) == cudaSuccess;
+        ok &= cudaEventRecord(dev->out_done[b], dev->s_out) == cudaSuccess;
+        if (!ok) return MMV_ERR_CUDA;
+    }
+    // the caller's stream continues when everything is back on the host
+    ok &= cudaEventRecord(dev->ev_end_k, dev->s_k) == cudaSuccess;
+    ok &= cudaEventRecord(dev->ev_end_out, dev->s_out) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(user, dev->ev_end_k, 0) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(user, dev->ev_end_out, 0) == cudaSuccess;
+    return ok ? MMV_OK : MMV_ERR_CUDA;
 }
 
 mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
@@ -498,6 +641,7 @@ mmv_status mmv_seg_scan_static(const void* x, const void* flags_u8, int64_t n, m
     prm.status = reinterpret_cast<uint64_t*>(ws + sizeof(WorkspaceHeader));
     prm.budget_ns = g_budget_ns.load();
     prm.debug_skip_span = -1;
+    prm.carry_in = nullptr;
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
     if (f16)
         seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);

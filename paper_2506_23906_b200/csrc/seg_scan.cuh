@@ -43,6 +43,9 @@ struct ScanParams {
     uint64_t* status;            // one word per span
     unsigned long long budget_ns;
     long long debug_skip_span;   // test hook: this span never publishes (-1 = off)
+    const void* carry_in;        // device pointer to one fp32 / int32, or null: the running sum that
+                                 // reaches element 0 from an earlier chunk of the same vector (element 0
+                                 // then continues that segment unless its flag is set)
 };
 
 // Scan geometry: a warp owns a UNIT of SCAN_UP consecutive pieces (the grain of the carry
@@ -341,6 +344,10 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         // first accumulator column of this warp's unit, in its lane quarter
         int obuf = 0;
         bool failed = false;
+        // carry handed in by the caller (null: none); only read here, used much later
+        const bool has_in = prm.carry_in != nullptr;
+        uint32_t base_bits = 0u;
+        if (has_in) base_bits = *static_cast<const uint32_t*>(prm.carry_in);
 
         MMV_T_DECL
         // stages the 32 x 32 block held in r (lane = row) and stores it with one TMA store
@@ -476,11 +483,11 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 tail_tile = fj ? tj : P::add(tail_tile, tj);
                 flag_tile = flag_tile || fj;
             }
-            const bool need_global = !exflag && tile != 0;      // the carry reaches back past the tile
+            const bool need_global = !exflag && (tile != 0 || has_in);      // the carry reaches back past the tile
             const bool skip_publish = (prm.debug_skip_span >= 0) && ((prm.debug_skip_span >> 2) == tile);
             if (w == 0 && lane == 0 && !skip_publish)
                 st_relaxed_gpu_u64(prm.status + tile,
-                                   pack_status((flag_tile || tile == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail_tile)));
+                                   pack_status((flag_tile || (tile == 0 && !has_in)) ? ST_PREFIX : ST_AGG, P::to_bits(tail_tile)));
             MMV_T_MARK(3)
 
             // ---- main pass: everything that does not need the carry of earlier units ----
@@ -492,7 +499,8 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 #pragma unroll 1
             for (int i = 0; i < UP; ++i) {
                 // the first look-back window travels while the last piece is processed
-                if (i == UP - 1 && need_global && w == 0) lookback_load<SCAN_LB_WORDS>(prm.status, tile - 1, lbw);
+                if (i == UP - 1 && need_global && w == 0 && tile != 0)
+                    lookback_load<SCAN_LB_WORDS>(prm.status, tile - 1, lbw, base_bits);
                 uint32_t fmi = fm[0], pmi = pm[0];
                 Acc toti = tot[0];
 #pragma unroll
@@ -584,11 +592,15 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             if (w == 0) {
                 Acc carry_tile = Acc(0);
                 if (tile != 0) {
-                    if (!lookback<P, SCAN_LB_WORDS>(prm.status, tile, carry_tile, abort_flag, budget, lbw, true)) {
+                    if (!lookback<P, SCAN_LB_WORDS>(prm.status, tile, carry_tile, abort_flag, budget, lbw, true, base_bits)) {
                         if (lane == 0) st_relaxed_gpu_u64(prm.status + tile, pack_status(ST_ABORT, 0u));
                         failed = true;
                         break;
                     }
+                    if (!flag_tile && lane == 0 && !skip_publish)
+                        st_relaxed_gpu_u64(prm.status + tile, pack_status(ST_PREFIX, P::to_bits(P::add(carry_tile, tail_tile))));
+                } else if (has_in) {
+                    carry_tile = P::from_bits(base_bits);           // the first tile of a later chunk
                     if (!flag_tile && lane == 0 && !skip_publish)
                         st_relaxed_gpu_u64(prm.status + tile, pack_status(ST_PREFIX, P::to_bits(P::add(carry_tile, tail_tile))));
                 }

@@ -75,5 +75,13 @@ def test_argument_errors_are_synchronous(lib):
     assert lib.mmv_seg_sum(16, 16, 1, -5, 1, 0, 16, None, 256, 4096, None) == 1
     assert lib.mmv_seg_sum(16, 16, 0, 8, 0, 0, 16, None, 256, 16, None) == 3        # flag form: workspace too small
     assert lib.mmv_seg_sum(16, 16, 0, 8, 0, 0, 16, 12, 256, 1 << 20, None) == 1     # misaligned segment counter
+    lib.mmv_seg_scan_host.argtypes = [vp, vp, i64, ci, vp, i64, vp, sz, vp]
+    lib.mmv_seg_scan_host_scratch_bytes.restype = sz
+    lib.mmv_seg_scan_host_scratch_bytes.argtypes = [ci, i64]
+    assert lib.mmv_seg_scan_host(16, 16, 8, 0, 16, 1000, 256, 1 << 30, None) == 1     # chunk not a multiple of 16384
+    assert lib.mmv_seg_scan_host(16, 16, 8, 0, 16, 16384, 256, 16, None) == 3         # scratch too small
+    assert lib.mmv_seg_scan_host(None, None, 0, 0, None, 16384, None, 0, None) == 0   # nothing to do
+    assert lib.mmv_seg_scan_host_scratch_bytes(0, 1000) == 0
+    assert lib.mmv_seg_scan_host_scratch_bytes(0, 16384) >= 2 * 16384 * 7
     assert lib.mmv_spmv_csr(None, None, None, None, None, -1, 1, 1, None, 0, None) == 1
     assert lib.mmv_spmv_csr(None, None, None, None, None, 0, 1, 0, None, 0, None) == 0

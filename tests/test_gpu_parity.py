@@ -162,6 +162,30 @@ def test_config3_reduced_and_config5_cases_reduced(mmv):
 
 
 # ---------------------------------------------------------------------------
+# scan of host-resident vectors, chunk by chunk (carry handed from chunk to chunk on the device)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("n,chunk,p", [(5 * TILE + 123, TILE, 0.0), (5 * TILE + 123, TILE, 1e-3), (7 * TILE, 2 * TILE, 0.3),
+                                       (TILE - 5, TILE, 0.01), (40 * TILE + 1, 8 * TILE, 1e-5), (3 * TILE, 4 * TILE, 0.5)])
+def test_scan_of_host_vectors_in_chunks(mmv, n, chunk, p):
+    rng = np.random.default_rng(n + chunk)
+    f = (rng.random(n) < p).astype(np.uint8)
+    f[::chunk] |= (rng.random(f[::chunk].shape[0]) < 0.5).astype(np.uint8)      # some chunks start a segment, some continue
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    xf = rng.uniform(-1, 1, n).astype(np.float16)
+    for x in (xi, xf):
+        xh, fh = torch.from_numpy(x).pin_memory(), torch.from_numpy(f).pin_memory()
+        scratch = mmv.host_scan_scratch(mmv.I8_TO_I32 if x.dtype == np.int8 else mmv.F16_TO_F32, chunk)
+        out = mmv.seg_scan_host(xh, fh, chunk=chunk, scratch=scratch)
+        assert mmv.last_async_status(scratch) == 0            # synchronises the stream
+        got = out.numpy()
+        if x.dtype == np.int8:
+            assert np.array_equal(got, oracle.seg_scan_i8(x, f))
+        else:
+            z, a = oracle.seg_scan_f16(x, f)
+            assert_fp(got, z, a, f"host scan n={n} chunk={chunk} p={p}")
+
+
+# ---------------------------------------------------------------------------
 # segmented sum over CSR offsets
 # ---------------------------------------------------------------------------
 def sum_csr(mmv, x, off, guard=16):
