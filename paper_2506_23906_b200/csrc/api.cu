@@ -205,7 +205,7 @@ __global__ void spmv_gather_kernel(const int32_t* __restrict__ col, const __half
 template <typename P>
 mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* off, long long nseg, int shift,
                           void* out, uint8_t* ws, const WorkspacePlan& plan, DeviceInfo* dev, cudaStream_t st,
-                          const long long* nseg_dev = nullptr) {
+                          const long long* nseg_dev = nullptr, const int* shape_sel = nullptr) {
     const int tiles = static_cast<int>(num_tiles_of(n_eff));
     int32_t* span_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
     {
@@ -231,9 +231,18 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();
     prm.nseg_dev = nseg_dev;
+    prm.shape_sel = shape_sel;
     const int grid = tiles < dev->sm_count ? tiles : dev->sm_count;
     // Long segments (few boundaries per 4096-element span): sixteen epilogue warps on the light path.
     // The segment count of the flag-encoded form is not known here; it takes the eight-warp kernel.
+    if (shape_sel) {
+        // flag-encoded segments: their number is only known on the device, which has left its choice
+        // in *shape_sel; both shapes are launched and the other one returns at once
+        seg_sum_kernel<P, 2><<<grid, SumShape<2>::kThreads, SumCfg<P, 2>::kSmemBytes, st>>>(tmap, values, prm);
+        seg_sum_kernel<P, 4><<<grid, SumShape<4>::kThreads, SumCfg<P, 4>::kSmemBytes, st>>>(tmap, values, prm);
+        g_launches += 2;
+        return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+    }
     bool many_warps = !nseg_dev && nseg > 0 && n_eff / nseg >= 256;
     if (g_force_groups.load() == 2) many_warps = false;
     if (g_force_groups.load() == 4) many_warps = true;
@@ -536,13 +545,14 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
         const long long cap = static_cast<long long>(dev->sm_count) * 8;
         const unsigned blocks = static_cast<unsigned>(nchunks < cap ? nchunks : cap);
         flag_count_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_count);
+        int* shape_sel = reinterpret_cast<int*>(ws + plan.cmp_off + 8);
         chunk_scan_kernel<<<1, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, nseg_dev,
-                                              reinterpret_cast<long long*>(d_num_segments), off, n);
+                                              reinterpret_cast<long long*>(d_num_segments), off, n, shape_sel);
         flag_scatter_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_base, off);
         g_launches += 3;
         if (cudaGetLastError() != cudaSuccess) return MMV_ERR_CUDA;
-        if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev);
-        return launch_seg_sum<I8Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev);
+        if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, shape_sel);
+        return launch_seg_sum<I8Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, shape_sel);
     }
     if (nseg == 0) return MMV_OK;
     if (!seg || !out) return MMV_ERR_INVALID_ARG;

@@ -84,11 +84,11 @@ flag_count_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks,
 }
 
 // One block: chunk_base = exclusive scan of chunk_count; K = total is written to nseg_dev and, when given,
-// to the caller's d_num_segments; off[K] = n closes the last segment.
+// to the caller's d_num_segments; off[K] = n closes the last segment; *shape_sel picks the kernel shape.
 __global__ void __launch_bounds__(1024)
 chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, int32_t* __restrict__ chunk_base,
                   long long* __restrict__ nseg_dev, long long* __restrict__ d_num_segments, int32_t* __restrict__ off,
-                  long long n) {
+                  long long n, int* __restrict__ shape_sel) {
     __shared__ int warp_sums[32];
     const long long per = (nchunks + blockDim.x - 1) / blockDim.x;
     const long long lo = static_cast<long long>(threadIdx.x) * per;
@@ -105,6 +105,8 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
         *nseg_dev = total;
         if (d_num_segments) *d_num_segments = total;
         off[total] = static_cast<int32_t>(n);
+        // long segments on average: the segmented-sum kernel with sixteen epilogue warps takes the call
+        *shape_sel = (total > 0 && n / total >= 256) ? 4 : 2;
     }
 }
 

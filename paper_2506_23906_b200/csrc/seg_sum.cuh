@@ -192,6 +192,8 @@ struct SumParams {
     unsigned long long budget_ns;
     const long long* nseg_dev;   // when not null: the number of segments is read from here (flag-encoded
                                  // segments, whose count is only known on the device); nseg is ignored
+    const int* shape_sel;        // when not null: both kernel shapes are launched and the one whose G
+                                 // differs from *shape_sel returns at once (the choice depends on nseg)
 };
 
 // span_q[s] = first index q in [0, nseg] with (off[q] << shift) >= s * SPAN, nseg + 1 if none.
@@ -243,6 +245,7 @@ template <typename P, int G>
 __global__ void __launch_bounds__(SumShape<G>::kThreads, 1)
 seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restrict__ xg, const SumParams prm) {
     using Acc = typename P::Acc;
+    if (prm.shape_sel && *prm.shape_sel != G) return;      // the other shape does this call
     using Cfg = SumCfg<P, G>;
     using Shape = SumShape<G>;
     constexpr int BPG = Shape::kBufsPerGroup;
