@@ -229,10 +229,33 @@ def event_time_ms(torch, fn, steps, flush=None):
     return total / steps
 
 
-def bench_configs(torch, mmv, peak, steps, warmup, l2_flush):
-    """Short measurements of the five configurations (device-resident inputs).  Timing only: parity at
-    these sizes is checked by tests/test_gpu_full_size.py, which makes the same calls."""
+def bench_configs(torch, mmv, peak, steps, warmup, l2_flush, cpu_leg):
+    """Short measurements of the five configurations (device-resident inputs).  With cpu_leg the
+    oracle is timed on one host core over the whole input of every configuration (the baseline leg)
+    and, its result being in hand, the device result is compared with it.  Parity at these sizes is
+    also a test: tests/test_gpu_full_size.py makes the same calls."""
     res = []
+
+    def baseline(units, run_oracle, compare):
+        """One run of the oracle over the whole configuration -> the record's cpu_baseline entry."""
+        if not cpu_leg:
+            return {}
+        import oracle
+        t0 = time.perf_counter()
+        want = run_oracle(oracle)
+        sec = time.perf_counter() - t0
+        d = {"value": units / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+             "sample": f"the whole configuration, one run, {sec:.2f} s"}
+        d.update(compare(oracle, want))
+        return {"cpu_baseline": d}
+
+    def fp_compare(got):
+        def cmp(oracle, want):
+            ok, ratio, i = oracle.check_fp(got, want[0], want[1])
+            if not ok:
+                raise SystemExit(f"bench: device result outside the bound (ratio {ratio} at {i})")
+            return {"device_result_worst_err_over_bound": ratio}
+        return cmp
 
     def rec(name, units, bytes_, ms, extra=None):
         d = {"config": name, "units": int(units), "ms": ms, "gelem_s": units / ms / 1e6,
@@ -255,7 +278,16 @@ def bench_configs(torch, mmv, peak, steps, warmup, l2_flush):
         ms = event_time_ms(torch, fn, steps, flush)
         assert mmv.last_async_status(ws) == 0
         bpe = (2 if dt == mmv.F16_TO_F32 else 1) + 1 + 4
-        rec(name, n, n * bpe, ms)
+        if dt == mmv.F16_TO_F32:
+            extra = baseline(n, lambda o: o.seg_scan_f16(x, f), fp_compare(out.cpu().numpy()))
+        else:
+            def cmp_int(oracle, want):
+                bad = int(np.count_nonzero(out.cpu().numpy() != want))
+                if bad:
+                    raise SystemExit(f"bench: {bad} mismatches in {name}")
+                return {"device_result_mismatches": 0}
+            extra = baseline(n, lambda o: o.seg_scan_i8(x, f), cmp_int)
+        rec(name, n, n * bpe, ms, extra)
         del xd, fd, out, ws
 
     x, f = gen.config1()
@@ -273,7 +305,7 @@ def bench_configs(torch, mmv, peak, steps, warmup, l2_flush):
     ms = event_time_ms(torch, fn, steps)
     assert mmv.last_async_status(ws) == 0
     rec("C2 seg-sum n=2^26 fp16 N(0,1), CSR offsets len U{1..4096}", n, 2 * n + 4 * (nseg + 1) + 4 * nseg, ms,
-        {"segments": nseg})
+        {"segments": nseg, **baseline(n, lambda o: o.seg_sum_csr_f16(x, off), fp_compare(out.cpu().numpy()))})
     del xd, od, out, ws
 
     # the same recipe four times larger (the n >= 2^28 point of the target), and the flag-encoded
@@ -290,7 +322,7 @@ def bench_configs(torch, mmv, peak, steps, warmup, l2_flush):
     ms = event_time_ms(torch, fn, steps)
     assert mmv.last_async_status(ws) == 0
     rec("C2x4 seg-sum n=2^28 fp16 N(0,1), CSR offsets len U{1..4096}", n, 2 * n + 4 * (nseg + 1) + 4 * nseg, ms,
-        {"segments": nseg})
+        {"segments": nseg, **baseline(n, lambda o: o.seg_sum_csr_f16(x, off), fp_compare(out.cpu().numpy()))})
     del od, ws
     f = gen.start_flags_of_offsets(off, n)
     fd = torch.from_numpy(f).cuda()
@@ -307,26 +339,29 @@ def bench_configs(torch, mmv, peak, steps, warmup, l2_flush):
     if k != nseg - int(np.count_nonzero(np.diff(off.astype(np.int64)) == 0)):
         raise SystemExit(f"bench: flag-form seg-sum found {k} segments")
     rec("N1 seg-sum (start flags) n=2^28 fp16 N(0,1), same segments as C2x4", n, 2 * n + n + 4 * k, ms,
-        {"segments": k})
+        {"segments": k, **baseline(n, lambda o: o.seg_sum_flags_f16(x, f), fp_compare(outf[:k].cpu().numpy()))})
     del xd, fd, out, outf, ws
 
     x, f = gen.config3()
     run_scan("C3 seg-scan n=2^28 int8 flags 1e-3", x, f)
 
-    rowptr, col, val, xv = gen.config4()
-    rows, nnz = rowptr.shape[0] - 1, val.shape[0]
-    rd, cd, vd, xd = (torch.from_numpy(t).cuda() for t in (rowptr, col, val, xv))
-    y = torch.empty(rows, dtype=torch.float32, device="cuda")
-    ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, nnz, rows)
-    fn = lambda: mmv.spmv_csr(rd, cd, vd, xd, y=y, workspace=ws)  # noqa: E731
-    for _ in range(warmup):
-        fn()
-    torch.cuda.synchronize()
-    ms = event_time_ms(torch, fn, steps)
-    assert mmv.last_async_status(ws) == 0
-    rec("C4 CSR SpMV 2^20 rows, nnz/row Zipf(1.5) cap 1e4", nnz, 6 * nnz + 4 * (rows + 1) + 4 * xv.shape[0] + 4 * rows,
-        ms, {"nnz": nnz})
-    del rd, cd, vd, xd, y, ws
+    # configuration 4, and the same with 10 % of the rows empty (the paper's corner case of empty rows)
+    for name, empty in (("C4 CSR SpMV 2^20 rows, nnz/row Zipf(1.5) cap 1e4", 0.0),
+                        ("C4e the same with 10 % of the rows empty", 0.1)):
+        rowptr, col, val, xv = gen.config4(empty_fraction=empty)
+        rows, nnz = rowptr.shape[0] - 1, val.shape[0]
+        rd, cd, vd, xd = (torch.from_numpy(t).cuda() for t in (rowptr, col, val, xv))
+        y = torch.empty(rows, dtype=torch.float32, device="cuda")
+        ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, nnz, rows)
+        fn = lambda: mmv.spmv_csr(rd, cd, vd, xd, y=y, workspace=ws)  # noqa: E731
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        ms = event_time_ms(torch, fn, steps)
+        assert mmv.last_async_status(ws) == 0
+        rec(name, nnz, 6 * nnz + 4 * (rows + 1) + 4 * xv.shape[0] + 4 * rows, ms,
+            {"nnz": nnz, **baseline(nnz, lambda o: o.spmv_csr(rowptr, col, val, xv), fp_compare(y.cpu().numpy()))})
+        del rd, cd, vd, xd, y, ws
     torch.cuda.empty_cache()
     return res
 
@@ -454,7 +489,7 @@ def run_ours(args):
         if world == 1 and not args.no_configs:
             def l2_flush():
                 l2_buf.zero_()
-            cfgs = bench_configs(torch, mmv, peak, min(args.steps, 20), max(3, args.warmup), l2_flush)
+            cfgs = bench_configs(torch, mmv, peak, min(args.steps, 20), max(3, args.warmup), l2_flush, not args.no_cpu)
             # the seven flag patterns of configuration 5 on the headline values
             xd = torch.from_numpy(x).cuda()
             od = torch.empty(n, dtype=torch.float32, device="cuda")

@@ -116,8 +116,9 @@ def test_config2_full_size_and_four_times_larger_with_both_encodings(mmv):
         torch.cuda.empty_cache()
 
 
-def test_config4_full_size(mmv):
-    rowptr, col, val, xv = gen.config4()
+@pytest.mark.parametrize("empty_fraction", [0.0, 0.1])
+def test_config4_full_size(mmv, empty_fraction):
+    rowptr, col, val, xv = gen.config4(empty_fraction=empty_fraction)
     rows = rowptr.shape[0] - 1
     ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, val.shape[0], rows)
     y = mmv.spmv_csr(torch.from_numpy(rowptr).cuda(), torch.from_numpy(col).cuda(), torch.from_numpy(val).cuda(),
@@ -125,4 +126,7 @@ def test_config4_full_size(mmv):
     assert mmv.last_async_status(ws) == 0
     want, a = oracle.spmv_csr(rowptr, col, val, xv)
     ok, ratio, i = oracle.check_fp(y.cpu().numpy(), want, a)
-    assert ok, f"config 4: ratio {ratio} at row {i}"
+    assert ok, f"config 4 (empty rows {empty_fraction}): ratio {ratio} at row {i}"
+    if empty_fraction:
+        lens = np.diff(rowptr.astype(np.int64))
+        assert (y.cpu().numpy()[lens == 0] == 0).all()
