@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS = 8000.0
 # the ~57 MB of output that are still in L2 when a launch ends; both scale with n.
 NCU_READ_BYTES_PER_ELEM = 3.001
 NCU_WRITE_BYTES_PER_ELEM = 4.0
-NCU_WRITE_L2_RESIDUE_BYTES = 58.9e6
+NCU_WRITE_L2_RESIDUE_BYTES = 59.0e6
 
 
 def parse_args():
@@ -507,6 +507,16 @@ def run_ours(args):
                               "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
                               "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
                 del fd
+            # the plain scan: no flag vector at all (6 B per element)
+            fn = lambda: mmv.seg_scan(xd, None, out=od, workspace=ws)  # noqa: E731
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            cms = event_time_ms(torch, fn, min(args.steps, 10))
+            assert mmv.last_async_status(ws) == 0
+            sweep.append({"case": "no flag vector (plain scan, 6 B/elem)", "ms": cms, "gelem_s": n / cms / 1e6,
+                          "gb_s": 6 * n / cms / 1e6, "frac_of_measured_peak": 6 * n / cms / 1e6 / peak,
+                          "frac_of_8tbs": 6 * n / cms / 1e6 / NOMINAL_HBM_GBS})
             line["configs"] = cfgs
             line["c5_density_sweep"] = sweep
         print(json.dumps(line))

@@ -86,7 +86,9 @@ size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, in
  *     out[i] = out[i-1] + x[i]    otherwise
  * x: n values (fp16 or int8 per dt).  seg: n flag bytes, or nseg+1 offsets with
  * off[0] == 0 and off[nseg] == n (empty segments allowed, they start nothing).
- * out: n values (fp32 or int32).  Elements past n are never written.
+ * With sf == MMV_SEG_FLAGS_U8, seg may be NULL: the whole vector is one segment
+ * (the plain inclusive scan, the case Algorithm 4.1 treats) and no flag bytes
+ * are read.  out: n values (fp32 or int32).  Elements past n are never written.
  */
 mmv_status mmv_seg_scan(const void *x, const void *seg, mmv_segfmt sf, int64_t n, int64_t nseg,
                         mmv_dtype dt, void *out,
@@ -179,7 +181,7 @@ mmv_status mmv_seg_scan_static_last_status(void *cuda_stream);
 
 /*
  * Segmented scan (Problem 2.1) of vectors that live in HOST memory: x_host (n values), flags_host
- * (n start-flag bytes) and out_host (n results) are host pointers.  The vectors are cut into
+ * (n start-flag bytes, or NULL for one segment) and out_host (n results) are host pointers.  The vectors are cut into
  * chunks of chunk_elems elements (a positive multiple of 16384); the chunks are copied to the
  * device, scanned and copied back on three internal streams, so that the copy-in, the kernels
  * and the copy-out of neighbouring chunks overlap; the running sum at the end of a chunk is

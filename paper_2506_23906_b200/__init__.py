@@ -136,11 +136,12 @@ def last_async_status(workspace: torch.Tensor, stream=None) -> int:
     return int(_lib.mmv_last_async_status(_ptr(workspace), _stream_ptr(stream)))
 
 
-def seg_scan(x: torch.Tensor, seg: torch.Tensor, out: torch.Tensor | None = None,
+def seg_scan(x: torch.Tensor, seg: torch.Tensor | None, out: torch.Tensor | None = None,
              workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
-    """mmv_seg_scan: segmented inclusive scan (Problem 2.1, Eq. 1) of x over seg."""
+    """mmv_seg_scan: segmented inclusive scan (Problem 2.1, Eq. 1) of x over seg; seg = None is the
+    plain inclusive scan (one segment, no flag vector is read)."""
     _check_cuda(x, seg, out, workspace)
-    dt, sf = _dtype_code(x), _seg_code(seg)
+    dt, sf = _dtype_code(x), (SEG_FLAGS_U8 if seg is None else _seg_code(seg))
     n = x.numel()
     nseg = seg.numel() - 1 if sf == SEG_OFFSETS_I32 else 0
     if out is None:
@@ -177,14 +178,14 @@ def host_scan_scratch(dt: int, chunk: int, device=None) -> torch.Tensor:
     return torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
 
 
-def seg_scan_host(x: torch.Tensor, flags: torch.Tensor, out: torch.Tensor | None = None, chunk: int = 1 << 26,
+def seg_scan_host(x: torch.Tensor, flags: torch.Tensor | None, out: torch.Tensor | None = None, chunk: int = 1 << 26,
                   scratch: torch.Tensor | None = None, stream=None) -> torch.Tensor:
     """mmv_seg_scan_host: the scan of HOST tensors (pinned memory recommended), copies and kernels
     of neighbouring chunks overlapped.  Returns ``out`` (a pinned host tensor unless one is given);
     the results are complete once the stream has been synchronised."""
-    if x.is_cuda or flags.is_cuda or (out is not None and out.is_cuda):
+    if x.is_cuda or (flags is not None and flags.is_cuda) or (out is not None and out.is_cuda):
         raise ValueError("seg_scan_host takes host tensors")
-    if flags.dtype != torch.uint8 or not x.is_contiguous() or not flags.is_contiguous():
+    if not x.is_contiguous() or (flags is not None and (flags.dtype != torch.uint8 or not flags.is_contiguous())):
         raise TypeError("contiguous values and uint8 start flags expected")
     dt = _dtype_code(x)
     n = x.numel()

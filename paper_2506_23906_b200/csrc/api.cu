@@ -323,7 +323,8 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
     if (n == 0) return MMV_OK;
     if (n >= (1ll << 36)) return MMV_ERR_UNSUPPORTED;
     if (sf == MMV_SEG_OFFSETS_I32 && n >= (1ll << 31)) return MMV_ERR_INVALID_ARG;
-    if (!x || !seg || !out || !workspace) return MMV_ERR_INVALID_ARG;
+    if (!x || !out || !workspace) return MMV_ERR_INVALID_ARG;
+    if (!seg && sf != MMV_SEG_FLAGS_U8) return MMV_ERR_INVALID_ARG;           // no flags = one segment; offsets must exist
     if (!aligned16(x) || !aligned16(seg) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
         return MMV_ERR_INVALID_ARG;
     if (sf == MMV_SEG_OFFSETS_I32 && nseg == 0) return MMV_ERR_INVALID_ARG;   // n > 0 needs a segment
@@ -431,7 +432,7 @@ mmv_status mmv_seg_scan_host(const void* x_host, const void* flags_host, int64_t
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
     if (chunk_elems <= 0 || chunk_elems % SCAN_TILE != 0 || chunk_elems >= (1ll << 36)) return MMV_ERR_INVALID_ARG;
     if (n == 0) return MMV_OK;
-    if (!x_host || !flags_host || !out_host || !device_scratch) return MMV_ERR_INVALID_ARG;
+    if (!x_host || !out_host || !device_scratch) return MMV_ERR_INVALID_ARG;      // flags_host may be null: one segment
     if (reinterpret_cast<uintptr_t>(device_scratch) & 255u) return MMV_ERR_INVALID_ARG;
     const HostScanPlan plan = plan_host_scan(dt, chunk_elems);
     if (device_scratch_bytes < plan.total) return MMV_ERR_WORKSPACE_TOO_SMALL;
@@ -465,8 +466,9 @@ mmv_status mmv_seg_scan_host(const void* x_host, const void* flags_host, int64_t
         if (c >= 2) ok &= cudaStreamWaitEvent(dev->s_in, dev->k_done[b], 0) == cudaSuccess;
         ok &= cudaMemcpyAsync(xd, static_cast<const uint8_t*>(x_host) + static_cast<size_t>(o) * eb, static_cast<size_t>(m) * eb,
                               cudaMemcpyHostToDevice, dev->s_in) == cudaSuccess;
-        ok &= cudaMemcpyAsync(fd, static_cast<const uint8_t*>(flags_host) + o, static_cast<size_t>(m), cudaMemcpyHostToDevice,
-                              dev->s_in) == cudaSuccess;
+        if (flags_host)
+            ok &= cudaMemcpyAsync(fd, static_cast<const uint8_t*>(flags_host) + o, static_cast<size_t>(m),
+                                  cudaMemcpyHostToDevice, dev->s_in) == cudaSuccess;
         ok &= cudaEventRecord(dev->in_done[b], dev->s_in) == cudaSuccess;
         // scan: needs the inputs, and the buffer's previous output (chunk c - 2) copied out
         ok &= cudaStreamWaitEvent(dev->s_k, dev->in_done[b], 0) == cudaSuccess;
@@ -478,7 +480,7 @@ mmv_status mmv_seg_scan_host(const void* x_host, const void* flags_host, int64_t
         if (!encode_out_map(&tmap_out, od, m)) return MMV_ERR_CUDA;
         ScanParams prm;
         prm.x = xd;
-        prm.flags = fd;
+        prm.flags = flags_host ? fd : nullptr;
         prm.out = od;
         prm.n = m;
         prm.num_tiles = static_cast<int>(num_scan_tiles_of(m));

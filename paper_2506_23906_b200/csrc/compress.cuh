@@ -93,13 +93,17 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
     const long long per = (nchunks + blockDim.x - 1) / blockDim.x;
     const long long lo = static_cast<long long>(threadIdx.x) * per;
     const long long hi = lo + per < nchunks ? lo + per : nchunks;
+    // (loads batched eight at a time: the kernel is one block, so it runs at the latency of its loads)
     int local = 0;
-    for (long long c = lo; c < hi; ++c) local += chunk_count[c];
+#pragma unroll 8
+    for (long long c = lo; c < hi; ++c) local += __ldg(chunk_count + c);
     int total;
     int run = block_exclusive_scan(local, &total, warp_sums);
+#pragma unroll 8
     for (long long c = lo; c < hi; ++c) {
+        const int cnt = __ldg(chunk_count + c);
         chunk_base[c] = run;
-        run += chunk_count[c];
+        run += cnt;
     }
     if (threadIdx.x == 0) {
         *nseg_dev = total;

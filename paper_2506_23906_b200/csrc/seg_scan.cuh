@@ -35,7 +35,7 @@ namespace mmv {
 
 struct ScanParams {
     const void* x;
-    const uint8_t* flags;
+    const uint8_t* flags;        // start flags, or null: one segment (the plain scan of Algorithm 4.1; no flag traffic)
     void* out;
     long long n;
     int num_tiles;
@@ -238,17 +238,17 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             const long long tbase = static_cast<long long>(tile) * SCAN_TILE;
             if (tbase + SCAN_TILE <= prm.n) {
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&bar_full[stage], Cfg::kStageBytes);
+                    mbar_arrive_expect_tx(&bar_full[stage], prm.flags ? Cfg::kStageBytes : Cfg::kXBytes);
 #pragma unroll
                     for (int i = 0; i < SCAN_UP; ++i)
                         tma_load_4d(xs + i * P::kSlabBytes, &tmap_x, &bar_full[stage], 0, 0, i, tile * SPANS_PER_TILE);
-                    tma_load_1d(fs, prm.flags + tbase, Cfg::kFlagBytes, &bar_full[stage]);
+                    if (prm.flags) tma_load_1d(fs, prm.flags + tbase, Cfg::kFlagBytes, &bar_full[stage]);
                 }
             } else {
                 // ragged last tile: plain loads, zero fill past n (MATMUL zero-pads its operand)
                 const long long cnt = prm.n - tbase;
 #pragma unroll 1
-                for (int v = lane; v < SCAN_TILE / 16; v += 32) {
+                for (int v = lane; v < (prm.flags ? SCAN_TILE / 16 : 0); v += 32) {
                     const int e0 = v * 16;
                     uint4 fv = make_uint4(0u, 0u, 0u, 0u);
                     if (e0 + 16 <= cnt) {
@@ -397,10 +397,13 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 const uint8_t* fs = sStage + stage * Cfg::kStageBytes + Cfg::kXBytes + w * SCAN_UNIT + lane * ROW;
 #pragma unroll
                 for (int i = 0; i < UP; ++i) {
-                    const uint4 a = *reinterpret_cast<const uint4*>(fs + i * PIECE);
-                    const uint4 b = *reinterpret_cast<const uint4*>(fs + i * PIECE + 16);
-                    const uint32_t any = a.x | a.y | a.z | a.w | b.x | b.y | b.z | b.w;
-                    fm[i] = any ? flag_bytes_to_mask(a, b) : 0u;
+                    fm[i] = 0u;
+                    if (prm.flags) {
+                        const uint4 a = *reinterpret_cast<const uint4*>(fs + i * PIECE);
+                        const uint4 b = *reinterpret_cast<const uint4*>(fs + i * PIECE + 16);
+                        const uint32_t any = a.x | a.y | a.z | a.w | b.x | b.y | b.z | b.w;
+                        fm[i] = any ? flag_bytes_to_mask(a, b) : 0u;
+                    }
                     pm[i] = __ballot_sync(0xffffffffu, fm[i] != 0u);
                 }
             }

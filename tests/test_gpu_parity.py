@@ -161,6 +161,31 @@ def test_config3_reduced_and_config5_cases_reduced(mmv):
         assert_fp(scan_f16(mmv, xv, f), z, a, f"config 5 / {case}")
 
 
+def test_plain_scan_without_a_flag_vector(mmv):
+    # seg = None: one segment, the kernel reads no flags at all; same result as all-zero flags
+    rng = np.random.default_rng(7)
+    for n in (1, 33, TILE - 1, 3 * TILE + 4099):
+        xi = rng.integers(-128, 128, n).astype(np.int8)
+        zero = np.zeros(n, np.uint8)
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+        got = mmv.seg_scan(dev(xi), None, workspace=ws).cpu().numpy()
+        assert mmv.last_async_status(ws) == 0
+        assert np.array_equal(got, oracle.seg_scan_i8(xi, zero))
+        xf = rng.uniform(-1, 1, n).astype(np.float16)
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+        got = mmv.seg_scan(dev(xf), None, workspace=ws).cpu().numpy()
+        z, a = oracle.seg_scan_f16(xf, zero)
+        assert_fp(got, z, a, f"plain scan n={n}")
+    # host vectors, chunked, no flags
+    n = 9 * TILE + 17
+    xf = rng.uniform(-1, 1, n).astype(np.float16)
+    scratch = mmv.host_scan_scratch(mmv.F16_TO_F32, 2 * TILE)
+    out = mmv.seg_scan_host(torch.from_numpy(xf).pin_memory(), None, chunk=2 * TILE, scratch=scratch)
+    assert mmv.last_async_status(scratch) == 0
+    z, a = oracle.seg_scan_f16(xf, np.zeros(n, np.uint8))
+    assert_fp(out.numpy(), z, a, "plain host scan")
+
+
 # ---------------------------------------------------------------------------
 # scan of host-resident vectors, chunk by chunk (carry handed from chunk to chunk on the device)
 # ---------------------------------------------------------------------------
