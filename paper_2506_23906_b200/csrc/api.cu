@@ -208,7 +208,7 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
                           const long long* nseg_dev = nullptr, const int* shape_sel = nullptr) {
     const int tiles = static_cast<int>(num_tiles_of(n_eff));
     int32_t* span_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
-    {
+    if (!shape_sel) {          // (the flag-encoded form has filled span_q while compacting its flags)
         const long long spans = static_cast<long long>(tiles) * SPANS_PER_TILE;
         const long long warps = spans + 1;
         const int threads = 256;
@@ -550,7 +550,9 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
         int* shape_sel = reinterpret_cast<int*>(ws + plan.cmp_off + 8);
         chunk_scan_kernel<<<1, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, nseg_dev,
                                               reinterpret_cast<long long*>(d_num_segments), off, n, shape_sel);
-        flag_scatter_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_base, off);
+        static_assert(CMP_CHUNK == TILE && SPAN == 4096, "a compaction chunk is one tile of four spans");
+        flag_scatter_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_base, off,
+                                                            reinterpret_cast<int32_t*>(ws + plan.tileq_off), nseg_dev);
         g_launches += 3;
         if (cudaGetLastError() != cudaSuccess) return MMV_ERR_CUDA;
         if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, shape_sel);

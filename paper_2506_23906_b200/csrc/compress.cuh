@@ -114,11 +114,21 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
     }
 }
 
-// off[chunk_base[c] + j] = position of the j-th start flag of chunk c (in order).
+// off[chunk_base[c] + j] = position of the j-th start flag of chunk c (in order).  A chunk is four
+// 4096-element spans of the segmented-sum kernel, and the number of starts in front of a span is
+// exactly that kernel's span_q entry (the first offset index at or after the span's start), so
+// the span partition comes for free here: span_q[s] = #starts before s * 4096, K when the span
+// starts at n, K + 1 ("none") beyond.
 __global__ void __launch_bounds__(CMP_THREADS)
 flag_scatter_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks, const int32_t* __restrict__ chunk_base,
-                    int32_t* __restrict__ off) {
+                    int32_t* __restrict__ off, int32_t* __restrict__ span_q, const long long* __restrict__ nseg_dev) {
     __shared__ int warp_sums[32];
+    constexpr int kThreadsPerSpan = 4096 / CMP_PER_THREAD;
+    const long long K = *nseg_dev;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const long long end = nchunks * CMP_CHUNK;
+        span_q[nchunks * (CMP_CHUNK / 4096)] = static_cast<int32_t>(end == n ? K : K + 1);
+    }
     for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
         const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
         uint32_t w[16];
@@ -128,6 +138,9 @@ flag_scatter_kernel(const uint8_t* __restrict__ f, long long n, long long nchunk
         for (int i = 0; i < 16; ++i) cnt += nonzero_bytes(w[i]);
         int total;
         int slot = chunk_base[c] + block_exclusive_scan(cnt, &total, warp_sums);
+        if (threadIdx.x % kThreadsPerSpan == 0)
+            span_q[c * (CMP_CHUNK / 4096) + threadIdx.x / kThreadsPerSpan] =
+                static_cast<int32_t>(base < n ? slot : (base == n ? K : K + 1));
         if (cnt) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
