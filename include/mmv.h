@@ -210,10 +210,10 @@ mmv_status mmv_seg_scan_host(const void *x_host, const void *flags_host, int64_t
 void mmv_debug_configure(int64_t wait_budget_ns, int64_t skip_publish_span);
 
 /*
- * Test hook.  The segmented-sum kernel exists with two and with four epilogue
+ * Test hook.  The segmented-sum kernel exists with two and with three epilogue
  * warpgroups; the library picks one from the average segment length.  groups =
- * 2 or 4 forces that variant for the offsets form (the SpMV and flag-encoded
- * paths always use two), 0 restores the automatic choice.
+ * 2 or 3 forces that variant for the offsets form and SpMV, 0 restores the
+ * automatic choice.
  */
 void mmv_debug_force_sum_groups(int groups);
 

@@ -75,9 +75,9 @@ DeviceInfo* device_info() {
         ok &= set_smem(seg_sum_kernel<F16Path, 2>, SumCfg<F16Path, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<I8Path, 2>, SumCfg<I8Path, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<BF16Path, 2>, SumCfg<BF16Path, 2>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<F16Path, 4>, SumCfg<F16Path, 4>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<I8Path, 4>, SumCfg<I8Path, 4>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<BF16Path, 4>, SumCfg<BF16Path, 4>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<F16Path, 3>, SumCfg<F16Path, 3>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<I8Path, 3>, SumCfg<I8Path, 3>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<BF16Path, 3>, SumCfg<BF16Path, 3>::kSmemBytes);
         d->ok = ok;
     });
     return d->ok ? d : nullptr;
@@ -233,27 +233,22 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     prm.nseg_dev = nseg_dev;
     prm.shape_sel = shape_sel;
     const int grid = tiles < dev->sm_count ? tiles : dev->sm_count;
-    // Long segments (few boundaries per 4096-element span): sixteen epilogue warps on the light path.
-    // The segment count of the flag-encoded form is not known here; it takes the eight-warp kernel.
     if (shape_sel) {
         // flag-encoded segments: their number is only known on the device, which has left its choice
         // in *shape_sel; both shapes are launched and the other one returns at once
         seg_sum_kernel<P, 2><<<grid, SumShape<2>::kThreads, SumCfg<P, 2>::kSmemBytes, st>>>(tmap, values, prm);
-        seg_sum_kernel<P, 4><<<grid, SumShape<4>::kThreads, SumCfg<P, 4>::kSmemBytes, st>>>(tmap, values, prm);
+        seg_sum_kernel<P, 3><<<grid, SumShape<3>::kThreads, SumCfg<P, 3>::kSmemBytes, st>>>(tmap, values, prm);
         g_launches += 2;
         return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
     }
-    bool many_warps = !nseg_dev && nseg > 0 && n_eff / nseg >= 256;
+    // Long segments (few boundaries per 4096-element span): twelve epilogue warps on the light path.
+    bool many_warps = nseg > 0 && n_eff / nseg >= 256;
     if (g_force_groups.load() == 2) many_warps = false;
-    if (g_force_groups.load() == 4) many_warps = true;
-    {
-        if (many_warps) {
-            seg_sum_kernel<P, 4><<<grid, SumShape<4>::kThreads, SumCfg<P, 4>::kSmemBytes, st>>>(tmap, values, prm);
-            ++g_launches;
-            return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
-        }
-    }
-    seg_sum_kernel<P, 2><<<grid, SumShape<2>::kThreads, SumCfg<P, 2>::kSmemBytes, st>>>(tmap, values, prm);
+    if (g_force_groups.load() == 3) many_warps = true;
+    if (many_warps)
+        seg_sum_kernel<P, 3><<<grid, SumShape<3>::kThreads, SumCfg<P, 3>::kSmemBytes, st>>>(tmap, values, prm);
+    else
+        seg_sum_kernel<P, 2><<<grid, SumShape<2>::kThreads, SumCfg<P, 2>::kSmemBytes, st>>>(tmap, values, prm);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
@@ -696,7 +691,7 @@ void mmv_debug_phase_cycles(unsigned long long* host16) {
 }
 #endif
 
-void mmv_debug_force_sum_groups(int groups) { g_force_groups.store(groups == 2 || groups == 4 ? groups : 0); }
+void mmv_debug_force_sum_groups(int groups) { g_force_groups.store(groups == 2 || groups == 3 ? groups : 0); }
 
 void mmv_debug_configure(int64_t wait_budget_ns, int64_t skip_publish_span) {
     g_budget_ns.store(wait_budget_ns > 0 ? static_cast<unsigned long long>(wait_budget_ns) : WAIT_BUDGET_NS);

@@ -109,8 +109,8 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
         *nseg_dev = total;
         if (d_num_segments) *d_num_segments = total;
         off[total] = static_cast<int32_t>(n);
-        // long segments on average: the segmented-sum kernel with sixteen epilogue warps takes the call
-        *shape_sel = (total > 0 && n / total >= 256) ? 4 : 2;
+        // long segments on average: the segmented-sum kernel with twelve epilogue warps takes the call
+        *shape_sel = (total > 0 && n / total >= 256) ? 3 : 2;
     }
 }
 

@@ -28,21 +28,22 @@
 
 namespace mmv {
 
-// The kernel comes with G = 2 or 4 epilogue warpgroups (4 G epilogue warps, then the TMA producer
+// The kernel comes with G = 2 or 3 epilogue warpgroups (4 G epilogue warps, then the TMA producer
 // warp and the MMA warp).  The epilogue is a chain of dependent instructions per span, so its
-// throughput grows with the number of warps: G = 4 (16 epilogue warps, at most 112 registers) is
-// used when segments are long and the light few-boundaries path does the work, G = 2 (8 warps,
-// 168 registers, the MMA warp one tile ahead) when boundaries are dense.
+// throughput grows with the number of warps: G = 3 (12 epilogue warps, 128 registers, one TMEM
+// buffer per group) is used when segments are long and the light few-boundaries path does the
+// work, G = 2 (8 warps, 168 registers, the MMA warp one tile ahead) when boundaries are dense.
+// (G = 4 compiles too but measured no better than 3: 96 registers make the general path spill.)
 constexpr int SUM_BUFS = 4;                                        // TMEM tile buffers, shared out among the warpgroups
 constexpr int SUM_TMEM_COLS = SUM_BUFS * PIECES_PER_SPAN * ROW;    // 512
 template <int G>
 struct SumShape {
-    static_assert(G == 2 || G == 4, "two or four epilogue warpgroups");
+    static_assert(G == 2 || G == 3 || G == 4, "two to four epilogue warpgroups");
     static constexpr int kEpiWarps = 4 * G;
     static constexpr int kProducerWarp = 4 * G;
     static constexpr int kMmaWarp = 4 * G + 1;
     static constexpr int kThreads = (4 * G + 2) * 32;
-    static constexpr int kBufsPerGroup = SUM_BUFS / G;
+    static constexpr int kBufsPerGroup = G == 2 ? 2 : 1;
 };
 constexpr int SUM_SPARSE_MAX = 8;                                  // spans with at most this many boundaries read single prefixes from TMEM
 constexpr int SUM_DIRECT_LEN = 4;                                  // segments this short are summed from the inputs
