@@ -214,7 +214,8 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
         const int threads = 256;
         const long long blocks = (warps * 32 + threads - 1) / threads;
         partition_offsets_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, shift, spans, span_q, n_eff,
-                                                                                 reinterpret_cast<WorkspaceHeader*>(ws), nseg_dev);
+                                                                                 reinterpret_cast<WorkspaceHeader*>(ws), nseg_dev,
+                                                                                 static_cast<uint32_t*>(out));
         ++g_launches;
     }
     CUtensorMap tmap;

@@ -197,28 +197,11 @@ struct SumParams {
                                  // differs from *shape_sel returns at once (the choice depends on nseg)
 };
 
-// span_q[s] = first index q in [0, nseg] with (off[q] << shift) >= s * SPAN, nseg + 1 if none.
-// One warp per span edge, 32-ary search.  The same launch validates the offsets (non-decreasing,
-// inside [0, n]) and records MMV_ERR_BAD_SEGMENTS otherwise; the main kernel never indexes
-// outside its tile whatever they hold.
-__global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, int shift, long long num_spans,
-                                         int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr,
-                                         const long long* __restrict__ nseg_dev) {
-    if (nseg_dev) nseg = *nseg_dev;
-    {
-        const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-        bool bad = false;
-        for (long long q = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q < nseg; q += stride) {
-            const long long a = static_cast<long long>(off[q]) << shift, b = static_cast<long long>(off[q + 1]) << shift;
-            bad |= (a > b) || (a < 0) || (b > n);
-        }
-        if (bad) report_error(hdr, 4u);
-    }
-    const long long warp = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+// First index q in [lo, hi) with (off[q] << shift) >= target, hi if none; the offsets are
+// non-decreasing.  One warp, 32-ary search (every lane probes the last element of its block).
+__device__ __forceinline__ long long first_index_at_least(const int32_t* __restrict__ off, int shift, long long lo, long long hi,
+                                                          long long target) {
     const int lane = threadIdx.x & 31;
-    if (warp > num_spans) return;
-    const long long target = warp * SPAN;
-    long long lo = 0, hi = nseg + 1;
     while (hi > lo) {
         const long long len = hi - lo;
         const long long step = (len + 31) / 32;
@@ -239,7 +222,37 @@ __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long l
             hi = ke - 1;
         }
     }
-    if (lane == 0) span_q[warp] = static_cast<int32_t>(lo);
+    return lo;
+}
+// The same out of line, for the rare jump over a long run of equal offsets in the epilogue.
+__device__ __noinline__ long long first_index_at_least_call(const int32_t* off, int shift, long long lo, long long hi,
+                                                            long long target) {
+    return first_index_at_least(off, shift, lo, hi, target);
+}
+
+// span_q[s] = first index q in [0, nseg] with (off[q] << shift) >= s * SPAN, nseg + 1 if none.
+// One warp per span edge.  The same launch validates the offsets (non-decreasing, inside [0, n]; it
+// records MMV_ERR_BAD_SEGMENTS otherwise, and the main kernel never indexes outside its tile
+// whatever they hold) and writes the zero of every EMPTY segment, so that the main kernel may jump
+// over long runs of equal offsets instead of visiting them one by one.
+__global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, int shift, long long num_spans,
+                                         int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr,
+                                         const long long* __restrict__ nseg_dev, uint32_t* __restrict__ out) {
+    if (nseg_dev) nseg = *nseg_dev;
+    {
+        const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+        bool bad = false;
+        for (long long q = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q < nseg; q += stride) {
+            const long long a = static_cast<long long>(off[q]) << shift, b = static_cast<long long>(off[q + 1]) << shift;
+            bad |= (a > b) || (a < 0) || (b > n);
+            if (a == b) out[q] = 0u;
+        }
+        if (bad) report_error(hdr, 4u);
+    }
+    const long long warp = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
+    if (warp > num_spans) return;
+    const long long lo = first_index_at_least(off, shift, 0, nseg + 1, warp * SPAN);
+    if ((threadIdx.x & 31) == 0) span_q[warp] = static_cast<int32_t>(lo);
 }
 
 template <typename P, int G>
@@ -775,7 +788,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 bool piece_has_start = false;
                 long long last_start = -1;
                 long long qp = q;              // batch pointer
-                int advance = 0;               // boundaries strictly before pend: consumed for good
+                long long advance = 0;         // boundaries strictly before pend: consumed for good
                 while (true) {
                     const long long qi = qp + lane;
                     long long b = -1, sb = -1;
@@ -841,6 +854,14 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     advance += __popc(__ballot_sync(0xffffffffu, mine && (b < pend)));
                     qp += cnt;
                     if (cnt < 32) break;
+                    // A whole batch at one position is a run of empty segments.  Their zeros were written
+                    // when the offsets were partitioned: jump to the first boundary behind the run.
+                    const long long b0 = __shfl_sync(0xffffffffu, b, 0);
+                    if (b0 == __shfl_sync(0xffffffffu, b, 31)) {
+                        const long long u = first_index_at_least_call(prm.off, sh, qp, nq, b0 + 1);
+                        if (b0 < pend) advance += u - qp;
+                        qp = u;
+                    }
                 }
                 q += advance;
                 if (piece_has_start) {

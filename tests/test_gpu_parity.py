@@ -261,6 +261,31 @@ def test_seg_sum_csr_edges(mmv):
     assert sum_csr(mmv, np.zeros(0, np.int8), off).tolist() == [0] * 8
 
 
+def test_seg_sum_long_runs_of_empty_segments(mmv):
+    # hundreds of thousands of empty segments in a row (at the start, in the middle of a span, exactly on a
+    # span edge, at the end): the kernel jumps over such runs instead of visiting them one by one
+    rng = np.random.default_rng(99)
+    n = 6 * TILE + 1000
+    cuts = np.sort(rng.choice(np.arange(1, n), 40, replace=False))
+    pieces = [np.zeros(300000, np.int64)]                                   # leading run at 0
+    for c in cuts:
+        pieces.append(np.asarray([c], np.int64))
+    pieces.append(np.full(250000, 2 * TILE + 777, np.int64))                # inside a span
+    pieces.append(np.full(250000, 3 * TILE, np.int64))                      # on a tile edge
+    pieces.append(np.full(400000, n, np.int64))                             # trailing run at n
+    off = np.sort(np.concatenate(pieces + [np.asarray([0, n], np.int64)])).astype(np.int32)
+    x = rng.integers(-128, 128, n).astype(np.int8)
+    want = oracle.seg_sum_csr_i8(x, off)
+    import time
+    t0 = time.time()
+    got = sum_csr(mmv, x, off)
+    assert np.array_equal(got, want)
+    xf = rng.standard_normal(n).astype(np.float16)
+    wantf, a = oracle.seg_sum_csr_f16(xf, off)
+    assert_fp(sum_csr(mmv, xf, off), wantf, a, "runs of empty segments")
+    assert time.time() - t0 < 5.0
+
+
 @pytest.mark.parametrize("maxlen", [3, 60, 3000])
 def test_seg_sum_csr_many_tiles_per_cta(mmv, maxlen):
     # more tiles than 2 x 148, so every CTA runs several tiles back to back in both warpgroups
