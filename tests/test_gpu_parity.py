@@ -286,6 +286,44 @@ def test_seg_sum_long_runs_of_empty_segments(mmv):
     assert time.time() - t0 < 5.0
 
 
+@pytest.mark.parametrize("seed", [1, 2, 3, 4])
+def test_seg_sum_mixed_runs_and_lengths_stress(mmv, seed):
+    # random mixtures of segment lengths (tiny, medium, long) and of runs of empty segments whose lengths sit
+    # around the batch and table sizes of the kernel (31..33, 63..65, 127..130, a few thousand), some of
+    # them pinned to row, piece, span and tile edges
+    rng = np.random.default_rng(seed)
+    n = 5 * TILE + int(rng.integers(0, 5000))
+    cuts = set(int(c) for c in rng.choice(np.arange(1, n), 300, replace=False))
+    cuts |= {32, 1024, 4096, TILE, 2 * TILE + 4096, 3 * TILE - 32, 4 * TILE + 1024, n - 1}
+    # a stretch of tiny segments
+    a = int(rng.integers(TILE, 2 * TILE))
+    cuts |= set(range(a, a + 700, int(rng.integers(1, 4))))
+    pos = np.asarray(sorted(c for c in cuts if 0 < c < n), np.int64)
+    reps = np.ones(pos.shape[0], np.int64)
+    run_lengths = [31, 32, 33, 63, 64, 65, 127, 128, 129, 130, 257, 3000, 5000]
+    where = rng.choice(pos.shape[0], len(run_lengths), replace=False)
+    for w, r in zip(where, run_lengths):
+        reps[w] = r
+    edge_idx = [int(np.searchsorted(pos, e)) for e in (4096, TILE, 3 * TILE - 32)]
+    for i, r in zip(edge_idx, (40, 129, 1000)):
+        reps[i] = r
+    body = np.repeat(pos, reps)
+    lead = int(rng.integers(0, 200))
+    trail = int(rng.integers(0, 200))
+    off = np.concatenate([np.zeros(1 + lead, np.int64), body, np.full(1 + trail, n, np.int64)]).astype(np.int32)
+    x = rng.integers(-128, 128, n).astype(np.int8)
+    assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
+    xf = rng.standard_normal(n).astype(np.float16)
+    want, a_ = oracle.seg_sum_csr_f16(xf, off)
+    assert_fp(sum_csr(mmv, xf, off), want, a_, f"stress seed {seed}")
+    for groups in (2, 3):
+        mmv.debug_force_sum_groups(groups)
+        try:
+            assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
+        finally:
+            mmv.debug_force_sum_groups(0)
+
+
 @pytest.mark.parametrize("maxlen", [3, 60, 3000])
 def test_seg_sum_csr_many_tiles_per_cta(mmv, maxlen):
     # more tiles than 2 x 148, so every CTA runs several tiles back to back in both warpgroups
