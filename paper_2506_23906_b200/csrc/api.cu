@@ -101,9 +101,12 @@ bool encode_span_map(CUtensorMap* map, const void* x, long long n, int elem_byte
     cuuint64_t strides[3] = {rb, rb * PIECE_ROWS, rb * PIECE_ROWS * pieces_per_unit};
     cuuint32_t box[4] = {ROW, PIECE_ROWS, 1, SPANS_PER_TILE};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = enc(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 4,
-                     const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     elem_bytes == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B,
+    const CUtensorMapDataType dtp = elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_UINT32
+                                  : elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_UINT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8;
+    const CUtensorMapSwizzle swz = elem_bytes == 4 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                 : elem_bytes == 2 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
+    CUresult r = enc(map, dtp, 4,
+                     const_cast<void*>(x), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
@@ -143,7 +146,7 @@ long long num_scan_tiles_of(long long n) { return (n + SCAN_TILE - 1) / SCAN_TIL
 
 WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     WorkspacePlan p{};
-    p.n_eff = (op == MMV_OP_SPMV_CSR) ? 2 * n : n;
+    p.n_eff = n;
     const long long tiles = num_tiles_of(p.n_eff);
     const long long units = (op == MMV_OP_SEG_SCAN) ? num_scan_tiles_of(n) * SPANS_PER_TILE : tiles * SPANS_PER_TILE;
     p.status_off = sizeof(WorkspaceHeader);
@@ -164,8 +167,9 @@ WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     return p;
 }
 
-// z(k) = val(k) * x(col(k)) in fp32 (Algorithm A.5, CsrGather), written as two bf16 halves
-// (hi = bf16(z), lo = bf16(z - hi)) so that the segmented sum can feed them to the tensor core.
+// z(k) = val(k) * x(col(k)) in fp32 (Algorithm A.5, CsrGather), written as a pair of bf16 values
+// (hi = bf16(z), lo = bf16(z - hi); 4 bytes per product) that the segmented sum feeds to the tensor
+// core as two K entries of one element.
 __global__ void spmv_gather_kernel(const int32_t* __restrict__ col, const __half* __restrict__ val,
                                    const float* __restrict__ x, uint32_t* __restrict__ prod, long long nnz) {
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
@@ -578,7 +582,7 @@ mmv_status mmv_spmv_csr(const int32_t* rowptr, const int32_t* col, const void* v
                         int64_t rows, int64_t cols, int64_t nnz, void* workspace, size_t workspace_bytes,
                         void* cuda_stream) {
     if (rows < 0 || cols < 0 || nnz < 0) return MMV_ERR_INVALID_ARG;
-    if (nnz >= (1ll << 30)) return MMV_ERR_INVALID_ARG;          // 2 * nnz must fit int32 offsets
+    if (nnz >= (1ll << 31)) return MMV_ERR_INVALID_ARG;          // int32 offsets cannot address more
     if (rows == 0) return MMV_OK;
     if (!rowptr || !y) return MMV_ERR_INVALID_ARG;
     if (!aligned16(rowptr) || !aligned16(y)) return MMV_ERR_INVALID_ARG;
@@ -606,7 +610,7 @@ mmv_status mmv_spmv_csr(const int32_t* rowptr, const int32_t* col, const void* v
                                                                               prod, nnz);
         ++g_launches;
     }
-    return launch_seg_sum<BF16Path>(prod, 2 * nnz, rowptr, rows, 1, y, ws, plan, dev, st);
+    return launch_seg_sum<BF16Path>(prod, nnz, rowptr, rows, 0, y, ws, plan, dev, st);
 }
 
 mmv_status mmv_last_async_status(const void* workspace, void* cuda_stream) {

@@ -12,10 +12,12 @@
 //                  of piece i of span w, the speculative block scan z = MATMUL(x, U_s) of
 //                  Algorithm A.1 (BlockSegScan); columns 32..63 (fp16) return the row itself
 //                  converted exactly to fp32.
-//   epilogue warps (lane = row; two warpgroups on alternating tiles)
+//   epilogue warps (lane = row; two warpgroups for fp16, three for int8, taking tiles in turn)
 //     pre-pass     flag bytes -> one 32-bit start mask per row; row totals (TMEM column 31);
-//                  from these the span's aggregate (sum of its open tail segment, any flag)
-//                  is formed with a handful of shuffles and published at once.
+//                  from these each span's aggregate (sum of its open tail segment, any flag) is
+//                  formed with a handful of shuffles; the four spans of a tile exchange theirs
+//                  through shared memory and the tile's first warp publishes ONE status word
+//                  for the tile.
 //     main pass    per piece: revert the speculation inside each row (Lemma A.1: subtract the
 //                  prefix just before the element's segment start; the first element of a
 //                  segment takes the input value itself), segmented scan of the 32 row tails
@@ -24,8 +26,9 @@
 //                  store.  Pieces without any flag skip the revert.  Pieces that reach back
 //                  to the start of the span (up to and including the first flagged one) are
 //                  parked in TMEM instead.
-//     look-back    decoupled look-back over the earlier spans' status words returns the carry
-//                  (this replaces the recursion of Section 4.2 / Algorithm A.1's Recurse); its
+//     look-back    the tile's first warp runs the decoupled look-back over the earlier tiles'
+//                  status words (this replaces the recursion of Section 4.2 / Algorithm A.1's
+//                  Recurse) and hands the carry to its siblings through shared memory; its
 //                  latency is covered by the main pass.  The parked pieces then receive the
 //                  carry on the elements before the span's first flag and are stored.
 #pragma once

@@ -9,17 +9,24 @@
 //   4-D TMA box, K-major, hardware swizzle) with the constant upper-triangular
 //   all-ones U_32 (B operand): TMEM lane 32w+l, column j = inclusive prefix at
 //   position j of row l of piece i of span w  --  z = MATMUL(x, U_s).
-//   The MMA warp runs one tile ahead (two TMEM buffers per warpgroup).
-//   Epilogue warps (lane = row) read the row totals (TMEM column 31) and only touch
-//   the segment boundaries, which they hold in registers (one offset per lane):
-//   a piece that contains a boundary has its 32 x 32 prefixes copied to shared
-//   memory and its row totals scanned with shuffles; every segment end inside it
-//   emits  prefix(end) - prefix(start-1)  (the DIFF of Algorithm 4.2 applied to the
-//   COMPRESSed speculative scan, but with prefixes local to the row or the piece so
-//   that magnitudes stay small); very short segments are summed directly from the
-//   input values; segments that cross pieces take the running sum of the open
-//   segment, and segments that cross spans take the carry of a decoupled look-back
-//   over per-span status words.  Pieces without a boundary only add their total.
+//   With two epilogue warpgroups the MMA warp runs one tile ahead (two TMEM buffers per group);
+//   the shape with three groups has one buffer per group.
+//   Epilogue warps (lane = row).  partition_offsets_kernel has stored, per span, the index of its
+//   first offset; a warp requests that index and the span's first 128 offsets one tile ahead.
+//     pre-pass     row totals (TMEM column 31) and the one prefix in front of the span's last
+//                  segment start give the span's aggregate, published at once.
+//     few boundaries (<= 8): each boundary's prefix is read straight from TMEM (one column, it
+//                  sits in the lane of its row), the 128 row totals are scanned with four
+//                  interleaved warp scans, and lane j emits the segment that ends at boundary j.
+//     general path the offsets go to a per-warp table in shared memory; a piece that contains a
+//                  boundary has its 32 x 32 prefixes copied to shared memory and its boundaries
+//                  walked 32 at a time; every segment end emits  prefix(end) - prefix(start-1)
+//                  (the DIFF of Algorithm 4.2 applied to the COMPRESSed speculative scan, but with
+//                  prefixes local to the row or the piece so that magnitudes stay small).
+//     Segments of at most four elements are summed from the input values themselves; segments
+//     that cross pieces take the running sum of the open segment; the one segment per span that
+//     began before it takes the carry of the sibling spans (shared memory) or of a decoupled
+//     look-back over per-span status words.  Pieces without a boundary only add their total.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -50,11 +57,31 @@ constexpr int SUM_DIRECT_LEN = 4;                                  // segments t
 constexpr int SUM_TBL = 128;                                       // boundaries of a span kept in shared memory
 constexpr int SUM_TBL_BYTES = (SUM_TBL + 4) * 4 + SUM_TBL * 4;     // offsets (one predecessor in front) + direct sums
 
-// bf16 values (the hi/lo halves of the fp32 products of SpMV): same geometry as fp16.
-struct BF16Path : F16Path {
-    static constexpr uint32_t kOneBits = 0x3F80u;                       // 1.0 in bf16
+// The fp32 products of SpMV, each stored as a pair of bf16 values (hi = bf16(z), lo = bf16(z - hi),
+// 4 bytes).  An ELEMENT of this path is one product; a row of 32 products is a 128-byte operand
+// row of 64 bf16 values (K = 64), and the constant operand adds both halves of every product into
+// the prefix:  B[k][j] = 1 iff floor(k / 2) <= j.  So the epilogue sees nnz elements, not 2 nnz.
+struct BF16Path {
+    using Acc = float;
+    static constexpr int kElemBytes = 4;
+    static constexpr bool kIsFloat = true;
+    static constexpr int kRowBytes = ROW * 4;              // 128-byte rows -> 128-byte swizzle
+    static constexpr int kSlabBytes = OPERAND_ROWS * kRowBytes;    // 16 KB
+    static constexpr int kMmaPerSlab = 4;                  // K = 16 bf16 values per instruction
+    static constexpr int kKStepBytes = 32;
+    static constexpr uint32_t kLayoutType = 2;             // SWIZZLE_128B
+    static constexpr uint32_t kSbo = 8 * kRowBytes;        // 1024
+    static constexpr uint32_t kOneBits = 0x3F80u;          // 1.0 in bf16
     static constexpr uint32_t kFmtBits = (1u << 7) | (1u << 10);        // A and B are bf16
+    __device__ static __forceinline__ Acc from_bits(uint32_t b) { return __uint_as_float(b); }
+    __device__ static __forceinline__ uint32_t to_bits(Acc v) { return __float_as_uint(v); }
+    __device__ static __forceinline__ Acc add(Acc a, Acc b) { return a + b; }
+    __device__ static __forceinline__ Acc sub(Acc a, Acc b) { return a - b; }
 };
+// one product = hi + lo, added in the order the tensor core sees them
+__device__ __forceinline__ float pair_value(uint32_t bits) {
+    return __uint_as_float(bits << 16) + __uint_as_float(bits & 0xffff0000u);
+}
 
 template <typename P>
 __device__ __forceinline__ typename P::Acc load_value(const void* base, long long idx);
@@ -64,7 +91,7 @@ __device__ __forceinline__ float load_value<F16Path>(const void* base, long long
 }
 template <>
 __device__ __forceinline__ float load_value<BF16Path>(const void* base, long long idx) {
-    return __bfloat162float(static_cast<const __nv_bfloat16*>(base)[idx]);
+    return pair_value(static_cast<const uint32_t*>(base)[idx]);
 }
 template <>
 __device__ __forceinline__ uint32_t load_value<I8Path>(const void* base, long long idx) {
@@ -80,7 +107,7 @@ __device__ __forceinline__ float elem_bits_to_acc<F16Path>(uint32_t bits) {
 }
 template <>
 __device__ __forceinline__ float elem_bits_to_acc<BF16Path>(uint32_t bits) {
-    return __uint_as_float(bits << 16);
+    return pair_value(bits);
 }
 template <>
 __device__ __forceinline__ uint32_t elem_bits_to_acc<I8Path>(uint32_t bits) {
@@ -107,6 +134,13 @@ struct ValueWindow {
 template <typename P>
 __device__ __forceinline__ void window_load(const void* xg, long long sb, int len, long long n, ValueWindow& win) {
     constexpr int EB = P::kElemBytes;                   // 2 or 1: a word of four elements is 8 or 4 bytes
+    if constexpr (EB == 4) {
+        // 4-byte elements: one load per element, nothing to align
+        win.wide = true;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) win.r[i] = (i < len && sb + i < n) ? static_cast<const uint32_t*>(xg)[sb + i] : 0u;
+        return;
+    }
     const long long base = sb & ~3ll;
     const int sh = static_cast<int>(sb & 3);
     win.r[0] = win.r[1] = win.r[2] = win.r[3] = 0u;
@@ -134,6 +168,12 @@ __device__ __forceinline__ typename P::Acc window_sum(const void* xg, long long 
     constexpr int EB = P::kElemBytes;
     const int sh = static_cast<int>(sb & 3);
     Acc val = Acc(0);
+    if constexpr (EB == 4) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (i < len) val = P::add(val, elem_bits_to_acc<P>(win.r[i]));
+        return val;
+    }
     if constexpr (EB == 2) {
         const int bits = sh * 16;
         const uint32_t a0 = bits >= 32 ? win.r[1] : win.r[0];
@@ -167,17 +207,18 @@ __device__ __forceinline__ bool sum_lookback(const uint64_t* status, long long s
 
 template <typename P, int G>
 struct SumCfg {
-    static constexpr int kStages = 4;
-    static constexpr int kBBytes = ROW * P::kRowBytes;               // constant U_32: 32 rows
+    static constexpr int kStages = P::kElemBytes == 4 ? 2 : 4;      // (the bf16-pair tiles are 64 KB)
+    static constexpr int kBBytes = ROW * P::kRowBytes;               // constant operand: 32 rows
     static constexpr int kXBytes = PIECES_PER_SPAN * P::kSlabBytes;  // four [128 x 32] operands
     static constexpr int kDumpBytes = PIECE * 4;                     // per epilogue warp
-    static constexpr int kStageOffset = 2048;                        // after the constant operand
+    static constexpr int kStageOffset = 4096;                        // after the constant operand
     static constexpr int kDumpOffset = kStageOffset + kStages * kXBytes;
     static constexpr int kRowpreOffset = kDumpOffset + SumShape<G>::kEpiWarps * kDumpBytes;
     static constexpr int kTblOffset = kRowpreOffset + SumShape<G>::kEpiWarps * PIECE_ROWS * 4;
     static constexpr int kBarOffset = kTblOffset + SumShape<G>::kEpiWarps * SUM_TBL_BYTES;
     static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
-    static_assert(kBBytes <= 2048, "constant operand fits its slot");
+    static_assert(kBBytes <= kStageOffset, "constant operand fits its slot");
+    static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of one CTA");
 };
 
 struct SumParams {
@@ -307,6 +348,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
     if (warp == Shape::kProducerWarp && lane == 0) tma_prefetch_desc(&tmap_x);
     {
         // constant B = U_32 stored K-major: row nn (output position), element k (input position): 1 iff k <= nn
+        // (bf16 pairs: element k is the two K entries 2k and 2k + 1, both set)
         constexpr int kVecPerRow = P::kRowBytes / 16;
         constexpr int kElemPerVec = 16 / P::kElemBytes;
         for (int v = threadIdx.x; v < ROW * kVecPerRow; v += Shape::kThreads) {
@@ -316,7 +358,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             for (int e = 0; e < kElemPerVec; ++e) {
                 const int k = cv * kElemPerVec + e;
                 if (k <= nn) {
-                    if constexpr (P::kElemBytes == 2) words[e >> 1] |= static_cast<uint32_t>(P::kOneBits) << ((e & 1) * 16);
+                    if constexpr (P::kElemBytes == 4) words[e] = P::kOneBits | (P::kOneBits << 16);   // both halves of product k
+                    else if constexpr (P::kElemBytes == 2) words[e >> 1] |= static_cast<uint32_t>(P::kOneBits) << ((e & 1) * 16);
                     else words[e >> 2] |= 1u << ((e & 3) * 8);
                 }
             }
