@@ -593,6 +593,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             win0.wide = false;
             if (isdir[0]) window_load<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), prm.n, win0);
             bool tcovers = covers;
+            ValueWindow wn[3];                 // direct sums of table entries 32..127 (general path only)
+            wn[0].wide = wn[1].wide = wn[2].wide = false;
             if (!sparse) {
                 // the general path keeps up to 128 boundaries in a shared-memory table
                 bool tc = false;
@@ -609,6 +611,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     tc |= (cq + lane + 32 * j >= nq) || (bj[j] > send);
                     isdir[j] = cq + lane + 32 * j < nq && sbj[j] >= 0 && bj[j] > sbj[j] && bj[j] - sbj[j] <= SUM_DIRECT_LEN &&
                                bj[j] > sbase && bj[j] <= send && bj[j] <= prm.n;
+                    // (the loads go out here, with those of entry 0; they are summed after the pre-pass)
+                    if (isdir[j]) window_load<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), prm.n, wn[j - 1]);
                 }
                 tcovers = __any_sync(0xffffffffu, tc) || covers;
             }
@@ -769,16 +773,9 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     tail = P::add(__shfl_sync(0xffffffffu, P::sub(totl, before), rl), after);
                 }
                 publish(tail);
-                // direct sums: the first 32 boundaries' values have arrived by now; the others (spans with
-                // more than 32 boundaries) are fetched here, all at once
+                // direct sums: the values were requested before the accumulators were awaited
                 dvt[lane] = isdir[0] ? window_sum<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), win0) : Acc(0);
                 if (!covers) {
-                    ValueWindow wn[3];
-#pragma unroll
-                    for (int j = 1; j < 4; ++j) {
-                        wn[j - 1].wide = false;
-                        if (isdir[j]) window_load<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), prm.n, wn[j - 1]);
-                    }
 #pragma unroll
                     for (int j = 1; j < 4; ++j)
                         dvt[lane + 32 * j] = isdir[j] ? window_sum<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), wn[j - 1]) : Acc(0);
