@@ -118,8 +118,10 @@ mmv_status mmv_seg_sum(const void *x, const void *seg, mmv_segfmt sf, int64_t n,
  * (Algorithm 4.4; Algorithms A.4-A.6):  y[r] = sum over k in
  * [rowptr[r], rowptr[r+1]) of val[k] * x[col[k]], fp32 products and sums, an
  * empty row gives exactly 0.  rowptr: rows+1 int32 with rowptr[0] == 0 and
- * rowptr[rows] == nnz; col: nnz int32 in [0, cols) (not checked; duplicates
- * simply add); val: nnz fp16; x: cols fp32; y: rows fp32.
+ * rowptr[rows] == nnz < 2^31; col: nnz int32 in [0, cols) (duplicates simply
+ * add; an index outside the range is never dereferenced, it contributes 0 and the
+ * call records MMV_ERR_INVALID_ARG in the workspace status); val: nnz fp16;
+ * x: cols fp32; y: rows fp32.
  */
 mmv_status mmv_spmv_csr(const int32_t *rowptr, const int32_t *col, const void *val_f16,
                         const float *x, float *y, int64_t rows, int64_t cols, int64_t nnz,

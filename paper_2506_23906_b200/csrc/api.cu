@@ -170,37 +170,39 @@ WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
 // z(k) = val(k) * x(col(k)) in fp32 (Algorithm A.5, CsrGather), written as a pair of bf16 values
 // (hi = bf16(z), lo = bf16(z - hi); 4 bytes per product) that the segmented sum feeds to the tensor
 // core as two K entries of one element.
+// A column index outside [0, cols) is never dereferenced: it reads as x = 0 and the call ends with
+// MMV_ERR_INVALID_ARG in the workspace status (the check costs nothing, the kernel waits on its loads).
+__device__ __forceinline__ float gather_x(const float* __restrict__ x, int c, long long cols, bool& bad) {
+    const bool oob = static_cast<unsigned long long>(static_cast<long long>(c)) >= static_cast<unsigned long long>(cols);
+    bad |= oob;
+    return oob ? 0.f : __ldg(x + c);
+}
+__device__ __forceinline__ uint32_t split_product(float z) {
+    const __nv_bfloat16 hi = __float2bfloat16_rn(z);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(z - __bfloat162float(hi));
+    return static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(lo)) << 16);
+}
 __global__ void spmv_gather_kernel(const int32_t* __restrict__ col, const __half* __restrict__ val,
-                                   const float* __restrict__ x, uint32_t* __restrict__ prod, long long nnz) {
+                                   const float* __restrict__ x, uint32_t* __restrict__ prod, long long nnz,
+                                   long long cols, WorkspaceHeader* hdr) {
     const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
     const long long nvec = nnz >> 2;
+    bool bad = false;
     for (long long v = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; v < nvec; v += stride) {
         const int4 c = __ldg(reinterpret_cast<const int4*>(col) + v);
         const uint2 hv = __ldg(reinterpret_cast<const uint2*>(val) + v);
         const __half2 h01 = *reinterpret_cast<const __half2*>(&hv.x);
         const __half2 h23 = *reinterpret_cast<const __half2*>(&hv.y);
-        float z[4];
-        z[0] = __low2float(h01) * __ldg(x + c.x);
-        z[1] = __high2float(h01) * __ldg(x + c.y);
-        z[2] = __low2float(h23) * __ldg(x + c.z);
-        z[3] = __high2float(h23) * __ldg(x + c.w);
-        uint32_t o[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const __nv_bfloat16 hi = __float2bfloat16_rn(z[e]);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(z[e] - __bfloat162float(hi));
-            o[e] = static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(lo)) << 16);
-        }
-        *(reinterpret_cast<uint4*>(prod) + v) = make_uint4(o[0], o[1], o[2], o[3]);
+        const float x0 = gather_x(x, c.x, cols, bad), x1 = gather_x(x, c.y, cols, bad);
+        const float x2 = gather_x(x, c.z, cols, bad), x3 = gather_x(x, c.w, cols, bad);
+        *(reinterpret_cast<uint4*>(prod) + v) =
+            make_uint4(split_product(__low2float(h01) * x0), split_product(__high2float(h01) * x1),
+                       split_product(__low2float(h23) * x2), split_product(__high2float(h23) * x3));
     }
     // ragged tail (nnz not a multiple of 4)
     const long long k = (nvec << 2) + static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (k < nnz) {
-        const float z = __half2float(val[k]) * __ldg(x + col[k]);
-        const __nv_bfloat16 hi = __float2bfloat16_rn(z);
-        const __nv_bfloat16 lo = __float2bfloat16_rn(z - __bfloat162float(hi));
-        prod[k] = static_cast<uint32_t>(__bfloat16_as_ushort(hi)) | (static_cast<uint32_t>(__bfloat16_as_ushort(lo)) << 16);
-    }
+    if (k < nnz) prod[k] = split_product(__half2float(val[k]) * gather_x(x, col[k], cols, bad));
+    if (bad) report_error(hdr, 1u);
 }
 
 // Shared launcher of the tiled segmented-sum kernel.  `values` holds n_eff elements of the
@@ -607,7 +609,7 @@ mmv_status mmv_spmv_csr(const int32_t* rowptr, const int32_t* col, const void* v
         if (blocks > cap) blocks = cap;
         if (blocks < 1) blocks = 1;
         spmv_gather_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(col, static_cast<const __half*>(val_f16), x,
-                                                                              prod, nnz);
+                                                                              prod, nnz, cols, reinterpret_cast<WorkspaceHeader*>(ws));
         ++g_launches;
     }
     return launch_seg_sum<BF16Path>(prod, nnz, rowptr, rows, 0, y, ws, plan, dev, st);

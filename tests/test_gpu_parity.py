@@ -433,6 +433,21 @@ def test_spmv_golden_and_random(mmv):
 # ---------------------------------------------------------------------------
 # robustness
 # ---------------------------------------------------------------------------
+def test_bad_column_indices_are_reported_not_dereferenced(mmv):
+    rowptr, col, val, xv = gen.config4(rows=4096)
+    col = col.copy()
+    col[[5, col.shape[0] // 2, col.shape[0] - 1]] = [-7, xv.shape[0], 2 ** 31 - 1]
+    ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, val.shape[0], 4096)
+    mmv.spmv_csr(dev(rowptr), dev(col), dev(val), dev(xv), workspace=ws)
+    assert mmv.last_async_status(ws) == 1          # MMV_ERR_INVALID_ARG, and the context is still usable
+    ok = col.copy()
+    ok[[5, col.shape[0] // 2, col.shape[0] - 1]] = 0
+    y = mmv.spmv_csr(dev(rowptr), dev(ok), dev(val), dev(xv), workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    want, a = oracle.spmv_csr(rowptr, ok, val, xv)
+    assert_fp(y.cpu().numpy(), want, a, "SpMV after a rejected call")
+
+
 def test_bad_offsets_are_reported_not_trapped(mmv):
     n = 50000
     x = dev(np.ones(n, np.int8))
