@@ -160,7 +160,7 @@ WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     const bool flagsum = op == MMV_OP_SEG_SUM && sf == MMV_SEG_FLAGS_U8;
     const long long nchunks = (n + CMP_CHUNK - 1) / CMP_CHUNK;
     p.cmp_off = p.prod_off + p.prod_bytes;
-    p.cmp_bytes = flagsum ? round_up(static_cast<size_t>(2 * nchunks) * sizeof(int32_t) + 16, 256) : 0;
+    p.cmp_bytes = flagsum ? round_up(static_cast<size_t>(2 * nchunks + 8) * sizeof(int32_t) + 16, 256) : 0;
     p.off_off = p.cmp_off + p.cmp_bytes;
     p.off_bytes = flagsum ? round_up(static_cast<size_t>(n + 1) * sizeof(int32_t), 256) : 0;
     p.total = p.off_off + p.off_bytes;
@@ -543,7 +543,7 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
         const long long nchunks = (n + CMP_CHUNK - 1) / CMP_CHUNK;
         long long* nseg_dev = reinterpret_cast<long long*>(ws + plan.cmp_off);
         int32_t* chunk_count = reinterpret_cast<int32_t*>(ws + plan.cmp_off + 16);
-        int32_t* chunk_base = chunk_count + nchunks;
+        int32_t* chunk_base = chunk_count + ((nchunks + 3) & ~3ll);      // 16-byte aligned: it is written as vectors
         int32_t* off = reinterpret_cast<int32_t*>(ws + plan.off_off);
         const uint8_t* f = static_cast<const uint8_t*>(seg);
         const long long cap = static_cast<long long>(dev->sm_count) * 8;
