@@ -7,8 +7,8 @@ One step = one pass of the segmented-scan hot path (tile load, tensor-core block
 prefix, flag pass, revert, carries, look-back, store) over the headline workload:
 the density-sweep configuration (n = 2^30 fp16 values uniform in [-1,1), fp32
 output) with Bernoulli(1e-3) start flags.  The line printed at the end also
-carries, under "configs", short measurements of all five configurations of
-the benchmark spec (N = 1 only).  Inputs are seeded and synthetic (mmv_inputs); they
+carries, under "configs", short measurements of all five benchmark
+configurations (N = 1 only).  Inputs are seeded and synthetic (mmv_inputs); they
 are generated on the host and uploaded before the timed region.  Every working
 set here is larger than the 126 MB L2 except configuration 1, for which a
 buffer larger than L2 is rewritten between timed launches.
