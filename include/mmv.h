@@ -20,6 +20,10 @@
  *     not be shared by calls that may overlap on the GPU.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL =
  *     the default stream); the call does not synchronise with the host.
+ *     mmv_seg_scan, mmv_seg_sum and mmv_spmv_csr enqueue nothing but a memset
+ *     and kernels, so they can be captured in a CUDA graph and replayed,
+ *     provided one call was made on the device before the capture (the first
+ *     call sets the kernels' attributes).
  *   - x, seg and out must be 16-byte aligned and must not overlap each other.
  *   - Argument errors are reported synchronously and nothing is enqueued.
  *     Conditions only the device can detect (a wait that ran out of its time

@@ -477,3 +477,46 @@ def test_lookback_wait_gives_up_with_a_status(mmv):
     out = mmv.seg_scan(x, f, workspace=ws)            # and the next call works
     assert mmv.last_async_status(ws) == 0
     assert np.array_equal(out.cpu().numpy(), np.arange(1, n + 1))
+
+
+# ---------------------------------------------------------------------------
+# the calls only enqueue a memset and kernels on the given stream: they can be captured in a CUDA
+# graph and replayed (the first call on a device, which sets the kernels' attributes, comes before)
+# ---------------------------------------------------------------------------
+def test_calls_replay_from_a_cuda_graph(mmv):
+    rng = np.random.default_rng(5)
+    n = 3 * TILE + 4001
+    x = rng.integers(-128, 128, n).astype(np.int8)
+    f = (rng.random(n) < 0.01).astype(np.uint8)
+    off = gen.offsets_from_lengths(rng.integers(0, 700, 400))
+    xs = rng.integers(-128, 128, int(off[-1])).astype(np.int8)
+    rowptr, col, val, xv = gen.config4(rows=3000, empty_fraction=0.1)
+    xd, fd, od_, xsd = dev(x), dev(f), dev(off), dev(xs)
+    rd, cd, vd, xvd = dev(rowptr), dev(col), dev(val), dev(xv)
+    ws1 = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    ws2 = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.I8_TO_I32, mmv.SEG_OFFSETS_I32, xs.shape[0], off.shape[0] - 1)
+    ws3 = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, val.shape[0], 3000)
+    o1 = torch.zeros(n, dtype=torch.int32, device="cuda")
+    o2 = torch.zeros(off.shape[0] - 1, dtype=torch.int32, device="cuda")
+    o3 = torch.zeros(3000, dtype=torch.float32, device="cuda")
+
+    def calls():
+        mmv.seg_scan(xd, fd, out=o1, workspace=ws1)
+        mmv.seg_sum(xsd, od_, out=o2, workspace=ws2)
+        mmv.spmv_csr(rd, cd, vd, xvd, y=o3, workspace=ws3)
+
+    calls()                                   # warm-up outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        calls()
+    for buf in (o1, o2, o3):
+        buf.zero_()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    assert mmv.last_async_status(ws1) == 0 and mmv.last_async_status(ws2) == 0 and mmv.last_async_status(ws3) == 0
+    assert np.array_equal(o1.cpu().numpy(), oracle.seg_scan_i8(x, f))
+    assert np.array_equal(o2.cpu().numpy(), oracle.seg_sum_csr_i8(xs, off))
+    want, a = oracle.spmv_csr(rowptr, col, val, xv)
+    assert_fp(o3.cpu().numpy(), want, a, "SpMV replayed from a graph")
