@@ -130,3 +130,35 @@ def test_config4_full_size(mmv, empty_fraction):
     if empty_fraction:
         lens = np.diff(rowptr.astype(np.int64))
         assert (y.cpu().numpy()[lens == 0] == 0).all()
+
+
+def test_scan_beyond_2_to_the_32_elements_closed_form(mmv):
+    """Index arithmetic past 2^32 elements: all-ones int8 values with a start flag every 1000 elements
+    (one period is not a divisor of the tile size, so the flags drift through every position of a
+    tile), for which the scan has the closed form z[i] = (i mod 1000) + 1; checked chunk by chunk on
+    the device.  A second launch without flags is checked against z[i] = i + 1 modulo 2^32."""
+    n = (1 << 32) + 12345
+    free, _ = torch.cuda.mem_get_info()
+    if free < 6 * n + (2 << 30):
+        pytest.skip("not enough device memory for a 2^32-element scan")
+    x = torch.ones(n, dtype=torch.int8, device="cuda")
+    f = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    f[::1000] = 1
+    out = torch.empty(n, dtype=torch.int32, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    mmv.seg_scan(x, f, out=out, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    step = 1 << 27
+    for o in range(0, n, step):
+        e = min(n, o + step)
+        idx = torch.arange(o, e, dtype=torch.int64, device="cuda")
+        assert torch.equal(out[o:e], (idx % 1000 + 1).to(torch.int32)), f"flagged scan wrong in [{o}, {e})"
+    del f
+    mmv.seg_scan(x, None, out=out, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    for o in range(0, n, step):
+        e = min(n, o + step)
+        idx = torch.arange(o + 1, e + 1, dtype=torch.int64, device="cuda")
+        want = (idx & 0xffffffff).to(torch.int64)
+        want = torch.where(want >= (1 << 31), want - (1 << 32), want).to(torch.int32)     # wrap-around modulo 2^32
+        assert torch.equal(out[o:e], want), f"plain scan wrong in [{o}, {e})"
