@@ -216,11 +216,10 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     int32_t* span_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
     if (!shape_sel) {          // (the flag-encoded form has filled span_q while compacting its flags)
         const long long spans = static_cast<long long>(tiles) * SPANS_PER_TILE;
-        const long long warps = spans + 1;
         const int threads = 256;
-        const long long blocks = (warps * 32 + threads - 1) / threads;
+        const long long blocks = (nseg + 1 + threads - 1) / threads;           // one thread per offset
         partition_offsets_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, shift, spans, span_q, n_eff,
-                                                                                 reinterpret_cast<WorkspaceHeader*>(ws), nseg_dev,
+                                                                                 reinterpret_cast<WorkspaceHeader*>(ws),
                                                                                  static_cast<uint32_t*>(out));
         ++g_launches;
     }

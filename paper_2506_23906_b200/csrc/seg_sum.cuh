@@ -271,29 +271,59 @@ __device__ __noinline__ long long first_index_at_least_call(const int32_t* off, 
     return first_index_at_least(off, shift, lo, hi, target);
 }
 
-// span_q[s] = first index q in [0, nseg] with (off[q] << shift) >= s * SPAN, nseg + 1 if none.
-// One warp per span edge.  The same launch validates the offsets (non-decreasing, inside [0, n]; it
-// records MMV_ERR_BAD_SEGMENTS otherwise, and the main kernel never indexes outside its tile
-// whatever they hold) and writes the zero of every EMPTY segment, so that the main kernel may jump
-// over long runs of equal offsets instead of visiting them one by one.
+// span_q[s] = first index i in [0, nseg] with bnd(i) = off[i] << shift >= s * SPAN, nseg + 1 if none,
+// for s = 0 .. num_spans.  One thread per offset index i: i is that first index exactly for the
+// spans s with bnd(i-1) < s * SPAN <= bnd(i), a range it writes itself (ranges of more than 32
+// spans, i.e. very long segments, are written by the whole warp).  The same pass validates the
+// offsets (non-decreasing, inside [0, n]; MMV_ERR_BAD_SEGMENTS otherwise -- entries may then be
+// missing or inconsistent, which the main kernel tolerates: it clamps what it reads and never
+// indexes outside its tile) and writes the zero of every EMPTY segment, so that the main kernel
+// may jump over long runs of equal offsets instead of visiting them one by one.
 __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, int shift, long long num_spans,
                                          int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr,
-                                         const long long* __restrict__ nseg_dev, uint32_t* __restrict__ out) {
-    if (nseg_dev) nseg = *nseg_dev;
-    {
-        const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-        bool bad = false;
-        for (long long q = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; q < nseg; q += stride) {
-            const long long a = static_cast<long long>(off[q]) << shift, b = static_cast<long long>(off[q + 1]) << shift;
-            bad |= (a > b) || (a < 0) || (b > n);
-            if (a == b) out[q] = 0u;
+                                         uint32_t* __restrict__ out) {
+    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;      // offset index
+    const int lane = threadIdx.x & 31;
+    long long lo = 0, hi = -1;                 // spans [lo, hi] get the value i
+    long long tlo = 0, thi = -1;               // spans behind the last offset get nseg + 1
+    if (i <= nseg) {
+        const long long cur = static_cast<long long>(off[i]) << shift;
+        long long prev = -1;
+        if (i >= 1) {
+            prev = static_cast<long long>(off[i - 1]) << shift;
+            if (prev > cur || prev < 0 || cur > n) report_error(hdr, 4u);
+            if (prev == cur) out[i - 1] = 0u;                      // segment i - 1 is empty
+            lo = (prev < 0 ? -1 : prev / SPAN) + 1;
+        } else if (cur < 0 || cur > n) {
+            report_error(hdr, 4u);
         }
-        if (bad) report_error(hdr, 4u);
+        hi = cur < 0 ? -1 : cur / SPAN;
+        if (hi > num_spans) hi = num_spans;
+        if (lo < 0) lo = 0;
+        if (i == nseg) {
+            tlo = hi + 1;
+            thi = num_spans;
+        }
     }
-    const long long warp = (static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x) >> 5;
-    if (warp > num_spans) return;
-    const long long lo = first_index_at_least(off, shift, 0, nseg + 1, warp * SPAN);
-    if ((threadIdx.x & 31) == 0) span_q[warp] = static_cast<int32_t>(lo);
+    if (hi - lo < 32) {
+        for (long long s = lo; s <= hi; ++s) span_q[s] = static_cast<int32_t>(i);
+        hi = lo - 1;
+    }
+    // long ranges, and the range behind the last offset: the whole warp writes them
+    unsigned todo = __ballot_sync(0xffffffffu, hi >= lo);
+    while (todo) {
+        const int src = __ffs(todo) - 1;
+        const long long l = __shfl_sync(0xffffffffu, lo, src), h = __shfl_sync(0xffffffffu, hi, src);
+        const long long v = __shfl_sync(0xffffffffu, i, src);
+        for (long long s = l + lane; s <= h; s += 32) span_q[s] = static_cast<int32_t>(v);
+        todo &= todo - 1;
+    }
+    todo = __ballot_sync(0xffffffffu, thi >= tlo);
+    if (todo) {
+        const int src = __ffs(todo) - 1;
+        const long long l = __shfl_sync(0xffffffffu, tlo, src), h = __shfl_sync(0xffffffffu, thi, src);
+        for (long long s = l + lane; s <= h; s += 32) span_q[s] = static_cast<int32_t>(nseg + 1);
+    }
 }
 
 template <typename P, int G>
@@ -511,6 +541,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         // extension would make the warp wait for the load on the spot.  `last_ok` says whether `last`
         // was loaded at all.)
         auto load_offsets = [&](long long q0, long long qe, int32_t (&raw)[4], int32_t& rawp, int32_t& last, bool& last_ok) {
+            if (q0 < 0) q0 = 0;
+            if (q0 > nq) q0 = nq;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const long long qi = q0 + lane + 32 * j;
@@ -554,7 +586,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             const uint32_t taddr = tmem_base + buf * (PIECES_PER_SPAN * ROW) + ((static_cast<uint32_t>(w) * 32u) << 16);
 
             // ---- the span's boundaries: one offset per lane (requested during the previous tile) ----
-            long long q = q_next;                              // first q with bnd(q) >= sbase
+            // (clamped: with offsets that are not sorted the partition may hold anything)
+            long long q = q_next < 0 ? 0 : (q_next > nq ? nq : q_next);     // first q with bnd(q) >= sbase
             const long long cq = q;                            // index held by lane 0 of the cache
             int32_t raw[4];
 #pragma unroll

@@ -256,6 +256,13 @@ def test_seg_sum_csr_edges(mmv):
     # segments that do not cover the ends of x: values outside [off[0], off[-1]) are ignored
     off = np.asarray([100, 5000, 5000, 40000], np.int32)
     assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
+    # segments that span more than 32 spans each, and more than 32 spans of ignored values at both ends
+    n = 150 * 4096 + 77
+    x = np.random.default_rng(2).integers(-128, 128, n).astype(np.int8)
+    off = np.asarray([34 * 4096 + 5, 34 * 4096 + 7, 70 * 4096, 70 * 4096 + 1, 110 * 4096 + 4095, 110 * 4096 + 4095], np.int32)
+    assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
+    off = np.asarray([0, 33 * 4096, n], np.int32)
+    assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off))
     # all segments empty, no values at all
     off = np.zeros(9, np.int32)
     assert sum_csr(mmv, np.zeros(0, np.int8), off).tolist() == [0] * 8
