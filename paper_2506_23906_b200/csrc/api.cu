@@ -211,14 +211,15 @@ __global__ void spmv_gather_kernel(const int32_t* __restrict__ col, const __half
 template <typename P>
 mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* off, long long nseg, int shift,
                           void* out, uint8_t* ws, const WorkspacePlan& plan, DeviceInfo* dev, cudaStream_t st,
-                          const long long* nseg_dev = nullptr, const int* shape_sel = nullptr) {
+                          const long long* nseg_dev = nullptr, bool have_partition = false) {
     const int tiles = static_cast<int>(num_tiles_of(n_eff));
     int32_t* span_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
-    if (!shape_sel) {          // (the flag-encoded form has filled span_q while compacting its flags)
+    if (!have_partition) {     // (the flag-encoded form has filled span_q while compacting its flags)
         const long long spans = static_cast<long long>(tiles) * SPANS_PER_TILE;
         const int threads = 256;
-        const long long blocks = (nseg + 1 + threads - 1) / threads;           // one thread per offset
-        partition_offsets_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, shift, spans, span_q, n_eff,
+        long long blocks = (nseg + 1 + threads - 1) / threads;                 // one thread per offset and round
+        if (blocks > 16ll * dev->sm_count) blocks = 16ll * dev->sm_count;
+        partition_offsets_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, spans, span_q, n_eff,
                                                                                  reinterpret_cast<WorkspaceHeader*>(ws),
                                                                                  static_cast<uint32_t*>(out));
         ++g_launches;
@@ -237,21 +238,10 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();
     prm.nseg_dev = nseg_dev;
-    prm.shape_sel = shape_sel;
     const int grid = tiles < dev->sm_count ? tiles : dev->sm_count;
-    if (shape_sel) {
-        // flag-encoded segments: their number is only known on the device, which has left its choice
-        // in *shape_sel; both shapes are launched and the other one returns at once
-        seg_sum_kernel<P, 2><<<grid, SumShape<2>::kThreads, SumCfg<P, 2>::kSmemBytes, st>>>(tmap, values, prm);
-        seg_sum_kernel<P, 3><<<grid, SumShape<3>::kThreads, SumCfg<P, 3>::kSmemBytes, st>>>(tmap, values, prm);
-        g_launches += 2;
-        return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
-    }
-    // Long segments (few boundaries per 4096-element span): twelve epilogue warps on the light path.
-    bool many_warps = nseg > 0 && n_eff / nseg >= 256;
-    if (g_force_groups.load() == 2) many_warps = false;
-    if (g_force_groups.load() == 3) many_warps = true;
-    if (many_warps)
+    // Twelve epilogue warps (three warpgroups) measured faster than eight at every segment density;
+    // the shape with two warpgroups stays available for tests and measurements.
+    if (g_force_groups.load() != 2)
         seg_sum_kernel<P, 3><<<grid, SumShape<3>::kThreads, SumCfg<P, 3>::kSmemBytes, st>>>(tmap, values, prm);
     else
         seg_sum_kernel<P, 2><<<grid, SumShape<2>::kThreads, SumCfg<P, 2>::kSmemBytes, st>>>(tmap, values, prm);
@@ -548,16 +538,15 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
         const long long cap = static_cast<long long>(dev->sm_count) * 8;
         const unsigned blocks = static_cast<unsigned>(nchunks < cap ? nchunks : cap);
         flag_count_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_count);
-        int* shape_sel = reinterpret_cast<int*>(ws + plan.cmp_off + 8);
         chunk_scan_kernel<<<1, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, nseg_dev,
-                                              reinterpret_cast<long long*>(d_num_segments), off, n, shape_sel);
+                                              reinterpret_cast<long long*>(d_num_segments), off, n);
         static_assert(CMP_CHUNK == TILE && SPAN == 4096, "a compaction chunk is one tile of four spans");
         flag_scatter_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_base, off,
                                                             reinterpret_cast<int32_t*>(ws + plan.tileq_off), nseg_dev);
         g_launches += 3;
         if (cudaGetLastError() != cudaSuccess) return MMV_ERR_CUDA;
-        if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, shape_sel);
-        return launch_seg_sum<I8Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, shape_sel);
+        if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, true);
+        return launch_seg_sum<I8Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, true);
     }
     if (nseg == 0) return MMV_OK;
     if (!seg || !out) return MMV_ERR_INVALID_ARG;

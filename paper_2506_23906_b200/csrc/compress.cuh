@@ -84,11 +84,11 @@ flag_count_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks,
 }
 
 // One block: chunk_base = exclusive scan of chunk_count; K = total is written to nseg_dev and, when given,
-// to the caller's d_num_segments; off[K] = n closes the last segment; *shape_sel picks the kernel shape.
+// to the caller's d_num_segments; off[K] = n closes the last segment.
 __global__ void __launch_bounds__(1024)
 chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, int32_t* __restrict__ chunk_base,
                   long long* __restrict__ nseg_dev, long long* __restrict__ d_num_segments, int32_t* __restrict__ off,
-                  long long n, int* __restrict__ shape_sel) {
+                  long long n) {
     __shared__ int warp_sums[32];
     // Each thread takes `per` consecutive counts, a multiple of four so that it can read and write
     // them as 16-byte vectors: with scalar accesses 64 bytes apart every instruction of a warp touches
@@ -123,8 +123,6 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
         *nseg_dev = total;
         if (d_num_segments) *d_num_segments = total;
         off[total] = static_cast<int32_t>(n);
-        // long segments on average: the segmented-sum kernel with twelve epilogue warps takes the call
-        *shape_sel = (total > 0 && n / total >= 256) ? 3 : 2;
     }
 }
 

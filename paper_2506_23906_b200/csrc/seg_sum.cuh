@@ -18,15 +18,24 @@
 //     few boundaries (<= 8): each boundary's prefix is read straight from TMEM (one column, it
 //                  sits in the lane of its row), the 128 row totals are scanned with four
 //                  interleaved warp scans, and lane j emits the segment that ends at boundary j.
-//     general path the offsets go to a per-warp table in shared memory; a piece that contains a
-//                  boundary has its 32 x 32 prefixes copied to shared memory and its boundaries
-//                  walked 32 at a time; every segment end emits  prefix(end) - prefix(start-1)
-//                  (the DIFF of Algorithm 4.2 applied to the COMPRESSed speculative scan, but with
-//                  prefixes local to the row or the piece so that magnitudes stay small).
-//     Segments of at most four elements are summed from the input values themselves; segments
-//     that cross pieces take the running sum of the open segment; the one segment per span that
-//     began before it takes the carry of the sibling spans (shared memory) or of a decoupled
-//     look-back over per-span status words.  Pieces without a boundary only add their total.
+//     general path every boundary of the span marks, in a per-warp bit table in shared memory, the
+//                  element it ends behind (one lane per boundary, 128 at a time); then, piece by
+//                  piece, the 32 x 32 prefixes go to shared memory and every lane walks the marked
+//                  elements of ITS row: a segment end emits  prefix(end) - prefix(previous end)
+//                  (the DIFF of Algorithm 4.2 applied to the COMPRESSed speculative scan, with
+//                  prefixes local to the row so that magnitudes stay small); a row's first end adds
+//                  what is open from the rows before it (segmented warp scan of row totals and
+//                  tails).  The output index of a row's first sum is the number of boundaries in
+//                  front of the row, so nothing is searched or sorted; only rows that contain
+//                  empty segments look their indices up in the offsets.
+//     Floating point: a difference of prefixes loses a small sum next to large values.  In the
+//     few-boundaries path segments of at most four elements are therefore summed from the input
+//     values themselves; in the general path any segment inside one row or two adjacent rows whose
+//     sum came out below 2^-10 of those rows' largest prefix is added up again from its values, and
+//     so is the segment of at most 32 elements that reaches back across the span's first element.
+//     The one segment per span that began before it (and is longer) takes the carry of the sibling
+//     spans (shared memory) or of a decoupled look-back over per-span status words.  Pieces
+//     without a boundary only add their total.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -38,9 +47,9 @@ namespace mmv {
 // The kernel comes with G = 2 or 3 epilogue warpgroups (4 G epilogue warps, then the TMA producer
 // warp and the MMA warp).  The epilogue is a chain of dependent instructions per span, so its
 // throughput grows with the number of warps: G = 3 (12 epilogue warps, 128 registers, one TMEM
-// buffer per group) is used when segments are long and the light few-boundaries path does the
-// work, G = 2 (8 warps, 168 registers, the MMA warp one tile ahead) when boundaries are dense.
-// (G = 4 compiles too but measured no better than 3: 96 registers make the general path spill.)
+// buffer per group) measured faster than G = 2 (8 warps, 168 registers, the MMA warp one tile
+// ahead) at every segment density and is what the library launches; G = 2 is kept for tests.
+// (G = 4 compiles too but measured no better than 3.)
 constexpr int SUM_BUFS = 4;                                        // TMEM tile buffers, shared out among the warpgroups
 constexpr int SUM_TMEM_COLS = SUM_BUFS * PIECES_PER_SPAN * ROW;    // 512
 template <int G>
@@ -53,9 +62,10 @@ struct SumShape {
     static constexpr int kBufsPerGroup = G == 2 ? 2 : 1;
 };
 constexpr int SUM_SPARSE_MAX = 8;                                  // spans with at most this many boundaries read single prefixes from TMEM
-constexpr int SUM_DIRECT_LEN = 4;                                  // segments this short are summed from the inputs
-constexpr int SUM_TBL = 128;                                       // boundaries of a span kept in shared memory
-constexpr int SUM_TBL_BYTES = (SUM_TBL + 4) * 4 + SUM_TBL * 4;     // offsets (one predecessor in front) + direct sums
+constexpr int SUM_DIRECT_LEN = 4;                                  // few-boundaries path: segments this short are summed from the inputs
+constexpr float SUM_CANCEL = 1.0f / 1024.0f;                       // general path: a sum this small against its prefixes is added up again
+constexpr int SUM_TBL = 128;                                       // boundaries a warp handles at a time (four per lane)
+constexpr int SUM_TBL_BYTES = 2 * (SPAN / ROW) * 4 + 16;           // per warp: marked elements and boundary counts of 128 rows, one counter
 
 // The fp32 products of SpMV, each stored as a pair of bf16 values (hi = bf16(z), lo = bf16(z - hi),
 // 4 bytes).  An ELEMENT of this path is one product; a row of 32 products is a 128-byte operand
@@ -213,8 +223,7 @@ struct SumCfg {
     static constexpr int kDumpBytes = PIECE * 4;                     // per epilogue warp
     static constexpr int kStageOffset = 4096;                        // after the constant operand
     static constexpr int kDumpOffset = kStageOffset + kStages * kXBytes;
-    static constexpr int kRowpreOffset = kDumpOffset + SumShape<G>::kEpiWarps * kDumpBytes;
-    static constexpr int kTblOffset = kRowpreOffset + SumShape<G>::kEpiWarps * PIECE_ROWS * 4;
+    static constexpr int kTblOffset = kDumpOffset + SumShape<G>::kEpiWarps * kDumpBytes;
     static constexpr int kBarOffset = kTblOffset + SumShape<G>::kEpiWarps * SUM_TBL_BYTES;
     static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
     static_assert(kBBytes <= kStageOffset, "constant operand fits its slot");
@@ -234,8 +243,6 @@ struct SumParams {
     unsigned long long budget_ns;
     const long long* nseg_dev;   // when not null: the number of segments is read from here (flag-encoded
                                  // segments, whose count is only known on the device); nseg is ignored
-    const int* shape_sel;        // when not null: both kernel shapes are launched and the one whose G
-                                 // differs from *shape_sel returns at once (the choice depends on nseg)
 };
 
 // First index q in [lo, hi) with (off[q] << shift) >= target, hi if none; the offsets are
@@ -279,50 +286,57 @@ __device__ __noinline__ long long first_index_at_least_call(const int32_t* off, 
 // missing or inconsistent, which the main kernel tolerates: it clamps what it reads and never
 // indexes outside its tile) and writes the zero of every EMPTY segment, so that the main kernel
 // may jump over long runs of equal offsets instead of visiting them one by one.
-__global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, int shift, long long num_spans,
+__global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, long long num_spans,
                                          int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr,
                                          uint32_t* __restrict__ out) {
-    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;      // offset index
     const int lane = threadIdx.x & 31;
-    long long lo = 0, hi = -1;                 // spans [lo, hi] get the value i
-    long long tlo = 0, thi = -1;               // spans behind the last offset get nseg + 1
-    if (i <= nseg) {
-        const long long cur = static_cast<long long>(off[i]) << shift;
-        long long prev = -1;
-        if (i >= 1) {
-            prev = static_cast<long long>(off[i - 1]) << shift;
-            if (prev > cur || prev < 0 || cur > n) report_error(hdr, 4u);
-            if (prev == cur) out[i - 1] = 0u;                      // segment i - 1 is empty
-            lo = (prev < 0 ? -1 : prev / SPAN) + 1;
-        } else if (cur < 0 || cur > n) {
-            report_error(hdr, 4u);
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    const int n32 = static_cast<int>(n < 0x7fffffffll ? n : 0x7fffffffll);
+    const int last_span = static_cast<int>(num_spans);
+    // (every warp makes the same number of rounds: the votes below need all its lanes; positions and span
+    //  indices fit 32 bits because the offsets do)
+    for (long long wbase = static_cast<long long>(blockIdx.x) * blockDim.x + (threadIdx.x & ~31); wbase <= nseg; wbase += stride) {
+        const long long i = wbase + lane;          // offset index
+        const bool exists = i <= nseg;
+        const int cur = exists ? off[i] : 0;
+        int prev = __shfl_up_sync(0xffffffffu, cur, 1);
+        if (lane == 0) prev = wbase >= 1 ? off[wbase - 1] : 0;
+        int lo = 0, hi = -1;                       // spans [lo, hi] get the value i
+        if (exists) {
+            if (i >= 1) {
+                if (prev > cur || prev < 0 || cur > n32) report_error(hdr, 4u);
+                if (prev == cur) out[i - 1] = 0u;                  // segment i - 1 is empty
+                lo = prev < 0 ? 0 : (prev >> 12) + 1;
+            } else if (cur < 0 || cur > n32) {
+                report_error(hdr, 4u);
+            }
+            hi = cur < 0 ? -1 : (cur >> 12);
+            if (hi > last_span) hi = last_span;
         }
-        hi = cur < 0 ? -1 : cur / SPAN;
-        if (hi > num_spans) hi = num_spans;
-        if (lo < 0) lo = 0;
-        if (i == nseg) {
-            tlo = hi + 1;
-            thi = num_spans;
+        static_assert(SPAN == 4096, "span index = position >> 12");
+        const bool is_last = exists && i == nseg;
+        unsigned todo = __ballot_sync(0xffffffffu, hi >= lo || is_last);
+        if (todo == 0u) continue;                  // no span starts between this warp's offsets
+        if (hi >= lo && hi - lo < 32) {
+            for (int s = lo; s <= hi; ++s) span_q[s] = static_cast<int32_t>(i);
+            lo = hi + 1;
         }
-    }
-    if (hi - lo < 32) {
-        for (long long s = lo; s <= hi; ++s) span_q[s] = static_cast<int32_t>(i);
-        hi = lo - 1;
-    }
-    // long ranges, and the range behind the last offset: the whole warp writes them
-    unsigned todo = __ballot_sync(0xffffffffu, hi >= lo);
-    while (todo) {
-        const int src = __ffs(todo) - 1;
-        const long long l = __shfl_sync(0xffffffffu, lo, src), h = __shfl_sync(0xffffffffu, hi, src);
-        const long long v = __shfl_sync(0xffffffffu, i, src);
-        for (long long s = l + lane; s <= h; s += 32) span_q[s] = static_cast<int32_t>(v);
-        todo &= todo - 1;
-    }
-    todo = __ballot_sync(0xffffffffu, thi >= tlo);
-    if (todo) {
-        const int src = __ffs(todo) - 1;
-        const long long l = __shfl_sync(0xffffffffu, tlo, src), h = __shfl_sync(0xffffffffu, thi, src);
-        for (long long s = l + lane; s <= h; s += 32) span_q[s] = static_cast<int32_t>(nseg + 1);
+        // long ranges, and the range behind the last offset: the whole warp writes them
+        todo = __ballot_sync(0xffffffffu, hi >= lo);
+        while (todo) {
+            const int src = __ffs(todo) - 1;
+            const int l = __shfl_sync(0xffffffffu, lo, src), h = __shfl_sync(0xffffffffu, hi, src);
+            const int v = static_cast<int>(wbase) + src;
+            for (int s = l + lane; s <= h; s += 32) span_q[s] = v;
+            todo &= todo - 1;
+        }
+        todo = __ballot_sync(0xffffffffu, is_last);
+        if (todo) {
+            const int src = __ffs(todo) - 1;
+            const int h0 = __shfl_sync(0xffffffffu, cur < 0 ? -1 : (cur >> 12), src);
+            for (int s = (h0 > last_span ? last_span : h0) + 1 + lane; s <= last_span; s += 32)
+                span_q[s] = static_cast<int32_t>(nseg + 1);
+        }
     }
 }
 
@@ -330,7 +344,6 @@ template <typename P, int G>
 __global__ void __launch_bounds__(SumShape<G>::kThreads, 1)
 seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restrict__ xg, const SumParams prm) {
     using Acc = typename P::Acc;
-    if (prm.shape_sel && *prm.shape_sel != G) return;      // the other shape does this call
     using Cfg = SumCfg<P, G>;
     using Shape = SumShape<G>;
     constexpr int BPG = Shape::kBufsPerGroup;
@@ -512,20 +525,14 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         const int g = warp >> 2;
         const int w = warp & 3;
         Acc* outp = static_cast<Acc*>(prm.out);
-        uint8_t* dump = smem + Cfg::kDumpOffset + warp * Cfg::kDumpBytes;      // [32 rows][32] swizzled by row
-        Acc* rowpre = reinterpret_cast<Acc*>(smem + Cfg::kRowpreOffset) + warp * PIECE_ROWS;
-        int32_t* tbl = reinterpret_cast<int32_t*>(smem + Cfg::kTblOffset + warp * SUM_TBL_BYTES);   // [0] = offset before the first
-        Acc* dvt = reinterpret_cast<Acc*>(tbl + SUM_TBL + 4);
+        // per row of the span: marked elements (bits), number of boundaries; boundaries at the span's first element
+        uint8_t* dump = smem + Cfg::kDumpOffset + warp * Cfg::kDumpBytes;      // [32 rows][32] prefixes of a piece, swizzled by row
+        uint32_t* emask = reinterpret_cast<uint32_t*>(smem + Cfg::kTblOffset + warp * SUM_TBL_BYTES);
+        uint32_t* ecnt = emask + SPAN / ROW;
+        uint32_t* nbase = ecnt + SPAN / ROW;
         const int sh = prm.off_shift;
         const long long nq = (prm.nseg_dev ? *prm.nseg_dev : prm.nseg) + 1;
         bool failed = false;
-        // inclusive prefix inside the piece at element offset j (0..1023)
-        auto piece_prefix = [&](int j, Acc& rowpart, int& row) -> Acc {
-            row = j >> 5;
-            const int pos = j & 31;
-            rowpart = *reinterpret_cast<const Acc*>(dump + row * 128 + ((((pos >> 2) ^ (row & 7)) << 4) | ((pos & 3) << 2)));
-            return P::add(rowpre[row], rowpart);
-        };
         // The boundaries of the NEXT tile's span are requested one tile ahead (first the span's first
         // offset index, then one offset per lane), so that their two dependent round trips never
         // sit on the critical path.
@@ -619,41 +626,80 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             MMV_T_MARK(9)
             // very short segments that end in this span are summed from the inputs; the loads go out
             // now and return while the accumulators are awaited
-            bool isdir[4] = {false, false, false, false};
+            bool isdir[1] = {false};
             isdir[0] = cq + lane >= 1 && cq + lane < nq && sbj[0] >= 0 && bj[0] > sbj[0] && bj[0] - sbj[0] <= SUM_DIRECT_LEN &&
                        bj[0] > sbase && bj[0] <= send && bj[0] <= prm.n;
+            // (the general path needs only the one that reaches back across the span's first element)
+            if (!sparse && !(lane == 0 && sbj[0] < sbase)) isdir[0] = false;
             ValueWindow win0;
             win0.wide = false;
             if (isdir[0]) window_load<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), prm.n, win0);
+            int xlen = 0;
+            Acc xval = Acc(0);
+            // ---- general path, first step: every boundary marks the element it ends behind.  emask[row] has
+            //      bit c set if a segment ends behind element c of that row of the span, ecnt[row] counts the
+            //      boundaries there (more than the bits if empty segments follow), nbase those exactly at the
+            //      span's first element.  The first 128 boundaries are in registers already. ----
+            const uint32_t sb32 = static_cast<uint32_t>(sbase);
             bool tcovers = covers;
-            ValueWindow wn[3];                 // direct sums of table entries 32..127 (general path only)
-            wn[0].wide = wn[1].wide = wn[2].wide = false;
-            if (!sparse) {
-                // the general path keeps up to 128 boundaries in a shared-memory table
-                bool tc = false;
-                tbl[1 + lane] = raw[0];
-                if (lane == 0) tbl[0] = rawp;
-#pragma unroll
-                for (int j = 1; j < 4; ++j) {
-                    int32_t pr = __shfl_up_sync(0xffffffffu, raw[j], 1);
-                    const int32_t wrap = __shfl_sync(0xffffffffu, raw[j - 1], 31);
-                    if (lane == 0) pr = wrap;
-                    if (cq + lane + 32 * j < nq) bj[j] = cvt(raw[j]);
-                    sbj[j] = cvt(pr);
-                    tbl[1 + lane + 32 * j] = raw[j];
-                    tc |= (cq + lane + 32 * j >= nq) || (bj[j] > send);
-                    isdir[j] = cq + lane + 32 * j < nq && sbj[j] >= 0 && bj[j] > sbj[j] && bj[j] - sbj[j] <= SUM_DIRECT_LEN &&
-                               bj[j] > sbase && bj[j] <= send && bj[j] <= prm.n;
-                    // (the loads go out here, with those of entry 0; they are summed after the pre-pass)
-                    if (isdir[j]) window_load<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), prm.n, wn[j - 1]);
+            int32_t yraw[4] = {kNoOffset, kNoOffset, kNoOffset, kNoOffset};
+            auto mark = [&](int32_t braw) -> bool {          // returns true if the boundary lies behind the span
+                const int rel = static_cast<int>(static_cast<uint32_t>(braw) - sb32);
+                if (braw >= 0) {
+                    if (rel == 0) {
+                        atomicAdd(nbase, 1u);
+                    } else if (rel > 0 && rel <= SPAN) {
+                        atomicOr(&emask[(rel - 1) >> 5], 1u << ((rel - 1) & 31));
+                        atomicAdd(&ecnt[(rel - 1) >> 5], 1u);
+                    }
                 }
-                tcovers = __any_sync(0xffffffffu, tc) || covers;
+                return rel > SPAN;
+            };
+            if (!sparse) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) emask[lane + 32 * j] = 0u;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) ecnt[lane + 32 * j] = 0u;
+                if (lane == 0) *nbase = 0u;
+                __syncwarp();
+                bool tc = false;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (j == 0 || !covers) {           // (if the first 32 reach past the span the others lie behind it)
+                        if (cq + lane + 32 * j < nq) tc |= mark(raw[j]);
+                        else tc = true;
+                    }
+                }
+                tcovers = covers || __any_sync(0xffffffffu, tc);
+                // General path: the segment that reaches back across the span's first element (it ends at the first
+                // boundary): with at most 32 elements its values themselves are added up, one per lane.  Its carry
+                // would be a difference of the previous span's prefixes, which loses a small sum next to large values.
+                if constexpr (P::kIsFloat) {
+                    const bool crossing = cq >= 1 && cq < nq && csb >= 0 && csb < sbase && cb > sbase && cb <= send && cb <= prm.n &&
+                                          cb - csb <= 32;
+                    xlen = __shfl_sync(0xffffffffu, crossing ? static_cast<int>(cb - csb) : 0, 0);
+                    if (xlen > 0) {
+                        const long long xsb = __shfl_sync(0xffffffffu, csb, 0);
+                        if (static_cast<int>(lane) < xlen) xval = load_value<P>(xg, xsb + lane);
+                    }
+                }
+                // the next 128 offsets travel behind the accumulator wait
+                if (!tcovers) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const long long qi = cq + SUM_TBL + lane + 32 * j;
+                        if (qi < nq) yraw[j] = prm.off[qi];
+                    }
+                }
             }
 
             MMV_T_MARK(0)
             if (!wait_bar(&bar_acc_full[buf], (k / BPG) & 1, abort_flag, budget)) { failed = true; break; }
             tc_fence_after_sync();
             MMV_T_MARK(1)
+            // request the next tile's offsets (its first index has arrived by now): they travel while this
+            // tile's boundaries are worked through
+            if (tile_n >= 0) load_offsets(q_next, qe_next, nraw, nrawp, nlast, nlast_ok);
 
             LookbackWindow<1> lbw;
             Acc tot[PIECES_PER_SPAN];
@@ -806,148 +852,207 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     tail = P::add(__shfl_sync(0xffffffffu, P::sub(totl, before), rl), after);
                 }
                 publish(tail);
-                // direct sums: the values were requested before the accumulators were awaited
-                dvt[lane] = isdir[0] ? window_sum<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), win0) : Acc(0);
-                if (!covers) {
-#pragma unroll
-                    for (int j = 1; j < 4; ++j)
-                        dvt[lane + 32 * j] = isdir[j] ? window_sum<P>(xg, sbj[j], static_cast<int>(bj[j] - sbj[j]), wn[j - 1]) : Acc(0);
-                }
-                __syncwarp();
                 MMV_T_MARK(2)
             }
-#pragma unroll 1
-            for (int i = 0; i < (sparse ? 0 : PIECES_PER_SPAN); ++i) {
-                const long long pbase = sbase + i * PIECE;
-                const long long pend = pbase + PIECE;
-                Acc toti = tot[0];
+            if (!sparse) {
+                // ---- general path, second step: the boundaries beyond the first 128 mark their elements, 128 at
+                //      a time with the next 128 offsets already requested.  128 equal offsets in a row are a run of
+                //      empty segments (their zeros were written when the offsets were partitioned): the run is
+                //      jumped over with a 32-ary search and only counted. ----
+                if (!tcovers) {
+                    long long tp = cq + SUM_TBL;            // index of yraw's first boundary
+                    while (true) {
+                        int32_t zraw[4] = {kNoOffset, kNoOffset, kNoOffset, kNoOffset};
 #pragma unroll
-                for (int t = 1; t < PIECES_PER_SPAN; ++t)
-                    if (i == t) toti = tot[t];
-                // any boundary with pbase <= bnd <= pend (END in (pbase, pend], START in [pbase, pend))?
-                bool touched = true;
-                if (tcovers) {
-                    bool t4 = false;
+                        for (int j = 0; j < 4; ++j) {
+                            const long long qi = tp + SUM_TBL + lane + 32 * j;
+                            if (qi < nq) zraw[j] = prm.off[qi];
+                        }
+                        const int32_t first = __shfl_sync(0xffffffffu, yraw[0], 0);
+                        bool beyond = false, same = true;
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) t4 |= (cq + lane + 32 * j >= q) && (bj[j] >= pbase) && (bj[j] <= pend);
-                    touched = __any_sync(0xffffffffu, t4);
-                }
-                if (!touched) {
-                    run = P::add(run, warp_sum<P>(toti));
-                    MMV_T_MARK(3)
-                    continue;
-                }
-
-                // ---- prefixes of the piece -> shared memory, exclusive scan of the 32 row totals ----
-                uint32_t r[32];
-                tmem_ld_32x32(taddr + i * ROW, r);
-                tmem_ld_wait();
+                        for (int j = 0; j < 4; ++j) {
+                            if (tp + lane + 32 * j < nq) beyond |= mark(yraw[j]);
+                            else beyond = true;
+                            same &= yraw[j] == first;
+                        }
+                        if (__any_sync(0xffffffffu, beyond)) break;
+                        tp += SUM_TBL;
 #pragma unroll
-                for (int c4 = 0; c4 < 8; ++c4)
-                    *reinterpret_cast<uint4*>(dump + lane * 128 + ((c4 ^ (lane & 7)) << 4)) =
-                        make_uint4(r[4 * c4], r[4 * c4 + 1], r[4 * c4 + 2], r[4 * c4 + 3]);
-                Acc inc = toti;
+                        for (int j = 0; j < 4; ++j) yraw[j] = zraw[j];
+                        if (__all_sync(0xffffffffu, same)) {
+                            const long long u = first_index_at_least_call(prm.off, sh, tp, nq, static_cast<long long>(first) + 1);
+                            if (u > tp) {
+                                const int rel = static_cast<int>(static_cast<uint32_t>(first) - sb32);
+                                if (lane == 0) {
+                                    if (rel == 0) atomicAdd(nbase, static_cast<uint32_t>(u - tp));
+                                    else if (rel > 0 && rel <= SPAN) atomicAdd(&ecnt[(rel - 1) >> 5], static_cast<uint32_t>(u - tp));
+                                }
+                                tp = u;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const Acc t = __shfl_up_sync(0xffffffffu, inc, o);
-                    if (static_cast<int>(lane) >= o) inc = P::add(t, inc);
-                }
-                rowpre[lane] = P::sub(inc, toti);
-                const Acc piece_total = __shfl_sync(0xffffffffu, inc, 31);
-                __syncwarp();
-                MMV_T_MARK(4)
-
-                // ---- boundaries with pbase <= bnd(q) <= pend, 32 at a time (sorted: a prefix of every batch) ----
-                bool piece_has_start = false;
-                long long last_start = -1;
-                long long qp = q;              // batch pointer
-                long long advance = 0;         // boundaries strictly before pend: consumed for good
-                while (true) {
-                    const long long qi = qp + lane;
-                    long long b = -1, sb = -1;
-                    Acc dv = Acc(0);
-                    const long long rel = qi - cq;
-                    const bool cached = rel < SUM_TBL;
-                    if (cached) {
-                        if (qi < nq) b = cvt(tbl[1 + rel]);
-                        if (qi >= 1 && qi < nq) sb = cvt(tbl[rel]);
-                        dv = dvt[rel];
-                    } else {
-                        if (qi < nq) b = static_cast<long long>(prm.off[qi]) << sh;
-                        if (qi >= 1 && qi < nq) sb = static_cast<long long>(prm.off[qi - 1]) << sh;
-                    }
-                    const bool in_piece = (qi < nq) && (b >= 0) && (b <= pend);
-                    const unsigned inm = __ballot_sync(0xffffffffu, in_piece);
-                    const int cnt = (inm == 0xffffffffu) ? 32 : (__ffs(~inm) - 1);
-                    const bool mine = static_cast<int>(lane) < cnt;
-                    bool deferred = false;
-                    Acc val = Acc(0);
-                    // as the END of segment qi-1: bnd in (pbase, pend], or 0 for leading empty segments
-                    if (mine && qi >= 1 && (b > pbase || (pbase == 0 && b == 0))) {
-                        if (sb > b || sb < 0 || b > prm.n) {
-                            report_error(prm.hdr, 4u);
-                        } else {
-                            if (b != sb) {
-                                if (b - sb <= SUM_DIRECT_LEN) {
-                                    // a very short segment: add the input values themselves
-                                    val = cached ? dv : direct_sum<P>(xg, sb, b);
-                                } else {
-                                    Acc ep, sp = Acc(0);
-                                    int erow, srow;
-                                    const Acc e_full = piece_prefix(static_cast<int>(b - 1 - pbase), ep, erow);
-                                    if (sb >= pbase) {
-                                        Acc s_full = Acc(0);
-                                        if (sb > pbase) s_full = piece_prefix(static_cast<int>(sb - 1 - pbase), sp, srow);
-                                        if (static_cast<int>((sb - pbase) >> 5) == erow)
-                                            val = ((sb - pbase) & 31) ? P::sub(ep, sp) : ep;   // inside one row
-                                        else
-                                            val = P::sub(e_full, s_full);
-                                    } else {
-                                        val = P::add(run, e_full);
-                                        deferred = sb < sbase;
-                                    }
+                                for (int j = 0; j < 4; ++j) {
+                                    const long long qi = tp + lane + 32 * j;
+                                    yraw[j] = qi < nq ? prm.off[qi] : kNoOffset;
                                 }
                             }
-                            if (!deferred) outp[qi - 1] = val;
+                        }
+                    }
+                }
+                __syncwarp();
+                MMV_T_MARK(3)
+
+                // ---- third step, lane = row: the piece's prefixes go to shared memory and every lane visits the
+                //      marked elements of its row, one sum each.  Inside the row a sum is the difference of two row
+                //      prefixes; the first one of a row adds what is open from the rows before (a segmented warp
+                //      scan of row totals and row tails).  A floating-point sum of a segment inside one row or two
+                //      adjacent rows that came out small against the prefixes it was taken from (cancellation:
+                //      under 2^-10 of the largest prefix of those rows) is added up again from the input values.  Output indices follow from the counts: the r-th row's first sum
+                //      belongs to boundary cq + nbase + (number of boundaries in the rows before). ----
+                const bool open_at_base = *nbase == 0u;          // the segment open at the span's first element began before it
+                long long obase = cq + static_cast<long long>(*nbase) - 1;     // output index of the span's first marked element
+                bool span_has_end = false;
+                // a very short segment that reaches back across the span's first element: summed from its values
+                const bool cross_done = xlen > 0 || __shfl_sync(0xffffffffu, isdir[0] ? 1 : 0, 0) != 0;
+                if (xlen > 0) {
+                    const Acc xsum = warp_sum<P>(xval);
+                    if (lane == 0) outp[cq - 1] = xsum;
+                } else if (lane == 0 && isdir[0]) {
+                    outp[cq - 1] = window_sum<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), win0);
+                }
+                // number of elements open at the end of the previous piece's last row (64: too many to matter),
+                // and the largest prefix magnitude of that row
+                int pc_len = open_at_base ? 64 : 0;
+                float pc_scale = 0.f;
+#pragma unroll 1
+                for (int i = 0; i < PIECES_PER_SPAN; ++i) {
+                    const long long pbase = sbase + i * PIECE;
+                    Acc toti = tot[0];
+#pragma unroll
+                    for (int t = 1; t < PIECES_PER_SPAN; ++t)
+                        if (i == t) toti = tot[t];
+                    const uint32_t m = emask[i * PIECE_ROWS + lane];
+                    const uint32_t cn = ecnt[i * PIECE_ROWS + lane];
+                    const unsigned hb = __ballot_sync(0xffffffffu, m != 0u);
+                    // output index of the row's first sum: exclusive scan of the boundary counts
+                    uint32_t cinc = cn;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t t = __shfl_up_sync(0xffffffffu, cinc, o);
+                        if (static_cast<int>(lane) >= o) cinc += t;
+                    }
+                    const long long orow = obase + (cinc - cn);
+                    obase += __shfl_sync(0xffffffffu, cinc, 31);
+                    if (hb == 0u) {
+                        run = P::add(run, warp_sum<P>(toti));
+                        pc_len = 64;
+                        continue;
+                    }
+                    float scale = 0.f;             // largest prefix magnitude of my row
+                    {
+                        uint32_t r[32];
+                        tmem_ld_32x32(taddr + i * ROW, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int c4 = 0; c4 < 8; ++c4)
+                            *reinterpret_cast<uint4*>(dump + lane * 128 + ((c4 ^ (lane & 7)) << 4)) =
+                                make_uint4(r[4 * c4], r[4 * c4 + 1], r[4 * c4 + 2], r[4 * c4 + 3]);
+                        if constexpr (P::kIsFloat) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) scale = fmaxf(scale, fabsf(__uint_as_float(r[c])));
+                        }
+                    }
+                    __syncwarp();
+                    MMV_T_MARK(4)
+
+                    // rows with empty segments among their boundaries look their output indices up in the offsets
+                    const bool dirty = cn != static_cast<uint32_t>(__popc(m));
+                    long long bp = orow + 1;                       // boundary index the next sum is looked for at
+                    const long long bend = bp + cn;
+                    const long long rowpos = pbase + lane * ROW;   // position of my row's first element
+                    Acc pv = Acc(0), first_pref = Acc(0);
+                    int cprev = -1, nend = 0, first_len = 0;
+                    long long first_oi = -1;
+                    uint32_t mm = m;
+                    while (mm) {                                   // (lanes differ in the number of marked elements)
+                        const int c = __ffs(mm) - 1;
+                        mm &= mm - 1;
+                        const Acc pc = *reinterpret_cast<const Acc*>(dump + lane * 128 + ((((c >> 2) ^ (lane & 7)) << 4) | ((c & 3) << 2)));
+                        long long oi = orow + nend;
+                        if (dirty) {
+                            const int32_t bpos = static_cast<int32_t>(rowpos + c + 1);
+                            while (bp + 1 < bend && prm.off[bp] < bpos) ++bp;
+                            oi = bp - 1;
+                            ++bp;
+                        }
+                        if (nend == 0) {
+                            first_pref = pc;
+                            first_len = c + 1;
+                            first_oi = oi;
+                        } else {
+                            Acc val = P::sub(pc, pv);
+                            if constexpr (P::kIsFloat) {
+                                if (fabsf(val) < scale * SUM_CANCEL)
+                                    val = direct_sum<P>(xg, rowpos + cprev + 1, rowpos + c + 1);
+                            }
+                            outp[oi] = val;
+                        }
+                        pv = pc;
+                        cprev = c;
+                        ++nend;
+                    }
+                    // what is open at the end of each row: the part behind its last marked element, or all of it
+                    const bool has_end = nend > 0;
+                    Acc v = has_end ? P::sub(toti, pv) : toti;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const Acc t = __shfl_up_sync(0xffffffffu, v, o);
+                        // rows lane - o + 1 .. lane without a marked element: the open part reaches further back
+                        const bool clear = static_cast<int>(lane) >= o && ((hb >> (lane - o + 1)) & ((1u << o) - 1u)) == 0u;
+                        if (clear) v = P::add(t, v);
+                    }
+                    // open sum at the START of my row: the inclusive value of the row before (plus the piece's carry
+                    // if no row before me has a marked element)
+                    Acc open = __shfl_up_sync(0xffffffffu, v, 1);
+                    if (lane == 0) open = Acc(0);
+                    const bool none_before = (hb & ((1u << lane) - 1u)) == 0u;
+                    if (none_before) open = P::add(run, open);
+                    // the previous row's open elements, if it has a marked element itself
+                    const int my_open = has_end ? 31 - cprev : 64;
+                    int c_len = __shfl_up_sync(0xffffffffu, my_open, 1);
+                    float c_scale = __shfl_up_sync(0xffffffffu, scale, 1);
+                    if (lane == 0) {
+                        c_len = pc_len;
+                        c_scale = pc_scale;
+                    }
+                    bool deferred = false;
+                    Acc fval = Acc(0);
+                    if (has_end) {
+                        fval = P::add(open, first_pref);
+                        const bool first_of_span = !span_has_end && none_before;
+                        if (first_of_span && open_at_base) {
+                            deferred = !cross_done;           // waits for the carry (or was summed from its values)
+                        } else {
+                            if constexpr (P::kIsFloat) {
+                                if (c_len < 64 && fabsf(fval) < fmaxf(scale, c_scale) * SUM_CANCEL)
+                                    fval = direct_sum<P>(xg, rowpos - c_len, rowpos + first_len);
+                            }
+                            if (first_oi >= 0) outp[first_oi] = fval;
                         }
                     }
                     const unsigned dm = __ballot_sync(0xffffffffu, deferred);
                     if (dm) {
                         const int src = __ffs(dm) - 1;
-                        def_r = __shfl_sync(0xffffffffu, qi, src) - 1;
-                        def_val = __shfl_sync(0xffffffffu, val, src);
+                        def_r = __shfl_sync(0xffffffffu, first_oi, src);
+                        def_val = __shfl_sync(0xffffffffu, fval, src);
                     }
-                    // as a START: bnd in [pbase, pend)
-                    const bool is_start = mine && (b >= pbase) && (b < pend);
-                    const unsigned sm = __ballot_sync(0xffffffffu, is_start);
-                    if (sm) {
-                        piece_has_start = true;
-                        last_start = __shfl_sync(0xffffffffu, b, 31 - __clz(sm));
-                    }
-                    advance += __popc(__ballot_sync(0xffffffffu, mine && (b < pend)));
-                    qp += cnt;
-                    if (cnt < 32) break;
-                    // A whole batch at one position is a run of empty segments.  Their zeros were written
-                    // when the offsets were partitioned: jump to the first boundary behind the run.
-                    const long long b0 = __shfl_sync(0xffffffffu, b, 0);
-                    if (b0 == __shfl_sync(0xffffffffu, b, 31)) {
-                        const long long u = first_index_at_least_call(prm.off, sh, qp, nq, b0 + 1);
-                        if (b0 < pend) advance += u - qp;
-                        qp = u;
-                    }
+                    span_has_end = true;
+                    // carries into the next piece
+                    run = __shfl_sync(0xffffffffu, v, 31);
+                    pc_len = __shfl_sync(0xffffffffu, my_open, 31);
+                    pc_scale = __shfl_sync(0xffffffffu, scale, 31);
+                    __syncwarp();
+                    MMV_T_MARK(5)
                 }
-                q += advance;
-                if (piece_has_start) {
-                    Acc sp2;
-                    int srow2;
-                    Acc before = Acc(0);
-                    if (last_start > pbase) before = piece_prefix(static_cast<int>(last_start - 1 - pbase), sp2, srow2);
-                    run = P::sub(piece_total, before);
-                } else {
-                    run = P::add(run, piece_total);
-                }
-                __syncwarp();
-                MMV_T_MARK(5)
             }
 
             // ---- the TMEM buffer is free; publish, look back, emit the segment that began before this span ----
@@ -955,8 +1060,6 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_acc_empty[buf]);
             MMV_T_MARK(6)
-            // request the next tile's offsets (its first index has arrived by now)
-            if (tile_n >= 0) load_offsets(q_next, qe_next, nraw, nrawp, nlast, nlast_ok);
             // Every warp waits on every phase of bar_agg (parity waits must not skip phases).  The carry
             // into this span is first sought among the tile's earlier spans (shared memory); only if
             // none of them holds a segment start does the look-back go out to the other CTAs' words.

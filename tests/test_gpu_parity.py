@@ -268,6 +268,33 @@ def test_seg_sum_csr_edges(mmv):
     assert sum_csr(mmv, np.zeros(0, np.int8), off).tolist() == [0] * 8
 
 
+def test_seg_sum_tiny_segments_next_to_large_values(mmv):
+    # segments of 1..4 small values between large ones: a difference of two prefixes would lose them in
+    # rounding (the bound is relative to the segment's own sum of magnitudes), so such sums have to come
+    # from the input values themselves; dense boundaries, every row of the tile layout has several
+    rng = np.random.default_rng(7)
+    nseg = 60000
+    lens = rng.integers(1, 9, nseg)
+    off = gen.offsets_from_lengths(lens)
+    n = int(off[-1])
+    big = rng.integers(0, 2, nseg).astype(bool)                      # every other segment holds large values
+    scale = np.where(big, 2000.0, 1e-3)
+    x = (rng.standard_normal(n) * np.repeat(scale, lens)).astype(np.float16)
+    want, a = oracle.seg_sum_csr_f16(x, off)
+    got = sum_csr(mmv, x, off)
+    assert_fp(got, want, a, "tiny next to large")
+    # the same with segment boundaries exactly at row, piece and span edges and lengths up to 32 (a segment
+    # inside one or two adjacent 32-element rows: the reach of the kernel's cancellation check)
+    lens = rng.integers(1, 33, 20000)
+    lens[::7] = 32
+    off = gen.offsets_from_lengths(lens)
+    n = int(off[-1])
+    scale = np.where(rng.integers(0, 3, lens.shape[0]) == 0, 3000.0, 2e-3)
+    x = (rng.standard_normal(n) * np.repeat(scale, lens)).astype(np.float16)
+    want, a = oracle.seg_sum_csr_f16(x, off)
+    assert_fp(sum_csr(mmv, x, off), want, a, "tiny next to large, longer")
+
+
 def test_seg_sum_long_runs_of_empty_segments(mmv):
     # hundreds of thousands of empty segments in a row (at the start, in the middle of a span, exactly on a
     # span edge, at the end): the kernel jumps over such runs instead of visiting them one by one
