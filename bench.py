@@ -376,6 +376,48 @@ def bench_configs(torch, mmv, peak, steps, warmup, l2_flush, cpu_leg):
         rec(name, nnz, 6 * nnz + 4 * (rows + 1) + 4 * xv.shape[0] + 4 * rows, ms,
             {"nnz": nnz, **baseline(nnz, lambda o: o.spmv_csr(rowptr, col, val, xv), fp_compare(y.cpu().numpy()))})
         del rd, cd, vd, xd, y, ws
+    # The paper's other segmented-sum shapes: segment lengths with the minimum / average / maximum of the
+    # matrices of its Table 5.1, about 2^26 fp16 values each (the dense-boundary regime of the kernel).
+    for kind in gen.ROW_LENGTH_MIXES:
+        x, off = gen.seg_sum_row_mix(kind, 1 << 26)
+        n, nseg = x.shape[0], off.shape[0] - 1
+        xd, od = torch.from_numpy(x).cuda(), torch.from_numpy(off).cuda()
+        out = torch.empty(nseg, dtype=torch.float32, device="cuda")
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, n, nseg)
+        fn = lambda: mmv.seg_sum(xd, od, out=out, workspace=ws)  # noqa: E731
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        ms = event_time_ms(torch, fn, steps)
+        assert mmv.last_async_status(ws) == 0
+        lens = np.diff(off.astype(np.int64))
+        rec(f"T5.1 seg-sum fp16, segment lengths min/avg/max {int(lens.min())}/{lens.mean():.0f}/{int(lens.max())} ({kind})",
+            n, 2 * n + 4 * (nseg + 1) + 4 * nseg, ms, {"segments": nseg})
+        del xd, od, out, ws
+
+    # The blocked sparse-attention matrices of the paper's SpMV experiment: 65,536 rows and columns,
+    # 2 global and 3 window blocks, block sizes 2..64, 2..8 random blocks ("b-X_r-Y").  One record for all
+    # twelve; bytes as for C4.  The vector (256 KB) stays in cache, unlike C4's.
+    bsa = []
+    for block in gen.BSA_BLOCKS:
+        for rb in gen.BSA_RANDOM:
+            rowptr, col, val, xv = gen.block_sparse_attention_csr(block, rb)
+            rows, nnz = rowptr.shape[0] - 1, val.shape[0]
+            rd, cd, vd, xd = (torch.from_numpy(t).cuda() for t in (rowptr, col, val, xv))
+            y = torch.empty(rows, dtype=torch.float32, device="cuda")
+            ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, nnz, rows)
+            fn = lambda: mmv.spmv_csr(rd, cd, vd, xd, y=y, workspace=ws)  # noqa: E731
+            for _ in range(warmup):
+                fn()
+            torch.cuda.synchronize()
+            ms = event_time_ms(torch, fn, steps, l2_flush if 6 * nnz < (256 << 20) else None)
+            assert mmv.last_async_status(ws) == 0
+            bytes_ = 6 * nnz + 4 * (rows + 1) + 4 * xv.shape[0] + 4 * rows
+            bsa.append({"matrix": f"b-{block}_r-{rb}", "nnz": nnz, "us": ms * 1e3, "gnnz_s": nnz / ms / 1e6,
+                        "gb_s": bytes_ / ms / 1e6})
+            del rd, cd, vd, xd, y, ws
+    res.append({"config": "BSA CSR SpMV, blocked sparse attention 65,536 x 65,536 (L2 flushed between launches of the small ones)",
+                "matrices": bsa})
     torch.cuda.empty_cache()
     return res
 

@@ -197,6 +197,89 @@ def csr_matrix(config: int, rows: int, cols: int, s: float = 1.5, cap: int = 10_
 
 
 # --------------------------------------------------------------------------
+# the paper's other SpMV / segmented-sum workloads, as synthetic stand-ins
+# --------------------------------------------------------------------------
+BSA_BLOCKS = (2, 4, 16, 64)          # block sizes of the blocked sparse-attention matrices (Section 5)
+BSA_RANDOM = (2, 4, 8)               # numbers of random attention blocks per block row
+
+
+def block_sparse_attention_csr(block: int, random_blocks: int, dim: int = 65536, global_blocks: int = 2,
+                               window_blocks: int = 3, config: int = 6):
+    """(rowptr int32, col int32, val fp16, x fp32) of a matrix with the blocked sparse-attention
+    pattern ("b-<block>_r-<random_blocks>"): dim x dim in dense blocks of `block` x `block`; block
+    row I holds the first `global_blocks` block columns, the `window_blocks` block columns centred
+    on I (clipped at the edges) and `random_blocks` block columns drawn uniformly (blocks that
+    coincide are kept once); the first `global_blocks` block rows are dense.  Column indices are
+    sorted inside every row.  Values are uniform in [-1, 1), the vector standard normal."""
+    if dim % block:
+        raise ValueError("dim must be a multiple of the block size")
+    nb = dim // block
+    g = min(global_blocks, nb)
+    half = window_blocks // 2
+    rnd = _rng(config, S_LENGTHS, block * 16 + random_blocks).integers(0, nb, size=(nb, random_blocks))
+    ar = np.arange(block, dtype=np.int64)
+    lens = np.empty(dim, np.int64)
+    col_parts = []
+    # the dense block rows
+    lens[:g * block] = dim
+    col_parts.append(np.tile(np.arange(dim, dtype=np.int32), g * block))
+    step = max(1, 4096 // block)                     # block rows per round: bounds the temporaries
+    for i0 in range(g, nb, step):
+        i1 = min(nb, i0 + step)
+        rows_i = np.arange(i0, i1, dtype=np.int64)
+        cand = [np.broadcast_to(np.arange(g, dtype=np.int64), (i1 - i0, g))]
+        cand.append(rows_i[:, None] + np.arange(-half, window_blocks - half, dtype=np.int64)[None, :])
+        cand.append(rnd[i0:i1])
+        c = np.concatenate(cand, axis=1)
+        c = np.where((c >= 0) & (c < nb), c, nb)     # out of range -> sentinel
+        c.sort(axis=1)
+        dup = np.zeros(c.shape, bool)
+        dup[:, 1:] = c[:, 1:] == c[:, :-1]
+        valid = (c < nb) & ~dup                      # [block rows, candidates], ascending block columns
+        k = valid.sum(axis=1)
+        lens[i0 * block:i1 * block] = np.repeat(k * block, block)
+        full = c[:, None, :, None] * block + ar[None, None, None, :]           # [I, row in block, candidate, column in block]
+        full = np.broadcast_to(full, (i1 - i0, block, c.shape[1], block))
+        mask = np.broadcast_to(valid[:, None, :, None], full.shape)
+        col_parts.append(full[mask].astype(np.int32))
+    rowptr = offsets_from_lengths(lens)
+    col = np.concatenate(col_parts)
+    nnz = int(rowptr[-1])
+    assert col.shape[0] == nnz
+    val = f16_uniform(config, nnz)
+    x = _rng(config, S_XVEC, 0).standard_normal(dim, dtype=np.float32)
+    return rowptr, col, val, x
+
+
+# Row-length mixes with the minimum / average / maximum of the sparse matrices whose rows the
+# paper takes its segment lengths from (Table 5.1): constant 2K; 18 / 119 / 204; 1 / 6 / 44;
+# 1 / 6 / 395K (a few huge rows among very short ones).
+ROW_LENGTH_MIXES = ("const2k", "mid", "short", "heavy")
+
+
+def row_length_mix(kind: str, rows: int, config: int = 7) -> np.ndarray:
+    rng = _rng(config, S_LENGTHS, ROW_LENGTH_MIXES.index(kind))
+    if kind == "const2k":
+        return np.full(rows, 2000, np.int64)
+    if kind == "mid":
+        return 18 + np.rint(186.0 * rng.beta(1.63, 1.37, size=rows)).astype(np.int64)      # 18..204, mean 119
+    lens = np.minimum(rng.geometric(1.0 / 6.0, size=rows), 44).astype(np.int64)          # 1..44, mean just under 6
+    if kind == "heavy":
+        lens = np.minimum(rng.geometric(1.0 / 5.4, size=rows), 44).astype(np.int64)
+        giants = rng.choice(rows, size=rows // 683_000 + 1, replace=False)
+        lens[giants] = 395_000
+    return lens
+
+
+def seg_sum_row_mix(kind: str, n_target: int, config: int = 7):
+    """(x fp16 N(0,1), offsets int32) with about n_target elements in rows drawn from the mix."""
+    mean = {"const2k": 2000.0, "mid": 119.0, "short": 5.9, "heavy": 6.0}[kind]
+    rows = max(1, int(n_target / mean))
+    off = offsets_from_lengths(row_length_mix(kind, rows, config))
+    return f16_normal(config, int(off[-1])), off
+
+
+# --------------------------------------------------------------------------
 # the five benchmark configurations (sizes can be scaled down for tests)
 # --------------------------------------------------------------------------
 C5_CASES = (

@@ -248,15 +248,17 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                     if (prm.flags) tma_load_1d(fs, prm.flags + tbase, Cfg::kFlagBytes, &bar_full[stage]);
                 }
             } else {
-                // ragged last tile: plain loads, zero fill past n (MATMUL zero-pads its operand)
+                // ragged last tile: 16-byte asynchronous copies, zero fill past n (MATMUL zero-pads its operand)
                 const long long cnt = prm.n - tbase;
 #pragma unroll 1
                 for (int v = lane; v < (prm.flags ? SCAN_TILE / 16 : 0); v += 32) {
                     const int e0 = v * 16;
-                    uint4 fv = make_uint4(0u, 0u, 0u, 0u);
                     if (e0 + 16 <= cnt) {
-                        fv = *reinterpret_cast<const uint4*>(prm.flags + tbase + e0);
-                    } else if (e0 < cnt) {
+                        cp_async_16(fs + e0, prm.flags + tbase + e0);
+                        continue;
+                    }
+                    uint4 fv = make_uint4(0u, 0u, 0u, 0u);
+                    if (e0 < cnt) {
                         __align__(16) uint8_t tmp[16];
 #pragma unroll 1
                         for (int e = 0; e < 16; ++e) tmp[e] = (e0 + e < cnt) ? prm.flags[tbase + e0 + e] : uint8_t(0);
@@ -269,20 +271,23 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 #pragma unroll 1
                 for (int v = lane; v < SCAN_TILE / kElemPerVec; v += 32) {
                     const int e0 = v * kElemPerVec;
-                    uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+                    const int w = e0 / SCAN_UNIT, i = (e0 % SCAN_UNIT) / PIECE, l = (e0 % PIECE) / ROW, j0 = e0 % ROW;
+                    uint8_t* dst = xs + i * P::kSlabBytes + swz_offset<P::kRowBytes>(w * PIECE_ROWS + l, j0 * P::kElemBytes);
                     if (e0 + kElemPerVec <= cnt) {
-                        xv = *reinterpret_cast<const uint4*>(xt + static_cast<size_t>(e0) * P::kElemBytes);
-                    } else if (e0 < cnt) {
+                        cp_async_16(dst, xt + static_cast<size_t>(e0) * P::kElemBytes);
+                        continue;
+                    }
+                    uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+                    if (e0 < cnt) {
                         __align__(16) uint8_t tmp[16];
 #pragma unroll 1
                         for (int b = 0; b < 16; ++b)
                             tmp[b] = (e0 + b / P::kElemBytes < cnt) ? xt[static_cast<size_t>(e0) * P::kElemBytes + b] : uint8_t(0);
                         xv = *reinterpret_cast<const uint4*>(tmp);
                     }
-                    const int w = e0 / SCAN_UNIT, i = (e0 % SCAN_UNIT) / PIECE, l = (e0 % PIECE) / ROW, j0 = e0 % ROW;
-                    *reinterpret_cast<uint4*>(xs + i * P::kSlabBytes +
-                                              swz_offset<P::kRowBytes>(w * PIECE_ROWS + l, j0 * P::kElemBytes)) = xv;
+                    *reinterpret_cast<uint4*>(dst) = xv;
                 }
+                cp_async_wait_all();
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar_full[stage]);

@@ -447,25 +447,28 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                         tma_load_4d(xs + i * P::kSlabBytes, &tmap_x, &bar_full[stage], 0, 0, i, tile * SPANS_PER_TILE);
                 }
             } else {
-                // ragged last tile: plain loads with zero fill past n (MATMUL zero-pads its operand)
+                // ragged last tile: 16-byte asynchronous copies with zero fill past n (MATMUL zero-pads its operand)
                 const long long cnt = prm.n - tbase;
                 constexpr int kElemPerVec = 16 / P::kElemBytes;
                 const uint8_t* xt = static_cast<const uint8_t*>(xg) + tbase * P::kElemBytes;
                 for (int v = lane; v < TILE / kElemPerVec; v += 32) {
                     const int e0 = v * kElemPerVec;
-                    uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+                    const int w = e0 / SPAN, i = (e0 % SPAN) / PIECE, l = (e0 % PIECE) / ROW, j0 = e0 % ROW;
+                    uint8_t* dst = xs + i * P::kSlabBytes + swz_offset<P::kRowBytes>(w * PIECE_ROWS + l, j0 * P::kElemBytes);
                     if (e0 + kElemPerVec <= cnt) {
-                        xv = *reinterpret_cast<const uint4*>(xt + static_cast<size_t>(e0) * P::kElemBytes);
-                    } else if (e0 < cnt) {
+                        cp_async_16(dst, xt + static_cast<size_t>(e0) * P::kElemBytes);
+                        continue;
+                    }
+                    uint4 xv = make_uint4(0u, 0u, 0u, 0u);
+                    if (e0 < cnt) {
                         __align__(16) uint8_t tmp[16];
                         for (int b = 0; b < 16; ++b)
                             tmp[b] = (e0 + b / P::kElemBytes < cnt) ? xt[static_cast<size_t>(e0) * P::kElemBytes + b] : uint8_t(0);
                         xv = *reinterpret_cast<const uint4*>(tmp);
                     }
-                    const int w = e0 / SPAN, i = (e0 % SPAN) / PIECE, l = (e0 % PIECE) / ROW, j0 = e0 % ROW;
-                    *reinterpret_cast<uint4*>(xs + i * P::kSlabBytes +
-                                              swz_offset<P::kRowBytes>(w * PIECE_ROWS + l, j0 * P::kElemBytes)) = xv;
+                    *reinterpret_cast<uint4*>(dst) = xv;
                 }
+                cp_async_wait_all();
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&bar_full[stage]);

@@ -132,6 +132,32 @@ def test_config4_full_size(mmv, empty_fraction):
         assert (y.cpu().numpy()[lens == 0] == 0).all()
 
 
+def test_block_sparse_attention_full_size(mmv):
+    # the largest of the blocked sparse-attention matrices at the paper's size: 65,536 rows, b-64_r-8
+    rowptr, col, val, xv = gen.block_sparse_attention_csr(64, 8)
+    rows, nnz = rowptr.shape[0] - 1, val.shape[0]
+    rd, cd, vd, xd = (torch.from_numpy(t).cuda() for t in (rowptr, col, val, xv))
+    ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, nnz, rows)
+    y = mmv.spmv_csr(rd, cd, vd, xd, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    want, a = oracle.spmv_csr(rowptr, col, val, xv)
+    ok, ratio, i = oracle.check_fp(y.cpu().numpy(), want, a)
+    assert ok, f"b-64_r-8: |err|/bound = {ratio:.3g} at row {i}"
+
+
+@pytest.mark.parametrize("kind", gen.ROW_LENGTH_MIXES)
+def test_row_length_mixes_at_bench_size(mmv, kind):
+    x, off = gen.seg_sum_row_mix(kind, 1 << 26)
+    nseg = off.shape[0] - 1
+    xd, od = torch.from_numpy(x).cuda(), torch.from_numpy(off).cuda()
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, x.shape[0], nseg)
+    got = mmv.seg_sum(xd, od, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    want, a = oracle.seg_sum_csr_f16(x, off)
+    ok, ratio, i = oracle.check_fp(got.cpu().numpy(), want, a)
+    assert ok, f"{kind}: |err|/bound = {ratio:.3g} at segment {i}"
+
+
 def test_scan_beyond_2_to_the_32_elements_closed_form(mmv):
     """Index arithmetic past 2^32 elements: all-ones int8 values with a start flag every 1000 elements
     (one period is not a divisor of the tile size, so the flags drift through every position of a

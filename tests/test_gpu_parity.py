@@ -464,6 +464,25 @@ def test_spmv_golden_and_random(mmv):
         assert (got[np.diff(rowptr) == 0] == 0).all()
 
 
+@pytest.mark.parametrize("block", gen.BSA_BLOCKS)
+@pytest.mark.parametrize("random_blocks", gen.BSA_RANDOM)
+def test_spmv_block_sparse_attention(mmv, block, random_blocks):
+    # the blocked sparse-attention matrices of Section 5 (global, window and random blocks), reduced to 8192 rows
+    rowptr, col, val, x = gen.block_sparse_attention_csr(block, random_blocks, dim=8192)
+    want, a = oracle.spmv_csr(rowptr, col, val, x)
+    assert_fp(spmv(mmv, rowptr, col, val, x), want, a, f"b-{block}_r-{random_blocks}")
+
+
+@pytest.mark.parametrize("kind", gen.ROW_LENGTH_MIXES)
+def test_seg_sum_row_length_mixes(mmv, kind):
+    # segment lengths with the minimum / average / maximum of the matrices of Table 5.1
+    x, off = gen.seg_sum_row_mix(kind, 3 << 20)
+    want, a = oracle.seg_sum_csr_f16(x, off)
+    assert_fp(sum_csr(mmv, x, off), want, a, kind)
+    xi = gen.i8_uniform(7, x.shape[0])
+    assert np.array_equal(sum_csr(mmv, xi, off), oracle.seg_sum_csr_i8(xi, off))
+
+
 # ---------------------------------------------------------------------------
 # robustness
 # ---------------------------------------------------------------------------
