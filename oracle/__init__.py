@@ -129,6 +129,28 @@ def new_i8_state():
     return {"v": np.zeros(1, np.int64), "open": False}
 
 
+def seg_scan_excl_f16(x, f):
+    """Segmented exclusive scan on fp16 values: e(i) = sum of the elements of i's segment in front
+    of i (0 at a segment start); returns (e, a) in float64, a = the same sum over |x|."""
+    xb, fb = _as_f16_bits(x), _as(f, np.uint8)
+    n = xb.shape[0]
+    assert fb.shape[0] == n
+    e = np.empty(n, np.float64)
+    a = np.empty(n, np.float64)
+    _load().mmv_oracle_seg_scan_excl_f16(_p(xb), _p(fb), ctypes.c_int64(n), _p(e), _p(a))
+    return e, a
+
+
+def seg_scan_excl_i8(x, f):
+    """Segmented exclusive scan on int8 values, int32 result (low 32 bits of the exact sum)."""
+    xb, fb = _as(x, np.int8), _as(f, np.uint8)
+    n = xb.shape[0]
+    assert fb.shape[0] == n
+    e = np.empty(n, np.int32)
+    _load().mmv_oracle_seg_scan_excl_i8(_p(xb), _p(fb), ctypes.c_int64(n), _p(e))
+    return e
+
+
 def flags_from_offsets(off, n):
     """f(i) = 1 iff i starts a non-empty segment of the CSR offsets ``off``."""
     off = _as(off, np.int32)

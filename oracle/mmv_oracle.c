@@ -108,6 +108,35 @@ void mmv_oracle_seg_scan_i8(const int8_t *x, const uint8_t *f, int64_t n,
 }
 
 /*
+ * Segmented EXCLUSIVE scan: e(i) = 0 if i = 0 or f(i) != 0, else z(i-1) with z the
+ * scan of Eq. (1); that is, the sum of the elements of i's segment in front of
+ * i.  a[i] is the sum of |x| over the same elements.  (The paper states the
+ * inclusive problem only; this is the usual companion definition.)
+ */
+void mmv_oracle_seg_scan_excl_f16(const uint16_t *x, const uint8_t *f, int64_t n, double *e, double *a)
+{
+    double run = 0.0, arun = 0.0;       /* sum of the open segment so far */
+    for (int64_t i = 0; i < n; ++i) {
+        double xi = half_bits_to_double(x[i]);
+        if (i == 0 || f[i] != 0) { run = 0.0; arun = 0.0; }
+        e[i] = run;
+        if (a) a[i] = arun;
+        run = run + xi;
+        arun = arun + fabs(xi);
+    }
+}
+
+void mmv_oracle_seg_scan_excl_i8(const int8_t *x, const uint8_t *f, int64_t n, int32_t *e)
+{
+    int64_t run = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (i == 0 || f[i] != 0) run = 0;
+        e[i] = (int32_t)(uint32_t)(uint64_t)run;     /* low 32 bits */
+        run = run + (int64_t)x[i];
+    }
+}
+
+/*
  * Start flags from CSR offsets: f(i) = 1 iff i is the start index off[r] of a
  * non-empty segment r.  Returns 0, or -1 if the offsets are not a
  * non-decreasing sequence from 0 to n.

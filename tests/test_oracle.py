@@ -421,3 +421,60 @@ def test_fp_bound_helper():
     assert ok and ratio <= 1.0
     ok, ratio, i = oracle.check_fp(np.asarray([1.0, 2e-6], np.float64), z, a)
     assert not ok and i == 1
+
+
+# --------------------------------------------------------------------------
+# exclusive variant: e(i) = sum of the elements of i's segment in front of i
+# --------------------------------------------------------------------------
+def brute_excl(x, f):
+    out = []
+    for i in range(len(x)):
+        s = i
+        while s > 0 and not f[s]:
+            s -= 1
+        out.append(sum(x[s:i], type(x[0])(0)))
+    return out
+
+
+def test_exclusive_scan_of_the_worked_example_and_exhaustively():
+    g = load_golden("sec2_worked_example.txt")
+    x, f = g["x"], g["f"]
+    # inclusive (2,4,3,6,7,3,4,6) shifted inside each segment: (0,2,0,3,6,0,3,4)
+    want = [z - xi for z, xi in zip(g["seg_scan"], x)]
+    assert want == [0, 2, 0, 3, 6, 0, 3, 4]
+    e, a = oracle.seg_scan_excl_f16(f16(x), u8(f))
+    assert e.tolist() == want and a.tolist() == want
+    assert oracle.seg_scan_excl_i8(np.asarray(x, np.int8), u8(f)).tolist() == want
+    rng = np.random.default_rng(17)
+    for n in range(1, 10):
+        x = rng.integers(-9, 10, n).tolist()
+        for bits in itertools.product([0, 1], repeat=n):
+            assert oracle.seg_scan_excl_i8(np.asarray(x, np.int8), u8(bits)).tolist() == brute_excl(x, bits), (x, bits)
+            assert oracle.seg_scan_excl_f16(f16(x), u8(bits))[0].tolist() == brute_excl(x, bits)
+
+
+def test_exclusive_scan_random_and_identities():
+    rng = np.random.default_rng(19)
+    for trial in range(60):
+        n = int(rng.integers(1, 80))
+        f = (rng.random(n) < rng.choice([0.03, 0.3, 0.8])).astype(np.uint8)
+        x = rng.standard_normal(n).astype(np.float16)
+        xq = [Fraction(float(v)) for v in x]
+        e, a = oracle.seg_scan_excl_f16(x, f)
+        want, want_a = brute_excl(xq, f.tolist()), brute_excl([abs(v) for v in xq], f.tolist())
+        for i in range(n):
+            assert abs(Fraction(float(e[i])) - want[i]) <= Fraction(1, 10 ** 12)
+            assert abs(Fraction(float(a[i])) - want_a[i]) <= Fraction(1, 10 ** 12)
+        xi = rng.integers(-128, 128, n).astype(np.int8)
+        ei = oracle.seg_scan_excl_i8(xi, f)
+        assert ei.tolist() == brute_excl(xi.astype(int).tolist(), f.tolist())
+        # exclusive + element = inclusive (exact in integers)
+        assert np.array_equal(ei.astype(np.int64) + xi, oracle.seg_scan_i8(xi, f).astype(np.int64))
+    # wrap-around: 2^25 elements of 127 pass 2^31
+    n = 1 << 25
+    e = oracle.seg_scan_excl_i8(np.full(n, 127, np.int8), np.zeros(n, np.uint8))
+    for i in (0, 1, (1 << 24) + 5, n - 1):
+        assert int(e[i]) == wrap32(127 * i)
+    # all flags: zero everywhere; no flags: prefix sums shifted by one
+    assert not oracle.seg_scan_excl_i8(np.full(100, 5, np.int8), np.ones(100, np.uint8)).any()
+    assert oracle.seg_scan_excl_f16(np.ones(50, np.float16), np.zeros(50, np.uint8))[0].tolist() == list(range(50))
