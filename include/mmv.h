@@ -217,9 +217,9 @@ void mmv_debug_configure(int64_t wait_budget_ns, int64_t skip_publish_span);
 
 /*
  * Test hook.  The segmented-sum kernel exists with two and with three epilogue
- * warpgroups; the library picks one from the average segment length.  groups =
- * 2 or 3 forces that variant for the offsets form and SpMV, 0 restores the
- * automatic choice.
+ * warpgroups; the library launches the one with three.  groups = 2 makes every
+ * later segmented sum and SpMV use the variant with two, 3 or 0 restore the
+ * default.
  */
 void mmv_debug_force_sum_groups(int groups);
 
