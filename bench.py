@@ -573,6 +573,18 @@ def run_ours(args):
             sweep.append({"case": "no flag vector (plain scan, 6 B/elem)", "ms": cms, "gelem_s": n / cms / 1e6,
                           "gb_s": 6 * n / cms / 1e6, "frac_of_measured_peak": 6 * n / cms / 1e6 / peak,
                           "frac_of_8tbs": 6 * n / cms / 1e6 / NOMINAL_HBM_GBS})
+            # the exclusive variant on the headline flags (same traffic)
+            fd = torch.from_numpy(f).cuda()
+            fn = lambda: mmv.seg_scan(xd, fd, out=od, workspace=ws, exclusive=True)  # noqa: E731
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            cms = event_time_ms(torch, fn, min(args.steps, 10))
+            assert mmv.last_async_status(ws) == 0
+            sweep.append({"case": f"exclusive scan, {args.case}", "ms": cms, "gelem_s": n / cms / 1e6,
+                          "gb_s": 7 * n / cms / 1e6, "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
+                          "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
+            del fd
             line["configs"] = cfgs
             line["c5_density_sweep"] = sweep
         print(json.dumps(line))

@@ -99,6 +99,18 @@ mmv_status mmv_seg_scan(const void *x, const void *seg, mmv_segfmt sf, int64_t n
                         void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Segmented EXCLUSIVE scan, the companion of Eq. 1: every element receives the
+ * sum of the elements of its segment in front of it,
+ *     out[i] = 0                      if i == 0 or i starts a segment
+ *     out[i] = out[i-1] + x[i-1]      otherwise
+ * (the inclusive result moved one element to the right inside each segment).
+ * Same arguments, layouts, workspace, ownership and errors as mmv_seg_scan.
+ */
+mmv_status mmv_seg_scan_exclusive(const void *x, const void *seg, mmv_segfmt sf, int64_t n, int64_t nseg,
+                                  mmv_dtype dt, void *out,
+                                  void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Segmented sum (Section 2: the last element of every segment of the
  * segmented scan; Algorithm 4.2 computes the same quantity).
  * Offsets form: out has nseg entries, out[r] = sum of x over [off[r], off[r+1]),

@@ -26,7 +26,7 @@ EXPORTS = (
     "mmv_workspace_bytes", "mmv_seg_scan", "mmv_seg_sum", "mmv_spmv_csr",
     "mmv_last_async_status", "mmv_status_string", "mmv_kernel_launch_count", "mmv_debug_configure",
     "mmv_seg_scan_static", "mmv_seg_scan_static_last_status", "mmv_debug_force_sum_groups",
-    "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes",
+    "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes", "mmv_seg_scan_exclusive",
 )
 STATIC_SCAN_MAX_N = 1 << 28
 
@@ -48,6 +48,8 @@ def _load() -> ctypes.CDLL:
     lib.mmv_workspace_bytes.argtypes = [ci, ci, ci, i64, i64]
     lib.mmv_seg_scan.restype = ci
     lib.mmv_seg_scan.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, sz, vp]
+    lib.mmv_seg_scan_exclusive.restype = ci
+    lib.mmv_seg_scan_exclusive.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, sz, vp]
     lib.mmv_seg_sum.restype = ci
     lib.mmv_seg_sum.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, vp, sz, vp]
     lib.mmv_spmv_csr.restype = ci
@@ -137,9 +139,10 @@ def last_async_status(workspace: torch.Tensor, stream=None) -> int:
 
 
 def seg_scan(x: torch.Tensor, seg: torch.Tensor | None, out: torch.Tensor | None = None,
-             workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+             workspace: torch.Tensor | None = None, stream=None, exclusive: bool = False) -> torch.Tensor:
     """mmv_seg_scan: segmented inclusive scan (Problem 2.1, Eq. 1) of x over seg; seg = None is the
-    plain inclusive scan (one segment, no flag vector is read)."""
+    plain inclusive scan (one segment, no flag vector is read).  exclusive=True calls
+    mmv_seg_scan_exclusive: each element gets the sum of its segment's elements in front of it."""
     _check_cuda(x, seg, out, workspace)
     dt, sf = _dtype_code(x), (SEG_FLAGS_U8 if seg is None else _seg_code(seg))
     n = x.numel()
@@ -148,10 +151,10 @@ def seg_scan(x: torch.Tensor, seg: torch.Tensor | None, out: torch.Tensor | None
         out = torch.empty(n, dtype=torch.float32 if dt == F16_TO_F32 else torch.int32, device=x.device)
     if workspace is None:
         workspace = alloc_workspace(OP_SEG_SCAN, dt, sf, n, nseg, x.device)
-    rc = _lib.mmv_seg_scan(_ptr(x), _ptr(seg), sf, n, nseg, dt, _ptr(out), _ptr(workspace),
-                           workspace.numel(), _stream_ptr(stream))
+    call = _lib.mmv_seg_scan_exclusive if exclusive else _lib.mmv_seg_scan
+    rc = call(_ptr(x), _ptr(seg), sf, n, nseg, dt, _ptr(out), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     if rc != MMV_OK:
-        raise MmvError(rc, "mmv_seg_scan")
+        raise MmvError(rc, "mmv_seg_scan_exclusive" if exclusive else "mmv_seg_scan")
     return out
 
 

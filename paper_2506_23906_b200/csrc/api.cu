@@ -72,6 +72,8 @@ DeviceInfo* device_info() {
         bool ok = true;
         ok &= set_smem(seg_scan_kernel<F16Path>, ScanCfg<F16Path>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<I8Path>, ScanCfg<I8Path>::kSmemBytes);
+        ok &= set_smem(seg_scan_kernel<F16Path, true>, ScanCfg<F16Path>::kSmemBytes);
+        ok &= set_smem(seg_scan_kernel<I8Path, true>, ScanCfg<I8Path>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<F16Path, 2>, SumCfg<F16Path, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<I8Path, 2>, SumCfg<I8Path, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<BF16Path, 2>, SumCfg<BF16Path, 2>::kSmemBytes);
@@ -306,8 +308,9 @@ size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, in
     return plan_workspace(op, sf, n).total;
 }
 
-mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
-                        void* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+namespace {
+mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
+                         void* out, void* workspace, size_t workspace_bytes, void* cuda_stream, bool exclusive) {
     if (n < 0 || nseg < 0) return MMV_ERR_INVALID_ARG;
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
@@ -359,12 +362,27 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
     prm.debug_skip_span = g_debug_skip_span.load();
     prm.carry_in = nullptr;
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
-    if (f16)
+    if (f16 && !exclusive)
         seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
-    else
+    else if (!exclusive)
         seg_scan_kernel<I8Path><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+    else if (f16)
+        seg_scan_kernel<F16Path, true><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+    else
+        seg_scan_kernel<I8Path, true><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+}
+}  // namespace
+
+mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
+                        void* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return seg_scan_impl(x, seg, sf, n, nseg, dt, out, workspace, workspace_bytes, cuda_stream, false);
+}
+
+mmv_status mmv_seg_scan_exclusive(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
+                                  void* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return seg_scan_impl(x, seg, sf, n, nseg, dt, out, workspace, workspace_bytes, cuda_stream, true);
 }
 
 // ---------------------------------------------------------------------------

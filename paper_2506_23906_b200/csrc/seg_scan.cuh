@@ -128,7 +128,11 @@ __device__ __forceinline__ bool wait_stage(const volatile int* stage_iter, int i
     return wait_bar(bar, parity, abort_flag, budget_ns);
 }
 
-template <typename P>
+// EX = true gives the exclusive variant: every element receives the sum of the elements of its
+// segment in FRONT of it (0 at a segment start), i.e. the inclusive result moved one element to
+// the right inside each segment.  The shift happens in registers just before a piece is staged for
+// its store; everything else is the same kernel.
+template <typename P, bool EX = false>
 __global__ void __launch_bounds__(ScanCfg<P>::kThreads, 1)
 seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_out,
                  const ScanParams prm) {
@@ -359,7 +363,16 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 
         MMV_T_DECL
         // stages the 32 x 32 block held in r (lane = row) and stores it with one TMA store
-        auto store_piece = [&](const uint32_t (&r)[32], long long prow) {
+        // (exclusive variant: `fmask` = start flags of this lane's row, `prev_last` = inclusive value of the
+        //  element in front of the piece)
+        auto store_piece = [&](uint32_t (&r)[32], long long prow, uint32_t fmask, Acc prev_last) {
+            if constexpr (EX) {
+                uint32_t up = __shfl_up_sync(0xffffffffu, r[31], 1);
+                if (lane == 0) up = P::to_bits(prev_last);
+#pragma unroll
+                for (int j = 31; j >= 1; --j) r[j] = ((fmask >> j) & 1u) ? 0u : r[j - 1];
+                r[0] = (fmask & 1u) ? 0u : up;
+            }
             uint8_t* ob = stg + obuf * Cfg::kOutBufBytes;
             if (lane == 0) tma_store_wait_read<Cfg::kOutBufs - 1>();   // the buffer about to be reused is free again
             __syncwarp();
@@ -504,6 +517,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             // ---- main pass: everything that does not need the carry of earlier units ----
             const long long row0 = s * (SCAN_UNIT / ROW);
             Acc run = Acc(0);                 // sum of the open segment inside this unit so far
+            Acc last_incl = Acc(0);           // exclusive variant: inclusive value of the last element of the piece before
             uint32_t fm0 = 0u, pm0 = 0u;      // masks of the first flagged piece
             LookbackWindow<SCAN_LB_WORDS> lbw;
             // (not unrolled: the body is large and the instruction cache is the scarcer resource)
@@ -585,11 +599,14 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                         if (j < f0) r[j] = P::to_bits(P::add(carry_row, P::from_bits(r[j])));
                 }
                 MMV_T_MARK(5)
+                Acc last_i = Acc(0);
+                if constexpr (EX) last_i = P::from_bits(__shfl_sync(0xffffffffu, r[31], 31));
                 if (i > i0) {
-                    store_piece(r, row0 + i * PIECE_ROWS);       // complete: no element reaches back past a flag
+                    store_piece(r, row0 + i * PIECE_ROWS, fmi, last_incl);       // complete: no element reaches back past a flag
                 } else {
                     tmem_st_32x32(taddr + i * N, r);             // parked until the carry is known
                 }
+                last_incl = last_i;            // (of piece i0 it is final already: its last element lies behind the flag)
                 MMV_T_MARK(4)
             }
             tmem_st_wait();
@@ -630,6 +647,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             // ---- parked pieces: add the carry in front of the unit's first flag, store ----
             const int l0 = pm0 ? (__ffs(pm0) - 1) : 32;                       // first flagged row of piece i0
             const int fpos = __ffs(__shfl_sync(0xffffffffu, fm0, l0 & 31)) - 1;  // its first flag
+            Acc prev_parked = carry;           // exclusive variant: what stands in front of the unit's first element
 #pragma unroll 1
             for (int i = 0; i <= i0 && i < UP; ++i) {
                 uint32_t r[32];
@@ -640,7 +658,10 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
                     if (j < limit) r[j] = P::to_bits(P::add(carry, P::from_bits(r[j])));
-                store_piece(r, row0 + i * PIECE_ROWS);
+                Acc last_p = Acc(0);
+                if constexpr (EX) last_p = P::from_bits(__shfl_sync(0xffffffffu, r[31], 31));
+                store_piece(r, row0 + i * PIECE_ROWS, i == i0 ? fm0 : 0u, prev_parked);
+                prev_parked = last_p;
             }
             MMV_T_MARK(7)
 

@@ -188,3 +188,27 @@ def test_scan_beyond_2_to_the_32_elements_closed_form(mmv):
         want = (idx & 0xffffffff).to(torch.int64)
         want = torch.where(want >= (1 << 31), want - (1 << 32), want).to(torch.int32)     # wrap-around modulo 2^32
         assert torch.equal(out[o:e], want), f"plain scan wrong in [{o}, {e})"
+
+
+def test_exclusive_scan_full_size(mmv, c5_values):
+    # the exclusive variant at the headline size: exclusive + element = inclusive, checked piecewise against the
+    # oracle's inclusive scan streamed over the array
+    n = 1 << 30
+    f = gen.config5_flags(n, "p1e-3")
+    xd, fd = torch.from_numpy(c5_values).cuda(), torch.from_numpy(f).cuda()
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+    out = mmv.seg_scan(xd, fd, workspace=ws, exclusive=True)
+    assert mmv.last_async_status(ws) == 0
+    state = oracle.new_f16_state()
+    worst = 0.0
+    for lo in range(0, n, STEP):
+        hi = min(n, lo + STEP)
+        z, a = oracle.seg_scan_f16(c5_values[lo:hi], f[lo:hi], state)
+        xs = c5_values[lo:hi].astype(np.float64)
+        want = z - xs                                           # exact in fp64 for these magnitudes
+        bound = oracle.fp_bound(np.maximum(a - np.abs(xs), 0.0))       # sum of |x| over the elements in front
+        got = out[lo:hi].cpu().numpy().astype(np.float64)
+        worst = max(worst, float(np.max(np.abs(got - want) / bound)))
+        starts = f[lo:hi] != 0
+        assert (got[starts] == 0.0).all()
+    assert worst <= 1.0, f"exclusive scan: |err|/bound = {worst}"

@@ -29,25 +29,25 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def scan_i8(mmv, x, f, guard=64):
+def scan_i8(mmv, x, f, guard=64, exclusive=False):
     n = x.shape[0]
     seg = dev(f)
     sf = mmv.SEG_FLAGS_U8 if f.dtype == np.uint8 else mmv.SEG_OFFSETS_I32
     ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, sf, n, max(0, f.shape[0] - 1))
     buf = torch.full((n + guard,), -777, dtype=torch.int32, device="cuda")
-    mmv.seg_scan(dev(x), seg, out=buf[:n], workspace=ws)
+    mmv.seg_scan(dev(x), seg, out=buf[:n], workspace=ws, exclusive=exclusive)
     assert mmv.last_async_status(ws) == 0
     got = buf.cpu().numpy()
     assert (got[n:] == -777).all(), "wrote past the end of the output"
     return got[:n]
 
 
-def scan_f16(mmv, x, f, guard=64):
+def scan_f16(mmv, x, f, guard=64, exclusive=False):
     n = x.shape[0]
     sf = mmv.SEG_FLAGS_U8 if f.dtype == np.uint8 else mmv.SEG_OFFSETS_I32
     ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.F16_TO_F32, sf, n, max(0, f.shape[0] - 1))
     buf = torch.full((n + guard,), -777.0, dtype=torch.float32, device="cuda")
-    mmv.seg_scan(dev(x), dev(f), out=buf[:n], workspace=ws)
+    mmv.seg_scan(dev(x), dev(f), out=buf[:n], workspace=ws, exclusive=exclusive)
     assert mmv.last_async_status(ws) == 0
     got = buf.cpu().numpy()
     assert (got[n:] == -777.0).all(), "wrote past the end of the output"
@@ -481,6 +481,43 @@ def test_seg_sum_row_length_mixes(mmv, kind):
     assert_fp(sum_csr(mmv, x, off), want, a, kind)
     xi = gen.i8_uniform(7, x.shape[0])
     assert np.array_equal(sum_csr(mmv, xi, off), oracle.seg_sum_csr_i8(xi, off))
+
+
+# ---------------------------------------------------------------------------
+# exclusive variant of the scan
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("n", [1, 31, 32, 33, 1023, 1025, 4096, TILE - 1, TILE, TILE + 1, 3 * TILE + 4097, 11 * TILE + 777])
+@pytest.mark.parametrize("p", [0.0, 1e-3, 0.05, 0.5, 1.0])
+def test_exclusive_scan(mmv, n, p):
+    rng = np.random.default_rng(n * 7 + int(p * 1000))
+    f = (rng.random(n) < p).astype(np.uint8)
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    assert np.array_equal(scan_i8(mmv, xi, f, exclusive=True), oracle.seg_scan_excl_i8(xi, f))
+    xf = rng.standard_normal(n).astype(np.float16)
+    want, a = oracle.seg_scan_excl_f16(xf, f)
+    got = scan_f16(mmv, xf, f, exclusive=True)
+    assert_fp(got, want, a, f"exclusive scan n={n} p={p}")
+    assert got[0] == 0.0 and (got[f != 0] == 0.0).all()        # exactly zero at every segment start
+
+
+def test_exclusive_scan_flags_on_edges_offsets_and_plain(mmv):
+    n = 5 * TILE + 100
+    rng = np.random.default_rng(3)
+    f = np.zeros(n, np.uint8)
+    f[[31, 32, 33, 1023, 1024, 4095, 4096, 4097, TILE - 1, TILE, TILE + 1, 2 * TILE + 4096, 4 * TILE, n - 1]] = 1
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    assert np.array_equal(scan_i8(mmv, xi, f, exclusive=True), oracle.seg_scan_excl_i8(xi, f))
+    xf = gen.f16_uniform(1, n)
+    want, a = oracle.seg_scan_excl_f16(xf, f)
+    assert_fp(scan_f16(mmv, xf, f, exclusive=True), want, a, "exclusive, flags on edges")
+    # the same segments as offsets (with empty segments in between)
+    off = np.asarray([0, 0, 31, 32, 33, 33, 1023, 1024, 4095, 4096, 4097, TILE - 1, TILE, TILE + 1, 2 * TILE + 4096,
+                      4 * TILE, n - 1, n, n], np.int32)
+    assert np.array_equal(scan_i8(mmv, xi, off, exclusive=True), oracle.seg_scan_excl_i8(xi, f))
+    # no flag vector: the plain exclusive scan
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    got = mmv.seg_scan(dev(xi), None, workspace=ws, exclusive=True).cpu().numpy()
+    assert np.array_equal(got, oracle.seg_scan_excl_i8(xi, np.zeros(n, np.uint8)))
 
 
 # ---------------------------------------------------------------------------
