@@ -82,6 +82,18 @@ def f16_normal(config: int, n: int, stream: int = S_VALUES) -> np.ndarray:
     return _full(f16_normal_chunk, n, np.float16, config, stream=stream)
 
 
+def bf16_bits_of(x32: np.ndarray) -> np.ndarray:
+    """float32 -> bfloat16 bit patterns (uint16), round to nearest even (a data-type conversion,
+    like the rounding to fp16 above; numpy has no bfloat16 type)."""
+    u = np.ascontiguousarray(x32, np.float32).view(np.uint32)
+    return ((u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
+
+
+def bf16_normal(config: int, n: int, stream: int = S_VALUES) -> np.ndarray:
+    """Standard normal values as bfloat16 bit patterns (uint16)."""
+    return bf16_bits_of(f16_normal(config, n, stream).astype(np.float32) * np.float32(1.0009765625))
+
+
 def i8_uniform(config: int, n: int, lo: int = -8, hi: int = 7) -> np.ndarray:
     return _full(i8_uniform_chunk, n, np.int8, config, lo=lo, hi=hi)
 

@@ -141,6 +141,44 @@ def seg_scan_excl_f16(x, f):
     return e, a
 
 
+def bf16_to_double(bits) -> np.ndarray:
+    """Exact decode of bfloat16 bit patterns (uint16) to float64."""
+    hb = _as(bits, np.uint16)
+    out = np.empty(hb.shape[0], np.float64)
+    _load().mmv_oracle_decode_bf16(_p(hb), ctypes.c_int64(hb.shape[0]), _p(out))
+    return out
+
+
+def seg_scan_bf16(xbits, f, exclusive: bool = False):
+    """Eq. (1) (or its exclusive companion) on bfloat16 values given as uint16 bit patterns: (z, a) in float64."""
+    x, fb = bf16_to_double(xbits), _as(f, np.uint8)
+    n = x.shape[0]
+    assert fb.shape[0] == n
+    z, a = np.empty(n, np.float64), np.empty(n, np.float64)
+    fn = _load().mmv_oracle_seg_scan_excl_f64 if exclusive else _load().mmv_oracle_seg_scan_f64
+    fn(_p(x), _p(fb), ctypes.c_int64(n), _p(z), _p(a))
+    return z, a
+
+
+def seg_sum_csr_bf16(xbits, off):
+    x, off = bf16_to_double(xbits), _as(off, np.int32)
+    _check_offsets(off, x.shape[0])
+    nseg = off.shape[0] - 1
+    out, a = np.empty(nseg, np.float64), np.empty(nseg, np.float64)
+    _load().mmv_oracle_seg_sum_csr_f64(_p(x), _p(off), ctypes.c_int64(nseg), _p(out), _p(a))
+    return out, a
+
+
+def seg_sum_flags_bf16(xbits, f):
+    x, fb = bf16_to_double(xbits), _as(f, np.uint8)
+    n = x.shape[0]
+    out, a = np.empty(max(n, 1), np.float64), np.empty(max(n, 1), np.float64)
+    lib = _load()
+    lib.mmv_oracle_seg_sum_flags_f64.restype = ctypes.c_int64
+    k = lib.mmv_oracle_seg_sum_flags_f64(_p(x), _p(fb), ctypes.c_int64(n), _p(out), _p(a))
+    return out[:k].copy(), a[:k].copy()
+
+
 def seg_scan_excl_i8(x, f):
     """Segmented exclusive scan on int8 values, int32 result (low 32 bits of the exact sum)."""
     xb, fb = _as(x, np.int8), _as(f, np.uint8)

@@ -221,6 +221,85 @@ void mmv_oracle_seg_sum_csr_i8(const int8_t *x, const int32_t *off, int64_t nseg
 }
 
 /* ------------------------------------------------------------------------ */
+/* bfloat16 values: decoded exactly to double, then the same definitions on   */
+/* double inputs (Eq. (1), its exclusive companion, the two segmented sums).  */
+/* ------------------------------------------------------------------------ */
+
+/* Exact decode of a bfloat16 bit pattern (1 sign, 8 exponent, 7 mantissa bits). */
+double mmv_oracle_bf16_to_double(uint16_t h)
+{
+    int sign = (h >> 15) & 1;
+    int e = (h >> 7) & 0xff;
+    int m = h & 0x7f;
+    double v;
+    if (e == 0) {
+        v = ldexp((double)m, -133);             /* zero and subnormals: m * 2^-7 * 2^-126 */
+    } else if (e == 255) {
+        v = m ? NAN : INFINITY;
+    } else {
+        v = ldexp((double)(m + 128), e - 134);  /* (1 + m/128) * 2^(e-127) */
+    }
+    return sign ? -v : v;
+}
+
+void mmv_oracle_decode_bf16(const uint16_t *h, int64_t n, double *out)
+{
+    for (int64_t i = 0; i < n; ++i) out[i] = mmv_oracle_bf16_to_double(h[i]);
+}
+
+void mmv_oracle_seg_scan_f64(const double *x, const uint8_t *f, int64_t n, double *z, double *a)
+{
+    double zp = 0.0, ap = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (i == 0 || f[i] != 0) { zp = x[i]; ap = fabs(x[i]); }
+        else                     { zp = zp + x[i]; ap = ap + fabs(x[i]); }
+        z[i] = zp;
+        if (a) a[i] = ap;
+    }
+}
+
+void mmv_oracle_seg_scan_excl_f64(const double *x, const uint8_t *f, int64_t n, double *e, double *a)
+{
+    double run = 0.0, arun = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (i == 0 || f[i] != 0) { run = 0.0; arun = 0.0; }
+        e[i] = run;
+        if (a) a[i] = arun;
+        run = run + x[i];
+        arun = arun + fabs(x[i]);
+    }
+}
+
+int64_t mmv_oracle_seg_sum_flags_f64(const double *x, const uint8_t *f, int64_t n, double *out, double *a)
+{
+    int64_t k = 0;
+    double zp = 0.0, ap = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (i == 0 || f[i] != 0) { zp = x[i]; ap = fabs(x[i]); }
+        else                     { zp += x[i]; ap += fabs(x[i]); }
+        if (i == n - 1 || f[i + 1] != 0) {
+            out[k] = zp;
+            if (a) a[k] = ap;
+            ++k;
+        }
+    }
+    return k;
+}
+
+void mmv_oracle_seg_sum_csr_f64(const double *x, const int32_t *off, int64_t nseg, double *out, double *a)
+{
+    for (int64_t r = 0; r < nseg; ++r) {
+        double s = 0.0, sa = 0.0;
+        for (int64_t i = off[r]; i < off[r + 1]; ++i) {
+            s += x[i];
+            sa += fabs(x[i]);
+        }
+        out[r] = s;
+        if (a) a[r] = sa;
+    }
+}
+
+/* ------------------------------------------------------------------------ */
 /* CSR SpMV: y(r) = sum_k val(k) * x(col(k)) over the row's entries.          */
 /* val is fp16 (bit patterns), x is fp32; both are decoded exactly to double */
 /* so each product is exact in double; a(r) = sum |val(k) * x(col(k))|.       */

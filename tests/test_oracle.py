@@ -6,6 +6,7 @@ from fractions import Fraction
 import numpy as np
 import pytest
 
+import mmv_inputs as gen
 import oracle
 from conftest import load_golden
 
@@ -478,3 +479,55 @@ def test_exclusive_scan_random_and_identities():
     # all flags: zero everywhere; no flags: prefix sums shifted by one
     assert not oracle.seg_scan_excl_i8(np.full(100, 5, np.int8), np.ones(100, np.uint8)).any()
     assert oracle.seg_scan_excl_f16(np.ones(50, np.float16), np.zeros(50, np.uint8))[0].tolist() == list(range(50))
+
+
+# --------------------------------------------------------------------------
+# bfloat16 inputs: exact decode, then the same definitions on double values
+# --------------------------------------------------------------------------
+def test_bf16_decode_matches_the_float32_bit_pattern_for_every_value():
+    bits = np.arange(65536, dtype=np.uint16)
+    got = oracle.bf16_to_double(bits)
+    want = (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)    # bf16 = top half of fp32
+    finite = np.isfinite(want)
+    assert np.array_equal(got[finite], want[finite])
+    assert np.array_equal(np.isnan(got), np.isnan(want)) and np.array_equal(np.isinf(got), np.isinf(want))
+    assert np.array_equal(np.signbit(got[~np.isnan(want)]), np.signbit(want[~np.isnan(want)]))
+    # rounding of the generator: nearest, ties to even
+    x = np.asarray([1.0, 1.00390625, 1.01171875, -2.5, 3.0e38, 1e-40], np.float32)
+    assert gen.bf16_bits_of(x).tolist() == [0x3F80, 0x3F80, 0x3F82, 0xC020, 0x7F62, 0x0001]
+
+
+def test_bf16_definitions_against_brute_force_and_the_fp16_functions():
+    rng = np.random.default_rng(23)
+    for trial in range(40):
+        n = int(rng.integers(1, 70))
+        f = (rng.random(n) < rng.choice([0.05, 0.3, 0.8])).astype(np.uint8)
+        xb = gen.bf16_bits_of(rng.standard_normal(n).astype(np.float32) * 100)
+        xq = [Fraction(float(v)) for v in oracle.bf16_to_double(xb)]
+        z, a = oracle.seg_scan_bf16(xb, f)
+        e, ea = oracle.seg_scan_bf16(xb, f, exclusive=True)
+        want, want_a = brute_scan(xq, f.tolist()), brute_scan([abs(v) for v in xq], f.tolist())
+        want_e = brute_excl(xq, f.tolist())
+        for i in range(n):
+            assert abs(Fraction(float(z[i])) - want[i]) <= Fraction(1, 10 ** 9)
+            assert abs(Fraction(float(a[i])) - want_a[i]) <= Fraction(1, 10 ** 9)
+            assert abs(Fraction(float(e[i])) - want_e[i]) <= Fraction(1, 10 ** 9)
+        s, _ = oracle.seg_sum_flags_bf16(xb, f)
+        ws = brute_sums(xq, f.tolist())
+        assert len(s) == len(ws)
+        for got, w in zip(s, ws):
+            assert abs(Fraction(float(got)) - w) <= Fraction(1, 10 ** 9)
+        off = oracle_offsets_of_flags(f)
+        sc, _ = oracle.seg_sum_csr_bf16(xb, off)
+        assert np.array_equal(sc, s)
+    # values representable in both 16-bit formats: the two routes must agree exactly
+    vals = rng.integers(-64, 65, 500).astype(np.float32) / 8
+    f = (rng.random(500) < 0.1).astype(np.uint8)
+    z16, a16 = oracle.seg_scan_f16(vals.astype(np.float16), f)
+    zb, ab = oracle.seg_scan_bf16(gen.bf16_bits_of(vals), f)
+    assert np.array_equal(z16, zb) and np.array_equal(a16, ab)
+
+
+def oracle_offsets_of_flags(f):
+    starts = [0] + [i for i in range(1, len(f)) if f[i]]
+    return np.asarray(starts + [len(f)], np.int32)
