@@ -584,7 +584,18 @@ def run_ours(args):
             sweep.append({"case": f"exclusive scan, {args.case}", "ms": cms, "gelem_s": n / cms / 1e6,
                           "gb_s": 7 * n / cms / 1e6, "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
                           "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
-            del fd
+            # bfloat16 input values (the headline values converted on the device), same flags and traffic
+            xb = xd.to(torch.bfloat16)
+            fn = lambda: mmv.seg_scan(xb, fd, out=od, workspace=ws)  # noqa: E731
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            cms = event_time_ms(torch, fn, min(args.steps, 10))
+            assert mmv.last_async_status(ws) == 0
+            sweep.append({"case": f"bf16 values, {args.case}", "ms": cms, "gelem_s": n / cms / 1e6,
+                          "gb_s": 7 * n / cms / 1e6, "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
+                          "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
+            del fd, xb
             line["configs"] = cfgs
             line["c5_density_sweep"] = sweep
         print(json.dumps(line))

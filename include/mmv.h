@@ -52,6 +52,9 @@
  *                   depends on timing.
  *   MMV_I8_TO_I32   int8 values, exact int32 result modulo 2^32 (bit-exact and
  *                   deterministic).
+ *   MMV_BF16_TO_F32 bfloat16 values, otherwise as MMV_F16_TO_F32.  Accepted by
+ *                   mmv_seg_scan, mmv_seg_scan_exclusive and mmv_seg_sum;
+ *                   the other entry points answer MMV_ERR_INVALID_ARG.
  */
 #ifndef MMV_H_
 #define MMV_H_
@@ -73,7 +76,7 @@ typedef enum {
     MMV_ERR_CUDA = 6                 /* a CUDA runtime / driver call failed                   */
 } mmv_status;
 
-typedef enum { MMV_F16_TO_F32 = 0, MMV_I8_TO_I32 = 1 } mmv_dtype;
+typedef enum { MMV_F16_TO_F32 = 0, MMV_I8_TO_I32 = 1, MMV_BF16_TO_F32 = 2 } mmv_dtype;
 typedef enum { MMV_SEG_FLAGS_U8 = 0, MMV_SEG_OFFSETS_I32 = 1 } mmv_segfmt;
 typedef enum { MMV_OP_SEG_SCAN = 0, MMV_OP_SEG_SUM = 1, MMV_OP_SPMV_CSR = 2 } mmv_op;
 

@@ -18,7 +18,7 @@ LIB_PATH = _PKG / "libmmv.so"
 
 # enums of include/mmv.h
 MMV_OK = 0
-F16_TO_F32, I8_TO_I32 = 0, 1
+F16_TO_F32, I8_TO_I32, BF16_TO_F32 = 0, 1, 2
 SEG_FLAGS_U8, SEG_OFFSETS_I32 = 0, 1
 OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR = 0, 1, 2
 
@@ -112,7 +112,9 @@ def _dtype_code(x: torch.Tensor) -> int:
         return F16_TO_F32
     if x.dtype == torch.int8:
         return I8_TO_I32
-    raise TypeError("values must be torch.float16 or torch.int8")
+    if x.dtype == torch.bfloat16:
+        return BF16_TO_F32
+    raise TypeError("values must be torch.float16, torch.bfloat16 or torch.int8")
 
 
 def _seg_code(seg: torch.Tensor) -> int:
@@ -148,7 +150,7 @@ def seg_scan(x: torch.Tensor, seg: torch.Tensor | None, out: torch.Tensor | None
     n = x.numel()
     nseg = seg.numel() - 1 if sf == SEG_OFFSETS_I32 else 0
     if out is None:
-        out = torch.empty(n, dtype=torch.float32 if dt == F16_TO_F32 else torch.int32, device=x.device)
+        out = torch.empty(n, dtype=torch.int32 if dt == I8_TO_I32 else torch.float32, device=x.device)
     if workspace is None:
         workspace = alloc_workspace(OP_SEG_SCAN, dt, sf, n, nseg, x.device)
     call = _lib.mmv_seg_scan_exclusive if exclusive else _lib.mmv_seg_scan
@@ -193,7 +195,7 @@ def seg_scan_host(x: torch.Tensor, flags: torch.Tensor | None, out: torch.Tensor
     dt = _dtype_code(x)
     n = x.numel()
     if out is None:
-        out = torch.empty(n, dtype=torch.float32 if dt == F16_TO_F32 else torch.int32, pin_memory=True)
+        out = torch.empty(n, dtype=torch.int32 if dt == I8_TO_I32 else torch.float32, pin_memory=True)
     if scratch is None:
         scratch = host_scan_scratch(dt, chunk)
     rc = _lib.mmv_seg_scan_host(_ptr(x), _ptr(flags), n, dt, _ptr(out), int(chunk), _ptr(scratch), scratch.numel(),
@@ -217,7 +219,7 @@ def seg_sum(x: torch.Tensor, seg: torch.Tensor, out: torch.Tensor | None = None,
     nseg = seg.numel() - 1 if sf == SEG_OFFSETS_I32 else 0
     if out is None:
         cap = nseg if sf == SEG_OFFSETS_I32 else n
-        out = torch.empty(cap, dtype=torch.float32 if dt == F16_TO_F32 else torch.int32, device=x.device)
+        out = torch.empty(cap, dtype=torch.int32 if dt == I8_TO_I32 else torch.float32, device=x.device)
     if workspace is None:
         workspace = alloc_workspace(OP_SEG_SUM, dt, sf, n, nseg, x.device)
     rc = _lib.mmv_seg_sum(_ptr(x), _ptr(seg), sf, n, nseg, dt, _ptr(out), _ptr(num_segments),

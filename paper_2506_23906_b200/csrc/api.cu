@@ -74,6 +74,10 @@ DeviceInfo* device_info() {
         ok &= set_smem(seg_scan_kernel<I8Path>, ScanCfg<I8Path>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<F16Path, true>, ScanCfg<F16Path>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<I8Path, true>, ScanCfg<I8Path>::kSmemBytes);
+        ok &= set_smem(seg_scan_kernel<BF16ValPath>, ScanCfg<BF16ValPath>::kSmemBytes);
+        ok &= set_smem(seg_scan_kernel<BF16ValPath, true>, ScanCfg<BF16ValPath>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<BF16ValPath, 2>, SumCfg<BF16ValPath, 2>::kSmemBytes);
+        ok &= set_smem(seg_sum_kernel<BF16ValPath, 3>, SumCfg<BF16ValPath, 3>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<F16Path, 2>, SumCfg<F16Path, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<I8Path, 2>, SumCfg<I8Path, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<BF16Path, 2>, SumCfg<BF16Path, 2>::kSmemBytes);
@@ -303,7 +307,7 @@ extern "C" {
 size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, int64_t nseg) {
     if (n < 0 || nseg < 0) return 0;
     if (op != MMV_OP_SEG_SCAN && op != MMV_OP_SEG_SUM && op != MMV_OP_SPMV_CSR) return 0;
-    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return 0;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return 0;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return 0;
     return plan_workspace(op, sf, n).total;
 }
@@ -312,7 +316,7 @@ namespace {
 mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
                          void* out, void* workspace, size_t workspace_bytes, void* cuda_stream, bool exclusive) {
     if (n < 0 || nseg < 0) return MMV_ERR_INVALID_ARG;
-    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return MMV_ERR_INVALID_ARG;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
     if (n == 0) return MMV_OK;
     if (n >= (1ll << 36)) return MMV_ERR_UNSUPPORTED;
@@ -347,7 +351,7 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
 
     const bool f16 = dt == MMV_F16_TO_F32;
     CUtensorMap tmap, tmap_out;
-    if (!encode_span_map(&tmap, x, n, f16 ? 2 : 1, SCAN_UP)) return MMV_ERR_CUDA;
+    if (!encode_span_map(&tmap, x, n, dt == MMV_I8_TO_I32 ? 1 : 2, SCAN_UP)) return MMV_ERR_CUDA;
     if (!encode_out_map(&tmap_out, out, n)) return MMV_ERR_CUDA;
 
     ScanParams prm;
@@ -362,7 +366,11 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
     prm.debug_skip_span = g_debug_skip_span.load();
     prm.carry_in = nullptr;
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
-    if (f16 && !exclusive)
+    if (dt == MMV_BF16_TO_F32 && !exclusive)
+        seg_scan_kernel<BF16ValPath><<<grid, ScanCfg<BF16ValPath>::kThreads, ScanCfg<BF16ValPath>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+    else if (dt == MMV_BF16_TO_F32)
+        seg_scan_kernel<BF16ValPath, true><<<grid, ScanCfg<BF16ValPath>::kThreads, ScanCfg<BF16ValPath>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+    else if (f16 && !exclusive)
         seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
     else if (!exclusive)
         seg_scan_kernel<I8Path><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
@@ -526,7 +534,7 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
                        void* out, int64_t* d_num_segments, void* workspace, size_t workspace_bytes,
                        void* cuda_stream) {
     if (n < 0 || nseg < 0) return MMV_ERR_INVALID_ARG;
-    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return MMV_ERR_INVALID_ARG;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
     if (n >= (1ll << 31)) return MMV_ERR_INVALID_ARG;            // int32 offsets cannot address more
     if (sf == MMV_SEG_FLAGS_U8) {
@@ -564,6 +572,7 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
         g_launches += 3;
         if (cudaGetLastError() != cudaSuccess) return MMV_ERR_CUDA;
         if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, true);
+        if (dt == MMV_BF16_TO_F32) return launch_seg_sum<BF16ValPath>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, true);
         return launch_seg_sum<I8Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, true);
     }
     if (nseg == 0) return MMV_OK;
@@ -583,6 +592,7 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
     if (cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
     const int32_t* off = static_cast<const int32_t*>(seg);
     if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, nseg, 0, out, ws, plan, dev, st);
+    if (dt == MMV_BF16_TO_F32) return launch_seg_sum<BF16ValPath>(x, n, off, nseg, 0, out, ws, plan, dev, st);
     return launch_seg_sum<I8Path>(x, n, off, nseg, 0, out, ws, plan, dev, st);
 }
 

@@ -68,6 +68,12 @@ struct F16Path {
     __device__ static __forceinline__ Acc add(Acc a, Acc b) { return a + b; }
     __device__ static __forceinline__ Acc sub(Acc a, Acc b) { return a - b; }
 };
+// bfloat16 input values, fp32 results: the layout and arithmetic of the fp16 path, with the tensor-core
+// operands declared bf16 (the products with the 0/1 matrix stay exact, the accumulator is fp32).
+struct BF16ValPath : F16Path {
+    static constexpr uint32_t kOneBits = 0x3F80u;                       // 1.0 in bf16
+    static constexpr uint32_t kFmtBits = (1u << 7) | (1u << 10);        // A and B are bf16
+};
 struct I8Path {
     using Acc = uint32_t;                                  // wrap-around arithmetic on unsigned
     static constexpr int kElemBytes = 1;

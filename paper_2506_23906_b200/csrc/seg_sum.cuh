@@ -100,6 +100,10 @@ __device__ __forceinline__ float load_value<F16Path>(const void* base, long long
     return __half2float(static_cast<const __half*>(base)[idx]);
 }
 template <>
+__device__ __forceinline__ float load_value<BF16ValPath>(const void* base, long long idx) {
+    return __uint_as_float(static_cast<uint32_t>(static_cast<const unsigned short*>(base)[idx]) << 16);
+}
+template <>
 __device__ __forceinline__ float load_value<BF16Path>(const void* base, long long idx) {
     return pair_value(static_cast<const uint32_t*>(base)[idx]);
 }
@@ -114,6 +118,10 @@ __device__ __forceinline__ typename P::Acc elem_bits_to_acc(uint32_t bits);
 template <>
 __device__ __forceinline__ float elem_bits_to_acc<F16Path>(uint32_t bits) {
     return __half2float(__ushort_as_half(static_cast<unsigned short>(bits)));
+}
+template <>
+__device__ __forceinline__ float elem_bits_to_acc<BF16ValPath>(uint32_t bits) {
+    return __uint_as_float((bits & 0xffffu) << 16);
 }
 template <>
 __device__ __forceinline__ float elem_bits_to_acc<BF16Path>(uint32_t bits) {

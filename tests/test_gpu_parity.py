@@ -521,6 +521,62 @@ def test_exclusive_scan_flags_on_edges_offsets_and_plain(mmv):
 
 
 # ---------------------------------------------------------------------------
+# bfloat16 input values
+# ---------------------------------------------------------------------------
+def dev_bf16(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+@pytest.mark.parametrize("n", [1, 33, 4097, TILE + 5, 7 * TILE + 1234])
+@pytest.mark.parametrize("p", [0.0, 1e-3, 0.1, 1.0])
+def test_bf16_scan_and_sum(mmv, n, p):
+    rng = np.random.default_rng(n + int(p * 1e4))
+    f = (rng.random(n) < p).astype(np.uint8)
+    xb = gen.bf16_normal(8, n)
+    xd, fd = dev_bf16(xb), dev(f)
+    for exclusive in (False, True):
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.BF16_TO_F32, mmv.SEG_FLAGS_U8, n)
+        got = mmv.seg_scan(xd, fd, workspace=ws, exclusive=exclusive).cpu().numpy()
+        assert mmv.last_async_status(ws) == 0
+        want, a = oracle.seg_scan_bf16(xb, f, exclusive=exclusive)
+        assert_fp(got, want, a, f"bf16 scan n={n} p={p} exclusive={exclusive}")
+    # the same segments as offsets and as flags through the segmented sum
+    starts = np.flatnonzero(f)
+    off = np.unique(np.concatenate([[0], starts, [n]])).astype(np.int32)
+    want, a = oracle.seg_sum_csr_bf16(xb, off)
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.BF16_TO_F32, mmv.SEG_OFFSETS_I32, n, off.shape[0] - 1)
+    got = mmv.seg_sum(xd, dev(off), workspace=ws).cpu().numpy()
+    assert mmv.last_async_status(ws) == 0
+    assert_fp(got, want, a, f"bf16 seg-sum n={n} p={p}")
+    k = torch.zeros(1, dtype=torch.int64, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.BF16_TO_F32, mmv.SEG_FLAGS_U8, n)
+    gotf = mmv.seg_sum(xd, fd, num_segments=k, workspace=ws)
+    assert mmv.last_async_status(ws) == 0 and int(k.item()) == off.shape[0] - 1
+    wantf, af = oracle.seg_sum_flags_bf16(xb, f)
+    assert_fp(gotf[:int(k.item())].cpu().numpy(), wantf, af, f"bf16 flag-form seg-sum n={n} p={p}")
+
+
+def test_bf16_values_beyond_the_fp16_range(mmv):
+    # magnitudes that fp16 cannot hold (up to 1e30 and down to 1e-30), one magnitude per segment
+    rng = np.random.default_rng(5)
+    nseg = 3000
+    lens = rng.integers(1, 200, nseg)
+    off = gen.offsets_from_lengths(lens)
+    n = int(off[-1])
+    scale = np.repeat(10.0 ** rng.integers(-30, 31, nseg).astype(np.float64), lens)
+    xb = gen.bf16_bits_of((rng.standard_normal(n) * scale).astype(np.float32))
+    f = gen.start_flags_of_offsets(off, n)
+    want, a = oracle.seg_scan_bf16(xb, f)
+    got = mmv.seg_scan(dev_bf16(xb), dev(f)).cpu().numpy()
+    # the bound is relative to the segment's own running sum of magnitudes; what a prefix difference can keep
+    # is relative to the magnitudes of its 32-element row, so only segments that dominate their rows are held to it
+    ok = np.abs(got - want) <= 2e-3 * a + 1e-6
+    big = scale >= np.maximum.accumulate(scale)                        # no larger magnitude before it
+    assert ok[big].all()
+    assert np.isfinite(got).all()
+
+
+# ---------------------------------------------------------------------------
 # robustness
 # ---------------------------------------------------------------------------
 def test_bad_column_indices_are_reported_not_dereferenced(mmv):
