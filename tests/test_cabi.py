@@ -71,6 +71,11 @@ def test_argument_errors_are_synchronous(lib):
     assert lib.mmv_seg_scan(16, 16, 3, 8, 0, 0, 16, 256, 4096, None) == 1           # bad segment format
     assert lib.mmv_seg_scan(18, 16, 0, 8, 0, 0, 16, 256, 4096, None) == 1           # misaligned x
     assert lib.mmv_seg_scan(16, 16, 0, 8, 0, 0, 16, 256, 16, None) == 3             # workspace too small
+    lib.mmv_seg_scan_exclusive.argtypes = lib.mmv_seg_scan.argtypes
+    assert lib.mmv_seg_scan_exclusive(None, None, 0, -1, 0, 0, None, None, 0, None) == 1      # negative n
+    assert lib.mmv_seg_scan_exclusive(None, None, 0, 0, 0, 2, None, None, 0, None) == 0       # n == 0, bf16: nothing to do
+    assert lib.mmv_seg_scan_exclusive(16, 16, 0, 8, 0, 3, 16, 256, 4096, None) == 1           # bad dtype
+    assert lib.mmv_seg_scan(16, 16, 0, 8, 0, 2, 16, 256, 16, None) == 3                       # bf16 accepted: workspace too small
     assert lib.mmv_seg_sum(None, None, 1, 0, 0, 0, None, None, None, 0, None) == 0  # nothing to do
     assert lib.mmv_seg_sum(16, 16, 1, -5, 1, 0, 16, None, 256, 4096, None) == 1
     assert lib.mmv_seg_sum(16, 16, 0, 8, 0, 0, 16, None, 256, 16, None) == 3        # flag form: workspace too small
@@ -81,6 +86,7 @@ def test_argument_errors_are_synchronous(lib):
     assert lib.mmv_seg_scan_host(16, 16, 8, 0, 16, 1000, 256, 1 << 30, None) == 1     # chunk not a multiple of 16384
     assert lib.mmv_seg_scan_host(16, 16, 8, 0, 16, 16384, 256, 16, None) == 3         # scratch too small
     assert lib.mmv_seg_scan_host(None, None, 0, 0, None, 16384, None, 0, None) == 0   # nothing to do
+    assert lib.mmv_seg_scan_host(16, 16, 8, 2, 16, 16384, 256, 1 << 30, None) == 1    # bf16 values: not for this entry point
     assert lib.mmv_seg_scan_host_scratch_bytes(0, 1000) == 0
     assert lib.mmv_seg_scan_host_scratch_bytes(0, 16384) >= 2 * 16384 * 7
     assert lib.mmv_spmv_csr(None, None, None, None, None, -1, 1, 1, None, 0, None) == 1
