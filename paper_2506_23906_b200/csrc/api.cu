@@ -223,11 +223,16 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     if (!have_partition) {     // (the flag-encoded form has filled span_q while compacting its flags)
         const long long spans = static_cast<long long>(tiles) * SPANS_PER_TILE;
         const int threads = 256;
-        long long blocks = (nseg + 1 + threads - 1) / threads;                 // one thread per offset and round
+        const int vec = nseg >= (1ll << 20) ? 4 : 1;                           // offsets per thread and round
+        long long blocks = (nseg + 1 + vec * threads - 1) / (vec * threads);
         if (blocks > 16ll * dev->sm_count) blocks = 16ll * dev->sm_count;
-        partition_offsets_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, spans, span_q, n_eff,
-                                                                                 reinterpret_cast<WorkspaceHeader*>(ws),
-                                                                                 static_cast<uint32_t*>(out));
+        WorkspaceHeader* hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+        if (vec == 4)
+            partition_offsets_kernel<4><<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, spans, span_q, n_eff, hdr,
+                                                                                          static_cast<uint32_t*>(out));
+        else
+            partition_offsets_kernel<1><<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, spans, span_q, n_eff, hdr,
+                                                                                          static_cast<uint32_t*>(out));
         ++g_launches;
     }
     CUtensorMap tmap;

@@ -287,63 +287,97 @@ __device__ __noinline__ long long first_index_at_least_call(const int32_t* off, 
 }
 
 // span_q[s] = first index i in [0, nseg] with bnd(i) = off[i] << shift >= s * SPAN, nseg + 1 if none,
-// for s = 0 .. num_spans.  One thread per offset index i: i is that first index exactly for the
-// spans s with bnd(i-1) < s * SPAN <= bnd(i), a range it writes itself (ranges of more than 32
+// for s = 0 .. num_spans.  Every offset index i is handled by one thread: i is that first index exactly
+// for the spans s with bnd(i-1) < s * SPAN <= bnd(i), a range the thread writes itself (ranges of more than 32
 // spans, i.e. very long segments, are written by the whole warp).  The same pass validates the
 // offsets (non-decreasing, inside [0, n]; MMV_ERR_BAD_SEGMENTS otherwise -- entries may then be
 // missing or inconsistent, which the main kernel tolerates: it clamps what it reads and never
 // indexes outside its tile) and writes the zero of every EMPTY segment, so that the main kernel
 // may jump over long runs of equal offsets instead of visiting them one by one.
+template <int VEC>       // offsets per lane and round: 4 when there are many (one 16-byte load each), else 1
 __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, long long num_spans,
                                          int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr,
                                          uint32_t* __restrict__ out) {
     const int lane = threadIdx.x & 31;
-    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    const long long stride = static_cast<long long>(VEC) * gridDim.x * blockDim.x;
     const int n32 = static_cast<int>(n < 0x7fffffffll ? n : 0x7fffffffll);
     const int last_span = static_cast<int>(num_spans);
-    // (every warp makes the same number of rounds: the votes below need all its lanes; positions and span
-    //  indices fit 32 bits because the offsets do)
-    for (long long wbase = static_cast<long long>(blockIdx.x) * blockDim.x + (threadIdx.x & ~31); wbase <= nseg; wbase += stride) {
-        const long long i = wbase + lane;          // offset index
-        const bool exists = i <= nseg;
-        const int cur = exists ? off[i] : 0;
-        int prev = __shfl_up_sync(0xffffffffu, cur, 1);
-        if (lane == 0) prev = wbase >= 1 ? off[wbase - 1] : 0;
-        int lo = 0, hi = -1;                       // spans [lo, hi] get the value i
-        if (exists) {
-            if (i >= 1) {
-                if (prev > cur || prev < 0 || cur > n32) report_error(hdr, 4u);
-                if (prev == cur) out[i - 1] = 0u;                  // segment i - 1 is empty
-                lo = prev < 0 ? 0 : (prev >> 12) + 1;
-            } else if (cur < 0 || cur > n32) {
-                report_error(hdr, 4u);
+    static_assert(SPAN == 4096, "span index = position >> 12");
+    // A warp takes 32 VEC consecutive offsets per round; with many offsets four per lane in one 16-byte
+    // load (the kernel is bound by the loads it has in flight).  Every warp makes the same number of rounds: the votes below
+    // need all its lanes.  Positions and span indices fit 32 bits because the offsets do.
+    for (long long wbase = VEC * (static_cast<long long>(blockIdx.x) * blockDim.x + (threadIdx.x & ~31)); wbase <= nseg; wbase += stride) {
+        const long long i0 = wbase + VEC * lane;   // my first offset index
+        int c[VEC];
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) c[e] = 0;
+        bool vector_load = false;
+        if constexpr (VEC == 4) {
+            if (i0 + 3 <= nseg) {
+                const int4 v = *reinterpret_cast<const int4*>(off + i0);
+                c[0] = v.x;
+                c[1] = v.y;
+                c[2] = v.z;
+                c[3] = v.w;
+                vector_load = true;
             }
-            hi = cur < 0 ? -1 : (cur >> 12);
-            if (hi > last_span) hi = last_span;
         }
-        static_assert(SPAN == 4096, "span index = position >> 12");
-        const bool is_last = exists && i == nseg;
-        unsigned todo = __ballot_sync(0xffffffffu, hi >= lo || is_last);
-        if (todo == 0u) continue;                  // no span starts between this warp's offsets
-        if (hi >= lo && hi - lo < 32) {
-            for (int s = lo; s <= hi; ++s) span_q[s] = static_cast<int32_t>(i);
-            lo = hi + 1;
+        if (!vector_load) {
+#pragma unroll
+            for (int e = 0; e < VEC; ++e)
+                if (i0 + e <= nseg) c[e] = off[i0 + e];
         }
-        // long ranges, and the range behind the last offset: the whole warp writes them
-        todo = __ballot_sync(0xffffffffu, hi >= lo);
-        while (todo) {
-            const int src = __ffs(todo) - 1;
-            const int l = __shfl_sync(0xffffffffu, lo, src), h = __shfl_sync(0xffffffffu, hi, src);
-            const int v = static_cast<int>(wbase) + src;
-            for (int s = l + lane; s <= h; s += 32) span_q[s] = v;
-            todo &= todo - 1;
+        int before = __shfl_up_sync(0xffffffffu, c[VEC - 1], 1);
+        if (lane == 0) before = wbase >= 1 ? off[wbase - 1] : 0;
+        int lo[VEC], hi[VEC];                      // spans [lo, hi] get the offset's index
+        bool any = false;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) {
+            const long long i = i0 + e;
+            const int cur = c[e], prev = e ? c[e - 1] : before;
+            lo[e] = 0;
+            hi[e] = -1;
+            if (i <= nseg) {
+                if (i >= 1) {
+                    if (prev > cur || prev < 0 || cur > n32) report_error(hdr, 4u);
+                    if (prev == cur) out[i - 1] = 0u;              // segment i - 1 is empty
+                    lo[e] = prev < 0 ? 0 : (prev >> 12) + 1;
+                } else if (cur < 0 || cur > n32) {
+                    report_error(hdr, 4u);
+                }
+                hi[e] = cur < 0 ? -1 : (cur >> 12);
+                if (hi[e] > last_span) hi[e] = last_span;
+                any |= hi[e] >= lo[e] || i == nseg;
+            }
         }
-        todo = __ballot_sync(0xffffffffu, is_last);
-        if (todo) {
-            const int src = __ffs(todo) - 1;
-            const int h0 = __shfl_sync(0xffffffffu, cur < 0 ? -1 : (cur >> 12), src);
-            for (int s = (h0 > last_span ? last_span : h0) + 1 + lane; s <= last_span; s += 32)
-                span_q[s] = static_cast<int32_t>(nseg + 1);
+        if (__ballot_sync(0xffffffffu, any) == 0u) continue;       // no span starts between this warp's offsets
+#pragma unroll 1
+        for (int e = 0; e < VEC; ++e) {
+            int l = lo[0], h = hi[0], cur = c[0];
+#pragma unroll
+            for (int t = 1; t < VEC; ++t)
+                if (e == t) { l = lo[t]; h = hi[t]; cur = c[t]; }
+            const long long i = i0 + e;
+            if (h >= l && h - l < 32) {
+                for (int sp = l; sp <= h; ++sp) span_q[sp] = static_cast<int32_t>(i);
+                l = h + 1;
+            }
+            // long ranges, and the range behind the last offset: the whole warp writes them
+            unsigned todo = __ballot_sync(0xffffffffu, h >= l);
+            while (todo) {
+                const int src = __ffs(todo) - 1;
+                const int ll = __shfl_sync(0xffffffffu, l, src), hh = __shfl_sync(0xffffffffu, h, src);
+                const int v = static_cast<int>(wbase) + VEC * src + e;
+                for (int sp = ll + lane; sp <= hh; sp += 32) span_q[sp] = v;
+                todo &= todo - 1;
+            }
+            todo = __ballot_sync(0xffffffffu, i == nseg);
+            if (todo) {
+                const int src = __ffs(todo) - 1;
+                const int h0 = __shfl_sync(0xffffffffu, cur < 0 ? -1 : (cur >> 12), src);
+                for (int sp = (h0 > last_span ? last_span : h0) + 1 + lane; sp <= last_span; sp += 32)
+                    span_q[sp] = static_cast<int32_t>(nseg + 1);
+            }
         }
     }
 }
