@@ -29,6 +29,10 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
+def dev_bf16(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
 def scan_i8(mmv, x, f, guard=64, exclusive=False):
     n = x.shape[0]
     seg = dev(f)
@@ -484,6 +488,87 @@ def test_seg_sum_row_length_mixes(mmv, kind):
 
 
 # ---------------------------------------------------------------------------
+# randomised shapes
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_seg_sum_random_shapes(mmv, seed):
+    # random sizes, segment-length laws (tiny, geometric, wide, with empty segments, with runs of them, constant),
+    # leading ignored elements, all three value types and both kernel shapes
+    rng = np.random.default_rng(seed)
+    for trial in range(40):
+        n = int(rng.choice([rng.integers(1, 300), rng.integers(300, 40000), rng.integers(40000, 6 * TILE)]))
+        kind = int(rng.integers(0, 6))
+        if kind == 0:
+            lens = rng.integers(0, 4, 4 * n)
+        elif kind == 1:
+            lens = rng.geometric(1 / rng.choice([2.0, 6.0, 40.0, 300.0]), 2 * n) - rng.integers(0, 2)
+        elif kind == 2:
+            lens = rng.integers(1, rng.choice([8, 64, 2000, 20000]), n)
+        elif kind == 3:
+            lens = rng.integers(1, 50, n)
+            lens[rng.random(n) < 0.3] = 0
+        elif kind == 4:
+            lens = rng.integers(1, 10, n)
+            for _ in range(3):
+                at = int(rng.integers(0, lens.shape[0]))
+                lens = np.concatenate([lens[:at], np.zeros(int(rng.choice([31, 32, 33, 127, 129, 300, 5000])), np.int64), lens[at:]])
+        else:
+            lens = np.full(n, rng.choice([1, 2, 31, 32, 33, 1024, 4096]))
+        lead = int(rng.integers(0, 40)) if rng.random() < 0.3 else 0
+        off = np.concatenate([[lead], lead + np.cumsum(np.maximum(lens, 0))])
+        off = off[off <= n]
+        if off.shape[0] < 2:
+            off = np.asarray([0, n])
+        off = off.astype(np.int32)
+        mmv.debug_force_sum_groups(int(rng.choice([0, 2, 3])))
+        try:
+            what = f"seed {seed} trial {trial} n={n} kind={kind}"
+            which = int(rng.integers(0, 3))
+            if which == 0:
+                x = rng.integers(-128, 128, n).astype(np.int8)
+                assert np.array_equal(sum_csr(mmv, x, off), oracle.seg_sum_csr_i8(x, off)), what
+            elif which == 1:
+                x = (rng.standard_normal(n) * rng.choice([1.0, 30.0])).astype(np.float16)
+                want, a = oracle.seg_sum_csr_f16(x, off)
+                assert_fp(sum_csr(mmv, x, off), want, a, what)
+            else:
+                xb = gen.bf16_bits_of(rng.standard_normal(n).astype(np.float32))
+                ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.BF16_TO_F32, mmv.SEG_OFFSETS_I32, n, off.shape[0] - 1)
+                got = mmv.seg_sum(dev_bf16(xb), dev(off), workspace=ws).cpu().numpy()
+                assert mmv.last_async_status(ws) == 0
+                want, a = oracle.seg_sum_csr_bf16(xb, off)
+                assert_fp(got, want, a, what)
+        finally:
+            mmv.debug_force_sum_groups(0)
+
+
+def test_spmv_random_shapes(mmv):
+    rng = np.random.default_rng(21)
+    for trial in range(40):
+        rows = int(rng.choice([rng.integers(1, 50), rng.integers(50, 5000), rng.integers(5000, 100000)]))
+        cols = int(rng.integers(1, 100000))
+        kind = int(rng.integers(0, 4))
+        if kind == 0:
+            lens = rng.integers(0, 4, rows)
+        elif kind == 1:
+            lens = rng.geometric(1 / rng.choice([2.0, 6.0, 60.0]), rows) - rng.integers(0, 2)
+        elif kind == 2:
+            lens = rng.integers(0, rng.choice([8, 200, 5000]), rows)
+        else:
+            lens = np.full(rows, rng.choice([1, 2, 32, 33]))
+        lens = np.maximum(lens, 0)
+        if lens.sum() > 2_000_000:
+            lens = lens // 8
+        rowptr = gen.offsets_from_lengths(lens)
+        nnz = int(rowptr[-1])
+        col = rng.integers(0, cols, nnz).astype(np.int32)
+        val = (rng.standard_normal(nnz) * rng.choice([1.0, 100.0])).astype(np.float16)
+        x = (rng.standard_normal(cols) * rng.choice([1.0, 1e-3, 50.0])).astype(np.float32)
+        want, a = oracle.spmv_csr(rowptr, col, val, x)
+        assert_fp(spmv(mmv, rowptr, col, val, x), want, a, f"trial {trial} rows={rows} nnz={nnz} kind={kind}")
+
+
+# ---------------------------------------------------------------------------
 # exclusive variant of the scan
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("n", [1, 31, 32, 33, 1023, 1025, 4096, TILE - 1, TILE, TILE + 1, 3 * TILE + 4097, 11 * TILE + 777])
@@ -523,10 +608,6 @@ def test_exclusive_scan_flags_on_edges_offsets_and_plain(mmv):
 # ---------------------------------------------------------------------------
 # bfloat16 input values
 # ---------------------------------------------------------------------------
-def dev_bf16(bits):
-    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
-
-
 @pytest.mark.parametrize("n", [1, 33, 4097, TILE + 5, 7 * TILE + 1234])
 @pytest.mark.parametrize("p", [0.0, 1e-3, 0.1, 1.0])
 def test_bf16_scan_and_sum(mmv, n, p):
