@@ -76,6 +76,10 @@ DeviceInfo* device_info() {
         ok &= set_smem(seg_scan_kernel<I8Path, true>, ScanCfg<I8Path>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<BF16ValPath>, ScanCfg<BF16ValPath>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<BF16ValPath, true>, ScanCfg<BF16ValPath>::kSmemBytes);
+        ok &= set_smem(seg_scan_kernel<F16Path, false, true>, ScanCfg<F16Path, true>::kSmemBytes);
+        ok &= set_smem(seg_scan_kernel<F16Path, true, true>, ScanCfg<F16Path, true>::kSmemBytes);
+        ok &= set_smem(seg_scan_kernel<BF16ValPath, false, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
+        ok &= set_smem(seg_scan_kernel<BF16ValPath, true, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<BF16ValPath, 2>, SumCfg<BF16ValPath, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<BF16ValPath, 3>, SumCfg<BF16ValPath, 3>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<F16Path, 2>, SumCfg<F16Path, 2>::kSmemBytes);
@@ -371,18 +375,25 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
     prm.debug_skip_span = g_debug_skip_span.load();
     prm.carry_in = nullptr;
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
-    if (dt == MMV_BF16_TO_F32 && !exclusive)
-        seg_scan_kernel<BF16ValPath><<<grid, ScanCfg<BF16ValPath>::kThreads, ScanCfg<BF16ValPath>::kSmemBytes, st>>>(tmap, tmap_out, prm);
-    else if (dt == MMV_BF16_TO_F32)
-        seg_scan_kernel<BF16ValPath, true><<<grid, ScanCfg<BF16ValPath>::kThreads, ScanCfg<BF16ValPath>::kSmemBytes, st>>>(tmap, tmap_out, prm);
-    else if (f16 && !exclusive)
-        seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
-    else if (!exclusive)
-        seg_scan_kernel<I8Path><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
-    else if (f16)
-        seg_scan_kernel<F16Path, true><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
-    else
-        seg_scan_kernel<I8Path, true><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+    // (no flag vector: the floating-point paths run the narrow-tile variant)
+    const bool plain = flags == nullptr;
+#define MMV_LAUNCH_SCAN(PATH, EXCL, PL)                                                                               \
+    seg_scan_kernel<PATH, EXCL, PL><<<grid, ScanCfg<PATH, PL>::kThreads, ScanCfg<PATH, PL>::kSmemBytes, st>>>(tmap, tmap_out, prm)
+    if (dt == MMV_I8_TO_I32) {
+        if (exclusive) MMV_LAUNCH_SCAN(I8Path, true, false);
+        else MMV_LAUNCH_SCAN(I8Path, false, false);
+    } else if (dt == MMV_BF16_TO_F32) {
+        if (plain && exclusive) MMV_LAUNCH_SCAN(BF16ValPath, true, true);
+        else if (plain) MMV_LAUNCH_SCAN(BF16ValPath, false, true);
+        else if (exclusive) MMV_LAUNCH_SCAN(BF16ValPath, true, false);
+        else MMV_LAUNCH_SCAN(BF16ValPath, false, false);
+    } else {
+        if (plain && exclusive) MMV_LAUNCH_SCAN(F16Path, true, true);
+        else if (plain) MMV_LAUNCH_SCAN(F16Path, false, true);
+        else if (exclusive) MMV_LAUNCH_SCAN(F16Path, true, false);
+        else MMV_LAUNCH_SCAN(F16Path, false, false);
+    }
+#undef MMV_LAUNCH_SCAN
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }

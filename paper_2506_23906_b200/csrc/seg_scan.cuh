@@ -64,26 +64,30 @@ constexpr int SCAN_LB_WORDS = 1;                            // look-back window:
 #define MMV_SCAN_I8_GROUPS 3
 #endif
 
-template <typename P>
+// PLAIN = the call has no flag vector (one segment): no row ever needs its own values back, so the
+// floating-point paths drop the identity half of the product and get the narrow tiles, the third
+// warpgroup and the flag-free stages of the int8 path.
+template <typename P, bool PLAIN = false>
 struct ScanCfg {
     // fp16: the product also returns the rows themselves (exact fp32 copies, columns 32..63), so a
     // tile needs 256 TMEM columns and each warpgroup has one buffer; int8: 128 columns, two buffers.
     // The epilogue is latency-bound, so the narrower int8 tiles are spread over a third warpgroup.
-    static constexpr int kN = P::kIsFloat ? 2 * ROW : ROW;               // accumulator columns per product
-    static constexpr int kGroups = P::kIsFloat ? 2 : MMV_SCAN_I8_GROUPS;
-    static constexpr int kBufsPerGroup = P::kIsFloat ? 1 : (kGroups == 2 ? 2 : 1);
+    static constexpr bool kWide = P::kIsFloat && !PLAIN;                 // [U | I] product
+    static constexpr int kN = kWide ? 2 * ROW : ROW;                     // accumulator columns per product
+    static constexpr int kGroups = kWide ? 2 : MMV_SCAN_I8_GROUPS;
+    static constexpr int kBufsPerGroup = kWide ? 1 : (kGroups == 2 ? 2 : 1);
     static constexpr int kBufs = kGroups * kBufsPerGroup;                // TMEM tile buffers
     static constexpr int kEpiWarps = 4 * kGroups;
     static constexpr int kProducerWarp = kEpiWarps;
     static constexpr int kMmaWarp = kEpiWarps + 1;
     static constexpr int kThreads = (kEpiWarps + 2) * 32;
     static constexpr int kTmemCols = 512;
-    static constexpr int kStages = P::kIsFloat ? 3 : (kGroups == 2 ? 4 : 3);
+    static constexpr int kStages = kWide ? 3 : (kGroups == 2 ? 4 : 3);
     static_assert(kBufs * SCAN_UP * kN <= kTmemCols, "tile buffers fit the tensor memory");
     static constexpr int kBBytes = kN * P::kRowBytes;                    // constant operand [U_32 | I_32] / U_32
     static constexpr int kBSlot = 4096;
     static constexpr int kXBytes = SCAN_UP * P::kSlabBytes;
-    static constexpr int kFlagBytes = SCAN_TILE;
+    static constexpr int kFlagBytes = PLAIN ? 0 : SCAN_TILE;
     static constexpr int kStageBytes = kXBytes + kFlagBytes;
     static constexpr int kStageOffset = kBSlot;
     static constexpr int kOutOffset = kStageOffset + kStages * kStageBytes;
@@ -132,12 +136,12 @@ __device__ __forceinline__ bool wait_stage(const volatile int* stage_iter, int i
 // segment in FRONT of it (0 at a segment start), i.e. the inclusive result moved one element to
 // the right inside each segment.  The shift happens in registers just before a piece is staged for
 // its store; everything else is the same kernel.
-template <typename P, bool EX = false>
-__global__ void __launch_bounds__(ScanCfg<P>::kThreads, 1)
+template <typename P, bool EX = false, bool PLAIN = false>
+__global__ void __launch_bounds__(ScanCfg<P, PLAIN>::kThreads, 1)
 seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_out,
                  const ScanParams prm) {
     using Acc = typename P::Acc;
-    using Cfg = ScanCfg<P>;
+    using Cfg = ScanCfg<P, PLAIN>;
     constexpr int S = Cfg::kStages;
     constexpr int N = Cfg::kN;
 
@@ -535,12 +539,12 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 uint32_t r[32];
                 uint32_t raw[P::kIsFloat ? 32 : 1];
                 tmem_ld_32x32(taddr + i * N, r);
-                if constexpr (P::kIsFloat) {
+                if constexpr (Cfg::kWide) {
                     if (pmi != 0u) tmem_ld_32x32(taddr + i * N + ROW, raw);
                 }
                 tmem_ld_wait();
                 MMV_T_MARK(4)
-                if (pmi == 0u) {
+                if (PLAIN || pmi == 0u) {
                     // no flag in the piece: plain prefix of the row totals, one add per element
                     Acc inc = toti;
 #pragma unroll

@@ -180,6 +180,19 @@ def test_plain_scan_without_a_flag_vector(mmv):
         got = mmv.seg_scan(dev(xf), None, workspace=ws).cpu().numpy()
         z, a = oracle.seg_scan_f16(xf, zero)
         assert_fp(got, z, a, f"plain scan n={n}")
+        # (the floating-point plain scan is a kernel variant of its own: exclusive and bfloat16 too)
+        got = mmv.seg_scan(dev(xf), None, exclusive=True).cpu().numpy()
+        e, ea = oracle.seg_scan_excl_f16(xf, zero)
+        assert_fp(got, e, ea, f"plain exclusive scan n={n}")
+        xb = gen.bf16_normal(9, n)
+        for exclusive in (False, True):
+            got = mmv.seg_scan(dev_bf16(xb), None, exclusive=exclusive).cpu().numpy()
+            zb, ab = oracle.seg_scan_bf16(xb, zero, exclusive=exclusive)
+            assert_fp(got, zb, ab, f"plain bf16 scan n={n} exclusive={exclusive}")
+    for n in (7 * TILE + 5, 40 * TILE + 31):                   # many tiles per warpgroup, a ragged end
+        xf = rng.uniform(-1, 1, n).astype(np.float16)
+        z, a = oracle.seg_scan_f16(xf, np.zeros(n, np.uint8))
+        assert_fp(mmv.seg_scan(dev(xf), None).cpu().numpy(), z, a, f"plain scan n={n}")
     # host vectors, chunked, no flags
     n = 9 * TILE + 17
     xf = rng.uniform(-1, 1, n).astype(np.float16)
