@@ -65,8 +65,8 @@ constexpr int SCAN_LB_WORDS = 1;                            // look-back window:
 #endif
 
 // PLAIN = the call has no flag vector (one segment): no row ever needs its own values back, so the
-// floating-point paths drop the identity half of the product and get the narrow tiles, the third
-// warpgroup and the flag-free stages of the int8 path.
+// floating-point paths drop the identity half of the product: narrow tiles (128 TMEM columns), so
+// four warpgroups with one tile each, four 32 KB stages without flag bytes, one staging buffer per warp.
 template <typename P, bool PLAIN = false>
 struct ScanCfg {
     // fp16: the product also returns the rows themselves (exact fp32 copies, columns 32..63), so a
@@ -74,7 +74,10 @@ struct ScanCfg {
     // The epilogue is latency-bound, so the narrower int8 tiles are spread over a third warpgroup.
     static constexpr bool kWide = P::kIsFloat && !PLAIN;                 // [U | I] product
     static constexpr int kN = kWide ? 2 * ROW : ROW;                     // accumulator columns per product
-    static constexpr int kGroups = kWide ? 2 : MMV_SCAN_I8_GROUPS;
+#ifndef MMV_SCAN_PLAIN_GROUPS
+#define MMV_SCAN_PLAIN_GROUPS 4
+#endif
+    static constexpr int kGroups = kWide ? 2 : ((PLAIN && P::kIsFloat) ? MMV_SCAN_PLAIN_GROUPS : MMV_SCAN_I8_GROUPS);
     static constexpr int kBufsPerGroup = kWide ? 1 : (kGroups == 2 ? 2 : 1);
     static constexpr int kBufs = kGroups * kBufsPerGroup;                // TMEM tile buffers
     static constexpr int kEpiWarps = 4 * kGroups;
@@ -82,7 +85,8 @@ struct ScanCfg {
     static constexpr int kMmaWarp = kEpiWarps + 1;
     static constexpr int kThreads = (kEpiWarps + 2) * 32;
     static constexpr int kTmemCols = 512;
-    static constexpr int kStages = kWide ? 3 : (kGroups == 2 ? 4 : 3);
+    static constexpr int kStages = kWide ? 3 : ((kGroups == 2 || kGroups == 4) ? 4 : 3);
+    static_assert(kStages >= kGroups, "the producer's closing round needs a stage per warpgroup");
     static_assert(kBufs * SCAN_UP * kN <= kTmemCols, "tile buffers fit the tensor memory");
     static constexpr int kBBytes = kN * P::kRowBytes;                    // constant operand [U_32 | I_32] / U_32
     static constexpr int kBSlot = 4096;
@@ -92,7 +96,7 @@ struct ScanCfg {
     static constexpr int kStageOffset = kBSlot;
     static constexpr int kOutOffset = kStageOffset + kStages * kStageBytes;
     static constexpr int kOutBufBytes = PIECE * 4;                       // 32 rows x 128 B
-    static constexpr int kOutBufs = 2;                                   // staging buffers per warp
+    static constexpr int kOutBufs = kGroups >= 4 ? 1 : 2;                // staging buffers per warp
     static constexpr int kOutBytes = kEpiWarps * kOutBufs * kOutBufBytes;
     static constexpr int kBarOffset = kOutOffset + kOutBytes;
     static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
