@@ -64,8 +64,8 @@ struct SumShape {
 constexpr int SUM_SPARSE_MAX = 8;                                  // spans with at most this many boundaries read single prefixes from TMEM
 constexpr int SUM_DIRECT_LEN = 4;                                  // few-boundaries path: segments this short are summed from the inputs
 constexpr float SUM_CANCEL = 1.0f / 1024.0f;                       // general path: a sum this small against its prefixes is added up again
-constexpr int SUM_TBL = 128;                                       // boundaries a warp handles at a time (four per lane)
-constexpr int SUM_TBL_BYTES = 2 * (SPAN / ROW) * 4 + 16;           // per warp: marked elements and boundary counts of 128 rows, one counter
+constexpr int SUM_CHUNK = 128;                                     // boundaries a warp handles at a time (four per lane)
+constexpr int SUM_MARK_BYTES = 2 * (SPAN / ROW) * 4 + 16;          // per warp: marked elements and boundary counts of 128 rows, one counter
 
 // The fp32 products of SpMV, each stored as a pair of bf16 values (hi = bf16(z), lo = bf16(z - hi),
 // 4 bytes).  An ELEMENT of this path is one product; a row of 32 products is a 128-byte operand
@@ -231,8 +231,8 @@ struct SumCfg {
     static constexpr int kDumpBytes = PIECE * 4;                     // per epilogue warp
     static constexpr int kStageOffset = 4096;                        // after the constant operand
     static constexpr int kDumpOffset = kStageOffset + kStages * kXBytes;
-    static constexpr int kTblOffset = kDumpOffset + SumShape<G>::kEpiWarps * kDumpBytes;
-    static constexpr int kBarOffset = kTblOffset + SumShape<G>::kEpiWarps * SUM_TBL_BYTES;
+    static constexpr int kMarkOffset = kDumpOffset + SumShape<G>::kEpiWarps * kDumpBytes;
+    static constexpr int kBarOffset = kMarkOffset + SumShape<G>::kEpiWarps * SUM_MARK_BYTES;
     static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
     static_assert(kBBytes <= kStageOffset, "constant operand fits its slot");
     static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of one CTA");
@@ -242,7 +242,7 @@ struct SumParams {
     const int32_t* off;          // nseg + 1 offsets
     long long nseg;
     long long n;                 // number of values
-    int off_shift;               // boundaries are off[q] << off_shift (1 for the hi/lo pairs of SpMV)
+    int off_shift;               // boundaries are off[q] << off_shift (0 in every current call)
     void* out;                   // nseg results
     int num_tiles;
     const int32_t* span_q;       // 4 * num_tiles + 1: first q with (off[q] << shift) >= span start
@@ -572,7 +572,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         Acc* outp = static_cast<Acc*>(prm.out);
         // per row of the span: marked elements (bits), number of boundaries; boundaries at the span's first element
         uint8_t* dump = smem + Cfg::kDumpOffset + warp * Cfg::kDumpBytes;      // [32 rows][32] prefixes of a piece, swizzled by row
-        uint32_t* emask = reinterpret_cast<uint32_t*>(smem + Cfg::kTblOffset + warp * SUM_TBL_BYTES);
+        uint32_t* emask = reinterpret_cast<uint32_t*>(smem + Cfg::kMarkOffset + warp * SUM_MARK_BYTES);
         uint32_t* ecnt = emask + SPAN / ROW;
         uint32_t* nbase = ecnt + SPAN / ROW;
         const int sh = prm.off_shift;
@@ -650,16 +650,15 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             const int tile_n = tile_of(k + 1);
             if (tile_n >= 0) load_span_q(tile_n, q_next, qe_next);
             MMV_T_MARK(10)
-            // table entry t <-> boundary index cq + t; lane holds entries lane + 32 j.  Block 0 first: it
+            // lane holds boundaries cq + lane + 32 j (j < 4).  The first 32 first: they
             // decides between the path for spans with few boundaries and the general one.
-            long long bj[4] = {-1, -1, -1, -1}, sbj[4] = {-1, -1, -1, -1};
+            long long cb = -1, csb = -1;                       // my boundary among the first 32, and the one before it
             {
                 int32_t pr = __shfl_up_sync(0xffffffffu, raw[0], 1);
                 if (lane == 0) pr = rawp;
-                if (cq + lane < nq) bj[0] = cvt(raw[0]);
-                if (cq + lane >= 1) sbj[0] = cvt(pr);
+                if (cq + lane < nq) cb = cvt(raw[0]);
+                if (cq + lane >= 1) csb = cvt(pr);
             }
-            const long long cb = bj[0], csb = sbj[0];          // the first 32 boundaries, one per lane
             // the first 32 entries cover the span if they reach past its end (or the end of the offsets)
             const bool covers = __any_sync(0xffffffffu, (q + lane >= nq) || (cb > send));
             // number of boundaries with sbase <= bnd <= send (a prefix of the lanes)
@@ -671,14 +670,13 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             MMV_T_MARK(9)
             // very short segments that end in this span are summed from the inputs; the loads go out
             // now and return while the accumulators are awaited
-            bool isdir[1] = {false};
-            isdir[0] = cq + lane >= 1 && cq + lane < nq && sbj[0] >= 0 && bj[0] > sbj[0] && bj[0] - sbj[0] <= SUM_DIRECT_LEN &&
-                       bj[0] > sbase && bj[0] <= send && bj[0] <= prm.n;
+            bool is_direct = cq + lane >= 1 && cq + lane < nq && csb >= 0 && cb > csb && cb - csb <= SUM_DIRECT_LEN &&
+                             cb > sbase && cb <= send && cb <= prm.n;
             // (the general path needs only the one that reaches back across the span's first element)
-            if (!sparse && !(lane == 0 && sbj[0] < sbase)) isdir[0] = false;
+            if (!sparse && !(lane == 0 && csb < sbase)) is_direct = false;
             ValueWindow win0;
             win0.wide = false;
-            if (isdir[0]) window_load<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), prm.n, win0);
+            if (is_direct) window_load<P>(xg, csb, static_cast<int>(cb - csb), prm.n, win0);
             int xlen = 0;
             Acc xval = Acc(0);
             // ---- general path, first step: every boundary marks the element it ends behind.  emask[row] has
@@ -732,7 +730,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (!tcovers) {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const long long qi = cq + SUM_TBL + lane + 32 * j;
+                        const long long qi = cq + SUM_CHUNK + lane + 32 * j;
                         if (qi < nq) yraw[j] = prm.off[qi];
                     }
                 }
@@ -836,7 +834,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 publish(tail);
                 run = tail;
                 MMV_T_MARK(2)
-                const Acc dval = isdir[0] ? window_sum<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), win0) : Acc(0);
+                const Acc dval = is_direct ? window_sum<P>(xg, csb, static_cast<int>(cb - csb), win0) : Acc(0);
                 const Acc plocal = __shfl_up_sync(0xffffffffu, mylocal, 1);
                 const Acc prp = __shfl_up_sync(0xffffffffu, myrp, 1);
                 const int prow = __shfl_up_sync(0xffffffffu, myrow, 1);
@@ -871,7 +869,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 }
                 MMV_T_MARK(5)
             } else {
-                // ---- general path: row totals, pre-pass, table of direct sums ----
+                // ---- general path: row totals, pre-pass ----
 #pragma unroll
                 for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * ROW + (ROW - 1)));
                 tmem_ld_wait();
@@ -905,12 +903,12 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 //      empty segments (their zeros were written when the offsets were partitioned): the run is
                 //      jumped over with a 32-ary search and only counted. ----
                 if (!tcovers) {
-                    long long tp = cq + SUM_TBL;            // index of yraw's first boundary
+                    long long tp = cq + SUM_CHUNK;            // index of yraw's first boundary
                     while (true) {
                         int32_t zraw[4] = {kNoOffset, kNoOffset, kNoOffset, kNoOffset};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
-                            const long long qi = tp + SUM_TBL + lane + 32 * j;
+                            const long long qi = tp + SUM_CHUNK + lane + 32 * j;
                             if (qi < nq) zraw[j] = prm.off[qi];
                         }
                         const int32_t first = __shfl_sync(0xffffffffu, yraw[0], 0);
@@ -922,7 +920,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                             same &= yraw[j] == first;
                         }
                         if (__any_sync(0xffffffffu, beyond)) break;
-                        tp += SUM_TBL;
+                        tp += SUM_CHUNK;
 #pragma unroll
                         for (int j = 0; j < 4; ++j) yraw[j] = zraw[j];
                         if (__all_sync(0xffffffffu, same)) {
@@ -957,12 +955,12 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 long long obase = cq + static_cast<long long>(*nbase) - 1;     // output index of the span's first marked element
                 bool span_has_end = false;
                 // a very short segment that reaches back across the span's first element: summed from its values
-                const bool cross_done = xlen > 0 || __shfl_sync(0xffffffffu, isdir[0] ? 1 : 0, 0) != 0;
+                const bool cross_done = xlen > 0 || __shfl_sync(0xffffffffu, is_direct ? 1 : 0, 0) != 0;
                 if (xlen > 0) {
                     const Acc xsum = warp_sum<P>(xval);
                     if (lane == 0) outp[cq - 1] = xsum;
-                } else if (lane == 0 && isdir[0]) {
-                    outp[cq - 1] = window_sum<P>(xg, sbj[0], static_cast<int>(bj[0] - sbj[0]), win0);
+                } else if (lane == 0 && is_direct) {
+                    outp[cq - 1] = window_sum<P>(xg, csb, static_cast<int>(cb - csb), win0);
                 }
                 // number of elements open at the end of the previous piece's last row (64: too many to matter),
                 // and the largest prefix magnitude of that row
