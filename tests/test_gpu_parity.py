@@ -670,6 +670,22 @@ def test_bf16_values_beyond_the_fp16_range(mmv):
     assert np.isfinite(got).all()
 
 
+def test_spmv_tiny_rows_next_to_large_rows(mmv):
+    # rows of 1..8 non-zeros whose products are around 1e-3 between rows whose products are around 1e3: the bound
+    # is relative to each row's own sum of magnitudes, so a tiny row must not drown in its neighbours' prefixes
+    rng = np.random.default_rng(31)
+    rows, cols = 50000, 4096
+    lens = rng.integers(1, 9, rows)
+    rowptr = gen.offsets_from_lengths(lens)
+    nnz = int(rowptr[-1])
+    col = rng.integers(0, cols, nnz).astype(np.int32)
+    big = np.repeat(rng.integers(0, 2, rows).astype(bool), lens)
+    val = (rng.standard_normal(nnz) * np.where(big, 1000.0, 1e-3)).astype(np.float16)
+    x = (0.5 + rng.random(cols)).astype(np.float32)                  # magnitudes of order 1: the products keep the contrast
+    want, a = oracle.spmv_csr(rowptr, col, val, x)
+    assert_fp(spmv(mmv, rowptr, col, val, x), want, a, "tiny rows next to large rows")
+
+
 # ---------------------------------------------------------------------------
 # robustness
 # ---------------------------------------------------------------------------
