@@ -141,6 +141,19 @@ def seg_scan_excl_f16(x, f):
     return e, a
 
 
+def compress(x, f) -> np.ndarray:
+    """COMPRESS (Section 2): the elements x(i) with f(i) != 0, in order, copied unchanged."""
+    x = np.ascontiguousarray(x)
+    fb = _as(f, np.uint8)
+    assert fb.shape[0] == x.shape[0]
+    out = np.empty_like(x)
+    lib = _load()
+    lib.mmv_oracle_compress.restype = ctypes.c_int64
+    k = lib.mmv_oracle_compress(_p(x.view(np.uint8)), _p(fb), ctypes.c_int64(x.shape[0]), ctypes.c_int(x.dtype.itemsize),
+                                _p(out.view(np.uint8)))
+    return out[:k].copy()
+
+
 def bf16_to_double(bits) -> np.ndarray:
     """Exact decode of bfloat16 bit patterns (uint16) to float64."""
     hb = _as(bits, np.uint16)

@@ -221,6 +221,22 @@ void mmv_oracle_seg_sum_csr_i8(const int8_t *x, const int32_t *off, int64_t nseg
 }
 
 /* ------------------------------------------------------------------------ */
+/* COMPRESS (Section 2): keep x(i) where f(i) != 0, in order.  Elements are   */
+/* copied as they are (elem_bytes each); returns the number kept.             */
+/* ------------------------------------------------------------------------ */
+int64_t mmv_oracle_compress(const uint8_t *x, const uint8_t *f, int64_t n, int elem_bytes, uint8_t *out)
+{
+    int64_t k = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (f[i] != 0) {
+            for (int b = 0; b < elem_bytes; ++b) out[k * elem_bytes + b] = x[i * elem_bytes + b];
+            ++k;
+        }
+    }
+    return k;
+}
+
+/* ------------------------------------------------------------------------ */
 /* bfloat16 values: decoded exactly to double, then the same definitions on   */
 /* double inputs (Eq. (1), its exclusive companion, the two segmented sums).  */
 /* ------------------------------------------------------------------------ */

@@ -532,3 +532,22 @@ def test_bf16_definitions_against_brute_force_and_the_fp16_functions():
 def oracle_offsets_of_flags(f):
     starts = [0] + [i for i in range(1, len(f)) if f[i]]
     return np.asarray(starts + [len(f)], np.int32)
+
+
+# --------------------------------------------------------------------------
+# COMPRESS (Section 2)
+# --------------------------------------------------------------------------
+def test_compress_of_the_worked_example_and_against_a_loop():
+    g = load_golden("sec2_worked_example.txt")
+    x, f = g["x"], g["f"]
+    assert oracle.compress(np.asarray(x, np.int8), u8(f)).tolist() == g["compress_x_f"]
+    assert oracle.compress(f16(x), u8(f)).tolist() == g["compress_x_f"]
+    rng = np.random.default_rng(29)
+    for trial in range(50):
+        n = int(rng.integers(0, 200))
+        f = (rng.random(n) < rng.choice([0.0, 0.1, 0.6, 1.0])).astype(np.uint8) * rng.integers(1, 256, n).astype(np.uint8)
+        for x in (rng.integers(-128, 128, n).astype(np.int8), rng.standard_normal(n).astype(np.float16),
+                  rng.integers(0, 65536, n).astype(np.uint16)):
+            want = [x[i] for i in range(n) if f[i]]
+            got = oracle.compress(x, f)
+            assert got.dtype == x.dtype and got.tolist() == [v.item() for v in want]
