@@ -595,7 +595,21 @@ def run_ours(args):
             sweep.append({"case": f"bf16 values, {args.case}", "ms": cms, "gelem_s": n / cms / 1e6,
                           "gb_s": 7 * n / cms / 1e6, "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
                           "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
-            del fd, xb
+            # COMPRESS of the headline values under the headline flags (flags are read twice: count, scatter)
+            outc = torch.empty(n, dtype=torch.float16, device="cuda")
+            kc = torch.zeros(1, dtype=torch.int64, device="cuda")
+            wsc = mmv.alloc_workspace(mmv.OP_COMPRESS, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+            fn = lambda: mmv.compress(xd, fd, out=outc, count=kc, workspace=wsc)  # noqa: E731
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            cms = event_time_ms(torch, fn, min(args.steps, 10))
+            kept = int(kc.item())
+            cbytes = n + 4 * kept
+            sweep.append({"case": f"COMPRESS, {args.case} ({kept} kept)", "ms": cms, "gelem_s": n / cms / 1e6,
+                          "gb_s": cbytes / cms / 1e6, "frac_of_measured_peak": cbytes / cms / 1e6 / peak,
+                          "frac_of_8tbs": cbytes / cms / 1e6 / NOMINAL_HBM_GBS})
+            del fd, xb, outc, wsc
             line["configs"] = cfgs
             line["c5_density_sweep"] = sweep
         print(json.dumps(line))

@@ -78,7 +78,7 @@ typedef enum {
 
 typedef enum { MMV_F16_TO_F32 = 0, MMV_I8_TO_I32 = 1, MMV_BF16_TO_F32 = 2 } mmv_dtype;
 typedef enum { MMV_SEG_FLAGS_U8 = 0, MMV_SEG_OFFSETS_I32 = 1 } mmv_segfmt;
-typedef enum { MMV_OP_SEG_SCAN = 0, MMV_OP_SEG_SUM = 1, MMV_OP_SPMV_CSR = 2 } mmv_op;
+typedef enum { MMV_OP_SEG_SCAN = 0, MMV_OP_SEG_SUM = 1, MMV_OP_SPMV_CSR = 2, MMV_OP_COMPRESS = 3 } mmv_op;
 
 /*
  * Bytes of device workspace the given call needs (a pure host computation).
@@ -131,6 +131,21 @@ mmv_status mmv_seg_scan_exclusive(const void *x, const void *seg, mmv_segfmt sf,
 mmv_status mmv_seg_sum(const void *x, const void *seg, mmv_segfmt sf, int64_t n, int64_t nseg,
                        mmv_dtype dt, void *out, int64_t *d_num_segments,
                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * COMPRESS (Section 2): the values x[i] with flag[i] != 0, in order, copied
+ * unchanged to out[0 .. K-1] (same element type as x: 2 bytes for
+ * MMV_F16_TO_F32 and MMV_BF16_TO_F32, 1 byte for MMV_I8_TO_I32); nothing
+ * beyond out[K-1] is touched.  Unlike the segment encodings above, flag[0] is
+ * an ordinary flag here.  K is written to *d_count (device pointer, int64,
+ * 8-byte aligned) when it is not NULL.  out needs room for n elements in the
+ * worst case; x, flags and out 16-byte aligned; n < 2^31.  Workspace:
+ * mmv_workspace_bytes(MMV_OP_COMPRESS, dt, MMV_SEG_FLAGS_U8, n, 0).  Three
+ * streaming kernels (counts per 16384-flag chunk, one-block scan, scatter);
+ * asynchronous on the stream like the other calls.
+ */
+mmv_status mmv_compress(const void *x, const void *flags, int64_t n, mmv_dtype dt, void *out, int64_t *d_count,
+                        void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * CSR sparse matrix times dense vector built on the segmented sum

@@ -20,13 +20,13 @@ LIB_PATH = _PKG / "libmmv.so"
 MMV_OK = 0
 F16_TO_F32, I8_TO_I32, BF16_TO_F32 = 0, 1, 2
 SEG_FLAGS_U8, SEG_OFFSETS_I32 = 0, 1
-OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR = 0, 1, 2
+OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR, OP_COMPRESS = 0, 1, 2, 3
 
 EXPORTS = (
     "mmv_workspace_bytes", "mmv_seg_scan", "mmv_seg_sum", "mmv_spmv_csr",
     "mmv_last_async_status", "mmv_status_string", "mmv_kernel_launch_count", "mmv_debug_configure",
     "mmv_seg_scan_static", "mmv_seg_scan_static_last_status", "mmv_debug_force_sum_groups",
-    "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes", "mmv_seg_scan_exclusive",
+    "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes", "mmv_seg_scan_exclusive", "mmv_compress",
 )
 STATIC_SCAN_MAX_N = 1 << 28
 
@@ -50,6 +50,8 @@ def _load() -> ctypes.CDLL:
     lib.mmv_seg_scan.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, sz, vp]
     lib.mmv_seg_scan_exclusive.restype = ci
     lib.mmv_seg_scan_exclusive.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, sz, vp]
+    lib.mmv_compress.restype = ci
+    lib.mmv_compress.argtypes = [vp, vp, i64, ci, vp, vp, vp, sz, vp]
     lib.mmv_seg_sum.restype = ci
     lib.mmv_seg_sum.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, vp, sz, vp]
     lib.mmv_spmv_csr.restype = ci
@@ -158,6 +160,27 @@ def seg_scan(x: torch.Tensor, seg: torch.Tensor | None, out: torch.Tensor | None
     if rc != MMV_OK:
         raise MmvError(rc, "mmv_seg_scan_exclusive" if exclusive else "mmv_seg_scan")
     return out
+
+
+def compress(x: torch.Tensor, flags: torch.Tensor, out: torch.Tensor | None = None, count: torch.Tensor | None = None,
+             workspace: torch.Tensor | None = None, stream=None):
+    """mmv_compress: COMPRESS of Section 2 -- the values x[i] with flags[i] != 0, in order.  Returns (out, count):
+    out has room for n values of x's type, count is an int64 device tensor holding K; out[:K] is the result."""
+    _check_cuda(x, flags, out, workspace)
+    if flags.dtype != torch.uint8:
+        raise TypeError("flags must be uint8")
+    dt, n = _dtype_code(x), x.numel()
+    if out is None:
+        out = torch.empty(n, dtype=x.dtype, device=x.device)
+    if count is None:
+        count = torch.zeros(1, dtype=torch.int64, device=x.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_COMPRESS, dt, SEG_FLAGS_U8, n, 0, x.device)
+    rc = _lib.mmv_compress(_ptr(x), _ptr(flags), n, dt, _ptr(out), _ptr(count), _ptr(workspace), workspace.numel(),
+                           _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_compress")
+    return out, count
 
 
 def seg_scan_static(x: torch.Tensor, flags: torch.Tensor, out: torch.Tensor, stream=None) -> torch.Tensor:

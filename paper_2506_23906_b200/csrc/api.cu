@@ -167,12 +167,12 @@ WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     p.tileq_bytes = (op != MMV_OP_SEG_SCAN) ? round_up(static_cast<size_t>(tiles * SPANS_PER_TILE + 1) * sizeof(int32_t), 256) : 0;
     p.prod_off = p.tileq_off + p.tileq_bytes;
     p.prod_bytes = (op == MMV_OP_SPMV_CSR) ? round_up(static_cast<size_t>(n) * 4, 256) : 0;
-    const bool flagsum = op == MMV_OP_SEG_SUM && sf == MMV_SEG_FLAGS_U8;
+    const bool flagsum = (op == MMV_OP_SEG_SUM && sf == MMV_SEG_FLAGS_U8) || op == MMV_OP_COMPRESS;
     const long long nchunks = (n + CMP_CHUNK - 1) / CMP_CHUNK;
     p.cmp_off = p.prod_off + p.prod_bytes;
     p.cmp_bytes = flagsum ? round_up(static_cast<size_t>(2 * nchunks + 8) * sizeof(int32_t) + 16, 256) : 0;
     p.off_off = p.cmp_off + p.cmp_bytes;
-    p.off_bytes = flagsum ? round_up(static_cast<size_t>(n + 1) * sizeof(int32_t), 256) : 0;
+    p.off_bytes = (flagsum && op != MMV_OP_COMPRESS) ? round_up(static_cast<size_t>(n + 1) * sizeof(int32_t), 256) : 0;
     p.total = p.off_off + p.off_bytes;
     return p;
 }
@@ -315,7 +315,7 @@ extern "C" {
 
 size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, int64_t nseg) {
     if (n < 0 || nseg < 0) return 0;
-    if (op != MMV_OP_SEG_SCAN && op != MMV_OP_SEG_SUM && op != MMV_OP_SPMV_CSR) return 0;
+    if (op != MMV_OP_SEG_SCAN && op != MMV_OP_SEG_SUM && op != MMV_OP_SPMV_CSR && op != MMV_OP_COMPRESS) return 0;
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return 0;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return 0;
     return plan_workspace(op, sf, n).total;
@@ -610,6 +610,45 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
     if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, nseg, 0, out, ws, plan, dev, st);
     if (dt == MMV_BF16_TO_F32) return launch_seg_sum<BF16ValPath>(x, n, off, nseg, 0, out, ws, plan, dev, st);
     return launch_seg_sum<I8Path>(x, n, off, nseg, 0, out, ws, plan, dev, st);
+}
+
+mmv_status mmv_compress(const void* x, const void* flags, int64_t n, mmv_dtype dt, void* out, int64_t* d_count,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (n < 0 || n >= (1ll << 31)) return MMV_ERR_INVALID_ARG;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return MMV_ERR_INVALID_ARG;
+    if (d_count && (reinterpret_cast<uintptr_t>(d_count) & 7u)) return MMV_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (n == 0) {
+        if (d_count && cudaMemsetAsync(d_count, 0, sizeof(int64_t), st) != cudaSuccess) return MMV_ERR_CUDA;
+        return MMV_OK;
+    }
+    if (!x || !flags || !out || !workspace) return MMV_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(flags) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return MMV_ERR_INVALID_ARG;
+    const WorkspacePlan plan = plan_workspace(MMV_OP_COMPRESS, MMV_SEG_FLAGS_U8, n);
+    if (workspace_bytes < plan.total) return MMV_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo* dev = device_info();
+    if (!dev) return MMV_ERR_CUDA;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (cudaMemsetAsync(ws, 0, sizeof(WorkspaceHeader), st) != cudaSuccess) return MMV_ERR_CUDA;
+    const long long nchunks = (n + CMP_CHUNK - 1) / CMP_CHUNK;
+    long long* count_dev = reinterpret_cast<long long*>(ws + plan.cmp_off);
+    int32_t* chunk_count = reinterpret_cast<int32_t*>(ws + plan.cmp_off + 16);
+    int32_t* chunk_base = chunk_count + ((nchunks + 3) & ~3ll);
+    const uint8_t* f = static_cast<const uint8_t*>(flags);
+    const long long cap = static_cast<long long>(dev->sm_count) * 8;
+    const unsigned blocks = static_cast<unsigned>(nchunks < cap ? nchunks : cap);
+    flag_count_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_count, false);
+    chunk_scan_kernel<<<1, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, count_dev, reinterpret_cast<long long*>(d_count),
+                                          nullptr, n);
+    if (dt == MMV_I8_TO_I32)
+        compress_values_kernel<uint8_t><<<blocks, CMP_THREADS, 0, st>>>(static_cast<const uint8_t*>(x), f, n, nchunks, chunk_base,
+                                                                       static_cast<uint8_t*>(out));
+    else
+        compress_values_kernel<unsigned short><<<blocks, CMP_THREADS, 0, st>>>(static_cast<const unsigned short*>(x), f, n, nchunks,
+                                                                              chunk_base, static_cast<unsigned short*>(out));
+    g_launches += 3;
+    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
 
 mmv_status mmv_spmv_csr(const int32_t* rowptr, const int32_t* col, const void* val_f16, const float* x, float* y,

@@ -19,8 +19,10 @@ __device__ __forceinline__ int nonzero_bytes(uint32_t w) {
     return __popc((((w & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w) & 0x80808080u);
 }
 
-// The 64 flag bytes of thread t of chunk c as 16 words (zero past n; byte 0 of the vector forced to 1).
-__device__ __forceinline__ void load_thread_flags(const uint8_t* __restrict__ f, long long n, long long base, uint32_t (&w)[16]) {
+// The 64 flag bytes of thread t of chunk c as 16 words (zero past n; with first_is_start byte 0 of the
+// vector is forced to 1: element 0 opens a segment whatever its flag says).
+__device__ __forceinline__ void load_thread_flags(const uint8_t* __restrict__ f, long long n, long long base, uint32_t (&w)[16],
+                                                  bool first_is_start = true) {
 #pragma unroll
     for (int v = 0; v < 4; ++v) {
         const long long p = base + 16 * v;
@@ -37,7 +39,7 @@ __device__ __forceinline__ void load_thread_flags(const uint8_t* __restrict__ f,
         w[4 * v + 2] = q.z;
         w[4 * v + 3] = q.w;
     }
-    if (base == 0) w[0] |= 1u;          // element 0 starts the first segment
+    if (base == 0 && first_is_start) w[0] |= 1u;          // element 0 starts the first segment
 }
 
 // Exclusive scan of one int per thread over the block; returns this thread's offset, *total = block sum.
@@ -69,11 +71,12 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* total, int* warp
 
 // chunk_count[c] = number of segment starts among the flags of chunk c.
 __global__ void __launch_bounds__(CMP_THREADS)
-flag_count_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks, int32_t* __restrict__ chunk_count) {
+flag_count_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks, int32_t* __restrict__ chunk_count,
+                  bool first_is_start = true) {
     __shared__ int warp_sums[32];
     for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
         uint32_t w[16];
-        load_thread_flags(f, n, c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD, w);
+        load_thread_flags(f, n, c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD, w, first_is_start);
         int cnt = 0;
 #pragma unroll
         for (int i = 0; i < 16; ++i) cnt += nonzero_bytes(w[i]);
@@ -122,7 +125,7 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
     if (threadIdx.x == 0) {
         *nseg_dev = total;
         if (d_num_segments) *d_num_segments = total;
-        off[total] = static_cast<int32_t>(n);
+        if (off) off[total] = static_cast<int32_t>(n);
     }
 }
 
@@ -160,6 +163,36 @@ flag_scatter_kernel(const uint8_t* __restrict__ f, long long n, long long nchunk
                 while (m) {
                     const int b = (__ffs(m) - 1) >> 3;
                     off[slot++] = static_cast<int32_t>(base + 4 * i + b);
+                    m &= m - 1;
+                }
+            }
+        }
+    }
+}
+
+// COMPRESS of the values themselves (Section 2): out[chunk_base[c] + j] = the value at the j-th non-zero flag
+// of chunk c.  T is the element as stored (2 bytes for fp16 / bf16, 1 byte for int8); nothing is converted.
+template <typename T>
+__global__ void __launch_bounds__(CMP_THREADS)
+compress_values_kernel(const T* __restrict__ x, const uint8_t* __restrict__ f, long long n, long long nchunks,
+                       const int32_t* __restrict__ chunk_base, T* __restrict__ out) {
+    __shared__ int warp_sums[32];
+    for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
+        const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
+        uint32_t w[16];
+        load_thread_flags(f, n, base, w, false);
+        int cnt = 0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) cnt += nonzero_bytes(w[i]);
+        int total;
+        long long slot = chunk_base[c] + block_exclusive_scan(cnt, &total, warp_sums);
+        if (cnt) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                uint32_t m = (((w[i] & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w[i]) & 0x80808080u;
+                while (m) {
+                    const int b = (__ffs(m) - 1) >> 3;
+                    out[slot++] = x[base + 4 * i + b];
                     m &= m - 1;
                 }
             }

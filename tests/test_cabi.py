@@ -89,5 +89,11 @@ def test_argument_errors_are_synchronous(lib):
     assert lib.mmv_seg_scan_host(16, 16, 8, 2, 16, 16384, 256, 1 << 30, None) == 1    # bf16 values: not for this entry point
     assert lib.mmv_seg_scan_host_scratch_bytes(0, 1000) == 0
     assert lib.mmv_seg_scan_host_scratch_bytes(0, 16384) >= 2 * 16384 * 7
+    lib.mmv_compress.argtypes = [vp, vp, i64, ci, vp, vp, vp, sz, vp]
+    assert lib.mmv_compress(None, None, 0, 0, None, None, None, 0, None) == 0           # nothing to do
+    assert lib.mmv_compress(None, None, -1, 0, None, None, None, 0, None) == 1
+    assert lib.mmv_compress(16, 16, 8, 0, 16, None, 256, 16, None) == 3                 # workspace too small
+    assert lib.mmv_compress(16, 16, 8, 0, 16, 12, 256, 1 << 20, None) == 1              # misaligned counter
+    assert lib.mmv_workspace_bytes(3, 0, 0, 1 << 20, 0) >= 512
     assert lib.mmv_spmv_csr(None, None, None, None, None, -1, 1, 1, None, 0, None) == 1
     assert lib.mmv_spmv_csr(None, None, None, None, None, 0, 1, 0, None, 0, None) == 0

@@ -501,6 +501,35 @@ def test_seg_sum_row_length_mixes(mmv, kind):
 
 
 # ---------------------------------------------------------------------------
+# COMPRESS (Section 2)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("n", [1, 63, 64, 65, TILE - 1, TILE, TILE + 1, 5 * TILE + 333])
+@pytest.mark.parametrize("p", [0.0, 0.01, 0.5, 1.0])
+def test_compress(mmv, n, p):
+    rng = np.random.default_rng(n + int(100 * p))
+    f = ((rng.random(n) < p) * rng.integers(1, 256, n)).astype(np.uint8)        # any non-zero byte keeps the element
+    for x in (rng.integers(-128, 128, n).astype(np.int8), rng.standard_normal(n).astype(np.float16)):
+        want = oracle.compress(x, f)
+        guard = torch.full((n + 8,), 77, dtype=torch.from_numpy(x[:1]).dtype, device="cuda")
+        out, count = mmv.compress(dev(x), dev(f), out=guard[:n])
+        k = int(count.item())
+        got = guard.cpu().numpy()
+        assert k == want.shape[0]
+        assert np.array_equal(got[:k].view(np.uint8), want.view(np.uint8))          # bit for bit
+        assert (got[max(k, 0):] == 77).all() if k == n else (got[n:] == 77).all()   # nothing past the end
+    xb = gen.bf16_normal(3, n)
+    out, count = mmv.compress(dev_bf16(xb), dev(f))
+    k = int(count.item())
+    assert np.array_equal(out[:k].view(torch.int16).cpu().numpy().view(np.uint16), oracle.compress(xb, f))
+
+
+def test_compress_of_the_paper_example(mmv):
+    g = __import__("conftest").load_golden("sec2_worked_example.txt")
+    out, count = mmv.compress(dev(np.asarray(g["x"], np.int8)), dev(np.asarray(g["f"], np.uint8)))
+    assert out[:int(count.item())].cpu().tolist() == g["compress_x_f"]
+
+
+# ---------------------------------------------------------------------------
 # randomised shapes
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("seed", [11, 12, 13])
