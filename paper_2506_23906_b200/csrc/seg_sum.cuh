@@ -687,16 +687,16 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             bool tcovers = covers;
             int32_t yraw[4] = {kNoOffset, kNoOffset, kNoOffset, kNoOffset};
             auto mark = [&](int32_t braw) -> bool {          // returns true if the boundary lies behind the span
-                const int rel = static_cast<int>(static_cast<uint32_t>(braw) - sb32);
-                if (braw >= 0) {
-                    if (rel == 0) {
-                        atomicAdd(nbase, 1u);
-                    } else if (rel > 0 && rel <= SPAN) {
-                        atomicOr(&emask[(rel - 1) >> 5], 1u << ((rel - 1) & 31));
-                        atomicAdd(&ecnt[(rel - 1) >> 5], 1u);
-                    }
+                // element the boundary ends behind, relative to the span (one unsigned test covers 1 <= rel <= SPAN;
+                // a negative offset wraps to a huge value and marks nothing)
+                const uint32_t e = static_cast<uint32_t>(braw) - sb32 - 1u;
+                if (e < static_cast<uint32_t>(SPAN)) {
+                    atomicOr(&emask[e >> 5], 1u << (e & 31u));
+                    atomicAdd(&ecnt[e >> 5], 1u);
+                } else if (e == 0xffffffffu && braw >= 0) {
+                    atomicAdd(nbase, 1u);
                 }
-                return rel > SPAN;
+                return static_cast<int>(e) >= SPAN;
             };
             if (!sparse) {
 #pragma unroll
@@ -1016,29 +1016,39 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     int cprev = -1, nend = 0, first_len = 0;
                     long long first_oi = -1;
                     uint32_t mm = m;
+                    const uint8_t* drow = dump + lane * 128;       // my row of the prefixes (16-byte groups swizzled by row)
+                    const int lx = static_cast<int>(lane & 7);
+                    auto prefix_at = [&](int c) -> Acc {
+                        return *reinterpret_cast<const Acc*>(drow + ((((c >> 2) ^ lx) << 4) | ((c & 3) << 2)));
+                    };
+                    auto index_of = [&](int c, int k) -> long long {          // output index of my k-th sum, which ends behind column c
+                        if (!dirty) return orow + k;
+                        const int32_t bpos = static_cast<int32_t>(rowpos + c + 1);
+                        while (bp + 1 < bend && prm.off[bp] < bpos) ++bp;
+                        return (bp++) - 1;
+                    };
+                    if (mm) {                                      // the row's first marked element: finished below
+                        const int c = __ffs(mm) - 1;
+                        mm &= mm - 1;
+                        first_pref = pv = prefix_at(c);
+                        first_len = c + 1;
+                        first_oi = index_of(c, 0);
+                        cprev = c;
+                        nend = 1;
+                    }
+                    float cancel_below = 0.f;
+                    if constexpr (P::kIsFloat) cancel_below = scale * SUM_CANCEL;
+                    Acc* po = outp + orow;                          // (rows without empty segments: sums at consecutive indices)
                     while (mm) {                                   // (lanes differ in the number of marked elements)
                         const int c = __ffs(mm) - 1;
                         mm &= mm - 1;
-                        const Acc pc = *reinterpret_cast<const Acc*>(dump + lane * 128 + ((((c >> 2) ^ (lane & 7)) << 4) | ((c & 3) << 2)));
-                        long long oi = orow + nend;
-                        if (dirty) {
-                            const int32_t bpos = static_cast<int32_t>(rowpos + c + 1);
-                            while (bp + 1 < bend && prm.off[bp] < bpos) ++bp;
-                            oi = bp - 1;
-                            ++bp;
+                        const Acc pc = prefix_at(c);
+                        Acc val = P::sub(pc, pv);
+                        if constexpr (P::kIsFloat) {
+                            if (fabsf(val) < cancel_below) val = direct_sum<P>(xg, rowpos + cprev + 1, rowpos + c + 1);
                         }
-                        if (nend == 0) {
-                            first_pref = pc;
-                            first_len = c + 1;
-                            first_oi = oi;
-                        } else {
-                            Acc val = P::sub(pc, pv);
-                            if constexpr (P::kIsFloat) {
-                                if (fabsf(val) < scale * SUM_CANCEL)
-                                    val = direct_sum<P>(xg, rowpos + cprev + 1, rowpos + c + 1);
-                            }
-                            outp[oi] = val;
-                        }
+                        if (dirty) outp[index_of(c, nend)] = val;
+                        else po[nend] = val;
                         pv = pc;
                         cprev = c;
                         ++nend;
