@@ -1000,8 +1000,14 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                             *reinterpret_cast<uint4*>(dump + lane * 128 + ((c4 ^ (lane & 7)) << 4)) =
                                 make_uint4(r[4 * c4], r[4 * c4 + 1], r[4 * c4 + 2], r[4 * c4 + 3]);
                         if constexpr (P::kIsFloat) {
+                            // (two chains of three-operand maxima)
+                            float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) scale = fmaxf(scale, fabsf(__uint_as_float(r[c])));
+                            for (int c = 0; c < 32; c += 4) {
+                                s0 = fmaxf(fmaxf(s0, fabsf(__uint_as_float(r[c]))), fabsf(__uint_as_float(r[c + 1])));
+                                s1 = fmaxf(fmaxf(s1, fabsf(__uint_as_float(r[c + 2]))), fabsf(__uint_as_float(r[c + 3])));
+                            }
+                            scale = fmaxf(s0, s1);
                         }
                     }
                     __syncwarp();
@@ -1056,12 +1062,14 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     // what is open at the end of each row: the part behind its last marked element, or all of it
                     const bool has_end = nend > 0;
                     Acc v = has_end ? P::sub(toti, pv) : toti;
+                    // rows back to (not including) the nearest one at or before mine that has a marked element: the
+                    // open part reaches that far back
+                    const uint32_t heads = hb & (0xffffffffu >> (31 - lane));
+                    const int reach = heads ? static_cast<int>(lane) - (31 - __clz(heads)) : static_cast<int>(lane);
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
                         const Acc t = __shfl_up_sync(0xffffffffu, v, o);
-                        // rows lane - o + 1 .. lane without a marked element: the open part reaches further back
-                        const bool clear = static_cast<int>(lane) >= o && ((hb >> (lane - o + 1)) & ((1u << o) - 1u)) == 0u;
-                        if (clear) v = P::add(t, v);
+                        if (o <= reach) v = P::add(t, v);
                     }
                     // open sum at the START of my row: the inclusive value of the row before (plus the piece's carry
                     // if no row before me has a marked element)
