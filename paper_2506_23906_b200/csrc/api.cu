@@ -256,12 +256,29 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     const int grid = tiles < dev->sm_count ? tiles : dev->sm_count;
     // Twelve epilogue warps (three warpgroups) measured faster than eight at every segment density;
     // the shape with two warpgroups stays available for tests and measurements.
-    if (g_force_groups.load() != 2)
-        seg_sum_kernel<P, 3><<<grid, SumShape<3>::kThreads, SumCfg<P, 3>::kSmemBytes, st>>>(tmap, values, prm);
-    else
-        seg_sum_kernel<P, 2><<<grid, SumShape<2>::kThreads, SumCfg<P, 2>::kSmemBytes, st>>>(tmap, values, prm);
+    // With the partition kernel right in front, the tiled kernel is launched with programmatic
+    // serialisation: its set-up (barriers, tensor memory, constant operand) overlaps the partition's end.
+    const bool overlap = !have_partition;
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    cudaError_t err;
+    if (g_force_groups.load() != 2) {
+        cfg.blockDim = dim3(SumShape<3>::kThreads);
+        cfg.dynamicSmemBytes = SumCfg<P, 3>::kSmemBytes;
+        err = cudaLaunchKernelEx(&cfg, seg_sum_kernel<P, 3>, tmap, values, prm);
+    } else {
+        cfg.blockDim = dim3(SumShape<2>::kThreads);
+        cfg.dynamicSmemBytes = SumCfg<P, 2>::kSmemBytes;
+        err = cudaLaunchKernelEx(&cfg, seg_sum_kernel<P, 2>, tmap, values, prm);
+    }
     ++g_launches;
-    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? MMV_OK : MMV_ERR_CUDA;
 }
 
 // f[off[r]] = 1 for every non-empty segment r (scratch flags of the offset-encoded scan).

@@ -14,6 +14,12 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start
+// while its predecessor in the stream still runs; it must wait here before it touches what the predecessor
+// (or anything before it) writes.  Without the attribute both instructions do nothing.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // 16-byte asynchronous copy global -> shared (the ragged last tile, which TMA's box cannot describe:
 // all of a lane's copies are in flight together instead of one load latency after the other)
 __device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {

@@ -300,6 +300,7 @@ __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long l
                                          uint32_t* __restrict__ out) {
     const int lane = threadIdx.x & 31;
     const long long stride = static_cast<long long>(VEC) * gridDim.x * blockDim.x;
+    griddep_launch_dependents();       // the tiled kernel may set itself up meanwhile (it waits before it reads)
     const int n32 = static_cast<int>(n < 0x7fffffffll ? n : 0x7fffffffll);
     const int last_span = static_cast<int>(num_spans);
     static_assert(SPAN == 4096, "span index = position >> 12");
@@ -457,6 +458,9 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Everything above (barriers, tensor memory, the constant operand) touched nothing a predecessor in the
+    // stream writes; from here on the kernel reads the span partition, the status words and the offsets.
+    griddep_wait();
 
     if (warp == Shape::kProducerWarp) {
         // =========================== producer ===========================
