@@ -141,6 +141,25 @@ def seg_scan_excl_f16(x, f):
     return e, a
 
 
+def seg_scan_minmax_f16(x, f, want_min: bool = False) -> np.ndarray:
+    """Segmented running maximum (or minimum) of fp16 values, float64 (exact: no arithmetic is involved)."""
+    xb, fb = _as_f16_bits(x), _as(f, np.uint8)
+    n = xb.shape[0]
+    assert fb.shape[0] == n
+    z = np.empty(n, np.float64)
+    _load().mmv_oracle_seg_scan_minmax_f16(_p(xb), _p(fb), ctypes.c_int64(n), ctypes.c_int(int(want_min)), _p(z))
+    return z
+
+
+def seg_scan_minmax_i8(x, f, want_min: bool = False) -> np.ndarray:
+    xb, fb = _as(x, np.int8), _as(f, np.uint8)
+    n = xb.shape[0]
+    assert fb.shape[0] == n
+    z = np.empty(n, np.int32)
+    _load().mmv_oracle_seg_scan_minmax_i8(_p(xb), _p(fb), ctypes.c_int64(n), ctypes.c_int(int(want_min)), _p(z))
+    return z
+
+
 def compress(x, f) -> np.ndarray:
     """COMPRESS (Section 2): the elements x(i) with f(i) != 0, in order, copied unchanged."""
     x = np.ascontiguousarray(x)

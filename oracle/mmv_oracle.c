@@ -221,6 +221,34 @@ void mmv_oracle_seg_sum_csr_i8(const int8_t *x, const int32_t *off, int64_t nseg
 }
 
 /* ------------------------------------------------------------------------ */
+/* Segmented running maximum / minimum: Eq. (1) with max or min in place of   */
+/* the addition (an operator without an inverse: Section 2 notes that the     */
+/* speculate-and-revert method needs a group, so this is the plain recurrence).*/
+/* want_min = 0: maximum, 1: minimum.                                         */
+/* ------------------------------------------------------------------------ */
+void mmv_oracle_seg_scan_minmax_f16(const uint16_t *x, const uint8_t *f, int64_t n, int want_min, double *z)
+{
+    double zp = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        double xi = half_bits_to_double(x[i]);
+        if (i == 0 || f[i] != 0) zp = xi;
+        else if (want_min ? (xi < zp) : (xi > zp)) zp = xi;
+        z[i] = zp;
+    }
+}
+
+void mmv_oracle_seg_scan_minmax_i8(const int8_t *x, const uint8_t *f, int64_t n, int want_min, int32_t *z)
+{
+    int32_t zp = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int32_t xi = (int32_t)x[i];
+        if (i == 0 || f[i] != 0) zp = xi;
+        else if (want_min ? (xi < zp) : (xi > zp)) zp = xi;
+        z[i] = zp;
+    }
+}
+
+/* ------------------------------------------------------------------------ */
 /* COMPRESS (Section 2): keep x(i) where f(i) != 0, in order.  Elements are   */
 /* copied as they are (elem_bytes each); returns the number kept.             */
 /* ------------------------------------------------------------------------ */

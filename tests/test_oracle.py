@@ -551,3 +551,37 @@ def test_compress_of_the_worked_example_and_against_a_loop():
             want = [x[i] for i in range(n) if f[i]]
             got = oracle.compress(x, f)
             assert got.dtype == x.dtype and got.tolist() == [v.item() for v in want]
+
+
+# --------------------------------------------------------------------------
+# segmented running maximum / minimum
+# --------------------------------------------------------------------------
+def test_segmented_running_max_and_min():
+    g = load_golden("sec2_worked_example.txt")
+    x, f = g["x"], g["f"]                       # x = (2,2,3,3,1,3,1,2), f = (1,0,1,0,0,1,0,0)
+    assert oracle.seg_scan_minmax_i8(np.asarray(x, np.int8), u8(f)).tolist() == [2, 2, 3, 3, 3, 3, 3, 3]
+    assert oracle.seg_scan_minmax_i8(np.asarray(x, np.int8), u8(f), want_min=True).tolist() == [2, 2, 3, 3, 1, 3, 1, 1]
+    assert oracle.seg_scan_minmax_f16(f16(x), u8(f)).tolist() == [2, 2, 3, 3, 3, 3, 3, 3]
+    rng = np.random.default_rng(37)
+    for trial in range(60):
+        n = int(rng.integers(1, 90))
+        f = (rng.random(n) < rng.choice([0.0, 0.1, 0.5, 1.0])).astype(np.uint8)
+        xi = rng.integers(-128, 128, n).astype(np.int8)
+        xf = rng.standard_normal(n).astype(np.float16)
+        for want_min in (False, True):
+            pick = min if want_min else max
+            def brute(v):
+                out = []
+                for i in range(n):
+                    s = i
+                    while s > 0 and not f[s]:
+                        s -= 1
+                    out.append(pick(v[s:i + 1]))
+                return out
+            assert oracle.seg_scan_minmax_i8(xi, f, want_min).tolist() == brute(xi.astype(int).tolist())
+            assert oracle.seg_scan_minmax_f16(xf, f, want_min).tolist() == brute(xf.astype(np.float64).tolist())
+        # duality, and the library routine when there is no flag
+        assert np.array_equal(oracle.seg_scan_minmax_f16(xf, f, True), -oracle.seg_scan_minmax_f16(-xf, f, False))
+        zero = np.zeros(n, np.uint8)
+        assert np.array_equal(oracle.seg_scan_minmax_i8(xi, zero), np.maximum.accumulate(xi.astype(np.int32)))
+        assert np.array_equal(oracle.seg_scan_minmax_f16(xf, zero, True), np.minimum.accumulate(xf.astype(np.float64)))
