@@ -595,6 +595,19 @@ def run_ours(args):
             sweep.append({"case": f"bf16 values, {args.case}", "ms": cms, "gelem_s": n / cms / 1e6,
                           "gb_s": 7 * n / cms / 1e6, "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
                           "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
+            # segmented running maximum and the plain running maximum (CUDA cores: the operator has no inverse)
+            wsm = mmv.alloc_workspace(mmv.OP_SEG_SCAN_MINMAX, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+            for label, fl, per in ((f"running maximum, {args.case}", fd, 7), ("running maximum, no flag vector", None, 6)):
+                fn = lambda: mmv.seg_scan_minmax(xd, fl, out=od, workspace=wsm)  # noqa: E731,B023
+                for _ in range(3):
+                    fn()
+                torch.cuda.synchronize()
+                cms = event_time_ms(torch, fn, min(args.steps, 10))
+                assert mmv.last_async_status(wsm) == 0
+                sweep.append({"case": label, "ms": cms, "gelem_s": n / cms / 1e6, "gb_s": per * n / cms / 1e6,
+                              "frac_of_measured_peak": per * n / cms / 1e6 / peak,
+                              "frac_of_8tbs": per * n / cms / 1e6 / NOMINAL_HBM_GBS})
+            del wsm
             # COMPRESS of the headline values under the headline flags (flags are read twice: count, scatter)
             outc = torch.empty(n, dtype=torch.float16, device="cuda")
             kc = torch.zeros(1, dtype=torch.int64, device="cuda")

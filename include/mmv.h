@@ -78,7 +78,9 @@ typedef enum {
 
 typedef enum { MMV_F16_TO_F32 = 0, MMV_I8_TO_I32 = 1, MMV_BF16_TO_F32 = 2 } mmv_dtype;
 typedef enum { MMV_SEG_FLAGS_U8 = 0, MMV_SEG_OFFSETS_I32 = 1 } mmv_segfmt;
-typedef enum { MMV_OP_SEG_SCAN = 0, MMV_OP_SEG_SUM = 1, MMV_OP_SPMV_CSR = 2, MMV_OP_COMPRESS = 3 } mmv_op;
+typedef enum {
+    MMV_OP_SEG_SCAN = 0, MMV_OP_SEG_SUM = 1, MMV_OP_SPMV_CSR = 2, MMV_OP_COMPRESS = 3, MMV_OP_SEG_SCAN_MINMAX = 4
+} mmv_op;
 
 /*
  * Bytes of device workspace the given call needs (a pure host computation).
@@ -131,6 +133,22 @@ mmv_status mmv_seg_scan_exclusive(const void *x, const void *seg, mmv_segfmt sf,
 mmv_status mmv_seg_sum(const void *x, const void *seg, mmv_segfmt sf, int64_t n, int64_t nseg,
                        mmv_dtype dt, void *out, int64_t *d_num_segments,
                        void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Segmented running maximum (want_min == 0) or minimum (want_min != 0): Eq. 1
+ * with max / min in place of the addition,
+ *     out[i] = x[i]                  if i == 0 or flags[i] != 0
+ *     out[i] = max(out[i-1], x[i])   otherwise.
+ * These operators have no inverse, so the matrix-product method (which reverts
+ * its speculation by subtracting: Section 2 asks for a group) does not apply;
+ * the scan runs on the CUDA cores and is exact.  x: n values, fp16
+ * (MMV_F16_TO_F32, out fp32) or int8 (MMV_I8_TO_I32, out int32); flags: n bytes
+ * or NULL (one segment); x, flags, out 16-byte aligned.  Workspace:
+ * mmv_workspace_bytes(MMV_OP_SEG_SCAN_MINMAX, dt, MMV_SEG_FLAGS_U8, n, 0).
+ * Errors and asynchrony as for mmv_seg_scan.
+ */
+mmv_status mmv_seg_scan_minmax(const void *x, const void *flags, int64_t n, mmv_dtype dt, int want_min, void *out,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * COMPRESS (Section 2): the values x[i] with flag[i] != 0, in order, copied

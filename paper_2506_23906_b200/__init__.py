@@ -20,13 +20,14 @@ LIB_PATH = _PKG / "libmmv.so"
 MMV_OK = 0
 F16_TO_F32, I8_TO_I32, BF16_TO_F32 = 0, 1, 2
 SEG_FLAGS_U8, SEG_OFFSETS_I32 = 0, 1
-OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR, OP_COMPRESS = 0, 1, 2, 3
+OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR, OP_COMPRESS, OP_SEG_SCAN_MINMAX = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "mmv_workspace_bytes", "mmv_seg_scan", "mmv_seg_sum", "mmv_spmv_csr",
     "mmv_last_async_status", "mmv_status_string", "mmv_kernel_launch_count", "mmv_debug_configure",
     "mmv_seg_scan_static", "mmv_seg_scan_static_last_status", "mmv_debug_force_sum_groups",
     "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes", "mmv_seg_scan_exclusive", "mmv_compress",
+    "mmv_seg_scan_minmax",
 )
 STATIC_SCAN_MAX_N = 1 << 28
 
@@ -50,6 +51,8 @@ def _load() -> ctypes.CDLL:
     lib.mmv_seg_scan.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, sz, vp]
     lib.mmv_seg_scan_exclusive.restype = ci
     lib.mmv_seg_scan_exclusive.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, sz, vp]
+    lib.mmv_seg_scan_minmax.restype = ci
+    lib.mmv_seg_scan_minmax.argtypes = [vp, vp, i64, ci, ci, vp, vp, sz, vp]
     lib.mmv_compress.restype = ci
     lib.mmv_compress.argtypes = [vp, vp, i64, ci, vp, vp, vp, sz, vp]
     lib.mmv_seg_sum.restype = ci
@@ -159,6 +162,22 @@ def seg_scan(x: torch.Tensor, seg: torch.Tensor | None, out: torch.Tensor | None
     rc = call(_ptr(x), _ptr(seg), sf, n, nseg, dt, _ptr(out), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     if rc != MMV_OK:
         raise MmvError(rc, "mmv_seg_scan_exclusive" if exclusive else "mmv_seg_scan")
+    return out
+
+
+def seg_scan_minmax(x: torch.Tensor, flags: torch.Tensor | None, want_min: bool = False, out: torch.Tensor | None = None,
+                    workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """mmv_seg_scan_minmax: segmented running maximum (or minimum) of fp16 / int8 values; flags = None is one segment."""
+    _check_cuda(x, flags, out, workspace)
+    dt, n = _dtype_code(x), x.numel()
+    if out is None:
+        out = torch.empty(n, dtype=torch.int32 if dt == I8_TO_I32 else torch.float32, device=x.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_SEG_SCAN_MINMAX, dt, SEG_FLAGS_U8, n, 0, x.device)
+    rc = _lib.mmv_seg_scan_minmax(_ptr(x), _ptr(flags), n, dt, int(bool(want_min)), _ptr(out), _ptr(workspace),
+                                  workspace.numel(), _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_seg_scan_minmax")
     return out
 
 

@@ -611,6 +611,65 @@ def test_spmv_random_shapes(mmv):
 
 
 # ---------------------------------------------------------------------------
+# segmented running maximum / minimum (exact: every comparison below is for equality)
+# ---------------------------------------------------------------------------
+MM_TILE = 4096
+
+
+def minmax(mmv, x, f, want_min, guard=64):
+    """The call with a guard band behind the output: nothing past n may be written."""
+    import torch
+    n = x.shape[0]
+    i8 = x.dtype == np.int8
+    buf = torch.full((n + guard,), -77, dtype=torch.int32 if i8 else torch.float32, device="cuda")
+    mmv.seg_scan_minmax(dev(x), None if f is None else dev(f), want_min=want_min, out=buf[:n])
+    torch.cuda.synchronize()
+    assert (buf[n:] == -77).all(), "wrote past the end of the output"
+    return buf[:n].cpu().numpy()
+
+
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 511, 513, MM_TILE - 1, MM_TILE, MM_TILE + 1, 3 * MM_TILE + 5, 40 * MM_TILE + 1234,
+                               300 * MM_TILE + 77])
+@pytest.mark.parametrize("p", [0.0, 1e-4, 1e-2, 0.5, 1.0])
+def test_seg_scan_minmax(mmv, n, p):
+    rng = np.random.default_rng(n * 11 + int(p * 10000))
+    f = (rng.random(n) < p).astype(np.uint8)
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    xf = rng.standard_normal(n).astype(np.float16)
+    for want_min in (False, True):
+        assert np.array_equal(minmax(mmv, xi, f, want_min), oracle.seg_scan_minmax_i8(xi, f, want_min))
+        assert np.array_equal(minmax(mmv, xf, f, want_min).astype(np.float64), oracle.seg_scan_minmax_f16(xf, f, want_min))
+
+
+def test_seg_scan_minmax_edges_and_long_carries(mmv):
+    # a ramp that falls: the running maximum is carried from element 0 across every tile, the minimum is the input
+    n = 700 * MM_TILE + 9
+    xf = np.linspace(60000.0, -60000.0, n).astype(np.float16)
+    got = minmax(mmv, xf, None, False)
+    assert (got == np.float32(xf[0])).all()
+    assert np.array_equal(minmax(mmv, xf, None, True), xf.astype(np.float32))
+    # flags on the edges of threads' 16-element runs, warps (512) and tiles; extreme values next to them
+    rng = np.random.default_rng(5)
+    n = 9 * MM_TILE + 100
+    f = np.zeros(n, np.uint8)
+    f[[0, 15, 16, 17, 511, 512, 513, MM_TILE - 1, MM_TILE, MM_TILE + 1, 3 * MM_TILE + 15, 5 * MM_TILE, n - 1]] = 1
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    xi[[14, 510, MM_TILE - 2, 5 * MM_TILE - 1]] = 127
+    xi[[18, 514, MM_TILE + 2, 5 * MM_TILE + 1]] = -128
+    xf = rng.standard_normal(n).astype(np.float16)
+    xf[[14, MM_TILE - 2]] = np.float16(65504.0)
+    xf[[18, MM_TILE + 2]] = np.float16(-65504.0)
+    for want_min in (False, True):
+        assert np.array_equal(minmax(mmv, xi, f, want_min), oracle.seg_scan_minmax_i8(xi, f, want_min))
+        assert np.array_equal(minmax(mmv, xf, f, want_min).astype(np.float64), oracle.seg_scan_minmax_f16(xf, f, want_min))
+    # the worked example of Section 2 (its values, its flags)
+    x = np.asarray([2, 2, 3, 3, 1, 3, 1, 2], np.int8)
+    fl = np.asarray([1, 0, 1, 0, 0, 1, 0, 0], np.uint8)
+    assert minmax(mmv, x, fl, False).tolist() == [2, 2, 3, 3, 3, 3, 3, 3]
+    assert minmax(mmv, x, fl, True).tolist() == [2, 2, 3, 3, 1, 3, 1, 1]
+
+
+# ---------------------------------------------------------------------------
 # exclusive variant of the scan
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("n", [1, 31, 32, 33, 1023, 1025, 4096, TILE - 1, TILE, TILE + 1, 3 * TILE + 4097, 11 * TILE + 777])
