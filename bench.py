@@ -57,7 +57,7 @@ def parse_args():
     ap.add_argument("--case", default="p1e-3", help="flag pattern of the headline workload")
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline")
-    ap.add_argument("--profile-case", default=None, choices=["scan_f16", "scan_i8", "seg_sum", "seg_sum_short", "seg_sum_mid", "spmv"],
+    ap.add_argument("--profile-case", default=None, choices=["scan_f16", "scan_i8", "seg_sum", "seg_sum_short", "seg_sum_mid", "spmv", "minmax"],
                     help="run one small case a few times and exit (the command profiled with ncu)")
     return ap.parse_args()
 
@@ -645,6 +645,14 @@ def run_profile_case(args):
         out = torch.empty(n, dtype=torch.float32 if f16 else torch.int32, device="cuda")
         ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.F16_TO_F32 if f16 else mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
         fn = lambda: mmv.seg_scan(xd, fd, out=out, workspace=ws)  # noqa: E731
+    elif args.profile_case == "minmax":
+        # the segmented running maximum on the flag pattern --case names (p0: no start at all)
+        x = gen.f16_uniform(5, n)
+        f = gen.config5_flags(n, args.case)
+        xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+        out = torch.empty(n, dtype=torch.float32, device="cuda")
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN_MINMAX, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+        fn = lambda: mmv.seg_scan_minmax(xd, fd, out=out, workspace=ws)  # noqa: E731
     elif args.profile_case in ("seg_sum", "seg_sum_short", "seg_sum_mid"):
         # configuration 2, or the Table 5.1 mixes with segment lengths 1/6/44 and 18/119/204 (dense boundaries)
         x, off = gen.config2(n) if args.profile_case == "seg_sum" else gen.seg_sum_row_mix(args.profile_case[8:], n)

@@ -81,6 +81,10 @@ DeviceInfo* device_info() {
         ok &= set_smem(seg_scan_kernel<F16Path, true, true>, ScanCfg<F16Path, true>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<BF16ValPath, false, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<BF16ValPath, true, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
+        ok &= set_smem(seg_scan_minmax_kernel<false, false>, MM_SMEM_BYTES);
+        ok &= set_smem(seg_scan_minmax_kernel<false, true>, MM_SMEM_BYTES);
+        ok &= set_smem(seg_scan_minmax_kernel<true, false>, MM_SMEM_BYTES);
+        ok &= set_smem(seg_scan_minmax_kernel<true, true>, MM_SMEM_BYTES);
         ok &= set_smem(seg_sum_kernel<BF16ValPath, 2>, SumCfg<BF16ValPath, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<BF16ValPath, 3>, SumCfg<BF16ValPath, 3>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<F16Path, 2>, SumCfg<F16Path, 2>::kSmemBytes);
@@ -159,11 +163,12 @@ WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     WorkspacePlan p{};
     p.n_eff = n;
     const long long tiles = num_tiles_of(p.n_eff);
-    const long long units = (op == MMV_OP_SEG_SCAN)          ? num_scan_tiles_of(n) * SPANS_PER_TILE
+    const long long units = (op == MMV_OP_SEG_SCAN)          ? num_scan_tiles_of(n) * SCAN_STATUS_STRIDE
                             : (op == MMV_OP_SEG_SCAN_MINMAX) ? (n + MM_TILE - 1) / MM_TILE
                                                              : tiles * SPANS_PER_TILE;
     p.status_off = sizeof(WorkspaceHeader);
-    p.status_bytes = round_up(static_cast<size_t>(units) * sizeof(uint64_t), 256);
+    const int stride = (op == MMV_OP_SEG_SCAN_MINMAX) ? MM_STATUS_STRIDE : (op == MMV_OP_SEG_SCAN) ? 1 : SUM_STATUS_STRIDE;
+    p.status_bytes = round_up(static_cast<size_t>(units) * sizeof(uint64_t) * stride, 256);
     p.flags_off = p.status_off + p.status_bytes;
     p.flags_bytes = (op == MMV_OP_SEG_SCAN && sf == MMV_SEG_OFFSETS_I32) ? round_up(static_cast<size_t>(n), 256) : 0;
     p.tileq_off = p.flags_off + p.flags_bytes;
@@ -299,13 +304,13 @@ __global__ void offsets_to_flags_kernel(const int32_t* __restrict__ off, long lo
 }
 
 // ---------------------------------------------------------------------------
-// Built-in scratch of mmv_seg_scan_static: header + one status word per 4096-element unit.
+// Built-in scratch of mmv_seg_scan_static: header + the status words (SCAN_STATUS_STRIDE per tile).
 // The symbol below is a host-side stand-in in host code; its device address is looked up once per
 // device with cudaGetSymbolAddress and only that address is ever handed to a kernel or a memset.
 // ---------------------------------------------------------------------------
 constexpr long long kStaticScanMaxN = MMV_STATIC_SCAN_MAX_N;
 constexpr size_t kStaticScratchBytes =
-    sizeof(WorkspaceHeader) + static_cast<size_t>((kStaticScanMaxN + SCAN_UNIT - 1) / SCAN_UNIT) * sizeof(uint64_t);
+    sizeof(WorkspaceHeader) + static_cast<size_t>((kStaticScanMaxN + SCAN_TILE - 1) / SCAN_TILE) * SCAN_STATUS_STRIDE * sizeof(uint64_t);
 static __device__ __align__(256) unsigned char g_static_scan_scratch[kStaticScratchBytes];
 
 struct StaticScratch {
@@ -450,7 +455,7 @@ HostScanPlan plan_host_scan(mmv_dtype dt, long long chunk) {
     HostScanPlan p{};
     const size_t eb = dt == MMV_F16_TO_F32 ? 2 : 1;
     p.status_off = 0;
-    p.status_bytes = round_up(static_cast<size_t>(num_scan_tiles_of(chunk)) * SPANS_PER_TILE * sizeof(uint64_t), 256);
+    p.status_bytes = round_up(static_cast<size_t>(num_scan_tiles_of(chunk)) * SCAN_STATUS_STRIDE * sizeof(uint64_t), 256);
     p.x_off = p.status_bytes;
     p.f_off = p.x_off + round_up(static_cast<size_t>(chunk) * eb, 256);
     p.out_off = p.f_off + round_up(static_cast<size_t>(chunk), 256);
@@ -662,11 +667,11 @@ mmv_status mmv_seg_scan_minmax(const void* x, const void* flags, int64_t n, mmv_
     const long long cap = static_cast<long long>(dev->sm_count) * MM_CTAS_PER_SM;
     const unsigned blocks = static_cast<unsigned>(prm.num_tiles < cap ? prm.num_tiles : cap);
     if (dt == MMV_F16_TO_F32) {
-        if (want_min) seg_scan_minmax_kernel<float, true><<<blocks, MM_THREADS, 0, st>>>(prm);
-        else seg_scan_minmax_kernel<float, false><<<blocks, MM_THREADS, 0, st>>>(prm);
+        if (want_min) seg_scan_minmax_kernel<false, true><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
+        else seg_scan_minmax_kernel<false, false><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
     } else {
-        if (want_min) seg_scan_minmax_kernel<int, true><<<blocks, MM_THREADS, 0, st>>>(prm);
-        else seg_scan_minmax_kernel<int, false><<<blocks, MM_THREADS, 0, st>>>(prm);
+        if (want_min) seg_scan_minmax_kernel<true, true><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
+        else seg_scan_minmax_kernel<true, false><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
     }
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
@@ -770,7 +775,7 @@ mmv_status mmv_seg_scan_static(const void* x, const void* flags_u8, int64_t n, m
 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     const long long tiles = num_scan_tiles_of(n);
-    const size_t used = sizeof(WorkspaceHeader) + static_cast<size_t>(tiles) * SPANS_PER_TILE * sizeof(uint64_t);
+    const size_t used = sizeof(WorkspaceHeader) + static_cast<size_t>(tiles) * SCAN_STATUS_STRIDE * sizeof(uint64_t);
     // the buffer keeps the previous call's words: everything this call reads must start at zero
     if (cudaMemsetAsync(ws, 0, used, st) != cudaSuccess) return MMV_ERR_CUDA;
 

@@ -168,21 +168,22 @@ struct LookbackWindow {
 // Issues the loads of the window whose nearest predecessor is `idx` (no wait on the data).
 // Positions before word 0 read as an inclusive prefix of `base_bits`: zero, or the carry that an
 // earlier call hands in when a long input is processed chunk by chunk.
-template <int W>
+// STRIDE: distance in words between the status words of consecutive positions (1: a dense array).
+template <int W, int STRIDE = 1>
 __device__ __forceinline__ void lookback_load(const uint64_t* status, long long idx, LookbackWindow<W>& win,
                                               uint32_t base_bits = 0u) {
     const long long first = idx - static_cast<long long>(W) * lane_id();
 #pragma unroll
     for (int q = 0; q < W; ++q) {
         const long long my = first - q;
-        win.w[q] = (my >= 0) ? ld_relaxed_gpu_u64(status + my) : pack_status(ST_PREFIX, base_bits);
+        win.w[q] = (my >= 0) ? ld_relaxed_gpu_u64(status + my * STRIDE) : pack_status(ST_PREFIX, base_bits);
     }
 }
 
 // Returns the carry into position s.  `win` may hold a window loaded earlier with lookback_load
 // (preloaded = true) so that the first round trip overlaps the caller's work.  Bounded: returns
 // false on time-out, when another role of the CTA aborted, or when a predecessor aborted.
-template <typename P, int W>
+template <typename P, int W, int STRIDE = 1>
 __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, typename P::Acc& carry,
                                          volatile int* abort_flag, uint64_t budget_ns, LookbackWindow<W>& win,
                                          bool preloaded, uint32_t base_bits = 0u) {
@@ -192,7 +193,7 @@ __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, ty
     long long idx = s - 1;
     uint64_t t0 = global_timer_ns();
     uint32_t polls = 0;
-    if (!preloaded) lookback_load<W>(status, idx, win, base_bits);
+    if (!preloaded) lookback_load<W, STRIDE>(status, idx, win, base_bits);
     while (true) {
         uint32_t tmask = 0u, rmask = 0u, xmask = 0u;
 #pragma unroll
@@ -236,7 +237,7 @@ __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, ty
 #ifdef MMV_PHASE_TIMERS
         if (lane == 0) atomicAdd(&g_phase_cycles[13], 1ull);      // polls after the first window
 #endif
-        lookback_load<W>(status, idx, win, base_bits);
+        lookback_load<W, STRIDE>(status, idx, win, base_bits);
     }
 }
 

@@ -59,7 +59,17 @@ struct ScanParams {
 constexpr int SCAN_UP = 4;
 constexpr int SCAN_UNIT = SCAN_UP * PIECE;                  // 4096 elements
 constexpr int SCAN_TILE = SPANS_PER_TILE * SCAN_UNIT;       // 16384 elements
-constexpr int SCAN_LB_WORDS = 1;                            // look-back window: 32 tiles per poll
+#ifndef MMV_SCAN_LB_WORDS
+#define MMV_SCAN_LB_WORDS 1
+#endif
+#ifndef MMV_SCAN_STATUS_STRIDE
+#define MMV_SCAN_STATUS_STRIDE 8
+#endif
+constexpr int SCAN_LB_WORDS = MMV_SCAN_LB_WORDS;            // look-back window: 32 tiles per poll and word
+// A tile publishes one status word; tile t uses word t * SCAN_STATUS_STRIDE of the workspace, so that every
+// word sits in a 32-byte sector of its own: the tiles in flight poll and write neighbouring words all the
+// time, and in a dense array those accesses queue at one sector.
+constexpr int SCAN_STATUS_STRIDE = MMV_SCAN_STATUS_STRIDE;
 #ifndef MMV_SCAN_I8_GROUPS
 #define MMV_SCAN_I8_GROUPS 3
 #endif
@@ -518,7 +528,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             const bool need_global = !exflag && (tile != 0 || has_in);      // the carry reaches back past the tile
             const bool skip_publish = (prm.debug_skip_span >= 0) && ((prm.debug_skip_span >> 2) == tile);
             if (w == 0 && lane == 0 && !skip_publish)
-                st_relaxed_gpu_u64(prm.status + tile,
+                st_relaxed_gpu_u64(prm.status + tile * SCAN_STATUS_STRIDE,
                                    pack_status((flag_tile || (tile == 0 && !has_in)) ? ST_PREFIX : ST_AGG, P::to_bits(tail_tile)));
             MMV_T_MARK(3)
 
@@ -533,7 +543,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             for (int i = 0; i < UP; ++i) {
                 // the first look-back window travels while the last piece is processed
                 if (i == UP - 1 && need_global && w == 0 && tile != 0)
-                    lookback_load<SCAN_LB_WORDS>(prm.status, tile - 1, lbw, base_bits);
+                    lookback_load<SCAN_LB_WORDS, SCAN_STATUS_STRIDE>(prm.status, tile - 1, lbw, base_bits);
                 uint32_t fmi = fm[0], pmi = pm[0];
                 Acc toti = tot[0];
 #pragma unroll
@@ -628,17 +638,17 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             if (w == 0) {
                 Acc carry_tile = Acc(0);
                 if (tile != 0) {
-                    if (!lookback<P, SCAN_LB_WORDS>(prm.status, tile, carry_tile, abort_flag, budget, lbw, true, base_bits)) {
-                        if (lane == 0) st_relaxed_gpu_u64(prm.status + tile, pack_status(ST_ABORT, 0u));
+                    if (!lookback<P, SCAN_LB_WORDS, SCAN_STATUS_STRIDE>(prm.status, tile, carry_tile, abort_flag, budget, lbw, true, base_bits)) {
+                        if (lane == 0) st_relaxed_gpu_u64(prm.status + tile * SCAN_STATUS_STRIDE, pack_status(ST_ABORT, 0u));
                         failed = true;
                         break;
                     }
                     if (!flag_tile && lane == 0 && !skip_publish)
-                        st_relaxed_gpu_u64(prm.status + tile, pack_status(ST_PREFIX, P::to_bits(P::add(carry_tile, tail_tile))));
+                        st_relaxed_gpu_u64(prm.status + tile * SCAN_STATUS_STRIDE, pack_status(ST_PREFIX, P::to_bits(P::add(carry_tile, tail_tile))));
                 } else if (has_in) {
                     carry_tile = P::from_bits(base_bits);           // the first tile of a later chunk
                     if (!flag_tile && lane == 0 && !skip_publish)
-                        st_relaxed_gpu_u64(prm.status + tile, pack_status(ST_PREFIX, P::to_bits(P::add(carry_tile, tail_tile))));
+                        st_relaxed_gpu_u64(prm.status + tile * SCAN_STATUS_STRIDE, pack_status(ST_PREFIX, P::to_bits(P::add(carry_tile, tail_tile))));
                 }
                 if (lane == 0) {
                     carry_slot[g] = P::to_bits(carry_tile);

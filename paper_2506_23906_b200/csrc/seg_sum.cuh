@@ -211,6 +211,14 @@ __device__ __forceinline__ typename P::Acc window_sum(const void* xg, long long 
     return val;
 }
 
+#ifndef MMV_SUM_STATUS_STRIDE
+#define MMV_SUM_STATUS_STRIDE 1
+#endif
+// Span s publishes word s * SUM_STATUS_STRIDE of the status area.  The scans spread their words over 32-byte
+// sectors and gain by it; here nearly every span holds a boundary and a look-back ends at its first word, and
+// a stride of 4 or 8 measured the same or slightly worse (a larger area to clear), so the array stays dense.
+constexpr int SUM_STATUS_STRIDE = MMV_SUM_STATUS_STRIDE;
+
 // The look-back of the segmented sum behind one signature for its three call sites.
 template <typename P>
 __device__ __forceinline__ bool sum_lookback(const uint64_t* status, long long s, typename P::Acc* carry,
@@ -218,7 +226,7 @@ __device__ __forceinline__ bool sum_lookback(const uint64_t* status, long long s
     LookbackWindow<1> win;
     win.w[0] = window;
     typename P::Acc c = typename P::Acc(0);
-    const bool ok = lookback<P, 1>(status, s, c, abort_flag, budget_ns, win, preloaded);
+    const bool ok = lookback<P, 1, SUM_STATUS_STRIDE>(status, s, c, abort_flag, budget_ns, win, preloaded);
     *carry = c;
     return ok;
 }
@@ -756,13 +764,13 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             // the span's aggregate: published before the boundaries are worked through, kept for the siblings
             auto publish = [&](Acc tail) {
                 if (lane == 0) {
-                    st_relaxed_gpu_u64(prm.status + s, pack_status((seen || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail)));
+                    st_relaxed_gpu_u64(prm.status + s * SUM_STATUS_STRIDE, pack_status((seen || s == 0) ? ST_PREFIX : ST_AGG, P::to_bits(tail)));
                     agg_slot[(g * 2 + (k & 1)) * SPANS_PER_TILE + w] = (static_cast<uint64_t>(seen ? 1u : 0u) << 32) | P::to_bits(tail);
                     mbar_arrive(&bar_agg[g]);
                 }
                 // the first window beyond the tile travels while the boundaries are processed
-                if (tile != 0 && !seen) lookback_load<1>(prm.status, s - w - 1, lbw);
-                if (pending) lookback_load<1>(prm.status, pend_s - w - 1, plw);
+                if (tile != 0 && !seen) lookback_load<1, SUM_STATUS_STRIDE>(prm.status, s - w - 1, lbw);
+                if (pending) lookback_load<1, SUM_STATUS_STRIDE>(prm.status, pend_s - w - 1, plw);
             };
             if (sparse) {
                 // ---- few boundaries (lane j <-> boundary j): the one prefix each boundary needs is read
@@ -1156,7 +1164,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (exflag || tile == 0) {
                     // the carry is complete inside the tile
                     if (!seen && lane == 0)
-                        st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(ex, run))));
+                        st_relaxed_gpu_u64(prm.status + s * SUM_STATUS_STRIDE, pack_status(ST_PREFIX, P::to_bits(P::add(ex, run))));
                     if (def_r >= 0 && lane == 0) outp[def_r] = P::add(ex, def_val);
                 } else if (seen) {
                     // The span's own word is final already; only the segment that ends here waits for the
@@ -1170,12 +1178,12 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 } else {
                     Acc carry_out = Acc(0);
                     if (!sum_lookback<P>(prm.status, s - w, &carry_out, abort_flag, budget, lbw.w[0], true)) {
-                        if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_ABORT, 0u));
+                        if (lane == 0) st_relaxed_gpu_u64(prm.status + s * SUM_STATUS_STRIDE, pack_status(ST_ABORT, 0u));
                         failed = true;
                         break;
                     }
                     const Acc carry = P::add(carry_out, ex);
-                    if (lane == 0) st_relaxed_gpu_u64(prm.status + s, pack_status(ST_PREFIX, P::to_bits(P::add(carry, run))));
+                    if (lane == 0) st_relaxed_gpu_u64(prm.status + s * SUM_STATUS_STRIDE, pack_status(ST_PREFIX, P::to_bits(P::add(carry, run))));
                     if (def_r >= 0 && lane == 0) outp[def_r] = P::add(carry, def_val);
                 }
             }
