@@ -210,6 +210,7 @@ __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, ty
         const int need = (static_cast<int>(lane) < L) ? W : ((static_cast<int>(lane) == L) ? qt + 1 : 0);
         const uint32_t need_mask = (1u << need) - 1u;
         const bool lane_ready = (rmask & need_mask) == need_mask;
+        bool reload = true;                   // after a step back every lane loads; on a retry only the lanes that wait
         if (__all_sync(0xffffffffu, lane_ready)) {
             if (__any_sync(0xffffffffu, (xmask & need_mask) != 0u)) return false;
             Acc v = Acc(0);
@@ -233,11 +234,12 @@ __device__ __forceinline__ bool lookback(const uint64_t* status, long long s, ty
                 if (global_timer_ns() - t0 > budget_ns) return false;
             }
             __nanosleep(40);        // keep the polling traffic in L2 small
+            reload = !lane_ready;
         }
 #ifdef MMV_PHASE_TIMERS
         if (lane == 0) atomicAdd(&g_phase_cycles[13], 1ull);      // polls after the first window
 #endif
-        lookback_load<W, STRIDE>(status, idx, win, base_bits);
+        if (reload) lookback_load<W, STRIDE>(status, idx, win, base_bits);
     }
 }
 
