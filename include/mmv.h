@@ -144,8 +144,12 @@ mmv_status mmv_seg_sum(const void *x, const void *seg, mmv_segfmt sf, int64_t n,
  * the scan runs on the CUDA cores and is exact.  x: n values, fp16
  * (MMV_F16_TO_F32, out fp32) or int8 (MMV_I8_TO_I32, out int32); flags: n bytes
  * or NULL (one segment); x, flags, out 16-byte aligned.  Workspace:
- * mmv_workspace_bytes(MMV_OP_SEG_SCAN_MINMAX, dt, MMV_SEG_FLAGS_U8, n, 0).
- * Errors and asynchrony as for mmv_seg_scan.
+ * mmv_workspace_bytes(MMV_OP_SEG_SCAN_MINMAX, dt, MMV_SEG_FLAGS_U8, n, 0)
+ * (256-byte aligned, owned by the caller, reusable once the call's work on the
+ * stream is done).  n < 2^36.  NaN values and the sign of a zero result are
+ * unspecified.  Errors and asynchrony as for mmv_seg_scan: argument errors are
+ * returned at once, a look-back that exceeds the time budget is reported by
+ * mmv_last_async_status (MMV_ERR_TIMEOUT).
  */
 mmv_status mmv_seg_scan_minmax(const void *x, const void *flags, int64_t n, mmv_dtype dt, int want_min, void *out,
                                void *workspace, size_t workspace_bytes, void *cuda_stream);
