@@ -664,6 +664,8 @@ mmv_status mmv_seg_scan_minmax(const void* x, const void* flags, int64_t n, mmv_
     prm.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();
+    const long long skip = g_debug_skip_span.load();
+    prm.debug_skip_run = skip >= 0 ? skip / (MM_TILE / SCAN_UNIT) : -1;      // the hook counts 4096-element spans
     const long long cap = static_cast<long long>(dev->sm_count) * MM_CTAS_PER_SM;
     const unsigned blocks = static_cast<unsigned>(prm.num_tiles < cap ? prm.num_tiles : cap);
     if (dt == MMV_F16_TO_F32) {

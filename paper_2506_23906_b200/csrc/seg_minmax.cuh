@@ -62,6 +62,7 @@ struct MinMaxParams {
     WorkspaceHeader* hdr;       // tile_counter and error, cleared by the caller
     uint64_t* status;           // one word per run, cleared by the caller; payload: the value as fp32 bits
     unsigned long long budget_ns;
+    long long debug_skip_run;   // test hook: this run never publishes a status word (-1: none)
 };
 
 template <bool MIN>
@@ -261,7 +262,8 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
             run_flg = run_flg || sub_flg;
         }
         const bool first = tile == 0;
-        if (tid == 0 && !published)
+        const bool silent = tile == prm.debug_skip_run;
+        if (tid == 0 && !published && !silent)
             st_relaxed_gpu_u64(prm.status + tile * MM_STATUS_STRIDE, pack_status((run_flg || first) ? ST_PREFIX : ST_AGG, __float_as_uint(run_val)));
         __syncthreads();                                   // every result of the run is parked
 
@@ -314,7 +316,7 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
                 for (int o = 16; o >= 1; o >>= 1) m = Op::f(m, __shfl_xor_sync(0xffffffffu, m, o));
                 if (lane == 0) early_val[warp] = m;
                 __syncthreads();
-                if (tid == 0) {
+                if (tid == 0 && next != prm.debug_skip_run) {
                     float r = early_val[0];
 #pragma unroll
                     for (int q = 1; q < MM_WARPS; ++q) r = Op::f(r, early_val[q]);
@@ -409,7 +411,7 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
                     st_relaxed_gpu_u64(prm.status + tile * MM_STATUS_STRIDE, pack_status(ST_ABORT, 0u));
                     report_error(prm.hdr, 5u);
                     s_failed = 1;
-                } else if (!run_flg && !first) {
+                } else if (!run_flg && !first && !silent) {
                     st_relaxed_gpu_u64(prm.status + tile * MM_STATUS_STRIDE, pack_status(ST_PREFIX, __float_as_uint(Op::f(carry, run_val))));
                 }
                 s_carry = carry;

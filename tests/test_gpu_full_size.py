@@ -212,3 +212,32 @@ def test_exclusive_scan_full_size(mmv, c5_values):
         starts = f[lo:hi] != 0
         assert (got[starts] == 0.0).all()
     assert worst <= 1.0, f"exclusive scan: |err|/bound = {worst}"
+
+
+def test_running_maximum_full_size(mmv, c5_values):
+    # the segmented running maximum at the headline size against the oracle, chunk by chunk: a chunk's elements in
+    # front of its first start take the maximum with the value carried out of the chunk before
+    n = 1 << 30
+    f = gen.config5_flags(n, "p1e-3")
+    xd, fd = torch.from_numpy(c5_values).cuda(), torch.from_numpy(f).cuda()
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN_MINMAX, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+    out = mmv.seg_scan_minmax(xd, fd, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    carry = -np.inf
+    for lo in range(0, n, STEP):
+        hi = min(n, lo + STEP)
+        z = oracle.seg_scan_minmax_f16(c5_values[lo:hi], f[lo:hi])
+        starts = np.flatnonzero(f[lo:hi])
+        first = int(starts[0]) if starts.size else hi - lo
+        z[:first] = np.maximum(z[:first], carry)
+        carry = z[-1]
+        assert np.array_equal(out[lo:hi].cpu().numpy().astype(np.float64), z), f"running maximum wrong in [{lo}, {hi})"
+    # and without a flag vector: every element is the maximum of all elements up to it
+    out = mmv.seg_scan_minmax(xd, None, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    carry = -np.inf
+    for lo in range(0, n, STEP):
+        hi = min(n, lo + STEP)
+        z = np.maximum(np.maximum.accumulate(c5_values[lo:hi].astype(np.float32)), np.float32(carry))
+        carry = z[-1]
+        assert np.array_equal(out[lo:hi].cpu().numpy(), z), f"plain running maximum wrong in [{lo}, {hi})"

@@ -827,6 +827,23 @@ def test_lookback_wait_gives_up_with_a_status(mmv):
     assert np.array_equal(out.cpu().numpy(), np.arange(1, n + 1))
 
 
+def test_minmax_lookback_wait_gives_up_with_a_status(mmv):
+    # the same for the running maximum: run 4 (spans 16..19) stays silent, the runs behind it give up
+    n = 40 * MM_TILE
+    x = np.arange(n, dtype=np.int64) % 100
+    x = dev(x.astype(np.int8))
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN_MINMAX, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    try:
+        mmv.debug_configure(20_000_000, 17)
+        mmv.seg_scan_minmax(x, None, workspace=ws)
+        assert mmv.last_async_status(ws) == 5
+    finally:
+        mmv.debug_configure(0, -1)
+    out = mmv.seg_scan_minmax(x, None, workspace=ws)   # and the next call works
+    assert mmv.last_async_status(ws) == 0
+    assert np.array_equal(out.cpu().numpy(), np.minimum(np.arange(n), 99))
+
+
 # ---------------------------------------------------------------------------
 # the calls only enqueue a memset and kernels on the given stream: they can be captured in a CUDA
 # graph and replayed (the first call on a device, which sets the kernels' attributes, comes before)
