@@ -5,10 +5,11 @@
 // is involved, so results are exact; the kernel is bound by instruction issue and by memory, and
 // is laid out to spend few instructions per element:
 //
-//  * a CTA of 512 threads takes a run of 16384 consecutive elements (runs are handed out by an
-//    atomic counter, so a run's predecessors have always started) as two halves of 8192; a thread
-//    scans 16 consecutive elements, a segmented warp scan (starts known from one ballot) and a
-//    16-lane scan of the warp aggregates give the prefix inside the run;
+//  * a CTA of 256 threads takes a run of 8192 consecutive elements (runs are handed out by an
+//    atomic counter, so a run's predecessors have always started) as two halves of 4096; a thread
+//    scans 16 consecutive elements, a segmented warp scan (starts known from one ballot) and the
+//    same scan over the eight warp aggregates give the prefix inside the run.  Four CTAs share an
+//    SM: with 512 threads and 16384-element runs, two per SM, the CTA-wide barriers cost 10 %;
 //  * everything per element is done on fp16: the maximum of fp16 values is one of them, and int8
 //    values are fp16 values too, so a thread's 16 elements live in eight packed registers and the
 //    results are parked in shared memory in place of the inputs;
@@ -28,13 +29,17 @@
 
 namespace mmv {
 
-constexpr int MM_THREADS = 512;
+#ifndef MMV_MM_THREADS
+#define MMV_MM_THREADS 256
+#endif
+constexpr int MM_THREADS = MMV_MM_THREADS;
 constexpr int MM_WARPS = MM_THREADS / 32;
 constexpr int MM_PER_THREAD = 16;
-constexpr int MM_SUB = MM_THREADS * MM_PER_THREAD;       // 8192 elements: one pass of the CTA
+constexpr int MM_SUB = MM_THREADS * MM_PER_THREAD;       // 4096 elements: one pass of the CTA
 constexpr int MM_SUBS = 2;
-constexpr int MM_TILE = MM_SUB * MM_SUBS;                // 16384 elements: one run, one status word
-constexpr int MM_CTAS_PER_SM = 2;
+constexpr int MM_TILE = MM_SUB * MM_SUBS;                // 8192 elements: one run, one status word
+static_assert(MM_WARPS <= 32 && 1024 % MM_THREADS == 0, "the warp aggregates are scanned by one warp");
+constexpr int MM_CTAS_PER_SM = 1024 / MM_THREADS;
 constexpr int MM_X_BYTES = MM_TILE * 2;                  // values (and, later, results) as fp16
 constexpr int MM_STAGE_BYTES = MM_X_BYTES + MM_TILE;     // ... and the flag bytes behind them
 constexpr int MM_SMEM_BYTES = 2 * MM_STAGE_BYTES;
@@ -218,7 +223,7 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
                 next = s_tile[b ^ 1];
                 stage(next, b ^ 1);                                     // the next run comes in behind everything below
             }
-            // ---- across the 16 warps: the same scan over one value per lane ----
+            // ---- across the warps: the same scan over one value per lane ----
             const float wv = lane < MM_WARPS ? warp_val[s][lane] : Op::identity();
             const int wf = lane < MM_WARPS ? warp_first[s][lane] : MM_SUB;
             const unsigned wstarts = __ballot_sync(0xffffffffu, wf < MM_SUB);

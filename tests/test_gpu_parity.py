@@ -613,7 +613,7 @@ def test_spmv_random_shapes(mmv):
 # ---------------------------------------------------------------------------
 # segmented running maximum / minimum (exact: every comparison below is for equality)
 # ---------------------------------------------------------------------------
-MM_TILE = 16384          # elements per status word of that kernel; a CTA pass covers half of it
+MM_TILE = 8192           # elements per status word of that kernel; a CTA pass covers half of it
 
 
 def minmax(mmv, x, f, want_min, guard=64):
@@ -628,8 +628,8 @@ def minmax(mmv, x, f, want_min, guard=64):
     return buf[:n].cpu().numpy()
 
 
-@pytest.mark.parametrize("n", [1, 15, 16, 17, 511, 513, 8191, 8192, 8193, MM_TILE - 1, MM_TILE, MM_TILE + 1, 3 * MM_TILE + 5,
-                               40 * MM_TILE + 8200, 300 * MM_TILE + 77])
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 511, 513, 4095, 4096, 4097, MM_TILE - 1, MM_TILE, MM_TILE + 1, 16383, 16385,
+                               3 * MM_TILE + 5, 40 * MM_TILE + 4100, 600 * MM_TILE + 77])
 @pytest.mark.parametrize("p", [0.0, 1e-4, 1e-2, 0.5, 1.0])
 def test_seg_scan_minmax(mmv, n, p):
     rng = np.random.default_rng(n * 11 + int(p * 10000))
@@ -643,16 +643,16 @@ def test_seg_scan_minmax(mmv, n, p):
 
 def test_seg_scan_minmax_edges_and_long_carries(mmv):
     # a ramp that falls: the running maximum is carried from element 0 across every tile, the minimum is the input
-    n = 200 * MM_TILE + 9
+    n = 400 * MM_TILE + 9
     xf = np.linspace(60000.0, -60000.0, n).astype(np.float16)
     got = minmax(mmv, xf, None, False)
     assert (got == np.float32(xf[0])).all()
     assert np.array_equal(minmax(mmv, xf, None, True), xf.astype(np.float32))
-    # flags on the edges of threads' 16-element runs, warps (512), CTA passes (8192) and runs; extreme values next to them
+    # flags on the edges of threads' 16-element runs, warps (512), CTA passes (4096) and runs; extreme values next to them
     rng = np.random.default_rng(5)
     n = 9 * MM_TILE + 100
     f = np.zeros(n, np.uint8)
-    f[[0, 15, 16, 17, 511, 512, 513, 8191, 8192, 8193, MM_TILE - 1, MM_TILE, MM_TILE + 1, 3 * MM_TILE + 15, 5 * MM_TILE, n - 1]] = 1
+    f[[0, 15, 16, 17, 511, 512, 513, 4095, 4096, 4097, MM_TILE - 1, MM_TILE, MM_TILE + 1, 3 * MM_TILE + 15, 5 * MM_TILE, n - 1]] = 1
     xi = rng.integers(-128, 128, n).astype(np.int8)
     xi[[14, 510, MM_TILE - 2, 5 * MM_TILE - 1]] = 127
     xi[[18, 514, MM_TILE + 2, 5 * MM_TILE + 1]] = -128
@@ -828,7 +828,7 @@ def test_lookback_wait_gives_up_with_a_status(mmv):
 
 
 def test_minmax_lookback_wait_gives_up_with_a_status(mmv):
-    # the same for the running maximum: run 4 (spans 16..19) stays silent, the runs behind it give up
+    # the same for the running maximum: the run that holds span 17 stays silent, the runs behind it give up
     n = 40 * MM_TILE
     x = np.arange(n, dtype=np.int64) % 100
     x = dev(x.astype(np.int8))
