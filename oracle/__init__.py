@@ -141,6 +141,16 @@ def seg_scan_excl_f16(x, f):
     return e, a
 
 
+def seg_scan_i8_wide(x, f) -> np.ndarray:
+    """Eq. (1) on int8 values with an int64 result: the exact sums, no wrap."""
+    xb, fb = _as(x, np.int8), _as(f, np.uint8)
+    n = xb.shape[0]
+    assert fb.shape[0] == n
+    z = np.empty(n, np.int64)
+    _load().mmv_oracle_seg_scan_i8_wide(_p(xb), _p(fb), ctypes.c_int64(n), _p(z))
+    return z
+
+
 def seg_scan_minmax_f16(x, f, want_min: bool = False) -> np.ndarray:
     """Segmented running maximum (or minimum) of fp16 values, float64 (exact: no arithmetic is involved)."""
     xb, fb = _as_f16_bits(x), _as(f, np.uint8)

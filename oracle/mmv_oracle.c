@@ -107,6 +107,17 @@ void mmv_oracle_seg_scan_i8(const int8_t *x, const uint8_t *f, int64_t n,
     if (state) state[0] = zp;
 }
 
+/* int8 values, int64 result: Eq. (1) without any wrap (|z| <= 128 n). */
+void mmv_oracle_seg_scan_i8_wide(const int8_t *x, const uint8_t *f, int64_t n, int64_t *z)
+{
+    int64_t zp = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (i == 0 || f[i] != 0) zp = (int64_t)x[i];
+        else                     zp = zp + (int64_t)x[i];
+        z[i] = zp;
+    }
+}
+
 /*
  * Segmented EXCLUSIVE scan: e(i) = 0 if i = 0 or f(i) != 0, else z(i-1) with z the
  * scan of Eq. (1); that is, the sum of the elements of i's segment in front of

@@ -585,3 +585,31 @@ def test_segmented_running_max_and_min():
         zero = np.zeros(n, np.uint8)
         assert np.array_equal(oracle.seg_scan_minmax_i8(xi, zero), np.maximum.accumulate(xi.astype(np.int32)))
         assert np.array_equal(oracle.seg_scan_minmax_f16(xf, zero, True), np.minimum.accumulate(xf.astype(np.float64)))
+
+
+# --------------------------------------------------------------------------
+# int8 values with an int64 result (no wrap)
+# --------------------------------------------------------------------------
+def test_wide_integer_scan():
+    g = load_golden("sec2_worked_example.txt")
+    x, f = g["x"], g["f"]                       # x = (2,2,3,3,1,3,1,2), f = (1,0,1,0,0,1,0,0)
+    assert oracle.seg_scan_i8_wide(np.asarray(x, np.int8), u8(f)).tolist() == [2, 4, 3, 6, 7, 3, 4, 6]
+    rng = np.random.default_rng(41)
+    for trial in range(40):
+        n = int(rng.integers(1, 200))
+        xi = rng.integers(-128, 128, n).astype(np.int8)
+        f = (rng.random(n) < rng.choice([0.0, 0.1, 0.5])).astype(np.uint8)
+        want, run = [], 0
+        for i in range(n):                      # the definition once more, on Python integers
+            run = int(xi[i]) if (i == 0 or f[i]) else run + int(xi[i])
+            want.append(run)
+        assert oracle.seg_scan_i8_wide(xi, f).tolist() == want
+        # its low 32 bits are the int32 scan; one segment is numpy's cumulative sum
+        assert np.array_equal(oracle.seg_scan_i8_wide(xi, f).astype(np.int32), oracle.seg_scan_i8(xi, f))
+        assert np.array_equal(oracle.seg_scan_i8_wide(xi, np.zeros(n, np.uint8)), np.cumsum(xi.astype(np.int64)))
+    # past the int32 range: 2^25 values of -128 reach -2^32 (the int32 scan wraps to 0 there), closed form -128 (i + 1)
+    n = 1 << 25
+    z = oracle.seg_scan_i8_wide(np.full(n, -128, np.int8), np.zeros(n, np.uint8))
+    assert z[-1] == -(1 << 32) and np.array_equal(z, -128 * np.arange(1, n + 1, dtype=np.int64))
+    z = oracle.seg_scan_i8_wide(np.full(n, 127, np.int8), np.zeros(n, np.uint8))
+    assert z[-1] == 127 * n and z[(1 << 24) + 5] == 127 * ((1 << 24) + 6)
