@@ -79,7 +79,8 @@ typedef enum {
 typedef enum { MMV_F16_TO_F32 = 0, MMV_I8_TO_I32 = 1, MMV_BF16_TO_F32 = 2 } mmv_dtype;
 typedef enum { MMV_SEG_FLAGS_U8 = 0, MMV_SEG_OFFSETS_I32 = 1 } mmv_segfmt;
 typedef enum {
-    MMV_OP_SEG_SCAN = 0, MMV_OP_SEG_SUM = 1, MMV_OP_SPMV_CSR = 2, MMV_OP_COMPRESS = 3, MMV_OP_SEG_SCAN_MINMAX = 4
+    MMV_OP_SEG_SCAN = 0, MMV_OP_SEG_SUM = 1, MMV_OP_SPMV_CSR = 2, MMV_OP_COMPRESS = 3, MMV_OP_SEG_SCAN_MINMAX = 4,
+    MMV_OP_SEG_SCAN_WIDE = 5
 } mmv_op;
 
 /*
@@ -152,6 +153,20 @@ mmv_status mmv_seg_sum(const void *x, const void *seg, mmv_segfmt sf, int64_t n,
  * mmv_last_async_status (MMV_ERR_TIMEOUT).
  */
 mmv_status mmv_seg_scan_minmax(const void *x, const void *flags, int64_t n, mmv_dtype dt, int want_min, void *out,
+                               void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Segmented inclusive scan (Problem 2.1, Eq. 1) of int8 values with int64
+ * results: the exact sums, where mmv_seg_scan's int32 results wrap from
+ * n = 2^24 on.  Inside a 4096-element tile every sum fits 32 bits; the carries
+ * between tiles are 64 bits wide.  Runs on the CUDA cores (the tensor-core
+ * path chains its tiles through 32-bit payloads).  x: n int8 values; flags: n
+ * bytes or NULL (one segment: the plain inclusive scan); out: n int64 values;
+ * x, flags, out 16-byte aligned; n < 2^36.  Workspace (256-byte aligned):
+ * mmv_workspace_bytes(MMV_OP_SEG_SCAN_WIDE, MMV_I8_TO_I32, MMV_SEG_FLAGS_U8, n, 0).
+ * Errors and asynchrony as for mmv_seg_scan.
+ */
+mmv_status mmv_seg_scan_i8_i64(const void *x, const void *flags, int64_t n, int64_t *out,
                                void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*

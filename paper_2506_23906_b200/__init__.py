@@ -20,14 +20,14 @@ LIB_PATH = _PKG / "libmmv.so"
 MMV_OK = 0
 F16_TO_F32, I8_TO_I32, BF16_TO_F32 = 0, 1, 2
 SEG_FLAGS_U8, SEG_OFFSETS_I32 = 0, 1
-OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR, OP_COMPRESS, OP_SEG_SCAN_MINMAX = 0, 1, 2, 3, 4
+OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR, OP_COMPRESS, OP_SEG_SCAN_MINMAX, OP_SEG_SCAN_WIDE = 0, 1, 2, 3, 4, 5
 
 EXPORTS = (
     "mmv_workspace_bytes", "mmv_seg_scan", "mmv_seg_sum", "mmv_spmv_csr",
     "mmv_last_async_status", "mmv_status_string", "mmv_kernel_launch_count", "mmv_debug_configure",
     "mmv_seg_scan_static", "mmv_seg_scan_static_last_status", "mmv_debug_force_sum_groups",
     "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes", "mmv_seg_scan_exclusive", "mmv_compress",
-    "mmv_seg_scan_minmax",
+    "mmv_seg_scan_minmax", "mmv_seg_scan_i8_i64",
 )
 STATIC_SCAN_MAX_N = 1 << 28
 
@@ -53,6 +53,8 @@ def _load() -> ctypes.CDLL:
     lib.mmv_seg_scan_exclusive.argtypes = [vp, vp, ci, i64, i64, ci, vp, vp, sz, vp]
     lib.mmv_seg_scan_minmax.restype = ci
     lib.mmv_seg_scan_minmax.argtypes = [vp, vp, i64, ci, ci, vp, vp, sz, vp]
+    lib.mmv_seg_scan_i8_i64.restype = ci
+    lib.mmv_seg_scan_i8_i64.argtypes = [vp, vp, i64, vp, vp, sz, vp]
     lib.mmv_compress.restype = ci
     lib.mmv_compress.argtypes = [vp, vp, i64, ci, vp, vp, vp, sz, vp]
     lib.mmv_seg_sum.restype = ci
@@ -178,6 +180,23 @@ def seg_scan_minmax(x: torch.Tensor, flags: torch.Tensor | None, want_min: bool 
                                   workspace.numel(), _stream_ptr(stream))
     if rc != MMV_OK:
         raise MmvError(rc, "mmv_seg_scan_minmax")
+    return out
+
+
+def seg_scan_wide(x: torch.Tensor, flags: torch.Tensor | None, out: torch.Tensor | None = None,
+                  workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """mmv_seg_scan_i8_i64: segmented inclusive scan of int8 values with int64 results (no wrap); flags = None is one segment."""
+    _check_cuda(x, flags, out, workspace)
+    if x.dtype != torch.int8:
+        raise TypeError("seg_scan_wide takes int8 values")
+    n = x.numel()
+    if out is None:
+        out = torch.empty(n, dtype=torch.int64, device=x.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_SEG_SCAN_WIDE, I8_TO_I32, SEG_FLAGS_U8, n, 0, x.device)
+    rc = _lib.mmv_seg_scan_i8_i64(_ptr(x), _ptr(flags), n, _ptr(out), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_seg_scan_i8_i64")
     return out
 
 

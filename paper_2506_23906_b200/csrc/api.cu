@@ -15,6 +15,7 @@
 #include "seg_sum.cuh"
 #include "compress.cuh"
 #include "seg_minmax.cuh"
+#include "seg_wide.cuh"
 
 namespace mmv {
 namespace {
@@ -165,14 +166,18 @@ WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     const long long tiles = num_tiles_of(p.n_eff);
     const long long units = (op == MMV_OP_SEG_SCAN)          ? num_scan_tiles_of(n) * SCAN_STATUS_STRIDE
                             : (op == MMV_OP_SEG_SCAN_MINMAX) ? (n + MM_TILE - 1) / MM_TILE
+                            : (op == MMV_OP_SEG_SCAN_WIDE)   ? (n + WD_TILE - 1) / WD_TILE
                                                              : tiles * SPANS_PER_TILE;
     p.status_off = sizeof(WorkspaceHeader);
-    const int stride = (op == MMV_OP_SEG_SCAN_MINMAX) ? MM_STATUS_STRIDE : (op == MMV_OP_SEG_SCAN) ? 1 : SUM_STATUS_STRIDE;
+    const int stride = (op == MMV_OP_SEG_SCAN_MINMAX) ? MM_STATUS_STRIDE
+                       : (op == MMV_OP_SEG_SCAN_WIDE)  ? WD_STATUS_STRIDE
+                       : (op == MMV_OP_SEG_SCAN)       ? 1
+                                                       : SUM_STATUS_STRIDE;
     p.status_bytes = round_up(static_cast<size_t>(units) * sizeof(uint64_t) * stride, 256);
     p.flags_off = p.status_off + p.status_bytes;
     p.flags_bytes = (op == MMV_OP_SEG_SCAN && sf == MMV_SEG_OFFSETS_I32) ? round_up(static_cast<size_t>(n), 256) : 0;
     p.tileq_off = p.flags_off + p.flags_bytes;
-    p.tileq_bytes = (op != MMV_OP_SEG_SCAN && op != MMV_OP_SEG_SCAN_MINMAX) ? round_up(static_cast<size_t>(tiles * SPANS_PER_TILE + 1) * sizeof(int32_t), 256) : 0;
+    p.tileq_bytes = (op != MMV_OP_SEG_SCAN && op != MMV_OP_SEG_SCAN_MINMAX && op != MMV_OP_SEG_SCAN_WIDE) ? round_up(static_cast<size_t>(tiles * SPANS_PER_TILE + 1) * sizeof(int32_t), 256) : 0;
     p.prod_off = p.tileq_off + p.tileq_bytes;
     p.prod_bytes = (op == MMV_OP_SPMV_CSR) ? round_up(static_cast<size_t>(n) * 4, 256) : 0;
     const bool flagsum = (op == MMV_OP_SEG_SUM && sf == MMV_SEG_FLAGS_U8) || op == MMV_OP_COMPRESS;
@@ -341,7 +346,7 @@ extern "C" {
 size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, int64_t nseg) {
     if (n < 0 || nseg < 0) return 0;
     if (op != MMV_OP_SEG_SCAN && op != MMV_OP_SEG_SUM && op != MMV_OP_SPMV_CSR && op != MMV_OP_COMPRESS &&
-        op != MMV_OP_SEG_SCAN_MINMAX)
+        op != MMV_OP_SEG_SCAN_MINMAX && op != MMV_OP_SEG_SCAN_WIDE)
         return 0;
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return 0;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return 0;
@@ -675,6 +680,39 @@ mmv_status mmv_seg_scan_minmax(const void* x, const void* flags, int64_t n, mmv_
         if (want_min) seg_scan_minmax_kernel<true, true><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
         else seg_scan_minmax_kernel<true, false><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
     }
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+}
+
+mmv_status mmv_seg_scan_i8_i64(const void* x, const void* flags, int64_t n, int64_t* out, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream) {
+    if (n < 0) return MMV_ERR_INVALID_ARG;
+    if (n == 0) return MMV_OK;
+    if (n >= (1ll << 36)) return MMV_ERR_UNSUPPORTED;
+    if (!x || !out || !workspace) return MMV_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(flags) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return MMV_ERR_INVALID_ARG;
+    const WorkspacePlan plan = plan_workspace(MMV_OP_SEG_SCAN_WIDE, MMV_SEG_FLAGS_U8, n);
+    if (workspace_bytes < plan.total) return MMV_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo* dev = device_info();
+    if (!dev) return MMV_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
+    WideParams prm;
+    prm.x = static_cast<const int8_t*>(x);
+    prm.flags = static_cast<const uint8_t*>(flags);
+    prm.out = reinterpret_cast<long long*>(out);
+    prm.n = n;
+    prm.num_tiles = (n + WD_TILE - 1) / WD_TILE;
+    prm.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+    prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
+    prm.budget_ns = g_budget_ns.load();
+    const long long skip = g_debug_skip_span.load();
+    prm.debug_skip_tile = skip >= 0 ? skip / (WD_TILE / SCAN_UNIT) : -1;       // the hook counts 4096-element spans
+    const long long cap = static_cast<long long>(dev->sm_count) * WD_CTAS_PER_SM;
+    const unsigned blocks = static_cast<unsigned>(prm.num_tiles < cap ? prm.num_tiles : cap);
+    seg_scan_wide_kernel<<<blocks, WD_THREADS, 0, st>>>(prm);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }

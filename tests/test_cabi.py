@@ -102,5 +102,11 @@ def test_argument_errors_are_synchronous(lib):
     assert lib.mmv_seg_scan_minmax(16, 16, 8, 0, 1, 16, 256, 16, None) == 3                # workspace too small
     assert lib.mmv_seg_scan_minmax(16, 18, 8, 0, 1, 16, 256, 1 << 20, None) == 1           # misaligned flags
     assert lib.mmv_workspace_bytes(4, 0, 0, 1 << 20, 0) >= 256 * 8
+    lib.mmv_seg_scan_i8_i64.argtypes = [vp, vp, i64, vp, vp, sz, vp]
+    assert lib.mmv_seg_scan_i8_i64(None, None, 0, None, None, 0, None) == 0                # nothing to do
+    assert lib.mmv_seg_scan_i8_i64(None, None, -1, None, None, 0, None) == 1
+    assert lib.mmv_seg_scan_i8_i64(16, 16, 8, 16, 256, 16, None) == 3                      # workspace too small
+    assert lib.mmv_seg_scan_i8_i64(16, 16, 8, 24, 256, 1 << 20, None) == 1                 # misaligned output
+    assert lib.mmv_workspace_bytes(5, 1, 0, 1 << 20, 0) >= 256 * 32
     assert lib.mmv_spmv_csr(None, None, None, None, None, -1, 1, 1, None, 0, None) == 1
     assert lib.mmv_spmv_csr(None, None, None, None, None, 0, 1, 0, None, 0, None) == 0

@@ -674,6 +674,72 @@ def test_seg_scan_minmax_edges_and_long_carries(mmv):
 
 
 # ---------------------------------------------------------------------------
+# int8 values with int64 results (no wrap): exact
+# ---------------------------------------------------------------------------
+WD_TILE = 4096
+
+
+def scan_wide(mmv, x, f, guard=64):
+    import torch
+    n = x.shape[0]
+    buf = torch.full((n + guard,), -77, dtype=torch.int64, device="cuda")
+    mmv.seg_scan_wide(dev(x), None if f is None else dev(f), out=buf[:n])
+    torch.cuda.synchronize()
+    assert (buf[n:] == -77).all(), "wrote past the end of the output"
+    return buf[:n].cpu().numpy()
+
+
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 511, 513, WD_TILE - 1, WD_TILE, WD_TILE + 1, 3 * WD_TILE + 5, 40 * WD_TILE + 1234,
+                               700 * WD_TILE + 77])
+@pytest.mark.parametrize("p", [0.0, 1e-4, 1e-2, 0.5, 1.0])
+def test_seg_scan_wide(mmv, n, p):
+    rng = np.random.default_rng(n * 13 + int(p * 10000))
+    f = (rng.random(n) < p).astype(np.uint8)
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    assert np.array_equal(scan_wide(mmv, xi, f), oracle.seg_scan_i8_wide(xi, f))
+
+
+def test_seg_scan_wide_past_the_int32_range_and_edges(mmv):
+    # 2^25 + 5 values of -128: the sums pass -2^32 (the int32 scan is back at 0 there); closed form -128 (i + 1)
+    n = (1 << 25) + 5
+    x = np.full(n, -128, np.int8)
+    got = scan_wide(mmv, x, None)
+    assert got[-1] == -128 * n and np.array_equal(got, -128 * np.arange(1, n + 1, dtype=np.int64))
+    # the same with one start late in the vector and one flag byte that is not 1
+    f = np.zeros(n, np.uint8)
+    f[(1 << 24) + 3] = 0x80
+    assert np.array_equal(scan_wide(mmv, x, f), oracle.seg_scan_i8_wide(x, f))
+    # flags on the edges of threads' 16-element runs, warps (512) and tiles; extreme values next to them
+    rng = np.random.default_rng(6)
+    n = 9 * WD_TILE + 100
+    f = np.zeros(n, np.uint8)
+    f[[0, 15, 16, 17, 511, 512, 513, WD_TILE - 1, WD_TILE, WD_TILE + 1, 3 * WD_TILE + 15, 5 * WD_TILE, n - 1]] = 1
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    assert np.array_equal(scan_wide(mmv, xi, f), oracle.seg_scan_i8_wide(xi, f))
+    # its low 32 bits are what the tensor-core scan returns
+    assert np.array_equal(scan_wide(mmv, xi, f).astype(np.int32), scan_i8(mmv, xi, f))
+    # the worked example of Section 2
+    x = np.asarray([2, 2, 3, 3, 1, 3, 1, 2], np.int8)
+    fl = np.asarray([1, 0, 1, 0, 0, 1, 0, 0], np.uint8)
+    assert scan_wide(mmv, x, fl).tolist() == [2, 4, 3, 6, 7, 3, 4, 6]
+
+
+def test_wide_lookback_wait_gives_up_with_a_status(mmv):
+    n = 40 * TILE
+    x = dev(np.ones(n, np.int8))
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN_WIDE, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    try:
+        mmv.debug_configure(20_000_000, 17)           # 20 ms budget, tile 17 stays silent
+        mmv.seg_scan_wide(x, None, workspace=ws)
+        assert mmv.last_async_status(ws) == 5
+    finally:
+        mmv.debug_configure(0, -1)
+    out = mmv.seg_scan_wide(x, None, workspace=ws)     # and the next call works
+    assert mmv.last_async_status(ws) == 0
+    assert np.array_equal(out.cpu().numpy(), np.arange(1, n + 1))
+
+
+# ---------------------------------------------------------------------------
 # exclusive variant of the scan
 # ---------------------------------------------------------------------------
 @pytest.mark.parametrize("n", [1, 31, 32, 33, 1023, 1025, 4096, TILE - 1, TILE, TILE + 1, 3 * TILE + 4097, 11 * TILE + 777])
