@@ -57,7 +57,7 @@ def parse_args():
     ap.add_argument("--case", default="p1e-3", help="flag pattern of the headline workload")
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline")
-    ap.add_argument("--profile-case", default=None, choices=["scan_f16", "scan_i8", "seg_sum", "seg_sum_short", "seg_sum_mid", "spmv", "minmax"],
+    ap.add_argument("--profile-case", default=None, choices=["scan_f16", "scan_i8", "seg_sum", "seg_sum_short", "seg_sum_mid", "spmv", "minmax", "wide"],
                     help="run one small case a few times and exit (the command profiled with ncu)")
     return ap.parse_args()
 
@@ -608,6 +608,20 @@ def run_ours(args):
                               "frac_of_measured_peak": per * n / cms / 1e6 / peak,
                               "frac_of_8tbs": per * n / cms / 1e6 / NOMINAL_HBM_GBS})
             del wsm
+            # int8 values with int64 results (10 B/elem): the headline flags over int8 values made on the device
+            xi8 = (xd * 127).to(torch.int8)
+            od64 = torch.empty(n, dtype=torch.int64, device="cuda")
+            wsw = mmv.alloc_workspace(mmv.OP_SEG_SCAN_WIDE, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+            fn = lambda: mmv.seg_scan_wide(xi8, fd, out=od64, workspace=wsw)  # noqa: E731
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            cms = event_time_ms(torch, fn, min(args.steps, 10))
+            assert mmv.last_async_status(wsw) == 0
+            sweep.append({"case": f"int8 -> int64 scan, {args.case} (10 B/elem)", "ms": cms, "gelem_s": n / cms / 1e6,
+                          "gb_s": 10 * n / cms / 1e6, "frac_of_measured_peak": 10 * n / cms / 1e6 / peak,
+                          "frac_of_8tbs": 10 * n / cms / 1e6 / NOMINAL_HBM_GBS})
+            del xi8, od64, wsw
             # COMPRESS of the headline values under the headline flags (flags are read twice: count, scatter)
             outc = torch.empty(n, dtype=torch.float16, device="cuda")
             kc = torch.zeros(1, dtype=torch.int64, device="cuda")
@@ -653,6 +667,14 @@ def run_profile_case(args):
         out = torch.empty(n, dtype=torch.float32, device="cuda")
         ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN_MINMAX, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
         fn = lambda: mmv.seg_scan_minmax(xd, fd, out=out, workspace=ws)  # noqa: E731
+    elif args.profile_case == "wide":
+        # int8 values with int64 results on the flag pattern --case names
+        x = gen.i8_uniform(3, n)
+        f = gen.config5_flags(n, args.case)
+        xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+        out = torch.empty(n, dtype=torch.int64, device="cuda")
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN_WIDE, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+        fn = lambda: mmv.seg_scan_wide(xd, fd, out=out, workspace=ws)  # noqa: E731
     elif args.profile_case in ("seg_sum", "seg_sum_short", "seg_sum_mid"):
         # configuration 2, or the Table 5.1 mixes with segment lengths 1/6/44 and 18/119/204 (dense boundaries)
         x, off = gen.config2(n) if args.profile_case == "seg_sum" else gen.seg_sum_row_mix(args.profile_case[8:], n)

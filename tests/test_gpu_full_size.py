@@ -241,3 +241,33 @@ def test_running_maximum_full_size(mmv, c5_values):
         z = np.maximum(np.maximum.accumulate(c5_values[lo:hi].astype(np.float32)), np.float32(carry))
         carry = z[-1]
         assert np.array_equal(out[lo:hi].cpu().numpy(), z), f"plain running maximum wrong in [{lo}, {hi})"
+
+
+def test_wide_integer_scan_full_size(mmv):
+    # int8 -> int64 at 2^30 elements, flags p = 1e-3, against the oracle chunk by chunk: a chunk's elements in front
+    # of its first start add the value carried out of the chunk before; then one segment of 2^30 values of -128,
+    # whose sums pass the int32 range 64 times over (closed form)
+    n = 1 << 30
+    f = gen.config5_flags(n, "p1e-3")
+    x = gen.i8_uniform(3, n)
+    xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN_WIDE, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    out = mmv.seg_scan_wide(xd, fd, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    carry = 0
+    for lo in range(0, n, STEP):
+        hi = min(n, lo + STEP)
+        z = oracle.seg_scan_i8_wide(x[lo:hi], f[lo:hi])
+        starts = np.flatnonzero(f[lo:hi])
+        first = int(starts[0]) if starts.size else hi - lo
+        z[:first] += carry
+        carry = int(z[-1])
+        assert np.array_equal(out[lo:hi].cpu().numpy(), z), f"int64 scan wrong in [{lo}, {hi})"
+    del xd, fd
+    xd = torch.full((n,), -128, dtype=torch.int8, device="cuda")
+    out = mmv.seg_scan_wide(xd, None, out=out, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    for lo in range(0, n, STEP):
+        hi = min(n, lo + STEP)
+        want = torch.arange(lo + 1, hi + 1, dtype=torch.int64, device="cuda") * -128
+        assert torch.equal(out[lo:hi], want), f"int64 plain scan wrong in [{lo}, {hi})"
