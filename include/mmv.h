@@ -158,8 +158,8 @@ mmv_status mmv_seg_scan_minmax(const void *x, const void *flags, int64_t n, mmv_
 /*
  * Segmented inclusive scan (Problem 2.1, Eq. 1) of int8 values with int64
  * results: the exact sums, where mmv_seg_scan's int32 results wrap from
- * n = 2^24 on.  Inside a 4096-element tile every sum fits 32 bits; the carries
- * between tiles are 64 bits wide.  Runs on the CUDA cores (the tensor-core
+ * n = 2^24 on.  Inside a tile of a few thousand elements every sum fits 32
+ * bits; the carries between tiles are 64 bits wide.  Runs on the CUDA cores (the tensor-core
  * path chains its tiles through 32-bit payloads).  x: n int8 values; flags: n
  * bytes or NULL (one segment: the plain inclusive scan); out: n int64 values;
  * x, flags, out 16-byte aligned; n < 2^36.  Workspace (256-byte aligned):

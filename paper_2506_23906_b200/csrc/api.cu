@@ -670,7 +670,7 @@ mmv_status mmv_seg_scan_minmax(const void* x, const void* flags, int64_t n, mmv_
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();
     const long long skip = g_debug_skip_span.load();
-    prm.debug_skip_run = skip >= 0 ? skip / (MM_TILE / SCAN_UNIT) : -1;      // the hook counts 4096-element spans
+    prm.debug_skip_run = skip >= 0 ? skip * SCAN_UNIT / MM_TILE : -1;        // the hook counts 4096-element spans
     const long long cap = static_cast<long long>(dev->sm_count) * MM_CTAS_PER_SM;
     const unsigned blocks = static_cast<unsigned>(prm.num_tiles < cap ? prm.num_tiles : cap);
     if (dt == MMV_F16_TO_F32) {
@@ -709,7 +709,7 @@ mmv_status mmv_seg_scan_i8_i64(const void* x, const void* flags, int64_t n, int6
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();
     const long long skip = g_debug_skip_span.load();
-    prm.debug_skip_tile = skip >= 0 ? skip / (WD_TILE / SCAN_UNIT) : -1;       // the hook counts 4096-element spans
+    prm.debug_skip_tile = skip >= 0 ? skip * SCAN_UNIT / WD_TILE : -1;         // the hook counts 4096-element spans
     const long long cap = static_cast<long long>(dev->sm_count) * WD_CTAS_PER_SM;
     const unsigned blocks = static_cast<unsigned>(prm.num_tiles < cap ? prm.num_tiles : cap);
     seg_scan_wide_kernel<<<blocks, WD_THREADS, 0, st>>>(prm);

@@ -1,10 +1,11 @@
 // Segmented inclusive scan of int8 values with int64 results: Eq. (1) without the wrap of the int32 path
 // (|z| <= 128 n needs more than 32 bits from n = 2^24 on).  The tensor-core scan accumulates in int32 and
 // chains its tiles through 32-bit status payloads; this variant keeps 32-bit arithmetic where it is exact --
-// inside a 4096-element tile no sum exceeds 2^19 -- and carries 64 bits between tiles.  It runs on the CUDA
+// inside a 2048-element tile no sum exceeds 2^18 -- and carries 64 bits between tiles.  It runs on the CUDA
 // cores with the structure of the running maximum / minimum (seg_minmax.cuh): a thread scans 16 consecutive
-// elements, a segmented warp scan whose limits come from one ballot and the same scan over the eight warp
-// aggregates give the sums inside the tile; tiles are handed out by an atomic counter and chained by a
+// elements, a segmented warp scan whose limits come from one ballot and the same scan over the four warp
+// aggregates give the sums inside the tile (CTAs of 128 threads, eight per SM: with 256 threads and 4096-element
+// tiles the CTA-wide barriers cost 7 % where segment starts are frequent); tiles are handed out by an atomic counter and chained by a
 // single-pass decoupled look-back over one status word per tile (one word per 32-byte sector); only the
 // elements in front of the tile's first segment start need the carry, so all others leave while the first warp
 // still looks back; inputs arrive by 16-byte asynchronous copies into one of two shared-memory buffers, and a
@@ -18,11 +19,15 @@
 
 namespace mmv {
 
-constexpr int WD_THREADS = 256;
+#ifndef MMV_WD_THREADS
+#define MMV_WD_THREADS 128
+#endif
+constexpr int WD_THREADS = MMV_WD_THREADS;
 constexpr int WD_WARPS = WD_THREADS / 32;
 constexpr int WD_PER_THREAD = 16;
-constexpr int WD_TILE = WD_THREADS * WD_PER_THREAD;      // 4096 elements: one pass of the CTA, one status word
-constexpr int WD_CTAS_PER_SM = 4;
+constexpr int WD_TILE = WD_THREADS * WD_PER_THREAD;      // 2048 elements: one pass of the CTA, one status word
+static_assert(WD_TILE <= 12288, "the buffers are static shared memory");
+constexpr int WD_CTAS_PER_SM = 1024 / WD_THREADS;
 constexpr int WD_STATUS_STRIDE = 4;                       // status words of consecutive tiles: one per 32-byte sector
 
 struct WideParams {

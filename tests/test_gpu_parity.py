@@ -676,7 +676,7 @@ def test_seg_scan_minmax_edges_and_long_carries(mmv):
 # ---------------------------------------------------------------------------
 # int8 values with int64 results (no wrap): exact
 # ---------------------------------------------------------------------------
-WD_TILE = 4096
+WD_TILE = 2048
 
 
 def scan_wide(mmv, x, f, guard=64):
@@ -689,8 +689,8 @@ def scan_wide(mmv, x, f, guard=64):
     return buf[:n].cpu().numpy()
 
 
-@pytest.mark.parametrize("n", [1, 15, 16, 17, 511, 513, WD_TILE - 1, WD_TILE, WD_TILE + 1, 3 * WD_TILE + 5, 40 * WD_TILE + 1234,
-                               700 * WD_TILE + 77])
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 511, 513, WD_TILE - 1, WD_TILE, WD_TILE + 1, 4095, 4097, 3 * WD_TILE + 5,
+                               40 * WD_TILE + 1234, 1400 * WD_TILE + 77])
 @pytest.mark.parametrize("p", [0.0, 1e-4, 1e-2, 0.5, 1.0])
 def test_seg_scan_wide(mmv, n, p):
     rng = np.random.default_rng(n * 13 + int(p * 10000))
