@@ -930,18 +930,28 @@ def test_calls_replay_from_a_cuda_graph(mmv):
     o1 = torch.zeros(n, dtype=torch.int32, device="cuda")
     o2 = torch.zeros(off.shape[0] - 1, dtype=torch.int32, device="cuda")
     o3 = torch.zeros(3000, dtype=torch.float32, device="cuda")
+    ws4 = mmv.alloc_workspace(mmv.OP_SEG_SCAN_MINMAX, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    ws5 = mmv.alloc_workspace(mmv.OP_SEG_SCAN_WIDE, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    ws6 = mmv.alloc_workspace(mmv.OP_COMPRESS, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    o4 = torch.zeros(n, dtype=torch.int32, device="cuda")
+    o5 = torch.zeros(n, dtype=torch.int64, device="cuda")
+    o6 = torch.zeros(n, dtype=torch.int8, device="cuda")
+    k6 = torch.zeros(1, dtype=torch.int64, device="cuda")
 
     def calls():
         mmv.seg_scan(xd, fd, out=o1, workspace=ws1)
         mmv.seg_sum(xsd, od_, out=o2, workspace=ws2)
         mmv.spmv_csr(rd, cd, vd, xvd, y=o3, workspace=ws3)
+        mmv.seg_scan_minmax(xd, fd, want_min=True, out=o4, workspace=ws4)
+        mmv.seg_scan_wide(xd, fd, out=o5, workspace=ws5)
+        mmv.compress(xd, fd, out=o6, count=k6, workspace=ws6)
 
     calls()                                   # warm-up outside the capture
     torch.cuda.synchronize()
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
         calls()
-    for buf in (o1, o2, o3):
+    for buf in (o1, o2, o3, o4, o5, o6, k6):
         buf.zero_()
     for _ in range(3):
         g.replay()
@@ -951,3 +961,8 @@ def test_calls_replay_from_a_cuda_graph(mmv):
     assert np.array_equal(o2.cpu().numpy(), oracle.seg_sum_csr_i8(xs, off))
     want, a = oracle.spmv_csr(rowptr, col, val, xv)
     assert_fp(o3.cpu().numpy(), want, a, "SpMV replayed from a graph")
+    assert mmv.last_async_status(ws4) == 0 and mmv.last_async_status(ws5) == 0
+    assert np.array_equal(o4.cpu().numpy(), oracle.seg_scan_minmax_i8(x, f, True))
+    assert np.array_equal(o5.cpu().numpy(), oracle.seg_scan_i8_wide(x, f))
+    kept = oracle.compress(x, f)
+    assert int(k6.item()) == kept.shape[0] and np.array_equal(o6[:kept.shape[0]].cpu().numpy(), kept)
