@@ -187,7 +187,7 @@ seg_scan_wide_kernel(const WideParams prm) {
             const int c = tid * 4 + q;
             outb[c ^ ((c >> 3) & 7)] = make_uint4(o[0], o[1], o[2], o[3]);
         }
-        __syncthreads();                                   // every result of the tile is parked
+        __syncwarp();                                      // a warp stores the results of its own lanes: no CTA-wide barrier
 
         // ---- where segment starts are rare: the NEXT tile's aggregate, ahead of time ----
         published = false;
@@ -224,8 +224,8 @@ seg_scan_wide_kernel(const WideParams prm) {
         const bool whole = t0 + WD_TILE <= prm.n;
         auto copy_out = [&](bool late, long long carry) {
 #pragma unroll
-            for (int k = 0; k < WD_TILE / 4 / WD_THREADS; ++k) {
-                const int c = k * WD_THREADS + tid;
+            for (int k = 0; k < WD_PER_THREAD / 4; ++k) {
+                const int c = warp * (32 * WD_PER_THREAD / 4) + k * 32 + lane;      // a chunk of four of my warp's elements
                 const int e = 4 * c;
                 const bool needs = e < tile_first;
                 if (warp == 0 ? !late : needs != late) continue;
