@@ -390,7 +390,6 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
         flags = f;
     }
 
-    const bool f16 = dt == MMV_F16_TO_F32;
     CUtensorMap tmap, tmap_out;
     if (!encode_span_map(&tmap, x, n, dt == MMV_I8_TO_I32 ? 1 : 2, SCAN_UP)) return MMV_ERR_CUDA;
     if (!encode_out_map(&tmap_out, out, n)) return MMV_ERR_CUDA;
