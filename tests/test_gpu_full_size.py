@@ -271,3 +271,49 @@ def test_wide_integer_scan_full_size(mmv):
         hi = min(n, lo + STEP)
         want = torch.arange(lo + 1, hi + 1, dtype=torch.int64, device="cuda") * -128
         assert torch.equal(out[lo:hi], want), f"int64 plain scan wrong in [{lo}, {hi})"
+
+
+def test_compress_full_size(mmv, c5_values):
+    # COMPRESS of the headline values under the headline flags: the kept values are x[f != 0], in order
+    n = 1 << 30
+    f = gen.config5_flags(n, "p1e-3")
+    xd, fd = torch.from_numpy(c5_values).cuda(), torch.from_numpy(f).cuda()
+    ws = mmv.alloc_workspace(mmv.OP_COMPRESS, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+    out, count = mmv.compress(xd, fd, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    k = int(count.item())
+    pos = 0
+    for lo in range(0, n, STEP):
+        hi = min(n, lo + STEP)
+        kept = oracle.compress(c5_values[lo:hi], f[lo:hi])
+        got = out[pos:pos + kept.shape[0]].cpu().numpy()
+        assert np.array_equal(got.view(np.uint16), kept.view(np.uint16)), f"COMPRESS wrong for the flags in [{lo}, {hi})"
+        pos += kept.shape[0]
+    assert pos == k
+
+
+def test_bf16_scan_full_size(mmv, c5_values):
+    # bfloat16 values (the headline values rounded to bf16 on the device) under the headline flags, against the
+    # oracle chunk by chunk: the elements in front of a chunk's first start add what the chunk before carried out
+    n = 1 << 30
+    f = gen.config5_flags(n, "p1e-3")
+    xb = torch.from_numpy(c5_values).cuda().to(torch.bfloat16)
+    fd = torch.from_numpy(f).cuda()
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.BF16_TO_F32, mmv.SEG_FLAGS_U8, n)
+    out = mmv.seg_scan(xb, fd, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    bits = xb.view(torch.int16)
+    carry_z, carry_a, worst = 0.0, 0.0, 0.0
+    for lo in range(0, n, STEP):
+        hi = min(n, lo + STEP)
+        z, a = oracle.seg_scan_bf16(bits[lo:hi].cpu().numpy().view(np.uint16), f[lo:hi])
+        starts = np.flatnonzero(f[lo:hi])
+        first = int(starts[0]) if starts.size else hi - lo
+        if lo > 0:
+            z[:first] += carry_z
+            a[:first] += carry_a
+        carry_z, carry_a = float(z[-1]), float(a[-1])
+        ok, ratio, i = oracle.check_fp(out[lo:hi].cpu().numpy(), z, a)
+        assert ok, f"bf16 scan: outside the bound at element {lo + i} (ratio {ratio})"
+        worst = max(worst, ratio)
+    assert worst <= 1.0
