@@ -161,6 +161,16 @@ def seg_scan_minmax_f16(x, f, want_min: bool = False) -> np.ndarray:
     return z
 
 
+def seg_scan_minmax_bf16(xbits, f, want_min: bool = False) -> np.ndarray:
+    """Segmented running maximum (or minimum) of bfloat16 values given as uint16 bit patterns, float64 (exact)."""
+    x, fb = bf16_to_double(xbits), _as(f, np.uint8)
+    n = x.shape[0]
+    assert fb.shape[0] == n
+    z = np.empty(n, np.float64)
+    _load().mmv_oracle_seg_scan_minmax_f64(_p(x), _p(fb), ctypes.c_int64(n), ctypes.c_int(int(want_min)), _p(z))
+    return z
+
+
 def seg_scan_minmax_i8(x, f, want_min: bool = False) -> np.ndarray:
     xb, fb = _as(x, np.int8), _as(f, np.uint8)
     n = xb.shape[0]

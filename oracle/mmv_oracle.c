@@ -248,6 +248,17 @@ void mmv_oracle_seg_scan_minmax_f16(const uint16_t *x, const uint8_t *f, int64_t
     }
 }
 
+/* The same on values given as doubles (bfloat16 inputs are decoded first). */
+void mmv_oracle_seg_scan_minmax_f64(const double *x, const uint8_t *f, int64_t n, int want_min, double *z)
+{
+    double zp = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        if (i == 0 || f[i] != 0) zp = x[i];
+        else if (want_min ? (x[i] < zp) : (x[i] > zp)) zp = x[i];
+        z[i] = zp;
+    }
+}
+
 void mmv_oracle_seg_scan_minmax_i8(const int8_t *x, const uint8_t *f, int64_t n, int want_min, int32_t *z)
 {
     int32_t zp = 0;

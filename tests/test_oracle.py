@@ -612,3 +612,29 @@ def test_wide_integer_scan():
     z = oracle.seg_scan_i8_wide(np.full(n, -128, np.int8), np.zeros(n, np.uint8))
     idx = np.arange(0, n, 4097)
     assert z[-1] == -(1 << 32) and z[(1 << 24) + 5] == -128 * ((1 << 24) + 6) and np.array_equal(z[idx], -128 * (idx + 1))
+
+
+def test_running_max_and_min_of_bfloat16_values():
+    g = load_golden("sec2_worked_example.txt")
+    x, f = g["x"], g["f"]                       # small integers: exact in bfloat16
+    xb = gen.bf16_bits_of(np.asarray(x, np.float32))
+    assert oracle.seg_scan_minmax_bf16(xb, u8(f)).tolist() == [2, 2, 3, 3, 3, 3, 3, 3]
+    assert oracle.seg_scan_minmax_bf16(xb, u8(f), want_min=True).tolist() == [2, 2, 3, 3, 1, 3, 1, 1]
+    rng = np.random.default_rng(43)
+    for trial in range(40):
+        n = int(rng.integers(1, 300))
+        f = (rng.random(n) < rng.choice([0.0, 0.05, 0.5])).astype(np.uint8)
+        # values that both 16-bit formats hold exactly: the fp16 function must agree
+        small = rng.integers(-200, 200, n).astype(np.float32) / 4.0
+        assert np.array_equal(oracle.seg_scan_minmax_bf16(gen.bf16_bits_of(small), f), oracle.seg_scan_minmax_f16(small.astype(np.float16), f))
+        # the whole bfloat16 range, far beyond fp16's: brute force on the decoded values, duality, one segment = numpy
+        xb = gen.bf16_bits_of((rng.standard_normal(n) * 10.0 ** rng.integers(-30, 30, n)).astype(np.float32))
+        xd = oracle.bf16_to_double(xb)
+        for want_min in (False, True):
+            want, run = [], 0.0
+            for i in range(n):
+                run = xd[i] if (i == 0 or f[i]) else (min(run, xd[i]) if want_min else max(run, xd[i]))
+                want.append(run)
+            assert oracle.seg_scan_minmax_bf16(xb, f, want_min).tolist() == want
+        assert np.array_equal(oracle.seg_scan_minmax_bf16(xb, f, True), -oracle.seg_scan_minmax_bf16(xb ^ np.uint16(0x8000), f, False))
+        assert np.array_equal(oracle.seg_scan_minmax_bf16(xb, np.zeros(n, np.uint8)), np.maximum.accumulate(xd))
