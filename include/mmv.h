@@ -142,8 +142,8 @@ mmv_status mmv_seg_sum(const void *x, const void *seg, mmv_segfmt sf, int64_t n,
  *     out[i] = max(out[i-1], x[i])   otherwise.
  * These operators have no inverse, so the matrix-product method (which reverts
  * its speculation by subtracting: Section 2 asks for a group) does not apply;
- * the scan runs on the CUDA cores and is exact.  x: n values, fp16
- * (MMV_F16_TO_F32, out fp32) or int8 (MMV_I8_TO_I32, out int32); flags: n bytes
+ * the scan runs on the CUDA cores and is exact.  x: n values, fp16 or bfloat16
+ * (MMV_F16_TO_F32, MMV_BF16_TO_F32: out fp32) or int8 (MMV_I8_TO_I32: out int32); flags: n bytes
  * or NULL (one segment); x, flags, out 16-byte aligned.  Workspace:
  * mmv_workspace_bytes(MMV_OP_SEG_SCAN_MINMAX, dt, MMV_SEG_FLAGS_U8, n, 0)
  * (256-byte aligned, owned by the caller, reusable once the call's work on the

@@ -82,10 +82,12 @@ DeviceInfo* device_info() {
         ok &= set_smem(seg_scan_kernel<F16Path, true, true>, ScanCfg<F16Path, true>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<BF16ValPath, false, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
         ok &= set_smem(seg_scan_kernel<BF16ValPath, true, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
-        ok &= set_smem(seg_scan_minmax_kernel<false, false>, MM_SMEM_BYTES);
-        ok &= set_smem(seg_scan_minmax_kernel<false, true>, MM_SMEM_BYTES);
-        ok &= set_smem(seg_scan_minmax_kernel<true, false>, MM_SMEM_BYTES);
-        ok &= set_smem(seg_scan_minmax_kernel<true, true>, MM_SMEM_BYTES);
+        ok &= set_smem(seg_scan_minmax_kernel<0, false>, MM_SMEM_BYTES);
+        ok &= set_smem(seg_scan_minmax_kernel<0, true>, MM_SMEM_BYTES);
+        ok &= set_smem(seg_scan_minmax_kernel<1, false>, MM_SMEM_BYTES);
+        ok &= set_smem(seg_scan_minmax_kernel<1, true>, MM_SMEM_BYTES);
+        ok &= set_smem(seg_scan_minmax_kernel<2, false>, MM_SMEM_BYTES);
+        ok &= set_smem(seg_scan_minmax_kernel<2, true>, MM_SMEM_BYTES);
         ok &= set_smem(seg_sum_kernel<BF16ValPath, 2>, SumCfg<BF16ValPath, 2>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<BF16ValPath, 3>, SumCfg<BF16ValPath, 3>::kSmemBytes);
         ok &= set_smem(seg_sum_kernel<F16Path, 2>, SumCfg<F16Path, 2>::kSmemBytes);
@@ -646,7 +648,7 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
 mmv_status mmv_seg_scan_minmax(const void* x, const void* flags, int64_t n, mmv_dtype dt, int want_min, void* out,
                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (n < 0) return MMV_ERR_INVALID_ARG;
-    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32) return MMV_ERR_INVALID_ARG;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return MMV_ERR_INVALID_ARG;
     if (n == 0) return MMV_OK;
     if (n >= (1ll << 36)) return MMV_ERR_UNSUPPORTED;
     if (!x || !out || !workspace) return MMV_ERR_INVALID_ARG;
@@ -673,11 +675,14 @@ mmv_status mmv_seg_scan_minmax(const void* x, const void* flags, int64_t n, mmv_
     const long long cap = static_cast<long long>(dev->sm_count) * MM_CTAS_PER_SM;
     const unsigned blocks = static_cast<unsigned>(prm.num_tiles < cap ? prm.num_tiles : cap);
     if (dt == MMV_F16_TO_F32) {
-        if (want_min) seg_scan_minmax_kernel<false, true><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
-        else seg_scan_minmax_kernel<false, false><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
+        if (want_min) seg_scan_minmax_kernel<0, true><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
+        else seg_scan_minmax_kernel<0, false><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
+    } else if (dt == MMV_I8_TO_I32) {
+        if (want_min) seg_scan_minmax_kernel<1, true><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
+        else seg_scan_minmax_kernel<1, false><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
     } else {
-        if (want_min) seg_scan_minmax_kernel<true, true><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
-        else seg_scan_minmax_kernel<true, false><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
+        if (want_min) seg_scan_minmax_kernel<2, true><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
+        else seg_scan_minmax_kernel<2, false><<<blocks, MM_THREADS, MM_SMEM_BYTES, st>>>(prm);
     }
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;

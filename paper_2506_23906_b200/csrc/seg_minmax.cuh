@@ -10,9 +10,9 @@
 //    scans 16 consecutive elements, a segmented warp scan (starts known from one ballot) and the
 //    same scan over the eight warp aggregates give the prefix inside the run.  Four CTAs share an
 //    SM: with 512 threads and 16384-element runs, two per SM, the CTA-wide barriers cost 10 %;
-//  * everything per element is done on fp16: the maximum of fp16 values is one of them, and int8
-//    values are fp16 values too, so a thread's 16 elements live in eight packed registers and the
-//    results are parked in shared memory in place of the inputs;
+//  * everything per element is done in the values' own 16-bit format (fp16 or bfloat16): the maximum
+//    of such values is one of them; int8 values are fp16 values too.  So a thread's 16 elements live
+//    in eight packed registers and the results are parked in shared memory in place of the inputs;
 //  * runs are chained with a single-pass decoupled look-back over one status word per run.  Only
 //    the elements in front of the run's first segment start need the carry, so all other results
 //    leave (fp32 / int32, coalesced 16-byte stores) while the first warp is still looking back;
@@ -21,7 +21,9 @@
 //
 // NaN inputs and the sign of a zero result are unspecified (max(+0, -0) may be either).
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_fp16.h>
+#include <type_traits>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include "common.cuh"
@@ -75,8 +77,27 @@ struct MinMaxOp {
     __device__ static __forceinline__ float f(float a, float b) { return MIN ? fminf(a, b) : fmaxf(a, b); }
     __device__ static __forceinline__ __half h(__half a, __half b) { return MIN ? __hmin(a, b) : __hmax(a, b); }
     __device__ static __forceinline__ __half2 h2(__half2 a, __half2 b) { return MIN ? __hmin2(a, b) : __hmax2(a, b); }
+    __device__ static __forceinline__ __nv_bfloat16 h(__nv_bfloat16 a, __nv_bfloat16 b) { return MIN ? __hmin(a, b) : __hmax(a, b); }
+    __device__ static __forceinline__ __nv_bfloat162 h2(__nv_bfloat162 a, __nv_bfloat162 b) { return MIN ? __hmin2(a, b) : __hmax2(a, b); }
     __device__ static __forceinline__ float identity() { return __int_as_float(MIN ? 0x7f800000 : 0xff800000); }
 };
+
+// The two 16-bit formats behind one set of names.
+__device__ __forceinline__ __half mm_lo(__half2 p) { return __low2half(p); }
+__device__ __forceinline__ __half mm_hi(__half2 p) { return __high2half(p); }
+__device__ __forceinline__ __nv_bfloat16 mm_lo(__nv_bfloat162 p) { return __low2bfloat16(p); }
+__device__ __forceinline__ __nv_bfloat16 mm_hi(__nv_bfloat162 p) { return __high2bfloat16(p); }
+__device__ __forceinline__ float mm_tof(__half v) { return __half2float(v); }
+__device__ __forceinline__ float mm_tof(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float2 mm_tof2(__half2 p) { return __half22float2(p); }
+__device__ __forceinline__ float2 mm_tof2(__nv_bfloat162 p) { return __bfloat1622float2(p); }
+__device__ __forceinline__ __half2 mm_dup(__half v) { return __half2half2(v); }
+__device__ __forceinline__ __nv_bfloat162 mm_dup(__nv_bfloat16 v) { return __bfloat162bfloat162(v); }
+__device__ __forceinline__ __half2 mm_pack(__half a, __half b) { return __halves2half2(a, b); }
+__device__ __forceinline__ __nv_bfloat162 mm_pack(__nv_bfloat16 a, __nv_bfloat16 b) { return __halves2bfloat162(a, b); }
+template <typename H> __device__ __forceinline__ H mm_fromf(float v);
+template <> __device__ __forceinline__ __half mm_fromf<__half>(float v) { return __float2half_rn(v); }
+template <> __device__ __forceinline__ __nv_bfloat16 mm_fromf<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
 // Bit i of the result: byte i of w is not zero.
 __device__ __forceinline__ uint32_t nonzero_byte_bits(uint32_t w) {
@@ -84,11 +105,16 @@ __device__ __forceinline__ uint32_t nonzero_byte_bits(uint32_t w) {
     return ((t & 0x01010101u) * 0x01020408u) >> 24 & 0xfu;
 }
 
-// INT8: the values are int8 and the results int32 (else fp16 and fp32); MIN selects the operator.
-template <bool INT8, bool MIN>
+// FMT 0: fp16 values, fp32 results; 1: int8 values (handled as fp16), int32 results; 2: bfloat16 values, fp32
+// results.  MIN selects the operator.
+template <int FMT, bool MIN>
 __global__ void __launch_bounds__(MM_THREADS, MM_CTAS_PER_SM)
 seg_scan_minmax_kernel(const MinMaxParams prm) {
     using Op = MinMaxOp<MIN>;
+    constexpr bool INT8 = FMT == 1;
+    using H = typename std::conditional<FMT == 2, __nv_bfloat16, __half>::type;
+    using H2 = typename std::conditional<FMT == 2, __nv_bfloat162, __half2>::type;
+    constexpr unsigned short kNeutralBits = FMT == 2 ? (MIN ? 0x7f80u : 0xff80u) : (MIN ? 0x7c00u : 0xfc00u);   // +inf / -inf
     constexpr int kElem = INT8 ? 1 : 2;                    // bytes per input value
     // int8 values land in the upper half of the value area: their fp16 results then never overwrite
     // a value that has not been read (the first half's results fill the lower half of the area, the
@@ -128,7 +154,7 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
                     xs[kRawOff + e] = in ? static_cast<const uint8_t*>(prm.x)[t0 + e] : static_cast<uint8_t>(MIN ? 0x7fu : 0x80u);
                 else
                     reinterpret_cast<unsigned short*>(xs)[e] =
-                        in ? static_cast<const unsigned short*>(prm.x)[t0 + e] : static_cast<unsigned short>(MIN ? 0x7c00u : 0xfc00u);
+                        in ? static_cast<const unsigned short*>(prm.x)[t0 + e] : kNeutralBits;
                 fs[e] = (in && prm.flags) ? prm.flags[t0 + e] : uint8_t(0);
             }
         }
@@ -160,7 +186,7 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
         for (int s = 0; s < MM_SUBS; ++s) {
             const int base = s * MM_SUB + tid * MM_PER_THREAD;          // my first element inside the run
             // ---- my 16 values as fp16 pairs, my 16 flags as bits ----
-            __half h[MM_PER_THREAD];
+            H h[MM_PER_THREAD];
             if constexpr (INT8) {
                 const uint4 a = *reinterpret_cast<const uint4*>(xs + kRawOff + base);
                 const uint32_t w[4] = {a.x, a.y, a.z, a.w};
@@ -173,9 +199,9 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
                 const uint32_t w[8] = {a.x, a.y, a.z, a.w, c.x, c.y, c.z, c.w};
 #pragma unroll
                 for (int k = 0; k < MM_PER_THREAD / 2; ++k) {
-                    const __half2 p = *reinterpret_cast<const __half2*>(&w[k]);
-                    h[2 * k] = __low2half(p);
-                    h[2 * k + 1] = __high2half(p);
+                    const H2 p = *reinterpret_cast<const H2*>(&w[k]);
+                    h[2 * k] = mm_lo(p);
+                    h[2 * k + 1] = mm_hi(p);
                 }
             }
             uint32_t fmask = 0u;                                        // bit j: element j starts a segment
@@ -185,7 +211,7 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
                     fmask = nonzero_byte_bits(f.x) | nonzero_byte_bits(f.y) << 4 | nonzero_byte_bits(f.z) << 8 | nonzero_byte_bits(f.w) << 12;
             }
             // ---- the recurrence inside the thread ----
-            __half run = h[0];
+            H run = h[0];
             if (fmask == 0u) {
 #pragma unroll
                 for (int j = 1; j < MM_PER_THREAD; ++j) {
@@ -202,7 +228,7 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
             // ---- segmented warp scan of the threads' open tails; the starts are known from one ballot ----
             const unsigned starts = __ballot_sync(0xffffffffu, fmask != 0u);
             const int seg_lane = 31 - __clz((starts & (lanes_below | (1u << lane))) | 1u);   // nearest lane at or below mine with a start (else 0)
-            float val = __half2float(run);
+            float val = mm_tof(run);
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const float tv = __shfl_up_sync(0xffffffffu, val, o);
@@ -244,17 +270,17 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
             // ---- what is open in front of my elements inside the run; finish my elements up to my first start ----
             float ex = ef ? ev : Op::f(pre, ev);
             if (!(ef || pre_flg)) ex = Op::f(run_val, ex);
-            const __half exh = __float2half_rn(ex);                     // exact: one of the values, or the identity
-            __half2 w2[MM_PER_THREAD / 2];
+            const H exh = mm_fromf<H>(ex);                              // exact: one of the values, or the identity
+            H2 w2[MM_PER_THREAD / 2];
             if (fmask == 0u) {
-                const __half2 ex2 = __half2half2(exh);
+                const H2 ex2 = mm_dup(exh);
 #pragma unroll
-                for (int k = 0; k < MM_PER_THREAD / 2; ++k) w2[k] = Op::h2(ex2, __halves2half2(h[2 * k], h[2 * k + 1]));
+                for (int k = 0; k < MM_PER_THREAD / 2; ++k) w2[k] = Op::h2(ex2, mm_pack(h[2 * k], h[2 * k + 1]));
             } else {
                 const int first_flag = __ffs(fmask) - 1;
 #pragma unroll
                 for (int k = 0; k < MM_PER_THREAD / 2; ++k)
-                    w2[k] = __halves2half2(2 * k < first_flag ? Op::h(exh, h[2 * k]) : h[2 * k],
+                    w2[k] = mm_pack(2 * k < first_flag ? Op::h(exh, h[2 * k]) : h[2 * k],
                                            2 * k + 1 < first_flag ? Op::h(exh, h[2 * k + 1]) : h[2 * k + 1]);
             }
             uint4* park = reinterpret_cast<uint4*>(xs + base * 2);
@@ -306,16 +332,16 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
                     m = static_cast<float>(mi);
                 } else {
                     const uint4* p4 = reinterpret_cast<const uint4*>(nx + tid * 64);
-                    __half2 m2 = *reinterpret_cast<const __half2*>(&p4[0].x);
+                    H2 m2 = *reinterpret_cast<const H2*>(&p4[0].x);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
                         const uint4 a = p4[k];
-                        m2 = Op::h2(m2, *reinterpret_cast<const __half2*>(&a.x));
-                        m2 = Op::h2(m2, *reinterpret_cast<const __half2*>(&a.y));
-                        m2 = Op::h2(m2, *reinterpret_cast<const __half2*>(&a.z));
-                        m2 = Op::h2(m2, *reinterpret_cast<const __half2*>(&a.w));
+                        m2 = Op::h2(m2, *reinterpret_cast<const H2*>(&a.x));
+                        m2 = Op::h2(m2, *reinterpret_cast<const H2*>(&a.y));
+                        m2 = Op::h2(m2, *reinterpret_cast<const H2*>(&a.z));
+                        m2 = Op::h2(m2, *reinterpret_cast<const H2*>(&a.w));
                     }
-                    m = __half2float(Op::h(__low2half(m2), __high2half(m2)));
+                    m = mm_tof(Op::h(mm_lo(m2), mm_hi(m2)));
                 }
 #pragma unroll
                 for (int o = 16; o >= 1; o >>= 1) m = Op::f(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -342,8 +368,8 @@ seg_scan_minmax_kernel(const MinMaxParams prm) {
                 const bool needs = e < run_first;
                 if (warp == 0 ? !late : needs != late) continue;
                 const uint2 r = *reinterpret_cast<const uint2*>(xs + c * 8);
-                const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&r.x));
-                const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&r.y));
+                const float2 lo = mm_tof2(*reinterpret_cast<const H2*>(&r.x));
+                const float2 hi = mm_tof2(*reinterpret_cast<const H2*>(&r.y));
                 float v[4] = {lo.x, lo.y, hi.x, hi.y};
                 if (needs) {
 #pragma unroll

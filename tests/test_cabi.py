@@ -98,7 +98,8 @@ def test_argument_errors_are_synchronous(lib):
     lib.mmv_seg_scan_minmax.argtypes = [vp, vp, i64, ci, ci, vp, vp, sz, vp]
     assert lib.mmv_seg_scan_minmax(None, None, 0, 0, 0, None, None, 0, None) == 0          # nothing to do
     assert lib.mmv_seg_scan_minmax(None, None, -1, 0, 0, None, None, 0, None) == 1
-    assert lib.mmv_seg_scan_minmax(16, 16, 8, 2, 0, 16, 256, 1 << 20, None) == 1           # bf16: not for this entry point
+    assert lib.mmv_seg_scan_minmax(16, 16, 8, 3, 0, 16, 256, 1 << 20, None) == 1           # bad dtype
+    assert lib.mmv_seg_scan_minmax(16, 16, 8, 2, 0, 16, 256, 16, None) == 3                # bf16 accepted: workspace too small
     assert lib.mmv_seg_scan_minmax(16, 16, 8, 0, 1, 16, 256, 16, None) == 3                # workspace too small
     assert lib.mmv_seg_scan_minmax(16, 18, 8, 0, 1, 16, 256, 1 << 20, None) == 1           # misaligned flags
     assert lib.mmv_workspace_bytes(4, 0, 0, 1 << 20, 0) >= 256 * 8

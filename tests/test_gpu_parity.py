@@ -641,6 +641,20 @@ def test_seg_scan_minmax(mmv, n, p):
         assert np.array_equal(minmax(mmv, xf, f, want_min).astype(np.float64), oracle.seg_scan_minmax_f16(xf, f, want_min))
 
 
+@pytest.mark.parametrize("n", [1, 17, 4097, MM_TILE + 5, 50 * MM_TILE + 123])
+@pytest.mark.parametrize("p", [0.0, 1e-3, 0.1, 1.0])
+def test_seg_scan_minmax_bf16(mmv, n, p):
+    # bfloat16 values over the whole exponent range (far beyond fp16's), exact comparison
+    rng = np.random.default_rng(n * 17 + int(p * 1000))
+    f = (rng.random(n) < p).astype(np.uint8)
+    xb = gen.bf16_bits_of((rng.standard_normal(n) * 10.0 ** rng.integers(-30, 30, n)).astype(np.float32))
+    for want_min in (False, True):
+        got = mmv.seg_scan_minmax(dev_bf16(xb), dev(f), want_min=want_min).cpu().numpy()
+        assert np.array_equal(got.astype(np.float64), oracle.seg_scan_minmax_bf16(xb, f, want_min))
+    got = mmv.seg_scan_minmax(dev_bf16(xb), None).cpu().numpy()
+    assert np.array_equal(got.astype(np.float64), oracle.seg_scan_minmax_bf16(xb, np.zeros(n, np.uint8)))
+
+
 def test_seg_scan_minmax_edges_and_long_carries(mmv):
     # a ramp that falls: the running maximum is carried from element 0 across every tile, the minimum is the input
     n = 400 * MM_TILE + 9
