@@ -137,10 +137,11 @@ class ClockSampler:
 # ---------------------------------------------------------------------------
 # the reference arm: the CPU oracle, as it stands
 # ---------------------------------------------------------------------------
-def time_oracle_scan(x, f, reps=2, got=None):
+def time_oracle_scan(x, f, reps=2, got=()):
     """Times the oracle's fp16 scan on (x, f).  The baseline leg has the oracle's result for the whole
-    workload in hand, so it also reports how far the device result `got` (a CUDA tensor) is from it,
-    as the largest |error| / bound over all elements."""
+    workload in hand, so it also reports how far each result in `got` (CUDA or host tensors: the device
+    scan and the chunked scan of the host vectors) is from it, as the largest |error| / bound over all
+    elements."""
     import oracle
     oracle.build()
     best, z, a = float("inf"), None, None
@@ -148,12 +149,13 @@ def time_oracle_scan(x, f, reps=2, got=None):
         t0 = time.perf_counter()
         z, a = oracle.seg_scan_f16(x, f)
         best = min(best, time.perf_counter() - t0)
-    worst = None
-    if got is not None:
-        worst, step = 0.0, 1 << 26
+    worst = []
+    for g in got:
+        w, step = 0.0, 1 << 26
         for o in range(0, x.shape[0], step):
-            _, ratio, _ = oracle.check_fp(got[o:o + step].cpu().numpy(), z[o:o + step], a[o:o + step])
-            worst = max(worst, ratio)
+            _, ratio, _ = oracle.check_fp(g[o:o + step].cpu().numpy(), z[o:o + step], a[o:o + step])
+            w = max(w, ratio)
+        worst.append(w)
     return best, worst
 
 
@@ -499,7 +501,9 @@ def run_ours(args):
     barrier()
     if mmv.last_async_status(scratch) != 0:
         raise SystemExit("bench: device-side error status (host scan)")
-    if not torch.allclose(oh[-(1 << 20):], od[-(1 << 20):].cpu(), rtol=1e-4, atol=1e-3):
+    # (the baseline leg below compares every element of this result with the oracle's; without that leg the
+    #  end of the vector is at least compared with the device scan)
+    if args.no_cpu and not torch.allclose(oh[-(1 << 20):], od[-(1 << 20):].cpu(), rtol=1e-4, atol=1e-3):
         raise SystemExit("bench: the chunked host scan and the device scan disagree")
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
@@ -531,15 +535,17 @@ def run_ours(args):
                          "traffic": (NCU_READ_BYTES_PER_ELEM + NCU_WRITE_BYTES_PER_ELEM) * n - NCU_WRITE_L2_RESIDUE_BYTES,
                          "traffic_source": "ncu capture at n=2^26 scaled by n (profiles/seg_scan_kernel_f16_n2p26_p1e-3.md)"},
         }
-        del xh, fh, oh
+        del xh, fh
         if not args.no_cpu:
             mmv.seg_scan(xd, fd, out=od, workspace=ws)
-            sec, worst = time_oracle_scan(x, f, reps=2, got=od)
+            sec, (worst, worst_host) = time_oracle_scan(x, f, reps=2, got=(od, oh))
             line["cpu_baseline"] = {"value": n / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                                     "sample": f"the whole headline workload (n=2^{args.log2n}), best of 2, {sec:.2f} s",
-                                    "device_result_worst_err_over_bound": worst}
-            if worst is not None and not worst <= 1.0:
-                raise SystemExit(f"bench: the device result is outside the bound (ratio {worst})")
+                                    "device_result_worst_err_over_bound": worst,
+                                    "host_vector_result_worst_err_over_bound": worst_host}
+            if not (worst <= 1.0 and worst_host <= 1.0):
+                raise SystemExit(f"bench: a result is outside the bound (device {worst}, host vectors {worst_host})")
+        del oh
         del xd, fd, od
         torch.cuda.empty_cache()
         if world == 1 and not args.no_configs:

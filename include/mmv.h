@@ -45,10 +45,15 @@
  *
  * Arithmetic
  *   MMV_F16_TO_F32  fp16 values, fp32 accumulation and output.  Results satisfy
- *                   |out - exact| <= 2e-3 * (sum of |x| over the summed range) + 1e-6
- *                   for inputs of the magnitude the library is specified for
- *                   (|x| of order 1); they are not bit-reproducible from run to
- *                   run because the grouping of the cross-tile carry chain
+ *                   |out - exact| <= 2e-3 * (sum of |x| over the summed range) + 1e-6.
+ *                   The scans (mmv_seg_scan, mmv_seg_scan_exclusive, the static and
+ *                   the host-vector form) hold this for any finite values whose
+ *                   sums stay finite in fp32: no result is ever formed as a
+ *                   difference of two prefixes, so a segment of tiny values
+ *                   behind a segment of huge ones keeps its own small bound.
+ *                   For mmv_seg_sum and mmv_spmv_csr see their comments.
+ *                   Floating-point results are not bit-reproducible from run
+ *                   to run because the grouping of the cross-tile carry chain
  *                   depends on timing.
  *   MMV_I8_TO_I32   int8 values, exact int32 result modulo 2^32 (bit-exact and
  *                   deterministic).

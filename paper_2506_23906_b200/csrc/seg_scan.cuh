@@ -18,9 +18,11 @@
 //                  formed with a handful of shuffles; the four spans of a tile exchange theirs
 //                  through shared memory and the tile's first warp publishes ONE status word
 //                  for the tile.
-//     main pass    per piece: revert the speculation inside each row (Lemma A.1: subtract the
-//                  prefix just before the element's segment start; the first element of a
-//                  segment takes the input value itself), segmented scan of the 32 row tails
+//     main pass    per piece: revert the speculation inside each row (Lemma A.1).  int8: subtract the
+//                  prefix just before the element's segment start, exact modulo 2^32.  Floating
+//                  point, where addition has no inverse: a piece that holds a start takes the rows
+//                  themselves (identity half) and forms the running sum since the last start, so
+//                  no prefix is ever subtracted from another.  Then a segmented scan of the 32 row tails
 //                  with shuffles, add the row carries (UpdateFirstSegment inside the span),
 //                  stage the 32 x 32 results in shared memory and write them with one TMA
 //                  store.  Pieces without any flag skip the revert.  Pieces that reach back
@@ -460,18 +462,28 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             tc_fence_after_sync();
 
             // ---- pre-pass: row totals, unit aggregate, publish ----
-            Acc tot[UP];
-#pragma unroll
-            for (int i = 0; i < UP; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * N + (ROW - 1)));
-            tmem_ld_wait();
             uint32_t anyp = 0u;
             int i0 = UP;                    // first piece with a flag
+            int istar = 0;                  // ... and the last one
 #pragma unroll
             for (int i = UP - 1; i >= 0; --i) {
                 anyp |= pm[i];
                 if (pm[i]) i0 = i;
             }
+#pragma unroll
+            for (int i = 0; i < UP; ++i)
+                if (pm[i]) istar = i;
             const bool flagged = anyp != 0u;
+            Acc tot[UP];
+#pragma unroll
+            for (int i = 0; i < UP; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * N + (ROW - 1)));
+            // floating point: the rows of the last flagged piece themselves (the identity half of the product)
+            // travel with the same wait; the tail behind the unit's last start is added up from them
+            uint32_t xr[Cfg::kWide ? 32 : 1];
+            if constexpr (Cfg::kWide) {
+                if (flagged) tmem_ld_32x32(taddr + istar * N + ROW, xr);
+            }
+            tmem_ld_wait();
             Acc tail_unit;
             if (!flagged) {
                 Acc t = tot[0];
@@ -479,10 +491,6 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 for (int i = 1; i < UP; ++i) t = P::add(t, tot[i]);
                 tail_unit = warp_sum<P>(t);
             } else {
-                int istar = 0;
-#pragma unroll
-                for (int i = 0; i < UP; ++i)
-                    if (pm[i]) istar = i;
                 uint32_t pms = pm[0], fms = fm[0];
                 Acc tots = tot[0];
 #pragma unroll
@@ -497,17 +505,24 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                     if (i > istar) after = P::add(after, tot[i]);
                 if (static_cast<int>(lane) > lstar) after = P::add(after, tots);
                 after = warp_sum<P>(after);
-                Acc before = Acc(0);
-                if (pl > 0) {
-                    before = P::from_bits(tmem_ld_32x1(taddr + istar * N + (pl - 1)));
-                    tmem_ld_wait();
-                }
-                Acc row_tail = P::sub(tots, before);
-                if constexpr (P::kIsFloat) {
-                    if (pl == ROW - 1) {          // the tail is a segment's first element: the input value itself
-                        row_tail = P::from_bits(tmem_ld_32x1(taddr + istar * N + ROW + (ROW - 1)));
+                Acc row_tail;
+                if constexpr (Cfg::kWide) {
+                    // Floating point addition has no inverse (Section 2 asks for a group): total - prefix(pl - 1)
+                    // would leave a small tail behind large values in the rounding of the two prefixes.  The
+                    // tail is the sum of the row's own values from its last start on (four partial sums, so
+                    // that the 32 additions are not one dependent chain).
+                    Acc part[4] = {Acc(0), Acc(0), Acc(0), Acc(0)};
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j >= pl) part[j & 3] = P::add(part[j & 3], P::from_bits(xr[j]));
+                    row_tail = P::add(P::add(part[0], part[1]), P::add(part[2], part[3]));
+                } else {
+                    Acc before = Acc(0);
+                    if (pl > 0) {
+                        before = P::from_bits(tmem_ld_32x1(taddr + istar * N + (pl - 1)));
                         tmem_ld_wait();
                     }
+                    row_tail = P::sub(tots, before);           // exact: integer arithmetic modulo 2^32 is a group
                 }
                 tail_unit = P::add(__shfl_sync(0xffffffffu, row_tail, lstar), after);
             }
@@ -562,11 +577,10 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                     if (i == q) { fmi = fm[q]; pmi = pm[q]; toti = tot[q]; }
                 if (i == i0) { fm0 = fmi; pm0 = pmi; }
                 uint32_t r[32];
-                uint32_t raw[P::kIsFloat ? 32 : 1];
-                tmem_ld_32x32(taddr + i * N, r);
-                if constexpr (Cfg::kWide) {
-                    if (pmi != 0u) tmem_ld_32x32(taddr + i * N + ROW, raw);
-                }
+                // a floating-point piece with a start takes its rows themselves (the identity half of the
+                // product), every other piece the speculative row prefixes
+                if constexpr (Cfg::kWide) tmem_ld_32x32(taddr + i * N + (pmi != 0u ? ROW : 0), r);
+                else tmem_ld_32x32(taddr + i * N, r);
                 tmem_ld_wait();
                 MMV_T_MARK(4)
                 if (PLAIN || pmi == 0u) {
@@ -577,24 +591,31 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                         const Acc t = __shfl_up_sync(0xffffffffu, inc, o);
                         if (static_cast<int>(lane) >= o) inc = P::add(t, inc);
                     }
-                    const Acc carry_row = P::add(run, P::sub(inc, toti));
+                    // (the exclusive value comes from the lane below, not as inc - toti: no subtraction in floating point)
+                    Acc exc = __shfl_up_sync(0xffffffffu, inc, 1);
+                    if (lane == 0) exc = Acc(0);
+                    const Acc carry_row = P::add(run, exc);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) r[j] = P::to_bits(P::add(carry_row, P::from_bits(r[j])));
                     run = P::add(run, __shfl_sync(0xffffffffu, inc, 31));
                 } else {
-                    // revert the speculation inside each row (Lemma A.1)
                     if constexpr (P::kIsFloat) {
-                        Acc base = Acc(0);
-                        uint32_t prev = 0u;
+                        // Reverting the speculation (Lemma A.1: z = prefix(j) - prefix(last start - 1)) is exact only in
+                        // a group, and a difference of two fp32 prefixes errs relative to the prefixes, not to the
+                        // segment behind them.  The same quantity is therefore formed without a subtraction, as the
+                        // running sum of the row's own values since the last start (since the row's beginning in
+                        // front of its first start).  One chain of 32 additions: splitting the row into two or four
+                        // independent chains measured slower (n = 2^30, every element a start: 1.17 / 1.19 / 1.22 ms),
+                        // the elements that continue the part before them cost more than the latency saved.
+                        Acc since = Acc(0);
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {
-                            const bool pj = (fmi >> j) & 1u;
-                            if (j > 0) base = pj ? P::from_bits(prev) : base;
-                            prev = r[j];
-                            // the first element of a segment is the input value itself, exactly
-                            r[j] = pj ? raw[j] : P::to_bits(P::sub(P::from_bits(r[j]), base));
+                            const Acc xj = P::from_bits(r[j]);
+                            since = ((fmi >> j) & 1u) ? xj : P::add(since, xj);
+                            r[j] = P::to_bits(since);
                         }
                     } else {
+                        // revert the speculation inside each row (Lemma A.1); exact modulo 2^32
                         Acc base = Acc(0);
                         uint32_t prev = 0u;
 #pragma unroll

@@ -203,6 +203,83 @@ def test_plain_scan_without_a_flag_vector(mmv):
     assert_fp(out.numpy(), z, a, "plain host scan")
 
 
+def _mixed_magnitude_segments(rng, nseg, max_len, small=1e-3, large=2e3):
+    """Segments of small values right behind segments of large ones (lengths 1..max_len, skewed to short)."""
+    lens = np.minimum(max_len, 1 + (rng.pareto(0.6, nseg) * 2).astype(np.int64))
+    lens[rng.integers(0, nseg, 8)] = max_len                       # a few of the longest, too
+    off = gen.offsets_from_lengths(lens)
+    n = int(off[-1])
+    scale = np.where(np.arange(nseg) % 2 == 0, large, small)       # every other segment is small
+    v = rng.standard_normal(n) * np.repeat(scale, lens)
+    f = oracle.flags_from_offsets(off, n)
+    return v, f, off
+
+
+def test_scan_tiny_segments_next_to_large_values(mmv):
+    # Floating-point addition is not a group (Section 2): prefix(j) - prefix(last start - 1) leaves a segment of
+    # values 1e-3 behind a segment of values 2e3 in the rounding of the prefixes, while the bound is relative to
+    # the segment's own sum of magnitudes.  Segment lengths 1 .. 5000: inside a row, across rows, pieces, units
+    # and tiles; inclusive and exclusive, flag- and offset-encoded, fp16 and bfloat16, device and host vectors.
+    rng = np.random.default_rng(2024)
+    v, f, off = _mixed_magnitude_segments(rng, 9000, 5000)
+    n = v.shape[0]
+    assert n > 20 * TILE
+    x = v.astype(np.float16)
+    z, a = oracle.seg_scan_f16(x, f)
+    assert_fp(scan_f16(mmv, x, f), z, a, "fp16 inclusive")
+    assert_fp(scan_f16(mmv, x, off), z, a, "fp16 inclusive, offsets")
+    e, ea = oracle.seg_scan_excl_f16(x, f)
+    assert_fp(scan_f16(mmv, x, f, exclusive=True), e, ea, "fp16 exclusive")
+    xb = gen.bf16_bits_of(v.astype(np.float32))
+    for exclusive in (False, True):
+        zb, ab = oracle.seg_scan_bf16(xb, f, exclusive=exclusive)
+        got = mmv.seg_scan(dev_bf16(xb), dev(f), exclusive=exclusive).cpu().numpy()
+        assert_fp(got, zb, ab, f"bf16 exclusive={exclusive}")
+    chunk = 4 * TILE
+    scratch = mmv.host_scan_scratch(mmv.F16_TO_F32, chunk)
+    out = mmv.seg_scan_host(torch.from_numpy(x).pin_memory(), torch.from_numpy(f).pin_memory(), chunk=chunk, scratch=scratch)
+    assert mmv.last_async_status(scratch) == 0
+    assert_fp(out.numpy(), z, a, "fp16 host vectors")
+    # dense starts: most rows of the layout hold several segments of both magnitudes
+    v, f, _ = _mixed_magnitude_segments(rng, 120000, 12)
+    x = v.astype(np.float16)
+    z, a = oracle.seg_scan_f16(x, f)
+    assert_fp(scan_f16(mmv, x, f), z, a, "fp16 inclusive, short segments")
+    e, ea = oracle.seg_scan_excl_f16(x, f)
+    assert_fp(scan_f16(mmv, x, f, exclusive=True), e, ea, "fp16 exclusive, short segments")
+
+
+def test_scan_mixed_magnitudes_inside_a_segment(mmv):
+    # The bound of an element is relative to the magnitudes IN FRONT of it in its segment: small values that
+    # open a segment keep a small bound even when large values follow in the same row, piece or unit, and
+    # large values that cancel (+a, -a) in front of a start must not leak into the segment behind it.
+    rng = np.random.default_rng(77)
+    n = 9 * TILE + 1500
+    v = rng.standard_normal(n) * 1e-3
+    f = (rng.random(n) < 0.004).astype(np.uint8)
+    starts = np.flatnonzero(f)
+    for s in starts[::3]:                                  # large values from the 3rd .. 40th element of a segment on
+        k = s + rng.integers(2, 40)
+        m = v[k:k + rng.integers(1, 200)].shape[0]
+        v[k:k + m] = rng.standard_normal(m) * 2e3
+    for s in starts[1::3]:                                 # a cancelling pair right in front of a start
+        if s >= 2:
+            v[s - 2], v[s - 1] = 3000.0, -3000.0
+    x = v.astype(np.float16)
+    z, a = oracle.seg_scan_f16(x, f)
+    assert_fp(scan_f16(mmv, x, f), z, a, "inclusive")
+    e, ea = oracle.seg_scan_excl_f16(x, f)
+    assert_fp(scan_f16(mmv, x, f, exclusive=True), e, ea, "exclusive")
+    # no start at all in long stretches: small leading values of the vector, large ones later (plain scan too)
+    v = rng.standard_normal(n) * 1e-3
+    v[3 * TILE + 517:] *= 1e6
+    x = v.astype(np.float16)
+    zero = np.zeros(n, np.uint8)
+    z, a = oracle.seg_scan_f16(x, zero)
+    assert_fp(scan_f16(mmv, x, zero), z, a, "one segment, flag vector")
+    assert_fp(mmv.seg_scan(dev(x), None).cpu().numpy(), z, a, "one segment, no flag vector")
+
+
 # ---------------------------------------------------------------------------
 # scan of host-resident vectors, chunk by chunk (carry handed from chunk to chunk on the device)
 # ---------------------------------------------------------------------------
