@@ -12,12 +12,23 @@
  *
  * Conventions for every entry point
  *   - All data pointers are DEVICE pointers unless a parameter says "host".
- *     The caller owns every buffer; the library never allocates, frees or
- *     keeps a pointer after the call returns.
+ *     The caller owns every buffer; the library allocates and frees no device
+ *     memory and keeps no pointer after the call returns.  Two entry points
+ *     hold resources of their own, each described at its declaration:
+ *     mmv_seg_scan_static (a fixed buffer inside the library's device image)
+ *     and mmv_seg_scan_host (three streams and nine events per device, made
+ *     at its first call and kept until the process exits).
  *   - `workspace` is caller-provided device scratch of at least
  *     mmv_workspace_bytes(...) bytes, 256-byte aligned; its content on entry is
  *     irrelevant (the call initialises what it needs on the stream) and it must
  *     not be shared by calls that may overlap on the GPU.
+ *   - Calls may overlap on the GPU (different streams, a workspace each).  The
+ *     tensor-core kernels (scan, segmented sum, SpMV) need every thread block
+ *     of their grid resident at once and are launched cooperatively: two such
+ *     calls that meet on the GPU run one after the other rather than side by
+ *     side, and where the process may use fewer SMs than the device reports
+ *     (an MPS thread limit, a green context) the launch is refused with
+ *     MMV_ERR_CUDA instead of stalling.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL =
  *     the default stream); the call does not synchronise with the host.
  *     mmv_seg_scan, mmv_seg_sum and mmv_spmv_csr enqueue nothing but a memset
@@ -122,6 +133,41 @@ mmv_status mmv_seg_scan_exclusive(const void *x, const void *seg, mmv_segfmt sf,
                                   void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * One vector cut into contiguous shards, one per GPU (Section 4.2, steps 3-6:
+ * the blocks' last values and flags are scanned and the result is added to the
+ * first segment of every block -- here a shard is the block, and the scan over
+ * the handful of shard records is done by every shard for itself).
+ *
+ * mmv_seg_scan_shard scans one shard as mmv_seg_scan would (flag-encoded
+ * segments; flags_u8 may be NULL: no start inside the shard) without the carry
+ * from the shards in front of it, and writes a 16-byte record to `summary`
+ * (device pointer, 16-byte aligned):
+ *     uint32  bits of the running sum at the shard's last element (fp32 / int32)
+ *     uint32  1 if a segment starts inside the shard, else 0
+ *     int64   index of the shard's first start, n if there is none
+ * first_shard != 0: element 0 opens a segment whatever its flag (Eq. 1).
+ * first_shard == 0: flag byte 0 counts like any other, and without it element 0
+ * continues the segment that reaches it from the shard in front.
+ * Workspace as for mmv_seg_scan (MMV_OP_SEG_SCAN, MMV_SEG_FLAGS_U8, n).
+ *
+ * The caller then gathers the records of all `world` shards, in shard order,
+ * into one buffer on every GPU (one all-gather of 16 bytes per shard: the only
+ * exchange of the path) and calls mmv_seg_scan_shard_finish on the same
+ * stream order: it folds the records of the shards in front of `rank` with
+ * (v1, f1) + (v2, f2) = (f2 ? v2 : v1 + v2, f1 | f2) and adds the resulting
+ * carry to out[0 .. first start of this shard).  With segment starts in every
+ * shard that touches a few elements; a shard without any start is rewritten
+ * once.  Both calls are asynchronous on cuda_stream; errors as for
+ * mmv_seg_scan (device-side status in the shard's workspace).
+ */
+#define MMV_SHARD_SUMMARY_BYTES 16
+mmv_status mmv_seg_scan_shard(const void *x, const void *flags_u8, int64_t n, mmv_dtype dt, int first_shard,
+                              void *out, void *summary,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream);
+mmv_status mmv_seg_scan_shard_finish(const void *summaries, int rank, int world, void *out, int64_t n,
+                                     mmv_dtype dt, void *cuda_stream);
+
+/*
  * Segmented sum (Section 2: the last element of every segment of the
  * segmented scan; Algorithm 4.2 computes the same quantity).
  * Offsets form: out has nseg entries, out[r] = sum of x over [off[r], off[r+1]),
@@ -135,6 +181,14 @@ mmv_status mmv_seg_scan_exclusive(const void *x, const void *seg, mmv_segfmt sf,
  * the workspace (COMPRESS, Section 2; the compaction step of Algorithm 4.2),
  * which therefore holds 4 (n + 1) bytes more than for the offsets form; nseg is
  * ignored.  n < 2^31 in both forms.
+ * Floating point: a sum is formed from differences of prefixes local to
+ * 32-element rows.  A segment that lies inside one row or two adjacent rows
+ * (in particular every segment of up to 32 elements) holds the bound for any
+ * finite values: a difference that came out small against its prefixes is
+ * added up again from the values themselves.  A longer segment holds it when
+ * the magnitudes inside its 4096-element span are within about 2^10 of each
+ * other; beyond that its absolute error is about 2^-22 of the largest prefix
+ * of the rows involved.
  */
 mmv_status mmv_seg_sum(const void *x, const void *seg, mmv_segfmt sf, int64_t n, int64_t nseg,
                        mmv_dtype dt, void *out, int64_t *d_num_segments,
@@ -192,8 +246,14 @@ mmv_status mmv_compress(const void *x, const void *flags, int64_t n, mmv_dtype d
 /*
  * CSR sparse matrix times dense vector built on the segmented sum
  * (Algorithm 4.4; Algorithms A.4-A.6):  y[r] = sum over k in
- * [rowptr[r], rowptr[r+1]) of val[k] * x[col[k]], fp32 products and sums, an
- * empty row gives exactly 0.  rowptr: rows+1 int32 with rowptr[0] == 0 and
+ * [rowptr[r], rowptr[r+1]) of val[k] * x[col[k]]; an empty row gives exactly
+ * 0.  Every product is formed in fp32 and handed to the tensor core as a pair
+ * of bfloat16 values (hi = bf16(z), lo = bf16(z - hi): relative error at most
+ * 2^-17 per product); the sums are fp32.  Rows of up to 32 non-zeros (and any
+ * row inside one or two adjacent 32-element rows of the product vector) hold
+ * the bound of "Arithmetic" above for any finite values; a longer row holds it
+ * when the magnitudes of the products inside a 4096-product span are within
+ * about 2^10 of each other (see mmv_seg_sum).  rowptr: rows+1 int32 with rowptr[0] == 0 and
  * rowptr[rows] == nnz < 2^31; col: nnz int32 in [0, cols) (duplicates simply
  * add; an index outside the range is never dereferenced, it contributes 0 and the
  * call records MMV_ERR_INVALID_ARG in the workspace status); val: nnz fp16;

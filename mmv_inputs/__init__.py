@@ -54,14 +54,16 @@ def i8_uniform_chunk(config: int, chunk: int, m: int = CHUNK, lo: int = -8, hi: 
     return _rng(config, S_VALUES, chunk).integers(lo, hi + 1, size=CHUNK, dtype=np.int8)[:m]
 
 
-def _full(fn, n: int, dtype, *a, **k) -> np.ndarray:
+def _full(fn, n: int, dtype, *a, first_chunk: int = 0, **k) -> np.ndarray:
     """All chunks of an array; chunks are independent, so large arrays are filled by a few threads
-    (numpy releases the GIL in the generators and conversions; the values do not depend on it)."""
+    (numpy releases the GIL in the generators and conversions; the values do not depend on it).
+    first_chunk > 0 gives the n elements that start at chunk `first_chunk` of a longer array
+    (a shard of it: the same values the whole array holds there)."""
     out = np.empty(n, dtype)
 
     def fill(cm):
         c, m = cm
-        out[c * CHUNK:c * CHUNK + m] = fn(*a, chunk=c, m=m, **k)
+        out[c * CHUNK:c * CHUNK + m] = fn(*a, chunk=first_chunk + c, m=m, **k)
 
     todo = list(_chunks(n))
     workers = min(len(todo), os.cpu_count() or 1, 16)
@@ -74,8 +76,8 @@ def _full(fn, n: int, dtype, *a, **k) -> np.ndarray:
     return out
 
 
-def f16_uniform(config: int, n: int, stream: int = S_VALUES) -> np.ndarray:
-    return _full(f16_uniform_chunk, n, np.float16, config, stream=stream)
+def f16_uniform(config: int, n: int, stream: int = S_VALUES, first_chunk: int = 0) -> np.ndarray:
+    return _full(f16_uniform_chunk, n, np.float16, config, stream=stream, first_chunk=first_chunk)
 
 
 def f16_normal(config: int, n: int, stream: int = S_VALUES) -> np.ndarray:
@@ -127,8 +129,8 @@ def flags_chunk(config: int, chunk: int, m: int = CHUNK, p: float = 1.0 / 64, pa
     return f
 
 
-def flags(config: int, n: int, p: float = 1.0 / 64, pattern: str = "bernoulli") -> np.ndarray:
-    return _full(flags_chunk, n, np.uint8, config, p=p, pattern=pattern)
+def flags(config: int, n: int, p: float = 1.0 / 64, pattern: str = "bernoulli", first_chunk: int = 0) -> np.ndarray:
+    return _full(flags_chunk, n, np.uint8, config, p=p, pattern=pattern, first_chunk=first_chunk)
 
 
 # --------------------------------------------------------------------------
@@ -325,10 +327,10 @@ def config4(rows: int = 1 << 20, cols: int | None = None, empty_fraction: float 
     return csr_matrix(4, rows, rows if cols is None else cols, empty_fraction=empty_fraction)
 
 
-def config5_values(n: int = 1 << 30):
-    return f16_uniform(5, n)
+def config5_values(n: int = 1 << 30, first_chunk: int = 0):
+    return f16_uniform(5, n, first_chunk=first_chunk)
 
 
-def config5_flags(n: int, case: str):
+def config5_flags(n: int, case: str, first_chunk: int = 0):
     kw = dict(C5_CASES)[case]
-    return flags(5, n, **kw)
+    return flags(5, n, first_chunk=first_chunk, **kw)

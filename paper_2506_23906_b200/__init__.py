@@ -27,8 +27,9 @@ EXPORTS = (
     "mmv_last_async_status", "mmv_status_string", "mmv_kernel_launch_count", "mmv_debug_configure",
     "mmv_seg_scan_static", "mmv_seg_scan_static_last_status", "mmv_debug_force_sum_groups",
     "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes", "mmv_seg_scan_exclusive", "mmv_compress",
-    "mmv_seg_scan_minmax", "mmv_seg_scan_i8_i64",
+    "mmv_seg_scan_minmax", "mmv_seg_scan_i8_i64", "mmv_seg_scan_shard", "mmv_seg_scan_shard_finish",
 )
+SHARD_SUMMARY_BYTES = 16
 STATIC_SCAN_MAX_N = 1 << 28
 
 
@@ -77,6 +78,10 @@ def _load() -> ctypes.CDLL:
     lib.mmv_seg_scan_host_scratch_bytes.argtypes = [ci, i64]
     lib.mmv_seg_scan_host.restype = ci
     lib.mmv_seg_scan_host.argtypes = [vp, vp, i64, ci, vp, i64, vp, sz, vp]
+    lib.mmv_seg_scan_shard.restype = ci
+    lib.mmv_seg_scan_shard.argtypes = [vp, vp, i64, ci, ci, vp, vp, vp, sz, vp]
+    lib.mmv_seg_scan_shard_finish.restype = ci
+    lib.mmv_seg_scan_shard_finish.argtypes = [vp, ci, ci, vp, i64, ci, vp]
     lib.mmv_debug_force_sum_groups.restype = None
     lib.mmv_debug_force_sum_groups.argtypes = [ci]
     return lib
@@ -164,6 +169,34 @@ def seg_scan(x: torch.Tensor, seg: torch.Tensor | None, out: torch.Tensor | None
     rc = call(_ptr(x), _ptr(seg), sf, n, nseg, dt, _ptr(out), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
     if rc != MMV_OK:
         raise MmvError(rc, "mmv_seg_scan_exclusive" if exclusive else "mmv_seg_scan")
+    return out
+
+
+def seg_scan_shard(x: torch.Tensor, flags: torch.Tensor | None, first_shard: bool, out: torch.Tensor, summary: torch.Tensor,
+                   workspace: torch.Tensor, stream=None) -> torch.Tensor:
+    """mmv_seg_scan_shard: scan of one contiguous shard of a longer vector, without the carry from the shards in
+    front of it; `summary` (16 bytes on the device, e.g. two int64) receives the shard's record."""
+    _check_cuda(x, flags, out, summary, workspace)
+    if summary.numel() * summary.element_size() < SHARD_SUMMARY_BYTES:
+        raise ValueError("summary needs 16 bytes")
+    rc = _lib.mmv_seg_scan_shard(_ptr(x), _ptr(flags), x.numel(), _dtype_code(x), 1 if first_shard else 0, _ptr(out),
+                                 _ptr(summary), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_seg_scan_shard")
+    return out
+
+
+def seg_scan_shard_finish(summaries: torch.Tensor, rank: int, world: int, out: torch.Tensor, x_dtype: torch.dtype,
+                          stream=None) -> torch.Tensor:
+    """mmv_seg_scan_shard_finish: fold the gathered records of the shards in front of `rank` and add the carry to
+    this shard's elements in front of its first start."""
+    _check_cuda(summaries, out)
+    if summaries.numel() * summaries.element_size() < world * SHARD_SUMMARY_BYTES:
+        raise ValueError("summaries needs 16 bytes per shard")
+    dt = I8_TO_I32 if x_dtype == torch.int8 else (BF16_TO_F32 if x_dtype == torch.bfloat16 else F16_TO_F32)
+    rc = _lib.mmv_seg_scan_shard_finish(_ptr(summaries), int(rank), int(world), _ptr(out), out.numel(), dt, _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_seg_scan_shard_finish")
     return out
 
 

@@ -28,9 +28,9 @@ std::atomic<int> g_force_groups{0};
 constexpr int kMaxDevices = 64;
 
 struct DeviceInfo {
-    std::once_flag once;
+    std::mutex lock;
+    std::atomic<bool> ok{false};
     int sm_count = 0;
-    bool ok = false;
     // copy-in / kernel / copy-out streams and their events for mmv_seg_scan_host (made on first use)
     std::once_flag pipe_once;
     bool pipe_ok = false;
@@ -62,43 +62,83 @@ bool set_smem(K kernel, int bytes) {
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
 }
 
+// Launch of a tiled tensor-core kernel (scan, segmented sum).  These kernels hand out their tiles in a fixed order
+// (tile = block + iteration * grid) and a tile waits for the carries of the tiles in front of it, so every CTA of
+// the grid has to be resident at the same time.  A cooperative launch makes the device guarantee that: the grid
+// starts only once all its CTAs fit together, whatever else runs on the GPU (another call of this library on a
+// second stream simply runs before or after it), and a grid that can never fit (fewer SMs than the device
+// reports: an MPS thread limit, a green context) is refused at launch instead of running into its time-out.
+// `programmatic`: the kernel may start while the kernel in front of it in the stream still runs (it waits with
+// griddepcontrol before it reads that kernel's results).  Measured: beside the cooperative attribute the early start
+// no longer happens for a launch made directly (configuration 2: 37.2 -> 39.2 us per call), while a call replayed
+// from a CUDA graph keeps it (32.8 vs 33.3 us); the attribute stays for the graph's sake.
+template <typename... KP, typename... A>
+cudaError_t launch_resident(void (*kernel)(KP...), int grid, int threads, int smem_bytes, cudaStream_t st, bool programmatic,
+                            const A&... args) {
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[2];
+    unsigned na = 0;
+    attr[na].id = cudaLaunchAttributeCooperative;
+    attr[na].val.cooperative = 1;
+    ++na;
+    if (programmatic) {
+        attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[na].val.programmaticStreamSerializationAllowed = 1;
+        ++na;
+    }
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(static_cast<unsigned>(threads));
+    cfg.dynamicSmemBytes = static_cast<size_t>(smem_bytes);
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = na;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, args...);
+    return err != cudaSuccess ? err : cudaGetLastError();
+}
+
 // Per-device one-time set-up: SM count and the kernels' dynamic shared-memory limits.
 DeviceInfo* device_info() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
     DeviceInfo* d = &g_dev[dev];
-    std::call_once(d->once, [d, dev] {
-        int sm = 0;
-        if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return;
-        d->sm_count = sm;
-        bool ok = true;
-        ok &= set_smem(seg_scan_kernel<F16Path>, ScanCfg<F16Path>::kSmemBytes);
-        ok &= set_smem(seg_scan_kernel<I8Path>, ScanCfg<I8Path>::kSmemBytes);
-        ok &= set_smem(seg_scan_kernel<F16Path, true>, ScanCfg<F16Path>::kSmemBytes);
-        ok &= set_smem(seg_scan_kernel<I8Path, true>, ScanCfg<I8Path>::kSmemBytes);
-        ok &= set_smem(seg_scan_kernel<BF16ValPath>, ScanCfg<BF16ValPath>::kSmemBytes);
-        ok &= set_smem(seg_scan_kernel<BF16ValPath, true>, ScanCfg<BF16ValPath>::kSmemBytes);
-        ok &= set_smem(seg_scan_kernel<F16Path, false, true>, ScanCfg<F16Path, true>::kSmemBytes);
-        ok &= set_smem(seg_scan_kernel<F16Path, true, true>, ScanCfg<F16Path, true>::kSmemBytes);
-        ok &= set_smem(seg_scan_kernel<BF16ValPath, false, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
-        ok &= set_smem(seg_scan_kernel<BF16ValPath, true, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
-        ok &= set_smem(seg_scan_minmax_kernel<0, false>, MM_SMEM_BYTES);
-        ok &= set_smem(seg_scan_minmax_kernel<0, true>, MM_SMEM_BYTES);
-        ok &= set_smem(seg_scan_minmax_kernel<1, false>, MM_SMEM_BYTES);
-        ok &= set_smem(seg_scan_minmax_kernel<1, true>, MM_SMEM_BYTES);
-        ok &= set_smem(seg_scan_minmax_kernel<2, false>, MM_SMEM_BYTES);
-        ok &= set_smem(seg_scan_minmax_kernel<2, true>, MM_SMEM_BYTES);
-        ok &= set_smem(seg_sum_kernel<BF16ValPath, 2>, SumCfg<BF16ValPath, 2>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<BF16ValPath, 3>, SumCfg<BF16ValPath, 3>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<F16Path, 2>, SumCfg<F16Path, 2>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<I8Path, 2>, SumCfg<I8Path, 2>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<BF16Path, 2>, SumCfg<BF16Path, 2>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<F16Path, 3>, SumCfg<F16Path, 3>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<I8Path, 3>, SumCfg<I8Path, 3>::kSmemBytes);
-        ok &= set_smem(seg_sum_kernel<BF16Path, 3>, SumCfg<BF16Path, 3>::kSmemBytes);
-        d->ok = ok;
-    });
-    return d->ok ? d : nullptr;
+    if (d->ok.load(std::memory_order_acquire)) return d;
+    // (only success is remembered: after a failed attempt the next call tries again)
+    std::lock_guard<std::mutex> guard(d->lock);
+    if (d->ok.load(std::memory_order_relaxed)) return d;
+    int sm = 0;
+    if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    d->sm_count = sm;
+    bool ok = true;
+    ok &= set_smem(seg_scan_kernel<F16Path>, ScanCfg<F16Path>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<I8Path>, ScanCfg<I8Path>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<F16Path, true>, ScanCfg<F16Path>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<I8Path, true>, ScanCfg<I8Path>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<BF16ValPath>, ScanCfg<BF16ValPath>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<BF16ValPath, true>, ScanCfg<BF16ValPath>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<F16Path, false, true>, ScanCfg<F16Path, true>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<F16Path, true, true>, ScanCfg<F16Path, true>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<BF16ValPath, false, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<BF16ValPath, true, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
+    ok &= set_smem(seg_scan_minmax_kernel<0, false>, MM_SMEM_BYTES);
+    ok &= set_smem(seg_scan_minmax_kernel<0, true>, MM_SMEM_BYTES);
+    ok &= set_smem(seg_scan_minmax_kernel<1, false>, MM_SMEM_BYTES);
+    ok &= set_smem(seg_scan_minmax_kernel<1, true>, MM_SMEM_BYTES);
+    ok &= set_smem(seg_scan_minmax_kernel<2, false>, MM_SMEM_BYTES);
+    ok &= set_smem(seg_scan_minmax_kernel<2, true>, MM_SMEM_BYTES);
+    ok &= set_smem(seg_sum_kernel<BF16ValPath, 2>, SumCfg<BF16ValPath, 2>::kSmemBytes);
+    ok &= set_smem(seg_sum_kernel<BF16ValPath, 3>, SumCfg<BF16ValPath, 3>::kSmemBytes);
+    ok &= set_smem(seg_sum_kernel<F16Path, 2>, SumCfg<F16Path, 2>::kSmemBytes);
+    ok &= set_smem(seg_sum_kernel<I8Path, 2>, SumCfg<I8Path, 2>::kSmemBytes);
+    ok &= set_smem(seg_sum_kernel<BF16Path, 2>, SumCfg<BF16Path, 2>::kSmemBytes);
+    ok &= set_smem(seg_sum_kernel<F16Path, 3>, SumCfg<F16Path, 3>::kSmemBytes);
+    ok &= set_smem(seg_sum_kernel<I8Path, 3>, SumCfg<I8Path, 3>::kSmemBytes);
+    ok &= set_smem(seg_sum_kernel<BF16Path, 3>, SumCfg<BF16Path, 3>::kSmemBytes);
+    if (!ok) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    d->ok.store(true, std::memory_order_release);
+    return d;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -274,26 +314,13 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     // With the partition kernel right in front, the tiled kernel is launched with programmatic
     // serialisation: its set-up (barriers, tensor memory, constant operand) overlaps the partition's end.
     const bool overlap = !have_partition;
-    cudaLaunchConfig_t cfg{};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.gridDim = dim3(static_cast<unsigned>(grid));
-    cfg.stream = st;
-    cfg.attrs = attr;
-    cfg.numAttrs = overlap ? 1 : 0;
     cudaError_t err;
-    if (g_force_groups.load() != 2) {
-        cfg.blockDim = dim3(SumShape<3>::kThreads);
-        cfg.dynamicSmemBytes = SumCfg<P, 3>::kSmemBytes;
-        err = cudaLaunchKernelEx(&cfg, seg_sum_kernel<P, 3>, tmap, values, prm);
-    } else {
-        cfg.blockDim = dim3(SumShape<2>::kThreads);
-        cfg.dynamicSmemBytes = SumCfg<P, 2>::kSmemBytes;
-        err = cudaLaunchKernelEx(&cfg, seg_sum_kernel<P, 2>, tmap, values, prm);
-    }
+    if (g_force_groups.load() != 2)
+        err = launch_resident(seg_sum_kernel<P, 3>, grid, SumShape<3>::kThreads, SumCfg<P, 3>::kSmemBytes, st, overlap, tmap, values, prm);
+    else
+        err = launch_resident(seg_sum_kernel<P, 2>, grid, SumShape<2>::kThreads, SumCfg<P, 2>::kSmemBytes, st, overlap, tmap, values, prm);
     ++g_launches;
-    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? MMV_OK : MMV_ERR_CUDA;
+    return err == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
 
 // f[off[r]] = 1 for every non-empty segment r (scratch flags of the offset-encoded scan).
@@ -321,21 +348,84 @@ constexpr size_t kStaticScratchBytes =
 static __device__ __align__(256) unsigned char g_static_scan_scratch[kStaticScratchBytes];
 
 struct StaticScratch {
-    std::once_flag once;
-    void* ptr = nullptr;
+    std::mutex lock;
+    std::atomic<void*> ptr{nullptr};
 };
 StaticScratch g_static_scratch[kMaxDevices];
 
-// Device address of the built-in scratch on the current device (nullptr on failure).
+// Device address of the built-in scratch on the current device (nullptr on failure).  Only a successful lookup
+// is remembered: after a failure (a first call made during stream capture, a transient error) the next call
+// tries again.
 void* static_scratch_ptr() {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
     StaticScratch* sc = &g_static_scratch[dev];
-    std::call_once(sc->once, [sc] {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scan_scratch) == cudaSuccess) sc->ptr = p;
-    });
-    return sc->ptr;
+    void* p = sc->ptr.load(std::memory_order_acquire);
+    if (p) return p;
+    std::lock_guard<std::mutex> guard(sc->lock);
+    p = sc->ptr.load(std::memory_order_relaxed);
+    if (p) return p;
+    if (cudaGetSymbolAddress(&p, g_static_scan_scratch) != cudaSuccess || !p) {
+        cudaGetLastError();            // the failure is reported through the return value, not left as a sticky error
+        return nullptr;
+    }
+    sc->ptr.store(p, std::memory_order_release);
+    return p;
+}
+
+// ---------------------------------------------------------------------------
+// One vector cut into contiguous shards (one per GPU): each shard is scanned by itself and described
+// by a 16-byte summary; the summaries of all shards are exchanged once (an all-gather, done by the
+// caller), every shard folds the ones in front of it into its carry and adds that carry to its
+// elements in front of its first start.  This is the block recursion of Section 4.2, steps 3-6 (scan
+// the blocks' last values and flags, then UpdateFirstSegment), with a shard as the block.
+// ---------------------------------------------------------------------------
+struct ShardSummary {
+    uint32_t value_bits;        // running sum at the shard's last element (fp32 or int32 bits), carry not included
+    uint32_t has_start;         // 1 if a segment starts inside the shard
+    long long first_start;      // index of the shard's first start, n if it has none
+};
+static_assert(sizeof(ShardSummary) == MMV_SHARD_SUMMARY_BYTES, "summary record is 16 bytes");
+
+__global__ void shard_summary_kernel(const uint32_t* __restrict__ out, long long n, const unsigned long long* __restrict__ first_word,
+                                     int first_shard, ShardSummary* __restrict__ summary) {
+    const unsigned long long w = *first_word;                   // n - (index of the first start), 0 = none
+    long long first = w ? n - static_cast<long long>(w) : n;
+    if (first_shard) first = 0;                                 // element 0 of the whole vector opens a segment
+    summary->value_bits = out[n - 1];
+    summary->has_start = first < n ? 1u : 0u;
+    summary->first_start = first;
+}
+
+// carry = fold of the summaries in front of `rank` with (v1, f1) + (v2, f2) = (f2 ? v2 : v1 + v2, f1 | f2);
+// out[i] += carry for i < first_start(rank)
+template <bool FP>
+__global__ void shard_finish_kernel(const ShardSummary* __restrict__ all, int rank, uint32_t* __restrict__ out, long long n) {
+    uint32_t carry_bits = 0u;
+    float cf = 0.f;
+    for (int r = 0; r < rank; ++r) {
+        const uint32_t v = all[r].value_bits;
+        if (FP) cf = all[r].has_start ? __uint_as_float(v) : cf + __uint_as_float(v);
+        else carry_bits = all[r].has_start ? v : carry_bits + v;
+    }
+    long long limit = all[rank].first_start;
+    if (limit > n) limit = n;
+    if (limit <= 0) return;
+    auto add = [&](uint32_t v) -> uint32_t { return FP ? __float_as_uint(cf + __uint_as_float(v)) : carry_bits + v; };
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    const long long tid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const long long nvec = limit >> 2;
+    uint4* o4 = reinterpret_cast<uint4*>(out);
+    for (long long v = tid; v < nvec; v += stride) {
+        uint4 q = o4[v];
+        q.x = add(q.x);
+        q.y = add(q.y);
+        q.z = add(q.z);
+        q.w = add(q.w);
+        o4[v] = q;
+    }
+    const long long k = (nvec << 2) + tid;
+    if (k < limit) out[k] = add(out[k]);
 }
 
 }  // namespace
@@ -356,8 +446,11 @@ size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, in
 }
 
 namespace {
+// shard: 0 = a whole vector; 1 = the first shard of a longer vector, 2 = a later shard (its flag byte 0 counts,
+// and without it element 0 continues the segment that reaches it).  For shards `summary` receives the record.
 mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
-                         void* out, void* workspace, size_t workspace_bytes, void* cuda_stream, bool exclusive) {
+                         void* out, void* workspace, size_t workspace_bytes, void* cuda_stream, bool exclusive,
+                         int shard = 0, void* summary = nullptr) {
     if (n < 0 || nseg < 0) return MMV_ERR_INVALID_ARG;
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return MMV_ERR_INVALID_ARG;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
@@ -407,11 +500,19 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
     prm.budget_ns = g_budget_ns.load();
     prm.debug_skip_span = g_debug_skip_span.load();
     prm.carry_in = nullptr;
+    prm.first_start = nullptr;
+    if (shard) {
+        // (header words behind the two counters, cleared with the header: the first-start word and a carry of zero)
+        prm.first_start = reinterpret_cast<unsigned long long*>(&hdr->reserved[0]);
+        if (shard == 2) prm.carry_in = &hdr->reserved[2];
+    }
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
     // (no flag vector: the floating-point paths run the narrow-tile variant)
     const bool plain = flags == nullptr;
+    cudaError_t err;
 #define MMV_LAUNCH_SCAN(PATH, EXCL, PL)                                                                               \
-    seg_scan_kernel<PATH, EXCL, PL><<<grid, ScanCfg<PATH, PL>::kThreads, ScanCfg<PATH, PL>::kSmemBytes, st>>>(tmap, tmap_out, prm)
+    err = launch_resident(seg_scan_kernel<PATH, EXCL, PL>, grid, ScanCfg<PATH, PL>::kThreads, ScanCfg<PATH, PL>::kSmemBytes, st, \
+                          false, tmap, tmap_out, prm)
     if (dt == MMV_I8_TO_I32) {
         if (exclusive) MMV_LAUNCH_SCAN(I8Path, true, false);
         else MMV_LAUNCH_SCAN(I8Path, false, false);
@@ -428,7 +529,14 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
     }
 #undef MMV_LAUNCH_SCAN
     ++g_launches;
-    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+    if (err != cudaSuccess) return MMV_ERR_CUDA;
+    if (shard) {
+        shard_summary_kernel<<<1, 1, 0, st>>>(static_cast<const uint32_t*>(out), n, prm.first_start, shard == 1 ? 1 : 0,
+                                              static_cast<ShardSummary*>(summary));
+        ++g_launches;
+        if (cudaGetLastError() != cudaSuccess) return MMV_ERR_CUDA;
+    }
+    return MMV_OK;
 }
 }  // namespace
 
@@ -440,6 +548,41 @@ mmv_status mmv_seg_scan(const void* x, const void* seg, mmv_segfmt sf, int64_t n
 mmv_status mmv_seg_scan_exclusive(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
                                   void* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return seg_scan_impl(x, seg, sf, n, nseg, dt, out, workspace, workspace_bytes, cuda_stream, true);
+}
+
+mmv_status mmv_seg_scan_shard(const void* x, const void* flags_u8, int64_t n, mmv_dtype dt, int first_shard, void* out,
+                              void* summary, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (!summary || (reinterpret_cast<uintptr_t>(summary) & 15u)) return MMV_ERR_INVALID_ARG;
+    if (n == 0) {
+        // an empty shard: no start, nothing summed
+        return cudaMemsetAsync(summary, 0, sizeof(ShardSummary), static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+    }
+    return seg_scan_impl(x, flags_u8, MMV_SEG_FLAGS_U8, n, 0, dt, out, workspace, workspace_bytes, cuda_stream, false,
+                         first_shard ? 1 : 2, summary);
+}
+
+mmv_status mmv_seg_scan_shard_finish(const void* summaries, int rank, int world, void* out, int64_t n, mmv_dtype dt,
+                                     void* cuda_stream) {
+    if (n < 0 || world <= 0 || rank < 0 || rank >= world) return MMV_ERR_INVALID_ARG;
+    if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return MMV_ERR_INVALID_ARG;
+    if (!summaries || (reinterpret_cast<uintptr_t>(summaries) & 15u)) return MMV_ERR_INVALID_ARG;
+    if (n == 0 || rank == 0) return MMV_OK;                        // nothing in front of the first shard
+    if (!out || !aligned16(out)) return MMV_ERR_INVALID_ARG;
+    DeviceInfo* dev = device_info();
+    if (!dev) return MMV_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int threads = 256;
+    long long blocks = ((n >> 2) + threads - 1) / threads;
+    const long long cap = static_cast<long long>(dev->sm_count) * 8;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    const ShardSummary* all = static_cast<const ShardSummary*>(summaries);
+    if (dt == MMV_I8_TO_I32)
+        shard_finish_kernel<false><<<static_cast<unsigned>(blocks), threads, 0, st>>>(all, rank, static_cast<uint32_t*>(out), n);
+    else
+        shard_finish_kernel<true><<<static_cast<unsigned>(blocks), threads, 0, st>>>(all, rank, static_cast<uint32_t*>(out), n);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
 
 // ---------------------------------------------------------------------------
@@ -555,13 +698,15 @@ mmv_status mmv_seg_scan_host(const void* x_host, const void* flags_host, int64_t
         prm.budget_ns = g_budget_ns.load();
         prm.debug_skip_span = -1;
         prm.carry_in = carry;
+        prm.first_start = nullptr;
         const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
         if (f16)
-            seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, dev->s_k>>>(tmap, tmap_out, prm);
+            ok &= launch_resident(seg_scan_kernel<F16Path>, grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, dev->s_k,
+                                  false, tmap, tmap_out, prm) == cudaSuccess;
         else
-            seg_scan_kernel<I8Path><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, dev->s_k>>>(tmap, tmap_out, prm);
+            ok &= launch_resident(seg_scan_kernel<I8Path>, grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, dev->s_k,
+                                  false, tmap, tmap_out, prm) == cudaSuccess;
         ++g_launches;
-        ok &= cudaGetLastError() == cudaSuccess;
         ok &= cudaEventRecord(dev->k_done[b], dev->s_k) == cudaSuccess;
         carry = od + static_cast<size_t>(m - 1) * 4;           // the running sum at the end of this chunk
         // copy out
@@ -836,15 +981,19 @@ mmv_status mmv_seg_scan_static(const void* x, const void* flags_u8, int64_t n, m
     prm.hdr = reinterpret_cast<WorkspaceHeader*>(ws);
     prm.status = reinterpret_cast<uint64_t*>(ws + sizeof(WorkspaceHeader));
     prm.budget_ns = g_budget_ns.load();
-    prm.debug_skip_span = -1;
+    prm.debug_skip_span = g_debug_skip_span.load();
     prm.carry_in = nullptr;
+    prm.first_start = nullptr;
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
+    cudaError_t err;
     if (f16)
-        seg_scan_kernel<F16Path><<<grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+        err = launch_resident(seg_scan_kernel<F16Path>, grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, st, false,
+                              tmap, tmap_out, prm);
     else
-        seg_scan_kernel<I8Path><<<grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st>>>(tmap, tmap_out, prm);
+        err = launch_resident(seg_scan_kernel<I8Path>, grid, ScanCfg<I8Path>::kThreads, ScanCfg<I8Path>::kSmemBytes, st, false,
+                              tmap, tmap_out, prm);
     ++g_launches;
-    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+    return err == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
 
 mmv_status mmv_seg_scan_static_last_status(void* cuda_stream) {

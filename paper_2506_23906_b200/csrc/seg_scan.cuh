@@ -51,6 +51,9 @@ struct ScanParams {
     const void* carry_in;        // device pointer to one fp32 / int32, or null: the running sum that
                                  // reaches element 0 from an earlier chunk of the same vector (element 0
                                  // then continues that segment unless its flag is set)
+    unsigned long long* first_start;   // device word, or null: receives n - (index of the vector's first start)
+                                 // by atomicMax (it begins at 0 = no start); used when the vector is one
+                                 // shard of a longer one, whose carry belongs in front of that index
 };
 
 // Scan geometry: a warp owns a UNIT of SCAN_UP consecutive pieces (the grain of the carry
@@ -96,16 +99,19 @@ struct ScanCfg {
 #define MMV_SCAN_PLAIN_GROUPS 4
 #endif
     static constexpr int kGroups = kWide ? 2 : ((PLAIN && P::kIsFloat) ? MMV_SCAN_PLAIN_GROUPS : MMV_SCAN_I8_GROUPS);
-    static constexpr int kBufsPerGroup = kWide ? 1 : (kGroups == 2 ? 2 : 1);
-    static constexpr int kBufs = kGroups * kBufsPerGroup;                // TMEM tile buffers
+    static constexpr int kTmemCols = 512;
+    // TMEM tile buffers: as many as fit.  Iteration `it` of the CTA uses buffer it % kBufs, whichever warpgroup
+    // takes it, so with more buffers than warpgroups (int8 with three groups: four) the products of a group's
+    // next tile are finished while all groups are still busy with their current ones
+    // (int8, n = 2^28: every second element a start 274 -> 266 us, p = 1e-3 280 -> 278 us).
+    static constexpr int kBufs = kTmemCols / (SCAN_UP * kN);
     static constexpr int kEpiWarps = 4 * kGroups;
     static constexpr int kProducerWarp = kEpiWarps;
     static constexpr int kMmaWarp = kEpiWarps + 1;
     static constexpr int kThreads = (kEpiWarps + 2) * 32;
-    static constexpr int kTmemCols = 512;
     static constexpr int kStages = kWide ? 3 : ((kGroups == 2 || kGroups == 4) ? 4 : 3);
     static_assert(kStages >= kGroups, "the producer's closing round needs a stage per warpgroup");
-    static_assert(kBufs * SCAN_UP * kN <= kTmemCols, "tile buffers fit the tensor memory");
+    static_assert(kBufs >= kGroups && kBufs * SCAN_UP * kN <= kTmemCols, "a tile buffer per warpgroup, all inside the tensor memory");
     static constexpr int kBBytes = kN * P::kRowBytes;                    // constant operand [U_32 | I_32] / U_32
     static constexpr int kBSlot = 4096;
     static constexpr int kXBytes = SCAN_UP * P::kSlabBytes;
@@ -117,7 +123,7 @@ struct ScanCfg {
     static constexpr int kOutBufs = kGroups >= 4 ? 1 : 2;                // staging buffers per warp
     static constexpr int kOutBytes = kEpiWarps * kOutBufs * kOutBufBytes;
     static constexpr int kBarOffset = kOutOffset + kOutBytes;
-    static constexpr int kSmemBytes = kBarOffset + 512 + 1024;
+    static constexpr int kSmemBytes = kBarOffset + 640 + 1024;        // barriers and small slots, alignment slack
     static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of one CTA");
     static_assert(kBBytes <= kBSlot, "constant operand fits its slot");
     static_assert(kStageOffset % 1024 == 0 && kStageBytes % 1024 == 0 && kOutOffset % 1024 == 0, "swizzle atoms");
@@ -185,12 +191,16 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     volatile int* stage_iter = tile_slot + S;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tile_slot + 2 * S);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    // smallest index of a start that this CTA has reported so far (its tiles come in ascending order, so only its
+    // first few units with a start ever go to the global word)
+    volatile long long* cta_first = reinterpret_cast<volatile long long*>((reinterpret_cast<uintptr_t>(tmem_slot + 2) + 7) & ~uintptr_t(7));
 
     const int warp = threadIdx.x >> 5;
     const uint32_t lane = lane_id();
     const uint64_t budget = prm.budget_ns;
 
     if (threadIdx.x == 0) {
+        *cta_first = 0x7fffffffffffffffll;
         for (int i = 0; i < S; ++i) {
             mbar_init(&bar_full[i], 1);
             mbar_init(&bar_empty[i], 4);      // the group's four warps, once their flag bytes are read
@@ -345,9 +355,8 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 if (++sentinels == Cfg::kGroups) break;
                 continue;
             }
-            const int g = it % Cfg::kGroups, k = it / Cfg::kGroups;
-            const int buf = g * Cfg::kBufsPerGroup + (k % Cfg::kBufsPerGroup);
-            if (!wait_bar(&bar_acc_empty[buf], ((k / Cfg::kBufsPerGroup) & 1) ^ 1, abort_flag, budget)) {
+            const int buf = it % Cfg::kBufs;
+            if (!wait_bar(&bar_acc_empty[buf], ((it / Cfg::kBufs) & 1) ^ 1, abort_flag, budget)) {
                 *abort_flag = 1;
                 if (lane == 0) report_error(prm.hdr, 5u);
                 break;
@@ -433,7 +442,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             if (tile < 0) break;
             MMV_T_MARK(0)
 
-            const int buf = g * Cfg::kBufsPerGroup + (k % Cfg::kBufsPerGroup);
+            const int buf = it % Cfg::kBufs;
             const uint32_t taddr = tmem_base + buf * (UP * N) + ((static_cast<uint32_t>(w) * 32u) << 16);
             const long long s = static_cast<long long>(tile) * SPANS_PER_TILE + w;      // this warp's unit
 
@@ -455,7 +464,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 }
             }
             MMV_T_MARK(1)
-            if (!wait_bar(&bar_acc_full[buf], (k / Cfg::kBufsPerGroup) & 1, abort_flag, budget)) { failed = true; break; }
+            if (!wait_bar(&bar_acc_full[buf], (it / Cfg::kBufs) & 1, abort_flag, budget)) { failed = true; break; }
             MMV_T_MARK(2)
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_empty[stage]);      // operands consumed, flags in registers
@@ -697,6 +706,13 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             // ---- parked pieces: add the carry in front of the unit's first flag, store ----
             const int l0 = pm0 ? (__ffs(pm0) - 1) : 32;                       // first flagged row of piece i0
             const int fpos = __ffs(__shfl_sync(0xffffffffu, fm0, l0 & 31)) - 1;  // its first flag
+            if (prm.first_start != nullptr && flagged && lane == 0) {
+                const long long gidx = s * SCAN_UNIT + i0 * PIECE + l0 * ROW + fpos;       // this unit's first start
+                if (gidx < *cta_first) {
+                    *cta_first = gidx;
+                    atomicMax(prm.first_start, static_cast<unsigned long long>(prm.n - gidx));
+                }
+            }
             Acc prev_parked = carry;           // exclusive variant: what stands in front of the unit's first element
 #pragma unroll 1
             for (int i = 0; i <= i0 && i < UP; ++i) {

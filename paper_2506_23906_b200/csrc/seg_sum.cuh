@@ -59,7 +59,6 @@ struct SumShape {
     static constexpr int kProducerWarp = 4 * G;
     static constexpr int kMmaWarp = 4 * G + 1;
     static constexpr int kThreads = (4 * G + 2) * 32;
-    static constexpr int kBufsPerGroup = G == 2 ? 2 : 1;
 };
 constexpr int SUM_SPARSE_MAX = 8;                                  // spans with at most this many boundaries read single prefixes from TMEM
 constexpr int SUM_DIRECT_LEN = 4;                                  // few-boundaries path: segments this short are summed from the inputs
@@ -397,7 +396,6 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
     using Acc = typename P::Acc;
     using Cfg = SumCfg<P, G>;
     using Shape = SumShape<G>;
-    constexpr int BPG = Shape::kBufsPerGroup;
     constexpr int S = Cfg::kStages;
 
     extern __shared__ uint8_t smem_raw[];
@@ -550,9 +548,10 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 if (++sentinels == 2) break;
                 continue;
             }
-            const int g = it % G, k = it / G;
-            const int buf = g * BPG + (k % BPG);
-            if (!wait_bar(&bar_acc_empty[buf], ((k / BPG) & 1) ^ 1, abort_flag, budget)) {
+            // iteration `it` uses buffer it % SUM_BUFS whichever warpgroup takes it: with three groups and four
+            // buffers the products of a group's next tile are finished while all groups are still busy
+            const int buf = it % SUM_BUFS;
+            if (!wait_bar(&bar_acc_empty[buf], ((it / SUM_BUFS) & 1) ^ 1, abort_flag, budget)) {
                 *abort_flag = 1;
                 if (lane == 0) report_error(prm.hdr, 5u);
                 break;
@@ -643,7 +642,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             // tile order it knows its tile without being told
             const int tile = tile_of(k);
             if (tile < 0) break;
-            const int buf = g * BPG + (k % BPG);
+            const int it = g + G * k;
+            const int buf = it % SUM_BUFS;
             const long long s = static_cast<long long>(tile) * SPANS_PER_TILE + w;
             const long long sbase = s * SPAN;
             const long long send = sbase + SPAN;
@@ -749,7 +749,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             }
 
             MMV_T_MARK(0)
-            if (!wait_bar(&bar_acc_full[buf], (k / BPG) & 1, abort_flag, budget)) { failed = true; break; }
+            if (!wait_bar(&bar_acc_full[buf], (it / SUM_BUFS) & 1, abort_flag, budget)) { failed = true; break; }
             tc_fence_after_sync();
             MMV_T_MARK(1)
             // request the next tile's offsets (its first index has arrived by now): they travel while this

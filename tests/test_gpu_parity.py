@@ -1005,6 +1005,48 @@ def test_minmax_lookback_wait_gives_up_with_a_status(mmv):
 # the calls only enqueue a memset and kernels on the given stream: they can be captured in a CUDA
 # graph and replayed (the first call on a device, which sets the kernels' attributes, comes before)
 # ---------------------------------------------------------------------------
+def test_calls_that_overlap_on_two_streams(mmv):
+    # The tiled kernels hand out their tiles in a fixed order and need every CTA of their grid resident; they are
+    # launched cooperatively, so two calls that overlap in time on two streams (each with a workspace of its own)
+    # run one after the other instead of sharing the SMs and waiting for tiles whose CTAs never started.  A 200 ms
+    # wait budget turns any such stall into MMV_ERR_TIMEOUT quickly; what is promised is that none occurs.
+    mmv.debug_configure(200_000_000, -1)
+    try:
+        n = (1 << 27) + 4321
+        rng = np.random.default_rng(99)
+        xs = [rng.integers(-128, 128, n).astype(np.int8) for _ in range(2)]
+        fs = [(rng.random(n) < p).astype(np.uint8) for p in (1e-5, 0.02)]
+        want = [oracle.seg_scan_i8(x, f) for x, f in zip(xs, fs)]
+        xd, fd = [dev(x) for x in xs], [dev(f) for f in fs]
+        outs = [torch.empty(n, dtype=torch.int32, device="cuda") for _ in range(2)]
+        wss = [mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n) for _ in range(2)]
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        torch.cuda.synchronize()
+        for _ in range(6):                               # back to back, no host synchronisation in between
+            for i in range(2):
+                mmv.seg_scan(xd[i], fd[i], out=outs[i], workspace=wss[i], stream=streams[i])
+        for i in range(2):
+            assert mmv.last_async_status(wss[i], streams[i]) == 0
+            assert np.array_equal(outs[i].cpu().numpy(), want[i])
+        # a scan beside a segmented sum
+        x2, off = gen.config2(1 << 24, max_len=300)
+        nseg = off.shape[0] - 1
+        x2d, offd = dev(x2), dev(off)
+        out2 = torch.empty(nseg, dtype=torch.float32, device="cuda")
+        ws2 = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, x2.shape[0], nseg)
+        torch.cuda.synchronize()
+        for _ in range(6):
+            mmv.seg_scan(xd[0], fd[0], out=outs[0], workspace=wss[0], stream=streams[0])
+            mmv.seg_sum(x2d, offd, out=out2, workspace=ws2, stream=streams[1])
+        assert mmv.last_async_status(wss[0], streams[0]) == 0
+        assert mmv.last_async_status(ws2, streams[1]) == 0
+        assert np.array_equal(outs[0].cpu().numpy(), want[0])
+        w2, a2 = oracle.seg_sum_csr_f16(x2, off)
+        assert_fp(out2.cpu().numpy(), w2, a2, "segmented sum beside a scan")
+    finally:
+        mmv.debug_configure(0, -1)
+
+
 def test_calls_replay_from_a_cuda_graph(mmv):
     rng = np.random.default_rng(5)
     n = 3 * TILE + 4001
@@ -1057,3 +1099,87 @@ def test_calls_replay_from_a_cuda_graph(mmv):
     assert np.array_equal(o5.cpu().numpy(), oracle.seg_scan_i8_wide(x, f))
     kept = oracle.compress(x, f)
     assert int(k6.item()) == kept.shape[0] and np.array_equal(o6[:kept.shape[0]].cpu().numpy(), kept)
+
+
+# ---------------------------------------------------------------------------
+# one vector scanned as contiguous shards (the multi-GPU path, all shards on this GPU)
+# ---------------------------------------------------------------------------
+def scan_in_shards(mmv, x, f, cuts):
+    """x/f cut at `cuts`: every shard is scanned by itself, the 16-byte records are gathered into one buffer
+    (here by device copies; across GPUs by one all-gather) and every shard adds its carry."""
+    n = x.shape[0]
+    edges = [0] + list(cuts) + [n]
+    world = len(edges) - 1
+    odt = torch.int32 if x.dtype == np.int8 else torch.float32
+    xd = dev_bf16(x) if x.dtype == np.uint16 else dev(x)
+    fd = dev(f)
+    out = torch.full((n + 64,), -777, dtype=odt, device="cuda")
+    gathered = torch.zeros(2 * world, dtype=torch.int64, device="cuda")
+    mine = [torch.zeros(2, dtype=torch.int64, device="cuda") for _ in range(world)]
+    wss = []
+    for r in range(world):
+        a, b = edges[r], edges[r + 1]
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, max(1, b - a))
+        wss.append(ws)
+        mmv.seg_scan_shard(xd[a:b], fd[a:b], r == 0, out[a:b], mine[r], ws)
+    for r in range(world):
+        gathered[2 * r:2 * r + 2] = mine[r]                       # the all-gather
+    for r in range(world):
+        a, b = edges[r], edges[r + 1]
+        mmv.seg_scan_shard_finish(gathered, r, world, out[a:b], xd.dtype)
+    for ws in wss:
+        assert mmv.last_async_status(ws) == 0
+    got = out.cpu().numpy()
+    assert (got[n:] == -777).all()
+    return got[:n], gathered.cpu().numpy().reshape(world, 2)
+
+
+@pytest.mark.parametrize("p", [0.0, 1e-5, 1e-3, 0.3])
+def test_scan_in_four_shards_matches_the_whole_vector(mmv, p):
+    rng = np.random.default_rng(int(p * 1e6) + 3)
+    n = 37 * TILE + 4321
+    cuts = [8 * TILE, 8 * TILE + 16 * 1000, 30 * TILE + 16]        # shard edges must keep 16-byte alignment of x, f, out
+    f = (rng.random(n) < p).astype(np.uint8)
+    f[cuts[1]] = 1                                                  # one shard begins with a start ...
+    f[cuts[2]] = 0                                                  # ... another continues the segment in front of it
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    got, rec = scan_in_shards(mmv, xi, f, cuts)
+    assert np.array_equal(got, oracle.seg_scan_i8(xi, f))
+    # the records: first start of every shard (flag byte 0 of shard 0 is not consulted: element 0 starts)
+    edges = [0] + cuts + [n]
+    for r in range(4):
+        fl = f[edges[r]:edges[r + 1]].copy()
+        if r == 0:
+            fl[0] = 1
+        nz = np.flatnonzero(fl)
+        assert rec[r, 1] == (nz[0] if nz.size else fl.shape[0])
+        assert (rec[r, 0] >> 32) == (1 if nz.size else 0)
+    xf = rng.uniform(-1, 1, n).astype(np.float16)
+    z, a = oracle.seg_scan_f16(xf, f)
+    assert_fp(scan_in_shards(mmv, xf, f, cuts)[0], z, a, f"fp16 in shards, p={p}")
+    xb = gen.bf16_normal(12, n)
+    zb, ab = oracle.seg_scan_bf16(xb, f)
+    assert_fp(scan_in_shards(mmv, xb, f, cuts)[0], zb, ab, f"bf16 in shards, p={p}")
+
+
+def test_scan_in_shards_edges(mmv):
+    # shards shorter than a tile, a single shard, a shard without any start between two that have one, and the
+    # flag-free call (no flag vector at all)
+    rng = np.random.default_rng(8)
+    n = 5 * TILE + 48
+    xi = rng.integers(-128, 128, n).astype(np.int8)
+    f = np.zeros(n, np.uint8)
+    f[[100, 4 * TILE + 7]] = 1
+    for cuts in ([], [16], [16, 32, 48], [TILE, 3 * TILE], [n - 16]):
+        got, _ = scan_in_shards(mmv, xi, f, cuts)
+        assert np.array_equal(got, oracle.seg_scan_i8(xi, f)), cuts
+    world, m = 3, TILE + 160
+    x3 = torch.from_numpy(xi[:world * m]).cuda()
+    out = torch.empty(world * m, dtype=torch.int32, device="cuda")
+    gathered = torch.zeros(2 * world, dtype=torch.int64, device="cuda")
+    for r in range(world):
+        ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, m)
+        mmv.seg_scan_shard(x3[r * m:(r + 1) * m], None, r == 0, out[r * m:(r + 1) * m], gathered[2 * r:2 * r + 2], ws)
+    for r in range(world):
+        mmv.seg_scan_shard_finish(gathered, r, world, out[r * m:(r + 1) * m], torch.int8)
+    assert np.array_equal(out.cpu().numpy(), oracle.seg_scan_i8(xi[:world * m], np.zeros(world * m, np.uint8)))

@@ -61,3 +61,53 @@ def test_static_scan_refuses_inputs_beyond_its_buffer(mmv):
                                       out.data_ptr(), None)
     assert rc == 3 and "workspace" in mmv.status_string(rc)
     assert mmv._lib.mmv_seg_scan_static(x.data_ptr(), f.data_ptr(), 0, mmv.I8_TO_I32, out.data_ptr(), None) == 0
+    # exactly the largest size is accepted (checked for real: all-ones values, one segment, closed form i + 1)
+    n = mmv.STATIC_SCAN_MAX_N
+    x = torch.ones(n, dtype=torch.int8, device="cuda")
+    f = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    out = torch.empty(n, dtype=torch.int32, device="cuda")
+    mmv.seg_scan_static(x, f, out)
+    assert mmv.seg_scan_static_last_status() == 0
+    step = 1 << 26
+    for o in range(0, n, step):
+        assert torch.equal(out[o:o + step], torch.arange(o + 1, o + step + 1, dtype=torch.int32, device="cuda"))
+
+
+def test_static_scan_allocates_nothing(mmv):
+    # what the entry point is for: after one warm-up call (module load, first-use set-up) a call changes neither
+    # the driver's free-memory figure nor the bytes PyTorch's allocator holds
+    n = 5 * 16384 + 77
+    rng = np.random.default_rng(5)
+    x = torch.from_numpy(rng.integers(-128, 128, n).astype(np.int8)).cuda()
+    f = torch.from_numpy((rng.random(n) < 0.01).astype(np.uint8)).cuda()
+    out = torch.empty(n, dtype=torch.int32, device="cuda")
+    mmv.seg_scan_static(x, f, out)
+    assert mmv.seg_scan_static_last_status() == 0
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    held0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+    for _ in range(3):
+        mmv.seg_scan_static(x, f, out)
+    assert mmv.seg_scan_static_last_status() == 0
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0
+    assert torch.cuda.memory_allocated() == held0 and torch.cuda.memory_reserved() == reserved0
+    assert np.array_equal(out.cpu().numpy(), oracle.seg_scan_i8(x.cpu().numpy(), f.cpu().numpy()))
+
+
+def test_static_scan_reports_a_wait_that_ran_out(mmv):
+    # the time-out path through mmv_seg_scan_static_last_status: one span never publishes its carry (host-side
+    # test switch, no GPU fault), its successors give up after 20 ms; the next call on the shared buffer works
+    n = 40 * 16384
+    x = torch.ones(n, dtype=torch.int8, device="cuda")
+    f = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    out = torch.empty(n, dtype=torch.int32, device="cuda")
+    mmv.debug_configure(20_000_000, 8)
+    try:
+        mmv.seg_scan_static(x, f, out)
+        assert mmv.seg_scan_static_last_status() == 5            # MMV_ERR_TIMEOUT
+    finally:
+        mmv.debug_configure(0, -1)
+    mmv.seg_scan_static(x, f, out)
+    assert mmv.seg_scan_static_last_status() == 0
+    assert torch.equal(out, torch.arange(1, n + 1, dtype=torch.int32, device="cuda"))
