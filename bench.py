@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
 # DRAM traffic of the headline kernel from the ncu capture of its n = 2^26 case
-# (profiles/seg_scan_kernel_f16_n2p26_p1e-3.md): reads 3.003 B/element, writes 4 B/element minus
+# (the summary of that capture is kept with the other profiles): reads 3.003 B/element, writes 4 B/element minus
 # the ~58 MB of output that are still in L2 when a launch ends; both scale with n.
 NCU_READ_BYTES_PER_ELEM = 3.003
 NCU_WRITE_BYTES_PER_ELEM = 4.0
@@ -192,9 +192,42 @@ def run_reference(args):
 # our arm
 # ---------------------------------------------------------------------------
 def shard_plan(world: int, rank: int, log2n: int):
-    """Work of one rank: the path has no exchange step, so every rank scans its own shard of the
-    same size (weak scaling) and only the timing is reduced (max over ranks)."""
-    return {"rank": rank, "world": world, "n": 1 << log2n, "collectives_on_data_path": 0}
+    """Work of one rank.  N = 1: the whole vector.  N > 1: ONE vector of world * 2^log2n elements cut into
+    contiguous shards, rank r holding elements [r * 2^log2n, (r + 1) * 2^log2n) (weak scaling: the shard size
+    is fixed).  Every shard is scanned by itself; the one exchange of the path is an all-gather of the
+    16-byte shard records, after which every rank folds the records in front of it into its carry."""
+    n = 1 << log2n
+    if n % gen.CHUNK and world > 1:
+        raise SystemExit("bench: shards are whole generator chunks (log2n >= 24) when --gpus > 1")
+    return {"rank": rank, "world": world, "n": n, "global_n": world * n,
+            "first_chunk": rank * (n // gen.CHUNK) if world > 1 else 0,
+            "collectives_on_data_path": 1 if world > 1 else 0}
+
+
+def shard_record(last_value_bits: int, first_start: int, n: int):
+    """The 16-byte record of a shard as two int64 words, laid out as mmv_seg_scan_shard writes it:
+    word 0 = value bits | has_start << 32, word 1 = index of the first start (n if none)."""
+    has = 1 if first_start < n else 0
+    return np.array([(int(last_value_bits) & 0xffffffff) | (has << 32), int(first_start)], dtype=np.int64)
+
+
+def fold_records(records, rank: int, is_float: bool = True):
+    """Carry into shard `rank`: the fold of the records in front of it with the operator of the segmented
+    scan on pairs, (v1, f1) + (v2, f2) = (f2 ? v2 : v1 + v2, f1 | f2) (Section 4.2, steps 3-5, applied to the
+    shards' last values and flags).  `records`: world x 2 int64 as gathered.  Written for the CPU test of the
+    shard plan and for the benchmark's own cross-check; the library folds on the device."""
+    rec = np.asarray(records, dtype=np.int64).reshape(-1, 2)
+    carry = np.float32(0.0) if is_float else 0
+    for r in range(rank):
+        bits = int(rec[r, 0]) & 0xffffffff
+        has = (int(rec[r, 0]) >> 32) & 1
+        if is_float:
+            v = np.array([bits], dtype=np.uint32).view(np.float32)[0]
+            carry = v if has else np.float32(carry + v)
+        else:
+            v = bits - (1 << 32) if bits >= (1 << 31) else bits
+            carry = v if has else ((carry + v + (1 << 31)) % (1 << 32)) - (1 << 31)
+    return carry
 
 
 def reduce_max_over_ranks(torch, dist, values, device):
@@ -433,13 +466,16 @@ def run_ours(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        # (a bounded time-out: a rank that dies leaves the others with an error, not with an endless wait)
+        import datetime
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local), timeout=datetime.timedelta(seconds=300))
 
     import paper_2506_23906_b200 as mmv
 
-    n = 1 << args.log2n
-    x = gen.f16_uniform(5, n)
-    f = gen.config5_flags(n, args.case)
+    plan = shard_plan(world, rank, args.log2n)
+    n = plan["n"]
+    x = gen.config5_values(n, first_chunk=plan["first_chunk"])
+    f = gen.config5_flags(n, args.case, first_chunk=plan["first_chunk"])
     peak, peak_kind = measured_peak()
 
     # pinned host buffers (end-to-end leg) and device-resident copies (kernel leg)
@@ -453,9 +489,25 @@ def run_ours(args):
     xd.copy_(xh)
     fd.copy_(fh)
     l2_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    # N > 1: this rank's 16-byte shard record and the gathered records of all ranks
+    my_record = torch.zeros(2, dtype=torch.int64, device="cuda")
+    records = torch.zeros(2 * world, dtype=torch.int64, device="cuda")
 
-    def step():
-        mmv.seg_scan(xd, fd, out=od, workspace=ws)
+    if world == 1:
+        def step():
+            mmv.seg_scan(xd, fd, out=od, workspace=ws)
+        load_step = step
+    else:
+        def step():
+            # shard scan -> one all-gather of the records (NCCL, the path's only exchange) -> local fold + carry
+            mmv.seg_scan_shard(xd, fd, rank == 0, od, my_record, ws)
+            dist.all_gather_into_tensor(records, my_record)
+            mmv.seg_scan_shard_finish(records, rank, world, od, torch.float16)
+
+        def load_step():
+            # the same kernels without the exchange: what keeps the GPU busy while the clocks are sampled (every
+            # rank makes its own number of these, so they must not contain a collective)
+            mmv.seg_scan_shard(xd, fd, rank == 0, od, my_record, ws)
 
     def barrier():
         torch.cuda.synchronize()
@@ -481,7 +533,7 @@ def run_ours(args):
         t_extra0 = time.perf_counter()
         while clk.count_between(t_load0, time.perf_counter()) < 6 and time.perf_counter() - t_extra0 < 1.5:
             for _ in range(16):
-                step()
+                load_step()
             torch.cuda.synchronize()
         t_load1 = time.perf_counter()
     clocks = clk.summary(t_load0, t_load1)
@@ -491,20 +543,39 @@ def run_ours(args):
         raise SystemExit("bench: device-side error status")
 
     # end to end: the library's call for HOST vectors (pinned): every step copies the 3 n input bytes
-    # to the device, scans, and brings the 4 n result bytes back, chunk by chunk on three streams
+    # to the device, scans, and brings the 4 n result bytes back, chunk by chunk on three streams.
+    # N > 1: the shard's inputs are copied in, the shard path above runs, the result is copied out.
     e2e_steps = max(1, min(args.steps, 5))
     e2e_chunk = min(1 << 25, n)
-    scratch = mmv.host_scan_scratch(mmv.F16_TO_F32, e2e_chunk)
-    def e2e_step():
-        mmv.seg_scan_host(xh, fh, out=oh, chunk=e2e_chunk, scratch=scratch)
+    if world == 1:
+        scratch = mmv.host_scan_scratch(mmv.F16_TO_F32, e2e_chunk)
+
+        def e2e_step():
+            mmv.seg_scan_host(xh, fh, out=oh, chunk=e2e_chunk, scratch=scratch)
+    else:
+        scratch = ws
+
+        def e2e_step():
+            xd.copy_(xh, non_blocking=True)
+            fd.copy_(fh, non_blocking=True)
+            step()
+            oh.copy_(od, non_blocking=True)
     e2e_step()
     barrier()
     if mmv.last_async_status(scratch) != 0:
         raise SystemExit("bench: device-side error status (host scan)")
     # (the baseline leg below compares every element of this result with the oracle's; without that leg the
     #  end of the vector is at least compared with the device scan)
-    if args.no_cpu and not torch.allclose(oh[-(1 << 20):], od[-(1 << 20):].cpu(), rtol=1e-4, atol=1e-3):
-        raise SystemExit("bench: the chunked host scan and the device scan disagree")
+    if (args.no_cpu or world > 1) and not torch.allclose(oh[-(1 << 20):], od[-(1 << 20):].cpu(), rtol=1e-4, atol=1e-3):
+        raise SystemExit("bench: the scan of the host vectors and the device scan disagree")
+    if world > 1:
+        # cross-check of the exchange: the carry this rank added must be the fold of the gathered records as
+        # the definition gives it, and element 0 must continue the shard in front (or start a segment)
+        carry = float(fold_records(records.cpu().numpy(), rank))
+        first = int(my_record.cpu()[1])
+        want0 = float(x[0]) + (0.0 if (rank == 0 or first == 0) else carry)
+        if abs(float(od[0].cpu()) - want0) > 2e-3 * (abs(carry) + 1.0) + 1e-6:
+            raise SystemExit(f"bench: rank {rank}: element 0 is {float(od[0].cpu())}, expected {want0}")
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         e2e_step()
@@ -522,21 +593,25 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": f"C5 seg-scan n=2^{args.log2n} fp16 U[-1,1) -> fp32, uint8 flags {args.case}",
                        "n_per_gpu": n, "timing": "inputs (7 B/elem working set) larger than L2; no flush needed",
-                       "parallelism": f"{world} independent shards, no collective"},
+                       "parallelism": ("one GPU" if world == 1 else
+                                       f"one vector of {world} x 2^{args.log2n} elements in {world} contiguous shards; per step one "
+                                       f"all-gather of {world} 16-byte shard records (NCCL), carries folded locally")},
             "clocks": clocks,
             "e2e": {"value": whole_job_value(world, n, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": 3 * n,
                     "d2h_bytes_per_step": 4 * n, "ms_per_step": e2e_ms, "steps": e2e_steps,
-                    "call": f"mmv_seg_scan_host, pinned host vectors, chunks of 2^{int(np.log2(e2e_chunk))} elements"},
+                    "call": (f"mmv_seg_scan_host, pinned host vectors, chunks of 2^{int(np.log2(e2e_chunk))} elements" if world == 1
+                             else "copy in, mmv_seg_scan_shard, all-gather, mmv_seg_scan_shard_finish, copy out (pinned host vectors)")},
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": peak_kind,
                          "frac_of_8tbs_nominal": achieved / NOMINAL_HBM_GBS,
                          "algorithmic_bytes_per_elem": 7,
+                         "algorithmic_bytes": bytes_per_launch,
                          "traffic": (NCU_READ_BYTES_PER_ELEM + NCU_WRITE_BYTES_PER_ELEM) * n - NCU_WRITE_L2_RESIDUE_BYTES,
-                         "traffic_source": "ncu capture at n=2^26 scaled by n (profiles/seg_scan_kernel_f16_n2p26_p1e-3.md)"},
+                         "traffic_kind": "constant from an ncu capture of this kernel at n=2^26, scaled by n (not a counter of this run)"},
         }
         del xh, fh
-        if not args.no_cpu:
+        if not args.no_cpu and world == 1:
             mmv.seg_scan(xd, fd, out=od, workspace=ws)
             sec, (worst, worst_host) = time_oracle_scan(x, f, reps=2, got=(od, oh))
             line["cpu_baseline"] = {"value": n / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
@@ -545,6 +620,15 @@ def run_ours(args):
                                     "host_vector_result_worst_err_over_bound": worst_host}
             if not (worst <= 1.0 and worst_host <= 1.0):
                 raise SystemExit(f"bench: a result is outside the bound (device {worst}, host vectors {worst_host})")
+            # the same definition chunk-parallel over all cores this process may use (sequential carry hand-over)
+            import oracle
+            best_all, used = float("inf"), 0
+            for _ in range(2):
+                t0 = time.perf_counter()
+                _, _, used = oracle.seg_scan_f16_all_cores(x, f)
+                best_all = min(best_all, time.perf_counter() - t0)
+            line["cpu_baseline_all_cores"] = {"value": n / best_all / 1e9, "unit": UNIT, "cores": used, "kind": "oracle, chunk-parallel",
+                                              "sample": f"the whole headline workload (n=2^{args.log2n}), best of 2, {best_all:.2f} s"}
         del oh
         del xd, fd, od
         torch.cuda.empty_cache()
@@ -565,7 +649,7 @@ def run_ours(args):
                 torch.cuda.synchronize()
                 cms = event_time_ms(torch, fn, min(args.steps, 10))
                 assert mmv.last_async_status(ws) == 0
-                sweep.append({"case": case, "ms": cms, "gelem_s": n / cms / 1e6, "gb_s": 7 * n / cms / 1e6,
+                sweep.append({"tag": case, "case": case, "ms": cms, "gelem_s": n / cms / 1e6, "gb_s": 7 * n / cms / 1e6,
                               "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
                               "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
                 del fd
@@ -576,7 +660,7 @@ def run_ours(args):
             torch.cuda.synchronize()
             cms = event_time_ms(torch, fn, min(args.steps, 10))
             assert mmv.last_async_status(ws) == 0
-            sweep.append({"case": "no flag vector (plain scan, 6 B/elem)", "ms": cms, "gelem_s": n / cms / 1e6,
+            sweep.append({"tag": "plain", "case": "no flag vector (plain scan, 6 B/elem)", "ms": cms, "gelem_s": n / cms / 1e6,
                           "gb_s": 6 * n / cms / 1e6, "frac_of_measured_peak": 6 * n / cms / 1e6 / peak,
                           "frac_of_8tbs": 6 * n / cms / 1e6 / NOMINAL_HBM_GBS})
             # the exclusive variant on the headline flags (same traffic)
@@ -587,7 +671,7 @@ def run_ours(args):
             torch.cuda.synchronize()
             cms = event_time_ms(torch, fn, min(args.steps, 10))
             assert mmv.last_async_status(ws) == 0
-            sweep.append({"case": f"exclusive scan, {args.case}", "ms": cms, "gelem_s": n / cms / 1e6,
+            sweep.append({"tag": "excl", "case": f"exclusive scan, {args.case}", "ms": cms, "gelem_s": n / cms / 1e6,
                           "gb_s": 7 * n / cms / 1e6, "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
                           "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
             # bfloat16 input values (the headline values converted on the device), same flags and traffic
@@ -598,7 +682,7 @@ def run_ours(args):
             torch.cuda.synchronize()
             cms = event_time_ms(torch, fn, min(args.steps, 10))
             assert mmv.last_async_status(ws) == 0
-            sweep.append({"case": f"bf16 values, {args.case}", "ms": cms, "gelem_s": n / cms / 1e6,
+            sweep.append({"tag": "bf16", "case": f"bf16 values, {args.case}", "ms": cms, "gelem_s": n / cms / 1e6,
                           "gb_s": 7 * n / cms / 1e6, "frac_of_measured_peak": 7 * n / cms / 1e6 / peak,
                           "frac_of_8tbs": 7 * n / cms / 1e6 / NOMINAL_HBM_GBS})
             # segmented running maximum and the plain running maximum (CUDA cores: the operator has no inverse)
@@ -610,7 +694,7 @@ def run_ours(args):
                 torch.cuda.synchronize()
                 cms = event_time_ms(torch, fn, min(args.steps, 10))
                 assert mmv.last_async_status(wsm) == 0
-                sweep.append({"case": label, "ms": cms, "gelem_s": n / cms / 1e6, "gb_s": per * n / cms / 1e6,
+                sweep.append({"tag": "max" if fl is not None else "max-plain", "case": label, "ms": cms, "gelem_s": n / cms / 1e6, "gb_s": per * n / cms / 1e6,
                               "frac_of_measured_peak": per * n / cms / 1e6 / peak,
                               "frac_of_8tbs": per * n / cms / 1e6 / NOMINAL_HBM_GBS})
             del wsm
@@ -624,7 +708,7 @@ def run_ours(args):
             torch.cuda.synchronize()
             cms = event_time_ms(torch, fn, min(args.steps, 10))
             assert mmv.last_async_status(wsw) == 0
-            sweep.append({"case": f"int8 -> int64 scan, {args.case} (10 B/elem)", "ms": cms, "gelem_s": n / cms / 1e6,
+            sweep.append({"tag": "i8->i64", "case": f"int8 -> int64 scan, {args.case} (10 B/elem)", "ms": cms, "gelem_s": n / cms / 1e6,
                           "gb_s": 10 * n / cms / 1e6, "frac_of_measured_peak": 10 * n / cms / 1e6 / peak,
                           "frac_of_8tbs": 10 * n / cms / 1e6 / NOMINAL_HBM_GBS})
             del xi8, od64, wsw
@@ -639,12 +723,18 @@ def run_ours(args):
             cms = event_time_ms(torch, fn, min(args.steps, 10))
             kept = int(kc.item())
             cbytes = n + 4 * kept
-            sweep.append({"case": f"COMPRESS, {args.case} ({kept} kept)", "ms": cms, "gelem_s": n / cms / 1e6,
+            sweep.append({"tag": "compress", "case": f"COMPRESS, {args.case} ({kept} kept)", "ms": cms, "gelem_s": n / cms / 1e6,
                           "gb_s": cbytes / cms / 1e6, "frac_of_measured_peak": cbytes / cms / 1e6 / peak,
                           "frac_of_8tbs": cbytes / cms / 1e6 / NOMINAL_HBM_GBS})
             del fd, xb, outc, wsc
             line["configs"] = cfgs
             line["c5_density_sweep"] = sweep
+            # a compact digest as the LAST key, so that the end of the line alone shows every case:
+            # [name, time in us, GB/s of algorithmic bytes, fraction of the nominal 8 TB/s]
+            digest = [[c["config"].split(" ")[0], round(c["ms"] * 1e3, 1), round(c["gb_s"]), round(c["frac_of_8tbs"], 3)]
+                      for c in cfgs if "ms" in c]
+            digest += [["C5/" + c["tag"], round(c["ms"] * 1e3, 1), round(c["gb_s"]), round(c["frac_of_8tbs"], 3)] for c in sweep]
+            line["digest_name_us_gbs_fracof8tbs"] = digest
         print(json.dumps(line))
     if world > 1:
         dist.barrier()

@@ -18,6 +18,7 @@ import numpy as np
 
 _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "mmv_oracle.c"
+_SRC_PAR = _HERE / "mmv_oracle_par.c"
 _LIB = _HERE / "libmmv_oracle.so"
 _lib = None
 
@@ -29,11 +30,11 @@ TOL_ABS = 1e-6
 
 def build(force: bool = False) -> Path:
     """Compile the oracle's C file into a shared library next to it."""
-    if force or not _LIB.exists() or _LIB.stat().st_mtime < _SRC.stat().st_mtime:
+    if force or not _LIB.exists() or _LIB.stat().st_mtime < max(_SRC.stat().st_mtime, _SRC_PAR.stat().st_mtime):
         tmp = _LIB.with_suffix(f".{os.getpid()}.tmp")
         subprocess.run(
-            ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fno-fast-math",
-             "-o", str(tmp), str(_SRC), "-lm"],
+            ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fno-fast-math", "-pthread",
+             "-o", str(tmp), str(_SRC), str(_SRC_PAR), "-lm"],
             check=True,
         )
         os.replace(tmp, _LIB)
@@ -100,6 +101,22 @@ def seg_scan_f16(x, f, state=None):
     if state is not None and n > 0:
         state["open"] = True
     return z, a
+
+
+def seg_scan_f16_all_cores(x, f, threads: int | None = None):
+    """Eq. (1) on fp16 values, chunk-parallel over `threads` host threads (default: the cores this
+    process may use) with a sequential carry hand-over between the chunks.  Returns (z, a, threads used)."""
+    xb, fb = _as_f16_bits(x), _as(f, np.uint8)
+    n = xb.shape[0]
+    assert fb.shape[0] == n
+    if threads is None:
+        threads = len(os.sched_getaffinity(0))
+    z = np.empty(n, np.float64)
+    a = np.empty(n, np.float64)
+    used = _load().mmv_oracle_seg_scan_f16_chunks(_p(xb), _p(fb), ctypes.c_int64(n), _p(z), _p(a), ctypes.c_int(int(threads)))
+    if used <= 0:
+        raise MemoryError("mmv_oracle_seg_scan_f16_chunks")
+    return z, a, int(used)
 
 
 def new_f16_state():

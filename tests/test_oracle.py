@@ -638,3 +638,32 @@ def test_running_max_and_min_of_bfloat16_values():
             assert oracle.seg_scan_minmax_bf16(xb, f, want_min).tolist() == want
         assert np.array_equal(oracle.seg_scan_minmax_bf16(xb, f, True), -oracle.seg_scan_minmax_bf16(xb ^ np.uint16(0x8000), f, False))
         assert np.array_equal(oracle.seg_scan_minmax_bf16(xb, np.zeros(n, np.uint8)), np.maximum.accumulate(xd))
+
+
+# ---------------------------------------------------------------------------
+# the all-cores form of the fp16 scan (timed beside the one-core oracle by the benchmark)
+# ---------------------------------------------------------------------------
+def test_all_cores_scan_equals_the_sequential_oracle():
+    # the paper's worked example of Section 2, cut into 3 chunks: (2,2,3 | 3,1,3 | 1,2) -> (2,4,3,6,7,3,4,6)
+    x = np.array([2, 2, 3, 3, 1, 3, 1, 2], np.float16)
+    f = np.array([1, 0, 1, 0, 0, 1, 0, 0], np.uint8)
+    z, a, used = oracle.seg_scan_f16_all_cores(x, f, threads=3)
+    assert used == 3 and z.tolist() == [2, 4, 3, 6, 7, 3, 4, 6] and a.tolist() == [2, 4, 3, 6, 7, 3, 4, 6]
+    rng = np.random.default_rng(31)
+    for n, p, threads in [(1, 0.5, 4), (7, 0.0, 8), (1000, 0.01, 7), (100003, 1e-4, 8), (100003, 0.0, 5), (4096, 1.0, 3),
+                          (50000, 0.3, 1)]:
+        x = rng.uniform(-1, 1, n).astype(np.float16)
+        f = (rng.random(n) < p).astype(np.uint8)
+        z0, a0 = oracle.seg_scan_f16(x, f)
+        z1, a1, used = oracle.seg_scan_f16_all_cores(x, f, threads=threads)
+        assert used == min(threads, n)
+        # one more fp64 addition per element than the sequential recurrence: equal to ~1e-16 of the magnitudes
+        assert np.all(np.abs(z1 - z0) <= 1e-13 * a0 + 1e-300), (n, p, threads)
+        assert np.all(np.abs(a1 - a0) <= 1e-13 * a0 + 1e-300), (n, p, threads)
+    # chunks without any start between chunks that have one: the carry passes through
+    n = 90
+    x = np.ones(n, np.float16)
+    f = np.zeros(n, np.uint8)
+    f[[5, 80]] = 1
+    z, _, _ = oracle.seg_scan_f16_all_cores(x, f, threads=9)
+    assert np.array_equal(z, oracle.seg_scan_f16(x, f)[0])
