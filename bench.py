@@ -731,8 +731,8 @@ def run_ours(args):
             line["c5_density_sweep"] = sweep
             # a compact digest as the LAST key, so that the end of the line alone shows every case:
             # [name, time in us, GB/s of algorithmic bytes, fraction of the nominal 8 TB/s]
-            digest = [[c["config"].split(" ")[0], round(c["ms"] * 1e3, 1), round(c["gb_s"]), round(c["frac_of_8tbs"], 3)]
-                      for c in cfgs if "ms" in c]
+            digest = [[c["config"].split(" ")[0] + (("/" + c["config"].split("(")[-1].rstrip(")")) if c["config"].startswith("T5.1") else ""),
+                       round(c["ms"] * 1e3, 1), round(c["gb_s"]), round(c["frac_of_8tbs"], 3)] for c in cfgs if "ms" in c]
             digest += [["C5/" + c["tag"], round(c["ms"] * 1e3, 1), round(c["gb_s"]), round(c["frac_of_8tbs"], 3)] for c in sweep]
             line["digest_name_us_gbs_fracof8tbs"] = digest
         print(json.dumps(line))

@@ -26,7 +26,7 @@ def build(force: bool = False, verbose: bool = False) -> Path:
         return LIB
     tmp = LIB.with_suffix(f".{os.getpid()}.tmp")
     cmd = [NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "--use_fast_math" if False else "-DNDEBUG",
+           "-shared", "-Xcompiler", "-fPIC", "-DNDEBUG",
            "-o", str(tmp)] + os.environ.get("MMV_NVCC_FLAGS", "").split() + [str(s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")

@@ -6,7 +6,10 @@
 
 namespace mmv {
 
-// Optional phase timers (compile with -DMMV_PHASE_TIMERS): cycles summed over all epilogue warps.
+// Phase timers, a supported build flag for performance work (MMV_NVCC_FLAGS=-DMMV_PHASE_TIMERS python
+// paper_2506_23906_b200/build.py --force): every epilogue warp adds the cycles it spends between the
+// MMV_T_MARK points of the scan and segmented-sum kernels to 16 global counters, which the extra export
+// mmv_debug_phase_cycles reads and clears.  Without the flag the macros are empty and nothing is compiled in.
 #ifdef MMV_PHASE_TIMERS
 __device__ unsigned long long g_phase_cycles[16];
 #define MMV_T_DECL long long t_prev = clock64(); unsigned long long t_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
@@ -104,14 +107,16 @@ __device__ __forceinline__ uint32_t swz_offset(uint32_t row, uint32_t byte_in_ro
     return row * RowBytes + (chunk << 4) + (byte_in_row & 15u);
 }
 
-// Shared-memory matrix descriptor of a K-major swizzled slab (see ptx.cuh for the fields).
+// Shared-memory matrix descriptor of a K-major swizzled slab: rows of RowBytes bytes, groups of 8 rows contiguous,
+// the 16-byte chunk index XOR-ed with a function of the row (swz_offset above).  `addr` = shared address of the
+// first row plus the byte offset of the K slice inside the row.
 __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t sbo_bytes, uint32_t layout_type) {
     uint64_t d = 0;
-    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);
-    d |= static_cast<uint64_t>(1) << 16;
-    d |= static_cast<uint64_t>(sbo_bytes >> 4) << 32;
-    d |= static_cast<uint64_t>(1) << 46;
-    d |= static_cast<uint64_t>(layout_type) << 61;
+    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);        // start address, bits [0,14)
+    d |= static_cast<uint64_t>(1) << 16;                       // leading byte offset (unused for swizzled K-major)
+    d |= static_cast<uint64_t>(sbo_bytes >> 4) << 32;          // stride byte offset: 8 rows
+    d |= static_cast<uint64_t>(1) << 46;                       // descriptor version (sm_100)
+    d |= static_cast<uint64_t>(layout_type) << 61;             // 2 = 128-byte, 4 = 64-byte, 6 = 32-byte swizzle
     return d;
 }
 

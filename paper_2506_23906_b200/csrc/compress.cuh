@@ -4,6 +4,9 @@
 // so the flag-encoded segmented sum is this compaction followed by the offset-encoded kernel.
 // Three small streaming kernels: per-chunk counts, one-block exclusive scan of the counts,
 // in-order scatter of the positions.  Element 0 always starts a segment, whatever f(0) holds.
+// The count pass is the only one that reads the flag bytes: it leaves one bit per flag (a 64-bit
+// mask per thread, n / 8 bytes in the workspace) and the scatter pass reads those instead, an
+// eighth of the bytes.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -13,11 +16,6 @@ namespace mmv {
 constexpr int CMP_THREADS = 256;
 constexpr int CMP_PER_THREAD = 64;                              // flag bytes per thread: four 16-byte vectors
 constexpr int CMP_CHUNK = CMP_THREADS * CMP_PER_THREAD;         // 16384 flags per block iteration
-
-// number of non-zero bytes of a word
-__device__ __forceinline__ int nonzero_bytes(uint32_t w) {
-    return __popc((((w & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w) & 0x80808080u);
-}
 
 // The 64 flag bytes of thread t of chunk c as 16 words (zero past n; with first_is_start byte 0 of the
 // vector is forced to 1: element 0 opens a segment whatever its flag says).
@@ -69,19 +67,32 @@ __device__ __forceinline__ int block_exclusive_scan(int v, int* total, int* warp
     return before + inc - v;
 }
 
-// chunk_count[c] = number of segment starts among the flags of chunk c.
+// bit b of the result = byte b of the 64 flag bytes in w is non-zero
+__device__ __forceinline__ unsigned long long flag_words_to_mask(const uint32_t (&w)[16]) {
+    uint32_t lo = 0u, hi = 0u;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const uint32_t t = (((w[i] & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w[i]) & 0x80808080u;      // bit 8b+7 set: byte b non-zero
+        const uint32_t four = (t * 0x00204081u) >> 28;                                        // those four bits, packed
+        if (i < 8) lo |= four << (4 * i);
+        else hi |= four << (4 * (i - 8));
+    }
+    return (static_cast<unsigned long long>(hi) << 32) | lo;
+}
+
+// chunk_count[c] = number of segment starts among the flags of chunk c; masks[c * CMP_THREADS + t] = the 64
+// flags of thread t as bits.
 __global__ void __launch_bounds__(CMP_THREADS)
 flag_count_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks, int32_t* __restrict__ chunk_count,
-                  bool first_is_start = true) {
+                  unsigned long long* __restrict__ masks, bool first_is_start = true) {
     __shared__ int warp_sums[32];
     for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
         uint32_t w[16];
         load_thread_flags(f, n, c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD, w, first_is_start);
-        int cnt = 0;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) cnt += nonzero_bytes(w[i]);
+        const unsigned long long m = flag_words_to_mask(w);
+        masks[c * CMP_THREADS + threadIdx.x] = m;
         int total;
-        block_exclusive_scan(cnt, &total, warp_sums);
+        block_exclusive_scan(__popcll(m), &total, warp_sums);
         if (threadIdx.x == 0) chunk_count[c] = total;
     }
 }
@@ -135,7 +146,7 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
 // the span partition comes for free here: span_q[s] = #starts before s * 4096, K when the span
 // starts at n, K + 1 ("none") beyond.
 __global__ void __launch_bounds__(CMP_THREADS)
-flag_scatter_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks, const int32_t* __restrict__ chunk_base,
+flag_scatter_kernel(const unsigned long long* __restrict__ masks, long long n, long long nchunks, const int32_t* __restrict__ chunk_base,
                     int32_t* __restrict__ off, int32_t* __restrict__ span_q, const long long* __restrict__ nseg_dev) {
     __shared__ int warp_sums[32];
     constexpr int kThreadsPerSpan = 4096 / CMP_PER_THREAD;
@@ -146,26 +157,15 @@ flag_scatter_kernel(const uint8_t* __restrict__ f, long long n, long long nchunk
     }
     for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
         const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
-        uint32_t w[16];
-        load_thread_flags(f, n, base, w);
-        int cnt = 0;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) cnt += nonzero_bytes(w[i]);
+        unsigned long long m = masks[c * CMP_THREADS + threadIdx.x];
         int total;
-        int slot = chunk_base[c] + block_exclusive_scan(cnt, &total, warp_sums);
+        int slot = chunk_base[c] + block_exclusive_scan(__popcll(m), &total, warp_sums);
         if (threadIdx.x % kThreadsPerSpan == 0)
             span_q[c * (CMP_CHUNK / 4096) + threadIdx.x / kThreadsPerSpan] =
                 static_cast<int32_t>(base < n ? slot : (base == n ? K : K + 1));
-        if (cnt) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                uint32_t m = (((w[i] & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w[i]) & 0x80808080u;     // bit 8b+7 set: byte b non-zero
-                while (m) {
-                    const int b = (__ffs(m) - 1) >> 3;
-                    off[slot++] = static_cast<int32_t>(base + 4 * i + b);
-                    m &= m - 1;
-                }
-            }
+        while (m) {
+            off[slot++] = static_cast<int32_t>(base + (__ffsll(static_cast<long long>(m)) - 1));
+            m &= m - 1;
         }
     }
 }
@@ -174,28 +174,17 @@ flag_scatter_kernel(const uint8_t* __restrict__ f, long long n, long long nchunk
 // of chunk c.  T is the element as stored (2 bytes for fp16 / bf16, 1 byte for int8); nothing is converted.
 template <typename T>
 __global__ void __launch_bounds__(CMP_THREADS)
-compress_values_kernel(const T* __restrict__ x, const uint8_t* __restrict__ f, long long n, long long nchunks,
+compress_values_kernel(const T* __restrict__ x, const unsigned long long* __restrict__ masks, long long nchunks,
                        const int32_t* __restrict__ chunk_base, T* __restrict__ out) {
     __shared__ int warp_sums[32];
     for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
         const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
-        uint32_t w[16];
-        load_thread_flags(f, n, base, w, false);
-        int cnt = 0;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) cnt += nonzero_bytes(w[i]);
+        unsigned long long m = masks[c * CMP_THREADS + threadIdx.x];
         int total;
-        long long slot = chunk_base[c] + block_exclusive_scan(cnt, &total, warp_sums);
-        if (cnt) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                uint32_t m = (((w[i] & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w[i]) & 0x80808080u;
-                while (m) {
-                    const int b = (__ffs(m) - 1) >> 3;
-                    out[slot++] = x[base + 4 * i + b];
-                    m &= m - 1;
-                }
-            }
+        long long slot = chunk_base[c] + block_exclusive_scan(__popcll(m), &total, warp_sums);
+        while (m) {
+            out[slot++] = x[base + (__ffsll(static_cast<long long>(m)) - 1)];
+            m &= m - 1;
         }
     }
 }

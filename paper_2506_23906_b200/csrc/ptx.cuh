@@ -36,16 +36,6 @@ __device__ __forceinline__ uint32_t lane_id() {
     asm volatile("mov.u32 %0, %%laneid;" : "=r"(l));
     return l;
 }
-// Elects one lane of a fully converged warp.
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred = 0;
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "elect.sync _|P, 0xffffffff;\n\t"
-        "selp.u32 %0, 1, 0, P;\n\t}"
-        : "=r"(pred));
-    return pred != 0;
-}
 // Makes generic-proxy writes to shared memory visible to the async proxy (TMA, tcgen05.mma).
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -107,14 +97,6 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* m, uin
         "r"(c3)
         : "memory");
 }
-// Tiled 2-D load global -> shared (c0 = innermost coordinate, must be a multiple of 16 bytes).
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* m, uint64_t* bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
-        : "memory");
-}
 // Untiled bulk copy global -> shared (both addresses 16-byte aligned, size a multiple of 16).
 __device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile(
@@ -167,20 +149,6 @@ __device__ __forceinline__ void tc_fence_after_sync() {
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
-}
-
-// Shared-memory matrix descriptor for a K-major operand stored with the 128-byte
-// swizzle: rows of 128 bytes, groups of 8 rows (1024 bytes) contiguous, 16-byte
-// chunk index XOR (row & 7).  `addr` = shared address of the first row plus the
-// byte offset of the K slice inside the 128-byte row.
-__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t addr) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((addr & 0x3FFFFu) >> 4);        // start address, bits [0,14)
-    d |= static_cast<uint64_t>(1) << 16;                       // leading byte offset (unused for swizzled K-major)
-    d |= static_cast<uint64_t>(1024 >> 4) << 32;               // stride byte offset: 8 rows * 128 B
-    d |= static_cast<uint64_t>(1) << 46;                       // descriptor version (sm_100)
-    d |= static_cast<uint64_t>(2) << 61;                       // layout: 128-byte swizzle
-    return d;
 }
 
 // Instruction descriptors (dense, no negate, both operands K-major).
@@ -257,10 +225,6 @@ __device__ __forceinline__ uint64_t ld_relaxed_gpu_u64(const uint64_t* p) {
     uint64_t v;
     asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
-}
-// Streaming 32-bit store (written once, never re-read by this kernel).
-__device__ __forceinline__ void st_cs_u32(uint32_t* p, uint32_t v) {
-    asm volatile("st.global.cs.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 }  // namespace mmv
