@@ -271,32 +271,43 @@ __global__ void spmv_gather_kernel(const int32_t* __restrict__ col, const __half
     const long long k = (nvec << 2) + static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (k < nnz) prod[k] = split_product(__half2float(val[k]) * gather_x(x, col[k], cols, bad));
     if (bad) report_error(hdr, 1u);
+    // This kernel is launched so that it may start while the kernel in front of it (the span partition of the row
+    // pointers, which it does not depend on) still runs; it ends only after that kernel has ended, so that whoever
+    // follows in the stream finds both finished.
+    griddep_wait();
+}
+
+// The span partition of the offset-encoded segmented sum (and the validation of the offsets, and the zeros of the
+// empty segments).  The header must have been cleared on the stream already.
+void launch_partition(const int32_t* off, long long nseg, long long n_eff, void* out, uint8_t* ws, const WorkspacePlan& plan,
+                      DeviceInfo* dev, cudaStream_t st) {
+    const long long spans = num_tiles_of(n_eff) * SPANS_PER_TILE;
+    int32_t* span_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
+    const int threads = 256;
+    const int vec = nseg >= (1ll << 20) ? 4 : 1;                           // offsets per thread and round
+    long long blocks = (nseg + 1 + vec * threads - 1) / (vec * threads);
+    if (blocks > 16ll * dev->sm_count) blocks = 16ll * dev->sm_count;
+    WorkspaceHeader* hdr = reinterpret_cast<WorkspaceHeader*>(ws);
+    if (vec == 4)
+        partition_offsets_kernel<4><<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, spans, span_q, n_eff, hdr,
+                                                                                      static_cast<uint32_t*>(out));
+    else
+        partition_offsets_kernel<1><<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, spans, span_q, n_eff, hdr,
+                                                                                      static_cast<uint32_t*>(out));
+    ++g_launches;
 }
 
 // Shared launcher of the tiled segmented-sum kernel.  `values` holds n_eff elements of the
 // path's type; boundaries are off[q] << shift.  The header and status words must have been
-// cleared on the stream already.
+// cleared on the stream already.  have_partition: span_q is filled already (by the compaction of
+// the flag-encoded form, or by launch_partition earlier in the stream).
 template <typename P>
 mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* off, long long nseg, int shift,
                           void* out, uint8_t* ws, const WorkspacePlan& plan, DeviceInfo* dev, cudaStream_t st,
                           const long long* nseg_dev = nullptr, bool have_partition = false) {
     const int tiles = static_cast<int>(num_tiles_of(n_eff));
     int32_t* span_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
-    if (!have_partition) {     // (the flag-encoded form has filled span_q while compacting its flags)
-        const long long spans = static_cast<long long>(tiles) * SPANS_PER_TILE;
-        const int threads = 256;
-        const int vec = nseg >= (1ll << 20) ? 4 : 1;                           // offsets per thread and round
-        long long blocks = (nseg + 1 + vec * threads - 1) / (vec * threads);
-        if (blocks > 16ll * dev->sm_count) blocks = 16ll * dev->sm_count;
-        WorkspaceHeader* hdr = reinterpret_cast<WorkspaceHeader*>(ws);
-        if (vec == 4)
-            partition_offsets_kernel<4><<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, spans, span_q, n_eff, hdr,
-                                                                                          static_cast<uint32_t*>(out));
-        else
-            partition_offsets_kernel<1><<<static_cast<unsigned>(blocks), threads, 0, st>>>(off, nseg, spans, span_q, n_eff, hdr,
-                                                                                          static_cast<uint32_t*>(out));
-        ++g_launches;
-    }
+    if (!have_partition) launch_partition(off, nseg, n_eff, out, ws, plan, dev, st);
     CUtensorMap tmap;
     if (!encode_span_map(&tmap, values, n_eff, P::kElemBytes, PIECES_PER_SPAN)) return MMV_ERR_CUDA;
     SumParams prm;
@@ -932,17 +943,32 @@ mmv_status mmv_spmv_csr(const int32_t* rowptr, const int32_t* col, const void* v
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     if (cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
     uint32_t* prod = reinterpret_cast<uint32_t*>(ws + plan.prod_off);
+    // The span partition of the row pointers first: the gather does not depend on it and is launched so that it
+    // may start at once (the partition is bound by its few loads in flight, 28 us for 2^20 rows, and leaves the
+    // GPU nearly empty); the tiled kernel behind the gather needs both.
+    launch_partition(rowptr, rows, nnz, y, ws, plan, dev, st);
     {
         const int threads = 256;
         long long blocks = ((nnz >> 2) + threads - 1) / threads;
         const long long cap = static_cast<long long>(dev->sm_count) * 16;
         if (blocks > cap) blocks = cap;
         if (blocks < 1) blocks = 1;
-        spmv_gather_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(col, static_cast<const __half*>(val_f16), x,
-                                                                              prod, nnz, cols, reinterpret_cast<WorkspaceHeader*>(ws));
+        cudaLaunchConfig_t cfg{};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.gridDim = dim3(static_cast<unsigned>(blocks));
+        cfg.blockDim = dim3(threads);
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t err = cudaLaunchKernelEx(&cfg, spmv_gather_kernel, col, static_cast<const __half*>(val_f16), x, prod,
+                                                   static_cast<long long>(nnz), static_cast<long long>(cols),
+                                                   reinterpret_cast<WorkspaceHeader*>(ws));
         ++g_launches;
+        if (err != cudaSuccess) return MMV_ERR_CUDA;
     }
-    return launch_seg_sum<BF16Path>(prod, nnz, rowptr, rows, 0, y, ws, plan, dev, st);
+    return launch_seg_sum<BF16Path>(prod, nnz, rowptr, rows, 0, y, ws, plan, dev, st, nullptr, true);
 }
 
 mmv_status mmv_last_async_status(const void* workspace, void* cuda_stream) {
