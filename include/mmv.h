@@ -355,6 +355,15 @@ void mmv_debug_configure(int64_t wait_budget_ns, int64_t skip_publish_span);
  */
 void mmv_debug_force_sum_groups(int groups);
 
+/*
+ * Test hook.  The floating-point scan with a flag vector exists in two shapes:
+ * 0 = wide tiles (every flag density), 2 = narrow tiles (fast where segment
+ * starts are rare, correct everywhere).  shape = 0 or 2 makes every later
+ * floating-point scan with a flag vector use that shape; any other value
+ * gives the choice back to the library.
+ */
+void mmv_debug_force_scan_shape(int shape);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,6 +28,7 @@ EXPORTS = (
     "mmv_seg_scan_static", "mmv_seg_scan_static_last_status", "mmv_debug_force_sum_groups",
     "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes", "mmv_seg_scan_exclusive", "mmv_compress",
     "mmv_seg_scan_minmax", "mmv_seg_scan_i8_i64", "mmv_seg_scan_shard", "mmv_seg_scan_shard_finish",
+    "mmv_debug_force_scan_shape",
 )
 SHARD_SUMMARY_BYTES = 16
 STATIC_SCAN_MAX_N = 1 << 28
@@ -82,6 +83,8 @@ def _load() -> ctypes.CDLL:
     lib.mmv_seg_scan_shard.argtypes = [vp, vp, i64, ci, ci, vp, vp, vp, sz, vp]
     lib.mmv_seg_scan_shard_finish.restype = ci
     lib.mmv_seg_scan_shard_finish.argtypes = [vp, ci, ci, vp, i64, ci, vp]
+    lib.mmv_debug_force_scan_shape.restype = None
+    lib.mmv_debug_force_scan_shape.argtypes = [ci]
     lib.mmv_debug_force_sum_groups.restype = None
     lib.mmv_debug_force_sum_groups.argtypes = [ci]
     return lib
@@ -100,6 +103,10 @@ def kernel_launch_count() -> int:
 
 def debug_configure(wait_budget_ns: int = 0, skip_publish_span: int = -1) -> None:
     _lib.mmv_debug_configure(int(wait_budget_ns), int(skip_publish_span))
+
+
+def debug_force_scan_shape(shape: int = -1) -> None:
+    _lib.mmv_debug_force_scan_shape(int(shape))
 
 
 def debug_force_sum_groups(groups: int = 0) -> None:

@@ -24,8 +24,10 @@ std::atomic<long long> g_launches{0};
 std::atomic<unsigned long long> g_budget_ns{WAIT_BUDGET_NS};
 std::atomic<long long> g_debug_skip_span{-1};
 std::atomic<int> g_force_groups{0};
+std::atomic<int> g_force_scan_shape{-1};      // test hook: -1 = the library chooses
 
 constexpr int kMaxDevices = 64;
+constexpr long long kScanProbeMinN = 1ll << 28;       // shortest vector for which the scan samples its flag density
 
 struct DeviceInfo {
     std::mutex lock;
@@ -115,10 +117,14 @@ DeviceInfo* device_info() {
     ok &= set_smem(seg_scan_kernel<I8Path, true>, ScanCfg<I8Path>::kSmemBytes);
     ok &= set_smem(seg_scan_kernel<BF16ValPath>, ScanCfg<BF16ValPath>::kSmemBytes);
     ok &= set_smem(seg_scan_kernel<BF16ValPath, true>, ScanCfg<BF16ValPath>::kSmemBytes);
-    ok &= set_smem(seg_scan_kernel<F16Path, false, true>, ScanCfg<F16Path, true>::kSmemBytes);
-    ok &= set_smem(seg_scan_kernel<F16Path, true, true>, ScanCfg<F16Path, true>::kSmemBytes);
-    ok &= set_smem(seg_scan_kernel<BF16ValPath, false, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
-    ok &= set_smem(seg_scan_kernel<BF16ValPath, true, true>, ScanCfg<BF16ValPath, true>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<F16Path, false, SCAN_PLAIN>, ScanCfg<F16Path, SCAN_PLAIN>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<F16Path, true, SCAN_PLAIN>, ScanCfg<F16Path, SCAN_PLAIN>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<BF16ValPath, false, SCAN_PLAIN>, ScanCfg<BF16ValPath, SCAN_PLAIN>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<BF16ValPath, true, SCAN_PLAIN>, ScanCfg<BF16ValPath, SCAN_PLAIN>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<F16Path, false, SCAN_NARROW>, ScanCfg<F16Path, SCAN_NARROW>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<F16Path, true, SCAN_NARROW>, ScanCfg<F16Path, SCAN_NARROW>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<BF16ValPath, false, SCAN_NARROW>, ScanCfg<BF16ValPath, SCAN_NARROW>::kSmemBytes);
+    ok &= set_smem(seg_scan_kernel<BF16ValPath, true, SCAN_NARROW>, ScanCfg<BF16ValPath, SCAN_NARROW>::kSmemBytes);
     ok &= set_smem(seg_scan_minmax_kernel<0, false>, MM_SMEM_BYTES);
     ok &= set_smem(seg_scan_minmax_kernel<0, true>, MM_SMEM_BYTES);
     ok &= set_smem(seg_scan_minmax_kernel<1, false>, MM_SMEM_BYTES);
@@ -515,31 +521,68 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
     prm.debug_skip_span = g_debug_skip_span.load();
     prm.carry_in = nullptr;
     prm.first_start = nullptr;
+    prm.probe_count = nullptr;
+    prm.probe_narrow_below = 0u;
     if (shard) {
         // (header words behind the two counters, cleared with the header: the first-start word and a carry of zero)
         prm.first_start = reinterpret_cast<unsigned long long*>(&hdr->reserved[0]);
         if (shard == 2) prm.carry_in = &hdr->reserved[2];
     }
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
-    // (no flag vector: the floating-point paths run the narrow-tile variant)
+    // (no flag vector: the floating-point paths run the narrow-tile shape without flag bytes; with a flag vector
+    //  the narrow-tile shape is for vectors with few starts -- see the probe below)
     const bool plain = flags == nullptr;
+    const int forced = g_force_scan_shape.load();
+    bool narrow = !plain && forced == SCAN_NARROW;
+    // A long floating-point vector with a flag vector: which shape is faster depends on how many tiles hold a
+    // start (n = 2^30: no start 1.37 ms wide / 1.24 narrow, p = 1e-5 1.22 / 1.16, p = 1e-4 1.15 / 1.18,
+    // p = 1e-3 1.13 / 1.40), which only the device can see.  A sampling kernel counts the starts in 256 KB of
+    // the flags, both shapes are launched, and the one the count does not ask for returns at once (about
+    // 6-8 us for the probe and the idle launch together, 0.6 % at n = 2^30 and 2.6 % at n = 2^28, hence only for
+    // vectors of 2^28 elements and more).  Fewer than one start per two tiles: narrow.  A vector whose starts all hide between the samples gets the slower shape, never a
+    // wrong result.
+    const bool probe = !plain && forced < 0 && dt != MMV_I8_TO_I32 && n >= kScanProbeMinN;
+    if (probe) {
+        unsigned int* cnt = &hdr->reserved[4];                        // cleared with the header
+        flag_density_probe_kernel<<<SCAN_PROBE_BLOCKS, SCAN_PROBE_THREADS, 0, st>>>(flags, n, cnt);
+        ++g_launches;
+        if (cudaGetLastError() != cudaSuccess) return MMV_ERR_CUDA;
+        prm.probe_count = cnt;
+        prm.probe_narrow_below = SCAN_PROBE_BYTES / SCAN_TILE / 2;    // half a start per tile on average
+    }
     cudaError_t err;
 #define MMV_LAUNCH_SCAN(PATH, EXCL, PL)                                                                               \
     err = launch_resident(seg_scan_kernel<PATH, EXCL, PL>, grid, ScanCfg<PATH, PL>::kThreads, ScanCfg<PATH, PL>::kSmemBytes, st, \
                           false, tmap, tmap_out, prm)
     if (dt == MMV_I8_TO_I32) {
-        if (exclusive) MMV_LAUNCH_SCAN(I8Path, true, false);
-        else MMV_LAUNCH_SCAN(I8Path, false, false);
+        if (exclusive) MMV_LAUNCH_SCAN(I8Path, true, SCAN_WIDE);
+        else MMV_LAUNCH_SCAN(I8Path, false, SCAN_WIDE);
     } else if (dt == MMV_BF16_TO_F32) {
-        if (plain && exclusive) MMV_LAUNCH_SCAN(BF16ValPath, true, true);
-        else if (plain) MMV_LAUNCH_SCAN(BF16ValPath, false, true);
-        else if (exclusive) MMV_LAUNCH_SCAN(BF16ValPath, true, false);
-        else MMV_LAUNCH_SCAN(BF16ValPath, false, false);
+        if (plain && exclusive) MMV_LAUNCH_SCAN(BF16ValPath, true, SCAN_PLAIN);
+        else if (plain) MMV_LAUNCH_SCAN(BF16ValPath, false, SCAN_PLAIN);
+        else {
+            if ((narrow || probe) && exclusive) MMV_LAUNCH_SCAN(BF16ValPath, true, SCAN_NARROW);
+            else if (narrow || probe) MMV_LAUNCH_SCAN(BF16ValPath, false, SCAN_NARROW);
+            if (probe) {
+                ++g_launches;
+                if (err != cudaSuccess) return MMV_ERR_CUDA;
+            }
+            if ((!narrow || probe) && exclusive) MMV_LAUNCH_SCAN(BF16ValPath, true, SCAN_WIDE);
+            else if (!narrow || probe) MMV_LAUNCH_SCAN(BF16ValPath, false, SCAN_WIDE);
+        }
     } else {
-        if (plain && exclusive) MMV_LAUNCH_SCAN(F16Path, true, true);
-        else if (plain) MMV_LAUNCH_SCAN(F16Path, false, true);
-        else if (exclusive) MMV_LAUNCH_SCAN(F16Path, true, false);
-        else MMV_LAUNCH_SCAN(F16Path, false, false);
+        if (plain && exclusive) MMV_LAUNCH_SCAN(F16Path, true, SCAN_PLAIN);
+        else if (plain) MMV_LAUNCH_SCAN(F16Path, false, SCAN_PLAIN);
+        else {
+            if ((narrow || probe) && exclusive) MMV_LAUNCH_SCAN(F16Path, true, SCAN_NARROW);
+            else if (narrow || probe) MMV_LAUNCH_SCAN(F16Path, false, SCAN_NARROW);
+            if (probe) {
+                ++g_launches;
+                if (err != cudaSuccess) return MMV_ERR_CUDA;
+            }
+            if ((!narrow || probe) && exclusive) MMV_LAUNCH_SCAN(F16Path, true, SCAN_WIDE);
+            else if (!narrow || probe) MMV_LAUNCH_SCAN(F16Path, false, SCAN_WIDE);
+        }
     }
 #undef MMV_LAUNCH_SCAN
     ++g_launches;
@@ -713,6 +756,8 @@ mmv_status mmv_seg_scan_host(const void* x_host, const void* flags_host, int64_t
         prm.debug_skip_span = -1;
         prm.carry_in = carry;
         prm.first_start = nullptr;
+        prm.probe_count = nullptr;
+        prm.probe_narrow_below = 0u;
         const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
         if (f16)
             ok &= launch_resident(seg_scan_kernel<F16Path>, grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, dev->s_k,
@@ -1015,6 +1060,8 @@ mmv_status mmv_seg_scan_static(const void* x, const void* flags_u8, int64_t n, m
     prm.debug_skip_span = g_debug_skip_span.load();
     prm.carry_in = nullptr;
     prm.first_start = nullptr;
+    prm.probe_count = nullptr;
+    prm.probe_narrow_below = 0u;
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
     cudaError_t err;
     if (f16)
@@ -1057,6 +1104,8 @@ void mmv_debug_phase_cycles(unsigned long long* host16) {
     cudaMemcpyToSymbol(g_phase_cycles, z, sizeof(z));
 }
 #endif
+
+void mmv_debug_force_scan_shape(int shape) { g_force_scan_shape.store(shape == SCAN_WIDE || shape == SCAN_NARROW ? shape : -1); }
 
 void mmv_debug_force_sum_groups(int groups) { g_force_groups.store(groups == 2 || groups == 3 ? groups : 0); }
 

@@ -70,12 +70,28 @@ struct F16Path {
     __device__ static __forceinline__ uint32_t to_bits(Acc v) { return __float_as_uint(v); }
     __device__ static __forceinline__ Acc add(Acc a, Acc b) { return a + b; }
     __device__ static __forceinline__ Acc sub(Acc a, Acc b) { return a - b; }
+    // two packed input values -> fp32 (low half first), and one value from memory
+    __device__ static __forceinline__ void unpack2(uint32_t w, float& lo, float& hi) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
+        lo = f.x;
+        hi = f.y;
+    }
+    __device__ static __forceinline__ float load_elem(const void* x, long long idx) {
+        return __half2float(static_cast<const __half*>(x)[idx]);
+    }
 };
 // bfloat16 input values, fp32 results: the layout and arithmetic of the fp16 path, with the tensor-core
 // operands declared bf16 (the products with the 0/1 matrix stay exact, the accumulator is fp32).
 struct BF16ValPath : F16Path {
     static constexpr uint32_t kOneBits = 0x3F80u;                       // 1.0 in bf16
     static constexpr uint32_t kFmtBits = (1u << 7) | (1u << 10);        // A and B are bf16
+    __device__ static __forceinline__ void unpack2(uint32_t w, float& lo, float& hi) {
+        lo = __uint_as_float(w << 16);
+        hi = __uint_as_float(w & 0xffff0000u);
+    }
+    __device__ static __forceinline__ float load_elem(const void* x, long long idx) {
+        return __uint_as_float(static_cast<uint32_t>(static_cast<const unsigned short*>(x)[idx]) << 16);
+    }
 };
 struct I8Path {
     using Acc = uint32_t;                                  // wrap-around arithmetic on unsigned

@@ -51,6 +51,9 @@ struct ScanParams {
     const void* carry_in;        // device pointer to one fp32 / int32, or null: the running sum that
                                  // reaches element 0 from an earlier chunk of the same vector (element 0
                                  // then continues that segment unless its flag is set)
+    const unsigned int* probe_count;   // device word, or null: number of starts a sampling kernel found in
+    unsigned int probe_narrow_below;   // SCAN_PROBE_BYTES flag bytes; the narrow shape runs iff it is below this,
+                                       // the wide shape iff it is not (the other launch returns at once)
     unsigned long long* first_start;   // device word, or null: receives n - (index of the vector's first start)
                                  // by atomicMax (it begins at 0 = no start); used when the vector is one
                                  // shard of a longer one, whose carry belongs in front of that index
@@ -85,20 +88,23 @@ constexpr int SCAN_STATUS_STRIDE = MMV_SCAN_STATUS_STRIDE;
 #define MMV_SCAN_I8_GROUPS 3
 #endif
 
-// PLAIN = the call has no flag vector (one segment): no row ever needs its own values back, so the
-// floating-point paths drop the identity half of the product: narrow tiles (128 TMEM columns), so
-// four warpgroups with one tile each, four 32 KB stages without flag bytes, one staging buffer per warp.
-template <typename P, bool PLAIN = false>
+// The kernel comes in three shapes.
+//   SCAN_WIDE    the product also returns the rows themselves ([U | I], 256 TMEM columns per fp16 tile), two
+//                warpgroups (int8: U only, 128 columns, three warpgroups).  Every flag density.
+//   SCAN_PLAIN   the call has no flag vector (one segment): no row ever needs its own values back, so the
+//                floating-point paths drop the identity half: narrow tiles (128 TMEM columns), four warpgroups
+//                with one tile each, four 32 KB stages without flag bytes, one staging buffer per warp.
+//   SCAN_NARROW  floating point with a flag vector in which starts are RARE: the narrow tiles and four
+//                warpgroups of SCAN_PLAIN, three 48 KB stages; the rare piece that holds a start fetches its
+//                rows from global memory instead of from identity columns.  Correct for every flag vector,
+//                fast only where few pieces hold a start (a tile can then wait for its carry in a quarter
+//                of the tensor memory while three others are worked on).
+constexpr int SCAN_WIDE = 0, SCAN_PLAIN = 1, SCAN_NARROW = 2;
+template <typename P, int MODE = SCAN_WIDE>
 struct ScanCfg {
-    // fp16: the product also returns the rows themselves (exact fp32 copies, columns 32..63), so a
-    // tile needs 256 TMEM columns and each warpgroup has one buffer; int8: 128 columns, two buffers.
-    // The epilogue is latency-bound, so the narrower int8 tiles are spread over a third warpgroup.
-    static constexpr bool kWide = P::kIsFloat && !PLAIN;                 // [U | I] product
+    static constexpr bool kWide = P::kIsFloat && MODE == SCAN_WIDE;      // [U | I] product
     static constexpr int kN = kWide ? 2 * ROW : ROW;                     // accumulator columns per product
-#ifndef MMV_SCAN_PLAIN_GROUPS
-#define MMV_SCAN_PLAIN_GROUPS 4
-#endif
-    static constexpr int kGroups = kWide ? 2 : ((PLAIN && P::kIsFloat) ? MMV_SCAN_PLAIN_GROUPS : MMV_SCAN_I8_GROUPS);
+    static constexpr int kGroups = kWide ? 2 : (P::kIsFloat ? 4 : MMV_SCAN_I8_GROUPS);
     static constexpr int kTmemCols = 512;
     // TMEM tile buffers: as many as fit.  Iteration `it` of the CTA uses buffer it % kBufs, whichever warpgroup
     // takes it, so with more buffers than warpgroups (int8 with three groups: four) the products of a group's
@@ -109,13 +115,12 @@ struct ScanCfg {
     static constexpr int kProducerWarp = kEpiWarps;
     static constexpr int kMmaWarp = kEpiWarps + 1;
     static constexpr int kThreads = (kEpiWarps + 2) * 32;
-    static constexpr int kStages = kWide ? 3 : ((kGroups == 2 || kGroups == 4) ? 4 : 3);
-    static_assert(kStages >= kGroups, "the producer's closing round needs a stage per warpgroup");
+    static constexpr int kStages = (P::kIsFloat && MODE == SCAN_PLAIN) ? 4 : 3;
     static_assert(kBufs >= kGroups && kBufs * SCAN_UP * kN <= kTmemCols, "a tile buffer per warpgroup, all inside the tensor memory");
     static constexpr int kBBytes = kN * P::kRowBytes;                    // constant operand [U_32 | I_32] / U_32
     static constexpr int kBSlot = 4096;
     static constexpr int kXBytes = SCAN_UP * P::kSlabBytes;
-    static constexpr int kFlagBytes = PLAIN ? 0 : SCAN_TILE;
+    static constexpr int kFlagBytes = MODE == SCAN_PLAIN ? 0 : SCAN_TILE;
     static constexpr int kStageBytes = kXBytes + kFlagBytes;
     static constexpr int kStageOffset = kBSlot;
     static constexpr int kOutOffset = kStageOffset + kStages * kStageBytes;
@@ -160,18 +165,79 @@ __device__ __forceinline__ bool wait_stage(const volatile int* stage_iter, int i
     return wait_bar(bar, parity, abort_flag, budget_ns);
 }
 
+// Flag density probe: SCAN_PROBE_BLOCKS blocks of 1 KB, spread evenly over the flag vector, are counted for
+// non-zero bytes (one 16-byte load per thread); the total goes to *count, which the caller has cleared.
+constexpr int SCAN_PROBE_BLOCKS = 256;
+constexpr int SCAN_PROBE_THREADS = 64;
+constexpr int SCAN_PROBE_BYTES = SCAN_PROBE_BLOCKS * SCAN_PROBE_THREADS * 16;     // 256 KB
+__global__ void __launch_bounds__(SCAN_PROBE_THREADS)
+flag_density_probe_kernel(const uint8_t* __restrict__ flags, long long n, unsigned int* __restrict__ count) {
+    const long long base = (static_cast<long long>(blockIdx.x) * (n / SCAN_PROBE_BLOCKS)) & ~15ll;
+    const long long p = base + threadIdx.x * 16;
+    unsigned int c = 0u;
+    if (p + 16 <= n) {
+        const uint4 q = *reinterpret_cast<const uint4*>(flags + p);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) c += __popc((((w[k] & 0x7F7F7F7Fu) + 0x7F7F7F7Fu) | w[k]) & 0x80808080u);
+    }
+    c = __reduce_add_sync(0xffffffffu, c);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(count, c);
+}
+
+// SCAN_NARROW only.  The 32 values of one row (elements e0 .. e0 + 31 of the vector, zero past n) as fp32 bit
+// patterns, fetched from global memory: that shape has no identity columns to take them from.
+template <typename P>
+__device__ __forceinline__ void load_row_from_memory(const void* x, long long e0, long long n, uint32_t (&r)[32]) {
+    if (e0 + ROW <= n) {
+        const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(x) + e0 * 2);
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const uint4 q = __ldg(p + v);
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                float a, b;
+                P::unpack2(w[k], a, b);
+                r[8 * v + 2 * k] = __float_as_uint(a);
+                r[8 * v + 2 * k + 1] = __float_as_uint(b);
+            }
+        }
+    } else {
+#pragma unroll 1
+        for (int j = 0; j < ROW; ++j) {
+            const float v = (e0 + j < n) ? P::load_elem(x, e0 + j) : 0.f;
+#pragma unroll
+            for (int q = 0; q < ROW; ++q)
+                if (q == j) r[q] = __float_as_uint(v);
+        }
+    }
+}
+// Sum of the elements pl .. 31 of the row that starts at element e0 (the tail behind a row's last start).
+template <typename P>
+__device__ __noinline__ float row_tail_from_memory(const void* x, long long e0, int pl, long long n) {
+    float t = 0.f;
+    for (int j = pl; j < ROW && e0 + j < n; ++j) t += P::load_elem(x, e0 + j);
+    return t;
+}
+
 // EX = true gives the exclusive variant: every element receives the sum of the elements of its
 // segment in FRONT of it (0 at a segment start), i.e. the inclusive result moved one element to
 // the right inside each segment.  The shift happens in registers just before a piece is staged for
 // its store; everything else is the same kernel.
-template <typename P, bool EX = false, bool PLAIN = false>
-__global__ void __launch_bounds__(ScanCfg<P, PLAIN>::kThreads, 1)
+template <typename P, bool EX = false, int MODE = SCAN_WIDE>
+__global__ void __launch_bounds__(ScanCfg<P, MODE>::kThreads, 1)
 seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_out,
                  const ScanParams prm) {
     using Acc = typename P::Acc;
-    using Cfg = ScanCfg<P, PLAIN>;
+    using Cfg = ScanCfg<P, MODE>;
+    constexpr bool PLAIN = MODE == SCAN_PLAIN;
     constexpr int S = Cfg::kStages;
     constexpr int N = Cfg::kN;
+
+    // Two shapes of this kernel may have been launched for one call (wide and narrow tiles); the one the sampled
+    // flag density does not ask for returns before it touches anything.
+    if (prm.probe_count != nullptr && ((*prm.probe_count < prm.probe_narrow_below) != (MODE == SCAN_NARROW))) return;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -255,26 +321,20 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 
     if (warp == Cfg::kProducerWarp) {
         // =========================== producer ===========================
-        int it = 0, sentinels = 0;
+        int it = 0;
         bool ok = true;
         while (ok) {
+            // static round-robin tile assignment: all CTAs are resident (cooperative launch, one CTA per
+            // SM), so iteration `it` of every CTA runs at about the same time and a tile's predecessors
+            // are always in flight or finished.  Every role of the CTA derives its tiles from the same
+            // formula, so the end of the work needs no message.
+            const int tile = static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
+            if (tile >= prm.num_tiles) break;
             const int stage = it % S;
             if (!wait_bar(&bar_empty[stage], ((it / S) & 1) ^ 1, abort_flag, budget)) { ok = false; break; }
-            // static round-robin tile assignment: all CTAs are resident (grid <= SM count, one CTA per
-            // SM), so iteration `it` of every CTA runs at about the same time and a tile's predecessors
-            // are always in flight or finished
-            int tile = static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x);
-            if (tile >= prm.num_tiles) tile = -1;
             if (lane == 0) {
                 tile_slot[stage] = tile;
                 stage_iter[stage] = it;
-            }
-            if (tile < 0) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bar_full[stage]);
-                ++it;
-                if (++sentinels == Cfg::kGroups) break;
-                continue;
             }
             uint8_t* xs = sStage + stage * Cfg::kStageBytes;
             uint8_t* fs = xs + Cfg::kXBytes;
@@ -343,17 +403,12 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
         // =========================== MMA issuer ===========================
         // Runs ahead of the epilogue: the products of a warpgroup's next tile go to its other buffer.
         constexpr uint32_t idesc = P::kIsFloat ? (make_idesc_f16_f32(128, N) | P::kFmtBits) : make_idesc_s8_s32(128, N);
-        int sentinels = 0;
-        for (int it = 0;; ++it) {
+        for (int it = 0; static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x) < prm.num_tiles; ++it) {
             const int stage = it % S;
             if (!wait_bar(&bar_full[stage], (it / S) & 1, abort_flag, budget)) {
                 *abort_flag = 1;
                 if (lane == 0) report_error(prm.hdr, 5u);
                 break;
-            }
-            if (tile_slot[stage] < 0) {
-                if (++sentinels == Cfg::kGroups) break;
-                continue;
             }
             const int buf = it % Cfg::kBufs;
             if (!wait_bar(&bar_acc_empty[buf], ((it / Cfg::kBufs) & 1) ^ 1, abort_flag, budget)) {
@@ -436,10 +491,10 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
 
         for (int k = 0;; ++k) {
             const int it = g + Cfg::kGroups * k;
+            if (static_cast<int>(blockIdx.x) + it * static_cast<int>(gridDim.x) >= prm.num_tiles) break;
             const int stage = it % S;
             if (!wait_stage(&stage_iter[stage], it, &bar_full[stage], (it / S) & 1, abort_flag, budget)) { failed = true; break; }
             const int tile = tile_slot[stage];
-            if (tile < 0) break;
             MMV_T_MARK(0)
 
             const int buf = it % Cfg::kBufs;
@@ -525,6 +580,11 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                     for (int j = 0; j < 32; ++j)
                         if (j >= pl) part[j & 3] = P::add(part[j & 3], P::from_bits(xr[j]));
                     row_tail = P::add(P::add(part[0], part[1]), P::add(part[2], part[3]));
+                } else if constexpr (P::kIsFloat) {
+                    // narrow tiles: the same sum, the row's values fetched from memory (only the lane of that row)
+                    row_tail = Acc(0);
+                    if (static_cast<int>(lane) == lstar)
+                        row_tail = row_tail_from_memory<P>(prm.x, s * SCAN_UNIT + istar * PIECE + lstar * ROW, pl, prm.n);
                 } else {
                     Acc before = Acc(0);
                     if (pl > 0) {
@@ -616,6 +676,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                         // front of its first start).  One chain of 32 additions: splitting the row into two or four
                         // independent chains measured slower (n = 2^30, every element a start: 1.17 / 1.19 / 1.22 ms),
                         // the elements that continue the part before them cost more than the latency saved.
+                        if constexpr (!Cfg::kWide) load_row_from_memory<P>(prm.x, (row0 + i * PIECE_ROWS + lane) * ROW, prm.n, r);
                         Acc since = Acc(0);
 #pragma unroll
                         for (int j = 0; j < 32; ++j) {

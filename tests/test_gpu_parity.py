@@ -1183,3 +1183,36 @@ def test_scan_in_shards_edges(mmv):
     for r in range(world):
         mmv.seg_scan_shard_finish(gathered, r, world, out[r * m:(r + 1) * m], torch.int8)
     assert np.array_equal(out.cpu().numpy(), oracle.seg_scan_i8(xi[:world * m], np.zeros(world * m, np.uint8)))
+
+
+# ---------------------------------------------------------------------------
+# the narrow-tile shape of the floating-point scan (chosen by the library where starts are rare) on every density
+# ---------------------------------------------------------------------------
+def test_scan_narrow_shape_is_correct_for_every_flag_vector(mmv):
+    # forced for all calls below: pieces that hold a start fetch their rows from memory instead of identity columns
+    mmv.debug_force_scan_shape(2)
+    try:
+        for n in (1, 33, 1025, 4097, TILE - 1, TILE + 1, 5 * TILE + 4099, 100_003):
+            test_scan_f16_sizes(mmv, n)
+        test_scan_flag_positions_around_row_and_tile_edges(mmv)
+        test_scan_closed_forms(mmv)
+        test_scan_with_offsets(mmv)
+        test_scan_tiny_segments_next_to_large_values(mmv)
+        test_scan_mixed_magnitudes_inside_a_segment(mmv)
+        for n, p in ((4097, 0.05), (3 * TILE + 4097, 1e-3), (11 * TILE + 777, 0.5), (11 * TILE + 777, 1.0)):
+            test_exclusive_scan(mmv, n, p)
+        for n, p in ((33, 1.0), (7 * TILE + 1234, 1e-3), (7 * TILE + 1234, 0.1)):
+            test_bf16_scan_and_sum(mmv, n, p)
+        test_bf16_values_beyond_the_fp16_range(mmv)
+        test_scan_in_four_shards_matches_the_whole_vector(mmv, 1e-5)
+        test_lookback_wait_gives_up_with_a_status(mmv)
+        # many tiles per warpgroup, few starts: the case the shape is for
+        rng = np.random.default_rng(4)
+        n = 300 * TILE + 77
+        x = rng.uniform(-1, 1, n).astype(np.float16)
+        for p in (0.0, 1e-6, 1e-4):
+            f = (rng.random(n) < p).astype(np.uint8)
+            z, a = oracle.seg_scan_f16(x, f)
+            assert_fp(scan_f16(mmv, x, f), z, a, f"narrow shape, p={p}")
+    finally:
+        mmv.debug_force_scan_shape(-1)
