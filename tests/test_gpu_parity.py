@@ -389,6 +389,28 @@ def test_seg_sum_tiny_segments_next_to_large_values(mmv):
     assert_fp(sum_csr(mmv, x, off), want, a, "tiny next to large, longer")
 
 
+def test_seg_sum_long_segments_at_the_edge_of_the_stated_magnitude_range(mmv):
+    # What the header promises for segments LONGER than two 32-element rows: the bound holds when the magnitudes
+    # inside a 4096-element span are within about 2^10 of each other.  Segments of 40 .. 3000 elements, every
+    # other one scaled by 2^-10 (so that a small segment's partial rows are differences of prefixes that still
+    # carry its big neighbour's values), also through SpMV's bf16-pair path.
+    rng = np.random.default_rng(41)
+    lens = rng.integers(40, 3000, 4000)
+    lens[::5] = rng.integers(33, 70, lens[::5].shape[0])         # many just beyond the reach of the cancellation check
+    off = gen.offsets_from_lengths(lens)
+    n = int(off[-1])
+    scale = np.where(np.arange(lens.shape[0]) % 2 == 0, 1.0, 2.0 ** -10)
+    x = (rng.standard_normal(n) * np.repeat(scale, lens)).astype(np.float16)
+    want, a = oracle.seg_sum_csr_f16(x, off)
+    assert_fp(sum_csr(mmv, x, off), want, a, "long segments, magnitudes 2^10 apart")
+    val = x
+    cols = n
+    col = np.arange(n, dtype=np.int32)
+    xv = np.ones(cols, np.float32)
+    wanty, ay = oracle.spmv_csr(off, col, val, xv)
+    assert_fp(spmv(mmv, off, col, val, xv), wanty, ay, "SpMV rows, magnitudes 2^10 apart")
+
+
 def test_seg_sum_long_runs_of_empty_segments(mmv):
     # hundreds of thousands of empty segments in a row (at the start, in the middle of a span, exactly on a
     # span edge, at the end): the kernel jumps over such runs instead of visiting them one by one
