@@ -310,10 +310,10 @@ void launch_partition(const int32_t* off, long long nseg, long long n_eff, void*
 template <typename P>
 mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* off, long long nseg, int shift,
                           void* out, uint8_t* ws, const WorkspacePlan& plan, DeviceInfo* dev, cudaStream_t st,
-                          const long long* nseg_dev = nullptr, bool have_partition = false) {
+                          const long long* nseg_dev = nullptr, bool have_partition = false, bool fused = false) {
     const int tiles = static_cast<int>(num_tiles_of(n_eff));
     int32_t* span_q = reinterpret_cast<int32_t*>(ws + plan.tileq_off);
-    if (!have_partition) launch_partition(off, nseg, n_eff, out, ws, plan, dev, st);
+    if (!have_partition && !fused) launch_partition(off, nseg, n_eff, out, ws, plan, dev, st);
     CUtensorMap tmap;
     if (!encode_span_map(&tmap, values, n_eff, P::kElemBytes, PIECES_PER_SPAN)) return MMV_ERR_CUDA;
     SumParams prm;
@@ -328,12 +328,14 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     prm.status = reinterpret_cast<uint64_t*>(ws + plan.status_off);
     prm.budget_ns = g_budget_ns.load();
     prm.nseg_dev = nseg_dev;
+    prm.fused_prologue = fused ? 1 : 0;
+    prm.status_words = static_cast<long long>(plan.status_bytes / sizeof(uint64_t));
     const int grid = tiles < dev->sm_count ? tiles : dev->sm_count;
     // Twelve epilogue warps (three warpgroups) measured faster than eight at every segment density;
     // the shape with two warpgroups stays available for tests and measurements.
     // With the partition kernel right in front, the tiled kernel is launched with programmatic
     // serialisation: its set-up (barriers, tensor memory, constant operand) overlaps the partition's end.
-    const bool overlap = !have_partition;
+    const bool overlap = !have_partition && !fused;
     cudaError_t err;
     if (g_force_groups.load() != 2)
         err = launch_resident(seg_sum_kernel<P, 3>, grid, SumShape<3>::kThreads, SumCfg<P, 3>::kSmemBytes, st, overlap, tmap, values, prm);
@@ -843,11 +845,17 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
     DeviceInfo* dev = device_info();
     if (!dev) return MMV_ERR_CUDA;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    if (cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
+    // Up to 2^18 segments, one launch: the tiled kernel clears the header and the status words and partitions the
+    // offsets itself, in front of a grid-wide barrier (it is launched cooperatively anyway).  Configuration 2:
+    // 39.5 -> 35.9 us per call (a memset, the partition kernel and the tiled kernel were three enqueues), n = 2^28
+    // 106 -> 104 us.  With millions of offsets the partition wants more threads than the tiled grid has (11.4 M
+    // offsets: 188 -> 210 us fused), so those calls keep the memset and the kernel of its own.
+    const bool fused = nseg <= (1ll << 18);
+    if (!fused && cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
     const int32_t* off = static_cast<const int32_t*>(seg);
-    if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, nseg, 0, out, ws, plan, dev, st);
-    if (dt == MMV_BF16_TO_F32) return launch_seg_sum<BF16ValPath>(x, n, off, nseg, 0, out, ws, plan, dev, st);
-    return launch_seg_sum<I8Path>(x, n, off, nseg, 0, out, ws, plan, dev, st);
+    if (dt == MMV_F16_TO_F32) return launch_seg_sum<F16Path>(x, n, off, nseg, 0, out, ws, plan, dev, st, nullptr, false, fused);
+    if (dt == MMV_BF16_TO_F32) return launch_seg_sum<BF16ValPath>(x, n, off, nseg, 0, out, ws, plan, dev, st, nullptr, false, fused);
+    return launch_seg_sum<I8Path>(x, n, off, nseg, 0, out, ws, plan, dev, st, nullptr, false, fused);
 }
 
 mmv_status mmv_seg_scan_minmax(const void* x, const void* flags, int64_t n, mmv_dtype dt, int want_min, void* out,

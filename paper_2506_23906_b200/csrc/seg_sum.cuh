@@ -37,6 +37,7 @@
 //     spans (shared memory) or of a decoupled look-back over per-span status words.  Pieces
 //     without a boundary only add their total.
 #pragma once
+#include <cooperative_groups.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include "../../include/mmv.h"
@@ -258,6 +259,10 @@ struct SumParams {
     unsigned long long budget_ns;
     const long long* nseg_dev;   // when not null: the number of segments is read from here (flag-encoded
                                  // segments, whose count is only known on the device); nseg is ignored
+    int fused_prologue;          // 1: the kernel itself clears the header and the status words and partitions the
+                                 // offsets (span_q, validation, zeros of empty segments) before a grid-wide
+                                 // barrier -- one launch per call instead of a memset and two kernels
+    long long status_words;      // number of 8-byte status words to clear in that case
 };
 
 // First index q in [lo, hi) with (off[q] << shift) >= target, hi if none; the offsets are
@@ -301,20 +306,22 @@ __device__ __noinline__ long long first_index_at_least_call(const int32_t* off, 
 // missing or inconsistent, which the main kernel tolerates: it clamps what it reads and never
 // indexes outside its tile) and writes the zero of every EMPTY segment, so that the main kernel
 // may jump over long runs of equal offsets instead of visiting them one by one.
+// (the work of one thread of `nthreads`, `tid` its index; every warp must come as a whole)
+// Returns true if this thread met an offset that is out of order or out of range (the caller reports it).
 template <int VEC>       // offsets per lane and round: 4 when there are many (one 16-byte load each), else 1
-__global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, long long num_spans,
-                                         int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr,
-                                         uint32_t* __restrict__ out) {
+__device__ __forceinline__ bool partition_offsets(const int32_t* __restrict__ off, long long nseg, long long num_spans,
+                                                  int32_t* __restrict__ span_q, long long n,
+                                                  uint32_t* __restrict__ out, long long tid, long long nthreads) {
     const int lane = threadIdx.x & 31;
-    const long long stride = static_cast<long long>(VEC) * gridDim.x * blockDim.x;
-    griddep_launch_dependents();       // the tiled kernel may set itself up meanwhile (it waits before it reads)
+    bool bad = false;
+    const long long stride = static_cast<long long>(VEC) * nthreads;
     const int n32 = static_cast<int>(n < 0x7fffffffll ? n : 0x7fffffffll);
     const int last_span = static_cast<int>(num_spans);
     static_assert(SPAN == 4096, "span index = position >> 12");
     // A warp takes 32 VEC consecutive offsets per round; with many offsets four per lane in one 16-byte
     // load (the kernel is bound by the loads it has in flight).  Every warp makes the same number of rounds: the votes below
     // need all its lanes.  Positions and span indices fit 32 bits because the offsets do.
-    for (long long wbase = VEC * (static_cast<long long>(blockIdx.x) * blockDim.x + (threadIdx.x & ~31)); wbase <= nseg; wbase += stride) {
+    for (long long wbase = VEC * (tid - lane); wbase <= nseg; wbase += stride) {
         const long long i0 = wbase + VEC * lane;   // my first offset index
         int c[VEC];
 #pragma unroll
@@ -347,11 +354,11 @@ __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long l
             hi[e] = -1;
             if (i <= nseg) {
                 if (i >= 1) {
-                    if (prev > cur || prev < 0 || cur > n32) report_error(hdr, 4u);
+                    if (prev > cur || prev < 0 || cur > n32) bad = true;
                     if (prev == cur) out[i - 1] = 0u;              // segment i - 1 is empty
                     lo[e] = prev < 0 ? 0 : (prev >> 12) + 1;
                 } else if (cur < 0 || cur > n32) {
-                    report_error(hdr, 4u);
+                    bad = true;
                 }
                 hi[e] = cur < 0 ? -1 : (cur >> 12);
                 if (hi[e] > last_span) hi[e] = last_span;
@@ -388,6 +395,17 @@ __global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long l
             }
         }
     }
+    return bad;
+}
+
+template <int VEC>
+__global__ void partition_offsets_kernel(const int32_t* __restrict__ off, long long nseg, long long num_spans,
+                                         int32_t* __restrict__ span_q, long long n, WorkspaceHeader* hdr,
+                                         uint32_t* __restrict__ out) {
+    griddep_launch_dependents();       // the kernel behind may set itself up meanwhile (it waits before it reads)
+    if (partition_offsets<VEC>(off, nseg, num_spans, span_q, n, out, static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x,
+                               static_cast<long long>(gridDim.x) * blockDim.x))
+        report_error(hdr, 4u);
 }
 
 template <typename P, int G>
@@ -467,6 +485,25 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
     // Everything above (barriers, tensor memory, the constant operand) touched nothing a predecessor in the
     // stream writes; from here on the kernel reads the span partition, the status words and the offsets.
     griddep_wait();
+    if (prm.fused_prologue) {
+        // The whole grid (resident as one: cooperative launch) first does what a memset and the partition kernel
+        // would do -- clear the header and the status words, partition and check the offsets, write the zeros of
+        // the empty segments -- then meets at one grid-wide barrier.  An error in the offsets is reported behind
+        // the barrier, when the header is certainly cleared.
+        const long long tid = static_cast<long long>(blockIdx.x) * Shape::kThreads + threadIdx.x;
+        const long long nthreads = static_cast<long long>(gridDim.x) * Shape::kThreads;
+        for (long long i = tid; i < prm.status_words; i += nthreads) prm.status[i] = 0ull;
+        if (tid < static_cast<long long>(sizeof(WorkspaceHeader) / sizeof(unsigned int))) reinterpret_cast<unsigned int*>(prm.hdr)[tid] = 0u;
+        const long long spans = static_cast<long long>(prm.num_tiles) * SPANS_PER_TILE;
+        bool bad;
+        if (prm.nseg >= (1ll << 20))
+            bad = partition_offsets<4>(prm.off, prm.nseg, spans, const_cast<int32_t*>(prm.span_q), prm.n, static_cast<uint32_t*>(prm.out), tid, nthreads);
+        else
+            bad = partition_offsets<1>(prm.off, prm.nseg, spans, const_cast<int32_t*>(prm.span_q), prm.n, static_cast<uint32_t*>(prm.out), tid, nthreads);
+        __threadfence();
+        cooperative_groups::this_grid().sync();
+        if (bad) report_error(prm.hdr, 4u);
+    }
 
     if (warp == Shape::kProducerWarp) {
         // =========================== producer ===========================
