@@ -492,7 +492,12 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     WorkspaceHeader* hdr = reinterpret_cast<WorkspaceHeader*>(ws);
-    if (cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
+    // Where nothing in front of the scan kernel uses the workspace header (no offsets to turn into flags, no
+    // density probe, no shard record), the kernel clears its workspace itself in front of a grid-wide barrier
+    // and the call is a single launch; otherwise a memset node does it.
+    const bool will_probe = seg != nullptr && g_force_scan_shape.load() < 0 && dt != MMV_I8_TO_I32 && n >= kScanProbeMinN;
+    const bool self_clear = sf == MMV_SEG_FLAGS_U8 && !will_probe && shard == 0;
+    if (!self_clear && cudaMemsetAsync(ws, 0, plan.status_off + plan.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
 
     const uint8_t* flags = static_cast<const uint8_t*>(seg);
     if (sf == MMV_SEG_OFFSETS_I32) {
@@ -525,6 +530,7 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
     prm.first_start = nullptr;
     prm.probe_count = nullptr;
     prm.probe_narrow_below = 0u;
+    prm.clear_words = self_clear ? static_cast<long long>(plan.status_bytes / sizeof(uint64_t)) : 0;
     if (shard) {
         // (header words behind the two counters, cleared with the header: the first-start word and a carry of zero)
         prm.first_start = reinterpret_cast<unsigned long long*>(&hdr->reserved[0]);
@@ -543,7 +549,7 @@ mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t 
     // 6-8 us for the probe and the idle launch together, 0.6 % at n = 2^30 and 2.6 % at n = 2^28, hence only for
     // vectors of 2^28 elements and more).  Fewer than one start per two tiles: narrow.  A vector whose starts all hide between the samples gets the slower shape, never a
     // wrong result.
-    const bool probe = !plain && forced < 0 && dt != MMV_I8_TO_I32 && n >= kScanProbeMinN;
+    const bool probe = will_probe;
     if (probe) {
         unsigned int* cnt = &hdr->reserved[4];                        // cleared with the header
         flag_density_probe_kernel<<<SCAN_PROBE_BLOCKS, SCAN_PROBE_THREADS, 0, st>>>(flags, n, cnt);
@@ -760,6 +766,7 @@ mmv_status mmv_seg_scan_host(const void* x_host, const void* flags_host, int64_t
         prm.first_start = nullptr;
         prm.probe_count = nullptr;
         prm.probe_narrow_below = 0u;
+        prm.clear_words = 0;
         const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
         if (f16)
             ok &= launch_resident(seg_scan_kernel<F16Path>, grid, ScanCfg<F16Path>::kThreads, ScanCfg<F16Path>::kSmemBytes, dev->s_k,
@@ -1070,6 +1077,7 @@ mmv_status mmv_seg_scan_static(const void* x, const void* flags_u8, int64_t n, m
     prm.first_start = nullptr;
     prm.probe_count = nullptr;
     prm.probe_narrow_below = 0u;
+    prm.clear_words = 0;
     const int grid = prm.num_tiles < dev->sm_count ? prm.num_tiles : dev->sm_count;
     cudaError_t err;
     if (f16)

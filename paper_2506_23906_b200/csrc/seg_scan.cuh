@@ -34,6 +34,7 @@
 //                  latency is covered by the main pass.  The parked pieces then receive the
 //                  carry on the elements before the span's first flag and are stored.
 #pragma once
+#include <cooperative_groups.h>
 #include "common.cuh"
 
 namespace mmv {
@@ -54,6 +55,8 @@ struct ScanParams {
     const unsigned int* probe_count;   // device word, or null: number of starts a sampling kernel found in
     unsigned int probe_narrow_below;   // SCAN_PROBE_BYTES flag bytes; the narrow shape runs iff it is below this,
                                        // the wide shape iff it is not (the other launch returns at once)
+    long long clear_words;             // > 0: the kernel itself clears the header and this many 8-byte status words in
+                                       // front of a grid-wide barrier (no memset node in front of the launch)
     unsigned long long* first_start;   // device word, or null: receives n - (index of the vector's first start)
                                  // by atomicMax (it begins at 0 = no start); used when the vector is one
                                  // shard of a longer one, whose carry belongs in front of that index
@@ -318,6 +321,15 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    if (prm.clear_words > 0) {
+        // the whole grid is resident (cooperative launch): it clears its own workspace and meets at a barrier
+        const long long tid = static_cast<long long>(blockIdx.x) * Cfg::kThreads + threadIdx.x;
+        const long long nthreads = static_cast<long long>(gridDim.x) * Cfg::kThreads;
+        for (long long i = tid; i < prm.clear_words; i += nthreads) prm.status[i] = 0ull;
+        if (tid < static_cast<long long>(sizeof(WorkspaceHeader) / sizeof(unsigned int))) reinterpret_cast<unsigned int*>(prm.hdr)[tid] = 0u;
+        __threadfence();
+        cooperative_groups::this_grid().sync();
+    }
 
     if (warp == Cfg::kProducerWarp) {
         // =========================== producer ===========================
