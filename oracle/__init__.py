@@ -329,6 +329,16 @@ def spmv_csr(rowptr, col, val, x):
     return y, a
 
 
+def mult_i8(x, y) -> np.ndarray:
+    """Element-wise product of two int8 vectors as int32 (Corollary 4.5)."""
+    xb, yb = _as(x, np.int8), _as(y, np.int8)
+    n = xb.shape[0]
+    assert yb.shape[0] == n
+    z = np.empty(n, np.int32)
+    _load().mmv_oracle_mult_i8(_p(xb), _p(yb), ctypes.c_int64(n), _p(z))
+    return z
+
+
 def fp_bound(a):
     """Per-element error allowance of the fp16 -> fp32 paths."""
     return TOL_REL * np.asarray(a, np.float64) + TOL_ABS

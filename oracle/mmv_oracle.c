@@ -384,3 +384,16 @@ void mmv_oracle_spmv_csr(const int32_t *rowptr, const int32_t *col, const uint16
         if (a) a[r] = sa;
     }
 }
+
+/*
+ * Element-wise product of two int8 vectors, int32 result (Section 4.3.1,
+ * Corollary 4.5: z(i) = x(i) y(i)).  The paper obtains each product as the last
+ * element of a segmented scan over the partial terms of the school method
+ * (Lemma 4.4); the quantity itself is the plain product, which is what is
+ * written here.  |x y| <= 2^14, so nothing wraps.
+ */
+void mmv_oracle_mult_i8(const int8_t *x, const int8_t *y, int64_t n, int32_t *z)
+{
+    for (int64_t i = 0; i < n; ++i) z[i] = (int32_t)x[i] * (int32_t)y[i];
+}
+

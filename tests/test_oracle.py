@@ -667,3 +667,32 @@ def test_all_cores_scan_equals_the_sequential_oracle():
     f[[5, 80]] = 1
     z, _, _ = oracle.seg_scan_f16_all_cores(x, f, threads=9)
     assert np.array_equal(z, oracle.seg_scan_f16(x, f)[0])
+
+
+# ---------------------------------------------------------------------------
+# element-wise integer product (Section 4.3.1, Lemma 4.4 / Corollary 4.5)
+# ---------------------------------------------------------------------------
+def test_mult_i8_against_python_integers_and_the_school_method():
+    # every pair of int8 values against Python's integers
+    v = np.arange(-128, 128, dtype=np.int64)
+    xs, ys = np.repeat(v, 256), np.tile(v, 256)
+    z = oracle.mult_i8(xs.astype(np.int8), ys.astype(np.int8))
+    assert z.tolist() == [int(a) * int(b) for a, b in zip(xs.tolist(), ys.tolist())]
+    # closed forms: x * 1 = x, x * 0 = 0, x * (-1) = -x, the two extremes
+    x = v.astype(np.int8)
+    assert np.array_equal(oracle.mult_i8(x, np.ones(256, np.int8)), v)
+    assert not oracle.mult_i8(x, np.zeros(256, np.int8)).any()
+    assert np.array_equal(oracle.mult_i8(x, np.full(256, -1, np.int8)), -v)
+    assert oracle.mult_i8(np.array([-128, 127], np.int8), np.array([-128, 127], np.int8)).tolist() == [16384, 16129]
+    # Lemma 4.4: the product is the sum of the partial terms of the school method, c_k = (bit k of y) ? x 2^k : 0,
+    # with bit 7 of a two's-complement byte weighing -2^7 -- i.e. the last element of a segmented scan over the
+    # terms of each product (Corollary 4.5), here with the oracle's own segmented sum over segments of 8 terms
+    bits = (ys.astype(np.uint8)[:, None] >> np.arange(8)) & 1
+    weights = np.array([1, 2, 4, 8, 16, 32, 64, -128], np.int64)
+    terms = bits * xs[:, None] * weights[None, :]
+    assert np.array_equal(terms.sum(axis=1), z)
+    t16 = terms.astype(np.float16)                      # every term is exactly an fp16 value
+    assert np.array_equal(t16.astype(np.int64), terms)
+    off = (np.arange(xs.shape[0] + 1) * 8).astype(np.int32)
+    sums, _ = oracle.seg_sum_csr_f16(t16.reshape(-1), off)
+    assert np.array_equal(sums.astype(np.int64), z)
