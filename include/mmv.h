@@ -96,7 +96,7 @@ typedef enum { MMV_F16_TO_F32 = 0, MMV_I8_TO_I32 = 1, MMV_BF16_TO_F32 = 2 } mmv_
 typedef enum { MMV_SEG_FLAGS_U8 = 0, MMV_SEG_OFFSETS_I32 = 1 } mmv_segfmt;
 typedef enum {
     MMV_OP_SEG_SCAN = 0, MMV_OP_SEG_SUM = 1, MMV_OP_SPMV_CSR = 2, MMV_OP_COMPRESS = 3, MMV_OP_SEG_SCAN_MINMAX = 4,
-    MMV_OP_SEG_SCAN_WIDE = 5
+    MMV_OP_SEG_SCAN_WIDE = 5, MMV_OP_MULT = 6
 } mmv_op;
 
 /*
@@ -242,6 +242,25 @@ mmv_status mmv_seg_scan_i8_i64(const void *x, const void *flags, int64_t n, int6
  */
 mmv_status mmv_compress(const void *x, const void *flags, int64_t n, mmv_dtype dt, void *out, int64_t *d_count,
                         void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Element-wise product of two int8 vectors through the segmented sum
+ * (Section 4.3.1, Lemma 4.4 / Corollary 4.5): out[i] = x[i] * y[i] as int32.
+ * Each product is the sum of the eight partial terms of the school method,
+ * c_k = (bit k of y[i]) ? x[i] 2^k : 0 with bit 7 weighing -2^7; the terms of all
+ * products are written to the workspace as one vector of 8 n fp16 values (every
+ * term is exactly representable) and its segments of eight are summed by the
+ * tensor-core kernel of mmv_seg_sum; the sums, exact integers in fp32, are
+ * rewritten in place as int32.  The result is exact.  The paper gives this
+ * construction for machines without a multiplier; here it is a demonstration
+ * of the method, far slower than a plain multiply.
+ * x, y: n int8 values; out: n int32, 16-byte aligned; n < 2^28.  Workspace:
+ * mmv_workspace_bytes(MMV_OP_MULT, MMV_I8_TO_I32, MMV_SEG_OFFSETS_I32, n, 0)
+ * (about 28 bytes per element).  Asynchronous on cuda_stream; errors as for
+ * mmv_seg_sum.
+ */
+mmv_status mmv_mult_i8(const int8_t *x, const int8_t *y, int64_t n, int32_t *out,
+                       void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * CSR sparse matrix times dense vector built on the segmented sum

@@ -20,7 +20,7 @@ LIB_PATH = _PKG / "libmmv.so"
 MMV_OK = 0
 F16_TO_F32, I8_TO_I32, BF16_TO_F32 = 0, 1, 2
 SEG_FLAGS_U8, SEG_OFFSETS_I32 = 0, 1
-OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR, OP_COMPRESS, OP_SEG_SCAN_MINMAX, OP_SEG_SCAN_WIDE = 0, 1, 2, 3, 4, 5
+OP_SEG_SCAN, OP_SEG_SUM, OP_SPMV_CSR, OP_COMPRESS, OP_SEG_SCAN_MINMAX, OP_SEG_SCAN_WIDE, OP_MULT = 0, 1, 2, 3, 4, 5, 6
 
 EXPORTS = (
     "mmv_workspace_bytes", "mmv_seg_scan", "mmv_seg_sum", "mmv_spmv_csr",
@@ -28,7 +28,7 @@ EXPORTS = (
     "mmv_seg_scan_static", "mmv_seg_scan_static_last_status", "mmv_debug_force_sum_groups",
     "mmv_seg_scan_host", "mmv_seg_scan_host_scratch_bytes", "mmv_seg_scan_exclusive", "mmv_compress",
     "mmv_seg_scan_minmax", "mmv_seg_scan_i8_i64", "mmv_seg_scan_shard", "mmv_seg_scan_shard_finish",
-    "mmv_debug_force_scan_shape",
+    "mmv_debug_force_scan_shape", "mmv_mult_i8",
 )
 SHARD_SUMMARY_BYTES = 16
 STATIC_SCAN_MAX_N = 1 << 28
@@ -83,6 +83,8 @@ def _load() -> ctypes.CDLL:
     lib.mmv_seg_scan_shard.argtypes = [vp, vp, i64, ci, ci, vp, vp, vp, sz, vp]
     lib.mmv_seg_scan_shard_finish.restype = ci
     lib.mmv_seg_scan_shard_finish.argtypes = [vp, ci, ci, vp, i64, ci, vp]
+    lib.mmv_mult_i8.restype = ci
+    lib.mmv_mult_i8.argtypes = [vp, vp, i64, vp, vp, sz, vp]
     lib.mmv_debug_force_scan_shape.restype = None
     lib.mmv_debug_force_scan_shape.argtypes = [ci]
     lib.mmv_debug_force_sum_groups.restype = None
@@ -204,6 +206,23 @@ def seg_scan_shard_finish(summaries: torch.Tensor, rank: int, world: int, out: t
     rc = _lib.mmv_seg_scan_shard_finish(_ptr(summaries), int(rank), int(world), _ptr(out), out.numel(), dt, _stream_ptr(stream))
     if rc != MMV_OK:
         raise MmvError(rc, "mmv_seg_scan_shard_finish")
+    return out
+
+
+def mult_i8(x: torch.Tensor, y: torch.Tensor, out: torch.Tensor | None = None, workspace: torch.Tensor | None = None,
+            stream=None) -> torch.Tensor:
+    """mmv_mult_i8: element-wise product of two int8 vectors through the segmented sum (Corollary 4.5), int32."""
+    _check_cuda(x, y, out, workspace)
+    if x.dtype != torch.int8 or y.dtype != torch.int8 or x.numel() != y.numel():
+        raise TypeError("two int8 vectors of the same length expected")
+    n = x.numel()
+    if out is None:
+        out = torch.empty(n, dtype=torch.int32, device=x.device)
+    if workspace is None:
+        workspace = alloc_workspace(OP_MULT, I8_TO_I32, SEG_OFFSETS_I32, n, 0, x.device)
+    rc = _lib.mmv_mult_i8(_ptr(x), _ptr(y), n, _ptr(out), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != MMV_OK:
+        raise MmvError(rc, "mmv_mult_i8")
     return out
 
 

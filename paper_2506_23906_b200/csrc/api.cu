@@ -450,6 +450,51 @@ __global__ void shard_finish_kernel(const ShardSummary* __restrict__ all, int ra
     if (k < limit) out[k] = add(out[k]);
 }
 
+// ---------------------------------------------------------------------------
+// Element-wise integer product through the segmented sum (Section 4.3.1, Lemma 4.4 / Corollary 4.5): the
+// product x(i) y(i) is the sum of the partial terms of the school method, c_k = (bit k of y) ? x 2^k : 0 (bit 7
+// of a two's-complement byte weighs -2^7); all terms of all products form one vector whose segments of 8 are
+// summed by the tensor-core kernel.  Every term (|c_k| <= 2^14, a shifted int8) is exactly an fp16 value and
+// every sum (|x y| <= 2^14) exactly an fp32 value, so the result is exact.
+// ---------------------------------------------------------------------------
+constexpr int MULT_TERMS = 8;
+__global__ void mult_expand_kernel(const int8_t* __restrict__ x, const int8_t* __restrict__ y, long long n,
+                                   __half* __restrict__ terms, int32_t* __restrict__ off) {
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i <= n; i += stride) {
+        off[i] = static_cast<int32_t>(i * MULT_TERMS);
+        if (i == n) break;
+        const int xi = x[i];
+        const unsigned yi = static_cast<unsigned char>(y[i]);
+        __half t[MULT_TERMS];
+#pragma unroll
+        for (int k = 0; k < MULT_TERMS; ++k) {
+            const int w = k == 7 ? -128 : (1 << k);
+            t[k] = __int2half_rn(((yi >> k) & 1u) ? xi * w : 0);          // exact: |x 2^k| <= 2^14
+        }
+        *reinterpret_cast<uint4*>(terms + i * MULT_TERMS) = *reinterpret_cast<const uint4*>(t);
+    }
+}
+// the sums are exact integers in fp32: rewrite them in place as int32
+__global__ void mult_to_int_kernel(float* __restrict__ io, long long n) {
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += stride)
+        reinterpret_cast<int32_t*>(io)[i] = __float2int_rn(io[i]);
+}
+
+struct MultPlan {
+    WorkspacePlan sum;          // the segmented sum over 8 n terms in n segments, at the workspace's base
+    size_t terms_off, off_off, total;
+};
+MultPlan plan_mult(long long n) {
+    MultPlan p{};
+    p.sum = plan_workspace(MMV_OP_SEG_SUM, MMV_SEG_OFFSETS_I32, n * MULT_TERMS);
+    p.terms_off = p.sum.total;
+    p.off_off = p.terms_off + round_up(static_cast<size_t>(n) * MULT_TERMS * sizeof(__half), 256);
+    p.total = p.off_off + round_up(static_cast<size_t>(n + 1) * sizeof(int32_t), 256);
+    return p;
+}
+
 }  // namespace
 }  // namespace mmv
 
@@ -459,6 +504,7 @@ extern "C" {
 
 size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, int64_t nseg) {
     if (n < 0 || nseg < 0) return 0;
+    if (op == MMV_OP_MULT) return n < (1ll << 28) ? plan_mult(n).total : 0;
     if (op != MMV_OP_SEG_SCAN && op != MMV_OP_SEG_SUM && op != MMV_OP_SPMV_CSR && op != MMV_OP_COMPRESS &&
         op != MMV_OP_SEG_SCAN_MINMAX && op != MMV_OP_SEG_SCAN_WIDE)
         return 0;
@@ -978,6 +1024,35 @@ mmv_status mmv_compress(const void* x, const void* flags, int64_t n, mmv_dtype d
         compress_values_kernel<unsigned short><<<blocks, CMP_THREADS, 0, st>>>(static_cast<const unsigned short*>(x), masks, nchunks,
                                                                               chunk_base, static_cast<unsigned short*>(out));
     g_launches += 3;
+    return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+}
+
+mmv_status mmv_mult_i8(const int8_t* x, const int8_t* y, int64_t n, int32_t* out, void* workspace, size_t workspace_bytes,
+                       void* cuda_stream) {
+    if (n < 0 || n >= (1ll << 28)) return MMV_ERR_INVALID_ARG;          // 8 n terms are addressed by int32 offsets
+    if (n == 0) return MMV_OK;
+    if (!x || !y || !out || !workspace) return MMV_ERR_INVALID_ARG;
+    if (!aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MMV_ERR_INVALID_ARG;
+    const MultPlan plan = plan_mult(n);
+    if (workspace_bytes < plan.total) return MMV_ERR_WORKSPACE_TOO_SMALL;
+    DeviceInfo* dev = device_info();
+    if (!dev) return MMV_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    __half* terms = reinterpret_cast<__half*>(ws + plan.terms_off);
+    int32_t* off = reinterpret_cast<int32_t*>(ws + plan.off_off);
+    const int threads = 256;
+    long long blocks = (n + threads) / threads;
+    const long long cap = static_cast<long long>(dev->sm_count) * 16;
+    if (blocks > cap) blocks = cap;
+    mult_expand_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(x, y, n, terms, off);
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) return MMV_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, plan.sum.status_off + plan.sum.status_bytes, st) != cudaSuccess) return MMV_ERR_CUDA;
+    const mmv_status rc = launch_seg_sum<F16Path>(terms, n * MULT_TERMS, off, n, 0, out, ws, plan.sum, dev, st);
+    if (rc != MMV_OK) return rc;
+    mult_to_int_kernel<<<static_cast<unsigned>(blocks), threads, 0, st>>>(reinterpret_cast<float*>(out), n);
+    ++g_launches;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }
 

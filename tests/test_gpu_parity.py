@@ -1238,3 +1238,25 @@ def test_scan_narrow_shape_is_correct_for_every_flag_vector(mmv):
             assert_fp(scan_f16(mmv, x, f), z, a, f"narrow shape, p={p}")
     finally:
         mmv.debug_force_scan_shape(-1)
+
+
+# ---------------------------------------------------------------------------
+# element-wise integer product through the segmented sum (Corollary 4.5)
+# ---------------------------------------------------------------------------
+def test_mult_i8_is_exact(mmv):
+    v = np.arange(-128, 128, dtype=np.int64)
+    xs, ys = np.repeat(v, 256).astype(np.int8), np.tile(v, 256).astype(np.int8)          # every pair of int8 values
+    got = mmv.mult_i8(dev(xs), dev(ys)).cpu().numpy()
+    assert np.array_equal(got, oracle.mult_i8(xs, ys))
+    rng = np.random.default_rng(6)
+    for n in (1, 7, 511, 513, 2049, 40 * TILE // 8 + 3, 300_001):
+        x = rng.integers(-128, 128, n).astype(np.int8)
+        y = rng.integers(-128, 128, n).astype(np.int8)
+        ws = mmv.alloc_workspace(mmv.OP_MULT, mmv.I8_TO_I32, mmv.SEG_OFFSETS_I32, n)
+        buf = torch.full((n + 16,), -777, dtype=torch.int32, device="cuda")
+        mmv.mult_i8(dev(x), dev(y), out=buf[:n], workspace=ws)
+        assert mmv.last_async_status(ws) == 0
+        g = buf.cpu().numpy()
+        assert (g[n:] == -777).all()
+        assert np.array_equal(g[:n], oracle.mult_i8(x, y)), n
+    assert mmv.mult_i8(dev(np.zeros(0, np.int8)), dev(np.zeros(0, np.int8))).numel() == 0
