@@ -817,13 +817,25 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 uint32_t vv[SUM_SPARSE_MAX];
 #pragma unroll
                 for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * ROW + (ROW - 1)));
-#pragma unroll
-                for (int j = 0; j < SUM_SPARSE_MAX; ++j) {
+                // (spans with at most two boundaries -- the usual case with long segments -- skip the other six slots
+                //  with one branch instead of issuing their predicated-off instructions: n = 2^28, lengths
+                //  U{1..4096}: 104.4 -> 98.9 us.  Replacing the four scans by one masked warp sum per boundary for
+                //  such spans measured slower again, 104 us.)
+                auto request = [&](int j) {
                     vv[j] = 0u;
                     if (j < nb_span) {
                         const int e = __shfl_sync(0xffffffffu, crel, j) - 1;                 // element before the boundary
                         if (e >= 0) vv[j] = tmem_ld_32x1(taddr + (e >> 10) * ROW + (e & 31));
                     }
+                };
+                request(0);
+                request(1);
+                if (nb_span > 2) {
+#pragma unroll
+                    for (int j = 2; j < SUM_SPARSE_MAX; ++j) request(j);
+                } else {
+#pragma unroll
+                    for (int j = 2; j < SUM_SPARSE_MAX; ++j) vv[j] = 0u;
                 }
                 tmem_ld_wait();
                 MMV_T_MARK(12)
@@ -852,10 +864,15 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 const int myrow = have ? (e >> 5) : -1;                  // row inside the span (0..127)
                 const int src = have ? (myrow & 31) : 0;
                 Acc mylocal = Acc(0), myrp = Acc(0);
-#pragma unroll
-                for (int j = 0; j < SUM_SPARSE_MAX; ++j) {
+                auto fetch = [&](int j) {
                     const uint32_t t = __shfl_sync(0xffffffffu, vv[j], src);
                     if (static_cast<int>(lane) == j) mylocal = P::from_bits(t);
+                };
+                fetch(0);
+                fetch(1);
+                if (nb_span > 2) {
+#pragma unroll
+                    for (int j = 2; j < SUM_SPARSE_MAX; ++j) fetch(j);
                 }
 #pragma unroll
                 for (int i = 0; i < PIECES_PER_SPAN; ++i) {
