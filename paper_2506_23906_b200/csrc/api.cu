@@ -234,7 +234,9 @@ WorkspacePlan plan_workspace(mmv_op op, mmv_segfmt sf, long long n) {
     p.cmp_off = p.prod_off + p.prod_bytes;
     p.cmp_bytes = flagsum ? round_up(static_cast<size_t>(2 * nchunks + 8) * sizeof(int32_t) + 16, 256) : 0;
     p.mask_off = p.cmp_off + p.cmp_bytes;
-    p.mask_bytes = flagsum ? round_up(static_cast<size_t>(nchunks) * CMP_THREADS * sizeof(unsigned long long), 256) : 0;
+    // (+ one int32 per warp of the count pass: the number of set flags of its chunk in front of it)
+    p.mask_bytes = flagsum ? round_up(static_cast<size_t>(nchunks) * CMP_THREADS * sizeof(unsigned long long), 256) +
+                                 round_up(static_cast<size_t>(nchunks) * CMP_WARPS * sizeof(int32_t), 256) : 0;
     p.off_off = p.mask_off + p.mask_bytes;
     p.off_bytes = (flagsum && op != MMV_OP_COMPRESS) ? round_up(static_cast<size_t>(n + 1) * sizeof(int32_t), 256) : 0;
     p.total = p.off_off + p.off_bytes;
@@ -872,11 +874,12 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
         const long long cap = static_cast<long long>(dev->sm_count) * 8;
         const unsigned blocks = static_cast<unsigned>(nchunks < cap ? nchunks : cap);
         unsigned long long* masks = reinterpret_cast<unsigned long long*>(ws + plan.mask_off);
-        flag_count_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_count, masks);
-        chunk_scan_kernel<<<1, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, nseg_dev,
+        int32_t* warp_off = reinterpret_cast<int32_t*>(ws + plan.mask_off + round_up(static_cast<size_t>(nchunks) * CMP_THREADS * sizeof(unsigned long long), 256));
+        flag_count_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_count, masks, warp_off);
+        chunk_scan_kernel<<<CMP_SCAN_BLOCKS, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, nseg_dev,
                                               reinterpret_cast<long long*>(d_num_segments), off, n);
         static_assert(CMP_CHUNK == TILE && SPAN == 4096, "a compaction chunk is one tile of four spans");
-        flag_scatter_kernel<<<blocks, CMP_THREADS, 0, st>>>(masks, n, nchunks, chunk_base, off,
+        flag_scatter_kernel<<<blocks, CMP_THREADS, 0, st>>>(masks, n, nchunks, chunk_base, warp_off, off,
                                                             reinterpret_cast<int32_t*>(ws + plan.tileq_off), nseg_dev);
         g_launches += 3;
         if (cudaGetLastError() != cudaSuccess) return MMV_ERR_CUDA;
@@ -1014,15 +1017,16 @@ mmv_status mmv_compress(const void* x, const void* flags, int64_t n, mmv_dtype d
     const long long cap = static_cast<long long>(dev->sm_count) * 8;
     const unsigned blocks = static_cast<unsigned>(nchunks < cap ? nchunks : cap);
     unsigned long long* masks = reinterpret_cast<unsigned long long*>(ws + plan.mask_off);
-    flag_count_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_count, masks, false);
-    chunk_scan_kernel<<<1, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, count_dev, reinterpret_cast<long long*>(d_count),
+    int32_t* warp_off = reinterpret_cast<int32_t*>(ws + plan.mask_off + round_up(static_cast<size_t>(nchunks) * CMP_THREADS * sizeof(unsigned long long), 256));
+    flag_count_kernel<<<blocks, CMP_THREADS, 0, st>>>(f, n, nchunks, chunk_count, masks, warp_off, false);
+    chunk_scan_kernel<<<CMP_SCAN_BLOCKS, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, count_dev, reinterpret_cast<long long*>(d_count),
                                           nullptr, n);
     if (dt == MMV_I8_TO_I32)
         compress_values_kernel<uint8_t><<<blocks, CMP_THREADS, 0, st>>>(static_cast<const uint8_t*>(x), masks, nchunks, chunk_base,
-                                                                       static_cast<uint8_t*>(out));
+                                                                       warp_off, static_cast<uint8_t*>(out));
     else
         compress_values_kernel<unsigned short><<<blocks, CMP_THREADS, 0, st>>>(static_cast<const unsigned short*>(x), masks, nchunks,
-                                                                              chunk_base, static_cast<unsigned short*>(out));
+                                                                              chunk_base, warp_off, static_cast<unsigned short*>(out));
     g_launches += 3;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
 }

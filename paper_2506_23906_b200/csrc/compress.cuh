@@ -82,34 +82,69 @@ __device__ __forceinline__ unsigned long long flag_words_to_mask(const uint32_t 
 
 // chunk_count[c] = number of segment starts among the flags of chunk c; masks[c * CMP_THREADS + t] = the 64
 // flags of thread t as bits.
+// warp_off[c * CMP_WARPS + w] = number of set flags of chunk c in front of warp w's 2048 flags: with it the
+// scatter passes need no block-wide barrier, a warp scan of its own 32 counts is enough.
+constexpr int CMP_WARPS = CMP_THREADS / 32;
 __global__ void __launch_bounds__(CMP_THREADS)
 flag_count_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks, int32_t* __restrict__ chunk_count,
-                  unsigned long long* __restrict__ masks, bool first_is_start = true) {
+                  unsigned long long* __restrict__ masks, int32_t* __restrict__ warp_off, bool first_is_start = true) {
     __shared__ int warp_sums[32];
     for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
         uint32_t w[16];
         load_thread_flags(f, n, c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD, w, first_is_start);
         const unsigned long long m = flag_words_to_mask(w);
         masks[c * CMP_THREADS + threadIdx.x] = m;
+        const int cnt = __popcll(m);
         int total;
-        block_exclusive_scan(__popcll(m), &total, warp_sums);
+        const int before = block_exclusive_scan(cnt, &total, warp_sums);
+        if ((threadIdx.x & 31) == 0) warp_off[c * CMP_WARPS + (threadIdx.x >> 5)] = before;
         if (threadIdx.x == 0) chunk_count[c] = total;
     }
 }
 
-// One block: chunk_base = exclusive scan of chunk_count; K = total is written to nseg_dev and, when given,
-// to the caller's d_num_segments; off[K] = n closes the last segment.
+// exclusive scan of one int per lane over the warp
+__device__ __forceinline__ int warp_exclusive_scan(int v) {
+    const int lane = threadIdx.x & 31;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    return inc - v;
+}
+
+// chunk_base = exclusive scan of chunk_count; K = total is written to nseg_dev and, when given, to the caller's
+// d_num_segments; off[K] = n closes the last segment.  A few blocks share the work: block b first adds up the
+// counts in front of its part (all its threads, 16-byte loads; the counts are a few hundred KB and stay in the
+// L2), then scans its part.  One block alone took 21 us for the 65,536 chunks of 2^30 flags.
+constexpr int CMP_SCAN_BLOCKS = 32;
 __global__ void __launch_bounds__(1024)
 chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, int32_t* __restrict__ chunk_base,
                   long long* __restrict__ nseg_dev, long long* __restrict__ d_num_segments, int32_t* __restrict__ off,
                   long long n) {
     __shared__ int warp_sums[32];
-    // Each thread takes `per` consecutive counts, a multiple of four so that it can read and write
-    // them as 16-byte vectors: with scalar accesses 64 bytes apart every instruction of a warp touches
-    // 32 sectors, and this one block then spends 20 us in its load/store unit.
-    const long long per = ((nchunks + blockDim.x - 1) / blockDim.x + 3) & ~3ll;
-    const long long lo = static_cast<long long>(threadIdx.x) * per;
-    const long long hi = lo + per < nchunks ? lo + per : nchunks;
+    __shared__ int s_front;
+    // parts are multiples of 4 * blockDim.x counts so that every thread reads and writes 16-byte vectors
+    const long long unit = 4ll * blockDim.x;
+    const long long part = ((nchunks + gridDim.x - 1) / gridDim.x + unit - 1) / unit * unit;
+    const long long p0 = static_cast<long long>(blockIdx.x) * part;
+    const long long p1 = p0 + part < nchunks ? p0 + part : nchunks;
+    // (1) the counts in front of my part
+    int front = 0;
+    for (long long c = 4ll * threadIdx.x; c < p0; c += unit) {          // p0 is a multiple of 4
+        const int4 v = __ldg(reinterpret_cast<const int4*>(chunk_count + c));
+        front += v.x + v.y + v.z + v.w;
+    }
+    int total;
+    block_exclusive_scan(front, &total, warp_sums);
+    if (threadIdx.x == 0) s_front = total;
+    __syncthreads();
+    int run_base = s_front;
+    // (2) my part: each thread takes `per` consecutive counts, a multiple of four
+    const long long per = part / blockDim.x;
+    const long long lo = p0 + static_cast<long long>(threadIdx.x) * per;
+    const long long hi = lo + per < p1 ? lo + per : p1;
     int local = 0;
     for (long long c = lo; c < hi; c += 4) {
         if (c + 4 <= hi) {
@@ -119,8 +154,7 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
             for (long long d = c; d < hi; ++d) local += __ldg(chunk_count + d);
         }
     }
-    int total;
-    int run = block_exclusive_scan(local, &total, warp_sums);
+    int run = run_base + block_exclusive_scan(local, &total, warp_sums);
     for (long long c = lo; c < hi; c += 4) {
         if (c + 4 <= hi) {
             const int4 v = __ldg(reinterpret_cast<const int4*>(chunk_count + c));
@@ -133,10 +167,12 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
             }
         }
     }
-    if (threadIdx.x == 0) {
-        *nseg_dev = total;
-        if (d_num_segments) *d_num_segments = total;
-        if (off) off[total] = static_cast<int32_t>(n);
+    // the block that holds the last chunk knows the grand total
+    if (threadIdx.x == 0 && p0 < nchunks && p1 == nchunks) {
+        const int grand = run_base + total;
+        *nseg_dev = grand;
+        if (d_num_segments) *d_num_segments = grand;
+        if (off) off[grand] = static_cast<int32_t>(n);
     }
 }
 
@@ -147,8 +183,8 @@ chunk_scan_kernel(const int32_t* __restrict__ chunk_count, long long nchunks, in
 // starts at n, K + 1 ("none") beyond.
 __global__ void __launch_bounds__(CMP_THREADS)
 flag_scatter_kernel(const unsigned long long* __restrict__ masks, long long n, long long nchunks, const int32_t* __restrict__ chunk_base,
-                    int32_t* __restrict__ off, int32_t* __restrict__ span_q, const long long* __restrict__ nseg_dev) {
-    __shared__ int warp_sums[32];
+                    const int32_t* __restrict__ warp_off, int32_t* __restrict__ off, int32_t* __restrict__ span_q,
+                    const long long* __restrict__ nseg_dev) {
     constexpr int kThreadsPerSpan = 4096 / CMP_PER_THREAD;
     const long long K = *nseg_dev;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -158,8 +194,7 @@ flag_scatter_kernel(const unsigned long long* __restrict__ masks, long long n, l
     for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
         const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
         unsigned long long m = masks[c * CMP_THREADS + threadIdx.x];
-        int total;
-        int slot = chunk_base[c] + block_exclusive_scan(__popcll(m), &total, warp_sums);
+        int slot = chunk_base[c] + warp_off[c * CMP_WARPS + (threadIdx.x >> 5)] + warp_exclusive_scan(__popcll(m));
         if (threadIdx.x % kThreadsPerSpan == 0)
             span_q[c * (CMP_CHUNK / 4096) + threadIdx.x / kThreadsPerSpan] =
                 static_cast<int32_t>(base < n ? slot : (base == n ? K : K + 1));
@@ -175,13 +210,11 @@ flag_scatter_kernel(const unsigned long long* __restrict__ masks, long long n, l
 template <typename T>
 __global__ void __launch_bounds__(CMP_THREADS)
 compress_values_kernel(const T* __restrict__ x, const unsigned long long* __restrict__ masks, long long nchunks,
-                       const int32_t* __restrict__ chunk_base, T* __restrict__ out) {
-    __shared__ int warp_sums[32];
+                       const int32_t* __restrict__ chunk_base, const int32_t* __restrict__ warp_off, T* __restrict__ out) {
     for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
         const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
         unsigned long long m = masks[c * CMP_THREADS + threadIdx.x];
-        int total;
-        long long slot = chunk_base[c] + block_exclusive_scan(__popcll(m), &total, warp_sums);
+        long long slot = chunk_base[c] + warp_off[c * CMP_WARPS + (threadIdx.x >> 5)] + warp_exclusive_scan(__popcll(m));
         while (m) {
             out[slot++] = x[base + (__ffsll(static_cast<long long>(m)) - 1)];
             m &= m - 1;
