@@ -550,14 +550,28 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
             for (int i = 0; i < UP; ++i)
                 if (pm[i]) istar = i;
             const bool flagged = anyp != 0u;
+            // the unit's last start: row lstar of piece istar, position pl in that row (known from the masks alone)
+            int lstar = 0, pl = 0;
+            if (flagged) {
+                uint32_t pms = pm[0], fms = fm[0];
+#pragma unroll
+                for (int i = 1; i < UP; ++i)
+                    if (istar == i) { pms = pm[i]; fms = fm[i]; }
+                lstar = 31 - __clz(pms);
+                pl = 31 - __clz(__shfl_sync(0xffffffffu, fms, lstar));
+            }
             Acc tot[UP];
 #pragma unroll
             for (int i = 0; i < UP; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * N + (ROW - 1)));
-            // floating point: the rows of the last flagged piece themselves (the identity half of the product)
-            // travel with the same wait; the tail behind the unit's last start is added up from them
+            // What the tail behind the unit's last start needs travels with the same wait.  Floating point: the rows
+            // of the last flagged piece themselves (the identity half of the product).  Integers: the prefix in
+            // front of that start.
             uint32_t xr[Cfg::kWide ? 32 : 1];
+            uint32_t before_bits = 0u;
             if constexpr (Cfg::kWide) {
                 if (flagged) tmem_ld_32x32(taddr + istar * N + ROW, xr);
+            } else if constexpr (!P::kIsFloat) {
+                if (flagged && pl > 0) before_bits = tmem_ld_32x1(taddr + istar * N + (pl - 1));
             }
             tmem_ld_wait();
             Acc tail_unit;
@@ -567,14 +581,10 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                 for (int i = 1; i < UP; ++i) t = P::add(t, tot[i]);
                 tail_unit = warp_sum<P>(t);
             } else {
-                uint32_t pms = pm[0], fms = fm[0];
                 Acc tots = tot[0];
 #pragma unroll
                 for (int i = 1; i < UP; ++i)
-                    if (istar == i) { pms = pm[i]; fms = fm[i]; tots = tot[i]; }
-                const int lstar = 31 - __clz(pms);
-                const uint32_t fmstar = __shfl_sync(0xffffffffu, fms, lstar);
-                const int pl = 31 - __clz(fmstar);            // last flag of the last flagged row
+                    if (istar == i) tots = tot[i];
                 Acc after = Acc(0);                            // totals of the rows behind it
 #pragma unroll
                 for (int i = 0; i < UP; ++i)
@@ -598,12 +608,7 @@ seg_scan_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constan
                     if (static_cast<int>(lane) == lstar)
                         row_tail = row_tail_from_memory<P>(prm.x, s * SCAN_UNIT + istar * PIECE + lstar * ROW, pl, prm.n);
                 } else {
-                    Acc before = Acc(0);
-                    if (pl > 0) {
-                        before = P::from_bits(tmem_ld_32x1(taddr + istar * N + (pl - 1)));
-                        tmem_ld_wait();
-                    }
-                    row_tail = P::sub(tots, before);           // exact: integer arithmetic modulo 2^32 is a group
+                    row_tail = P::sub(tots, P::from_bits(before_bits));      // exact: integer arithmetic modulo 2^32 is a group
                 }
                 tail_unit = P::add(__shfl_sync(0xffffffffu, row_tail, lstar), after);
             }
