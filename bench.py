@@ -57,6 +57,8 @@ def parse_args():
     ap.add_argument("--case", default="p1e-3", help="flag pattern of the headline workload")
     ap.add_argument("--no-configs", action="store_true", help="skip the per-configuration table")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline")
+    ap.add_argument("--scan-shape", type=int, default=-1, choices=[-1, 0, 2],
+                    help="with --profile-case: force the wide (0) or narrow (2) tiles of the floating-point scan (-1: the library chooses)")
     ap.add_argument("--profile-case", default=None, choices=["scan_f16", "scan_i8", "seg_sum", "seg_sum_short", "seg_sum_mid", "spmv", "minmax", "wide"],
                     help="run one small case a few times and exit (the command profiled with ncu)")
     return ap.parse_args()
@@ -746,6 +748,7 @@ def run_profile_case(args):
     import torch
     import paper_2506_23906_b200 as mmv
     torch.cuda.set_device(0)
+    mmv.debug_force_scan_shape(args.scan_shape)
     n = 1 << min(args.log2n, 27)
     if args.profile_case in ("scan_f16", "scan_i8"):
         f16 = args.profile_case == "scan_f16"
