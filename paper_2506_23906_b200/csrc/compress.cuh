@@ -85,6 +85,7 @@ __device__ __forceinline__ unsigned long long flag_words_to_mask(const uint32_t 
 // warp_off[c * CMP_WARPS + w] = number of set flags of chunk c in front of warp w's 2048 flags: with it the
 // scatter passes need no block-wide barrier, a warp scan of its own 32 counts is enough.
 constexpr int CMP_WARPS = CMP_THREADS / 32;
+constexpr int CMP_BATCH = 4;               // chunks a block of a scatter pass requests together
 __global__ void __launch_bounds__(CMP_THREADS)
 flag_count_kernel(const uint8_t* __restrict__ f, long long n, long long nchunks, int32_t* __restrict__ chunk_count,
                   unsigned long long* __restrict__ masks, int32_t* __restrict__ warp_off, bool first_is_start = true) {
@@ -191,16 +192,34 @@ flag_scatter_kernel(const unsigned long long* __restrict__ masks, long long n, l
         const long long end = nchunks * CMP_CHUNK;
         span_q[nchunks * (CMP_CHUNK / 4096)] = static_cast<int32_t>(end == n ? K : K + 1);
     }
-    for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
-        const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
-        unsigned long long m = masks[c * CMP_THREADS + threadIdx.x];
-        int slot = chunk_base[c] + warp_off[c * CMP_WARPS + (threadIdx.x >> 5)] + warp_exclusive_scan(__popcll(m));
-        if (threadIdx.x % kThreadsPerSpan == 0)
-            span_q[c * (CMP_CHUNK / 4096) + threadIdx.x / kThreadsPerSpan] =
-                static_cast<int32_t>(base < n ? slot : (base == n ? K : K + 1));
-        while (m) {
-            off[slot++] = static_cast<int32_t>(base + (__ffsll(static_cast<long long>(m)) - 1));
-            m &= m - 1;
+    // (four chunks per round, their loads requested together: the pass is bound by the latency of its loads)
+    for (long long c0 = blockIdx.x; c0 < nchunks; c0 += static_cast<long long>(CMP_BATCH) * gridDim.x) {
+        unsigned long long mk[CMP_BATCH];
+        int start[CMP_BATCH];
+#pragma unroll
+        for (int k = 0; k < CMP_BATCH; ++k) {
+            const long long c = c0 + static_cast<long long>(k) * gridDim.x;
+            mk[k] = 0ull;
+            start[k] = 0;
+            if (c < nchunks) {
+                mk[k] = masks[c * CMP_THREADS + threadIdx.x];
+                start[k] = chunk_base[c] + warp_off[c * CMP_WARPS + (threadIdx.x >> 5)];
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < CMP_BATCH; ++k) {
+            const long long c = c0 + static_cast<long long>(k) * gridDim.x;
+            if (c >= nchunks) break;
+            const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
+            unsigned long long m = mk[k];
+            int slot = start[k] + warp_exclusive_scan(__popcll(m));
+            if (threadIdx.x % kThreadsPerSpan == 0)
+                span_q[c * (CMP_CHUNK / 4096) + threadIdx.x / kThreadsPerSpan] =
+                    static_cast<int32_t>(base < n ? slot : (base == n ? K : K + 1));
+            while (m) {
+                off[slot++] = static_cast<int32_t>(base + (__ffsll(static_cast<long long>(m)) - 1));
+                m &= m - 1;
+            }
         }
     }
 }
@@ -211,13 +230,30 @@ template <typename T>
 __global__ void __launch_bounds__(CMP_THREADS)
 compress_values_kernel(const T* __restrict__ x, const unsigned long long* __restrict__ masks, long long nchunks,
                        const int32_t* __restrict__ chunk_base, const int32_t* __restrict__ warp_off, T* __restrict__ out) {
-    for (long long c = blockIdx.x; c < nchunks; c += gridDim.x) {
-        const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
-        unsigned long long m = masks[c * CMP_THREADS + threadIdx.x];
-        long long slot = chunk_base[c] + warp_off[c * CMP_WARPS + (threadIdx.x >> 5)] + warp_exclusive_scan(__popcll(m));
-        while (m) {
-            out[slot++] = x[base + (__ffsll(static_cast<long long>(m)) - 1)];
-            m &= m - 1;
+    for (long long c0 = blockIdx.x; c0 < nchunks; c0 += static_cast<long long>(CMP_BATCH) * gridDim.x) {
+        unsigned long long mk[CMP_BATCH];
+        int start[CMP_BATCH];
+#pragma unroll
+        for (int k = 0; k < CMP_BATCH; ++k) {
+            const long long c = c0 + static_cast<long long>(k) * gridDim.x;
+            mk[k] = 0ull;
+            start[k] = 0;
+            if (c < nchunks) {
+                mk[k] = masks[c * CMP_THREADS + threadIdx.x];
+                start[k] = chunk_base[c] + warp_off[c * CMP_WARPS + (threadIdx.x >> 5)];
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < CMP_BATCH; ++k) {
+            const long long c = c0 + static_cast<long long>(k) * gridDim.x;
+            if (c >= nchunks) break;
+            const long long base = c * CMP_CHUNK + static_cast<long long>(threadIdx.x) * CMP_PER_THREAD;
+            unsigned long long m = mk[k];
+            long long slot = start[k] + warp_exclusive_scan(__popcll(m));
+            while (m) {
+                out[slot++] = x[base + (__ffsll(static_cast<long long>(m)) - 1)];
+                m &= m - 1;
+            }
         }
     }
 }
