@@ -1022,10 +1022,10 @@ mmv_status mmv_compress(const void* x, const void* flags, int64_t n, mmv_dtype d
     chunk_scan_kernel<<<CMP_SCAN_BLOCKS, 1024, 0, st>>>(chunk_count, nchunks, chunk_base, count_dev, reinterpret_cast<long long*>(d_count),
                                           nullptr, n);
     if (dt == MMV_I8_TO_I32)
-        compress_values_kernel<uint8_t><<<blocks, CMP_THREADS, 0, st>>>(static_cast<const uint8_t*>(x), masks, nchunks, chunk_base,
+        compress_values_kernel<uint8_t><<<blocks, CMP_THREADS, 0, st>>>(static_cast<const uint8_t*>(x), masks, n, nchunks, chunk_base,
                                                                        warp_off, static_cast<uint8_t*>(out));
     else
-        compress_values_kernel<unsigned short><<<blocks, CMP_THREADS, 0, st>>>(static_cast<const unsigned short*>(x), masks, nchunks,
+        compress_values_kernel<unsigned short><<<blocks, CMP_THREADS, 0, st>>>(static_cast<const unsigned short*>(x), masks, n, nchunks,
                                                                               chunk_base, warp_off, static_cast<unsigned short*>(out));
     g_launches += 3;
     return cudaGetLastError() == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;

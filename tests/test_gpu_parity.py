@@ -622,6 +622,38 @@ def test_compress(mmv, n, p):
     assert np.array_equal(out[:k].view(torch.int16).cpu().numpy().view(np.uint16), oracle.compress(xb, f))
 
 
+def test_compress_with_dense_and_sparse_stretches(mmv):
+    # stretches of 2048 elements (one warp's share of a chunk) with 0, a few, 127, 128, 129, half and all flags
+    # set, in random order: both routes of the scatter pass, every phase of the output inside a 16-byte vector
+    rng = np.random.default_rng(5)
+    counts = [0, 1, 3, 40, 127, 128, 129, 500, 1024, 2047, 2048]
+    for trial in range(3):
+        pieces = []
+        for _ in range(40):
+            k = int(rng.choice(counts))
+            piece = np.zeros(2048, np.uint8)
+            piece[rng.choice(2048, k, replace=False)] = rng.integers(1, 256, k)
+            pieces.append(piece)
+        f = np.concatenate(pieces)[: 40 * 2048 - int(rng.integers(0, 2048))]
+        n = f.shape[0]
+        for x in (rng.integers(-128, 128, n).astype(np.int8), rng.standard_normal(n).astype(np.float16)):
+            want = oracle.compress(x, f)
+            guard = torch.full((n + 8,), 77, dtype=torch.from_numpy(x[:1]).dtype, device="cuda")
+            out, count = mmv.compress(dev(x), dev(f), out=guard[:n])
+            k = int(count.item())
+            got = guard.cpu().numpy()
+            assert k == want.shape[0]
+            assert np.array_equal(got[:k].view(np.uint8), want.view(np.uint8))
+            assert (got[n:] == 77).all()
+        # the same flags as segment starts of a flag-encoded segmented sum (positions instead of values)
+        xi = gen.i8_uniform(9, n)
+        kd = torch.zeros(1, dtype=torch.int64, device="cuda")
+        got = mmv.seg_sum(dev(xi), dev(f), num_segments=kd)
+        want = oracle.seg_sum_flags_i8(xi, f)
+        assert int(kd.item()) == want.shape[0]
+        assert np.array_equal(got[: want.shape[0]].cpu().numpy(), want)
+
+
 def test_compress_of_the_paper_example(mmv):
     g = __import__("conftest").load_golden("sec2_worked_example.txt")
     out, count = mmv.compress(dev(np.asarray(g["x"], np.int8)), dev(np.asarray(g["f"], np.uint8)))
