@@ -393,6 +393,24 @@ def bench_configs(torch, mmv, peak, steps, warmup, l2_flush, cpu_leg):
         {"segments": k, **baseline(n, lambda o: o.seg_sum_flags_f16(x, f), fp_compare(outf[:k].cpu().numpy()))})
     del xd, fd, out, outf, ws
 
+    # and sixteen times larger: the fixed cost of a call (launch, set-up, the partition of the offsets and the
+    # grid-wide barrier behind it, the first loads: about 10 us) is a tenth of the call at n = 2^28 and a
+    # fortieth here, so this line shows the rate the kernel sustains
+    x, off = gen.config2(1 << 30)
+    n, nseg = x.shape[0], off.shape[0] - 1
+    xd, od = torch.from_numpy(x).cuda(), torch.from_numpy(off).cuda()
+    out = torch.empty(nseg, dtype=torch.float32, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, n, nseg)
+    fn = lambda: mmv.seg_sum(xd, od, out=out, workspace=ws)  # noqa: E731
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ms = event_time_ms(torch, fn, steps)
+    assert mmv.last_async_status(ws) == 0
+    rec("C2x16 seg-sum n=2^30 fp16 N(0,1), CSR offsets len U{1..4096}", n, 2 * n + 4 * (nseg + 1) + 4 * nseg, ms,
+        {"segments": nseg, **baseline(n, lambda o: o.seg_sum_csr_f16(x, off), fp_compare(out.cpu().numpy()))})
+    del xd, od, out, ws
+
     x, f = gen.config3()
     run_scan("C3 seg-scan n=2^28 int8 flags 1e-3", x, f)
 
