@@ -322,7 +322,7 @@ mmv_status launch_seg_sum(const void* values, long long n_eff, const int32_t* of
     prm.off = off;
     prm.nseg = nseg;
     prm.n = n_eff;
-    prm.off_shift = shift;
+    (void)shift;
     prm.out = out;
     prm.num_tiles = tiles;
     prm.span_q = span_q;

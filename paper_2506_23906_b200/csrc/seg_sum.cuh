@@ -29,8 +29,9 @@
 //                  front of the row, so nothing is searched or sorted; only rows that contain
 //                  empty segments look their indices up in the offsets.
 //     Floating point: a difference of prefixes loses a small sum next to large values.  In the
-//     few-boundaries path segments of at most four elements are therefore summed from the input
-//     values themselves; in the general path any segment inside one row or two adjacent rows whose
+//     few-boundaries path segments of at most 32 elements are therefore summed from the input
+//     values themselves (up to four: from two words requested ahead; more: one element per lane,
+//     such segments are rare there); in the general path any segment inside one row or two adjacent rows whose
 //     sum came out below 2^-10 of those rows' largest prefix is added up again from its values, and
 //     so is the segment of at most 32 elements that reaches back across the span's first element.
 //     The one segment per span that began before it (and is longer) takes the carry of the sibling
@@ -250,7 +251,6 @@ struct SumParams {
     const int32_t* off;          // nseg + 1 offsets
     long long nseg;
     long long n;                 // number of values
-    int off_shift;               // boundaries are off[q] << off_shift (0 in every current call)
     void* out;                   // nseg results
     int num_tiles;
     const int32_t* span_q;       // 4 * num_tiles + 1: first q with (off[q] << shift) >= span start
@@ -623,7 +623,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         uint32_t* emask = reinterpret_cast<uint32_t*>(smem + Cfg::kMarkOffset + warp * SUM_MARK_BYTES);
         uint32_t* ecnt = emask + SPAN / ROW;
         uint32_t* nbase = ecnt + SPAN / ROW;
-        const int sh = prm.off_shift;
+        constexpr int sh = 0;             // (boundaries are the offsets themselves)
         const long long nq = (prm.nseg_dev ? *prm.nseg_dev : prm.nseg) + 1;
         bool failed = false;
         // The boundaries of the NEXT tile's span are requested one tile ahead (first the span's first
@@ -633,8 +633,6 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             const int t = static_cast<int>(blockIdx.x) + (g + G * kk) * static_cast<int>(gridDim.x);
             return t < prm.num_tiles ? t : -1;
         };
-        // raw offset -> position (index checks against nq are made where an entry is used)
-        auto cvt = [&](int32_t raw) -> long long { return static_cast<long long>(raw) << sh; };
         constexpr int32_t kNoOffset = 0;
         // offsets q0 + lane + 32 j (j < 4), the one before q0, and the last one below the span's end
         // (No arithmetic may touch a prefetched value before the tile that uses it: even a sign
@@ -683,7 +681,6 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
             const int buf = it % SUM_BUFS;
             const long long s = static_cast<long long>(tile) * SPANS_PER_TILE + w;
             const long long sbase = s * SPAN;
-            const long long send = sbase + SPAN;
             const uint32_t taddr = tmem_base + buf * (PIECES_PER_SPAN * ROW) + ((static_cast<uint32_t>(w) * 32u) << 16);
 
             // ---- the span's boundaries: one offset per lane (requested during the previous tile) ----
@@ -694,38 +691,47 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
 #pragma unroll
             for (int j = 0; j < 4; ++j) raw[j] = nraw[j];
             const int32_t rawp = nrawp;
-            const long long last_b = nlast_ok ? cvt(nlast) : -1ll;   // last boundary below the span's end
+            const int32_t last_raw = nlast;                    // last boundary below the span's end (if nlast_ok)
+            const bool last_ok = nlast_ok;
             MMV_T_MARK(8)
             const int tile_n = tile_of(k + 1);
             if (tile_n >= 0) load_span_q(tile_n, q_next, qe_next);
             MMV_T_MARK(10)
             // lane holds boundaries cq + lane + 32 j (j < 4).  The first 32 first: they
             // decides between the path for spans with few boundaries and the general one.
-            long long cb = -1, csb = -1;                       // my boundary among the first 32, and the one before it
+            // (Positions are below 2^31 because the offsets are 32-bit, so what follows is 32-bit arithmetic; the span's
+            //  end may be 2^31 itself, so boundaries are compared relative to the span's first element.)
+            int cb = -1, csb = -1;                             // my boundary among the first 32, and the one before it; -1: none
             {
                 int32_t pr = __shfl_up_sync(0xffffffffu, raw[0], 1);
                 if (lane == 0) pr = rawp;
-                if (cq + lane < nq) cb = cvt(raw[0]);
-                if (cq + lane >= 1) csb = cvt(pr);
+                if (cq + lane < nq) cb = raw[0];
+                if (cq + lane >= 1) csb = pr;
             }
+            const int sb32i = static_cast<int>(sbase);
+            const int n32i = static_cast<int>(prm.n);
+            const int crel = static_cast<int>(static_cast<unsigned>(cb) - static_cast<unsigned>(sb32i));      // (meaningful where cb >= 0)
             // the first 32 entries cover the span if they reach past its end (or the end of the offsets)
-            const bool covers = __any_sync(0xffffffffu, (q + lane >= nq) || (cb > send));
+            const bool covers = __any_sync(0xffffffffu, (q + lane >= nq) || (cb >= 0 && crel > SPAN));
             // number of boundaries with sbase <= bnd <= send (a prefix of the lanes)
-            const int nb_span = __popc(__ballot_sync(0xffffffffu, (cq + lane < nq) && (cb >= 0) && (cb <= send)));
+            const int nb_span = __popc(__ballot_sync(0xffffffffu, cb >= 0 && crel <= SPAN));
             const bool sparse = covers && nb_span <= SUM_SPARSE_MAX;
             // the last segment start inside the span, or -1
-            const int lastrel = (last_b >= sbase && last_b < send) ? static_cast<int>(last_b - sbase) : -1;
+            const int last_d = static_cast<int>(static_cast<unsigned>(last_raw) - static_cast<unsigned>(sb32i));
+            const int lastrel = (last_ok && static_cast<unsigned>(last_d) < static_cast<unsigned>(SPAN)) ? last_d : -1;
             const bool seen = lastrel >= 0;   // a segment start lies inside this span
             MMV_T_MARK(9)
             // very short segments that end in this span are summed from the inputs; the loads go out
             // now and return while the accumulators are awaited
-            bool is_direct = cq + lane >= 1 && cq + lane < nq && csb >= 0 && cb > csb && cb - csb <= SUM_DIRECT_LEN &&
-                             cb > sbase && cb <= send && cb <= prm.n;
+            const int seglen = static_cast<int>(static_cast<unsigned>(cb) - static_cast<unsigned>(csb));     // (meaningful where both exist)
+            // (one unsigned test each: 1 <= length <= SUM_DIRECT_LEN, and the end inside (sbase, send])
+            bool is_direct = csb >= 0 && cb >= 0 && static_cast<unsigned>(seglen - 1) < static_cast<unsigned>(SUM_DIRECT_LEN) &&
+                             static_cast<unsigned>(crel - 1) < static_cast<unsigned>(SPAN) && cb <= n32i;
             // (the general path needs only the one that reaches back across the span's first element)
-            if (!sparse && !(lane == 0 && csb < sbase)) is_direct = false;
+            if (!sparse && !(lane == 0 && csb < sb32i)) is_direct = false;
             ValueWindow win0;
             win0.wide = false;
-            if (is_direct) window_load<P>(xg, csb, static_cast<int>(cb - csb), prm.n, win0);
+            if (is_direct) window_load<P>(xg, csb, seglen, prm.n, win0);
             int xlen = 0;
             Acc xval = Acc(0);
             // ---- general path, first step: every boundary marks the element it ends behind.  emask[row] has
@@ -767,11 +773,12 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 // boundary): with at most 32 elements its values themselves are added up, one per lane.  Its carry
                 // would be a difference of the previous span's prefixes, which loses a small sum next to large values.
                 if constexpr (P::kIsFloat) {
-                    const bool crossing = cq >= 1 && cq < nq && csb >= 0 && csb < sbase && cb > sbase && cb <= send && cb <= prm.n &&
-                                          cb - csb <= 32;
-                    xlen = __shfl_sync(0xffffffffu, crossing ? static_cast<int>(cb - csb) : 0, 0);
+                    // (lane 0's boundary and the one before it)
+                    const bool crossing = csb >= 0 && cb >= 0 && csb < sb32i && static_cast<unsigned>(crel - 1) < static_cast<unsigned>(SPAN) &&
+                                          cb <= n32i && seglen <= 32;
+                    xlen = __shfl_sync(0xffffffffu, crossing ? seglen : 0, 0);
                     if (xlen > 0) {
-                        const long long xsb = __shfl_sync(0xffffffffu, csb, 0);
+                        const long long xsb = __shfl_sync(0xffffffffu, csb, 0);      // (widened: an element index)
                         if (static_cast<int>(lane) < xlen) xval = load_value<P>(xg, xsb + lane);
                     }
                 }
@@ -813,7 +820,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 // ---- few boundaries (lane j <-> boundary j): the one prefix each boundary needs is read
                 //      straight from TMEM (one column; it sits in the lane of its row), together with the
                 //      row totals (column 31), with a single wait ----
-                const int crel = static_cast<int>(cb - sbase);          // 0..SPAN for lanes < nb_span
+                // (crel = cb - sbase is 0..SPAN for lanes < nb_span)
                 uint32_t vv[SUM_SPARSE_MAX];
 #pragma unroll
                 for (int i = 0; i < PIECES_PER_SPAN; ++i) tot[i] = P::from_bits(tmem_ld_32x1(taddr + i * ROW + (ROW - 1)));
@@ -900,28 +907,38 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                 publish(tail);
                 run = tail;
                 MMV_T_MARK(2)
-                const Acc dval = is_direct ? window_sum<P>(xg, csb, static_cast<int>(cb - csb), win0) : Acc(0);
+                const Acc dval = is_direct ? window_sum<P>(xg, csb, seglen, win0) : Acc(0);
                 const Acc plocal = __shfl_up_sync(0xffffffffu, mylocal, 1);
                 const Acc prp = __shfl_up_sync(0xffffffffu, myrp, 1);
                 const int prow = __shfl_up_sync(0xffffffffu, myrow, 1);
                 const long long qi = cq + lane;
                 bool deferred = false;
+                bool redo = false;        // a short segment whose sum is taken again from its values, at the end of this path
                 Acc val = Acc(0);
                 // lane j: boundary j as the END of segment qi-1 (bnd in (sbase, send], or 0 for leading empties)
-                if (static_cast<int>(lane) < nb_span && qi >= 1 && (cb > sbase || (sbase == 0 && cb == 0))) {
-                    if (csb > cb || csb < 0 || cb > prm.n) {
+                if (static_cast<int>(lane) < nb_span && qi >= 1 && (crel > 0 || (sb32i == 0 && cb == 0))) {
+                    if (csb > cb || csb < 0 || cb > n32i) {
                         report_error(prm.hdr, 4u);
                     } else {
                         if (cb != csb) {
-                            if (cb - csb <= SUM_DIRECT_LEN) {
+                            if (seglen <= SUM_DIRECT_LEN) {
                                 val = dval;
-                            } else if (csb > sbase) {
+                            } else if (csb > sb32i) {
                                 // the start is the previous boundary (lane - 1), inside this span
                                 val = (prow == myrow) ? P::sub(mylocal, plocal)
                                                       : P::sub(P::add(myrp, mylocal), P::add(prp, plocal));
+                                if constexpr (P::kIsFloat) redo = seglen <= 32;
                             } else {
                                 val = P::add(myrp, mylocal);        // from the span's first element
-                                deferred = csb < sbase;
+                                deferred = csb < sb32i;
+                                // (short and reaching back across the span's first element: its carry would be a difference
+                                //  of the previous span's prefixes)
+                                if constexpr (P::kIsFloat) {
+                                    if (deferred && seglen <= 32) {
+                                        deferred = false;
+                                        redo = true;
+                                    }
+                                }
                             }
                         }
                         if (!deferred) outp[qi - 1] = val;
@@ -932,6 +949,24 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     const int srcl = __ffs(dm) - 1;
                     def_r = cq + srcl - 1;
                     def_val = __shfl_sync(0xffffffffu, val, srcl);
+                }
+                // Floating point: a difference of prefixes loses a small sum next to large values, and this path has no
+                // row-wide magnitudes to judge a difference by (the general path does).  Every segment of 5 to 32 elements
+                // that starts behind the span's first element or in front of it is therefore added up again from its
+                // values, one element per lane (a single round trip to memory; with so few boundaries in the span such
+                // segments are rare).
+                if constexpr (P::kIsFloat) {
+                    unsigned rm = __ballot_sync(0xffffffffu, redo);
+                    while (rm) {
+                        const int j = __ffs(rm) - 1;
+                        rm &= rm - 1;
+                        const long long sbj = __shfl_sync(0xffffffffu, csb, j);
+                        const int lenj = __shfl_sync(0xffffffffu, seglen, j);
+                        Acc v = Acc(0);
+                        if (static_cast<int>(lane) < lenj) v = load_value<P>(xg, sbj + lane);
+                        v = warp_sum<P>(v);
+                        if (static_cast<int>(lane) == j) outp[qi - 1] = v;
+                    }
                 }
                 MMV_T_MARK(5)
             } else {
@@ -1026,7 +1061,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     const Acc xsum = warp_sum<P>(xval);
                     if (lane == 0) outp[cq - 1] = xsum;
                 } else if (lane == 0 && is_direct) {
-                    outp[cq - 1] = window_sum<P>(xg, csb, static_cast<int>(cb - csb), win0);
+                    outp[cq - 1] = window_sum<P>(xg, csb, seglen, win0);
                 }
                 // number of elements open at the end of the previous piece's last row (64: too many to matter),
                 // and the largest prefix magnitude of that row

@@ -389,6 +389,32 @@ def test_seg_sum_tiny_segments_next_to_large_values(mmv):
     assert_fp(sum_csr(mmv, x, off), want, a, "tiny next to large, longer")
 
 
+@pytest.mark.parametrize("tiny_len", [5, 10, 20, 32])
+def test_seg_sum_short_tiny_segments_between_long_large_ones(mmv, tiny_len):
+    # spans with few boundaries (long segments of magnitude 2e3) that also hold a segment of 5 to 32 values of
+    # magnitude 1e-3: a difference of the span's prefixes would lose it; the stated bound holds for it at any
+    # magnitudes
+    rng = np.random.default_rng(tiny_len)
+    lens = []
+    while sum(lens) < 6 * TILE:
+        lens += [int(rng.integers(1200, 1800)), tiny_len]
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    n = int(off[-1])
+    scale = np.repeat(np.where(np.arange(len(lens)) % 2 == 0, 2e3, 1e-3), lens)
+    x = (rng.standard_normal(n) * scale).astype(np.float16)
+    want, a = oracle.seg_sum_csr_f16(x, off)
+    got = sum_csr(mmv, x, off)
+    short = np.diff(off) <= 32
+    assert_fp(got[short], want[short], a[short], f"short segments of {tiny_len}")
+    # the products of SpMV take the same path (pairs of bf16 values): rows of the same lengths
+    col = rng.integers(0, 1000, n).astype(np.int32)
+    val = (rng.standard_normal(n) * scale).astype(np.float16)
+    xv = rng.standard_normal(1000).astype(np.float32)
+    wy, ay = oracle.spmv_csr(off, col, val, xv)
+    gy = mmv.spmv_csr(dev(off), dev(col), dev(val), dev(xv)).cpu().numpy()
+    assert_fp(gy[short], wy[short], ay[short], f"short rows of {tiny_len}")
+
+
 def test_seg_sum_long_segments_at_the_edge_of_the_stated_magnitude_range(mmv):
     # What the header promises for segments LONGER than two 32-element rows: the bound holds when the magnitudes
     # inside a 4096-element span are within about 2^10 of each other.  Segments of 40 .. 3000 elements, every
