@@ -415,6 +415,39 @@ def test_seg_sum_short_tiny_segments_between_long_large_ones(mmv, tiny_len):
     assert_fp(gy[short], wy[short], ay[short], f"short rows of {tiny_len}")
 
 
+@pytest.mark.parametrize("seed", [1, 2])
+def test_seg_sum_short_segments_of_any_magnitude_random(mmv, seed):
+    # per-segment magnitudes 1e-3, 1 or 2e3 at random; four laws of segment lengths (few boundaries per span,
+    # dozens, many, long segments with clusters of short ones); every segment of up to 32 elements holds the bound
+    rng = np.random.default_rng(seed)
+    for trial in range(24):
+        n_target = int(rng.choice([3 * TILE, 7 * TILE + 123]))
+        mode = trial % 4
+        lens, tot = [], 0
+        while tot < n_target:
+            if mode == 0:
+                l = int(rng.choice([rng.integers(1, 33), rng.integers(300, 3000)], p=[0.3, 0.7]))
+            elif mode == 1:
+                l = int(rng.choice([rng.integers(1, 33), rng.integers(60, 400)], p=[0.4, 0.6]))
+            elif mode == 2:
+                l = int(rng.integers(1, 40))
+            else:
+                l = int(rng.choice([rng.integers(1, 33), rng.integers(3000, 20000)], p=[0.6, 0.4]))
+            lens.append(l)
+            tot += l
+        off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+        scale = np.repeat(rng.choice([1e-3, 1.0, 2e3], len(lens), p=[0.3, 0.3, 0.4]), lens)
+        x = (rng.standard_normal(int(off[-1])) * scale).astype(np.float16)
+        want, a = oracle.seg_sum_csr_f16(x, off)
+        mmv.debug_force_sum_groups(int(rng.choice([0, 2, 3])))
+        try:
+            got = sum_csr(mmv, x, off)
+        finally:
+            mmv.debug_force_sum_groups(0)
+        short = np.asarray(lens) <= 32
+        assert_fp(got[short], want[short], a[short], f"trial {trial}, law {mode}")
+
+
 def test_seg_sum_long_segments_at_the_edge_of_the_stated_magnitude_range(mmv):
     # What the header promises for segments LONGER than two 32-element rows: the bound holds when the magnitudes
     # inside a 4096-element span are within about 2^10 of each other.  Segments of 40 .. 3000 elements, every
