@@ -180,7 +180,7 @@ mmv_status mmv_seg_scan_shard_finish(const void *summaries, int rank, int world,
  * is not NULL.  The start flags are first compacted into K + 1 offsets inside
  * the workspace (COMPRESS, Section 2; the compaction step of Algorithm 4.2),
  * which therefore holds 4 (n + 1) bytes more than for the offsets form; nseg is
- * ignored.  n < 2^31 in both forms.
+ * ignored.  n < 2^31 in both forms, nseg < 2^31 - 1 (MMV_ERR_INVALID_ARG otherwise).
  * Floating point: a sum is formed from differences of prefixes local to
  * 32-element rows.  A segment that lies inside one row or two adjacent rows
  * (in particular every segment of up to 32 elements) holds the bound for any
@@ -273,7 +273,7 @@ mmv_status mmv_mult_i8(const int8_t *x, const int8_t *y, int64_t n, int32_t *out
  * the bound of "Arithmetic" above for any finite values; a longer row holds it
  * when the magnitudes of the products inside a 4096-product span are within
  * about 2^10 of each other (see mmv_seg_sum).  rowptr: rows+1 int32 with rowptr[0] == 0 and
- * rowptr[rows] == nnz < 2^31; col: nnz int32 in [0, cols) (duplicates simply
+ * rowptr[rows] == nnz < 2^31 (and rows < 2^31 - 1); col: nnz int32 in [0, cols) (duplicates simply
  * add; an index outside the range is never dereferenced, it contributes 0 and the
  * call records MMV_ERR_INVALID_ARG in the workspace status); val: nnz fp16;
  * x: cols fp32; y: rows fp32.

@@ -847,6 +847,7 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return MMV_ERR_INVALID_ARG;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
     if (n >= (1ll << 31)) return MMV_ERR_INVALID_ARG;            // int32 offsets cannot address more
+    if (nseg >= (1ll << 31) - 1) return MMV_ERR_INVALID_ARG;     // offset indices are kept in 32 bits (empty segments may outnumber n)
     if (sf == MMV_SEG_FLAGS_U8) {
         // COMPRESS the start flags into offsets (in the workspace), then the offset-encoded kernel with
         // the segment count read on the device.
@@ -1065,6 +1066,7 @@ mmv_status mmv_spmv_csr(const int32_t* rowptr, const int32_t* col, const void* v
                         void* cuda_stream) {
     if (rows < 0 || cols < 0 || nnz < 0) return MMV_ERR_INVALID_ARG;
     if (nnz >= (1ll << 31)) return MMV_ERR_INVALID_ARG;          // int32 offsets cannot address more
+    if (rows >= (1ll << 31) - 1) return MMV_ERR_INVALID_ARG;     // row indices are kept in 32 bits (empty rows may outnumber nnz)
     if (rows == 0) return MMV_OK;
     if (!rowptr || !y) return MMV_ERR_INVALID_ARG;
     if (!aligned16(rowptr) || !aligned16(y)) return MMV_ERR_INVALID_ARG;

@@ -78,6 +78,8 @@ def test_argument_errors_are_synchronous(lib):
     assert lib.mmv_seg_scan(16, 16, 0, 8, 0, 2, 16, 256, 16, None) == 3                       # bf16 accepted: workspace too small
     assert lib.mmv_seg_sum(None, None, 1, 0, 0, 0, None, None, None, 0, None) == 0  # nothing to do
     assert lib.mmv_seg_sum(16, 16, 1, -5, 1, 0, 16, None, 256, 4096, None) == 1
+    assert lib.mmv_seg_sum(16, 16, 1, 8, (1 << 31) - 1, 0, 16, None, 256, 1 << 40, None) == 1   # more segments than 32-bit indices hold
+    assert lib.mmv_spmv_csr(16, 16, 16, 16, 16, (1 << 31) - 1, 8, 8, 256, 1 << 40, None) == 1    # ... or rows
     assert lib.mmv_seg_sum(16, 16, 0, 8, 0, 0, 16, None, 256, 16, None) == 3        # flag form: workspace too small
     assert lib.mmv_seg_sum(16, 16, 0, 8, 0, 0, 16, 12, 256, 1 << 20, None) == 1     # misaligned segment counter
     lib.mmv_seg_scan_host.argtypes = [vp, vp, i64, ci, vp, i64, vp, sz, vp]
