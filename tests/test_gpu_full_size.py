@@ -257,10 +257,13 @@ def test_wide_integer_scan_full_size(mmv):
         assert torch.equal(out[lo:hi], want), f"int64 plain scan wrong in [{lo}, {hi})"
 
 
-def test_compress_full_size(mmv, c5_values):
-    # COMPRESS of the headline values under the headline flags: the kept values are x[f != 0], in order
+@pytest.mark.parametrize("case", ["p1e-3", "p0.5"])
+def test_compress_full_size(mmv, c5_values, case):
+    # COMPRESS of the headline values under the headline flags (one in a thousand kept: every lane walks its own
+    # mask) and under the flags with every second element kept (warps stage their kept values in shared
+    # memory): the kept values are x[f != 0], in order
     n = 1 << 30
-    f = gen.config5_flags(n, "p1e-3")
+    f = gen.config5_flags(n, case)
     xd, fd = torch.from_numpy(c5_values).cuda(), torch.from_numpy(f).cuda()
     ws = mmv.alloc_workspace(mmv.OP_COMPRESS, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
     out, count = mmv.compress(xd, fd, workspace=ws)
