@@ -142,6 +142,30 @@ def test_row_length_mixes_at_bench_size(mmv, kind):
     assert ok, f"{kind}: |err|/bound = {ratio:.3g} at segment {i}"
 
 
+@pytest.mark.parametrize("seglen", [1000, 3_000_001])
+def test_seg_sum_just_below_2_to_the_31_elements_closed_form(mmv, seglen):
+    """The largest input the offset encoding admits (positions are 32-bit): all-ones int8 values in segments of a
+    constant length that is no divisor of the span size, short ones (general path) and long ones (few-boundaries
+    path, carries across thousands of spans); every sum is the segment's length."""
+    n = (1 << 31) - 16
+    free, _ = torch.cuda.mem_get_info()
+    if free < n + (1 << 30):
+        pytest.skip("not enough device memory")
+    x = torch.ones(n, dtype=torch.int8, device="cuda")
+    nseg = (n + seglen - 1) // seglen
+    off = torch.arange(nseg + 1, dtype=torch.int64, device="cuda") * seglen
+    off[-1] = n
+    off = off.to(torch.int32)
+    ws = mmv.alloc_workspace(mmv.OP_SEG_SUM, mmv.I8_TO_I32, mmv.SEG_OFFSETS_I32, n, nseg)
+    out = mmv.seg_sum(x, off, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    want = torch.full((nseg,), seglen, dtype=torch.int32, device="cuda")
+    want[-1] = n - seglen * (nseg - 1)
+    assert torch.equal(out, want)
+    del x, off, out, ws
+    torch.cuda.empty_cache()
+
+
 def test_scan_beyond_2_to_the_32_elements_closed_form(mmv):
     """Index arithmetic past 2^32 elements: all-ones int8 values with a start flag every 1000 elements
     (one period is not a divisor of the tile size, so the flags drift through every position of a
