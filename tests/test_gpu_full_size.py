@@ -166,6 +166,35 @@ def test_seg_sum_just_below_2_to_the_31_elements_closed_form(mmv, seglen):
     torch.cuda.empty_cache()
 
 
+def test_spmv_just_below_2_to_the_31_products_closed_form(mmv):
+    """The largest matrix the 32-bit row pointers admit: every value 1, x = 1, rows of 777 products (the last one
+    shorter), columns spread over x; y(r) = length of row r, exactly (sums of ones below 2^24)."""
+    nnz = (1 << 31) - 16
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12 * nnz + (2 << 30):
+        pytest.skip("not enough device memory")
+    rowlen, cols = 777, 1 << 20
+    rows = (nnz + rowlen - 1) // rowlen
+    rowptr = torch.arange(rows + 1, dtype=torch.int64, device="cuda") * rowlen
+    rowptr[-1] = nnz
+    rowptr = rowptr.to(torch.int32)
+    col = torch.empty(nnz, dtype=torch.int32, device="cuda")
+    step = 1 << 28
+    for o in range(0, nnz, step):
+        e = min(nnz, o + step)
+        col[o:e] = ((torch.arange(o, e, dtype=torch.int64, device="cuda") * 2654435761) % cols).to(torch.int32)
+    val = torch.ones(nnz, dtype=torch.float16, device="cuda")
+    xv = torch.ones(cols, dtype=torch.float32, device="cuda")
+    ws = mmv.alloc_workspace(mmv.OP_SPMV_CSR, mmv.F16_TO_F32, mmv.SEG_OFFSETS_I32, nnz, rows)
+    y = mmv.spmv_csr(rowptr, col, val, xv, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    want = torch.full((rows,), float(rowlen), dtype=torch.float32, device="cuda")
+    want[-1] = float(nnz - rowlen * (rows - 1))
+    assert torch.equal(y, want)
+    del rowptr, col, val, xv, ws, y
+    torch.cuda.empty_cache()
+
+
 def test_scan_beyond_2_to_the_32_elements_closed_form(mmv):
     """Index arithmetic past 2^32 elements: all-ones int8 values with a start flag every 1000 elements
     (one period is not a divisor of the tile size, so the flags drift through every position of a
