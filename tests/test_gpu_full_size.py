@@ -195,6 +195,37 @@ def test_spmv_just_below_2_to_the_31_products_closed_form(mmv):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("period", [1, 3, 1000])
+def test_compress_just_below_2_to_the_31_elements_closed_form(mmv, period):
+    """COMPRESS at its largest size: x(i) = (i mod 251) - 125, every period-th element kept (all of them, a
+    third: the staged route; one in a thousand: the sparse loop), so kept(j) = x(period * j)."""
+    n = (1 << 31) - 16
+    free, _ = torch.cuda.mem_get_info()
+    if free < 4 * n + (2 << 30):
+        pytest.skip("not enough device memory")
+    x = torch.empty(n, dtype=torch.int8, device="cuda")
+    f = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    step = 1 << 28
+    for o in range(0, n, step):
+        e = min(n, o + step)
+        idx = torch.arange(o, e, dtype=torch.int64, device="cuda")
+        x[o:e] = (idx % 251 - 125).to(torch.int8)
+        f[o:e] = (idx % period == 0).to(torch.uint8) * 7
+        del idx
+    ws = mmv.alloc_workspace(mmv.OP_COMPRESS, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
+    out, count = mmv.compress(x, f, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    k = (n + period - 1) // period
+    assert int(count.item()) == k
+    for o in range(0, k, step):
+        e = min(k, o + step)
+        j = torch.arange(o, e, dtype=torch.int64, device="cuda")
+        assert torch.equal(out[o:e], ((j * period) % 251 - 125).to(torch.int8)), f"kept values wrong in [{o}, {e})"
+        del j
+    del x, f, out, ws
+    torch.cuda.empty_cache()
+
+
 def test_scan_beyond_2_to_the_32_elements_closed_form(mmv):
     """Index arithmetic past 2^32 elements: all-ones int8 values with a start flag every 1000 elements
     (one period is not a divisor of the tile size, so the flags drift through every position of a
