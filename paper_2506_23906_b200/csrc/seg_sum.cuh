@@ -951,7 +951,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     def_val = __shfl_sync(0xffffffffu, val, srcl);
                 }
                 // Floating point: a difference of prefixes loses a small sum next to large values, and this path has no
-                // row-wide magnitudes to judge a difference by (the general path does).  Every segment of 5 to 32 elements
+                // row-wide magnitudes to measure a difference against (the general path has).  Every segment of 5 to 32 elements
                 // that starts behind the span's first element or in front of it is therefore added up again from its
                 // values, one element per lane (a single round trip to memory; with so few boundaries in the span such
                 // segments are rare).
