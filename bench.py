@@ -59,7 +59,7 @@ def parse_args():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU baseline")
     ap.add_argument("--scan-shape", type=int, default=-1, choices=[-1, 0, 2],
                     help="with --profile-case: force the wide (0) or narrow (2) tiles of the floating-point scan (-1: the library chooses)")
-    ap.add_argument("--profile-case", default=None, choices=["scan_f16", "scan_i8", "seg_sum", "seg_sum_short", "seg_sum_mid", "spmv", "minmax", "wide"],
+    ap.add_argument("--profile-case", default=None, choices=["scan_f16", "scan_i8", "seg_sum", "seg_sum_short", "seg_sum_mid", "spmv", "minmax", "wide", "compress"],
                     help="run one small case a few times and exit (the command profiled with ncu)")
     return ap.parse_args()
 
@@ -792,6 +792,15 @@ def run_profile_case(args):
         out = torch.empty(n, dtype=torch.int64, device="cuda")
         ws = mmv.alloc_workspace(mmv.OP_SEG_SCAN_WIDE, mmv.I8_TO_I32, mmv.SEG_FLAGS_U8, n)
         fn = lambda: mmv.seg_scan_wide(xd, fd, out=out, workspace=ws)  # noqa: E731
+    elif args.profile_case == "compress":
+        # COMPRESS of fp16 values under the flag pattern --case names (p0.5: the staged route of warps with many kept elements)
+        x = gen.f16_uniform(5, n)
+        f = gen.config5_flags(n, args.case)
+        xd, fd = torch.from_numpy(x).cuda(), torch.from_numpy(f).cuda()
+        out = torch.empty(n, dtype=torch.float16, device="cuda")
+        kc = torch.zeros(1, dtype=torch.int64, device="cuda")
+        ws = mmv.alloc_workspace(mmv.OP_COMPRESS, mmv.F16_TO_F32, mmv.SEG_FLAGS_U8, n)
+        fn = lambda: mmv.compress(xd, fd, out=out, count=kc, workspace=ws)  # noqa: E731
     elif args.profile_case in ("seg_sum", "seg_sum_short", "seg_sum_mid"):
         # configuration 2, or the Table 5.1 mixes with segment lengths 1/6/44 and 18/119/204 (dense boundaries)
         x, off = gen.config2(n) if args.profile_case == "seg_sum" else gen.seg_sum_row_mix(args.profile_case[8:], n)
