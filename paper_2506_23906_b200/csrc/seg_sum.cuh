@@ -237,7 +237,10 @@ struct SumCfg {
     static constexpr int kStages = P::kElemBytes == 4 ? 2 : 4;      // (the bf16-pair tiles are 64 KB)
     static constexpr int kBBytes = ROW * P::kRowBytes;               // constant operand: 32 rows
     static constexpr int kXBytes = PIECES_PER_SPAN * P::kSlabBytes;  // four [128 x 32] operands
-    static constexpr int kDumpBytes = PIECE * 4;                     // per epilogue warp
+    static constexpr int kDumpRowBytes = ROW * 4 + 16;               // rows of 36 words: 16-byte stores and single-word loads
+                                                                     // both spread over the banks, and a prefix is at
+                                                                     // row + 4 c (no swizzle to undo per look-up)
+    static constexpr int kDumpBytes = PIECE_ROWS * kDumpRowBytes;    // per epilogue warp
     static constexpr int kStageOffset = 4096;                        // after the constant operand
     static constexpr int kDumpOffset = kStageOffset + kStages * kXBytes;
     static constexpr int kMarkOffset = kDumpOffset + SumShape<G>::kEpiWarps * kDumpBytes;
@@ -619,7 +622,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
         const int w = warp & 3;
         Acc* outp = static_cast<Acc*>(prm.out);
         // per row of the span: marked elements (bits), number of boundaries; boundaries at the span's first element
-        uint8_t* dump = smem + Cfg::kDumpOffset + warp * Cfg::kDumpBytes;      // [32 rows][32] prefixes of a piece, swizzled by row
+        uint8_t* dump = smem + Cfg::kDumpOffset + warp * Cfg::kDumpBytes;      // [32 rows][32] prefixes of a piece, rows padded
         uint32_t* emask = reinterpret_cast<uint32_t*>(smem + Cfg::kMarkOffset + warp * SUM_MARK_BYTES);
         uint32_t* ecnt = emask + SPAN / ROW;
         uint32_t* nbase = ecnt + SPAN / ROW;
@@ -1098,7 +1101,7 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                         tmem_ld_wait();
 #pragma unroll
                         for (int c4 = 0; c4 < 8; ++c4)
-                            *reinterpret_cast<uint4*>(dump + lane * 128 + ((c4 ^ (lane & 7)) << 4)) =
+                            *reinterpret_cast<uint4*>(dump + lane * Cfg::kDumpRowBytes + (c4 << 4)) =
                                 make_uint4(r[4 * c4], r[4 * c4 + 1], r[4 * c4 + 2], r[4 * c4 + 3]);
                         if constexpr (P::kIsFloat) {
                             // (two chains of three-operand maxima)
@@ -1123,11 +1126,8 @@ seg_sum_kernel(const __grid_constant__ CUtensorMap tmap_x, const void* __restric
                     int cprev = -1, nend = 0, first_len = 0;
                     long long first_oi = -1;
                     uint32_t mm = m;
-                    const uint8_t* drow = dump + lane * 128;       // my row of the prefixes (16-byte groups swizzled by row)
-                    const int lx = static_cast<int>(lane & 7);
-                    auto prefix_at = [&](int c) -> Acc {
-                        return *reinterpret_cast<const Acc*>(drow + ((((c >> 2) ^ lx) << 4) | ((c & 3) << 2)));
-                    };
+                    const uint8_t* drow = dump + lane * Cfg::kDumpRowBytes;       // my row of the prefixes
+                    auto prefix_at = [&](int c) -> Acc { return *reinterpret_cast<const Acc*>(drow + (c << 2)); };
                     auto index_of = [&](int c, int k) -> long long {          // output index of my k-th sum, which ends behind column c
                         if (!dirty) return orow + k;
                         const int32_t bpos = static_cast<int32_t>(rowpos + c + 1);
