@@ -285,7 +285,9 @@ mmv_status mmv_spmv_csr(const int32_t *rowptr, const int32_t *col, const void *v
 /*
  * Synchronises `cuda_stream` and returns the device-side status that the last
  * call using `workspace` recorded (MMV_OK if none), or MMV_ERR_CUDA if the
- * stream itself reports an error.
+ * stream itself reports an error.  A call that had nothing to do (no elements,
+ * no segments, no rows, no non-zeros) and was handed a workspace records
+ * MMV_OK in it; a workspace no call has seen yet holds no status.
  */
 mmv_status mmv_last_async_status(const void *workspace, void *cuda_stream);
 

@@ -518,13 +518,22 @@ size_t mmv_workspace_bytes(mmv_op op, mmv_dtype dt, mmv_segfmt sf, int64_t n, in
 namespace {
 // shard: 0 = a whole vector; 1 = the first shard of a longer vector, 2 = a later shard (its flag byte 0 counts,
 // and without it element 0 continues the segment that reaches it).  For shards `summary` receives the record.
+// A call that has nothing to do still leaves MMV_OK for mmv_last_async_status when it is handed a workspace
+// (a workspace that was never used would otherwise answer with whatever its memory holds).
+mmv_status nothing_to_do(void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    if (workspace && !(reinterpret_cast<uintptr_t>(workspace) & 255u) && workspace_bytes >= sizeof(WorkspaceHeader) &&
+        cudaMemsetAsync(workspace, 0, sizeof(WorkspaceHeader), static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return MMV_ERR_CUDA;
+    return MMV_OK;
+}
+
 mmv_status seg_scan_impl(const void* x, const void* seg, mmv_segfmt sf, int64_t n, int64_t nseg, mmv_dtype dt,
                          void* out, void* workspace, size_t workspace_bytes, void* cuda_stream, bool exclusive,
                          int shard = 0, void* summary = nullptr) {
     if (n < 0 || nseg < 0) return MMV_ERR_INVALID_ARG;
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return MMV_ERR_INVALID_ARG;
     if (sf != MMV_SEG_FLAGS_U8 && sf != MMV_SEG_OFFSETS_I32) return MMV_ERR_INVALID_ARG;
-    if (n == 0) return MMV_OK;
+    if (n == 0) return nothing_to_do(workspace, workspace_bytes, cuda_stream);
     if (n >= (1ll << 36)) return MMV_ERR_UNSUPPORTED;
     if (sf == MMV_SEG_OFFSETS_I32 && n >= (1ll << 31)) return MMV_ERR_INVALID_ARG;
     if (!x || !out || !workspace) return MMV_ERR_INVALID_ARG;
@@ -854,7 +863,7 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
         cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
         if (n == 0) {
             if (d_num_segments && cudaMemsetAsync(d_num_segments, 0, sizeof(int64_t), st) != cudaSuccess) return MMV_ERR_CUDA;
-            return MMV_OK;
+            return nothing_to_do(workspace, workspace_bytes, cuda_stream);
         }
         if (!x || !seg || !out || !workspace) return MMV_ERR_INVALID_ARG;
         if (!aligned16(x) || !aligned16(seg) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
@@ -888,12 +897,13 @@ mmv_status mmv_seg_sum(const void* x, const void* seg, mmv_segfmt sf, int64_t n,
         if (dt == MMV_BF16_TO_F32) return launch_seg_sum<BF16ValPath>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, true);
         return launch_seg_sum<I8Path>(x, n, off, 0, 0, out, ws, plan, dev, st, nseg_dev, true);
     }
-    if (nseg == 0) return MMV_OK;
+    if (nseg == 0) return nothing_to_do(workspace, workspace_bytes, cuda_stream);
     if (!seg || !out) return MMV_ERR_INVALID_ARG;
     if (!aligned16(seg) || !aligned16(out)) return MMV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (n == 0) {                                                // every segment is empty
-        return cudaMemsetAsync(out, 0, static_cast<size_t>(nseg) * 4, st) == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+        if (cudaMemsetAsync(out, 0, static_cast<size_t>(nseg) * 4, st) != cudaSuccess) return MMV_ERR_CUDA;
+        return nothing_to_do(workspace, workspace_bytes, cuda_stream);
     }
     if (!x || !workspace) return MMV_ERR_INVALID_ARG;
     if (!aligned16(x) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MMV_ERR_INVALID_ARG;
@@ -919,7 +929,7 @@ mmv_status mmv_seg_scan_minmax(const void* x, const void* flags, int64_t n, mmv_
                                void* workspace, size_t workspace_bytes, void* cuda_stream) {
     if (n < 0) return MMV_ERR_INVALID_ARG;
     if (dt != MMV_F16_TO_F32 && dt != MMV_I8_TO_I32 && dt != MMV_BF16_TO_F32) return MMV_ERR_INVALID_ARG;
-    if (n == 0) return MMV_OK;
+    if (n == 0) return nothing_to_do(workspace, workspace_bytes, cuda_stream);
     if (n >= (1ll << 36)) return MMV_ERR_UNSUPPORTED;
     if (!x || !out || !workspace) return MMV_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(flags) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
@@ -961,7 +971,7 @@ mmv_status mmv_seg_scan_minmax(const void* x, const void* flags, int64_t n, mmv_
 mmv_status mmv_seg_scan_i8_i64(const void* x, const void* flags, int64_t n, int64_t* out, void* workspace,
                                size_t workspace_bytes, void* cuda_stream) {
     if (n < 0) return MMV_ERR_INVALID_ARG;
-    if (n == 0) return MMV_OK;
+    if (n == 0) return nothing_to_do(workspace, workspace_bytes, cuda_stream);
     if (n >= (1ll << 36)) return MMV_ERR_UNSUPPORTED;
     if (!x || !out || !workspace) return MMV_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(flags) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
@@ -999,7 +1009,7 @@ mmv_status mmv_compress(const void* x, const void* flags, int64_t n, mmv_dtype d
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (n == 0) {
         if (d_count && cudaMemsetAsync(d_count, 0, sizeof(int64_t), st) != cudaSuccess) return MMV_ERR_CUDA;
-        return MMV_OK;
+        return nothing_to_do(workspace, workspace_bytes, cuda_stream);
     }
     if (!x || !flags || !out || !workspace) return MMV_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(flags) || !aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
@@ -1035,7 +1045,7 @@ mmv_status mmv_compress(const void* x, const void* flags, int64_t n, mmv_dtype d
 mmv_status mmv_mult_i8(const int8_t* x, const int8_t* y, int64_t n, int32_t* out, void* workspace, size_t workspace_bytes,
                        void* cuda_stream) {
     if (n < 0 || n >= (1ll << 28)) return MMV_ERR_INVALID_ARG;          // 8 n terms are addressed by int32 offsets
-    if (n == 0) return MMV_OK;
+    if (n == 0) return nothing_to_do(workspace, workspace_bytes, cuda_stream);
     if (!x || !y || !out || !workspace) return MMV_ERR_INVALID_ARG;
     if (!aligned16(out) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return MMV_ERR_INVALID_ARG;
     const MultPlan plan = plan_mult(n);
@@ -1067,12 +1077,13 @@ mmv_status mmv_spmv_csr(const int32_t* rowptr, const int32_t* col, const void* v
     if (rows < 0 || cols < 0 || nnz < 0) return MMV_ERR_INVALID_ARG;
     if (nnz >= (1ll << 31)) return MMV_ERR_INVALID_ARG;          // int32 offsets cannot address more
     if (rows >= (1ll << 31) - 1) return MMV_ERR_INVALID_ARG;     // row indices are kept in 32 bits (empty rows may outnumber nnz)
-    if (rows == 0) return MMV_OK;
+    if (rows == 0) return nothing_to_do(workspace, workspace_bytes, cuda_stream);
     if (!rowptr || !y) return MMV_ERR_INVALID_ARG;
     if (!aligned16(rowptr) || !aligned16(y)) return MMV_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (nnz == 0) {
-        return cudaMemsetAsync(y, 0, static_cast<size_t>(rows) * 4, st) == cudaSuccess ? MMV_OK : MMV_ERR_CUDA;
+        if (cudaMemsetAsync(y, 0, static_cast<size_t>(rows) * 4, st) != cudaSuccess) return MMV_ERR_CUDA;
+        return nothing_to_do(workspace, workspace_bytes, cuda_stream);
     }
     if (!col || !val_f16 || !x || !workspace || cols == 0) return MMV_ERR_INVALID_ARG;
     if (!aligned16(col) || !aligned16(val_f16) || !aligned16(x) || (reinterpret_cast<uintptr_t>(workspace) & 255u))

@@ -713,6 +713,31 @@ def test_compress_with_dense_and_sparse_stretches(mmv):
         assert np.array_equal(got[: want.shape[0]].cpu().numpy(), want)
 
 
+def test_calls_with_nothing_to_do_leave_ok_in_a_fresh_workspace(mmv):
+    # a workspace that no call has used yet (all bytes set) is handed to calls without elements, segments, rows
+    # or non-zeros: the status read back afterwards is MMV_OK, not whatever the memory held
+    def fresh():
+        return torch.full((4096,), 0xFF, dtype=torch.uint8, device="cuda")
+    e16 = torch.empty(0, dtype=torch.float16, device="cuda")
+    e8 = torch.empty(0, dtype=torch.uint8, device="cuda")
+    ws = fresh()
+    mmv.seg_scan(e16, e8, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    ws = fresh()
+    mmv.seg_scan_minmax(e16, e8, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    ws = fresh()
+    mmv.compress(e16, e8, workspace=ws)
+    assert mmv.last_async_status(ws) == 0
+    ws = fresh()
+    out = mmv.seg_sum(e16, torch.zeros(4, dtype=torch.int32, device="cuda"), workspace=ws)      # three empty segments
+    assert out.cpu().tolist() == [0.0, 0.0, 0.0] and mmv.last_async_status(ws) == 0
+    ws = fresh()
+    y = mmv.spmv_csr(torch.zeros(3, dtype=torch.int32, device="cuda"), torch.empty(0, dtype=torch.int32, device="cuda"), e16,
+                     torch.ones(5, dtype=torch.float32, device="cuda"), workspace=ws)                # two rows, no non-zeros
+    assert y.cpu().tolist() == [0.0, 0.0] and mmv.last_async_status(ws) == 0
+
+
 def test_compress_of_the_paper_example(mmv):
     g = __import__("conftest").load_golden("sec2_worked_example.txt")
     out, count = mmv.compress(dev(np.asarray(g["x"], np.int8)), dev(np.asarray(g["f"], np.uint8)))
